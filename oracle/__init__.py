@@ -1,0 +1,181 @@
+"""ctypes front end of the rTop-k CPU oracle (test infrastructure only).
+
+The oracle restates Algorithm 1 (node body and master average) and
+Definitions 1-3 of the rTop-k paper as plain CPU code; see the header of
+``rtopk_oracle.cpp`` for the readings it fixes.  Only tests, the smoke check
+and the benchmark's CPU-baseline leg import this package; the CUDA library
+never does.
+
+All array arguments are C-contiguous numpy arrays; bfloat16 gradients are
+passed as ``uint16`` bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+import sys
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "rtopk_oracle.cpp")
+_LIB = os.path.join(_HERE, "librtopk_oracle.so")
+
+GRAD_F32, GRAD_BF16 = 0, 1
+SCALE_MEAN, SCALE_SUM = 0, 1
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with the host compiler (no fast-math, no contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-pthread", "-ffp-contract=off",
+               "-fno-fast-math", "-Wall", "-Wextra", "-o", _LIB, _SRC]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        build()
+        L = C.CDLL(_LIB)
+        u32p, f32p, f64p, i64p = (C.POINTER(C.c_uint32), C.POINTER(C.c_float),
+                                  C.POINTER(C.c_double), C.POINTER(C.c_int64))
+        L.oracle_set_threads.argtypes = [C.c_int]
+        L.oracle_get_threads.restype = C.c_int
+        L.oracle_philox4x32_10.argtypes = [u32p, u32p, u32p]
+        L.oracle_scale_draw.argtypes = [C.c_uint64, C.c_uint32]
+        L.oracle_scale_draw.restype = C.c_uint32
+        L.oracle_draw.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint32]
+        L.oracle_draw.restype = C.c_uint32
+        L.oracle_floyd_from_draws.argtypes = [C.c_int64, C.c_int64, u32p, u32p]
+        L.oracle_sample_positions.argtypes = [C.c_int64, C.c_int64, C.c_uint64, C.c_uint32,
+                                              C.c_uint32, C.c_uint32, u32p]
+        L.oracle_top_r.argtypes = [f32p, C.c_int64, C.c_int64, u32p]
+        L.oracle_sparsify.argtypes = [C.c_void_p, C.c_int, C.c_int64, f32p, C.c_int64, C.c_int64,
+                                      C.c_int32, C.c_int32, C.c_int64, C.c_int64, C.c_uint64,
+                                      C.c_uint32, u32p, f32p]
+        L.oracle_sparsify_segmented.argtypes = [C.c_void_p, C.c_int, C.c_int64, f32p, C.c_int64,
+                                                C.c_int64, C.c_int32, C.c_int32, C.c_int32, i64p,
+                                                i64p, i64p, C.c_uint64, C.c_uint32, u32p, f32p]
+        L.oracle_aggregate.argtypes = [u32p, f32p, C.c_int64, C.c_int32, C.c_int64, C.c_int,
+                                       f64p, f32p]
+        _lib = L
+    return _lib
+
+
+def _p(a: np.ndarray, ty):
+    return a.ctypes.data_as(C.POINTER(ty))
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        raise ValueError(f"oracle: {what} rejected its arguments (code {rc})")
+
+
+def set_threads(n: int) -> None:
+    lib().oracle_set_threads(int(n))
+
+
+def philox4x32_10(ctr, key) -> np.ndarray:
+    c = np.asarray(ctr, dtype=np.uint32).copy()
+    k = np.asarray(key, dtype=np.uint32).copy()
+    assert c.shape == (4,) and k.shape == (2,)
+    out = np.zeros(4, dtype=np.uint32)
+    lib().oracle_philox4x32_10(_p(c, C.c_uint32), _p(k, C.c_uint32), _p(out, C.c_uint32))
+    return out
+
+
+def scale_draw(u: int, n: int) -> int:
+    return int(lib().oracle_scale_draw(int(u), int(n)))
+
+
+def draw(seed: int, step: int, worker: int, segment: int, j: int) -> int:
+    return int(lib().oracle_draw(int(seed), int(step), int(worker), int(segment), int(j)))
+
+
+def floyd_from_draws(r: int, k: int, t) -> np.ndarray:
+    t = np.ascontiguousarray(t, dtype=np.uint32)
+    assert t.shape == (k,)
+    pos = np.zeros(k, dtype=np.uint32)
+    _check(lib().oracle_floyd_from_draws(r, k, _p(t, C.c_uint32), _p(pos, C.c_uint32)), "floyd")
+    return pos
+
+
+def sample_positions(r: int, k: int, seed: int, step: int, worker: int, segment: int = 0) -> np.ndarray:
+    pos = np.zeros(k, dtype=np.uint32)
+    _check(lib().oracle_sample_positions(r, k, seed, step, worker, segment, _p(pos, C.c_uint32)),
+           "sample_positions")
+    return pos
+
+
+def top_r(a: np.ndarray, r: int) -> np.ndarray:
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    L = np.zeros(r, dtype=np.uint32)
+    _check(lib().oracle_top_r(_p(a, C.c_float), a.shape[0], r, _p(L, C.c_uint32)), "top_r")
+    return L
+
+
+def _grad_args(grad: np.ndarray):
+    assert grad.ndim == 2 and grad.flags.c_contiguous
+    if grad.dtype == np.float32:
+        return GRAD_F32
+    if grad.dtype == np.uint16:
+        return GRAD_BF16
+    raise TypeError("grad must be float32 or uint16 (bfloat16 bits)")
+
+
+def sparsify(grad: np.ndarray, residual: np.ndarray, d: int, r: int, k: int, seed: int, step: int,
+             worker_base: int = 0):
+    """Algorithm 1 node body on W rows; ``residual`` (float32, W x ld_m) is updated in place.
+    Returns (msg_idx [W,k] uint32, msg_val [W,k] float32)."""
+    dt = _grad_args(grad)
+    assert residual.dtype == np.float32 and residual.ndim == 2 and residual.flags.c_contiguous
+    W = grad.shape[0]
+    assert residual.shape[0] == W
+    idx = np.zeros((W, k), dtype=np.uint32)
+    val = np.zeros((W, k), dtype=np.float32)
+    _check(lib().oracle_sparsify(grad.ctypes.data, dt, grad.shape[1], _p(residual, C.c_float),
+                                 residual.shape[1], d, W, worker_base, r, k, seed, step,
+                                 _p(idx, C.c_uint32), _p(val, C.c_float)), "sparsify")
+    return idx, val
+
+
+def sparsify_segmented(grad: np.ndarray, residual: np.ndarray, d: int, seg_off, seg_r, seg_k,
+                       seed: int, step: int, worker_base: int = 0):
+    dt = _grad_args(grad)
+    assert residual.dtype == np.float32 and residual.ndim == 2 and residual.flags.c_contiguous
+    W = grad.shape[0]
+    off = np.ascontiguousarray(seg_off, dtype=np.int64)
+    rr = np.ascontiguousarray(seg_r, dtype=np.int64)
+    kk = np.ascontiguousarray(seg_k, dtype=np.int64)
+    S = rr.shape[0]
+    assert off.shape == (S + 1,) and kk.shape == (S,)
+    K = int(kk.sum())
+    idx = np.zeros((W, K), dtype=np.uint32)
+    val = np.zeros((W, K), dtype=np.float32)
+    _check(lib().oracle_sparsify_segmented(grad.ctypes.data, dt, grad.shape[1],
+                                           _p(residual, C.c_float), residual.shape[1], d, W,
+                                           worker_base, S, _p(off, C.c_int64), _p(rr, C.c_int64),
+                                           _p(kk, C.c_int64), seed, step, _p(idx, C.c_uint32),
+                                           _p(val, C.c_float)), "sparsify_segmented")
+    return idx, val
+
+
+def aggregate(msg_idx: np.ndarray, msg_val: np.ndarray, d: int, scale_mode: int = SCALE_MEAN):
+    """Algorithm 1 master average.  Returns (out64 float64 [d], out32 float32 [d])."""
+    idx = np.ascontiguousarray(msg_idx, dtype=np.uint32)
+    val = np.ascontiguousarray(msg_val, dtype=np.float32)
+    W, k = idx.shape
+    o64 = np.zeros(d, dtype=np.float64)
+    o32 = np.zeros(d, dtype=np.float32)
+    _check(lib().oracle_aggregate(_p(idx, C.c_uint32), _p(val, C.c_float), d, W, k, scale_mode,
+                                  _p(o64, C.c_double), _p(o32, C.c_float)), "aggregate")
+    return o64, o32
+
+
+if __name__ == "__main__":
+    print(build(force="--force" in sys.argv))

@@ -1,0 +1,289 @@
+// rTop-k CPU oracle -- TEST INFRASTRUCTURE, not a product path.
+//
+// A plain, slow, single-pass-per-definition restatement of the data-parallel
+// hot path of rTop-k (Barnes, Inan, Isik, Ozgur: "rTop-k: A Statistical
+// Estimation Approach to Distributed SGD"):
+//
+//   Algorithm 1, node body:   a = g + m ; ghat = rTop_k(a) ; m' = a - ghat ; send ghat
+//   Algorithm 1, master:      ghat = (1/n) * sum_i ghat_i
+//   Definition 1 (top-r), Definition 2 (random-k), Definition 3 (rTop-k).
+//
+// Only the tests, the smoke check and the benchmark's cpu_baseline leg may call
+// this file.  It shares no code, header, table or constant generator with the
+// CUDA library.  Nothing here is blocked, fused or reordered: the top-r set is
+// a full sort, the k-subset is the sequential Floyd loop, the aggregate is a
+// dense double-precision accumulation in worker order.
+//
+// Readings where the paper is silent (fixed by the library's contract):
+//   * ties in |a| (Def. 1 says "a permutation"): larger magnitude first, then
+//     the lower index;
+//   * "uniformly at random" (Def. 3): Floyd's subset algorithm on positions
+//     0..r-1 of the top-r set numbered by ascending index, driven by
+//     Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) with
+//     counter = (j, worker, segment, step), key = (seed lo, seed hi);
+//   * a, m, message values and the update are IEEE binary32; the add is one
+//     round-to-nearest add; magnitudes are compared through the bit pattern
+//     with the sign cleared (so NaN > Inf > finite, and -0 ties with +0);
+//   * m' is a bit copy of a outside the sent set and +0.0f inside it;
+//   * messages are listed by ascending index.
+//
+// Pins (tests/test_oracle_*.py): Philox against published known answers; the
+// draw scaling against big-integer arithmetic; Floyd against exhaustive
+// enumeration (every k-subset equally often); top-r against brute force and
+// library sorts; the whole operator against the closed form in the proof of
+// Proposition 1 and the limits k = r (Def. 1) and r = d (Def. 2).
+
+#include <algorithm>
+#include <cstdint>
+#include <cstring>
+#include <thread>
+#include <vector>
+
+namespace {
+
+enum { ORACLE_OK = 0, ORACLE_BAD_ARG = 1 };
+enum { GRAD_F32 = 0, GRAD_BF16 = 1 };
+enum { SCALE_MEAN = 0, SCALE_SUM = 1 };
+
+int g_threads = 1;
+
+// ---- Philox4x32-10, from the published definition (SC'11, Section 3.3) ------
+// One round: two 32x32->64 products of counter words 0 and 2 with the two
+// round multipliers; the high halves are XORed with counter words 1 and 3 and
+// with the key and cross over; the low halves pass through.  Between rounds
+// the key words are bumped by the two Weyl constants (golden ratio, sqrt(3)-1).
+void philox4x32_10(const uint32_t c_in[4], const uint32_t k_in[2], uint32_t out[4]) {
+  const uint64_t MUL_A = 0xD2511F53u;  // multiplies counter word 0
+  const uint64_t MUL_B = 0xCD9E8D57u;  // multiplies counter word 2
+  const uint32_t WEYL_0 = 0x9E3779B9u;
+  const uint32_t WEYL_1 = 0xBB67AE85u;
+  uint32_t c0 = c_in[0], c1 = c_in[1], c2 = c_in[2], c3 = c_in[3];
+  uint32_t k0 = k_in[0], k1 = k_in[1];
+  for (int round = 0; round < 10; ++round) {
+    const uint64_t pa = MUL_A * (uint64_t)c0;
+    const uint64_t pb = MUL_B * (uint64_t)c2;
+    const uint32_t n0 = (uint32_t)(pb >> 32) ^ c1 ^ k0;
+    const uint32_t n1 = (uint32_t)pb;
+    const uint32_t n2 = (uint32_t)(pa >> 32) ^ c3 ^ k1;
+    const uint32_t n3 = (uint32_t)pa;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += WEYL_0;
+    k1 += WEYL_1;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// floor(u * n / 2^64): maps a 64-bit uniform word onto {0, ..., n-1}.
+uint32_t scale_draw(uint64_t u, uint32_t n) {
+  return (uint32_t)(((unsigned __int128)u * (unsigned __int128)n) >> 64);
+}
+
+// The draw Floyd's loop makes at iteration j: uniform on {0, ..., j}.
+uint32_t draw_t(uint64_t seed, uint32_t step, uint32_t worker, uint32_t segment, uint32_t j) {
+  const uint32_t ctr[4] = {j, worker, segment, step};
+  const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+  uint32_t x[4];
+  philox4x32_10(ctr, key, x);
+  const uint64_t u = ((uint64_t)x[1] << 32) | (uint64_t)x[0];
+  return scale_draw(u, j + 1u);
+}
+
+// Floyd's k-of-r subset algorithm, sequential, with the draws supplied:
+// t[i] is the draw of iteration j = r-k+i and must lie in {0..j}.
+// Writes the k chosen positions in ascending order.
+void floyd_from_draws(int64_t r, int64_t k, const uint32_t* t, uint32_t* pos) {
+  std::vector<uint8_t> in_set((size_t)r, 0);
+  for (int64_t j = r - k; j < r; ++j) {
+    const uint32_t tj = t[j - (r - k)];
+    if (!in_set[tj]) in_set[tj] = 1;
+    else             in_set[(size_t)j] = 1;
+  }
+  int64_t n = 0;
+  for (int64_t p = 0; p < r; ++p)
+    if (in_set[(size_t)p]) pos[n++] = (uint32_t)p;
+}
+
+void sample_positions(int64_t r, int64_t k, uint64_t seed, uint32_t step, uint32_t worker,
+                      uint32_t segment, uint32_t* pos) {
+  std::vector<uint32_t> t((size_t)k);
+  for (int64_t j = r - k; j < r; ++j)
+    t[(size_t)(j - (r - k))] = draw_t(seed, step, worker, segment, (uint32_t)j);
+  floyd_from_draws(r, k, t.data(), pos);
+}
+
+inline uint32_t float_bits(float x) { uint32_t b; std::memcpy(&b, &x, 4); return b; }
+inline float bits_float(uint32_t b) { float x; std::memcpy(&x, &b, 4); return x; }
+inline uint32_t magnitude_key(float x) { return float_bits(x) & 0x7FFFFFFFu; }
+
+struct KeyIdx { uint32_t key; uint32_t idx; };
+
+// Definition 1: indices of the r largest-magnitude entries, ties to the lower
+// index; returned in ascending index order.
+void top_r_indices(const float* a, int64_t d, int64_t r, uint32_t* L) {
+  std::vector<KeyIdx> order((size_t)d);
+  for (int64_t i = 0; i < d; ++i) order[(size_t)i] = KeyIdx{magnitude_key(a[i]), (uint32_t)i};
+  std::sort(order.begin(), order.end(), [](const KeyIdx& x, const KeyIdx& y) {
+    if (x.key != y.key) return x.key > y.key;
+    return x.idx < y.idx;
+  });
+  for (int64_t p = 0; p < r; ++p) L[p] = order[(size_t)p].idx;
+  std::sort(L, L + r);
+}
+
+inline float widen_grad(const void* grad, int dtype, int64_t i) {
+  if (dtype == GRAD_F32) return ((const float*)grad)[i];
+  const uint16_t h = ((const uint16_t*)grad)[i];   // bfloat16 = top half of binary32
+  return bits_float((uint32_t)h << 16);
+}
+
+// One worker, one slice [0, d) of its vector (Algorithm 1 node body).
+// grad/residual point at the slice; idx_base is added to reported indices.
+void sparsify_slice(const void* grad, int dtype, float* residual, int64_t d, int64_t r, int64_t k,
+                    uint64_t seed, uint32_t step, uint32_t worker, uint32_t segment,
+                    uint32_t idx_base, uint32_t* msg_idx, float* msg_val) {
+  // a = g + m   (materialised in the residual buffer)
+  for (int64_t i = 0; i < d; ++i) {
+    const float s = widen_grad(grad, dtype, i) + residual[i];   // one binary32 add
+    residual[i] = s;
+  }
+  // I <- indices of the r largest-magnitude components
+  std::vector<uint32_t> L((size_t)r);
+  top_r_indices(residual, d, r, L.data());
+  // I <- random k-subset of I
+  std::vector<uint32_t> pos((size_t)k);
+  sample_positions(r, k, seed, step, worker, segment, pos.data());
+  // ghat <- a restricted to I ;  m' <- a - ghat
+  for (int64_t q = 0; q < k; ++q) {
+    const uint32_t i = L[pos[(size_t)q]];
+    msg_idx[q] = idx_base + i;
+    msg_val[q] = residual[i];
+    residual[i] = 0.0f;
+  }
+}
+
+template <class F>
+void for_each_row(int W, F&& body) {
+  const int nt = std::max(1, std::min(g_threads, W));
+  if (nt == 1) { for (int w = 0; w < W; ++w) body(w); return; }
+  std::vector<std::thread> pool;
+  for (int t = 0; t < nt; ++t)
+    pool.emplace_back([&, t] { for (int w = t; w < W; w += nt) body(w); });
+  for (auto& th : pool) th.join();
+}
+
+}  // namespace
+
+extern "C" {
+
+// Rows (workers) are independent; this only sets how many host threads walk them.
+void oracle_set_threads(int n) { g_threads = n < 1 ? 1 : n; }
+int  oracle_get_threads(void) { return g_threads; }
+
+void oracle_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* out) {
+  philox4x32_10(ctr, key, out);
+}
+
+uint32_t oracle_scale_draw(uint64_t u, uint32_t n) { return scale_draw(u, n); }
+
+uint32_t oracle_draw(uint64_t seed, uint32_t step, uint32_t worker, uint32_t segment, uint32_t j) {
+  return draw_t(seed, step, worker, segment, j);
+}
+
+int oracle_floyd_from_draws(int64_t r, int64_t k, const uint32_t* t, uint32_t* pos) {
+  if (r < 1 || k < 1 || k > r || !t || !pos) return ORACLE_BAD_ARG;
+  for (int64_t j = r - k; j < r; ++j)
+    if ((int64_t)t[j - (r - k)] > j) return ORACLE_BAD_ARG;
+  floyd_from_draws(r, k, t, pos);
+  return ORACLE_OK;
+}
+
+int oracle_sample_positions(int64_t r, int64_t k, uint64_t seed, uint32_t step, uint32_t worker,
+                            uint32_t segment, uint32_t* pos) {
+  if (r < 1 || k < 1 || k > r || r > 0x7FFFFFFF || !pos) return ORACLE_BAD_ARG;
+  sample_positions(r, k, seed, step, worker, segment, pos);
+  return ORACLE_OK;
+}
+
+int oracle_top_r(const float* a, int64_t d, int64_t r, uint32_t* L) {
+  if (!a || !L || d < 1 || r < 1 || r > d || d > 0x7FFFFFFF) return ORACLE_BAD_ARG;
+  top_r_indices(a, d, r, L);
+  return ORACLE_OK;
+}
+
+// Algorithm 1 node body for W workers held as rows of grad (W x ld_g) and
+// residual (W x ld_m, updated in place).  Row w is worker worker_base + w.
+// Messages: msg_idx / msg_val are W x k, ascending index within a row.
+int oracle_sparsify(const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
+                    int64_t d, int32_t W, int32_t worker_base, int64_t r, int64_t k, uint64_t seed,
+                    uint32_t step, uint32_t* msg_idx, float* msg_val) {
+  if (!grad || !residual || !msg_idx || !msg_val) return ORACLE_BAD_ARG;
+  if (d < 1 || d > 0x7FFFFFFF || W < 1 || k < 1 || k > r || r > d || ld_g < d || ld_m < d)
+    return ORACLE_BAD_ARG;
+  if (grad_dtype != GRAD_F32 && grad_dtype != GRAD_BF16) return ORACLE_BAD_ARG;
+  const size_t gsz = grad_dtype == GRAD_F32 ? 4 : 2;
+  for_each_row(W, [&](int w) {
+    sparsify_slice((const char*)grad + (size_t)w * (size_t)ld_g * gsz, grad_dtype,
+                   residual + (size_t)w * (size_t)ld_m, d, r, k, seed, step,
+                   (uint32_t)(worker_base + w), 0u, 0u,
+                   msg_idx + (size_t)w * (size_t)k, msg_val + (size_t)w * (size_t)k);
+  });
+  return ORACLE_OK;
+}
+
+// Per-tensor variant: the vector is cut at seg_off[0..S] (seg_off[0] = 0,
+// seg_off[S] = d) and rTop-k with (seg_r[s], seg_k[s]) is applied to every
+// slice independently; the Philox counter carries s.  A row's message holds
+// K = sum_s seg_k[s] entries: slice 0's first, each with flat indices.
+int oracle_sparsify_segmented(const void* grad, int grad_dtype, int64_t ld_g, float* residual,
+                              int64_t ld_m, int64_t d, int32_t W, int32_t worker_base, int32_t S,
+                              const int64_t* seg_off, const int64_t* seg_r, const int64_t* seg_k,
+                              uint64_t seed, uint32_t step, uint32_t* msg_idx, float* msg_val) {
+  if (!grad || !residual || !msg_idx || !msg_val || !seg_off || !seg_r || !seg_k) return ORACLE_BAD_ARG;
+  if (d < 1 || d > 0x7FFFFFFF || W < 1 || S < 1 || ld_g < d || ld_m < d) return ORACLE_BAD_ARG;
+  if (grad_dtype != GRAD_F32 && grad_dtype != GRAD_BF16) return ORACLE_BAD_ARG;
+  if (seg_off[0] != 0 || seg_off[S] != d) return ORACLE_BAD_ARG;
+  int64_t K = 0;
+  for (int s = 0; s < S; ++s) {
+    const int64_t len = seg_off[s + 1] - seg_off[s];
+    if (len < 1 || seg_k[s] < 1 || seg_k[s] > seg_r[s] || seg_r[s] > len) return ORACLE_BAD_ARG;
+    K += seg_k[s];
+  }
+  const size_t gsz = grad_dtype == GRAD_F32 ? 4 : 2;
+  for_each_row(W, [&](int w) {
+    int64_t at = 0;
+    for (int s = 0; s < S; ++s) {
+      const int64_t lo = seg_off[s], len = seg_off[s + 1] - lo;
+      sparsify_slice((const char*)grad + ((size_t)w * (size_t)ld_g + (size_t)lo) * gsz, grad_dtype,
+                     residual + (size_t)w * (size_t)ld_m + (size_t)lo, len, seg_r[s], seg_k[s],
+                     seed, step, (uint32_t)(worker_base + w), (uint32_t)s, (uint32_t)lo,
+                     msg_idx + (size_t)w * (size_t)K + (size_t)at,
+                     msg_val + (size_t)w * (size_t)K + (size_t)at);
+      at += seg_k[s];
+    }
+  });
+  return ORACLE_OK;
+}
+
+// Algorithm 1, master: dense sum of the W sparse messages in double precision,
+// workers in order, scaled by 1/W (mean) or 1 (sum).  out64 (optional) receives
+// the double result; out32 (optional) the same rounded once to binary32.
+int oracle_aggregate(const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
+                     int scale_mode, double* out64, float* out32) {
+  if (!msg_idx || !msg_val || d < 1 || W < 1 || k < 1) return ORACLE_BAD_ARG;
+  if (scale_mode != SCALE_MEAN && scale_mode != SCALE_SUM) return ORACLE_BAD_ARG;
+  std::vector<double> acc((size_t)d, 0.0);
+  for (int32_t w = 0; w < W; ++w)
+    for (int64_t q = 0; q < k; ++q) {
+      const uint32_t i = msg_idx[(size_t)w * (size_t)k + (size_t)q];
+      if ((int64_t)i >= d) return ORACLE_BAD_ARG;
+      acc[i] += (double)msg_val[(size_t)w * (size_t)k + (size_t)q];
+    }
+  for (int64_t i = 0; i < d; ++i) {
+    const double v = scale_mode == SCALE_MEAN ? acc[(size_t)i] / (double)W : acc[(size_t)i];
+    if (out64) out64[i] = v;
+    if (out32) out32[i] = (float)v;
+  }
+  return ORACLE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,372 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, checked without a GPU.
+
+Each test ties one piece of ``oracle/`` to something other than itself: published
+known answers (Philox), big-integer arithmetic (draw scaling), exhaustive enumeration
+(Floyd yields every k-subset equally often, Definition 3's "uniformly at random"),
+brute force and library sorts (Definition 1), the closed form in the proof of
+Proposition 1, the limits k = r (Definition 1) and r = d (Definition 2), and the
+identities of Algorithm 1 (m' = a - ghat; the master's 1/n average).
+"""
+import itertools
+import math
+import os
+from collections import Counter
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ----------------------------------------------------------------------------- Philox
+def _golden_lines(kind):
+    with open(os.path.join(GOLDEN, "philox4x32_10_known_answers.txt")) as f:
+        for line in f:
+            tok = line.split()
+            if tok and tok[0] == kind:
+                yield tok[1:]
+
+
+def test_philox_known_answers():
+    n = 0
+    for tok in _golden_lines("kat"):
+        w = [int(t, 16) for t in tok]
+        got = oracle.philox4x32_10(w[0:4], w[4:6])
+        assert [int(x) for x in got] == w[6:10]
+        n += 1
+    assert n >= 2
+
+
+def test_philox_cxx_standard_10000th_value():
+    for tok in _golden_lines("nth"):
+        n, seed, want = (int(t) for t in tok)
+        block, word = divmod(n - 1, 4)
+        got = oracle.philox4x32_10([block, 0, 0, 0], [seed, 0])
+        assert int(got[word]) == want
+
+
+def test_scale_draw_matches_big_integer_floor():
+    rng = np.random.default_rng(1)
+    cases = [(0, 1), (0, 7), (2**64 - 1, 1), (2**64 - 1, 7), (2**63, 2), (2**63 - 1, 2),
+             (2**64 - 1, 2**31), (2**64 - 1, 2**32 - 1)]
+    for _ in range(2000):
+        cases.append((int(rng.integers(0, 2**64, dtype=np.uint64)), int(rng.integers(1, 2**32))))
+    for u, n in cases:
+        assert oracle.scale_draw(u, n) == (u * n) >> 64
+
+
+def test_draw_uses_words_0_and_1_and_counter_layout():
+    # t_j = floor(((x1 << 32) | x0) * (j + 1) / 2^64), counter = (j, worker, segment, step),
+    # key = (seed lo, seed hi): the library's reading of "uniformly at random".
+    seed = 0x0123456789ABCDEF
+    for step, worker, seg, j in [(0, 0, 0, 0), (3, 2, 1, 77), (9, 31, 5, 2**28 - 1)]:
+        x = oracle.philox4x32_10([j, worker, seg, step], [seed & 0xFFFFFFFF, seed >> 32])
+        u = (int(x[1]) << 32) | int(x[0])
+        assert oracle.draw(seed, step, worker, seg, j) == (u * (j + 1)) >> 64
+
+
+def test_draw_streams_differ_across_seed_step_worker_segment():
+    base = [oracle.draw(7, 1, 2, 3, j) for j in range(1000, 1200)]
+    for args in [(8, 1, 2, 3), (7, 2, 2, 3), (7, 1, 3, 3), (7, 1, 2, 4), (7 + 2**32, 1, 2, 3)]:
+        other = [oracle.draw(*args, j) for j in range(1000, 1200)]
+        assert sum(a == b for a, b in zip(base, other)) < 10
+    assert all(0 <= t <= j for t, j in zip(base, range(1000, 1200)))
+
+
+# ----------------------------------------------------------------------------- Floyd
+@pytest.mark.parametrize("r", [1, 2, 3, 4, 5, 6, 7])
+def test_floyd_is_uniform_over_k_subsets_exhaustively(r):
+    # Over all admissible draw tuples every k-subset of {0..r-1} must appear equally often.
+    for k in range(1, r + 1):
+        ranges = [range(j + 1) for j in range(r - k, r)]
+        counts = Counter()
+        for t in itertools.product(*ranges):
+            pos = oracle.floyd_from_draws(r, k, np.array(t, dtype=np.uint32))
+            assert len(set(pos.tolist())) == k and list(pos) == sorted(pos)
+            counts[tuple(pos.tolist())] += 1
+        total = math.prod(j + 1 for j in range(r - k, r))
+        assert len(counts) == math.comb(r, k)
+        assert set(counts.values()) == {total // math.comb(r, k)}
+
+
+def test_floyd_limits():
+    # k = r: every position; k = 1: the single draw of iteration r-1
+    for r in (1, 5, 64):
+        t = np.array([oracle.draw(3, 0, 0, 0, j) for j in range(r)], dtype=np.uint32)
+        assert oracle.floyd_from_draws(r, r, t).tolist() == list(range(r))
+        assert oracle.sample_positions(r, r, 3, 0, 0).tolist() == list(range(r))
+    for r in (1, 9, 1000):
+        assert oracle.sample_positions(r, 1, 11, 4, 2, 1).tolist() == [oracle.draw(11, 4, 2, 1, r - 1)]
+    with pytest.raises(ValueError):
+        oracle.floyd_from_draws(4, 2, np.array([3, 0], dtype=np.uint32))  # t_2 = 3 > 2
+
+
+def _chi2_ok(observed, expected, dof, z=5.0):
+    stat = float(((observed - expected) ** 2 / expected).sum())
+    return abs(stat - dof) < z * math.sqrt(2 * dof), stat
+
+
+def test_sampler_inclusion_frequencies_are_k_over_r():
+    # each position is kept with probability k/r: its hit count over n seeds is Binomial(n, k/r)
+    r, k, n = 50, 10, 20000
+    hits = np.zeros(r)
+    for seed in range(n):
+        hits[oracle.sample_positions(r, k, seed, 0, 0)] += 1
+    assert hits.sum() == n * k
+    p = k / r
+    stat = float(((hits - n * p) ** 2 / (n * p * (1 - p))).sum())
+    assert abs(stat - r) < 6 * math.sqrt(2 * r), stat
+
+
+def test_sampler_subset_frequencies_small_case():
+    r, k, n = 5, 2, 20000
+    counts = Counter()
+    for step in range(n):
+        counts[tuple(oracle.sample_positions(r, k, 99, step, 1).tolist())] += 1
+    obs = np.array([counts[c] for c in itertools.combinations(range(r), k)], dtype=float)
+    ok, stat = _chi2_ok(obs, n / math.comb(r, k), math.comb(r, k) - 1)
+    assert ok, stat
+
+
+# ----------------------------------------------------------------------------- top-r
+def _key(x: np.ndarray) -> np.ndarray:
+    return np.ascontiguousarray(x, dtype=np.float32).view(np.uint32) & 0x7FFFFFFF
+
+
+def brute_top_r(a, r):
+    """Definition 1 with ties to the lower index, by a plain Python sort."""
+    key = _key(a).tolist()
+    order = sorted(range(len(key)), key=lambda i: (-key[i], i))
+    return sorted(order[:r])
+
+
+def test_top_r_brute_force_tiny_with_ties():
+    values = np.array([0.0, -0.0, 0.5, -0.5, 1.0, -2.0], dtype=np.float32)
+    for d in range(1, 6):
+        for combo in itertools.product(range(len(values)), repeat=d):
+            a = values[list(combo)]
+            for r in range(1, d + 1):
+                assert oracle.top_r(a, r).tolist() == brute_top_r(a, r)
+
+
+def test_top_r_matches_library_sorts_on_tie_free_data():
+    rng = np.random.default_rng(5)
+    d = 20011
+    mags = rng.permutation(d).astype(np.float32) * np.float32(0.125) + np.float32(1.0)
+    a = (mags * rng.choice([-1.0, 1.0], d)).astype(np.float32)
+    assert len(np.unique(np.abs(a))) == d
+    order = np.argsort(-np.abs(a).astype(np.float64), kind="stable")
+    for r in (1, 2, 100, d // 100, d - 1, d):
+        got = oracle.top_r(a, r)
+        assert got.tolist() == sorted(order[:r].tolist())
+        tk = torch.topk(torch.from_numpy(np.abs(a)), r).indices.numpy()
+        assert set(got.tolist()) == set(tk.tolist())
+
+
+def test_top_r_adversarial_ties_and_specials():
+    a = np.full(1000, -3.25, dtype=np.float32)
+    assert oracle.top_r(a, 17).tolist() == list(range(17))
+    # duplicated magnitudes across the threshold: the lower indices win
+    a = np.array([1, -2, 2, 1, -2, 0, 2, 1], dtype=np.float32)
+    assert oracle.top_r(a, 3).tolist() == [1, 2, 4]
+    assert oracle.top_r(a, 5).tolist() == [0, 1, 2, 4, 6]
+    # order by bit pattern with the sign cleared: NaN > Inf > finite > denormal > zero
+    a = np.array([0.0, 1e-45, -np.inf, np.nan, 3e38, -1e-45, -0.0], dtype=np.float32)
+    assert oracle.top_r(a, 1).tolist() == [3]
+    assert oracle.top_r(a, 2).tolist() == [2, 3]
+    assert oracle.top_r(a, 3).tolist() == [2, 3, 4]
+    assert oracle.top_r(a, 4).tolist() == [1, 2, 3, 4]
+    assert oracle.top_r(a, 6).tolist() == [0, 1, 2, 3, 4, 5]
+
+
+# ----------------------------------------------------------------------------- node body
+def _spiky(rng, W, d):
+    x = rng.standard_normal((W, d)) * 1e-3
+    m = rng.random((W, d)) < 0.05
+    return np.where(m, rng.standard_normal((W, d)), x).astype(np.float32)
+
+
+def _scatter(idx, val, d):
+    out = np.zeros(d, dtype=np.float32)
+    out[idx] = val
+    return out
+
+
+@pytest.mark.parametrize("d,r,k", [(1, 1, 1), (2, 2, 1), (5, 3, 2), (33, 7, 7), (1023, 100, 10),
+                                   (4097, 4097, 41), (4098, 400, 1)])
+def test_sparsify_identities_of_algorithm_1(d, r, k):
+    rng = np.random.default_rng(d)
+    W = 3
+    g = _spiky(rng, W, d)
+    m0 = _spiky(rng, W, d) * 0.5
+    a = g + m0                                     # numpy float32 add: IEEE round-to-nearest
+    m = m0.copy()
+    idx, val = oracle.sparsify(g, m, d, r, k, seed=42, step=6, worker_base=10)
+    for w in range(W):
+        T = brute_top_r(a[w], r)
+        pos = oracle.sample_positions(r, k, 42, 6, 10 + w, 0)
+        want = [T[p] for p in pos]
+        assert idx[w].tolist() == want                           # U = k-subset of the top-r set
+        assert len(set(want)) == k and set(want) <= set(T)
+        assert val[w].view(np.uint32).tolist() == a[w][want].view(np.uint32).tolist()
+        assert (m[w][want].view(np.uint32) == 0).all()           # sent slots hold +0.0
+        back = m[w].copy()
+        back[want] = val[w]
+        assert (back.view(np.uint32) == a[w].view(np.uint32)).all()   # sent + residual = a
+        assert np.count_nonzero(_scatter(idx[w], val[w], d)) <= k
+
+
+def test_limit_k_equals_r_is_top_r():
+    rng = np.random.default_rng(8)
+    d, r = 5000, 123
+    g = np.stack([rng.permutation(d) + 1.0 for _ in range(2)]) * rng.choice([-1.0, 1.0], (2, d))
+    g = (g * 0.25).astype(np.float32)               # distinct magnitudes: top-r is unique
+    m = np.zeros_like(g)
+    idx, val = oracle.sparsify(g, m, d, r, r, seed=1, step=0)
+    for w in range(2):
+        want = np.sort(np.argsort(-np.abs(g[w]), kind="stable")[:r])
+        assert idx[w].tolist() == want.tolist()
+        # top_r(a) itself: a - m' is a on the top-r set and 0 elsewhere
+        assert np.array_equal(g[w] - m[w], _scatter(want, g[w][want], d))
+
+
+def test_limit_r_equals_d_is_random_k():
+    rng = np.random.default_rng(9)
+    d, k = 3001, 30
+    g1 = rng.standard_normal((2, d)).astype(np.float32)
+    g2 = rng.standard_normal((2, d)).astype(np.float32)
+    i1, v1 = oracle.sparsify(g1, np.zeros_like(g1), d, d, k, seed=5, step=2)
+    i2, v2 = oracle.sparsify(g2, np.zeros_like(g2), d, d, k, seed=5, step=2)
+    assert np.array_equal(i1, i2)                     # the subset does not look at the values
+    for w in range(2):
+        assert i1[w].tolist() == oracle.sample_positions(d, k, 5, 2, w).tolist()
+        assert np.array_equal(v1[w], g1[w][i1[w]])
+
+
+def test_proposition_1_closed_form_monte_carlo():
+    # E||a - rTop_k(a)||^2 = (1 - k/r) sum_{j<=r} a_(j)^2 + sum_{j>r} a_(j)^2   (proof of Prop. 1),
+    # E[rTop_k(a)] = (k/r) top_r(a), and every draw satisfies ||a - C(a)||^2 <= ||a||^2.
+    rng = np.random.default_rng(10)
+    d, r, k, n = 300, 40, 10, 6000
+    a = (rng.standard_normal(d) * np.exp(rng.standard_normal(d))).astype(np.float32)
+    sq = np.sort(a.astype(np.float64) ** 2)[::-1]
+    closed = (1 - k / r) * sq[:r].sum() + sq[r:].sum()
+    errs = np.zeros(n)
+    mean_vec = np.zeros(d)
+    g = np.repeat(a[None, :], 1, axis=0)
+    for s in range(n):
+        m = np.zeros((1, d), dtype=np.float32)
+        idx, val = oracle.sparsify(g, m, d, r, k, seed=1000 + s, step=s % 7)
+        errs[s] = (m[0].astype(np.float64) ** 2).sum()
+        mean_vec[idx[0]] += val[0]
+    assert (errs <= (a.astype(np.float64) ** 2).sum() + 1e-9).all()
+    assert abs(errs.mean() - closed) < 4 * errs.std() / math.sqrt(n)
+    assert abs(closed - (1 - k / d) * sq.sum()) >= 0 and closed <= (1 - k / d) * sq.sum() + 1e-9
+    top = np.zeros(d)
+    T = brute_top_r(a, r)
+    top[T] = a[T]
+    dev = mean_vec / n - (k / r) * top
+    sigma = np.sqrt((k / r) * (1 - k / r) / n) * np.abs(top)
+    assert (np.abs(dev) <= 5 * sigma + 1e-12).all()
+
+
+def test_step_counter_and_resume():
+    rng = np.random.default_rng(11)
+    W, d, r, k = 2, 2000, 100, 20
+    grads = [_spiky(rng, W, d) for _ in range(6)]
+    m_all = np.zeros((W, d), dtype=np.float32)
+    out_all = [oracle.sparsify(grads[t], m_all, d, r, k, seed=3, step=t) for t in range(6)]
+    m_a = np.zeros((W, d), dtype=np.float32)
+    for t in range(3):
+        oracle.sparsify(grads[t], m_a, d, r, k, seed=3, step=t)
+    m_b = m_a.copy()                                  # "checkpoint": the residual is the only state
+    out_b = [oracle.sparsify(grads[t], m_b, d, r, k, seed=3, step=t) for t in range(3, 6)]
+    assert np.array_equal(m_b.view(np.uint32), m_all.view(np.uint32))
+    for (i1, v1), (i2, v2) in zip(out_all[3:], out_b):
+        assert np.array_equal(i1, i2) and np.array_equal(v1.view(np.uint32), v2.view(np.uint32))
+
+
+def test_bf16_gradient_is_widened_exactly():
+    rng = np.random.default_rng(12)
+    W, d, r, k = 2, 999, 50, 5
+    gf = torch.from_numpy(_spiky(rng, W, d)).to(torch.bfloat16)
+    bits = gf.view(torch.int16).numpy().view(np.uint16).copy()
+    m0 = _spiky(rng, W, d)
+    m1, m2 = m0.copy(), m0.copy()
+    i1, v1 = oracle.sparsify(bits, m1, d, r, k, seed=1, step=1)
+    i2, v2 = oracle.sparsify(gf.to(torch.float32).numpy().copy(), m2, d, r, k, seed=1, step=1)
+    assert np.array_equal(i1, i2) and np.array_equal(v1.view(np.uint32), v2.view(np.uint32))
+    assert np.array_equal(m1.view(np.uint32), m2.view(np.uint32))
+
+
+def test_segmented_is_rtopk_per_slice():
+    rng = np.random.default_rng(13)
+    W, sizes = 2, [700, 301, 1024, 5]
+    off = np.concatenate([[0], np.cumsum(sizes)])
+    d = int(off[-1])
+    seg_r = [70, 301, 10, 2]
+    seg_k = [7, 30, 10, 1]
+    g = _spiky(rng, W, d)
+    m0 = _spiky(rng, W, d)
+    m = m0.copy()
+    idx, val = oracle.sparsify_segmented(g, m, d, off, seg_r, seg_k, seed=21, step=4, worker_base=3)
+    a = g + m0
+    for w in range(W):
+        at = 0
+        for s, (lo, n) in enumerate(zip(off[:-1], sizes)):
+            T = brute_top_r(a[w, lo:lo + n], seg_r[s])
+            pos = oracle.sample_positions(seg_r[s], seg_k[s], 21, 4, 3 + w, s)
+            want = [int(lo) + T[p] for p in pos]
+            assert idx[w, at:at + seg_k[s]].tolist() == want
+            assert np.array_equal(val[w, at:at + seg_k[s]], a[w][want])
+            at += seg_k[s]
+        back = m[w].copy()
+        back[idx[w]] = val[w]
+        assert np.array_equal(back.view(np.uint32), a[w].view(np.uint32))
+    # one segment covering the vector is the plain operator
+    m1, m2 = m0.copy(), m0.copy()
+    i1, v1 = oracle.sparsify_segmented(g, m1, d, [0, d], [90], [9], seed=2, step=0)
+    i2, v2 = oracle.sparsify(g, m2, d, 90, 9, seed=2, step=0)
+    assert np.array_equal(i1, i2) and np.array_equal(v1, v2) and np.array_equal(m1, m2)
+
+
+# ----------------------------------------------------------------------------- master
+def test_aggregate_worked_example():
+    # two workers, d = 4: worker 0 sends (0: 1, 2: 2), worker 1 sends (2: 4, 3: 8)
+    idx = np.array([[0, 2], [2, 3]], dtype=np.uint32)
+    val = np.array([[1, 2], [4, 8]], dtype=np.float32)
+    o64, o32 = oracle.aggregate(idx, val, 4)
+    assert o64.tolist() == [0.5, 0.0, 3.0, 4.0] and o32.tolist() == [0.5, 0.0, 3.0, 4.0]
+    s64, _ = oracle.aggregate(idx, val, 4, oracle.SCALE_SUM)
+    assert s64.tolist() == [1.0, 0.0, 6.0, 8.0]
+
+
+def test_aggregate_against_numpy_and_special_cases():
+    rng = np.random.default_rng(14)
+    d, W, k = 5000, 5, 400
+    idx = np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)]).astype(np.uint32)
+    val = (rng.standard_normal((W, k)) * np.exp(3 * rng.standard_normal((W, k)))).astype(np.float32)
+    o64, o32 = oracle.aggregate(idx, val, d)
+    ref = np.zeros(d)
+    np.add.at(ref, idx.ravel().astype(np.int64), val.ravel().astype(np.float64))
+    # the sum of five doubles depends on order only in the last bits
+    assert np.allclose(o64, ref / W, rtol=1e-14, atol=0)
+    assert np.array_equal(o32, o64.astype(np.float32))
+    # W = 1: the update is the message itself
+    o64, o32 = oracle.aggregate(idx[:1], val[:1], d)
+    assert np.array_equal(o32, _scatter(idx[0], val[0], d))
+    # disjoint supports: exact
+    idx_d = np.arange(W * k, dtype=np.uint32).reshape(W, k)
+    o64, _ = oracle.aggregate(idx_d, val, d)
+    assert np.array_equal(o64[: W * k], val.ravel().astype(np.float64) / W)
+
+
+def test_bad_arguments_are_rejected():
+    g = np.zeros((1, 8), dtype=np.float32)
+    m = np.zeros((1, 8), dtype=np.float32)
+    for d, r, k in [(8, 4, 5), (8, 9, 1), (8, 4, 0), (9, 4, 1)]:
+        with pytest.raises(ValueError):
+            oracle.sparsify(g, m, d, r, k, seed=0, step=0)
