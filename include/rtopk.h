@@ -1,0 +1,197 @@
+/*
+ * rtopk.h -- C ABI of the rTop-k sparsification / aggregation library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the data-parallel hot path of
+ *   Barnes, Inan, Isik, Ozgur, "rTop-k: A Statistical Estimation Approach to Distributed SGD":
+ * for W workers whose gradient vectors are held as the rows of one matrix on one GPU,
+ *
+ *   node body   (Algorithm 1):  a = g + m ;  ghat = rTop_k(a) ;  m' = a - ghat ;  send ghat
+ *   rTop_k      (Definition 3): keep a uniformly random k-subset U of the r largest-magnitude
+ *                               coordinates (Definition 1, top-r), zero the rest
+ *   master      (Algorithm 1):  ghat = (1/n) sum_i ghat_i          (n = W here)
+ *
+ * Conventions fixed where the paper is silent:
+ *   - magnitudes are ordered by the binary32 bit pattern with the sign cleared; ties go to the
+ *     lower index ("pi is a permutation" in Definition 1 leaves this open);
+ *   - U is drawn with Floyd's subset algorithm over positions 0..r-1 of the top-r set listed by
+ *     ascending index; iteration j (j = r-k .. r-1) draws t_j = floor(u64 * (j+1) / 2^64) with
+ *     u64 = (x1 << 32) | x0 and (x0..x3) = Philox4x32-10(counter = (j, worker, segment, step),
+ *     key = (seed low word, seed high word)); t_j joins U's positions unless already there, in
+ *     which case j does;
+ *   - a, m, message values and the dense update are binary32; g may be binary32 or bfloat16
+ *     (widened exactly); the add is one round-to-nearest add, and a NaN sum is stored as the
+ *     default quiet NaN 0x7FC00000 (IEEE 754 leaves NaN payloads to the implementation);
+ *   - a message is k (index, value) pairs in ascending index order; m' is a bit copy of a
+ *     outside U and +0.0f on U.
+ *
+ * Pointers are DEVICE pointers owned by the caller unless a parameter is documented as host
+ * memory.  Calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL = default stream)
+ * and return without synchronising unless stated.  Every function returns an rtopk_status; on a
+ * non-zero status detected on the host nothing has been enqueued and no buffer was written.
+ * Conditions only the device can detect (an internal bounded wait that gave up) are reported by
+ * rtopk_poll_status.  A context serialises its scratch memory: calls that share a context must be
+ * ordered on one stream (or otherwise not overlap on the GPU).
+ */
+#ifndef RTOPK_H_
+#define RTOPK_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct rtopk_ctx rtopk_ctx;
+
+typedef enum {
+  RTOPK_OK = 0,
+  RTOPK_ERR_INVALID_ARG = 1, /* null/misaligned pointer, size out of range, k > r, r > d, ... */
+  RTOPK_ERR_ALLOC = 2,       /* device or host allocation failed */
+  RTOPK_ERR_CUDA = 3,        /* a CUDA runtime call failed; see rtopk_last_cuda_error */
+  RTOPK_ERR_UNSUPPORTED = 4, /* valid request the build does not cover */
+  RTOPK_ERR_INTERNAL = 5     /* device-side bounded wait expired or an internal invariant broke */
+} rtopk_status;
+
+/* gradient element type; residual, message values and the update are always binary32 */
+enum { RTOPK_F32 = 0, RTOPK_BF16 = 1 };
+
+/* scaling of the aggregated update: 1/W as in Algorithm 1's master step, or the plain sum */
+enum { RTOPK_SCALE_MEAN = 0, RTOPK_SCALE_SUM = 1 };
+
+/* rtopk_set_option keys */
+enum {
+  RTOPK_OPT_SELECT_PATH = 0, /* 0 = automatic (sampled threshold with exact fallback),
+                                1 = always the multi-pass radix select over the full vector */
+  RTOPK_OPT_PROFILE = 1      /* 1 = record CUDA events between the phases of each call on the
+                                caller's stream (read with rtopk_get_phase_times); 0 = off */
+};
+
+/* Phases of one call, in stream order.  STREAM is the single pass over the full vectors that
+ * performs a = g + m, writes it back and gathers the coordinates above the threshold. */
+enum {
+  RTOPK_PHASE_SUBSET = 0,    /* scratch clearing + the k-of-r subset (Definition 3's U, as positions) */
+  RTOPK_PHASE_THRESHOLD = 1, /* sampled threshold estimate */
+  RTOPK_PHASE_STREAM = 2,    /* fused add / write-back / candidate gathering over W x d elements */
+  RTOPK_PHASE_EXACT = 3,     /* full-vector radix passes (fallback; near-empty launches otherwise) */
+  RTOPK_PHASE_SELECT = 4,    /* exact r-th largest among the candidates */
+  RTOPK_PHASE_EMIT = 5,      /* messages + residual zeroing (m' = a - ghat) */
+  RTOPK_PHASE_AGGREGATE = 6, /* master average (rtopk_step only) */
+  RTOPK_N_PHASES = 7
+};
+
+/* Per-slice facts of the last sparsify call (one slice = one worker row, or one tensor of one
+ * worker row in the segmented calls). */
+typedef struct {
+  uint32_t tau_key;     /* bit pattern (sign cleared) of the r-th largest magnitude */
+  uint32_t tie_quota;   /* how many coordinates with exactly that magnitude are inside the top-r set */
+  uint32_t n_greater;   /* coordinates with a strictly larger magnitude */
+  uint32_t n_candidates;/* coordinates that survived the first threshold */
+  uint32_t used_fallback; /* 1 if the sampled threshold missed and the full radix select ran */
+  uint32_t reserved[3];
+} rtopk_stats;
+
+int rtopk_version(void);
+const char* rtopk_status_string(int status);
+/* cudaError_t (as int) of the last failing runtime call seen by this context, 0 if none. */
+int rtopk_last_cuda_error(const rtopk_ctx* ctx);
+
+/*
+ * Creates a context on `device` with scratch sized for calls up to the given maxima:
+ * vectors of at most d_max elements, W_max rows, r_max / k_max per slice summed over a row's
+ * slices (for the plain calls: r and k), segments_max slices per row (1 for the plain calls).
+ * The context owns its scratch (cudaMalloc) until rtopk_destroy.  d_max < 2^31.
+ * Errors: INVALID_ARG, ALLOC, CUDA.
+ */
+int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int64_t r_max,
+                 int64_t k_max, int32_t segments_max);
+int rtopk_destroy(rtopk_ctx* ctx);
+int rtopk_set_option(rtopk_ctx* ctx, int option, int64_t value);
+
+/*
+ * Algorithm 1, node body, for W workers at once (add residual, Definition 3, residual update).
+ *   grad      [in]      W x ld_g elements of grad_dtype, row-major; row w is worker worker_base+w;
+ *                       never written.
+ *   residual  [in/out]  W x ld_m binary32; on entry m (zero before the first step), on return m'.
+ *   d                   vector length, 1 <= k <= r <= d < 2^31 (Definition 3's 1 <= k <= r <= d).
+ *   ld_g, ld_m          row strides in elements, >= d, multiples of 4 (binary32) / 8 (bfloat16);
+ *                       base pointers 16-byte aligned.  Padding columns are neither read nor written.
+ *   worker_base         global id of row 0; enters the Philox counter so that a run sharded over
+ *                       several GPUs draws the same subsets as the single-GPU run.
+ *   seed, step          RNG key and the training step t; the caller advances step every round.
+ *   msg_idx, msg_val [out]  W x k: row w holds worker w's k (index, value) pairs, ascending index.
+ * Errors: INVALID_ARG (also when a size exceeds the context's maxima), CUDA.
+ */
+int rtopk_sparsify(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,
+                   int64_t ld_m, int64_t d, int32_t W, int32_t worker_base, int64_t r, int64_t k,
+                   uint64_t seed, uint32_t step, uint32_t* msg_idx, float* msg_val, void* stream);
+
+/*
+ * Algorithm 1, master step: out_i = scale * sum_w [i in U_w] val_{w,i}, scale = 1/W or 1.
+ * Sums run in double precision in worker order and are rounded once, so the result does not depend
+ * on scheduling.  msg_idx rows must be ascending (as rtopk_sparsify writes them) with entries < d.
+ *   msg_idx, msg_val [in]  W x k;   out [out]  d binary32, fully overwritten.
+ * Errors: INVALID_ARG, CUDA.
+ */
+int rtopk_aggregate(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d,
+                    int32_t W, int64_t k, int scale_mode, float* out, void* stream);
+
+/* One round of Algorithm 1's communication path: rtopk_sparsify followed by rtopk_aggregate of
+ * the W messages it produced.  Arguments as in the two calls. */
+int rtopk_step(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,
+               int64_t ld_m, int64_t d, int32_t W, int32_t worker_base, int64_t r, int64_t k,
+               uint64_t seed, uint32_t step, int scale_mode, uint32_t* msg_idx, float* msg_val,
+               float* out, void* stream);
+
+/*
+ * Per-tensor variant: every row is cut into S slices at seg_off[0..S] (HOST array, seg_off[0] = 0,
+ * seg_off[S] = d) and Definition 3 is applied to each slice with its own (seg_r[s], seg_k[s])
+ * (HOST arrays), the slice number entering the Philox counter.  A row's message has
+ * K = sum_s seg_k[s] pairs: slice 0's first; indices are positions in the whole vector, so the
+ * row is still ascending and rtopk_aggregate applies unchanged with k = K.
+ * The host arrays are read before the call returns.
+ */
+int rtopk_sparsify_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g,
+                             float* residual, int64_t ld_m, int64_t d, int32_t W,
+                             int32_t worker_base, int32_t S, const int64_t* seg_off,
+                             const int64_t* seg_r, const int64_t* seg_k, uint64_t seed,
+                             uint32_t step, uint32_t* msg_idx, float* msg_val, void* stream);
+int rtopk_step_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g,
+                         float* residual, int64_t ld_m, int64_t d, int32_t W, int32_t worker_base,
+                         int32_t S, const int64_t* seg_off, const int64_t* seg_r,
+                         const int64_t* seg_k, uint64_t seed, uint32_t step, int scale_mode,
+                         uint32_t* msg_idx, float* msg_val, float* out, void* stream);
+
+/*
+ * rtopk_step with HOST gradient and HOST results: copies h_grad (W x ld_g, ideally pinned) to a
+ * device staging buffer owned by the context (allocated on first use), runs the step against the
+ * DEVICE residual, and copies the messages and the dense update back to h_msg_idx, h_msg_val
+ * (W x k) and h_out (d).  All copies are enqueued on `stream`; the call returns without waiting.
+ */
+int rtopk_step_host(rtopk_ctx* ctx, const void* h_grad, int grad_dtype, int64_t ld_g,
+                    float* residual, int64_t ld_m, int64_t d, int32_t W, int32_t worker_base,
+                    int64_t r, int64_t k, uint64_t seed, uint32_t step, int scale_mode,
+                    uint32_t* h_msg_idx, float* h_msg_val, float* h_out, void* stream);
+
+/*
+ * The k-of-r subset alone (Definition 3's U as positions in the top-r list): writes the k chosen
+ * positions of (seed, step, worker, segment), ascending, to pos (device, k entries).
+ */
+int rtopk_sample_positions(rtopk_ctx* ctx, int64_t r, int64_t k, uint64_t seed, uint32_t step,
+                           uint32_t worker, uint32_t segment, uint32_t* pos, void* stream);
+
+/* Waits for `stream` and returns RTOPK_ERR_INTERNAL if any kernel of this context has raised the
+ * device-side error flag since the last poll (the flag is then cleared), else RTOPK_OK. */
+int rtopk_poll_status(rtopk_ctx* ctx, void* stream);
+
+/* Waits for `stream`, then writes the duration in milliseconds of each phase of the last call
+ * made with RTOPK_OPT_PROFILE on into ms[0..RTOPK_N_PHASES) (host); -1 where not recorded. */
+int rtopk_get_phase_times(rtopk_ctx* ctx, float* ms, void* stream);
+
+/* Waits for `stream` and copies the statistics of slice `slice` (row-major over rows x segments)
+ * of the last sparsify call into *out (host). */
+int rtopk_get_stats(rtopk_ctx* ctx, int32_t slice, rtopk_stats* out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RTOPK_H_ */

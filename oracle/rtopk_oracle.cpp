@@ -24,6 +24,8 @@
 //   * a, m, message values and the update are IEEE binary32; the add is one
 //     round-to-nearest add; magnitudes are compared through the bit pattern
 //     with the sign cleared (so NaN > Inf > finite, and -0 ties with +0);
+//   * IEEE 754 leaves the payload of a NaN result to the implementation, so a NaN sum is stored as
+//     the default quiet NaN (bit pattern 0x7FC00000);
 //   * m' is a bit copy of a outside the sent set and +0.0f inside it;
 //   * messages are listed by ascending index.
 //
@@ -143,7 +145,8 @@ void sparsify_slice(const void* grad, int dtype, float* residual, int64_t d, int
                     uint32_t idx_base, uint32_t* msg_idx, float* msg_val) {
   // a = g + m   (materialised in the residual buffer)
   for (int64_t i = 0; i < d; ++i) {
-    const float s = widen_grad(grad, dtype, i) + residual[i];   // one binary32 add
+    float s = widen_grad(grad, dtype, i) + residual[i];   // one binary32 add
+    if (s != s) s = bits_float(0x7FC00000u);              // NaN payloads are not portable: store the default NaN
     residual[i] = s;
   }
   // I <- indices of the r largest-magnitude components

@@ -1,0 +1,203 @@
+"""ctypes binding of librtopk.so with the same entry-point names as include/rtopk.h.
+
+Argument marshalling only: every step of the path runs in the library's kernels.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "librtopk.so")
+
+GRAD_F32, GRAD_BF16 = 0, 1
+SCALE_MEAN, SCALE_SUM = 0, 1
+OPT_SELECT_PATH, OPT_PROFILE = 0, 1
+PHASES = ("subset", "threshold", "stream", "exact", "select", "emit", "aggregate")
+
+_vp, _i32, _i64, _u32, _u64, _int = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_uint64, C.c_int
+
+# name -> (restype, argtypes); every symbol include/rtopk.h declares
+EXPORTS = {
+    "rtopk_version": (_int, []),
+    "rtopk_status_string": (C.c_char_p, [_int]),
+    "rtopk_last_cuda_error": (_int, [_vp]),
+    "rtopk_create": (_int, [C.POINTER(_vp), _int, _i64, _i32, _i64, _i64, _i32]),
+    "rtopk_destroy": (_int, [_vp]),
+    "rtopk_set_option": (_int, [_vp, _int, _i64]),
+    "rtopk_sparsify": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _i64, _u64, _u32,
+                              _vp, _vp, _vp]),
+    "rtopk_aggregate": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _int, _vp, _vp]),
+    "rtopk_step": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _i64, _u64, _u32, _int,
+                          _vp, _vp, _vp, _vp]),
+    "rtopk_sparsify_segmented": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i32,
+                                        C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64), _u64, _u32,
+                                        _vp, _vp, _vp]),
+    "rtopk_step_segmented": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i32,
+                                    C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64), _u64, _u32, _int,
+                                    _vp, _vp, _vp, _vp]),
+    "rtopk_step_host": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _i64, _u64, _u32,
+                               _int, _vp, _vp, _vp, _vp]),
+    "rtopk_sample_positions": (_int, [_vp, _i64, _i64, _u64, _u32, _u32, _u32, _vp, _vp]),
+    "rtopk_poll_status": (_int, [_vp, _vp]),
+    "rtopk_get_phase_times": (_int, [_vp, _vp, _vp]),
+    "rtopk_get_stats": (_int, [_vp, _i32, _vp, _vp]),
+}
+
+_lib: Optional[C.CDLL] = None
+
+
+class RTopKError(RuntimeError):
+    def __init__(self, status: int, what: str, detail: str = ""):
+        self.status = status
+        super().__init__(f"{what}: status {status} ({detail})")
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library() -> C.CDLL:
+    """Loads librtopk.so and declares every exported symbol.  Raises if it is not built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2005_10761_b200.build` "
+                               "(there is no CPU fallback)")
+        lib = C.CDLL(_LIB_PATH)
+        for name, (res, args) in EXPORTS.items():
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = lib
+    return _lib
+
+
+class Stats(C.Structure):
+    _fields_ = [("tau_key", _u32), ("tie_quota", _u32), ("n_greater", _u32), ("n_candidates", _u32),
+                ("used_fallback", _u32), ("reserved", _u32 * 3)]
+
+
+def _i64_array(xs: Sequence[int]):
+    return (_i64 * len(xs))(*[int(x) for x in xs])
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+class RTopK:
+    """A library context on one device.  Methods mirror the C entry points; tensors must live on
+    that device (except the pinned host tensors of :meth:`step_host`) and are passed by pointer."""
+
+    def __init__(self, d_max: int, W_max: int, r_max: int, k_max: int, segments_max: int = 1,
+                 device: Optional[int] = None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("rTop-k needs a CUDA device: there is no CPU fallback")
+        self._lib = load_library()
+        self.device = torch.cuda.current_device() if device is None else int(device)
+        h = _vp()
+        rc = self._lib.rtopk_create(C.byref(h), self.device, d_max, W_max, r_max, k_max, segments_max)
+        self._h = h
+        if rc != 0:
+            self._h = None
+            raise RTopKError(rc, "rtopk_create", self._lib.rtopk_status_string(rc).decode())
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            self._lib.rtopk_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc: int, what: str) -> None:
+        if rc != 0:
+            detail = self._lib.rtopk_status_string(rc).decode()
+            if rc == 3:
+                detail += f", cudaError {self._lib.rtopk_last_cuda_error(self._h)}"
+            raise RTopKError(rc, what, detail)
+
+    @staticmethod
+    def _grad_dtype(grad: torch.Tensor) -> int:
+        if grad.dtype == torch.float32:
+            return GRAD_F32
+        if grad.dtype == torch.bfloat16:
+            return GRAD_BF16
+        raise TypeError("gradient must be float32 or bfloat16")
+
+    def set_option(self, option: int, value: int) -> None:
+        self._check(self._lib.rtopk_set_option(self._h, option, value), "rtopk_set_option")
+
+    def sparsify(self, grad, residual, d, r, k, seed, step, msg_idx, msg_val, worker_base=0) -> None:
+        W = grad.shape[0]
+        rc = self._lib.rtopk_sparsify(self._h, grad.data_ptr(), self._grad_dtype(grad), grad.stride(0),
+                                      residual.data_ptr(), residual.stride(0), d, W, worker_base, r, k,
+                                      seed, step, msg_idx.data_ptr(), msg_val.data_ptr(), _stream())
+        self._check(rc, "rtopk_sparsify")
+
+    def aggregate(self, msg_idx, msg_val, d, out, scale_mode=SCALE_MEAN) -> None:
+        W, k = msg_idx.shape
+        rc = self._lib.rtopk_aggregate(self._h, msg_idx.data_ptr(), msg_val.data_ptr(), d, W, k, scale_mode,
+                                       out.data_ptr(), _stream())
+        self._check(rc, "rtopk_aggregate")
+
+    def step(self, grad, residual, d, r, k, seed, step, msg_idx, msg_val, out, worker_base=0,
+             scale_mode=SCALE_MEAN) -> None:
+        W = grad.shape[0]
+        rc = self._lib.rtopk_step(self._h, grad.data_ptr(), self._grad_dtype(grad), grad.stride(0),
+                                  residual.data_ptr(), residual.stride(0), d, W, worker_base, r, k, seed, step,
+                                  scale_mode, msg_idx.data_ptr(), msg_val.data_ptr(), out.data_ptr(), _stream())
+        self._check(rc, "rtopk_step")
+
+    def sparsify_segmented(self, grad, residual, d, seg_off, seg_r, seg_k, seed, step, msg_idx, msg_val,
+                           worker_base=0) -> None:
+        W, S = grad.shape[0], len(seg_r)
+        rc = self._lib.rtopk_sparsify_segmented(self._h, grad.data_ptr(), self._grad_dtype(grad), grad.stride(0),
+                                                residual.data_ptr(), residual.stride(0), d, W, worker_base, S,
+                                                _i64_array(seg_off), _i64_array(seg_r), _i64_array(seg_k),
+                                                seed, step, msg_idx.data_ptr(), msg_val.data_ptr(), _stream())
+        self._check(rc, "rtopk_sparsify_segmented")
+
+    def step_segmented(self, grad, residual, d, seg_off, seg_r, seg_k, seed, step, msg_idx, msg_val, out,
+                       worker_base=0, scale_mode=SCALE_MEAN) -> None:
+        W, S = grad.shape[0], len(seg_r)
+        rc = self._lib.rtopk_step_segmented(self._h, grad.data_ptr(), self._grad_dtype(grad), grad.stride(0),
+                                            residual.data_ptr(), residual.stride(0), d, W, worker_base, S,
+                                            _i64_array(seg_off), _i64_array(seg_r), _i64_array(seg_k), seed,
+                                            step, scale_mode, msg_idx.data_ptr(), msg_val.data_ptr(),
+                                            out.data_ptr(), _stream())
+        self._check(rc, "rtopk_step_segmented")
+
+    def step_host(self, h_grad, residual, d, r, k, seed, step, h_msg_idx, h_msg_val, h_out, worker_base=0,
+                  scale_mode=SCALE_MEAN) -> None:
+        W = h_grad.shape[0]
+        rc = self._lib.rtopk_step_host(self._h, h_grad.data_ptr(), self._grad_dtype(h_grad), h_grad.stride(0),
+                                       residual.data_ptr(), residual.stride(0), d, W, worker_base, r, k, seed,
+                                       step, scale_mode, h_msg_idx.data_ptr(), h_msg_val.data_ptr(),
+                                       h_out.data_ptr(), _stream())
+        self._check(rc, "rtopk_step_host")
+
+    def sample_positions(self, r, k, seed, step, worker, segment, pos) -> None:
+        rc = self._lib.rtopk_sample_positions(self._h, r, k, seed, step, worker, segment, pos.data_ptr(),
+                                              _stream())
+        self._check(rc, "rtopk_sample_positions")
+
+    def poll_status(self) -> None:
+        self._check(self._lib.rtopk_poll_status(self._h, _stream()), "rtopk_poll_status")
+
+    def phase_times(self) -> dict:
+        ms = (C.c_float * len(PHASES))()
+        self._check(self._lib.rtopk_get_phase_times(self._h, ms, _stream()), "rtopk_get_phase_times")
+        return {name: float(ms[i]) for i, name in enumerate(PHASES)}
+
+    def stats(self, slice_index: int) -> dict:
+        s = Stats()
+        self._check(self._lib.rtopk_get_stats(self._h, slice_index, C.byref(s), _stream()), "rtopk_get_stats")
+        return {f: getattr(s, f) for f, _ in Stats._fields_ if f != "reserved"}

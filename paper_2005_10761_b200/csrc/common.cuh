@@ -1,0 +1,272 @@
+// Shared device-side definitions of the rTop-k library: slice descriptors, selection state,
+// scans, the bounded decoupled look-back and Philox4x32-10.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace rtopk {
+
+// ----------------------------------------------------------------------------- geometry
+constexpr int kThreads = 256;                 // threads per block of the streaming kernels
+constexpr int kWarps = kThreads / 32;
+constexpr int kIter = 4;                      // 4-element vectors per thread per chunk
+constexpr int kWarpSpan = 32 * kIter * 4;     // 512 consecutive elements per warp
+constexpr int kChunk = kWarps * kWarpSpan;    // 4096 elements per block of the collect kernels
+constexpr int kHistChunks = 16;               // chunks per block of the histogram kernels
+constexpr int kCandTile = 2048;               // candidates per block of the candidate kernels
+constexpr int kCandPer = kCandTile / kThreads;
+
+// radix digits of the 31-bit magnitude key, most significant first: 11 + 11 + 9 bits
+constexpr int kBins = 2048;
+__host__ __device__ constexpr int digit_bits(int pass) { return pass < 2 ? 11 : 9; }
+__host__ __device__ constexpr int digit_shift(int pass) { return pass == 0 ? 20 : (pass == 1 ? 9 : 0); }
+__host__ __device__ constexpr int resolved_before(int pass) { return pass == 0 ? 0 : (pass == 1 ? 11 : 22); }
+
+constexpr uint32_t kNoQuota = 0xFFFFFFFFu;
+constexpr int kSampleMax = 32768;             // sampled elements per slice (threshold estimate)
+constexpr int kSampleThreads = 1024;
+
+// stage of the full-vector radix select of one slice
+enum : uint32_t { STAGE_PASS0 = 0, STAGE_PASS1 = 1, STAGE_PASS2 = 2, STAGE_COLLECT = 3, STAGE_DONE = 4 };
+enum : uint32_t { FLAG_GENERAL = 1u, FLAG_FELL_BACK = 2u };
+enum : uint32_t { ERR_LOOKBACK_TIMEOUT = 1u, ERR_CANDIDATE_OVERFLOW = 2u, ERR_SELECT_INCONSISTENT = 4u };
+
+// One slice: a worker row, or one tensor of a worker row.  Offsets are in elements.
+struct Slice {
+  int64_t g_off;        // slice start relative to the gradient base pointer
+  int64_t m_off;        // slice start relative to the residual base pointer
+  uint32_t len;         // number of coordinates d_s
+  uint32_t r, k;
+  uint32_t row;         // local row (worker_base + row is the global worker id)
+  uint32_t segment;
+  uint32_t idx_base;    // index of the slice's first coordinate in the whole vector
+  uint32_t head;        // (slice start) mod 4: elements of the first aligned vector before the slice
+  uint32_t msg_off;     // start of the slice's k pairs in the flattened message arrays
+  uint32_t cand_off, cand_cap;
+  uint32_t chunk_begin; // first collect tile (all slices are numbered one after another)
+  uint32_t hist_begin;  // first histogram block
+  uint32_t ctile_begin; // first candidate tile
+  uint32_t samp_off;    // start in the draw buffer (k entries)
+  uint32_t first_off;   // start in the first-occurrence table (r entries)
+  uint32_t sel_off;     // start in the selection bitmap / its prefix counts (32-bit words)
+  uint32_t pad;
+};
+
+// Selection state of one slice, advanced kernel by kernel.
+struct SelState {
+  uint32_t tau_lo;      // collect threshold: keys above it are candidates ...
+  uint32_t eq_quota;    // ... and the first eq_quota keys equal to it (kNoQuota = all)
+  uint32_t prefix;      // resolved high bits of the r-th largest key
+  uint32_t resolved;    // how many of the 31 bits are resolved
+  uint32_t n_gt;        // keys strictly above the resolved prefix bucket
+  uint32_t need;        // rank of the r-th largest inside the bucket (1-based)
+  uint32_t n_cand;      // candidates written
+  uint32_t stage;
+  uint32_t flags;
+  uint32_t n_cand_first;// candidates of the sampled-threshold pass (statistics)
+  uint32_t pad[2];
+};
+
+struct Scratch {
+  Slice* slices;
+  SelState* state;
+  uint32_t* hist;         // [slices][kBins]
+  uint32_t* done;         // [slices] block-completion counters
+  uint32_t* tickets;      // [4] dynamic tile counters
+  unsigned long long* look_a;   // look-back words of the first collect
+  unsigned long long* look_b;   // ... of the fallback collect
+  unsigned long long* look_e;   // ... of the emit pass
+  uint32_t* cand_idx;
+  float* cand_val;
+  uint32_t* draws;        // t_j
+  uint32_t* first;        // first-occurrence table F
+  uint32_t* sel;          // selection bitmap over positions
+  uint32_t* sel_pre;      // exclusive popcount prefix per bitmap word
+  uint32_t* error;        // device error flags
+};
+
+struct Launch {
+  Scratch s;
+  const void* grad;
+  float* residual;
+  uint32_t* msg_idx;
+  float* msg_val;
+  uint32_t n_slices;
+  uint32_t worker_base;
+  uint32_t seed_lo, seed_hi;
+  uint32_t step;
+};
+
+// ----------------------------------------------------------------------------- small helpers
+__device__ __forceinline__ uint32_t lane_id() { return threadIdx.x & 31; }
+__device__ __forceinline__ uint32_t mag_key(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
+
+__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v) {
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    uint32_t n = __shfl_up_sync(0xFFFFFFFFu, v, o);
+    if (lane_id() >= (uint32_t)o) v += n;
+  }
+  return v;
+}
+
+__device__ __forceinline__ uint32_t warp_sum(uint32_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+
+// index of the slice that owns global tile `t`: the last s with begin(s) <= t
+template <typename F>
+__device__ __forceinline__ uint32_t find_slice(uint32_t n, uint32_t t, F begin) {
+  uint32_t lo = 0, hi = n;
+  while (hi - lo > 1) {
+    uint32_t mid = (lo + hi) >> 1;
+    if (begin(mid) <= t) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// ----------------------------------------------------------------------------- look-back
+// Decoupled look-back over tiles of one slice, carrying two 31-bit counters.  Word layout:
+// bits 63..62 = 0 empty / 1 tile aggregate / 2 inclusive prefix; bits 61..31 = A; bits 30..0 = B.
+// Tiles are handed out by a ticket counter, so every predecessor of a waiting tile is already
+// running and publishes its aggregate before it waits itself.  Waits are bounded: on expiry the
+// error flag is raised and a zero prefix is returned (all later writes stay bounds-checked).
+constexpr unsigned long long kLookAgg = 1ull << 62, kLookIncl = 2ull << 62;
+constexpr uint32_t kLookMask31 = 0x7FFFFFFFu;
+constexpr int kLookSpinLimit = 1 << 22;
+
+__device__ __forceinline__ unsigned long long look_pack(unsigned long long flag, uint32_t a, uint32_t b) {
+  return flag | ((unsigned long long)(a & kLookMask31) << 31) | (unsigned long long)(b & kLookMask31);
+}
+__device__ __forceinline__ unsigned long long ld_relaxed(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_relaxed(unsigned long long* p, unsigned long long v) {
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+// Called by all 32 lanes of one warp.  `words` points at the slice's tile 0, `tile` is the tile
+// inside the slice, (aggA, aggB) the tile's own counts.  Returns the exclusive prefix in
+// (exA, exB) on every lane.
+__device__ __forceinline__ void lookback_exclusive(unsigned long long* words, uint32_t tile, uint32_t aggA,
+                                                   uint32_t aggB, uint32_t& exA, uint32_t& exB,
+                                                   uint32_t* error) {
+  const uint32_t lane = lane_id();
+  if (tile == 0) {
+    if (lane == 0) st_relaxed(words, look_pack(kLookIncl, aggA, aggB));
+    exA = 0; exB = 0;
+    return;
+  }
+  if (lane == 0) st_relaxed(words + tile, look_pack(kLookAgg, aggA, aggB));
+  uint32_t sumA = 0, sumB = 0;
+  int64_t top = (int64_t)tile - 1;          // newest tile not yet accounted for
+  bool failed = false;
+  while (true) {
+    const int64_t mine = top - lane;
+    unsigned long long w = kLookIncl;       // lanes before tile 0 read as "inclusive, zero"
+    if (mine >= 0) {
+      int spins = 0;
+      w = ld_relaxed(words + mine);
+      while ((w >> 62) == 0) {
+        if (++spins > kLookSpinLimit) { failed = true; break; }
+        __nanosleep(40);
+        w = ld_relaxed(words + mine);
+      }
+    }
+    if (__any_sync(0xFFFFFFFFu, failed)) { failed = true; break; }
+    const uint32_t incl_mask = __ballot_sync(0xFFFFFFFFu, (w >> 62) == 2);
+    const uint32_t stop = incl_mask ? (uint32_t)(__ffs(incl_mask) - 1) : 32u;   // first inclusive lane
+    const bool use = lane <= stop;
+    sumA += warp_sum(use ? (uint32_t)((w >> 31) & kLookMask31) : 0u);
+    sumB += warp_sum(use ? (uint32_t)(w & kLookMask31) : 0u);
+    if (incl_mask) break;
+    top -= 32;
+  }
+  if (failed) {
+    if (lane == 0) atomicOr(error, ERR_LOOKBACK_TIMEOUT);
+    sumA = 0; sumB = 0;
+  }
+  if (lane == 0) st_relaxed(words + tile, look_pack(kLookIncl, sumA + aggA, sumB + aggB));
+  exA = sumA; exB = sumB;
+}
+
+// ----------------------------------------------------------------------------- digit pick
+// Given a complete histogram of one digit (bins [0, nbins)) in shared memory and the rank `need`
+// (1-based, counted from the largest digit), finds the digit D with
+//   count(digit > D) < need <= count(digit >= D)
+// and returns D and count(digit > D).  Called by every thread of the block; `scratch` holds
+// blockDim.x / 32 + 2 words.  Returns false if the histogram holds fewer than `need` keys.
+__device__ __forceinline__ bool pick_digit(const uint32_t* hist, int nbins, uint32_t need, uint32_t* scratch,
+                                           uint32_t& D, uint32_t& above) {
+  const int nthreads = blockDim.x;
+  const int per = (nbins + nthreads - 1) / nthreads;
+  // thread t owns bins [hi - per + 1, hi] counted from the top: t = 0 holds the largest digits
+  const int hi = nbins - 1 - (int)threadIdx.x * per;
+  uint32_t mine = 0;
+  for (int i = 0; i < per; ++i) {
+    const int b = hi - i;
+    if (b >= 0) mine += hist[b];
+  }
+  // inclusive scan over threads (from the top digits downwards)
+  uint32_t incl = warp_incl_scan(mine);
+  const uint32_t warp = threadIdx.x >> 5, nwarps = (nthreads + 31) >> 5;
+  if (lane_id() == 31) scratch[warp] = incl;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t run = 0;
+    for (uint32_t w = 0; w < nwarps; ++w) { uint32_t v = scratch[w]; scratch[w] = run; run += v; }
+    scratch[nwarps] = 0xFFFFFFFFu;      // result: digit
+    scratch[nwarps + 1] = 0;            // result: above
+  }
+  __syncthreads();
+  incl += scratch[warp];
+  const uint32_t excl = incl - mine;
+  if (excl < need && need <= incl) {     // the crossing lies in this thread's bins
+    uint32_t run = excl;
+    for (int i = 0; i < per; ++i) {
+      const int b = hi - i;
+      if (b < 0) break;
+      const uint32_t h = hist[b];
+      if (run + h >= need) { scratch[nwarps] = (uint32_t)b; scratch[nwarps + 1] = run; break; }
+      run += h;
+    }
+  }
+  __syncthreads();
+  D = scratch[nwarps];
+  above = scratch[nwarps + 1];
+  __syncthreads();
+  return D != 0xFFFFFFFFu;
+}
+
+// ----------------------------------------------------------------------------- Philox4x32-10
+// Salmon, Moraes, Dror, Shaw, "Parallel Random Numbers: As Easy as 1, 2, 3" (SC'11): ten rounds;
+// each multiplies counter words 0 and 2 by the two round multipliers, XORs the high halves with
+// words 1 and 3 and the round key, and bumps the key by the Weyl constants.
+__device__ __forceinline__ uint2 philox4x32_10_lo(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                  uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int i = 0; i < 10; ++i) {
+    const uint32_t h0 = __umulhi(0xD2511F53u, c0), l0 = 0xD2511F53u * c0;
+    const uint32_t h1 = __umulhi(0xCD9E8D57u, c2), l1 = 0xCD9E8D57u * c2;
+    c0 = h1 ^ c1 ^ k0; c1 = l1;
+    c2 = h0 ^ c3 ^ k1; c3 = l0;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  return make_uint2(c0, c1);   // output words 0 and 1
+}
+
+// Floyd iteration j draws uniformly from {0..j}: floor(u64 * (j+1) / 2^64), u64 = (x1 << 32) | x0.
+__device__ __forceinline__ uint32_t floyd_draw(uint32_t j, uint32_t worker, uint32_t segment, uint32_t step,
+                                               uint32_t seed_lo, uint32_t seed_hi) {
+  const uint2 x = philox4x32_10_lo(j, worker, segment, step, seed_lo, seed_hi);
+  const unsigned long long u = ((unsigned long long)x.y << 32) | x.x;
+  return (uint32_t)__umul64hi(u, (unsigned long long)j + 1ull);
+}
+
+}  // namespace rtopk

@@ -1,0 +1,590 @@
+// Host side of the rTop-k library: argument checks, scratch layout, and the launch sequence of
+// one round of Algorithm 1's communication path (node body for W workers, then the master's
+// average).  All device work is enqueued on the caller's stream; nothing here synchronises
+// except the explicitly documented status / statistics reads.
+#include "../../include/rtopk.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "aggregate.cuh"
+#include "common.cuh"
+#include "sampler.cuh"
+#include "select.cuh"
+
+using namespace rtopk;
+
+struct rtopk_ctx {
+  int device = 0;
+  int64_t d_max = 0, r_max = 0, k_max = 0;
+  int32_t W_max = 0, S_max = 0;
+  int select_path = 0;
+  int last_cuda_error = 0;
+  // device scratch (one allocation each)
+  Slice* d_slices = nullptr;
+  SelState* d_state = nullptr;
+  char* d_zero = nullptr;        // counters, histograms, look-back words, bitmaps: cleared per call
+  size_t zero_bytes = 0;
+  uint32_t* d_first = nullptr;   // first-occurrence tables: set to 0xFF per call
+  size_t first_entries = 0;
+  uint32_t* d_cand_idx = nullptr;
+  float* d_cand_val = nullptr;
+  size_t cand_entries = 0;
+  uint32_t* d_draws = nullptr;
+  uint32_t* d_sel_pre = nullptr;
+  size_t sel_words = 0;
+  uint32_t* d_error = nullptr;
+  uint32_t* d_agg_starts = nullptr;
+  size_t agg_start_entries = 0;
+  void* d_stage = nullptr;       // host-call staging: gradient, messages, update
+  size_t stage_bytes = 0;
+  std::vector<Slice> cached_slices;   // what d_slices currently holds
+  uint32_t last_n_slices = 0;
+  // optional per-phase timing (RTOPK_OPT_PROFILE): events recorded on the caller's stream
+  int profile = 0;
+  cudaEvent_t ev[RTOPK_N_PHASES + 1] = {};
+  bool ev_valid[RTOPK_N_PHASES + 1] = {};
+};
+
+namespace {
+
+constexpr int kVersion = 100;
+constexpr size_t kSampleSmemBytes = (size_t)(kSampleMax + kBins + 64) * sizeof(uint32_t);
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int cuda_fail(rtopk_ctx* ctx, cudaError_t e) {
+  if (ctx) ctx->last_cuda_error = (int)e;
+  return RTOPK_ERR_CUDA;
+}
+#define RTOPK_CUDA(ctx, call)                                   \
+  do {                                                          \
+    cudaError_t e__ = (call);                                   \
+    if (e__ != cudaSuccess) return cuda_fail((ctx), e__);       \
+  } while (0)
+
+// Marks the boundary before phase `i` (i = RTOPK_N_PHASES: the end of the last phase).
+void mark(rtopk_ctx* ctx, int i, cudaStream_t st) {
+  if (!ctx->profile) return;
+  ctx->ev_valid[i] = cudaEventRecord(ctx->ev[i], st) == cudaSuccess;
+}
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+uint32_t cand_capacity(uint64_t len, uint64_t r) {
+  const uint64_t c = 2 * r + 1024;
+  return (uint32_t)(c < len ? c : len);
+}
+
+// Layout of one call: the slice table plus every per-call scratch offset.
+struct Plan {
+  std::vector<Slice> slices;
+  uint32_t n_chunks = 0, n_hist_blocks = 0, n_ctiles = 0;
+  size_t cand_entries = 0, draw_entries = 0, first_entries = 0, sel_words = 0;
+  uint32_t k_draw_max = 0, words_all_max = 0;
+  bool any_select = false, any_sampler = false, any_all = false;
+  uint32_t K_row = 0;
+};
+
+int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32_t W, int32_t S,
+              const int64_t* seg_off, const int64_t* seg_r, const int64_t* seg_k, Plan& P) {
+  uint64_t K = 0, R = 0;
+  for (int s = 0; s < S; ++s) {
+    const int64_t len = seg_off[s + 1] - seg_off[s];
+    if (len < 1 || seg_k[s] < 1 || seg_k[s] > seg_r[s] || seg_r[s] > len) return RTOPK_ERR_INVALID_ARG;
+    K += (uint64_t)seg_k[s];
+    R += (uint64_t)seg_r[s];
+  }
+  if (seg_off[0] != 0 || seg_off[S] != d) return RTOPK_ERR_INVALID_ARG;
+  if ((int64_t)K > ctx->k_max || (int64_t)R > ctx->r_max) return RTOPK_ERR_INVALID_ARG;
+  if (K * (uint64_t)W >= (1ull << 32)) return RTOPK_ERR_INVALID_ARG;
+  P.K_row = (uint32_t)K;
+  P.slices.resize((size_t)W * (size_t)S);
+  uint64_t chunks = 0, hblocks = 0, ctiles = 0, cand = 0, draws = 0, first = 0, selw = 0;
+  for (int w = 0; w < W; ++w) {
+    uint64_t msg_at = (uint64_t)w * K;
+    for (int s = 0; s < S; ++s) {
+      Slice& sl = P.slices[(size_t)w * S + s];
+      std::memset(&sl, 0, sizeof(sl));
+      const int64_t lo = seg_off[s], len = seg_off[s + 1] - lo;
+      sl.g_off = (int64_t)w * ld_g + lo;
+      sl.m_off = (int64_t)w * ld_m + lo;
+      sl.len = (uint32_t)len;
+      sl.r = (uint32_t)seg_r[s];
+      sl.k = (uint32_t)seg_k[s];
+      sl.row = (uint32_t)w;
+      sl.segment = (uint32_t)s;
+      sl.idx_base = (uint32_t)lo;
+      sl.head = (uint32_t)(lo & 3);
+      sl.msg_off = (uint32_t)msg_at;
+      msg_at += sl.k;
+      const uint32_t nchunks = (uint32_t)((sl.head + (uint64_t)sl.len + kChunk - 1) / kChunk);
+      sl.chunk_begin = (uint32_t)chunks;
+      sl.hist_begin = (uint32_t)hblocks;
+      chunks += nchunks;
+      hblocks += (nchunks + kHistChunks - 1) / kHistChunks;
+      sl.ctile_begin = (uint32_t)ctiles;
+      sl.cand_off = (uint32_t)cand;
+      if (sl.r < sl.len) {
+        sl.cand_cap = cand_capacity(sl.len, sl.r);
+        cand += sl.cand_cap;
+        ctiles += (sl.cand_cap + kCandTile - 1) / kCandTile;
+        P.any_select = true;
+      } else {
+        sl.cand_cap = 0;
+        P.any_all = true;
+        const uint32_t nw = (sl.r + 31) / 32;
+        if (nw > P.words_all_max) P.words_all_max = nw;
+      }
+      sl.samp_off = (uint32_t)draws;
+      sl.first_off = (uint32_t)first;
+      sl.sel_off = (uint32_t)selw;
+      if (sl.k < sl.r) {
+        draws += sl.k;
+        first += sl.r;
+        selw += (sl.r + 31) / 32;
+        P.any_sampler = true;
+        if (sl.k > P.k_draw_max) P.k_draw_max = sl.k;
+      }
+    }
+  }
+  if (chunks >= (1ull << 31) || cand >= (1ull << 32) || first >= (1ull << 32)) return RTOPK_ERR_INVALID_ARG;
+  P.n_chunks = (uint32_t)chunks; P.n_hist_blocks = (uint32_t)hblocks; P.n_ctiles = (uint32_t)ctiles;
+  P.cand_entries = cand; P.draw_entries = draws; P.first_entries = first; P.sel_words = selw;
+  return RTOPK_OK;
+}
+
+// Carves the per-call zeroed region.  Returns the bytes used.
+size_t carve_zero(const rtopk_ctx* ctx, const Plan& P, Scratch& s) {
+  char* p = ctx->d_zero;
+  size_t at = 0;
+  auto take = [&](size_t bytes) { char* q = p + at; at = align_up(at + bytes, 256); return q; };
+  s.tickets = (uint32_t*)take(4 * sizeof(uint32_t));
+  s.done = (uint32_t*)take(P.slices.size() * sizeof(uint32_t));
+  s.hist = (uint32_t*)take(P.slices.size() * kBins * sizeof(uint32_t));
+  s.look_a = (unsigned long long*)take((size_t)P.n_chunks * 8);
+  s.look_b = (unsigned long long*)take((size_t)P.n_chunks * 8);
+  s.look_e = (unsigned long long*)take((size_t)P.n_ctiles * 8);
+  s.sel = (uint32_t*)take(P.sel_words * sizeof(uint32_t));
+  return at;
+}
+
+size_t zero_region_bytes(size_t slices, size_t chunks, size_t ctiles, size_t sel_words) {
+  size_t at = 0;
+  auto take = [&](size_t bytes) { at = align_up(at + bytes, 256); };
+  take(16); take(slices * 4); take(slices * kBins * 4); take(chunks * 8); take(chunks * 8); take(ctiles * 8);
+  take(sel_words * 4);
+  return at;
+}
+
+int check_common(const rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, const float* residual,
+                 int64_t ld_m, int64_t d, int32_t W, int32_t worker_base, const uint32_t* msg_idx,
+                 const float* msg_val) {
+  if (!ctx || !grad || !residual || !msg_idx || !msg_val) return RTOPK_ERR_INVALID_ARG;
+  if (grad_dtype != RTOPK_F32 && grad_dtype != RTOPK_BF16) return RTOPK_ERR_INVALID_ARG;
+  if (d < 1 || d > ctx->d_max || W < 1 || W > ctx->W_max || worker_base < 0) return RTOPK_ERR_INVALID_ARG;
+  const int64_t g_mult = grad_dtype == RTOPK_F32 ? 4 : 8;
+  if (ld_g < d || ld_m < d || (ld_g % g_mult) != 0 || (ld_m % 4) != 0) return RTOPK_ERR_INVALID_ARG;
+  if (((uintptr_t)grad & 15u) || ((uintptr_t)residual & 15u) || ((uintptr_t)msg_idx & 3u) ||
+      ((uintptr_t)msg_val & 3u))
+    return RTOPK_ERR_INVALID_ARG;
+  return RTOPK_OK;
+}
+
+template <typename GradT>
+int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st) {
+  const uint32_t n = (uint32_t)P.slices.size();
+  if (ctx->select_path == 0) {
+    mark(ctx, RTOPK_PHASE_THRESHOLD, st);
+    k_sample<GradT><<<n, kSampleThreads, kSampleSmemBytes, st>>>(L);
+    mark(ctx, RTOPK_PHASE_STREAM, st);
+    k_collect<GradT, true, false><<<P.n_chunks, kThreads, 0, st>>>(L);
+    mark(ctx, RTOPK_PHASE_EXACT, st);
+    if (P.any_select) {
+      for (int pass = 0; pass < 3; ++pass) k_hist<float, false><<<P.n_hist_blocks, kThreads, 0, st>>>(L, pass);
+      k_collect<float, false, true><<<P.n_chunks, kThreads, 0, st>>>(L);
+    }
+  } else {
+    mark(ctx, RTOPK_PHASE_THRESHOLD, st);
+    k_init_state<<<(n + 127) / 128, 128, 0, st>>>(L, 1u);
+    mark(ctx, RTOPK_PHASE_STREAM, st);
+    k_hist<GradT, true><<<P.n_hist_blocks, kThreads, 0, st>>>(L, 0);
+    mark(ctx, RTOPK_PHASE_EXACT, st);
+    if (P.any_select) {
+      for (int pass = 1; pass < 3; ++pass) k_hist<float, false><<<P.n_hist_blocks, kThreads, 0, st>>>(L, pass);
+      k_collect<float, false, true><<<P.n_chunks, kThreads, 0, st>>>(L);
+    }
+  }
+  return RTOPK_OK;
+}
+
+int upload_slices(rtopk_ctx* ctx, const Plan& P, cudaStream_t st) {
+  const size_t bytes = P.slices.size() * sizeof(Slice);
+  if (ctx->cached_slices.size() == P.slices.size() &&
+      std::memcmp(ctx->cached_slices.data(), P.slices.data(), bytes) == 0)
+    return RTOPK_OK;
+  RTOPK_CUDA(ctx, cudaMemcpyAsync(ctx->d_slices, P.slices.data(), bytes, cudaMemcpyHostToDevice, st));
+  ctx->cached_slices = P.slices;
+  return RTOPK_OK;
+}
+
+int run_sampler(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st) {
+  if (!P.any_sampler) return RTOPK_OK;
+  const uint32_t n = (uint32_t)P.slices.size();
+  RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_first, 0xFF, P.first_entries * sizeof(uint32_t), st));
+  const dim3 grid((P.k_draw_max + kDrawThreads - 1) / kDrawThreads, n);
+  k_draw<<<grid, kDrawThreads, 0, st>>>(L);
+  k_resolve<<<grid, kDrawThreads, 0, st>>>(L);
+  k_sel_scan<<<n, kScanThreads, 0, st>>>(L);
+  return RTOPK_OK;
+}
+
+int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
+                  int64_t d, int32_t W, int32_t worker_base, int32_t S, const int64_t* seg_off,
+                  const int64_t* seg_r, const int64_t* seg_k, uint64_t seed, uint32_t step, uint32_t* msg_idx,
+                  float* msg_val, cudaStream_t st, uint32_t* K_out) {
+  int rc = check_common(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, msg_idx, msg_val);
+  if (rc) return rc;
+  if (S < 1 || S > ctx->S_max || !seg_off || !seg_r || !seg_k) return RTOPK_ERR_INVALID_ARG;
+  Plan P;
+  rc = make_plan(ctx, ld_g, ld_m, d, W, S, seg_off, seg_r, seg_k, P);
+  if (rc) return rc;
+  if (P.cand_entries > ctx->cand_entries || P.first_entries > ctx->first_entries ||
+      P.sel_words > ctx->sel_words)
+    return RTOPK_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return RTOPK_ERR_CUDA;
+  Launch L;
+  std::memset(&L, 0, sizeof(L));
+  const size_t zbytes = carve_zero(ctx, P, L.s);
+  if (zbytes > ctx->zero_bytes) return RTOPK_ERR_INVALID_ARG;
+  L.s.slices = ctx->d_slices; L.s.state = ctx->d_state;
+  L.s.cand_idx = ctx->d_cand_idx; L.s.cand_val = ctx->d_cand_val;
+  L.s.draws = ctx->d_draws; L.s.first = ctx->d_first; L.s.sel_pre = ctx->d_sel_pre;
+  L.s.error = ctx->d_error;
+  L.grad = grad; L.residual = residual; L.msg_idx = msg_idx; L.msg_val = msg_val;
+  L.n_slices = (uint32_t)P.slices.size();
+  L.worker_base = (uint32_t)worker_base;
+  L.seed_lo = (uint32_t)seed; L.seed_hi = (uint32_t)(seed >> 32);
+  L.step = step;
+
+  rc = upload_slices(ctx, P, st);
+  if (rc) return rc;
+  ctx->last_n_slices = L.n_slices;
+  mark(ctx, RTOPK_PHASE_SUBSET, st);
+  RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero, 0, zbytes, st));
+  rc = run_sampler(ctx, P, L, st);
+  if (rc) return rc;
+  rc = grad_dtype == RTOPK_F32 ? launch_select<float>(ctx, P, L, st) : launch_select<__nv_bfloat16>(ctx, P, L, st);
+  if (rc) return rc;
+  mark(ctx, RTOPK_PHASE_SELECT, st);
+  if (P.any_select) {
+    for (int pass = 0; pass < 3; ++pass) k_cand_hist<<<P.n_ctiles, kThreads, 0, st>>>(L, pass);
+    mark(ctx, RTOPK_PHASE_EMIT, st);
+    k_emit<<<P.n_ctiles, kThreads, 0, st>>>(L);
+  } else {
+    mark(ctx, RTOPK_PHASE_EMIT, st);
+  }
+  if (P.any_all) {
+    const dim3 grid((P.words_all_max + kThreads - 1) / kThreads, L.n_slices);
+    k_emit_all<<<grid, kThreads, 0, st>>>(L, P.words_all_max);
+  }
+  mark(ctx, RTOPK_PHASE_AGGREGATE, st);
+  ctx->ev_valid[RTOPK_N_PHASES] = false;   // closed by the aggregate of a step call, if any
+  RTOPK_CUDA(ctx, cudaGetLastError());
+  if (K_out) *K_out = P.K_row;
+  return RTOPK_OK;
+}
+
+int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
+                   int scale_mode, float* out, cudaStream_t st) {
+  if (!ctx || !msg_idx || !msg_val || !out) return RTOPK_ERR_INVALID_ARG;
+  if (d < 1 || d > ctx->d_max || W < 1 || W > ctx->W_max || k < 1 || k > d) return RTOPK_ERR_INVALID_ARG;
+  if (scale_mode != RTOPK_SCALE_MEAN && scale_mode != RTOPK_SCALE_SUM) return RTOPK_ERR_INVALID_ARG;
+  if (((uintptr_t)out & 15u) || ((uintptr_t)msg_idx & 3u) || ((uintptr_t)msg_val & 3u)) return RTOPK_ERR_INVALID_ARG;
+  if ((uint64_t)k * (uint64_t)W >= (1ull << 32)) return RTOPK_ERR_INVALID_ARG;
+  const uint32_t ntiles = (uint32_t)((d + kAggTile - 1) / kAggTile);
+  if ((size_t)W * (ntiles + 1) > ctx->agg_start_entries) return RTOPK_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return RTOPK_ERR_CUDA;
+  const dim3 sgrid((ntiles + 1 + kAggThreads - 1) / kAggThreads, (uint32_t)W);
+  k_agg_starts<<<sgrid, kAggThreads, 0, st>>>(msg_idx, (uint32_t)W, (uint32_t)k, ntiles, ctx->d_agg_starts);
+  k_aggregate<<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, ctx->d_agg_starts, (uint32_t)d, (uint32_t)W,
+                                              (uint32_t)k, scale_mode == RTOPK_SCALE_MEAN ? 1 : 0, out);
+  mark(ctx, RTOPK_N_PHASES, st);
+  RTOPK_CUDA(ctx, cudaGetLastError());
+  return RTOPK_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int rtopk_version(void) { return kVersion; }
+
+const char* rtopk_status_string(int status) {
+  switch (status) {
+    case RTOPK_OK: return "ok";
+    case RTOPK_ERR_INVALID_ARG: return "invalid argument";
+    case RTOPK_ERR_ALLOC: return "allocation failed";
+    case RTOPK_ERR_CUDA: return "CUDA runtime error";
+    case RTOPK_ERR_UNSUPPORTED: return "unsupported";
+    case RTOPK_ERR_INTERNAL: return "internal error (device-side wait expired or invariant broken)";
+    default: return "unknown status";
+  }
+}
+
+int rtopk_last_cuda_error(const rtopk_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int64_t r_max, int64_t k_max,
+                 int32_t segments_max) {
+  if (!out) return RTOPK_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (d_max < 1 || d_max >= (1ll << 31) || W_max < 1 || W_max > 65535 || r_max < 1 || r_max > d_max ||
+      k_max < 1 || k_max > r_max || segments_max < 1 || segments_max > 65535)
+    return RTOPK_ERR_INVALID_ARG;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) return RTOPK_ERR_CUDA;
+  rtopk_ctx* ctx = new (std::nothrow) rtopk_ctx();
+  if (!ctx) return RTOPK_ERR_ALLOC;
+  ctx->device = device; ctx->d_max = d_max; ctx->W_max = W_max; ctx->r_max = r_max; ctx->k_max = k_max;
+  ctx->S_max = segments_max;
+  DeviceGuard guard(device);
+  if (!guard.ok) { delete ctx; return RTOPK_ERR_CUDA; }
+  const size_t W = (size_t)W_max, S = (size_t)segments_max, slices = W * S;
+  const size_t chunks = W * ((size_t)d_max / kChunk + 2 * S + 1);
+  const size_t cand_row = std::min<size_t>((size_t)d_max, 2 * (size_t)r_max + 1024 * S);
+  const size_t ctiles = W * (cand_row / kCandTile + 1 + S);
+  ctx->cand_entries = W * cand_row;
+  ctx->first_entries = W * (size_t)r_max;
+  ctx->sel_words = W * ((size_t)r_max / 32 + S + 1);
+  ctx->zero_bytes = zero_region_bytes(slices, chunks, ctiles, ctx->sel_words);
+  ctx->agg_start_entries = W * ((size_t)(d_max + kAggTile - 1) / kAggTile + 2);
+  if (ctx->cand_entries >= (1ull << 32) || ctx->first_entries >= (1ull << 32)) { delete ctx; return RTOPK_ERR_INVALID_ARG; }
+  cudaError_t e = cudaSuccess;
+  auto alloc = [&](void** p, size_t bytes) { if (e == cudaSuccess) e = cudaMalloc(p, bytes ? bytes : 16); };
+  alloc((void**)&ctx->d_slices, slices * sizeof(Slice));
+  alloc((void**)&ctx->d_state, slices * sizeof(SelState));
+  alloc((void**)&ctx->d_zero, ctx->zero_bytes);
+  alloc((void**)&ctx->d_first, ctx->first_entries * sizeof(uint32_t));
+  alloc((void**)&ctx->d_cand_idx, ctx->cand_entries * sizeof(uint32_t));
+  alloc((void**)&ctx->d_cand_val, ctx->cand_entries * sizeof(float));
+  alloc((void**)&ctx->d_draws, W * (size_t)k_max * sizeof(uint32_t));
+  alloc((void**)&ctx->d_sel_pre, ctx->sel_words * sizeof(uint32_t));
+  alloc((void**)&ctx->d_error, 16);
+  alloc((void**)&ctx->d_agg_starts, ctx->agg_start_entries * sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_sample<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSampleSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_sample<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSampleSmemBytes);
+  for (int i = 0; i <= RTOPK_N_PHASES && e == cudaSuccess; ++i) e = cudaEventCreate(&ctx->ev[i]);
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_error, 0, 16);
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_state, 0, slices * sizeof(SelState));
+  if (e != cudaSuccess) {
+    const int rc = e == cudaErrorMemoryAllocation ? RTOPK_ERR_ALLOC : RTOPK_ERR_CUDA;
+    cudaGetLastError();
+    rtopk_destroy(ctx);
+    return rc;
+  }
+  *out = ctx;
+  return RTOPK_OK;
+}
+
+int rtopk_destroy(rtopk_ctx* ctx) {
+  if (!ctx) return RTOPK_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  void* ptrs[] = {ctx->d_slices, ctx->d_state, ctx->d_zero, ctx->d_first, ctx->d_cand_idx, ctx->d_cand_val,
+                  ctx->d_draws, ctx->d_sel_pre, ctx->d_error, ctx->d_agg_starts, ctx->d_stage};
+  for (void* p : ptrs) if (p) cudaFree(p);
+  for (cudaEvent_t ev : ctx->ev) if (ev) cudaEventDestroy(ev);
+  delete ctx;
+  return RTOPK_OK;
+}
+
+int rtopk_set_option(rtopk_ctx* ctx, int option, int64_t value) {
+  if (!ctx) return RTOPK_ERR_INVALID_ARG;
+  if (option == RTOPK_OPT_SELECT_PATH && (value == 0 || value == 1)) { ctx->select_path = (int)value; return RTOPK_OK; }
+  if (option == RTOPK_OPT_PROFILE && (value == 0 || value == 1)) {
+    ctx->profile = (int)value;
+    for (bool& v : ctx->ev_valid) v = false;
+    return RTOPK_OK;
+  }
+  return RTOPK_ERR_INVALID_ARG;
+}
+
+int rtopk_sparsify(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
+                   int64_t d, int32_t W, int32_t worker_base, int64_t r, int64_t k, uint64_t seed, uint32_t step,
+                   uint32_t* msg_idx, float* msg_val, void* stream) {
+  const int64_t off[2] = {0, d};
+  return sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed, step,
+                       msg_idx, msg_val, (cudaStream_t)stream, nullptr);
+}
+
+int rtopk_sparsify_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,
+                             int64_t ld_m, int64_t d, int32_t W, int32_t worker_base, int32_t S,
+                             const int64_t* seg_off, const int64_t* seg_r, const int64_t* seg_k, uint64_t seed,
+                             uint32_t step, uint32_t* msg_idx, float* msg_val, void* stream) {
+  return sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, S, seg_off, seg_r, seg_k,
+                       seed, step, msg_idx, msg_val, (cudaStream_t)stream, nullptr);
+}
+
+int rtopk_aggregate(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
+                    int scale_mode, float* out, void* stream) {
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, out, (cudaStream_t)stream);
+}
+
+int rtopk_step(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
+               int64_t d, int32_t W, int32_t worker_base, int64_t r, int64_t k, uint64_t seed, uint32_t step,
+               int scale_mode, uint32_t* msg_idx, float* msg_val, float* out, void* stream) {
+  if (!out || ((uintptr_t)out & 15u) || (scale_mode != RTOPK_SCALE_MEAN && scale_mode != RTOPK_SCALE_SUM))
+    return RTOPK_ERR_INVALID_ARG;
+  const int rc = rtopk_sparsify(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, r, k, seed, step,
+                                msg_idx, msg_val, stream);
+  if (rc) return rc;
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, out, (cudaStream_t)stream);
+}
+
+int rtopk_step_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,
+                         int64_t ld_m, int64_t d, int32_t W, int32_t worker_base, int32_t S, const int64_t* seg_off,
+                         const int64_t* seg_r, const int64_t* seg_k, uint64_t seed, uint32_t step, int scale_mode,
+                         uint32_t* msg_idx, float* msg_val, float* out, void* stream) {
+  if (!out || ((uintptr_t)out & 15u) || (scale_mode != RTOPK_SCALE_MEAN && scale_mode != RTOPK_SCALE_SUM))
+    return RTOPK_ERR_INVALID_ARG;
+  uint32_t K = 0;
+  const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, S, seg_off, seg_r,
+                               seg_k, seed, step, msg_idx, msg_val, (cudaStream_t)stream, &K);
+  if (rc) return rc;
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, K, scale_mode, out, (cudaStream_t)stream);
+}
+
+int rtopk_step_host(rtopk_ctx* ctx, const void* h_grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
+                    int64_t d, int32_t W, int32_t worker_base, int64_t r, int64_t k, uint64_t seed, uint32_t step,
+                    int scale_mode, uint32_t* h_msg_idx, float* h_msg_val, float* h_out, void* stream) {
+  if (!ctx || !h_grad || !h_msg_idx || !h_msg_val || !h_out) return RTOPK_ERR_INVALID_ARG;
+  if (grad_dtype != RTOPK_F32 && grad_dtype != RTOPK_BF16) return RTOPK_ERR_INVALID_ARG;
+  if (d < 1 || d > ctx->d_max || W < 1 || W > ctx->W_max || k < 1 || k > r || r > d || ld_g < d)
+    return RTOPK_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return RTOPK_ERR_CUDA;
+  const size_t gsz = grad_dtype == RTOPK_F32 ? 4 : 2;
+  const size_t g_bytes = align_up((size_t)W * (size_t)ld_g * gsz, 256);
+  const size_t mi_bytes = align_up((size_t)W * (size_t)k * 4, 256);
+  const size_t out_bytes = align_up((size_t)d * 4, 256);
+  const size_t total = g_bytes + 2 * mi_bytes + out_bytes;
+  if (total > ctx->stage_bytes) {
+    // first use (or a larger shape): the one place a call allocates, and therefore waits
+    RTOPK_CUDA(ctx, cudaStreamSynchronize(st));
+    if (ctx->d_stage) { cudaFree(ctx->d_stage); ctx->d_stage = nullptr; ctx->stage_bytes = 0; }
+    const cudaError_t e = cudaMalloc(&ctx->d_stage, total);
+    if (e != cudaSuccess) { cudaGetLastError(); ctx->last_cuda_error = (int)e; return RTOPK_ERR_ALLOC; }
+    ctx->stage_bytes = total;
+  }
+  char* base = (char*)ctx->d_stage;
+  void* d_grad = base;
+  uint32_t* d_idx = (uint32_t*)(base + g_bytes);
+  float* d_val = (float*)(base + g_bytes + mi_bytes);
+  float* d_out = (float*)(base + g_bytes + 2 * mi_bytes);
+  RTOPK_CUDA(ctx, cudaMemcpyAsync(d_grad, h_grad, (size_t)W * (size_t)ld_g * gsz, cudaMemcpyHostToDevice, st));
+  const int rc = rtopk_step(ctx, d_grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, r, k, seed, step,
+                            scale_mode, d_idx, d_val, d_out, stream);
+  if (rc) return rc;
+  RTOPK_CUDA(ctx, cudaMemcpyAsync(h_msg_idx, d_idx, (size_t)W * (size_t)k * 4, cudaMemcpyDeviceToHost, st));
+  RTOPK_CUDA(ctx, cudaMemcpyAsync(h_msg_val, d_val, (size_t)W * (size_t)k * 4, cudaMemcpyDeviceToHost, st));
+  RTOPK_CUDA(ctx, cudaMemcpyAsync(h_out, d_out, (size_t)d * 4, cudaMemcpyDeviceToHost, st));
+  return RTOPK_OK;
+}
+
+int rtopk_sample_positions(rtopk_ctx* ctx, int64_t r, int64_t k, uint64_t seed, uint32_t step, uint32_t worker,
+                           uint32_t segment, uint32_t* pos, void* stream) {
+  if (!ctx || !pos || k < 1 || k > r || r > ctx->r_max || k > ctx->k_max) return RTOPK_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return RTOPK_ERR_CUDA;
+  Plan P;
+  P.slices.resize(1);
+  Slice& sl = P.slices[0];
+  std::memset(&sl, 0, sizeof(sl));
+  sl.len = (uint32_t)r; sl.r = (uint32_t)r; sl.k = (uint32_t)k; sl.row = 0; sl.segment = segment;
+  P.any_sampler = k < r;
+  P.k_draw_max = (uint32_t)k;
+  P.first_entries = (size_t)r;
+  P.sel_words = ((size_t)r + 31) / 32;
+  Launch L;
+  std::memset(&L, 0, sizeof(L));
+  const size_t zbytes = carve_zero(ctx, P, L.s);
+  if (zbytes > ctx->zero_bytes) return RTOPK_ERR_INVALID_ARG;
+  L.s.slices = ctx->d_slices; L.s.state = ctx->d_state; L.s.draws = ctx->d_draws; L.s.first = ctx->d_first;
+  L.s.sel_pre = ctx->d_sel_pre; L.s.error = ctx->d_error;
+  L.n_slices = 1; L.worker_base = worker; L.seed_lo = (uint32_t)seed; L.seed_hi = (uint32_t)(seed >> 32);
+  L.step = step;
+  int rc = upload_slices(ctx, P, st);
+  if (rc) return rc;
+  RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero, 0, zbytes, st));
+  rc = run_sampler(ctx, P, L, st);
+  if (rc) return rc;
+  const uint32_t nwords = (uint32_t)((r + 31) / 32);
+  k_positions<<<(nwords + kThreads - 1) / kThreads, kThreads, 0, st>>>(L, pos);
+  RTOPK_CUDA(ctx, cudaGetLastError());
+  return RTOPK_OK;
+}
+
+int rtopk_poll_status(rtopk_ctx* ctx, void* stream) {
+  if (!ctx) return RTOPK_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return RTOPK_ERR_CUDA;
+  uint32_t flags = 0;
+  RTOPK_CUDA(ctx, cudaMemcpyAsync(&flags, ctx->d_error, sizeof(flags), cudaMemcpyDeviceToHost, st));
+  RTOPK_CUDA(ctx, cudaStreamSynchronize(st));
+  if (flags) {
+    RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_error, 0, sizeof(flags), st));
+    return RTOPK_ERR_INTERNAL;
+  }
+  return RTOPK_OK;
+}
+
+int rtopk_get_phase_times(rtopk_ctx* ctx, float* ms, void* stream) {
+  if (!ctx || !ms) return RTOPK_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return RTOPK_ERR_CUDA;
+  RTOPK_CUDA(ctx, cudaStreamSynchronize((cudaStream_t)stream));
+  for (int i = 0; i < RTOPK_N_PHASES; ++i) {
+    ms[i] = -1.0f;
+    if (ctx->profile && ctx->ev_valid[i] && ctx->ev_valid[i + 1]) {
+      float t = 0.f;
+      if (cudaEventElapsedTime(&t, ctx->ev[i], ctx->ev[i + 1]) == cudaSuccess) ms[i] = t;
+      else cudaGetLastError();
+    }
+  }
+  return RTOPK_OK;
+}
+
+int rtopk_get_stats(rtopk_ctx* ctx, int32_t slice, rtopk_stats* out, void* stream) {
+  if (!ctx || !out || slice < 0 || (uint32_t)slice >= ctx->last_n_slices) return RTOPK_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return RTOPK_ERR_CUDA;
+  SelState s;
+  RTOPK_CUDA(ctx, cudaMemcpyAsync(&s, ctx->d_state + slice, sizeof(s), cudaMemcpyDeviceToHost, st));
+  RTOPK_CUDA(ctx, cudaStreamSynchronize(st));
+  std::memset(out, 0, sizeof(*out));
+  out->tau_key = s.prefix;
+  out->tie_quota = s.need;
+  out->n_greater = s.n_gt;
+  out->n_candidates = s.n_cand;
+  out->used_fallback = (s.flags & FLAG_FELL_BACK) ? 1u : 0u;
+  return RTOPK_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,352 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle, element by element.
+
+Bar: message indices, message values and the residual are bit-exact; the aggregated update is
+within 1e-6 * max|g| of the oracle's double-precision result (and, because the library sums in a
+fixed order in double precision, in fact equal to its binary32 rounding).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2005_10761_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+AUTO, EXACT = 0, 1
+
+
+@pytest.fixture(scope="module")
+def lib():
+    import paper_2005_10761_b200 as pkg
+    from paper_2005_10761_b200 import build
+    build.build()
+    return pkg
+
+
+def _ctx(lib, d, W, r, k, S=1, path=AUTO):
+    ctx = lib.RTopK(d_max=d, W_max=W, r_max=r, k_max=k, segments_max=S)
+    ctx.set_option(0, path)
+    return ctx
+
+
+def _bits(x):
+    return np.ascontiguousarray(x).view(np.uint32)
+
+
+def _pad(a: np.ndarray, mult=8, fill=0.0):
+    W, d = a.shape
+    ld = wl.round_up(d, mult)
+    out = np.full((W, ld), fill, dtype=a.dtype)
+    out[:, :d] = a
+    return out
+
+
+def run_gpu(lib, g, m0, d, r, k, seed, step, worker_base=0, path=AUTO, ctx=None, bf16=False):
+    """g, m0: float32 numpy [W, ld] (g is converted to bfloat16 on request).  Returns numpy
+    (idx, val, m') from rtopk_sparsify."""
+    W = g.shape[0]
+    own = ctx is None
+    if own:
+        ctx = _ctx(lib, d, W, r, k, path=path)
+    tg = torch.from_numpy(g).cuda()
+    if bf16:
+        tg = tg.to(torch.bfloat16)
+    tm = torch.from_numpy(m0.copy()).cuda()
+    idx = torch.full((W, k), -1, dtype=torch.int32, device="cuda")
+    val = torch.full((W, k), float("nan"), dtype=torch.float32, device="cuda")
+    ctx.sparsify(tg, tm, d, r, k, seed, step, idx, val, worker_base=worker_base)
+    ctx.poll_status()
+    stats = [ctx.stats(w) for w in range(W)]
+    if own:
+        ctx.close()
+    return idx.cpu().numpy().view(np.uint32), val.cpu().numpy(), tm.cpu().numpy(), stats
+
+
+def check_against_oracle(lib, g, m0, d, r, k, seed=1, step=0, worker_base=0, path=AUTO, bf16=False):
+    if bf16:
+        gb = torch.from_numpy(g).to(torch.bfloat16)
+        g_or = gb.view(torch.int16).numpy().view(np.uint16).copy()
+    else:
+        g_or = g
+    m_or = m0.copy()
+    o_idx, o_val = oracle.sparsify(g_or, m_or, d, r, k, seed, step, worker_base)
+    g_idx, g_val, g_m, stats = run_gpu(lib, g, m0, d, r, k, seed, step, worker_base, path, bf16=bf16)
+    for w in range(g.shape[0]):
+        assert np.array_equal(g_idx[w], o_idx[w]), (
+            f"indices differ: worker {w} d={d} r={r} k={k} path={path} stats={stats[w]} "
+            f"first mismatch at {np.flatnonzero(g_idx[w] != o_idx[w])[:5]} gpu={g_idx[w][:8]} oracle={o_idx[w][:8]}")
+        assert np.array_equal(_bits(g_val[w]), _bits(o_val[w])), f"values differ: worker {w}"
+        assert np.array_equal(_bits(g_m[w, :d]), _bits(m_or[w, :d])), (
+            f"residual differs: worker {w}, at {np.flatnonzero(_bits(g_m[w, :d]) != _bits(m_or[w, :d]))[:5]}")
+        # padding columns are neither read nor written
+        assert np.array_equal(_bits(g_m[w, d:]), _bits(m0[w, d:]))
+    return stats
+
+
+def _spiky(rng, W, d, p=0.02):
+    x = rng.standard_normal((W, d)) * 1e-3
+    m = rng.random((W, d)) < p
+    return np.where(m, rng.standard_normal((W, d)), x).astype(np.float32)
+
+
+SMALL = [(1, 1, 1), (2, 2, 1), (3, 2, 2), (5, 3, 2), (31, 7, 3), (33, 33, 4), (1023, 100, 10), (4097, 41, 41),
+         (4098, 4098, 17), (5003, 1, 1), (12289, 900, 90), (40001, 400, 40)]
+
+
+@pytest.mark.parametrize("path", [AUTO, EXACT])
+@pytest.mark.parametrize("d,r,k", SMALL)
+def test_small_and_ragged_sizes(lib, d, r, k, path):
+    rng = np.random.default_rng(d * 7 + r)
+    W = 3
+    g = _pad(_spiky(rng, W, d), fill=7.0)          # poisoned padding: must never be selected
+    m0 = _pad(_spiky(rng, W, d) * 0.5, fill=-9.0)
+    check_against_oracle(lib, g, m0, d, r, k, seed=d, step=3, worker_base=5, path=path)
+
+
+@pytest.mark.parametrize("path", [AUTO, EXACT])
+def test_heavy_ties(lib, path):
+    rng = np.random.default_rng(2)
+    W, d = 2, 70001
+    cases = {
+        "all_equal": np.full((W, d), -3.25, dtype=np.float32),
+        "mostly_zero": np.where(rng.random((W, d)) < 0.01, rng.standard_normal((W, d)), 0.0).astype(np.float32),
+        "signed_zero": np.where(rng.random((W, d)) < 0.5, 0.0, -0.0).astype(np.float32),
+        "three_levels": rng.choice(np.array([0.5, -0.5, 1.0, -2.0, 0.0], dtype=np.float32), (W, d)),
+        "quantised": (np.round(rng.standard_normal((W, d)) * 4) / 4).astype(np.float32),
+    }
+    for name, g in cases.items():
+        g = _pad(g)
+        m0 = np.zeros_like(g)
+        for r, k in [(700, 70), (35000, 35), (1, 1), (d, 700), (d - 1, d - 1)]:
+            stats = check_against_oracle(lib, g, m0, d, r, k, seed=9, step=1, path=path)
+            assert stats is not None, name
+
+
+@pytest.mark.parametrize("path", [AUTO, EXACT])
+def test_non_finite_and_denormal_values(lib, path):
+    rng = np.random.default_rng(3)
+    W, d = 2, 9001
+    g = _spiky(rng, W, d)
+    g[:, 5] = np.nan; g[:, 77] = np.inf; g[:, 4000] = -np.inf; g[:, 8999] = 1e-45; g[:, 100] = -1e-42
+    g = _pad(g)
+    m0 = np.zeros_like(g)
+    for r, k in [(3, 3), (90, 9), (9001, 90)]:
+        check_against_oracle(lib, g, m0, d, r, k, seed=4, step=0, path=path)
+
+
+def test_multi_tile_many_workers_and_worker_base(lib):
+    rng = np.random.default_rng(4)
+    W, d, r, k = 7, 300007, 3000, 300
+    g = _pad(_spiky(rng, W, d, p=0.01))
+    m0 = _pad(_spiky(rng, W, d, p=0.01) * 0.3)
+    for path in (AUTO, EXACT):
+        check_against_oracle(lib, g, m0, d, r, k, seed=0xDEADBEEF12345, step=77, worker_base=1000, path=path)
+
+
+def test_limits_topk_and_randomk(lib):
+    rng = np.random.default_rng(5)
+    W, d = 2, 50000
+    g = _pad(_spiky(rng, W, d))
+    m0 = np.zeros_like(g)
+    for path in (AUTO, EXACT):
+        check_against_oracle(lib, g, m0, d, 500, 500, seed=1, step=2, path=path)      # k = r: Definition 1
+        check_against_oracle(lib, g, m0, d, d, 50, seed=1, step=2, path=path)         # r = d: Definition 2
+        check_against_oracle(lib, g, m0, d, d, d, seed=1, step=2, path=path)          # everything is sent
+
+
+def test_bf16_gradient(lib):
+    rng = np.random.default_rng(6)
+    W, d, r, k = 3, 100003, 1000, 100
+    g = _pad(_spiky(rng, W, d))
+    m0 = _pad(_spiky(rng, W, d) * 0.25)
+    for path in (AUTO, EXACT):
+        check_against_oracle(lib, g, m0, d, r, k, seed=6, step=6, path=path, bf16=True)
+
+
+@pytest.mark.parametrize("name", ["c2", "c3_f32"])
+def test_ten_steps_with_carried_residual(lib, name):
+    cfg = wl.scaled(wl.configs()[name], d=250007, W=3)
+    ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
+    m_gpu = wl.zero_residual(cfg, "cuda")
+    m_or = np.zeros((cfg.W, cfg.ld), dtype=np.float32)
+    idx = torch.zeros((cfg.W, cfg.k), dtype=torch.int32, device="cuda")
+    val = torch.zeros((cfg.W, cfg.k), dtype=torch.float32, device="cuda")
+    for t in range(cfg.steps):
+        g = wl.gradient(cfg, t, "cuda")
+        ctx.sparsify(g, m_gpu, cfg.d, cfg.r, cfg.k, cfg.seed, t, idx, val)
+        o_idx, o_val = oracle.sparsify(g.cpu().numpy(), m_or, cfg.d, cfg.r, cfg.k, cfg.seed, t)
+        assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx), f"step {t}"
+        assert np.array_equal(_bits(val.cpu().numpy()), _bits(o_val)), f"step {t}"
+        assert np.array_equal(_bits(m_gpu.cpu().numpy()), _bits(m_or)), f"step {t}"
+    ctx.poll_status()
+    ctx.close()
+
+
+def test_segmented_per_tensor_selection(lib):
+    rng = np.random.default_rng(7)
+    W = 3
+    sizes = [70001, 3, 4099, 12288, 50001, 1]       # unaligned cuts, tiny tensors, multi-tile tensors
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    d = int(off[-1])
+    seg_r = [700, 3, 4099, 100, 5000, 1]
+    seg_k = [70, 1, 40, 100, 50, 1]
+    K = sum(seg_k)
+    g = _pad(_spiky(rng, W, d))
+    m0 = _pad(_spiky(rng, W, d) * 0.5)
+    m_or = m0.copy()
+    o_idx, o_val = oracle.sparsify_segmented(g, m_or, d, off, seg_r, seg_k, seed=8, step=5, worker_base=2)
+    for path in (AUTO, EXACT):
+        ctx = _ctx(lib, d, W, sum(seg_r), K, S=len(sizes), path=path)
+        tg, tm = torch.from_numpy(g).cuda(), torch.from_numpy(m0.copy()).cuda()
+        idx = torch.zeros((W, K), dtype=torch.int32, device="cuda")
+        val = torch.zeros((W, K), dtype=torch.float32, device="cuda")
+        out = torch.empty(wl.round_up(d, 4), dtype=torch.float32, device="cuda")
+        ctx.step_segmented(tg, tm, d, off, seg_r, seg_k, 8, 5, idx, val, out, worker_base=2)
+        ctx.poll_status()
+        assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx)
+        assert np.array_equal(_bits(val.cpu().numpy()), _bits(o_val))
+        assert np.array_equal(_bits(tm.cpu().numpy()[:, :d]), _bits(m_or[:, :d]))
+        o64, o32 = oracle.aggregate(o_idx, o_val, d)
+        assert np.array_equal(_bits(out.cpu().numpy()[:d]), _bits(o32))
+        ctx.close()
+
+
+@pytest.mark.parametrize("W,d,k", [(1, 1000, 10), (4, 4096, 400), (5, 100001, 2000), (16, 300000, 3000),
+                                   (32, 50000, 50000 // 3), (300, 20000, 50)])
+def test_aggregate_against_oracle(lib, W, d, k):
+    rng = np.random.default_rng(W * 31 + k)
+    idx = np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)]).astype(np.uint32)
+    val = (rng.standard_normal((W, k)) * np.exp(2 * rng.standard_normal((W, k)))).astype(np.float32)
+    ctx = _ctx(lib, d, W, k, k)
+    t_idx = torch.from_numpy(idx.view(np.int32)).cuda()
+    t_val = torch.from_numpy(val).cuda()
+    out = torch.full((wl.round_up(d, 4),), float("nan"), dtype=torch.float32, device="cuda")
+    for mode in (lib.SCALE_MEAN, lib.SCALE_SUM):
+        ctx.aggregate(t_idx, t_val, d, out, scale_mode=mode)
+        o64, o32 = oracle.aggregate(idx, val, d, mode)
+        got = out.cpu().numpy()[:d]
+        tol = 1e-6 * float(np.abs(val).max())
+        assert np.abs(got.astype(np.float64) - o64).max() <= tol      # the stated bar
+        assert np.array_equal(_bits(got), _bits(o32))                  # and the stronger fact
+    ctx.close()
+
+
+def test_step_is_sparsify_then_aggregate(lib):
+    cfg = wl.configs()["c1"]
+    ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
+    g = wl.gradient(cfg, 0, "cuda")
+    m = wl.zero_residual(cfg, "cuda")
+    idx = torch.zeros((cfg.W, cfg.k), dtype=torch.int32, device="cuda")
+    val = torch.zeros((cfg.W, cfg.k), dtype=torch.float32, device="cuda")
+    out = torch.empty(cfg.d, dtype=torch.float32, device="cuda")
+    ctx.step(g, m, cfg.d, cfg.r, cfg.k, cfg.seed, 0, idx, val, out)
+    ctx.poll_status()
+    m_or = np.zeros((cfg.W, cfg.ld), dtype=np.float32)
+    g_host = g.cpu().numpy()
+    o_idx, o_val = oracle.sparsify(g_host, m_or, cfg.d, cfg.r, cfg.k, cfg.seed, 0)
+    o64, o32 = oracle.aggregate(o_idx, o_val, cfg.d)
+    assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx)
+    assert np.array_equal(_bits(val.cpu().numpy()), _bits(o_val))
+    assert np.array_equal(_bits(m.cpu().numpy()), _bits(m_or))
+    got = out.cpu().numpy()
+    assert np.abs(got.astype(np.float64) - o64).max() <= 1e-6 * float(np.abs(g_host).max())
+    assert np.array_equal(_bits(got), _bits(o32))
+    # the sampled threshold did its job on this configuration (no fallback)
+    assert all(ctx.stats(w)["used_fallback"] == 0 for w in range(cfg.W))
+    ctx.close()
+
+
+def test_step_host_matches_device_call(lib):
+    cfg = wl.scaled(wl.configs()["c1"], d=200003, W=3)
+    ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
+    g = wl.gradient(cfg, 0, "cpu").pin_memory()
+    m1, m2 = wl.zero_residual(cfg, "cuda"), wl.zero_residual(cfg, "cuda")
+    idx_d = torch.zeros((cfg.W, cfg.k), dtype=torch.int32, device="cuda")
+    val_d = torch.zeros((cfg.W, cfg.k), dtype=torch.float32, device="cuda")
+    out_d = torch.empty(cfg.ld, dtype=torch.float32, device="cuda")
+    ctx.step(g.cuda(), m1, cfg.d, cfg.r, cfg.k, 3, 1, idx_d, val_d, out_d)
+    idx_h = torch.zeros((cfg.W, cfg.k), dtype=torch.int32).pin_memory()
+    val_h = torch.zeros((cfg.W, cfg.k), dtype=torch.float32).pin_memory()
+    out_h = torch.zeros(cfg.d, dtype=torch.float32).pin_memory()
+    ctx.step_host(g, m2, cfg.d, cfg.r, cfg.k, 3, 1, idx_h, val_h, out_h)
+    torch.cuda.synchronize()
+    assert torch.equal(idx_h, idx_d.cpu()) and torch.equal(val_h.view(torch.int32), val_d.cpu().view(torch.int32))
+    assert torch.equal(out_h.view(torch.int32), out_d.cpu()[: cfg.d].view(torch.int32))
+    assert torch.equal(m1.view(torch.int32), m2.view(torch.int32))
+    ctx.close()
+
+
+@pytest.mark.parametrize("r,k", [(1, 1), (2, 1), (7, 3), (64, 64), (1000, 1), (1000, 999), (16384, 1024),
+                                 (111739, 11173), (2684354, 671088)])
+def test_sampler_positions_against_oracle(lib, r, k):
+    ctx = _ctx(lib, r, 1, r, k)
+    pos = torch.zeros(k, dtype=torch.int32, device="cuda")
+    for seed, step, worker, seg in [(0, 0, 0, 0), (0xABCDEF0123456789, 9, 31, 5)]:
+        ctx.sample_positions(r, k, seed, step, worker, seg, pos)
+        want = oracle.sample_positions(r, k, seed, step, worker, seg)
+        assert np.array_equal(pos.cpu().numpy().view(np.uint32), want)
+    ctx.close()
+
+
+def test_repeated_runs_are_bit_identical(lib):
+    cfg = wl.scaled(wl.configs()["c1"], d=500000, W=4)
+    g = wl.gradient(cfg, 0, "cuda")
+    ref = None
+    ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
+    for _ in range(20):
+        m = wl.zero_residual(cfg, "cuda")
+        idx = torch.zeros((cfg.W, cfg.k), dtype=torch.int32, device="cuda")
+        val = torch.zeros((cfg.W, cfg.k), dtype=torch.float32, device="cuda")
+        out = torch.empty(cfg.ld, dtype=torch.float32, device="cuda")
+        ctx.step(g, m, cfg.d, cfg.r, cfg.k, 5, 5, idx, val, out)
+        got = (idx.cpu(), val.cpu().view(torch.int32), m.cpu().view(torch.int32), out.cpu().view(torch.int32))
+        if ref is None:
+            ref = got
+        else:
+            assert all(torch.equal(a, b) for a, b in zip(ref, got))
+    ctx.close()
+
+
+def test_fallback_is_taken_and_exact_when_the_sample_misleads(lib):
+    # large values only in a region the strided sample sees little of: the estimate is too high or
+    # too low, the count check fails and the exact path must repair it
+    W, d, r, k = 2, 400000, 4000, 400
+    rng = np.random.default_rng(11)
+    g = (rng.standard_normal((W, d)) * 1e-3).astype(np.float32)
+    g[:, 1000:1000 + 6000] = rng.standard_normal((W, 6000)).astype(np.float32) * 5     # a dense hot band
+    g = _pad(g)
+    m0 = np.zeros_like(g)
+    stats = check_against_oracle(lib, g, m0, d, r, k, seed=12, step=0, path=AUTO)
+    g2 = np.zeros((W, d), dtype=np.float32)                                              # ties overflow the list
+    g2[:, ::2] = 1.0
+    g2 = _pad(g2)
+    stats2 = check_against_oracle(lib, g2, np.zeros_like(g2), d, r, k, seed=12, step=0, path=AUTO)
+    assert any(s["used_fallback"] for s in stats + stats2)
+
+
+def test_bad_arguments_return_invalid_arg_and_write_nothing(lib):
+    d, W, r, k = 4096, 2, 64, 8
+    ctx = _ctx(lib, d, W, r, k)
+    g = torch.zeros((W, d), dtype=torch.float32, device="cuda")
+    m = torch.ones((W, d), dtype=torch.float32, device="cuda")
+    idx = torch.zeros((W, k), dtype=torch.int32, device="cuda")
+    val = torch.zeros((W, k), dtype=torch.float32, device="cuda")
+    out = torch.zeros(d, dtype=torch.float32, device="cuda")
+    bad = [dict(r=8, k=9), dict(r=d + 1, k=8), dict(r=64, k=0), dict(d=d + 4), dict(r=128, k=8)]
+    for kw in bad:
+        a = dict(d=d, r=r, k=k)
+        a.update(kw)
+        with pytest.raises(lib.RTopKError) as e:
+            ctx.sparsify(g, m, a["d"], a["r"], a["k"], 0, 0, idx, val)
+        assert e.value.status == 1
+    with pytest.raises(lib.RTopKError):
+        ctx.sparsify(g[:, 1:], m, d - 1, r, k, 0, 0, idx, val)          # misaligned base / stride
+    with pytest.raises(lib.RTopKError):
+        ctx.aggregate(idx, val, d, out, scale_mode=7)
+    with pytest.raises(lib.RTopKError):
+        lib.RTopK(d_max=1 << 31, W_max=1, r_max=1, k_max=1)
+    torch.cuda.synchronize()
+    assert bool((m == 1).all())
+    ctx.poll_status()
+    ctx.close()

@@ -273,6 +273,19 @@ def test_proposition_1_closed_form_monte_carlo():
     assert (np.abs(dev) <= 5 * sigma + 1e-12).all()
 
 
+def test_nan_sums_are_stored_as_the_default_quiet_nan():
+    # IEEE 754 does not fix the payload of a NaN result; the contract does (0x7FC00000)
+    g = np.zeros((1, 8), dtype=np.float32)
+    g.view(np.uint32)[0, 2] = 0x7FFFFFFF
+    g.view(np.uint32)[0, 5] = 0xFFC12345
+    g[0, 6] = np.inf
+    m = np.zeros((1, 8), dtype=np.float32)
+    m[0, 6] = -np.inf                                  # inf - inf
+    idx, val = oracle.sparsify(g, m, 8, 3, 3, seed=0, step=0)
+    assert idx[0].tolist() == [2, 5, 6]                # equal keys: lower index first
+    assert val.view(np.uint32)[0].tolist() == [0x7FC00000] * 3
+
+
 def test_step_counter_and_resume():
     rng = np.random.default_rng(11)
     W, d, r, k = 2, 2000, 100, 20
