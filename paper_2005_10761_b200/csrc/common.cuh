@@ -78,7 +78,13 @@ struct Scratch {
   unsigned long long* look_a;   // look-back words of the first collect
   unsigned long long* look_b;   // ... of the fallback collect
   unsigned long long* look_e;   // ... of the emit pass
-  uint32_t* cand_idx;
+  uint32_t* cursor;       // [slices] next free entry of the raw candidate buffer
+  uint32_t* chunk_start;  // [chunks] where a chunk's run sits in the raw buffer ...
+  uint32_t* chunk_count;  // ... its length ...
+  uint32_t* chunk_dst;    // ... and its place in chunk order
+  uint32_t* raw_idx;      // candidates in reservation order
+  float* raw_val;
+  uint32_t* cand_idx;     // candidates in index order
   float* cand_val;
   uint32_t* draws;        // t_j
   uint32_t* first;        // first-occurrence table F

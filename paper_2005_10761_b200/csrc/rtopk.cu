@@ -15,6 +15,7 @@
 #include "common.cuh"
 #include "sampler.cuh"
 #include "select.cuh"
+#include "stream.cuh"
 
 using namespace rtopk;
 
@@ -33,6 +34,10 @@ struct rtopk_ctx {
   size_t first_entries = 0;
   uint32_t* d_cand_idx = nullptr;
   float* d_cand_val = nullptr;
+  uint32_t* d_raw_idx = nullptr;
+  float* d_raw_val = nullptr;
+  uint32_t* d_chunk_tab = nullptr;   // chunk_start | chunk_count | chunk_dst
+  size_t chunk_tab_entries = 0;
   size_t cand_entries = 0;
   uint32_t* d_draws = nullptr;
   uint32_t* d_sel_pre = nullptr;
@@ -45,6 +50,7 @@ struct rtopk_ctx {
   std::vector<Slice> cached_slices;   // what d_slices currently holds
   uint32_t last_n_slices = 0;
   // optional per-phase timing (RTOPK_OPT_PROFILE): events recorded on the caller's stream
+  int stream_blocks[2] = {0, 0};      // persistent grid of k_stream per gradient dtype
   int profile = 0;
   cudaEvent_t ev[RTOPK_N_PHASES + 1] = {};
   bool ev_valid[RTOPK_N_PHASES + 1] = {};
@@ -95,6 +101,7 @@ struct Plan {
   size_t cand_entries = 0, draw_entries = 0, first_entries = 0, sel_words = 0;
   uint32_t k_draw_max = 0, words_all_max = 0;
   bool any_select = false, any_sampler = false, any_all = false;
+  bool uniform = false;               // every slice has the same number of chunks (plain calls)
   uint32_t K_row = 0;
 };
 
@@ -111,6 +118,7 @@ int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32
   if ((int64_t)K > ctx->k_max || (int64_t)R > ctx->r_max) return RTOPK_ERR_INVALID_ARG;
   if (K * (uint64_t)W >= (1ull << 32)) return RTOPK_ERR_INVALID_ARG;
   P.K_row = (uint32_t)K;
+  P.uniform = (S == 1);
   P.slices.resize((size_t)W * (size_t)S);
   uint64_t chunks = 0, hblocks = 0, ctiles = 0, cand = 0, draws = 0, first = 0, selw = 0;
   for (int w = 0; w < W; ++w) {
@@ -127,7 +135,7 @@ int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32
       sl.row = (uint32_t)w;
       sl.segment = (uint32_t)s;
       sl.idx_base = (uint32_t)lo;
-      sl.head = (uint32_t)(lo & 3);
+      sl.head = (uint32_t)(lo & 7);   // slices sit on an 8-element grid: 16-byte bulk copies for both dtypes
       sl.msg_off = (uint32_t)msg_at;
       msg_at += sl.k;
       const uint32_t nchunks = (uint32_t)((sl.head + (uint64_t)sl.len + kChunk - 1) / kChunk);
@@ -173,6 +181,7 @@ size_t carve_zero(const rtopk_ctx* ctx, const Plan& P, Scratch& s) {
   auto take = [&](size_t bytes) { char* q = p + at; at = align_up(at + bytes, 256); return q; };
   s.tickets = (uint32_t*)take(4 * sizeof(uint32_t));
   s.done = (uint32_t*)take(P.slices.size() * sizeof(uint32_t));
+  s.cursor = (uint32_t*)take(P.slices.size() * sizeof(uint32_t));
   s.hist = (uint32_t*)take(P.slices.size() * kBins * sizeof(uint32_t));
   s.look_a = (unsigned long long*)take((size_t)P.n_chunks * 8);
   s.look_b = (unsigned long long*)take((size_t)P.n_chunks * 8);
@@ -184,7 +193,7 @@ size_t carve_zero(const rtopk_ctx* ctx, const Plan& P, Scratch& s) {
 size_t zero_region_bytes(size_t slices, size_t chunks, size_t ctiles, size_t sel_words) {
   size_t at = 0;
   auto take = [&](size_t bytes) { at = align_up(at + bytes, 256); };
-  take(16); take(slices * 4); take(slices * kBins * 4); take(chunks * 8); take(chunks * 8); take(ctiles * 8);
+  take(16); take(slices * 4); take(slices * 4); take(slices * kBins * 4); take(chunks * 8); take(chunks * 8); take(ctiles * 8);
   take(sel_words * 4);
   return at;
 }
@@ -210,7 +219,16 @@ int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t s
     mark(ctx, RTOPK_PHASE_THRESHOLD, st);
     k_sample<GradT><<<n, kSampleThreads, kSampleSmemBytes, st>>>(L);
     mark(ctx, RTOPK_PHASE_STREAM, st);
-    k_collect<GradT, true, false><<<P.n_chunks, kThreads, 0, st>>>(L);
+    {
+      const uint32_t per = (uint32_t)((P.slices[0].head + (uint64_t)P.slices[0].len + kChunk - 1) / kChunk);
+      const uint32_t uniform = P.uniform ? per : 0u;
+      const int blocks = ctx->stream_blocks[sizeof(GradT) == 4 ? 0 : 1];
+      k_stream<GradT><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
+      if (P.any_select) {
+        k_cand_scan<<<n, kOrderThreads, 0, st>>>(L);
+        k_cand_gather<<<(P.n_chunks + kWarps - 1) / kWarps, kThreads, 0, st>>>(L, P.n_chunks, uniform);
+      }
+    }
     mark(ctx, RTOPK_PHASE_EXACT, st);
     if (P.any_select) {
       for (int pass = 0; pass < 3; ++pass) k_hist<float, false><<<P.n_hist_blocks, kThreads, 0, st>>>(L, pass);
@@ -272,6 +290,11 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   if (zbytes > ctx->zero_bytes) return RTOPK_ERR_INVALID_ARG;
   L.s.slices = ctx->d_slices; L.s.state = ctx->d_state;
   L.s.cand_idx = ctx->d_cand_idx; L.s.cand_val = ctx->d_cand_val;
+  L.s.raw_idx = ctx->d_raw_idx; L.s.raw_val = ctx->d_raw_val;
+  if ((size_t)P.n_chunks > ctx->chunk_tab_entries) return RTOPK_ERR_INVALID_ARG;
+  L.s.chunk_start = ctx->d_chunk_tab;
+  L.s.chunk_count = ctx->d_chunk_tab + ctx->chunk_tab_entries;
+  L.s.chunk_dst = ctx->d_chunk_tab + 2 * ctx->chunk_tab_entries;
   L.s.draws = ctx->d_draws; L.s.first = ctx->d_first; L.s.sel_pre = ctx->d_sel_pre;
   L.s.error = ctx->d_error;
   L.grad = grad; L.residual = residual; L.msg_idx = msg_idx; L.msg_val = msg_val;
@@ -381,6 +404,10 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   alloc((void**)&ctx->d_first, ctx->first_entries * sizeof(uint32_t));
   alloc((void**)&ctx->d_cand_idx, ctx->cand_entries * sizeof(uint32_t));
   alloc((void**)&ctx->d_cand_val, ctx->cand_entries * sizeof(float));
+  alloc((void**)&ctx->d_raw_idx, ctx->cand_entries * sizeof(uint32_t));
+  alloc((void**)&ctx->d_raw_val, ctx->cand_entries * sizeof(float));
+  ctx->chunk_tab_entries = chunks;
+  alloc((void**)&ctx->d_chunk_tab, 3 * chunks * sizeof(uint32_t));
   alloc((void**)&ctx->d_draws, W * (size_t)k_max * sizeof(uint32_t));
   alloc((void**)&ctx->d_sel_pre, ctx->sel_words * sizeof(uint32_t));
   alloc((void**)&ctx->d_error, 16);
@@ -388,6 +415,17 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_sample<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSampleSmemBytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_sample<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSampleSmemBytes);
   for (int i = 0; i <= RTOPK_N_PHASES && e == cudaSuccess; ++i) e = cudaEventCreate(&ctx->ev[i]);
+  if (e == cudaSuccess) {
+    int sms = 0, per_f32 = 0, per_bf16 = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<float>));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<__nv_bfloat16>));
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_f32, k_stream<float>, kStreamThreads, sizeof(StreamSmem<float>));
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_bf16, k_stream<__nv_bfloat16>, kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>));
+    if (e == cudaSuccess && (per_f32 < 1 || per_bf16 < 1)) e = cudaErrorLaunchOutOfResources;
+    ctx->stream_blocks[0] = sms * per_f32;
+    ctx->stream_blocks[1] = sms * per_bf16;
+  }
   if (e == cudaSuccess) e = cudaMemset(ctx->d_error, 0, 16);
   if (e == cudaSuccess) e = cudaMemset(ctx->d_state, 0, slices * sizeof(SelState));
   if (e != cudaSuccess) {
@@ -404,6 +442,7 @@ int rtopk_destroy(rtopk_ctx* ctx) {
   if (!ctx) return RTOPK_ERR_INVALID_ARG;
   DeviceGuard guard(ctx->device);
   void* ptrs[] = {ctx->d_slices, ctx->d_state, ctx->d_zero, ctx->d_first, ctx->d_cand_idx, ctx->d_cand_val,
+                  ctx->d_raw_idx, ctx->d_raw_val, ctx->d_chunk_tab,
                   ctx->d_draws, ctx->d_sel_pre, ctx->d_error, ctx->d_agg_starts, ctx->d_stage};
   for (void* p : ptrs) if (p) cudaFree(p);
   for (cudaEvent_t ev : ctx->ev) if (ev) cudaEventDestroy(ev);

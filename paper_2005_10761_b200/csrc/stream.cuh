@@ -1,0 +1,304 @@
+// k_stream: the one pass over the W x d gradient and residual matrices (Algorithm 1's g + m).
+//
+// Persistent blocks; each has one producer warp and eight consumer warps.  The producer takes chunk
+// tickets from a global counter and stages the chunk's residual and gradient bytes into shared
+// memory with 1-D bulk async copies (TMA) that complete on an mbarrier; a ring of kStages buffers
+// keeps loads in flight while the consumers work.  The consumers form a = g + m, store it back,
+// flag the keys >= the sampled threshold, and append them -- in index order inside the chunk
+// (packed prefix sums) -- to a run of the slice's raw candidate buffer reserved with one atomicAdd
+// per chunk.  The run's start and length go into a per-chunk table; k_cand_scan / k_cand_gather
+// then lay the runs out in chunk order, which makes the final list independent of the order in
+// which chunks happened to reserve their runs.  No block ever waits on another block.
+//
+// The only waits are on the block's own mbarriers; they are bounded, and on expiry the error flag
+// is raised and the block leaves through a path every consumer takes together.
+#pragma once
+
+#include "common.cuh"
+#include "select.cuh"
+
+namespace rtopk {
+
+constexpr int kStages = 2;
+constexpr int kConsumers = kThreads;             // 256 = 8 warps
+constexpr int kStreamThreads = kConsumers + 32;  // + producer warp
+constexpr int kWaitLimit = 1 << 24;
+
+struct StageDesc { uint32_t slice, chunk, valid, pad; };
+
+template <typename GradT>
+struct StreamSmem {
+  alignas(128) float m[kStages][kChunk];
+  alignas(128) GradT g[kStages][kChunk];
+  alignas(8) unsigned long long full[kStages];
+  unsigned long long empty[kStages];
+  StageDesc desc[kStages];
+  uint32_t wA[2][kWarps];
+  uint32_t ex[2];
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait for the phase with the given parity to complete.
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity) {
+  for (int i = 0; i < kWaitLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+// 1-D bulk async copy global -> shared (TMA); src, dst 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+// Barrier over the consumer threads only (the producer warp never joins it).
+__device__ __forceinline__ void consumer_sync() {
+  asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory");
+}
+// ... with an OR-reduction of a predicate: every consumer learns whether any of them failed.
+__device__ __forceinline__ bool consumer_any(bool flag) {
+  uint32_t out;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.or.pred p, 2, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(out) : "r"((uint32_t)flag), "n"(kConsumers) : "memory");
+  return out != 0;
+}
+
+template <typename GradT> struct SmemGrad;
+template <> struct SmemGrad<float> {
+  static __device__ __forceinline__ float4 ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+  static __device__ __forceinline__ float ld1(const float* p) { return *p; }
+};
+template <> struct SmemGrad<__nv_bfloat16> {
+  static __device__ __forceinline__ float4 ld4(const __nv_bfloat16* p) {
+    const uint2 v = *reinterpret_cast<const uint2*>(p);
+    float4 f;
+    f.x = __uint_as_float(v.x << 16); f.y = __uint_as_float(v.x & 0xFFFF0000u);
+    f.z = __uint_as_float(v.y << 16); f.w = __uint_as_float(v.y & 0xFFFF0000u);
+    return f;
+  }
+  static __device__ __forceinline__ float ld1(const __nv_bfloat16* p) {
+    return __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t*>(p)) << 16);
+  }
+};
+
+template <typename GradT>
+__global__ void __launch_bounds__(kStreamThreads) k_stream(Launch L, uint32_t total_tiles, uint32_t uniform_chunks) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  StreamSmem<GradT>& sm = *reinterpret_cast<StreamSmem<GradT>*>(smem_raw);
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], kWarps); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const Slice* slices = L.s.slices;
+
+  if (warp == kWarps) {
+    // ------------------------------------------------------------------ producer (one lane)
+    if (lane != 0) return;
+    const char* grad = static_cast<const char*>(L.grad);
+    for (uint32_t i = 0;; ++i) {
+      const uint32_t stage = i % kStages, phase = (i / kStages) & 1u;
+      const uint32_t tile = blockIdx.x + i * gridDim.x;
+      if (!mbar_wait(&sm.empty[stage], phase ^ 1u)) { atomicOr(L.s.error, ERR_LOOKBACK_TIMEOUT); return; }
+      if (tile >= total_tiles) {
+        sm.desc[stage].valid = 0;
+        mbar_arrive(&sm.full[stage]);
+        return;
+      }
+      const uint32_t sl = uniform_chunks ? tile / uniform_chunks
+                                         : find_slice(L.n_slices, tile, [&](uint32_t s) { return slices[s].chunk_begin; });
+      const Slice* S = slices + sl;
+      const uint32_t head = S->head, span = head + S->len;
+      const uint32_t c = tile - S->chunk_begin;
+      const uint32_t e0 = c * (uint32_t)kChunk;
+      const uint32_t n_el = min((uint32_t)kChunk, span - e0);
+      const uint32_t bytes_m = (n_el * 4u + 15u) & ~15u;
+      const uint32_t bytes_g = (n_el * (uint32_t)sizeof(GradT) + 15u) & ~15u;
+      sm.desc[stage].slice = sl; sm.desc[stage].chunk = c; sm.desc[stage].valid = 1;
+      mbar_arrive_expect_tx(&sm.full[stage], bytes_m + bytes_g);
+      bulk_load(sm.m[stage], L.residual + (S->m_off - head) + e0, bytes_m, &sm.full[stage]);
+      bulk_load(sm.g[stage], grad + ((S->g_off - head) + (int64_t)e0) * (int64_t)sizeof(GradT), bytes_g, &sm.full[stage]);
+    }
+  }
+
+  // -------------------------------------------------------------------- consumers
+  uint32_t cur_slice = 0xFFFFFFFFu;
+  Slice S;
+  uint32_t tau = 0x80000000u;
+  for (uint32_t i = 0;; ++i) {
+    const uint32_t stage = i % kStages, phase = (i / kStages) & 1u, buf = i & 1u;
+    const bool arrived = mbar_wait(&sm.full[stage], phase);
+    if (consumer_any(!arrived)) {                 // every consumer leaves together
+      if (tid == 0) atomicOr(L.s.error, ERR_LOOKBACK_TIMEOUT);
+      return;
+    }
+    const StageDesc d = sm.desc[stage];
+    if (!d.valid) return;
+    if (d.slice != cur_slice) {
+      cur_slice = d.slice;
+      S = slices[cur_slice];
+      tau = L.s.state[cur_slice].tau_lo;
+    }
+    const uint32_t head = S.head, span = head + S.len;
+    const uint32_t e_w = d.chunk * (uint32_t)kChunk + warp * (uint32_t)kWarpSpan;   // element on the slice's grid
+    const uint32_t l_w = warp * (uint32_t)kWarpSpan;                                 // same, inside the chunk
+    float a[kIter][4];
+#pragma unroll
+    for (int it = 0; it < kIter; ++it) {
+      const uint32_t l = l_w + it * 128u + lane * 4u;
+      const float4 m4 = *reinterpret_cast<const float4*>(&sm.m[stage][l]);
+      const float4 g4 = SmemGrad<GradT>::ld4(&sm.g[stage][l]);
+      a[it][0] = ef_add(g4.x, m4.x); a[it][1] = ef_add(g4.y, m4.y);
+      a[it][2] = ef_add(g4.z, m4.z); a[it][3] = ef_add(g4.w, m4.w);
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.empty[stage]);      // the stage may be refilled from here on
+    float* res = L.residual + (S.m_off - head);
+    uint32_t maskA = 0;
+#pragma unroll
+    for (int it = 0; it < kIter; ++it) {
+      const uint32_t e = e_w + it * 128u + lane * 4u;
+      uint32_t valid;
+      if (e >= head && e + 4u <= span) {
+        valid = 0xFu;
+        __stcs(reinterpret_cast<float4*>(res + e), make_float4(a[it][0], a[it][1], a[it][2], a[it][3]));
+      } else {
+        valid = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (e + j >= head && e + j < span) { valid |= 1u << j; res[e + j] = a[it][j]; }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        maskA |= (uint32_t)(((valid >> j) & 1u) && mag_key(a[it][j]) >= tau) << (it * 4 + j);
+    }
+    uint32_t packA = 0;
+#pragma unroll
+    for (int it = 0; it < kIter; ++it) packA |= (uint32_t)__popc((maskA >> (it * 4)) & 0xFu) << (it * 8);
+    const uint32_t inclA = warp_incl_scan(packA);
+    const uint32_t totA = __shfl_sync(0xFFFFFFFFu, inclA, 31);
+    const uint32_t exLaneA = inclA - packA;
+    uint32_t wA = 0;
+#pragma unroll
+    for (int it = 0; it < kIter; ++it) wA += (totA >> (it * 8)) & 0xFFu;
+    if (lane == 0) sm.wA[buf][warp] = wA;
+    consumer_sync();
+    if (tid == 0) {
+      uint32_t bA = 0;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) bA += sm.wA[buf][w];
+      const uint32_t start = bA ? atomicAdd(&L.s.cursor[cur_slice], bA) : 0u;
+      const uint32_t tile = S.chunk_begin + d.chunk;
+      L.s.chunk_start[tile] = start;
+      L.s.chunk_count[tile] = bA;
+      sm.ex[buf] = start;
+    }
+    consumer_sync();
+    if (maskA) {
+      uint32_t before = sm.ex[buf];
+      for (uint32_t w = 0; w < warp; ++w) before += sm.wA[buf][w];
+      uint32_t* cidx = L.s.raw_idx + S.cand_off;
+      float* cval = L.s.raw_val + S.cand_off;
+#pragma unroll
+      for (int it = 0; it < kIter; ++it) {
+        const uint32_t bits = (maskA >> (it * 4)) & 0xFu;
+        if (bits) {
+          uint32_t pos = before + ((exLaneA >> (it * 8)) & 0xFFu);
+          const uint32_t e = e_w + it * 128u + lane * 4u;
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if ((bits >> j) & 1u) {
+              if (pos < S.cand_cap) { cidx[pos] = e + j - head; cval[pos] = a[it][j]; }
+              ++pos;
+            }
+        }
+        before += (totA >> (it * 8)) & 0xFFu;
+      }
+    }
+  }
+}
+
+// Chunk-order layout of the raw runs, one block per slice: chunk_dst = exclusive prefix of the
+// chunk counts; the total is the slice's candidate count.
+constexpr int kOrderThreads = 1024;
+__global__ void __launch_bounds__(kOrderThreads) k_cand_scan(Launch L) {
+  __shared__ uint32_t s_warp[32];
+  __shared__ uint32_t s_carry, s_total;
+  const Slice S = L.s.slices[blockIdx.x];
+  if (S.r == S.len) return;
+  const uint32_t n = slice_chunks(S);
+  const uint32_t* cnt = L.s.chunk_count + S.chunk_begin;
+  uint32_t* dst = L.s.chunk_dst + S.chunk_begin;
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) s_carry = 0;
+  __syncthreads();
+  for (uint32_t base = 0; base < n; base += kOrderThreads) {
+    const uint32_t c = base + tid;
+    const uint32_t v = c < n ? cnt[c] : 0u;
+    const uint32_t incl = warp_incl_scan(v);
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      const uint32_t x = s_warp[lane];
+      const uint32_t xi = warp_incl_scan(x);
+      s_warp[lane] = xi - x;
+      if (lane == 31) s_total = xi;
+    }
+    __syncthreads();
+    const uint32_t carry = s_carry;
+    if (c < n) dst[c] = carry + s_warp[warp] + incl - v;
+    __syncthreads();
+    if (tid == 0) s_carry = carry + s_total;
+    __syncthreads();
+  }
+  if (tid == 0) {
+    SelState* st = &L.s.state[blockIdx.x];
+    st->n_cand = s_carry;
+    st->n_cand_first = s_carry;
+  }
+}
+
+// Copies every chunk's run to its place in chunk order (one warp per chunk).
+__global__ void __launch_bounds__(kThreads) k_cand_gather(Launch L, uint32_t total_tiles, uint32_t uniform_chunks) {
+  const uint32_t tile = blockIdx.x * kWarps + (threadIdx.x >> 5);
+  if (tile >= total_tiles) return;
+  const uint32_t lane = lane_id();
+  const Slice* slices = L.s.slices;
+  const uint32_t sl = uniform_chunks ? tile / uniform_chunks
+                                     : find_slice(L.n_slices, tile, [&](uint32_t s) { return slices[s].chunk_begin; });
+  const uint32_t count = L.s.chunk_count[tile];
+  if (count == 0) return;
+  const Slice* S = slices + sl;
+  const uint32_t cap = S->cand_cap, off = S->cand_off;
+  if (cap == 0) return;
+  const uint32_t n_cand = L.s.state[sl].n_cand;
+  if (n_cand > cap) return;                       // overflowed: the exact path rebuilds the list
+  const uint32_t src = L.s.chunk_start[tile], dst = L.s.chunk_dst[tile];
+  for (uint32_t i = lane; i < count; i += 32) {
+    L.s.cand_idx[off + dst + i] = L.s.raw_idx[off + src + i];
+    L.s.cand_val[off + dst + i] = L.s.raw_val[off + src + i];
+  }
+}
+
+}  // namespace rtopk
