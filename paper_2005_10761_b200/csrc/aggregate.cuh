@@ -1,11 +1,14 @@
 // Master step of Algorithm 1: ghat = (1/n) sum_i ghat_i, from the n = W sparse messages.
 //
-// Sort-free and atomic-free: every message row is ascending in index, so each worker's entries for
-// an output range [lo, lo + kAggTile) are one contiguous run, found by binary search (k_agg_starts).
-// The block that owns the range adds them worker by worker into a shared-memory tile of doubles (a worker's indices are distinct,
-// so there is no conflict inside a round), and writes the tile once -- the zero fill of the dense
-// output and the scatter are the same pass.  The sum order is fixed (worker 0, 1, ...), so the
-// result is bit-reproducible.
+// Sort-free and atomic-free.  Every message row is ascending in index, so each worker's entries for
+// an output range [lo, lo + kAggTile) are one contiguous run, found by binary search
+// (k_agg_starts).  Sums run in double precision in worker order (0, 1, ...) and are rounded once, so
+// the result is bit-reproducible.
+//
+//   k_aggregate_sparse  (W * k << d, the usual case): the output has been cleared by a memset and
+//                       only the coordinates that some worker sent are computed;
+//   k_aggregate         (dense messages): a block adds the runs worker by worker into a shared
+//                       tile of doubles and writes the tile once (zero fill and scatter in one pass).
 #pragma once
 
 #include "common.cuh"
@@ -14,6 +17,8 @@ namespace rtopk {
 
 constexpr int kAggTile = 4096;
 constexpr int kAggThreads = 256;
+constexpr int kAggStage = 1024;   // entries of one output tile staged in shared memory
+constexpr int kAggMaxW = 1024;    // workers the sparse kernel keeps run tables for
 
 __device__ __forceinline__ uint32_t lower_bound_u32(const uint32_t* a, uint32_t n, uint32_t key) {
   uint32_t lo = 0, hi = n;
@@ -41,8 +46,11 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(const uint32_t* __res
                                                            uint32_t W, uint32_t K, int mean,
                                                            float* __restrict__ out) {
   __shared__ double acc[kAggTile];
-  __shared__ uint32_t s_beg[kAggThreads], s_end[kAggThreads];
-  const uint32_t tid = threadIdx.x;
+  __shared__ uint32_t s_beg[kAggThreads], s_pre[kAggThreads + 1];
+  __shared__ uint32_t st_idx[kAggStage];
+  __shared__ float st_val[kAggStage];
+  __shared__ uint32_t s_warp[kAggThreads / 32];
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t ntiles = gridDim.x;
   const uint32_t lo = blockIdx.x * (uint32_t)kAggTile;
   const uint32_t hi = min(d, lo + (uint32_t)kAggTile);
@@ -50,49 +58,152 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(const uint32_t* __res
   for (uint32_t w0 = 0; w0 < W; w0 += kAggThreads) {
     const uint32_t nw = min((uint32_t)kAggThreads, W - w0);
     __syncthreads();
+    // each worker's run for this tile, and the exclusive prefix of the run lengths
+    uint32_t cnt = 0;
     if (tid < nw) {
       const uint32_t* st = starts + (size_t)(w0 + tid) * (ntiles + 1) + blockIdx.x;
-      s_beg[tid] = __ldg(st); s_end[tid] = __ldg(st + 1);
+      const uint32_t b = __ldg(st), e = __ldg(st + 1);
+      s_beg[tid] = b;
+      cnt = e > b ? e - b : 0u;
     }
+    const uint32_t incl = warp_incl_scan(cnt);
+    if (lane == 31) s_warp[warp] = incl;
     __syncthreads();
-    // round w adds worker w's entries; the next worker's first entry per thread is fetched early
-    uint32_t nxt_i = 0; float nxt_v = 0.f;
-    {
-      const uint32_t b = s_beg[0], e = s_end[0];
-      if (b + tid < e) { nxt_i = __ldg(msg_idx + (size_t)w0 * K + b + tid); nxt_v = __ldg(msg_val + (size_t)w0 * K + b + tid); }
-    }
-    for (uint32_t w = 0; w < nw; ++w) {
-      const uint32_t b = s_beg[w], e = s_end[w];
-      const uint32_t cur_i = nxt_i; const float cur_v = nxt_v;
-      if (w + 1 < nw) {
-        const uint32_t b2 = s_beg[w + 1], e2 = s_end[w + 1];
-        const size_t row2 = (size_t)(w0 + w + 1) * K;
-        if (b2 + tid < e2) { nxt_i = __ldg(msg_idx + row2 + b2 + tid); nxt_v = __ldg(msg_val + row2 + b2 + tid); }
-      }
-      const size_t row = (size_t)(w0 + w) * K;
-      // the unsigned range check keeps a malformed (unsorted / out-of-range) row inside the tile
-      if (b + tid < e && cur_i - lo < (uint32_t)kAggTile) acc[cur_i - lo] += (double)cur_v;
-      for (uint32_t q = b + tid + kAggThreads; q < e; q += kAggThreads) {
-        const uint32_t i = __ldg(msg_idx + row + q) - lo;
-        if (i < (uint32_t)kAggTile) acc[i] += (double)__ldg(msg_val + row + q);
+    uint32_t woff = 0;
+    for (uint32_t w = 0; w < warp; ++w) woff += s_warp[w];
+    s_pre[tid] = woff + incl - cnt;
+    if (tid == kAggThreads - 1) s_pre[kAggThreads] = woff + incl;
+    __syncthreads();
+    const uint32_t total = s_pre[kAggThreads];
+    if (total <= (uint32_t)kAggStage) {
+      // stage every entry of the tile with one round of loads, then add worker by worker
+      for (uint32_t q = tid; q < total; q += kAggThreads) {
+        uint32_t a = 0, b = nw;                       // last worker with s_pre[w] <= q
+        while (b - a > 1) { const uint32_t mid = (a + b) >> 1; if (s_pre[mid] <= q) a = mid; else b = mid; }
+        const size_t at = (size_t)(w0 + a) * K + s_beg[a] + (q - s_pre[a]);
+        st_idx[q] = __ldg(msg_idx + at);
+        st_val[q] = __ldg(msg_val + at);
       }
       __syncthreads();
+      for (uint32_t w = 0; w < nw; ++w) {
+        const uint32_t b = s_pre[w], e = s_pre[w + 1];
+        if (e > b) {                                   // block-uniform
+          for (uint32_t q = b + tid; q < e; q += kAggThreads) {
+            const uint32_t i = st_idx[q] - lo;        // the unsigned check keeps a malformed row inside the tile
+            if (i < (uint32_t)kAggTile) acc[i] += (double)st_val[q];
+          }
+          __syncthreads();
+        }
+      }
+    } else {
+      for (uint32_t w = 0; w < nw; ++w) {
+        const uint32_t b = s_beg[w], n = s_pre[w + 1] - s_pre[w];
+        const size_t row = (size_t)(w0 + w) * K;
+        for (uint32_t q = tid; q < n; q += kAggThreads) {
+          const uint32_t i = __ldg(msg_idx + row + b + q) - lo;
+          if (i < (uint32_t)kAggTile) acc[i] += (double)__ldg(msg_val + row + b + q);
+        }
+        __syncthreads();
+      }
     }
   }
   __syncthreads();
   const double inv = (double)W;
   if (hi - lo == (uint32_t)kAggTile) {
     for (uint32_t i = tid * 4; i < (uint32_t)kAggTile; i += kAggThreads * 4) {
+      const double a0 = acc[i + 0], a1 = acc[i + 1], a2 = acc[i + 2], a3 = acc[i + 3];
       float4 o;
-      o.x = (float)(mean ? acc[i + 0] / inv : acc[i + 0]);
-      o.y = (float)(mean ? acc[i + 1] / inv : acc[i + 1]);
-      o.z = (float)(mean ? acc[i + 2] / inv : acc[i + 2]);
-      o.w = (float)(mean ? acc[i + 3] / inv : acc[i + 3]);
+      o.x = (float)(mean && a0 != 0.0 ? a0 / inv : a0);   // most entries are zero: skip their division
+      o.y = (float)(mean && a1 != 0.0 ? a1 / inv : a1);
+      o.z = (float)(mean && a2 != 0.0 ? a2 / inv : a2);
+      o.w = (float)(mean && a3 != 0.0 ? a3 / inv : a3);
       __stcs(reinterpret_cast<float4*>(out + lo + i), o);
     }
   } else {
     for (uint32_t i = tid; i < hi - lo; i += kAggThreads)
       out[lo + i] = (float)(mean ? acc[i] / inv : acc[i]);
+  }
+}
+
+// A block stages the entries of its tile (all workers' runs, in worker order); the entry of the
+// lowest worker that holds a coordinate owns it and sums that coordinate over the workers in
+// ascending order (binary search in each staged run): the same fixed-order sum as k_aggregate.
+__global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(const uint32_t* __restrict__ msg_idx,
+                                                                  const float* __restrict__ msg_val,
+                                                                  const uint32_t* __restrict__ starts, uint32_t d,
+                                                                  uint32_t W, uint32_t K, int mean,
+                                                                  float* __restrict__ out) {
+  __shared__ uint32_t s_beg[kAggMaxW], s_pre[kAggMaxW + 1];
+  __shared__ uint32_t st_idx[kAggStage];
+  __shared__ float st_val[kAggStage];
+  __shared__ uint32_t s_warp[kAggThreads / 32];
+  __shared__ uint32_t s_carry;
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t ntiles = gridDim.x;
+  const uint32_t lo = blockIdx.x * (uint32_t)kAggTile;
+  if (tid == 0) s_carry = 0;
+  __syncthreads();
+  for (uint32_t w0 = 0; w0 < W; w0 += kAggThreads) {
+    const uint32_t w = w0 + tid;
+    uint32_t cnt = 0;
+    if (w < W) {
+      const uint32_t* st = starts + (size_t)w * (ntiles + 1) + blockIdx.x;
+      const uint32_t b = __ldg(st), e = __ldg(st + 1);
+      s_beg[w] = b;
+      cnt = e > b ? e - b : 0u;
+    }
+    const uint32_t incl = warp_incl_scan(cnt);
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    uint32_t woff = s_carry;
+    for (uint32_t x = 0; x < warp; ++x) woff += s_warp[x];
+    if (w < W) s_pre[w] = woff + incl - cnt;
+    __syncthreads();
+    if (tid == kAggThreads - 1) s_carry = woff + incl;
+    __syncthreads();
+  }
+  const uint32_t total = s_carry;
+  if (total == 0) return;
+  if (tid == 0) s_pre[W] = total;
+  const bool staged = total <= (uint32_t)kAggStage;
+  __syncthreads();
+  auto worker_of = [&](uint32_t q) {                 // last worker with s_pre[w] <= q
+    uint32_t a = 0, b = W;
+    while (b - a > 1) { const uint32_t mid = (a + b) >> 1; if (s_pre[mid] <= q) a = mid; else b = mid; }
+    return a;
+  };
+  if (staged) {
+    for (uint32_t q = tid; q < total; q += kAggThreads) {
+      const uint32_t a = worker_of(q);
+      const size_t at = (size_t)a * K + s_beg[a] + (q - s_pre[a]);
+      st_idx[q] = __ldg(msg_idx + at);
+      st_val[q] = __ldg(msg_val + at);
+    }
+    __syncthreads();
+  }
+  auto idx_at = [&](uint32_t w, uint32_t j) {        // j-th entry of worker w's run in this tile
+    return staged ? st_idx[s_pre[w] + j] : __ldg(msg_idx + (size_t)w * K + s_beg[w] + j);
+  };
+  auto val_at = [&](uint32_t w, uint32_t j) {
+    return staged ? st_val[s_pre[w] + j] : __ldg(msg_val + (size_t)w * K + s_beg[w] + j);
+  };
+  for (uint32_t q = tid; q < total; q += kAggThreads) {
+    const uint32_t w = worker_of(q);
+    const uint32_t idx = idx_at(w, q - s_pre[w]);
+    if (idx - lo >= (uint32_t)kAggTile || idx >= d) continue;   // malformed row: ignore
+    double sum = 0.0;
+    bool owner = true;
+    for (uint32_t x = 0; x < W; ++x) {
+      if (x == w) { sum += (double)val_at(w, q - s_pre[w]); continue; }
+      const uint32_t n = s_pre[x + 1] - s_pre[x];
+      uint32_t a = 0, b = n;
+      while (a < b) { const uint32_t mid = (a + b) >> 1; if (idx_at(x, mid) < idx) a = mid + 1; else b = mid; }
+      if (a < n && idx_at(x, a) == idx) {
+        if (x < w) { owner = false; break; }          // a lower worker owns this coordinate
+        sum += (double)val_at(x, a);
+      }
+    }
+    if (owner) out[idx] = (float)(mean ? sum / (double)W : sum);
   }
 }
 

@@ -66,7 +66,8 @@ struct SelState {
   uint32_t stage;
   uint32_t flags;
   uint32_t n_cand_first;// candidates of the sampled-threshold pass (statistics)
-  uint32_t pad[2];
+  uint32_t tau_hi;      // sampled upper estimate of the r-th largest key (0x7FFFFFFF = none)
+  uint32_t pad;
 };
 
 struct Scratch {
@@ -74,7 +75,7 @@ struct Scratch {
   SelState* state;
   uint32_t* hist;         // [slices][kBins]
   uint32_t* done;         // [slices] block-completion counters
-  uint32_t* tickets;      // [4] dynamic tile counters
+  uint32_t* tickets;      // [0..2] dynamic tile counters; [3] slices whose sampled threshold missed
   unsigned long long* look_a;   // look-back words of the first collect
   unsigned long long* look_b;   // ... of the fallback collect
   unsigned long long* look_e;   // ... of the emit pass
@@ -103,6 +104,7 @@ struct Launch {
   uint32_t worker_base;
   uint32_t seed_lo, seed_hi;
   uint32_t step;
+  uint32_t general_primary;   // 1: the full-vector radix select is the main path, not a fallback
 };
 
 // ----------------------------------------------------------------------------- small helpers

@@ -6,6 +6,7 @@
 
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -50,7 +51,13 @@ struct rtopk_ctx {
   std::vector<Slice> cached_slices;   // what d_slices currently holds
   uint32_t last_n_slices = 0;
   // optional per-phase timing (RTOPK_OPT_PROFILE): events recorded on the caller's stream
+  int sms = 0;
+  int finish_max_clusters[5] = {0, 0, 0, 0, 0};   // co-resident k_finish clusters of size 1, 2, 4, 8, 16
   int stream_blocks[2] = {0, 0};      // persistent grid of k_stream per gradient dtype
+  // work that does not depend on the data (the k-of-r subset, clearing the dense update) runs on a
+  // side stream next to the streaming pass
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   int profile = 0;
   cudaEvent_t ev[RTOPK_N_PHASES + 1] = {};
   bool ev_valid[RTOPK_N_PHASES + 1] = {};
@@ -91,7 +98,7 @@ struct DeviceGuard {
 
 uint32_t cand_capacity(uint64_t len, uint64_t r) {
   const uint64_t c = 2 * r + 1024;
-  return (uint32_t)(c < len ? c : len);
+  return (uint32_t)(((c < len ? c : len) + 31u) & ~31ull);     // multiples of 32 keep every list 128-byte aligned
 }
 
 // Layout of one call: the slice table plus every per-call scratch offset.
@@ -231,18 +238,22 @@ int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t s
     }
     mark(ctx, RTOPK_PHASE_EXACT, st);
     if (P.any_select) {
-      for (int pass = 0; pass < 3; ++pass) k_hist<float, false><<<P.n_hist_blocks, kThreads, 0, st>>>(L, pass);
-      k_collect<float, false, true><<<P.n_chunks, kThreads, 0, st>>>(L);
+      const uint32_t hgrid = std::min<uint32_t>(P.n_hist_blocks, (uint32_t)ctx->sms * 8u);
+      const uint32_t cgrid = std::min<uint32_t>(P.n_chunks, (uint32_t)ctx->sms * 4u);
+      for (int pass = 0; pass < 3; ++pass) k_hist<float, false><<<hgrid, kThreads, 0, st>>>(L, pass, P.n_hist_blocks);
+      k_collect<float, false, true><<<cgrid, kThreads, 0, st>>>(L, P.n_chunks);
     }
   } else {
     mark(ctx, RTOPK_PHASE_THRESHOLD, st);
     k_init_state<<<(n + 127) / 128, 128, 0, st>>>(L, 1u);
     mark(ctx, RTOPK_PHASE_STREAM, st);
-    k_hist<GradT, true><<<P.n_hist_blocks, kThreads, 0, st>>>(L, 0);
+    const uint32_t hgrid = std::min<uint32_t>(P.n_hist_blocks, (uint32_t)ctx->sms * 8u);
+    const uint32_t cgrid = std::min<uint32_t>(P.n_chunks, (uint32_t)ctx->sms * 4u);
+    k_hist<GradT, true><<<hgrid, kThreads, 0, st>>>(L, 0, P.n_hist_blocks);
     mark(ctx, RTOPK_PHASE_EXACT, st);
     if (P.any_select) {
-      for (int pass = 1; pass < 3; ++pass) k_hist<float, false><<<P.n_hist_blocks, kThreads, 0, st>>>(L, pass);
-      k_collect<float, false, true><<<P.n_chunks, kThreads, 0, st>>>(L);
+      for (int pass = 1; pass < 3; ++pass) k_hist<float, false><<<hgrid, kThreads, 0, st>>>(L, pass, P.n_hist_blocks);
+      k_collect<float, false, true><<<cgrid, kThreads, 0, st>>>(L, P.n_chunks);
     }
   }
   return RTOPK_OK;
@@ -272,7 +283,7 @@ int run_sampler(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st)
 int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
                   int64_t d, int32_t W, int32_t worker_base, int32_t S, const int64_t* seg_off,
                   const int64_t* seg_r, const int64_t* seg_k, uint64_t seed, uint32_t step, uint32_t* msg_idx,
-                  float* msg_val, cudaStream_t st, uint32_t* K_out) {
+                  float* msg_val, cudaStream_t st, uint32_t* K_out, float* clear_out = nullptr) {
   int rc = check_common(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, msg_idx, msg_val);
   if (rc) return rc;
   if (S < 1 || S > ctx->S_max || !seg_off || !seg_r || !seg_k) return RTOPK_ERR_INVALID_ARG;
@@ -302,24 +313,45 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   L.worker_base = (uint32_t)worker_base;
   L.seed_lo = (uint32_t)seed; L.seed_hi = (uint32_t)(seed >> 32);
   L.step = step;
+  L.general_primary = ctx->select_path == 1 ? 1u : 0u;
 
   rc = upload_slices(ctx, P, st);
   if (rc) return rc;
   ctx->last_n_slices = L.n_slices;
   mark(ctx, RTOPK_PHASE_SUBSET, st);
   RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero, 0, zbytes, st));
-  rc = run_sampler(ctx, P, L, st);
-  if (rc) return rc;
+  const bool forked = P.any_sampler || clear_out != nullptr;
+  if (forked) {
+    // work that does not depend on the data runs beside the streaming pass: the k-of-r subset and,
+    // for a step call, the clearing of the dense update
+    RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_fork, st));
+    RTOPK_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
+    rc = run_sampler(ctx, P, L, ctx->side);
+    if (rc) return rc;
+    if (clear_out) RTOPK_CUDA(ctx, cudaMemsetAsync(clear_out, 0, (size_t)d * sizeof(float), ctx->side));
+    RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_join, ctx->side));
+  }
   rc = grad_dtype == RTOPK_F32 ? launch_select<float>(ctx, P, L, st) : launch_select<__nv_bfloat16>(ctx, P, L, st);
   if (rc) return rc;
+  if (forked) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0));
   mark(ctx, RTOPK_PHASE_SELECT, st);
   if (P.any_select) {
-    for (int pass = 0; pass < 3; ++pass) k_cand_hist<<<P.n_ctiles, kThreads, 0, st>>>(L, pass);
-    mark(ctx, RTOPK_PHASE_EMIT, st);
-    k_emit<<<P.n_ctiles, kThreads, 0, st>>>(L);
-  } else {
-    mark(ctx, RTOPK_PHASE_EMIT, st);
+    // the largest cluster size that still lets every slice's cluster be resident at once
+    int cs = 1;
+    for (int i = 4; i >= 0; --i)
+      if ((int)L.n_slices <= ctx->finish_max_clusters[i]) { cs = 1 << i; break; }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)cs * L.n_slices, 1, 1);
+    cfg.blockDim = dim3(kFinishThreads, 1, 1);
+    cfg.dynamicSmemBytes = kFinishSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    RTOPK_CUDA(ctx, cudaLaunchKernelEx(&cfg, k_finish, L));
   }
+  mark(ctx, RTOPK_PHASE_EMIT, st);
   if (P.any_all) {
     const dim3 grid((P.words_all_max + kThreads - 1) / kThreads, L.n_slices);
     k_emit_all<<<grid, kThreads, 0, st>>>(L, P.words_all_max);
@@ -331,8 +363,14 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   return RTOPK_OK;
 }
 
+bool aggregate_is_sparse(int64_t d, int32_t W, int64_t k) {
+  return W <= kAggMaxW && (uint64_t)W * (uint64_t)k * 8ull <= (uint64_t)d;
+}
+
+// `out_cleared`: the caller has already zeroed `out` in stream order (the step calls do it beside
+// the streaming pass).
 int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
-                   int scale_mode, float* out, cudaStream_t st) {
+                   int scale_mode, float* out, cudaStream_t st, bool out_cleared = false) {
   if (!ctx || !msg_idx || !msg_val || !out) return RTOPK_ERR_INVALID_ARG;
   if (d < 1 || d > ctx->d_max || W < 1 || W > ctx->W_max || k < 1 || k > d) return RTOPK_ERR_INVALID_ARG;
   if (scale_mode != RTOPK_SCALE_MEAN && scale_mode != RTOPK_SCALE_SUM) return RTOPK_ERR_INVALID_ARG;
@@ -344,8 +382,16 @@ int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val
   if (!guard.ok) return RTOPK_ERR_CUDA;
   const dim3 sgrid((ntiles + 1 + kAggThreads - 1) / kAggThreads, (uint32_t)W);
   k_agg_starts<<<sgrid, kAggThreads, 0, st>>>(msg_idx, (uint32_t)W, (uint32_t)k, ntiles, ctx->d_agg_starts);
-  k_aggregate<<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, ctx->d_agg_starts, (uint32_t)d, (uint32_t)W,
-                                              (uint32_t)k, scale_mode == RTOPK_SCALE_MEAN ? 1 : 0, out);
+  const int mean = scale_mode == RTOPK_SCALE_MEAN ? 1 : 0;
+  if (aggregate_is_sparse(d, W, k)) {
+    // few coordinates are touched: clear the update, then compute only what was sent
+    if (!out_cleared) RTOPK_CUDA(ctx, cudaMemsetAsync(out, 0, (size_t)d * sizeof(float), st));
+    k_aggregate_sparse<<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, ctx->d_agg_starts, (uint32_t)d,
+                                                       (uint32_t)W, (uint32_t)k, mean, out);
+  } else {
+    k_aggregate<<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, ctx->d_agg_starts, (uint32_t)d, (uint32_t)W,
+                                                (uint32_t)k, mean, out);
+  }
   mark(ctx, RTOPK_N_PHASES, st);
   RTOPK_CUDA(ctx, cudaGetLastError());
   return RTOPK_OK;
@@ -388,7 +434,7 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   if (!guard.ok) { delete ctx; return RTOPK_ERR_CUDA; }
   const size_t W = (size_t)W_max, S = (size_t)segments_max, slices = W * S;
   const size_t chunks = W * ((size_t)d_max / kChunk + 2 * S + 1);
-  const size_t cand_row = std::min<size_t>((size_t)d_max, 2 * (size_t)r_max + 1024 * S);
+  const size_t cand_row = std::min<size_t>((size_t)d_max, 2 * (size_t)r_max + 1024 * S) + 32 * S;
   const size_t ctiles = W * (cand_row / kCandTile + 1 + S);
   ctx->cand_entries = W * cand_row;
   ctx->first_entries = W * (size_t)r_max;
@@ -415,6 +461,25 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_sample<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSampleSmemBytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_sample<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSampleSmemBytes);
   for (int i = 0; i <= RTOPK_N_PHASES && e == cudaSuccess; ++i) e = cudaEventCreate(&ctx->ev[i]);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFinishSmemBytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+  for (int i = 0; i < 5 && e == cudaSuccess; ++i) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1u << i, 1, 1);
+    cfg.blockDim = dim3(kFinishThreads, 1, 1);
+    cfg.dynamicSmemBytes = kFinishSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1u << i; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, k_finish, &cfg) == cudaSuccess) ctx->finish_max_clusters[i] = n;
+    else cudaGetLastError();
+  }
+  if (e == cudaSuccess && ctx->finish_max_clusters[0] < 1) e = cudaErrorLaunchOutOfResources;
   if (e == cudaSuccess) {
     int sms = 0, per_f32 = 0, per_bf16 = 0;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
@@ -423,6 +488,7 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
     if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_f32, k_stream<float>, kStreamThreads, sizeof(StreamSmem<float>));
     if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_bf16, k_stream<__nv_bfloat16>, kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>));
     if (e == cudaSuccess && (per_f32 < 1 || per_bf16 < 1)) e = cudaErrorLaunchOutOfResources;
+    ctx->sms = sms;
     ctx->stream_blocks[0] = sms * per_f32;
     ctx->stream_blocks[1] = sms * per_bf16;
   }
@@ -446,6 +512,9 @@ int rtopk_destroy(rtopk_ctx* ctx) {
                   ctx->d_draws, ctx->d_sel_pre, ctx->d_error, ctx->d_agg_starts, ctx->d_stage};
   for (void* p : ptrs) if (p) cudaFree(p);
   for (cudaEvent_t ev : ctx->ev) if (ev) cudaEventDestroy(ev);
+  if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+  if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+  if (ctx->side) cudaStreamDestroy(ctx->side);
   delete ctx;
   return RTOPK_OK;
 }
@@ -487,10 +556,13 @@ int rtopk_step(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, f
                int scale_mode, uint32_t* msg_idx, float* msg_val, float* out, void* stream) {
   if (!out || ((uintptr_t)out & 15u) || (scale_mode != RTOPK_SCALE_MEAN && scale_mode != RTOPK_SCALE_SUM))
     return RTOPK_ERR_INVALID_ARG;
-  const int rc = rtopk_sparsify(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, r, k, seed, step,
-                                msg_idx, msg_val, stream);
+  if (!ctx || d < 1 || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
+  const bool sparse = W >= 1 && k >= 1 && aggregate_is_sparse(d, W, k);
+  const int64_t off[2] = {0, d};
+  const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed,
+                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, sparse ? out : nullptr);
   if (rc) return rc;
-  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, out, (cudaStream_t)stream);
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, out, (cudaStream_t)stream, sparse);
 }
 
 int rtopk_step_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,
@@ -499,11 +571,15 @@ int rtopk_step_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64
                          uint32_t* msg_idx, float* msg_val, float* out, void* stream) {
   if (!out || ((uintptr_t)out & 15u) || (scale_mode != RTOPK_SCALE_MEAN && scale_mode != RTOPK_SCALE_SUM))
     return RTOPK_ERR_INVALID_ARG;
+  if (!ctx || d < 1 || d > ctx->d_max || S < 1 || S > ctx->S_max || !seg_k) return RTOPK_ERR_INVALID_ARG;
+  int64_t Ksum = 0;
+  for (int s = 0; s < S; ++s) Ksum += seg_k[s] > 0 ? seg_k[s] : 0;
+  const bool sparse = W >= 1 && Ksum >= 1 && aggregate_is_sparse(d, W, Ksum);
   uint32_t K = 0;
   const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, S, seg_off, seg_r,
-                               seg_k, seed, step, msg_idx, msg_val, (cudaStream_t)stream, &K);
+                               seg_k, seed, step, msg_idx, msg_val, (cudaStream_t)stream, &K, sparse ? out : nullptr);
   if (rc) return rc;
-  return aggregate_impl(ctx, msg_idx, msg_val, d, W, K, scale_mode, out, (cudaStream_t)stream);
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, K, scale_mode, out, (cudaStream_t)stream, sparse);
 }
 
 int rtopk_step_host(rtopk_ctx* ctx, const void* h_grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,

@@ -5,11 +5,13 @@
 //   k_collect       one streaming pass: a = g + m -> residual, keys above the threshold are appended
 //                   to an index-ordered candidate list (ballot/prefix compaction + look-back)
 //   k_hist          full-vector radix histogram pass (exact path and fallback)
-//   k_cand_hist     radix select of the r-th largest key among the candidates
-//   k_emit          walks the candidates in index order, numbers the members of the top-r set and
+//   k_finish        one cluster per slice: exact r-th largest key among the candidates, then a walk
+//                   over the candidates in index order that numbers the members of the top-r set and
 //                   writes the ones the k-of-r sampler chose as (index, value) messages, zeroing
 //                   their residual slots (m' = a - ghat)
 #pragma once
+
+#include <cooperative_groups.h>
 
 #include "common.cuh"
 
@@ -92,7 +94,7 @@ __global__ void k_init_state(Launch L, uint32_t general) {
   st.tau_lo = 0x80000000u;           // above every key: nothing is a candidate
   st.eq_quota = kNoQuota;
   st.prefix = 0; st.n_gt = 0; st.need = S.r; st.n_cand = 0; st.n_cand_first = 0;
-  st.pad[0] = st.pad[1] = 0;
+  st.tau_hi = 0x7FFFFFFFu; st.pad = 0;
   if (S.r == S.len) { st.resolved = 31; st.stage = STAGE_DONE; st.flags = 0; }   // top-r is everything
   else { st.resolved = 0; st.stage = STAGE_PASS0; st.flags = general ? FLAG_GENERAL : 0u; }
   L.s.state[s] = st;
@@ -100,69 +102,124 @@ __global__ void k_init_state(Launch L, uint32_t general) {
 
 // ----------------------------------------------------------------------------- sampled threshold
 // One block per slice.  Reads up to kSampleMax coordinates of a = g + m in 128-byte groups spread
-// evenly over the slice, and picks as threshold the sample key whose sample rank, scaled to the
-// slice, lies six standard deviations above r.  The collect pass then verifies the count; a miss
-// is repaired by the exact path, so the estimate only affects speed, never the result.
-template <typename GradT>
-__global__ void __launch_bounds__(kSampleThreads) k_sample(Launch L) {
-  extern __shared__ uint32_t smem[];
-  uint32_t* keys = smem;
-  uint32_t* hist = smem + kSampleMax;
-  uint32_t* scratch = hist + kBins;
-  const uint32_t sl = blockIdx.x;
-  const Slice S = L.s.slices[sl];
-  const uint32_t tid = threadIdx.x;
-  SelState st;
-  st.eq_quota = kNoQuota; st.prefix = 0; st.resolved = 0; st.n_gt = 0; st.need = S.r;
-  st.n_cand = 0; st.n_cand_first = 0; st.stage = STAGE_PASS0; st.flags = 0; st.pad[0] = st.pad[1] = 0;
-  if (S.r == S.len) {
-    st.tau_lo = 0x80000000u; st.resolved = 31; st.stage = STAGE_DONE;
-    if (tid == 0) L.s.state[sl] = st;
-    return;
-  }
-  const float* m = L.residual;
-  uint32_t n_s, rho;
-  if (S.len <= (uint32_t)kSampleMax) {
-    n_s = S.len; rho = S.r;
-    for (uint32_t i = tid; i < n_s; i += kSampleThreads)
-      keys[i] = mag_key(ef_add(Grad<GradT>::ld1(L.grad, S.g_off + i), m[S.m_off + i]));
-  } else {
-    const uint32_t v0 = (S.head + 3u) >> 2, v1 = (S.head + S.len) >> 2;   // fully valid vectors
-    const uint32_t ngroups_avail = (v1 - v0) >> 3;
-    const uint32_t G = min((uint32_t)(kSampleMax / 32), ngroups_avail);
-    n_s = G * 32u;
-    const int64_t base_g = S.g_off - S.head, base_m = S.m_off - S.head;
-    for (uint32_t n = tid; n < G * 8u; n += kSampleThreads) {
-      const uint32_t gi = n >> 3, vv = n & 7u;
-      const uint32_t vec = v0 + (uint32_t)(((uint64_t)gi * ngroups_avail) / G) * 8u + vv;
-      const float4 g4 = Grad<GradT>::ld4(L.grad, base_g + (int64_t)vec * 4);
-      const float4 m4 = __ldg(reinterpret_cast<const float4*>(m + base_m + (int64_t)vec * 4));
-      keys[n * 4 + 0] = mag_key(ef_add(g4.x, m4.x));
-      keys[n * 4 + 1] = mag_key(ef_add(g4.y, m4.y));
-      keys[n * 4 + 2] = mag_key(ef_add(g4.z, m4.z));
-      keys[n * 4 + 3] = mag_key(ef_add(g4.w, m4.w));
-    }
-    const float expect = (float)n_s * ((float)S.r / (float)S.len);
-    const float target = expect + 6.0f * sqrtf(expect) + 8.0f;
-    rho = target >= (float)n_s ? n_s : (uint32_t)target;
-  }
-  __syncthreads();
-  uint32_t prefix = 0, need = rho;
+// evenly over the slice and brackets the r-th largest key from below (tau_lo: the keys >= tau_lo
+// must number at least r) and from above (tau_hi).  The streaming pass gathers the keys >= tau_lo
+// and counts them; a miss is repaired by the exact path, and a tau_hi that is too low only costs
+// k_finish one more round, so the estimates affect speed, never the result.
+//
+// Both sample ranks are small (about 1.4 % of the sample), so the bulk is never histogrammed: every
+// thread keeps only the maximum of its 32 keys, and the rho-th largest of the 1024 maxima is a lower
+// bound of the rho-th largest key (there are at least rho keys that large).  tau_lo is that bound at
+// rank expect + 6 sigma; tau_hi the same at rank (expect - 6 sigma) * 3/4, which as a sample rank
+// stays clearly above the r-th largest.  Samples whose ranks exceed the thread count take a radix
+// select over all sample keys instead.
+__device__ __forceinline__ uint32_t block_select_desc(uint32_t key, bool has, uint32_t rank, uint32_t* hist,
+                                                      uint32_t* scratch) {
+  // rank-th largest (1-based) of one key per thread; three radix passes of one increment per thread
+  uint32_t prefix = 0, need = rank;
   for (int pass = 0; pass < 3; ++pass) {
     const int bits = digit_bits(pass), shift = digit_shift(pass);
-    for (uint32_t b = tid; b < (uint32_t)kBins; b += kSampleThreads) hist[b] = 0;
+    for (uint32_t b = threadIdx.x; b < (uint32_t)kBins; b += blockDim.x) hist[b] = 0;
     __syncthreads();
-    for (uint32_t i = tid; i < n_s; i += kSampleThreads) {
-      const uint32_t key = keys[i];
-      if (pass == 0 || (key >> (shift + bits)) == prefix) atomicAdd(&hist[(key >> shift) & ((1u << bits) - 1u)], 1u);
-    }
+    if (has && (pass == 0 || (key >> (shift + bits)) == prefix)) atomicAdd(&hist[(key >> shift) & ((1u << bits) - 1u)], 1u);
     __syncthreads();
     uint32_t D, above;
     pick_digit(hist, 1 << bits, need, scratch, D, above);
     need -= above;
     prefix = (prefix << bits) | D;
   }
-  st.tau_lo = prefix;
+  return prefix;
+}
+
+template <typename GradT>
+__global__ void __launch_bounds__(kSampleThreads) k_sample(Launch L) {
+  extern __shared__ uint32_t smem[];
+  uint32_t* keys = smem;                       // [kSampleMax]
+  uint32_t* hist = smem + kSampleMax;          // [kBins]
+  uint32_t* scratch = hist + kBins;            // [64]
+  const uint32_t sl = blockIdx.x;
+  const Slice S = L.s.slices[sl];
+  const uint32_t tid = threadIdx.x;
+  SelState st;
+  st.eq_quota = kNoQuota; st.prefix = 0; st.resolved = 0; st.n_gt = 0; st.need = S.r;
+  st.n_cand = 0; st.n_cand_first = 0; st.stage = STAGE_PASS0; st.flags = 0; st.tau_hi = 0x7FFFFFFFu; st.pad = 0;
+  if (S.r == S.len) {
+    st.tau_lo = 0x80000000u; st.resolved = 31; st.stage = STAGE_DONE;
+    if (tid == 0) L.s.state[sl] = st;
+    return;
+  }
+  const float* m = L.residual;
+  uint32_t n_s, rho_lo, rho_hi, mine = 0;
+  if (S.len <= (uint32_t)kSampleMax) {
+    n_s = S.len; rho_lo = S.r; rho_hi = max(1u, S.r - S.r / 4u);   // the sample is the whole slice
+    for (uint32_t i = tid; i < n_s; i += kSampleThreads) {
+      const uint32_t key = mag_key(ef_add(Grad<GradT>::ld1(L.grad, S.g_off + i), m[S.m_off + i]));
+      keys[i] = key;
+      mine = max(mine, key);
+    }
+  } else {
+    const uint32_t v0 = (S.head + 3u) >> 2, v1 = (S.head + S.len) >> 2;   // fully valid vectors
+    const uint32_t ngroups_avail = (v1 - v0) >> 3;
+    const uint32_t G = min((uint32_t)(kSampleMax / 32), ngroups_avail);
+    n_s = G * 32u;
+    const int64_t base_g = S.g_off - S.head, base_m = S.m_off - S.head;
+    // all of a thread's sample loads are issued before the first use (one memory latency in total)
+    constexpr int kPer = kSampleMax / 4 / kSampleThreads;
+    float4 g4[kPer], m4[kPer];
+#pragma unroll
+    for (int u = 0; u < kPer; ++u) {
+      const uint32_t n = tid + u * kSampleThreads;
+      if (n < G * 8u) {
+        const uint32_t gi = n >> 3, vv = n & 7u;
+        // group gi of G sits at floor(gi * avail / G); G is 1024 whenever avail >= 1024, else avail
+        const uint32_t grp = G == (uint32_t)(kSampleMax / 32) ? (uint32_t)(((uint64_t)gi * ngroups_avail) >> 10) : gi;
+        const uint32_t vec = v0 + grp * 8u + vv;
+        g4[u] = Grad<GradT>::ld4(L.grad, base_g + (int64_t)vec * 4);
+        m4[u] = __ldg(reinterpret_cast<const float4*>(m + base_m + (int64_t)vec * 4));
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kPer; ++u) {
+      const uint32_t n = tid + u * kSampleThreads;
+      if (n < G * 8u) {
+        const uint32_t k0 = mag_key(ef_add(g4[u].x, m4[u].x)), k1 = mag_key(ef_add(g4[u].y, m4[u].y));
+        const uint32_t k2 = mag_key(ef_add(g4[u].z, m4[u].z)), k3 = mag_key(ef_add(g4[u].w, m4[u].w));
+        keys[n * 4 + 0] = k0; keys[n * 4 + 1] = k1; keys[n * 4 + 2] = k2; keys[n * 4 + 3] = k3;
+        mine = max(max(mine, max(k0, k1)), max(k2, k3));
+      }
+    }
+    const float expect = (float)n_s * ((float)S.r / (float)S.len);
+    const float margin = 6.0f * sqrtf(expect) + 8.0f;
+    rho_lo = expect + margin >= (float)n_s ? n_s : (uint32_t)(expect + margin);
+    rho_hi = expect - margin < 2.0f ? 1u : (uint32_t)((expect - margin) * 0.75f);
+  }
+  __syncthreads();
+  const uint32_t n_holders = min(n_s, (uint32_t)kSampleThreads);     // threads that hold at least one key
+  uint32_t tau_lo, tau_hi;
+  if (rho_lo <= n_holders) {
+    tau_lo = block_select_desc(mine, tid < n_holders, rho_lo, hist, scratch);
+    tau_hi = block_select_desc(mine, tid < n_holders, rho_hi, hist, scratch);
+  } else {
+    // radix select of the rho_lo-th largest over all sample keys; no upper estimate
+    uint32_t prefix = 0, need = rho_lo;
+    for (int pass = 0; pass < 3; ++pass) {
+      const int bits = digit_bits(pass), shift = digit_shift(pass);
+      for (uint32_t b = tid; b < (uint32_t)kBins; b += kSampleThreads) hist[b] = 0;
+      __syncthreads();
+      for (uint32_t i = tid; i < n_s; i += kSampleThreads) {
+        const uint32_t key = keys[i];
+        if (pass == 0 || (key >> (shift + bits)) == prefix) atomicAdd(&hist[(key >> shift) & ((1u << bits) - 1u)], 1u);
+      }
+      __syncthreads();
+      uint32_t D, above;
+      pick_digit(hist, 1 << bits, need, scratch, D, above);
+      need -= above;
+      prefix = (prefix << bits) | D;
+    }
+    tau_lo = prefix; tau_hi = 0x7FFFFFFFu;
+  }
+  st.tau_lo = tau_lo;
+  st.tau_hi = max(tau_hi, tau_lo);
   if (tid == 0) L.s.state[sl] = st;
 }
 
@@ -171,18 +228,24 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(Launch L) {
 // eq_quota keys == tau_lo in index order.  The candidate list keeps index order: inside a block by
 // ballot-free packed prefix sums, across blocks by the look-back on (count above, count equal).
 template <typename GradT, bool FUSE, bool TIES>
-__global__ void __launch_bounds__(kThreads) k_collect(Launch L) {
+__global__ void __launch_bounds__(kThreads) k_collect(Launch L, uint32_t total_tiles) {
   __shared__ uint32_t s_tile, s_wA[kWarps], s_wB[kWarps], s_ex[2];
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (!FUSE && !L.general_primary && L.s.tickets[3] == 0) return;   // no slice needs the exact path
+  const Slice* slices = L.s.slices;
+  // persistent blocks; tiles are handed out by ticket so that the look-back only ever waits on
+  // tiles whose blocks are already running
+  while (true) {
+  __syncthreads();
   if (tid == 0) s_tile = atomicAdd(&L.s.tickets[FUSE ? 0 : 1], 1u);
   __syncthreads();
   const uint32_t tile = s_tile;
-  const Slice* slices = L.s.slices;
+  if (tile >= total_tiles) return;
   const uint32_t sl = find_slice(L.n_slices, tile, [&](uint32_t i) { return slices[i].chunk_begin; });
   const Slice S = slices[sl];
   SelState* st = &L.s.state[sl];
   if (!FUSE) {
-    if (!((st->flags & FLAG_GENERAL) && st->stage == STAGE_COLLECT)) return;
+    if (!((st->flags & FLAG_GENERAL) && st->stage == STAGE_COLLECT)) continue;
   }
   const uint32_t tau = st->tau_lo;
   const uint32_t quota = TIES ? st->eq_quota : kNoQuota;
@@ -242,7 +305,7 @@ __global__ void __launch_bounds__(kThreads) k_collect(Launch L) {
     }
   }
   __syncthreads();
-  if ((maskA | maskB) == 0) return;
+  if ((maskA | maskB) == 0) continue;
   uint32_t gt_before = s_ex[0], eq_before = s_ex[1];
   for (uint32_t w = 0; w < warp; ++w) { gt_before += s_wA[w]; eq_before += s_wB[w]; }
   uint32_t* cidx = L.s.cand_idx + S.cand_off;
@@ -266,6 +329,7 @@ __global__ void __launch_bounds__(kThreads) k_collect(Launch L) {
     }
     gt_before += (totA >> (it * 8)) & 0xFFu;
     eq_before += (totB >> (it * 8)) & 0xFFu;
+  }
   }
 }
 
@@ -329,175 +393,322 @@ __device__ __forceinline__ bool first_pass_missed(const SelState* st, const Slic
 // add and the write-back; otherwise a is read from the residual buffer.  Pass p > 0 counts only keys
 // whose higher bits equal the resolved prefix.
 template <typename GradT, bool FUSE>
-__global__ void __launch_bounds__(kThreads) k_hist(Launch L, int pass) {
+__global__ void __launch_bounds__(kThreads) k_hist(Launch L, int pass, uint32_t total_blocks) {
   __shared__ uint32_t hist_s[kBins];
   __shared__ uint32_t scratch[kWarps + 2];
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (!FUSE && !L.general_primary && L.s.tickets[3] == 0) return;   // no slice needs the exact path
   const Slice* slices = L.s.slices;
-  const uint32_t sl = find_slice(L.n_slices, blockIdx.x, [&](uint32_t i) { return slices[i].hist_begin; });
-  const Slice S = slices[sl];
-  SelState* st = &L.s.state[sl];
-  const uint32_t flags = st->flags;
-  const bool fell_back = !(flags & FLAG_GENERAL) && !FUSE && pass == 0 && S.r < S.len && first_pass_missed(st, S);
-  const bool counting = (flags & FLAG_GENERAL) ? st->stage == (uint32_t)pass : fell_back;
-  const bool add_only = FUSE && S.r == S.len;      // nothing to select, but a = g + m is still due
-  if (!counting && !add_only) return;
-  const uint32_t prefix = st->prefix;
   const int bits = digit_bits(pass), shift = digit_shift(pass);
-  for (uint32_t b = tid; b < (uint32_t)kBins; b += kThreads) hist_s[b] = 0;
-  __syncthreads();
-  const uint32_t nchunks = slice_chunks(S);
-  const uint32_t hb = blockIdx.x - S.hist_begin;
-  const uint32_t c0 = hb * kHistChunks, c1 = min(nchunks, c0 + kHistChunks);
-  const uint32_t span = S.head + S.len;
-  const int64_t base_g = S.g_off - S.head, base_m = S.m_off - S.head;
-  for (uint32_t c = c0; c < c1; ++c) {
-    const uint32_t e_w = c * (uint32_t)kChunk + warp * (uint32_t)kWarpSpan;
-    float a[kIter][4];
-    uint32_t valid[kIter];
-#pragma unroll
-    for (int it = 0; it < kIter; ++it)
-      valid[it] = load_vec<GradT, FUSE>(L.grad, L.residual, base_g, base_m, e_w + it * 128u + lane * 4u,
-                                        S.head, span, a[it]);
-    if (counting) {
+  for (uint32_t unit = blockIdx.x; unit < total_blocks; unit += gridDim.x) {
+    __syncthreads();                                   // hist_s / scratch of the previous unit are free
+    const uint32_t sl = find_slice(L.n_slices, unit, [&](uint32_t i) { return slices[i].hist_begin; });
+    const Slice S = slices[sl];
+    SelState* st = &L.s.state[sl];
+    const uint32_t flags = st->flags;
+    const bool fell_back = !(flags & FLAG_GENERAL) && !FUSE && pass == 0 && S.r < S.len && first_pass_missed(st, S);
+    const bool counting = (flags & FLAG_GENERAL) ? st->stage == (uint32_t)pass : fell_back;
+    const bool add_only = FUSE && S.r == S.len;      // nothing to select, but a = g + m is still due
+    if (!counting && !add_only) continue;
+    const uint32_t prefix = st->prefix;
+    for (uint32_t b = tid; b < (uint32_t)kBins; b += kThreads) hist_s[b] = 0;
+    __syncthreads();
+    const uint32_t nchunks = slice_chunks(S);
+    const uint32_t hb = unit - S.hist_begin;
+    const uint32_t c0 = hb * kHistChunks, c1 = min(nchunks, c0 + kHistChunks);
+    const uint32_t span = S.head + S.len;
+    const int64_t base_g = S.g_off - S.head, base_m = S.m_off - S.head;
+    for (uint32_t c = c0; c < c1; ++c) {
+      const uint32_t e_w = c * (uint32_t)kChunk + warp * (uint32_t)kWarpSpan;
+      float a[kIter][4];
+      uint32_t valid[kIter];
 #pragma unroll
       for (int it = 0; it < kIter; ++it)
+        valid[it] = load_vec<GradT, FUSE>(L.grad, L.residual, base_g, base_m, e_w + it * 128u + lane * 4u,
+                                          S.head, span, a[it]);
+      if (counting) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const uint32_t key = mag_key(a[it][j]);
-          if (((valid[it] >> j) & 1u) && (pass == 0 || (key >> (shift + bits)) == prefix))
-            atomicAdd(&hist_s[(key >> shift) & ((1u << bits) - 1u)], 1u);
-        }
-    }
-  }
-  if (!counting) return;
-  __syncthreads();
-  uint32_t* gh = L.s.hist + (size_t)sl * kBins;
-  for (uint32_t b = tid; b < (1u << bits); b += kThreads) {
-    const uint32_t v = hist_s[b];
-    if (v) atomicAdd(gh + b, v);
-  }
-  const uint32_t nblocks = (nchunks + kHistChunks - 1) / kHistChunks;
-  if (is_last_block(&L.s.done[sl], nblocks)) finish_pass(L, sl, S, pass, true, fell_back, hist_s, scratch);
-}
-
-__device__ __forceinline__ uint32_t slice_ctiles(const Slice& S) {
-  return (S.cand_cap + kCandTile - 1) / kCandTile;
-}
-
-// One digit of the radix select among the candidates of each slice.
-__global__ void __launch_bounds__(kThreads) k_cand_hist(Launch L, int pass) {
-  __shared__ uint32_t hist_s[kBins];
-  __shared__ uint32_t scratch[kWarps + 2];
-  const uint32_t tid = threadIdx.x;
-  const Slice* slices = L.s.slices;
-  const uint32_t sl = find_slice(L.n_slices, blockIdx.x, [&](uint32_t i) { return slices[i].ctile_begin; });
-  const Slice S = slices[sl];
-  SelState* st = &L.s.state[sl];
-  if (st->resolved != (uint32_t)resolved_before(pass)) return;
-  const uint32_t n_cand = st->n_cand;
-  if (n_cand < S.r || n_cand > S.cand_cap) {       // cannot happen once the exact path has run
-    if (tid == 0 && blockIdx.x == S.ctile_begin) atomicOr(L.s.error, ERR_CANDIDATE_OVERFLOW);
-    return;
-  }
-  const uint32_t prefix = st->prefix;
-  const int bits = digit_bits(pass), shift = digit_shift(pass);
-  for (uint32_t b = tid; b < (uint32_t)kBins; b += kThreads) hist_s[b] = 0;
-  __syncthreads();
-  const uint32_t t0 = (blockIdx.x - S.ctile_begin) * (uint32_t)kCandTile;
-  const float* cval = L.s.cand_val + S.cand_off;
+        for (int it = 0; it < kIter; ++it)
 #pragma unroll
-  for (int q = 0; q < kCandPer; ++q) {
-    const uint32_t i = t0 + q * kThreads + tid;
-    if (i < n_cand) {
-      const uint32_t key = mag_key(cval[i]);
-      if (pass == 0 || (key >> (shift + bits)) == prefix) atomicAdd(&hist_s[(key >> shift) & ((1u << bits) - 1u)], 1u);
-    }
-  }
-  __syncthreads();
-  uint32_t* gh = L.s.hist + (size_t)sl * kBins;
-  for (uint32_t b = tid; b < (1u << bits); b += kThreads) {
-    const uint32_t v = hist_s[b];
-    if (v) atomicAdd(gh + b, v);
-  }
-  if (is_last_block(&L.s.done[sl], slice_ctiles(S))) finish_pass(L, sl, S, pass, false, false, hist_s, scratch);
-}
-
-// ----------------------------------------------------------------------------- emit
-// Position p of a top-r member = number of members with a lower index.  Members are the candidates
-// with key > tau plus the first `quota` candidates with key == tau.  Position p is sent iff the
-// sampler's bitmap has bit p; its place in the message is the number of selected positions below p.
-__device__ __forceinline__ bool position_selected(const Launch& L, const Slice& S, uint32_t p, uint32_t& slot) {
-  if (S.k == S.r) { slot = p; return true; }
-  const uint32_t word = L.s.sel[S.sel_off + (p >> 5)];
-  slot = L.s.sel_pre[S.sel_off + (p >> 5)] + __popc(word & ((1u << (p & 31u)) - 1u));
-  return (word >> (p & 31u)) & 1u;
-}
-
-__global__ void __launch_bounds__(kThreads) k_emit(Launch L) {
-  __shared__ uint32_t s_tile, s_wA[kWarps], s_wB[kWarps], s_ex[2];
-  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) s_tile = atomicAdd(&L.s.tickets[2], 1u);
-  __syncthreads();
-  const uint32_t tile = s_tile;
-  const Slice* slices = L.s.slices;
-  const uint32_t sl = find_slice(L.n_slices, tile, [&](uint32_t i) { return slices[i].ctile_begin; });
-  const Slice S = slices[sl];
-  const SelState* st = &L.s.state[sl];
-  if (S.r == S.len || st->resolved != 31) return;
-  const uint32_t n_cand = st->n_cand;
-  if (n_cand < S.r || n_cand > S.cand_cap) return;
-  const uint32_t tau = st->prefix, quota = st->need;
-  const uint32_t ct = tile - S.ctile_begin;
-  const uint32_t i_w = ct * (uint32_t)kCandTile + warp * (uint32_t)(kCandPer * 32);
-  const uint32_t* cidx = L.s.cand_idx + S.cand_off;
-  const float* cval = L.s.cand_val + S.cand_off;
-  float val[kCandPer];
-  uint32_t ballA[kCandPer], ballB[kCandPer];
-  uint32_t wA = 0, wB = 0;
-#pragma unroll
-  for (int q = 0; q < kCandPer; ++q) {
-    const uint32_t i = i_w + q * 32u + lane;
-    bool isA = false, isB = false;
-    val[q] = 0.f;
-    if (i < n_cand) {
-      val[q] = cval[i];
-      const uint32_t key = mag_key(val[q]);
-      isA = key > tau; isB = key == tau;
-    }
-    ballA[q] = __ballot_sync(0xFFFFFFFFu, isA);
-    ballB[q] = __ballot_sync(0xFFFFFFFFu, isB);
-    wA += __popc(ballA[q]); wB += __popc(ballB[q]);
-  }
-  if (lane == 0) { s_wA[warp] = wA; s_wB[warp] = wB; }
-  __syncthreads();
-  if (warp == 0) {
-    uint32_t bA = 0, bB = 0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) { bA += s_wA[w]; bB += s_wB[w]; }
-    uint32_t exA, exB;
-    lookback_exclusive(L.s.look_e + S.ctile_begin, ct, bA, bB, exA, exB, L.s.error);
-    if (lane == 0) { s_ex[0] = exA; s_ex[1] = exB; }
-  }
-  __syncthreads();
-  uint32_t gt_before = s_ex[0], eq_before = s_ex[1];
-  for (uint32_t w = 0; w < warp; ++w) { gt_before += s_wA[w]; eq_before += s_wB[w]; }
-  const uint32_t lt = (1u << lane) - 1u;
-#pragma unroll
-  for (int q = 0; q < kCandPer; ++q) {
-    const bool isA = (ballA[q] >> lane) & 1u, isB = (ballB[q] >> lane) & 1u;
-    const uint32_t g = gt_before + __popc(ballA[q] & lt), e = eq_before + __popc(ballB[q] & lt);
-    if (isA || (isB && e < quota)) {
-      const uint32_t p = g + min(e, quota);
-      uint32_t slot;
-      if (p < S.r && position_selected(L, S, p, slot) && slot < S.k) {
-        const uint32_t idx = cidx[i_w + q * 32u + lane];
-        L.msg_idx[S.msg_off + slot] = S.idx_base + idx;
-        L.msg_val[S.msg_off + slot] = val[q];
-        L.residual[S.m_off + idx] = 0.0f;
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t key = mag_key(a[it][j]);
+            if (((valid[it] >> j) & 1u) && (pass == 0 || (key >> (shift + bits)) == prefix))
+              atomicAdd(&hist_s[(key >> shift) & ((1u << bits) - 1u)], 1u);
+          }
       }
     }
-    gt_before += __popc(ballA[q]); eq_before += __popc(ballB[q]);
+    if (!counting) continue;
+    __syncthreads();
+    uint32_t* gh = L.s.hist + (size_t)sl * kBins;
+    for (uint32_t b = tid; b < (1u << bits); b += kThreads) {
+      const uint32_t v = hist_s[b];
+      if (v) atomicAdd(gh + b, v);
+    }
+    const uint32_t nblocks = (nchunks + kHistChunks - 1) / kHistChunks;
+    if (is_last_block(&L.s.done[sl], nblocks)) finish_pass(L, sl, S, pass, true, fell_back, hist_s, scratch);
+  }
+}
+
+// ----------------------------------------------------------------------------- finish
+// One thread-block cluster per slice finishes the selection in a single launch:
+//   1. the r-th largest key among the slice's candidates.  It lies in [lo_key, hi_key): after the
+//      exact path that is the resolved radix bucket and n_gt counts the keys above it; after the
+//      sampled pass it is [tau_lo, tau_hi] and the keys above are still uncounted.  Each round
+//      spreads the interval over 2047 equal power-of-two buckets (the candidates are nearly uniform
+//      over so narrow a range, so the shared-memory increments do not pile up on a few addresses)
+//      plus one bucket for "above"; every CTA histograms its contiguous share, the CTAs read each
+//      other's histograms through distributed shared memory and pick the bucket redundantly;
+//   2. with tau and the tie quota known, every warp counts the members (key > tau, or key == tau)
+//      in its contiguous part; the counts are exchanged, giving each warp its first position;
+//   3. each warp walks its part in index order, numbers the members of the top-r set and writes the
+//      ones the sampler chose as (index, value) messages, zeroing their residual slots.
+constexpr int kMaxCluster = 16;
+constexpr int kFinishThreads = 1024;
+constexpr int kFinishWarps = kFinishThreads / 32;
+constexpr int kFinishCache = 46 * 1024;   // candidate values a CTA keeps in shared memory (184 KB)
+constexpr int kFinishBatch = 8;           // independent loads in flight per thread
+constexpr int kFinishSelWords = 2048;     // bitmap words (64 Ki positions) a CTA keeps in shared memory
+
+struct alignas(16) FinishSmem {           // the value cache behind it is read as float4
+  uint32_t hist[kBins];
+  uint32_t red[kBins];                 // the cluster's histogram, summed by every CTA for itself
+  uint32_t sel[kFinishSelWords];       // the sampler's bitmap over this CTA's positions ...
+  uint32_t sel_pre[kFinishSelWords];   // ... and its running popcount
+  uint32_t scratch[kFinishWarps + 2];
+  uint32_t counts[2 * kMaxCluster];    // (members above tau, equal to tau) of every CTA's share
+  uint32_t warpA[kFinishWarps], warpB[kFinishWarps];
+};
+static_assert(sizeof(FinishSmem) % 16 == 0, "the value cache must start 16-byte aligned");
+constexpr size_t kFinishSmemBytes = sizeof(FinishSmem) + (size_t)kFinishCache * sizeof(float);
+
+__global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
+  namespace cg = cooperative_groups;
+  extern __shared__ __align__(16) unsigned char finish_raw[];
+  FinishSmem& sm = *reinterpret_cast<FinishSmem*>(finish_raw);
+  float* cache = reinterpret_cast<float*>(finish_raw + sizeof(FinishSmem));
+  cg::cluster_group cluster = cg::this_cluster();
+  const uint32_t CS = cluster.num_blocks();                    // 1, 2, 4, 8 or 16
+  const uint32_t q = cluster.block_rank();
+  const uint32_t sl = blockIdx.x / CS;
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const Slice S = L.s.slices[sl];
+  SelState* st = &L.s.state[sl];
+  // every early exit below depends on the slice only, so a cluster leaves as a whole
+  if (S.r == S.len) return;
+  const uint32_t n_cand = st->n_cand;
+  if (st->resolved > 31) return;                               // an earlier pass already failed
+  if (n_cand < S.r || n_cand > S.cand_cap) {                   // cannot happen once the exact path ran
+    if (q == 0 && tid == 0) atomicOr(L.s.error, ERR_CANDIDATE_OVERFLOW);
+    return;
+  }
+  uint32_t n_gt = st->n_gt, need = st->need, lo_key, hi_key;
+  bool count_above;
+  if (st->flags & FLAG_GENERAL) {
+    const uint32_t free_bits = 31u - st->resolved;
+    lo_key = st->prefix << free_bits; hi_key = lo_key + (1u << free_bits); count_above = false;
+  } else {
+    lo_key = st->tau_lo; hi_key = st->tau_hi + 1u; count_above = true; n_gt = 0; need = S.r;
+  }
+  const uint32_t* cidx = L.s.cand_idx + S.cand_off;
+  const float* cval = L.s.cand_val + S.cand_off;
+  const uint32_t per = ((n_cand + CS - 1) / CS + 31u) & ~31u;
+  const uint32_t lo = min(n_cand, q * per), hi = min(n_cand, lo + per);
+  const uint32_t n_mine = hi - lo;
+  const uint32_t n_cached = min(n_mine, (uint32_t)kFinishCache);
+
+  // my share of the candidate values -> shared memory (the share starts 128-byte aligned)
+  {
+    const float4* src = reinterpret_cast<const float4*>(cval + lo);
+    float4* dst = reinterpret_cast<float4*>(cache);
+    const uint32_t nv = n_cached >> 2;
+    for (uint32_t base = tid; base < nv; base += kFinishThreads * 4) {
+      float4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) if (base + u * kFinishThreads < nv) v[u] = __ldg(src + base + u * kFinishThreads);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) if (base + u * kFinishThreads < nv) dst[base + u * kFinishThreads] = v[u];
+    }
+    for (uint32_t i = (nv << 2) + tid; i < n_cached; i += kFinishThreads) cache[i] = __ldg(cval + lo + i);
+  }
+  __syncthreads();
+  auto value_at = [&](uint32_t i) -> float { return i < n_cached ? cache[i] : __ldg(cval + lo + i); };
+  // visits every key of my share once (order is irrelevant to the callers)
+  auto for_each_key = [&](auto&& f) {
+    const float4* c4 = reinterpret_cast<const float4*>(cache);
+    const uint32_t nv = n_cached >> 2;
+    for (uint32_t t = tid; t < nv; t += kFinishThreads) {
+      const float4 v = c4[t];
+      f(mag_key(v.x)); f(mag_key(v.y)); f(mag_key(v.z)); f(mag_key(v.w));
+    }
+    for (uint32_t i = (nv << 2) + tid; i < n_cached; i += kFinishThreads) f(mag_key(cache[i]));
+    for (uint32_t base = n_cached + tid; base < n_mine; base += kFinishThreads * kFinishBatch) {
+      float v[kFinishBatch];
+#pragma unroll
+      for (int u = 0; u < kFinishBatch; ++u) {
+        const uint32_t i = base + u * kFinishThreads;
+        v[u] = i < n_mine ? __ldg(cval + lo + i) : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < kFinishBatch; ++u)
+        if (base + u * kFinishThreads < n_mine) f(mag_key(v[u]));
+    }
+  };
+
+  for (int round = 0; (hi_key - lo_key > 1u || count_above) && round < 8; ++round) {
+    const uint32_t width = hi_key - lo_key;                    // >= 1
+    uint32_t sh = 0;
+    while (((width - 1u) >> sh) >= (uint32_t)(kBins - 1)) ++sh;
+    for (uint32_t b = tid; b < (uint32_t)kBins; b += kFinishThreads) sm.hist[b] = 0;
+    __syncthreads();
+    uint32_t n_above = 0;                                      // keys above the interval: counted in registers
+    for_each_key([&](uint32_t key) {
+      if (key >= hi_key) ++n_above;
+      else if (key >= lo_key) atomicAdd(&sm.hist[(key - lo_key) >> sh], 1u);
+    });
+    if (count_above) {
+      n_above = warp_sum(n_above);
+      if (lane == 0 && n_above) atomicAdd(&sm.hist[kBins - 1], n_above);
+    }
+    cluster.sync();
+    // every CTA sums the cluster's histograms for itself (independent remote loads, one latency)
+    // and picks the bucket redundantly: no broadcast, no serial section in one CTA
+    for (uint32_t b = tid; b < (uint32_t)kBins; b += kFinishThreads) {
+      uint32_t part[kMaxCluster];
+#pragma unroll
+      for (int rr = 0; rr < kMaxCluster; ++rr)
+        part[rr] = (uint32_t)rr < CS ? cluster.map_shared_rank(sm.hist, rr)[b] : 0u;
+      uint32_t sum = 0;
+#pragma unroll
+      for (int rr = 0; rr < kMaxCluster; ++rr) sum += part[rr];
+      sm.red[b] = sum;
+    }
+    __syncthreads();
+    uint32_t D, above;
+    pick_digit(sm.red, kBins, need, sm.scratch, D, above);
+    cluster.sync();                                            // all remote reads of sm.hist are done
+    if (D == 0xFFFFFFFFu) {                                    // fewer keys than the rank asked for
+      if (q == 0 && tid == 0) { atomicOr(L.s.error, ERR_SELECT_INCONSISTENT); st->resolved = 32; }
+      return;
+    }
+    if (D == (uint32_t)(kBins - 1)) {
+      // only possible while the keys above the interval were being counted: the sampled upper
+      // estimate was too low and the target lies above it
+      lo_key = hi_key; hi_key = 0x80000000u;
+    } else {
+      n_gt += above; need -= above;
+      lo_key += D << sh;
+      hi_key = min(hi_key, lo_key + (1u << sh));
+    }
+    count_above = false;
+  }
+  if (hi_key - lo_key != 1u) {                                 // did not converge (cannot happen: <= 5 rounds)
+    if (q == 0 && tid == 0) { atomicOr(L.s.error, ERR_SELECT_INCONSISTENT); st->resolved = 32; }
+    return;
+  }
+  const uint32_t tau = lo_key, quota = need;
+  if (q == 0 && tid == 0) { st->prefix = tau; st->resolved = 31; st->n_gt = n_gt; st->need = need; }
+
+  // Members of my share (keys above tau, keys equal to tau), per warp: warp w owns the w-th
+  // contiguous part of the share, so that the walk below needs no block-wide barrier.
+  const uint32_t wper = ((n_mine + kFinishWarps - 1) / kFinishWarps + 127u) & ~127u;   // multiple of 128
+  const uint32_t w_lo = min(n_mine, warp * wper), w_hi = min(n_mine, w_lo + wper);
+  auto load4 = [&](uint32_t i, float (&v)[4]) {               // values i..i+3 of my share (i % 4 == 0)
+    if (i + 4u <= n_cached) {
+      const float4 x = *reinterpret_cast<const float4*>(cache + i);
+      v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+    } else if (i >= n_cached && i + 4u <= n_mine) {
+      const float4 x = __ldg(reinterpret_cast<const float4*>(cval + lo + i));
+      v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) v[j] = i + j < n_mine ? value_at(i + j) : 0.f;
+    }
+  };
+  uint32_t cA = 0, cB = 0;
+  for (uint32_t base = w_lo; base < w_hi; base += 128u) {
+    const uint32_t i0 = base + lane * 4u;
+    float v[4];
+    load4(i0, v);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t key = mag_key(v[j]);
+      const bool in = i0 + j < w_hi;
+      cA += in && key > tau; cB += in && key == tau;
+    }
+  }
+  cA = warp_sum(cA); cB = warp_sum(cB);
+  if (lane == 0) { sm.warpA[warp] = cA; sm.warpB[warp] = cB; }
+  __syncthreads();
+  if (tid < CS) {
+    uint32_t tA = 0, tB = 0;
+#pragma unroll
+    for (int w = 0; w < kFinishWarps; ++w) { tA += sm.warpA[w]; tB += sm.warpB[w]; }
+    uint32_t* c = cluster.map_shared_rank(sm.counts, tid);   // my counts, into CTA `tid`
+    c[2 * q] = tA; c[2 * q + 1] = tB;
+  }
+  cluster.sync();                                              // last remote access of the kernel
+  uint32_t gt_before = 0, eq_before = 0;
+  for (uint32_t p = 0; p < q; ++p) { gt_before += sm.counts[2 * p]; eq_before += sm.counts[2 * p + 1]; }
+
+  // the part of the sampler's bitmap that covers my members' positions -> shared memory
+  const uint32_t pos0 = gt_before + min(eq_before, quota);
+  const uint32_t pos1 = min(S.r, pos0 + sm.counts[2 * q] + sm.counts[2 * q + 1]);
+  const uint32_t word0 = pos0 >> 5, nwords = pos1 > pos0 ? ((pos1 + 31u) >> 5) - word0 : 0u;
+  const bool sel_all = S.k == S.r;
+  const bool sel_cached = !sel_all && nwords <= (uint32_t)kFinishSelWords;
+  if (sel_cached)
+    for (uint32_t w = tid; w < nwords; w += kFinishThreads) {
+      sm.sel[w] = L.s.sel[S.sel_off + word0 + w];
+      sm.sel_pre[w] = L.s.sel_pre[S.sel_off + word0 + w];
+    }
+  __syncthreads();
+  auto selected = [&](uint32_t p, uint32_t& slot) -> bool {
+    if (sel_all) { slot = p; return true; }
+    const uint32_t wi = p >> 5;
+    const uint32_t word = sel_cached ? sm.sel[wi - word0] : L.s.sel[S.sel_off + wi];
+    if (!((word >> (p & 31u)) & 1u)) return false;
+    const uint32_t pre = sel_cached ? sm.sel_pre[wi - word0] : L.s.sel_pre[S.sel_off + wi];
+    slot = pre + __popc(word & ((1u << (p & 31u)) - 1u));
+    return true;
+  };
+
+  // walk my warp's part in index order: 4 consecutive candidates per lane, 128 per step
+  for (uint32_t w = 0; w < warp; ++w) { gt_before += sm.warpA[w]; eq_before += sm.warpB[w]; }
+  for (uint32_t base = w_lo; base < w_hi; base += 128u) {
+    const uint32_t i0 = base + lane * 4u;
+    float v[4];
+    load4(i0, v);
+    uint32_t mA = 0, mB = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t key = mag_key(v[j]);
+      const bool in = i0 + j < w_hi;
+      mA |= (uint32_t)(in && key > tau) << j;
+      mB |= (uint32_t)(in && key == tau) << j;
+    }
+    const uint32_t pack = (uint32_t)__popc(mA) | ((uint32_t)__popc(mB) << 16);   // <= 128 each per warp
+    const uint32_t incl = warp_incl_scan(pack);
+    const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    const uint32_t excl = incl - pack;
+    uint32_t g = gt_before + (excl & 0xFFFFu), e = eq_before + (excl >> 16);
+    if (mA | mB) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const bool isA = (mA >> j) & 1u, isB = (mB >> j) & 1u;
+        if (isA || (isB && e < quota)) {
+          const uint32_t p = g + min(e, quota);
+          uint32_t slot;
+          if (p < S.r && selected(p, slot) && slot < S.k) {
+            const uint32_t idx = cidx[lo + i0 + j];
+            L.msg_idx[S.msg_off + slot] = S.idx_base + idx;
+            L.msg_val[S.msg_off + slot] = v[j];
+            L.residual[S.m_off + idx] = 0.0f;
+          }
+        }
+        g += isA; e += isB;
+      }
+    }
+    gt_before += tot & 0xFFFFu; eq_before += tot >> 16;
   }
 }
 

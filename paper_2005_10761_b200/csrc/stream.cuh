@@ -27,7 +27,7 @@ constexpr int kWaitLimit = 1 << 24;
 struct StageDesc { uint32_t slice, chunk, valid, pad; };
 
 template <typename GradT>
-struct StreamSmem {
+struct alignas(128) StreamSmem {
   alignas(128) float m[kStages][kChunk];
   alignas(128) GradT g[kStages][kChunk];
   alignas(8) unsigned long long full[kStages];
@@ -274,8 +274,10 @@ __global__ void __launch_bounds__(kOrderThreads) k_cand_scan(Launch L) {
   }
   if (tid == 0) {
     SelState* st = &L.s.state[blockIdx.x];
-    st->n_cand = s_carry;
-    st->n_cand_first = s_carry;
+    const uint32_t total = s_carry;
+    st->n_cand = total;
+    st->n_cand_first = total;
+    if (total < S.r || total > S.cand_cap) atomicAdd(&L.s.tickets[3], 1u);   // wakes the exact path
   }
 }
 

@@ -232,6 +232,30 @@ def test_aggregate_against_oracle(lib, W, d, k):
     ctx.close()
 
 
+def test_aggregate_sparse_path_many_workers_and_crowded_tiles(lib):
+    rng = np.random.default_rng(99)
+    cases = []
+    d, W, k = 2_000_003, 300, 500                      # more workers than one block batch
+    cases.append((d, np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)])))
+    d, W, k = 1_000_000, 8, 2000                       # every entry inside the first output tiles
+    cases.append((d, np.stack([np.sort(rng.choice(6000, k, replace=False)) for _ in range(W)])))
+    d, W, k = 3_000_000, 16, 3000                      # identical supports: every coordinate shared by all
+    same = np.sort(rng.choice(d, k, replace=False))
+    cases.append((d, np.stack([same] * W)))
+    for d, idx in cases:
+        idx = idx.astype(np.uint32)
+        W, k = idx.shape
+        val = (rng.standard_normal((W, k)) * np.exp(2 * rng.standard_normal((W, k)))).astype(np.float32)
+        ctx = _ctx(lib, d, W, k, k)
+        out = torch.full((wl.round_up(d, 4),), float("nan"), dtype=torch.float32, device="cuda")
+        ctx.aggregate(torch.from_numpy(idx.view(np.int32)).cuda(), torch.from_numpy(val).cuda(), d, out)
+        o64, o32 = oracle.aggregate(idx, val, d)
+        got = out.cpu().numpy()[:d]
+        assert np.abs(got.astype(np.float64) - o64).max() <= 1e-6 * float(np.abs(val).max())
+        assert np.array_equal(_bits(got), _bits(o32))
+        ctx.close()
+
+
 def test_step_is_sparsify_then_aggregate(lib):
     cfg = wl.configs()["c1"]
     ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
