@@ -38,11 +38,20 @@ def gather_messages(idx_local: torch.Tensor, val_local: torch.Tensor, W_total: i
         dist.all_gather_into_tensor(idx_all, idx_local.contiguous(), group=group)
         dist.all_gather_into_tensor(val_all, val_local.contiguous(), group=group)
         return idx_all, val_all
-    idx_parts = [torch.empty((c, k), dtype=idx_local.dtype, device=idx_local.device) for c in counts]
-    val_parts = [torch.empty((c, k), dtype=val_local.dtype, device=val_local.device) for c in counts]
-    dist.all_gather(idx_parts, idx_local.contiguous(), group=group)
-    dist.all_gather(val_parts, val_local.contiguous(), group=group)
-    return torch.cat(idx_parts), torch.cat(val_parts)
+    # uneven shards: pad every block to the largest shard, gather, then drop the padding rows
+    cmax = max(counts)
+
+    def padded(x):
+        buf = torch.zeros((cmax, k), dtype=x.dtype, device=x.device)
+        buf[: x.shape[0]] = x
+        return buf
+
+    idx_pad = torch.empty((world * cmax, k), dtype=idx_local.dtype, device=idx_local.device)
+    val_pad = torch.empty((world * cmax, k), dtype=val_local.dtype, device=val_local.device)
+    dist.all_gather_into_tensor(idx_pad, padded(idx_local), group=group)
+    dist.all_gather_into_tensor(val_pad, padded(val_local), group=group)
+    keep = torch.cat([torch.arange(r * cmax, r * cmax + c, device=idx_local.device) for r, c in enumerate(counts)])
+    return idx_pad.index_select(0, keep), val_pad.index_select(0, keep)
 
 
 def sharded_round(sparsify: Callable, aggregate: Callable, grad_local: torch.Tensor,
