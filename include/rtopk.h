@@ -179,6 +179,38 @@ int rtopk_step_host(rtopk_ctx* ctx, const void* h_grad, int grad_dtype, int64_t 
 int rtopk_sample_positions(rtopk_ctx* ctx, int64_t r, int64_t k, uint64_t seed, uint32_t step,
                            uint32_t worker, uint32_t segment, uint32_t* pos, void* stream);
 
+/*
+ * rtopk_sample_positions without a context and without any allocation.  (The paper has no
+ * counterpart: this exists for the sake of callers, not of the method.)
+ *
+ * Who needs it: code that must not call cudaMalloc / cudaFree while it runs -- a training process
+ * whose framework has already claimed the device memory for its own caching allocator, so that a
+ * late cudaMalloc may fail or fragment it; a latency-critical loop with other streams in flight,
+ * where the device-wide synchronisation hidden in cudaMalloc / cudaFree stalls everything; a host
+ * program whose rules forbid allocation after start-up.  rtopk_create allocates its scratch, so
+ * such callers cannot use a context; this call needs none.
+ *
+ * Its scratch (draw buffer, first-occurrence table, position bitmap and prefix: about 8.7 MB) is a
+ * fixed array inside the library's device image.  Every GPU that loads the library holds that
+ * array until the process exits, whether or not this call is ever made.
+ *
+ *   r, k      1 <= k <= r <= RTOPK_STATIC_MAX_R; a larger r returns RTOPK_ERR_UNSUPPORTED and
+ *             nothing is enqueued (use a context for larger sets).
+ *   pos [out] device, k entries: the chosen positions, ascending; same values as
+ *             rtopk_sample_positions for the same (r, k, seed, step, worker, segment).
+ * Works on the current device.  The first call on a device looks up the array's device address
+ * (once per device); make that first call outside any stream capture.
+ * All calls on a device share the one array, which still holds the previous call's contents: the
+ * parts that must start clean are cleared at the start of every call, in stream order.  Two calls
+ * whose work overlaps on the GPU (different streams, no ordering between them) race on the array
+ * and give undefined positions; order them.
+ * Calls no cudaMalloc, cudaFree or other allocating routine.
+ * Errors: INVALID_ARG (null pos, k < 1, k > r), UNSUPPORTED (r too large), CUDA.
+ */
+#define RTOPK_STATIC_MAX_R (1 << 20)
+int rtopk_sample_positions_static(int64_t r, int64_t k, uint64_t seed, uint32_t step, uint32_t worker,
+                                  uint32_t segment, uint32_t* pos, void* stream);
+
 /* Waits for `stream` and returns RTOPK_ERR_INTERNAL if any kernel of this context has raised the
  * device-side error flag since the last poll (the flag is then cleared), else RTOPK_OK. */
 int rtopk_poll_status(rtopk_ctx* ctx, void* stream);

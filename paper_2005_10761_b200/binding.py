@@ -42,6 +42,7 @@ EXPORTS = {
     "rtopk_step_host": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _i64, _u64, _u32,
                                _int, _vp, _vp, _vp, _vp]),
     "rtopk_sample_positions": (_int, [_vp, _i64, _i64, _u64, _u32, _u32, _u32, _vp, _vp]),
+    "rtopk_sample_positions_static": (_int, [_i64, _i64, _u64, _u32, _u32, _u32, _vp, _vp]),
     "rtopk_poll_status": (_int, [_vp, _vp]),
     "rtopk_get_phase_times": (_int, [_vp, _vp, _vp]),
     "rtopk_get_stats": (_int, [_vp, _i32, _vp, _vp]),
@@ -74,6 +75,19 @@ def load_library() -> C.CDLL:
             fn.argtypes = args
         _lib = lib
     return _lib
+
+
+STATIC_MAX_R = 1 << 20
+
+
+def sample_positions_static(r: int, k: int, seed: int, step: int, worker: int, segment: int, pos) -> None:
+    """rtopk_sample_positions_static: the k-of-r positions without a context and without any device
+    allocation, for callers that must not allocate (see include/rtopk.h).  ``pos`` is a device tensor
+    of k 32-bit entries on the current device.  Raises RTopKError (status 4) if r > STATIC_MAX_R."""
+    lib = load_library()
+    rc = lib.rtopk_sample_positions_static(r, k, seed, step, worker, segment, pos.data_ptr(), _stream())
+    if rc != 0:
+        raise RTopKError(rc, "rtopk_sample_positions_static", lib.rtopk_status_string(rc).decode())
 
 
 class Stats(C.Structure):

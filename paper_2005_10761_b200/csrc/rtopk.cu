@@ -9,6 +9,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -700,6 +701,82 @@ int rtopk_get_stats(rtopk_ctx* ctx, int32_t slice, rtopk_stats* out, void* strea
   out->n_candidates = s.n_cand;
   out->used_fallback = (s.flags & FLAG_FELL_BACK) ? 1u : 0u;
   return RTOPK_OK;
+}
+
+// ----------------------------------------------------------------------------- no-allocation call
+// Scratch of rtopk_sample_positions_static: one slice descriptor, then the draw buffer, the
+// first-occurrence table, the position bitmap and its prefix, each sized for RTOPK_STATIC_MAX_R.
+// The array lives in the device image; its name below is only a host-side handle, the device
+// address comes from cudaGetSymbolAddress (once per device).
+namespace {
+constexpr size_t kStaticR = (size_t)RTOPK_STATIC_MAX_R;
+constexpr size_t kStaticSliceBytes = 256;
+constexpr size_t kStaticDrawsOff = kStaticSliceBytes;
+constexpr size_t kStaticFirstOff = kStaticDrawsOff + kStaticR * 4;
+constexpr size_t kStaticSelOff = kStaticFirstOff + kStaticR * 4;
+constexpr size_t kStaticPreOff = kStaticSelOff + (kStaticR / 32 + 8) * 4;
+constexpr size_t kStaticBytes = kStaticPreOff + (kStaticR / 32 + 8) * 4;
+static_assert(sizeof(Slice) <= kStaticSliceBytes, "slice descriptor must fit its slot");
+}  // namespace
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+namespace {
+constexpr int kStaticMaxDevices = 64;
+std::mutex g_static_mutex;
+unsigned char* g_static_ptr[kStaticMaxDevices] = {};
+
+// Writes the one-slice table the subset kernels read (no host-to-device copy needed).
+__global__ void k_static_slice(Slice* slot, uint32_t r, uint32_t k, uint32_t segment) {
+  if (blockIdx.x != 0 || threadIdx.x != 0) return;
+  Slice s;
+  s.g_off = 0; s.m_off = 0; s.len = r; s.r = r; s.k = k; s.row = 0; s.segment = segment; s.idx_base = 0;
+  s.head = 0; s.msg_off = 0; s.cand_off = 0; s.cand_cap = 0; s.chunk_begin = 0; s.hist_begin = 0;
+  s.ctile_begin = 0; s.samp_off = 0; s.first_off = 0; s.sel_off = 0; s.pad = 0;
+  *slot = s;
+}
+}  // namespace
+
+int rtopk_sample_positions_static(int64_t r, int64_t k, uint64_t seed, uint32_t step, uint32_t worker,
+                                  uint32_t segment, uint32_t* pos, void* stream) {
+  if (!pos || k < 1 || k > r) return RTOPK_ERR_INVALID_ARG;
+  if (r > (int64_t)RTOPK_STATIC_MAX_R) return RTOPK_ERR_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return RTOPK_ERR_CUDA;
+  unsigned char* base = nullptr;
+  {
+    // set-up, once per device, with that device current: the symbol's device address
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+      void* p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return RTOPK_ERR_CUDA; }
+      g_static_ptr[dev] = static_cast<unsigned char*>(p);
+    }
+    base = g_static_ptr[dev];
+  }
+  Launch L;
+  std::memset(&L, 0, sizeof(L));
+  L.s.slices = reinterpret_cast<Slice*>(base);
+  L.s.draws = reinterpret_cast<uint32_t*>(base + kStaticDrawsOff);
+  L.s.first = reinterpret_cast<uint32_t*>(base + kStaticFirstOff);
+  L.s.sel = reinterpret_cast<uint32_t*>(base + kStaticSelOff);
+  L.s.sel_pre = reinterpret_cast<uint32_t*>(base + kStaticPreOff);
+  L.n_slices = 1; L.worker_base = worker; L.seed_lo = (uint32_t)seed; L.seed_hi = (uint32_t)(seed >> 32);
+  L.step = step;
+  const uint32_t nwords = (uint32_t)((r + 31) / 32);
+  k_static_slice<<<1, 32, 0, st>>>(L.s.slices, (uint32_t)r, (uint32_t)k, segment);
+  if (k < r) {
+    // the array keeps the previous call's contents: the table starts at "never drawn", the bitmap at zero
+    if (cudaMemsetAsync(L.s.first, 0xFF, (size_t)r * sizeof(uint32_t), st) != cudaSuccess) return RTOPK_ERR_CUDA;
+    if (cudaMemsetAsync(L.s.sel, 0, (size_t)nwords * sizeof(uint32_t), st) != cudaSuccess) return RTOPK_ERR_CUDA;
+    const dim3 grid(((uint32_t)k + kDrawThreads - 1) / kDrawThreads, 1);
+    k_draw<<<grid, kDrawThreads, 0, st>>>(L);
+    k_resolve<<<grid, kDrawThreads, 0, st>>>(L);
+    k_sel_scan<<<1, kScanThreads, 0, st>>>(L);
+  }
+  k_positions<<<(nwords + kThreads - 1) / kThreads, kThreads, 0, st>>>(L, pos);
+  return cudaGetLastError() == cudaSuccess ? RTOPK_OK : RTOPK_ERR_CUDA;
 }
 
 }  // extern "C"
