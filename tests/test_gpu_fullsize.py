@@ -1,0 +1,176 @@
+"""Parity at the full sizes of the named configurations, in the launch configuration bench.py times
+(rtopk_step / rtopk_step_segmented on all W rows).
+
+The oracle's full sort is too slow for every row at these sizes, so per configuration
+  * a sample of worker rows is followed through the steps by the oracle and compared bit for bit
+    (indices, values, residual row);
+  * every row is checked on the GPU against properties that hold at any size: exactly k strictly
+    ascending in-range indices, values are a bit copy of a = g + m at those indices, sent + residual
+    reassembles a exactly, sent slots hold +0, every sent key is at least the reported threshold and
+    the number of keys above the threshold matches the reported count;
+  * the dense update is compared with the oracle's aggregate of the very messages the GPU produced
+    (all W rows), bit for bit, which also meets the 1e-6 * max|g| bar.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2005_10761_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def lib():
+    import paper_2005_10761_b200 as pkg
+    from paper_2005_10761_b200 import build
+    build.build()
+    oracle.set_threads(8)
+    return pkg
+
+
+def _bits(t: torch.Tensor) -> torch.Tensor:
+    return t.view(torch.int32)
+
+
+def _host_grad(cfg, g_rows: torch.Tensor) -> np.ndarray:
+    if cfg.grad_dtype == "bf16":
+        return g_rows.cpu().view(torch.int16).numpy().view(np.uint16).copy()
+    return g_rows.cpu().numpy().copy()
+
+
+def _check_rows_on_gpu(cfg, ctx, g, m_prev, m_new, idx, val, seg):
+    """Size-independent properties, all W rows, computed with torch on the device."""
+    d = cfg.d
+    S = len(cfg.seg_r) if seg else 1
+    for w in range(cfg.W):
+        a = g[w, :d].to(torch.float32) + m_prev[w, :d]
+        i = idx[w].to(torch.int64)
+        assert bool((i[1:] > i[:-1]).all()) and int(i[0]) >= 0 and int(i[-1]) < d
+        assert torch.equal(_bits(val[w]), _bits(a[i]))
+        assert bool((_bits(m_new[w, :d][i]) == 0).all())
+        back = m_new[w, :d].clone()
+        back[i] = val[w]
+        assert torch.equal(_bits(back), _bits(a))
+        key = _bits(a) & 0x7FFFFFFF
+        at = 0
+        for s in range(S):
+            st = ctx.stats(w * S + s)
+            lo, hi = (cfg.seg_off[s], cfg.seg_off[s + 1]) if seg else (0, d)
+            r_s, k_s = (cfg.seg_r[s], cfg.seg_k[s]) if seg else (cfg.r, cfg.k)
+            if r_s < hi - lo:
+                ks = key[lo:hi]
+                n_gt = int((ks > st["tau_key"]).sum())
+                n_eq = int((ks == st["tau_key"]).sum())
+                assert n_gt == st["n_greater"] and n_gt < r_s <= n_gt + n_eq      # tau is the r-th largest
+                assert st["tie_quota"] == r_s - n_gt
+                sent = key[i[at:at + k_s]]
+                assert bool((sent >= st["tau_key"]).all())                        # U is inside the top-r set
+            at += k_s
+
+
+def _run_config(lib, cfg, steps, sample_rows, path=0):
+    seg = cfg.seg_off is not None
+    K = cfg.k_total
+    ctx = lib.RTopK(d_max=cfg.d, W_max=cfg.W, r_max=cfg.r, k_max=K, segments_max=len(cfg.seg_r) if seg else 1)
+    ctx.set_option(0, path)
+    m = wl.zero_residual(cfg, "cuda")
+    idx = torch.zeros((cfg.W, K), dtype=torch.int32, device="cuda")
+    val = torch.zeros((cfg.W, K), dtype=torch.float32, device="cuda")
+    out = torch.empty(wl.round_up(cfg.d, 4), dtype=torch.float32, device="cuda")
+    m_or = np.zeros((len(sample_rows), cfg.ld), dtype=np.float32)
+    for t in range(steps):
+        g = wl.gradient(cfg, t, "cuda")
+        m_prev = m.clone()
+        if seg:
+            ctx.step_segmented(g, m, cfg.d, cfg.seg_off, cfg.seg_r, cfg.seg_k, cfg.seed, t, idx, val, out)
+        else:
+            ctx.step(g, m, cfg.d, cfg.r, cfg.k, cfg.seed, t, idx, val, out)
+        ctx.poll_status()
+        _check_rows_on_gpu(cfg, ctx, g, m_prev, m, idx, val, seg)
+        del m_prev
+        # sampled rows against the oracle (each row is an independent worker: worker_base = its id)
+        idx_h, val_h = idx.cpu().numpy().view(np.uint32), val.cpu().numpy()
+        for n, w in enumerate(sample_rows):
+            g_h = _host_grad(cfg, g[w:w + 1])
+            if seg:
+                o_idx, o_val = oracle.sparsify_segmented(g_h, m_or[n:n + 1], cfg.d, cfg.seg_off, cfg.seg_r, cfg.seg_k,
+                                                         cfg.seed, t, worker_base=w)
+            else:
+                o_idx, o_val = oracle.sparsify(g_h, m_or[n:n + 1], cfg.d, cfg.r, cfg.k, cfg.seed, t, worker_base=w)
+            assert np.array_equal(idx_h[w], o_idx[0]), f"{cfg.name} step {t} worker {w}: indices"
+            assert np.array_equal(val_h[w].view(np.uint32), o_val[0].view(np.uint32)), f"{cfg.name} step {t} worker {w}: values"
+            assert np.array_equal(m[w].cpu().numpy().view(np.uint32), m_or[n].view(np.uint32)), f"{cfg.name} step {t} worker {w}: residual"
+        # the update against the oracle's aggregate of the GPU's own messages
+        o64, o32 = oracle.aggregate(idx_h, val_h, cfg.d)
+        got = out.cpu().numpy()[: cfg.d]
+        gmax = float(g.to(torch.float32).abs().max())
+        assert np.abs(got.astype(np.float64) - o64).max() <= 1e-6 * gmax
+        assert np.array_equal(got.view(np.uint32), o32.view(np.uint32))
+        del g
+    fallbacks = sum(ctx.stats(s)["used_fallback"] for s in range(cfg.W * (len(cfg.seg_r) if seg else 1)))
+    ctx.close()
+    return fallbacks
+
+
+def test_c1_every_row(lib):
+    cfg = wl.configs()["c1"]
+    _run_config(lib, cfg, 1, list(range(cfg.W)))
+
+
+def test_c2_three_steps_with_carried_residual(lib):
+    assert _run_config(lib, wl.configs()["c2"], 3, [0, 5]) == 0       # the sampled bracket holds on this data
+
+
+def test_c2_paper_setting_five_nodes(lib):
+    _run_config(lib, wl.configs()["c2_n5"], 1, [4])
+
+
+def test_c2_exact_path_full_size(lib):
+    _run_config(lib, wl.configs()["c2"], 1, [7], path=1)
+
+
+@pytest.mark.parametrize("name", ["c3_f32", "c3_bf16"])
+def test_c3_two_steps(lib, name):
+    _run_config(lib, wl.configs()[name], 2, [3])
+
+
+def test_c4_per_tensor_lstm_shapes(lib):
+    _run_config(lib, wl.configs()["c4"], 1, [6])
+
+
+def test_c5_quarter_billion_coordinates(lib):
+    cfg = wl.configs()["c5_W4_r100_k10"]
+    free, _ = torch.cuda.mem_get_info()
+    if free < 24e9:
+        pytest.skip("not enough free device memory on this (shared) GPU")
+    _run_config(lib, cfg, 1, [2])
+
+
+def test_c5_limits_topk_and_randomk(lib):
+    free, _ = torch.cuda.mem_get_info()
+    if free < 16e9:
+        pytest.skip("not enough free device memory on this (shared) GPU")
+    # k = r (Definition 1): every member of the top-r set is sent -- properties on the device
+    _run_config(lib, wl.configs()["c5_W1_topk"], 1, [])
+    # r = d (Definition 2): the subset does not depend on the values; positions are indices
+    cfg = wl.configs()["c5_W1_randk"]
+    ctx = lib.RTopK(d_max=cfg.d, W_max=1, r_max=cfg.r, k_max=cfg.k)
+    g = wl.gradient(cfg, 0, "cuda")
+    m = wl.zero_residual(cfg, "cuda")
+    idx = torch.zeros((1, cfg.k), dtype=torch.int32, device="cuda")
+    val = torch.zeros((1, cfg.k), dtype=torch.float32, device="cuda")
+    out = torch.empty(cfg.d, dtype=torch.float32, device="cuda")
+    ctx.step(g, m, cfg.d, cfg.r, cfg.k, cfg.seed, 0, idx, val, out)
+    ctx.poll_status()
+    want = oracle.sample_positions(cfg.d, cfg.k, cfg.seed, 0, 0)
+    assert np.array_equal(idx.cpu().numpy().view(np.uint32)[0], want)
+    i = idx[0].to(torch.int64)
+    assert torch.equal(_bits(val[0]), _bits(g[0, : cfg.d][i]))
+    back = m[0, : cfg.d].clone()
+    back[i] = val[0]
+    assert torch.equal(_bits(back), _bits(g[0, : cfg.d]))
+    assert torch.equal(_bits(out[i]), _bits(val[0]))                  # W = 1: the update is the message
+    assert int((out != 0).sum()) <= cfg.k
+    ctx.close()
