@@ -55,7 +55,7 @@ def recorded_traffic(workload: str, launch_bytes: float):
     """DRAM bytes per launch of the streaming kernel from the committed ncu summary, scaled by the
     algorithmic bytes when the capture was taken on a smaller case; None if there is no summary or
     the kernel sources changed since."""
-    path = os.path.join(ROOT, "profiles", "k_collect_traffic.txt")
+    path = os.path.join(ROOT, "profiles", "k_stream_traffic.txt")
     try:
         kv = {}
         with open(path) as f:
@@ -320,7 +320,7 @@ def main():
     stream_bytes = W * d * (gsz + 8)
     stream_ms = phases.get("stream")
     achieved = stream_bytes / (stream_ms * 1e-3) / 1e9 if stream_ms else None
-    roofline = {"bound": "hbm", "kernel": "k_collect (fused add + write-back + candidate gather)",
+    roofline = {"bound": "hbm", "kernel": "k_stream (fused add + write-back + candidate gather)",
                 "achieved": achieved, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None,
                 "traffic": recorded_traffic(cfg.name, stream_bytes),

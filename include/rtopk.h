@@ -69,13 +69,13 @@ enum {
 /* Phases of one call, in stream order.  STREAM is the single pass over the full vectors that
  * performs a = g + m, writes it back and gathers the coordinates above the threshold. */
 enum {
-  RTOPK_PHASE_SUBSET = 0,    /* scratch clearing + the k-of-r subset (Definition 3's U, as positions) */
-  RTOPK_PHASE_THRESHOLD = 1, /* sampled threshold estimate */
-  RTOPK_PHASE_STREAM = 2,    /* fused add / write-back / candidate gathering over W x d elements */
-  RTOPK_PHASE_EXACT = 3,     /* full-vector radix passes (fallback; near-empty launches otherwise) */
-  RTOPK_PHASE_SELECT = 4,    /* exact r-th largest among the candidates */
-  RTOPK_PHASE_EMIT = 5,      /* messages + residual zeroing (m' = a - ghat) */
-  RTOPK_PHASE_AGGREGATE = 6, /* master average (rtopk_step only) */
+  RTOPK_PHASE_SUBSET = 0,    /* scratch clearing; the k-of-r subset itself runs beside the stream pass */
+  RTOPK_PHASE_THRESHOLD = 1, /* sampled bracket of the r-th largest magnitude */
+  RTOPK_PHASE_STREAM = 2,    /* the one kernel over W x d elements: add, write-back, candidate gathering */
+  RTOPK_PHASE_ORDER = 3,     /* candidate runs laid out in index order; count check */
+  RTOPK_PHASE_EXACT = 4,     /* full-vector radix passes (fallback; near-empty launches otherwise) */
+  RTOPK_PHASE_FINISH = 5,    /* exact threshold among the candidates, messages, residual zeroing */
+  RTOPK_PHASE_AGGREGATE = 6, /* master average (step calls only) */
   RTOPK_N_PHASES = 7
 };
 

@@ -16,7 +16,7 @@ _LIB_PATH = os.path.join(_HERE, "librtopk.so")
 GRAD_F32, GRAD_BF16 = 0, 1
 SCALE_MEAN, SCALE_SUM = 0, 1
 OPT_SELECT_PATH, OPT_PROFILE = 0, 1
-PHASES = ("subset", "threshold", "stream", "exact", "select", "emit", "aggregate")
+PHASES = ("subset", "threshold", "stream", "order", "exact", "finish", "aggregate")
 
 _vp, _i32, _i64, _u32, _u64, _int = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_uint64, C.c_int
 

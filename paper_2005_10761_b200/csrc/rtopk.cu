@@ -107,7 +107,7 @@ struct Plan {
   std::vector<Slice> slices;
   uint32_t n_chunks = 0, n_hist_blocks = 0, n_ctiles = 0;
   size_t cand_entries = 0, draw_entries = 0, first_entries = 0, sel_words = 0;
-  uint32_t k_draw_max = 0, words_all_max = 0;
+  uint32_t k_draw_max = 0, words_all_max = 0, cap_max = 0, chunks_max = 0;
   bool any_select = false, any_sampler = false, any_all = false;
   bool uniform = false;               // every slice has the same number of chunks (plain calls)
   uint32_t K_row = 0;
@@ -150,12 +150,14 @@ int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32
       sl.chunk_begin = (uint32_t)chunks;
       sl.hist_begin = (uint32_t)hblocks;
       chunks += nchunks;
+      if (nchunks > P.chunks_max) P.chunks_max = nchunks;
       hblocks += (nchunks + kHistChunks - 1) / kHistChunks;
       sl.ctile_begin = (uint32_t)ctiles;
       sl.cand_off = (uint32_t)cand;
       if (sl.r < sl.len) {
         sl.cand_cap = cand_capacity(sl.len, sl.r);
         cand += sl.cand_cap;
+        if (sl.cand_cap > P.cap_max) P.cap_max = sl.cand_cap;
         ctiles += (sl.cand_cap + kCandTile - 1) / kCandTile;
         P.any_select = true;
       } else {
@@ -232,6 +234,7 @@ int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t s
       const uint32_t uniform = P.uniform ? per : 0u;
       const int blocks = ctx->stream_blocks[sizeof(GradT) == 4 ? 0 : 1];
       k_stream<GradT><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
+      mark(ctx, RTOPK_PHASE_ORDER, st);
       if (P.any_select) {
         k_cand_scan<<<n, kOrderThreads, 0, st>>>(L);
         k_cand_gather<<<(P.n_chunks + kWarps - 1) / kWarps, kThreads, 0, st>>>(L, P.n_chunks, uniform);
@@ -251,6 +254,7 @@ int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t s
     const uint32_t hgrid = std::min<uint32_t>(P.n_hist_blocks, (uint32_t)ctx->sms * 8u);
     const uint32_t cgrid = std::min<uint32_t>(P.n_chunks, (uint32_t)ctx->sms * 4u);
     k_hist<GradT, true><<<hgrid, kThreads, 0, st>>>(L, 0, P.n_hist_blocks);
+    mark(ctx, RTOPK_PHASE_ORDER, st);
     mark(ctx, RTOPK_PHASE_EXACT, st);
     if (P.any_select) {
       for (int pass = 1; pass < 3; ++pass) k_hist<float, false><<<hgrid, kThreads, 0, st>>>(L, pass, P.n_hist_blocks);
@@ -335,7 +339,7 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   rc = grad_dtype == RTOPK_F32 ? launch_select<float>(ctx, P, L, st) : launch_select<__nv_bfloat16>(ctx, P, L, st);
   if (rc) return rc;
   if (forked) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0));
-  mark(ctx, RTOPK_PHASE_SELECT, st);
+  mark(ctx, RTOPK_PHASE_FINISH, st);
   if (P.any_select) {
     // the largest cluster size that still lets every slice's cluster be resident at once
     int cs = 1;
@@ -352,7 +356,6 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
     cfg.attrs = attr; cfg.numAttrs = 1;
     RTOPK_CUDA(ctx, cudaLaunchKernelEx(&cfg, k_finish, L));
   }
-  mark(ctx, RTOPK_PHASE_EMIT, st);
   if (P.any_all) {
     const dim3 grid((P.words_all_max + kThreads - 1) / kThreads, L.n_slices);
     k_emit_all<<<grid, kThreads, 0, st>>>(L, P.words_all_max);

@@ -108,20 +108,27 @@ __global__ void k_init_state(Launch L, uint32_t general) {
 // k_finish one more round, so the estimates affect speed, never the result.
 //
 // Both sample ranks are small (about 1.4 % of the sample), so the bulk is never histogrammed: every
-// thread keeps only the maximum of its 32 keys, and the rho-th largest of the 1024 maxima is a lower
-// bound of the rho-th largest key (there are at least rho keys that large).  tau_lo is that bound at
+// thread keeps only the maximum of each group of 4 sampled keys, and the rho-th largest of these
+// 8192 maxima is a lower bound of the rho-th largest key (there are at least rho keys that large;
+// with groups this small the bound is within a few per cent of the exact sample rank).  tau_lo is that bound at
 // rank expect + 6 sigma; tau_hi the same at rank (expect - 6 sigma) * 3/4, which as a sample rank
 // stays clearly above the r-th largest.  Samples whose ranks exceed the thread count take a radix
 // select over all sample keys instead.
-__device__ __forceinline__ uint32_t block_select_desc(uint32_t key, bool has, uint32_t rank, uint32_t* hist,
-                                                      uint32_t* scratch) {
-  // rank-th largest (1-based) of one key per thread; three radix passes of one increment per thread
+constexpr int kSampleHold = 8;   // maxima a thread keeps (one per 4 sampled keys)
+
+// rank-th largest (1-based) of the held keys of all threads: slot u of thread t is in use iff
+// t + u * blockDim.x < n_held.  Three radix passes of at most kSampleHold increments per thread.
+__device__ __forceinline__ uint32_t block_select_desc(const uint32_t (&key)[kSampleHold], uint32_t n_held,
+                                                      uint32_t rank, uint32_t* hist, uint32_t* scratch) {
   uint32_t prefix = 0, need = rank;
   for (int pass = 0; pass < 3; ++pass) {
     const int bits = digit_bits(pass), shift = digit_shift(pass);
     for (uint32_t b = threadIdx.x; b < (uint32_t)kBins; b += blockDim.x) hist[b] = 0;
     __syncthreads();
-    if (has && (pass == 0 || (key >> (shift + bits)) == prefix)) atomicAdd(&hist[(key >> shift) & ((1u << bits) - 1u)], 1u);
+#pragma unroll
+    for (int u = 0; u < kSampleHold; ++u)
+      if (threadIdx.x + u * blockDim.x < n_held && (pass == 0 || (key[u] >> (shift + bits)) == prefix))
+        atomicAdd(&hist[(key[u] >> shift) & ((1u << bits) - 1u)], 1u);
     __syncthreads();
     uint32_t D, above;
     pick_digit(hist, 1 << bits, need, scratch, D, above);
@@ -149,13 +156,21 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(Launch L) {
     return;
   }
   const float* m = L.residual;
-  uint32_t n_s, rho_lo, rho_hi, mine = 0;
+  uint32_t n_s, rho_lo, rho_hi, n_held;
+  uint32_t mine[kSampleHold];
+#pragma unroll
+  for (int u = 0; u < kSampleHold; ++u) mine[u] = 0;
   if (S.len <= (uint32_t)kSampleMax) {
     n_s = S.len; rho_lo = S.r; rho_hi = max(1u, S.r - S.r / 4u);   // the sample is the whole slice
-    for (uint32_t i = tid; i < n_s; i += kSampleThreads) {
-      const uint32_t key = mag_key(ef_add(Grad<GradT>::ld1(L.grad, S.g_off + i), m[S.m_off + i]));
-      keys[i] = key;
-      mine = max(mine, key);
+    n_held = min(n_s, (uint32_t)(kSampleHold * kSampleThreads));
+#pragma unroll
+    for (int u = 0; u < kSampleMax / kSampleThreads; ++u) {        // slot u % kSampleHold
+      const uint32_t i = tid + u * kSampleThreads;
+      if (i < n_s) {
+        const uint32_t key = mag_key(ef_add(Grad<GradT>::ld1(L.grad, S.g_off + i), m[S.m_off + i]));
+        keys[i] = key;
+        mine[u % kSampleHold] = max(mine[u % kSampleHold], key);
+      }
     }
   } else {
     const uint32_t v0 = (S.head + 3u) >> 2, v1 = (S.head + S.len) >> 2;   // fully valid vectors
@@ -165,6 +180,8 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(Launch L) {
     const int64_t base_g = S.g_off - S.head, base_m = S.m_off - S.head;
     // all of a thread's sample loads are issued before the first use (one memory latency in total)
     constexpr int kPer = kSampleMax / 4 / kSampleThreads;
+    static_assert(kPer == kSampleHold, "one held maximum per sampled vector");
+    n_held = G * 8u;
     float4 g4[kPer], m4[kPer];
 #pragma unroll
     for (int u = 0; u < kPer; ++u) {
@@ -185,7 +202,7 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(Launch L) {
         const uint32_t k0 = mag_key(ef_add(g4[u].x, m4[u].x)), k1 = mag_key(ef_add(g4[u].y, m4[u].y));
         const uint32_t k2 = mag_key(ef_add(g4[u].z, m4[u].z)), k3 = mag_key(ef_add(g4[u].w, m4[u].w));
         keys[n * 4 + 0] = k0; keys[n * 4 + 1] = k1; keys[n * 4 + 2] = k2; keys[n * 4 + 3] = k3;
-        mine = max(max(mine, max(k0, k1)), max(k2, k3));
+        mine[u] = max(max(k0, k1), max(k2, k3));
       }
     }
     const float expect = (float)n_s * ((float)S.r / (float)S.len);
@@ -194,11 +211,10 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(Launch L) {
     rho_hi = expect - margin < 2.0f ? 1u : (uint32_t)((expect - margin) * 0.75f);
   }
   __syncthreads();
-  const uint32_t n_holders = min(n_s, (uint32_t)kSampleThreads);     // threads that hold at least one key
   uint32_t tau_lo, tau_hi;
-  if (rho_lo <= n_holders) {
-    tau_lo = block_select_desc(mine, tid < n_holders, rho_lo, hist, scratch);
-    tau_hi = block_select_desc(mine, tid < n_holders, rho_hi, hist, scratch);
+  if (rho_lo <= n_held) {
+    tau_lo = block_select_desc(mine, n_held, rho_lo, hist, scratch);
+    tau_hi = block_select_desc(mine, n_held, rho_hi, hist, scratch);
   } else {
     // radix select of the rho_lo-th largest over all sample keys; no upper estimate
     uint32_t prefix = 0, need = rho_lo;
