@@ -17,7 +17,9 @@ namespace rtopk {
 
 constexpr int kAggTile = 4096;
 constexpr int kAggThreads = 256;
-constexpr int kAggStage = 1024;   // entries of one output tile staged in shared memory
+constexpr int kAggStage = 1024;   // entries of one output tile staged in shared memory (dense kernel)
+constexpr int kAggSparseTile = 16384;   // output coordinates per block of the sparse kernel
+constexpr int kAggSparseStage = 2048;   // entries of one such tile staged in shared memory
 constexpr int kAggMaxW = 1024;    // workers the sparse kernel keeps run tables for
 
 __device__ __forceinline__ uint32_t lower_bound_u32(const uint32_t* a, uint32_t n, uint32_t key) {
@@ -29,15 +31,15 @@ __device__ __forceinline__ uint32_t lower_bound_u32(const uint32_t* a, uint32_t 
   return lo;
 }
 
-// starts[w * (ntiles + 1) + t] = first entry of worker w with index >= t * kAggTile (K for t = ntiles)
+// starts[w * (ntiles + 1) + t] = first entry of worker w with index >= t * tile_size (K for t = ntiles)
 __global__ void __launch_bounds__(kAggThreads) k_agg_starts(const uint32_t* __restrict__ msg_idx, uint32_t W,
-                                                            uint32_t K, uint32_t ntiles,
+                                                            uint32_t K, uint32_t ntiles, uint32_t tile_size,
                                                             uint32_t* __restrict__ starts) {
   const uint32_t t = blockIdx.x * kAggThreads + threadIdx.x;
   const uint32_t w = blockIdx.y;
   if (t > ntiles || w >= W) return;
   const uint32_t* row = msg_idx + (size_t)w * K;
-  starts[(size_t)w * (ntiles + 1) + t] = t == ntiles ? K : lower_bound_u32(row, K, t * (uint32_t)kAggTile);
+  starts[(size_t)w * (ntiles + 1) + t] = t == ntiles ? K : lower_bound_u32(row, K, t * tile_size);
 }
 
 __global__ void __launch_bounds__(kAggThreads) k_aggregate(const uint32_t* __restrict__ msg_idx,
@@ -134,13 +136,13 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(const uint32_t
                                                                   uint32_t W, uint32_t K, int mean,
                                                                   float* __restrict__ out) {
   __shared__ uint32_t s_beg[kAggMaxW], s_pre[kAggMaxW + 1];
-  __shared__ uint32_t st_idx[kAggStage];
-  __shared__ float st_val[kAggStage];
+  __shared__ uint32_t st_idx[kAggSparseStage];
+  __shared__ float st_val[kAggSparseStage];
   __shared__ uint32_t s_warp[kAggThreads / 32];
   __shared__ uint32_t s_carry;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t ntiles = gridDim.x;
-  const uint32_t lo = blockIdx.x * (uint32_t)kAggTile;
+  const uint32_t lo = blockIdx.x * (uint32_t)kAggSparseTile;
   if (tid == 0) s_carry = 0;
   __syncthreads();
   for (uint32_t w0 = 0; w0 < W; w0 += kAggThreads) {
@@ -165,7 +167,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(const uint32_t
   const uint32_t total = s_carry;
   if (total == 0) return;
   if (tid == 0) s_pre[W] = total;
-  const bool staged = total <= (uint32_t)kAggStage;
+  const bool staged = total <= (uint32_t)kAggSparseStage;
   __syncthreads();
   auto worker_of = [&](uint32_t q) {                 // last worker with s_pre[w] <= q
     uint32_t a = 0, b = W;
@@ -187,10 +189,34 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(const uint32_t
   auto val_at = [&](uint32_t w, uint32_t j) {
     return staged ? st_val[s_pre[w] + j] : __ldg(msg_val + (size_t)w * K + s_beg[w] + j);
   };
+  // Most coordinates are sent by a single worker.  Two bitmaps over the tile find the ones that are
+  // not: the second entry that sets a coordinate's "seen" bit also sets its "shared" bit.
+  __shared__ uint32_t s_seen[kAggSparseTile / 32], s_shared[kAggSparseTile / 32];
+  if (staged) {
+    for (uint32_t i = tid; i < (uint32_t)(kAggSparseTile / 32); i += kAggThreads) { s_seen[i] = 0; s_shared[i] = 0; }
+    __syncthreads();
+    for (uint32_t q = tid; q < total; q += kAggThreads) {
+      const uint32_t local = st_idx[q] - lo;
+      if (local < (uint32_t)kAggSparseTile) {
+        const uint32_t bit = 1u << (local & 31u);
+        if (atomicOr(&s_seen[local >> 5], bit) & bit) atomicOr(&s_shared[local >> 5], bit);
+      }
+    }
+    __syncthreads();
+  }
   for (uint32_t q = tid; q < total; q += kAggThreads) {
+    if (staged) {
+      const uint32_t idx = st_idx[q], local = idx - lo;
+      if (local >= (uint32_t)kAggSparseTile || idx >= d) continue;    // malformed row: ignore
+      if (!((s_shared[local >> 5] >> (local & 31u)) & 1u)) {    // sole sender: the sum is the value
+        const double v = (double)st_val[q];
+        out[idx] = (float)(mean ? v / (double)W : v);
+        continue;
+      }
+    }
     const uint32_t w = worker_of(q);
     const uint32_t idx = idx_at(w, q - s_pre[w]);
-    if (idx - lo >= (uint32_t)kAggTile || idx >= d) continue;   // malformed row: ignore
+    if (idx - lo >= (uint32_t)kAggSparseTile || idx >= d) continue;   // malformed row: ignore
     double sum = 0.0;
     bool owner = true;
     for (uint32_t x = 0; x < W; ++x) {

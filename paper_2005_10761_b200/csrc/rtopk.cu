@@ -368,7 +368,7 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
 }
 
 bool aggregate_is_sparse(int64_t d, int32_t W, int64_t k) {
-  return W <= kAggMaxW && (uint64_t)W * (uint64_t)k * 8ull <= (uint64_t)d;
+  return W <= kAggMaxW && (uint64_t)W * (uint64_t)k * 16ull <= (uint64_t)d;   // <= 1024 entries per tile on average
 }
 
 // `out_cleared`: the caller has already zeroed `out` in stream order (the step calls do it beside
@@ -380,14 +380,16 @@ int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val
   if (scale_mode != RTOPK_SCALE_MEAN && scale_mode != RTOPK_SCALE_SUM) return RTOPK_ERR_INVALID_ARG;
   if (((uintptr_t)out & 15u) || ((uintptr_t)msg_idx & 3u) || ((uintptr_t)msg_val & 3u)) return RTOPK_ERR_INVALID_ARG;
   if ((uint64_t)k * (uint64_t)W >= (1ull << 32)) return RTOPK_ERR_INVALID_ARG;
-  const uint32_t ntiles = (uint32_t)((d + kAggTile - 1) / kAggTile);
+  const bool sparse = aggregate_is_sparse(d, W, k);
+  const uint32_t tile = sparse ? (uint32_t)kAggSparseTile : (uint32_t)kAggTile;
+  const uint32_t ntiles = (uint32_t)((d + tile - 1) / tile);
   if ((size_t)W * (ntiles + 1) > ctx->agg_start_entries) return RTOPK_ERR_INVALID_ARG;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return RTOPK_ERR_CUDA;
   const dim3 sgrid((ntiles + 1 + kAggThreads - 1) / kAggThreads, (uint32_t)W);
-  k_agg_starts<<<sgrid, kAggThreads, 0, st>>>(msg_idx, (uint32_t)W, (uint32_t)k, ntiles, ctx->d_agg_starts);
+  k_agg_starts<<<sgrid, kAggThreads, 0, st>>>(msg_idx, (uint32_t)W, (uint32_t)k, ntiles, tile, ctx->d_agg_starts);
   const int mean = scale_mode == RTOPK_SCALE_MEAN ? 1 : 0;
-  if (aggregate_is_sparse(d, W, k)) {
+  if (sparse) {
     // few coordinates are touched: clear the update, then compute only what was sent
     if (!out_cleared) RTOPK_CUDA(ctx, cudaMemsetAsync(out, 0, (size_t)d * sizeof(float), st));
     k_aggregate_sparse<<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, ctx->d_agg_starts, (uint32_t)d,

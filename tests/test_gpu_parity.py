@@ -235,7 +235,7 @@ def test_aggregate_against_oracle(lib, W, d, k):
 def test_aggregate_sparse_path_many_workers_and_crowded_tiles(lib):
     rng = np.random.default_rng(99)
     cases = []
-    d, W, k = 2_000_003, 300, 500                      # more workers than one block batch
+    d, W, k = 3_000_017, 300, 500                      # more workers than one block batch
     cases.append((d, np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)])))
     d, W, k = 1_000_000, 8, 2000                       # every entry inside the first output tiles
     cases.append((d, np.stack([np.sort(rng.choice(6000, k, replace=False)) for _ in range(W)])))
