@@ -54,7 +54,8 @@ struct rtopk_ctx {
   // optional per-phase timing (RTOPK_OPT_PROFILE): events recorded on the caller's stream
   int sms = 0;
   int finish_max_clusters[5] = {0, 0, 0, 0, 0};   // co-resident k_finish clusters of size 1, 2, 4, 8, 16
-  int stream_blocks[2] = {0, 0};      // persistent grid of k_stream per gradient dtype
+  int stream_blocks[2] = {0, 0};
+  int exact_blocks = 0;               // cooperative grid of k_exact (all blocks resident)      // persistent grid of k_stream per gradient dtype
   // work that does not depend on the data (the k-of-r subset, clearing the dense update) runs on a
   // side stream next to the streaming pass
   cudaStream_t side = nullptr;
@@ -222,9 +223,22 @@ int check_common(const rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t
   return RTOPK_OK;
 }
 
+// Passes first_pass..2 of the full-vector radix select plus the ordered collect, as one cooperative
+// launch (its blocks meet at grid barriers, so all of them must be resident).
+int launch_exact(rtopk_ctx* ctx, const Plan& P, const Launch& L, int first_pass, cudaStream_t st) {
+  Launch Lc = L;
+  int fp = first_pass;
+  uint32_t nh = P.n_hist_blocks, nc = P.n_chunks;
+  void* args[] = {&Lc, &fp, &nh, &nc};
+  RTOPK_CUDA(ctx, cudaLaunchCooperativeKernel((const void*)k_exact, dim3((unsigned)ctx->exact_blocks), dim3(kThreads),
+                                              args, 0, st));
+  return RTOPK_OK;
+}
+
 template <typename GradT>
 int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st) {
   const uint32_t n = (uint32_t)P.slices.size();
+  int rc = RTOPK_OK;
   if (ctx->select_path == 0) {
     mark(ctx, RTOPK_PHASE_THRESHOLD, st);
     k_sample<GradT><<<n, kSampleThreads, kSampleSmemBytes, st>>>(L);
@@ -242,23 +256,20 @@ int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t s
     }
     mark(ctx, RTOPK_PHASE_EXACT, st);
     if (P.any_select) {
-      const uint32_t hgrid = std::min<uint32_t>(P.n_hist_blocks, (uint32_t)ctx->sms * 8u);
-      const uint32_t cgrid = std::min<uint32_t>(P.n_chunks, (uint32_t)ctx->sms * 4u);
-      for (int pass = 0; pass < 3; ++pass) k_hist<float, false><<<hgrid, kThreads, 0, st>>>(L, pass, P.n_hist_blocks);
-      k_collect<float, false, true><<<cgrid, kThreads, 0, st>>>(L, P.n_chunks);
+      rc = launch_exact(ctx, P, L, 0, st);
+      if (rc) return rc;
     }
   } else {
     mark(ctx, RTOPK_PHASE_THRESHOLD, st);
     k_init_state<<<(n + 127) / 128, 128, 0, st>>>(L, 1u);
     mark(ctx, RTOPK_PHASE_STREAM, st);
     const uint32_t hgrid = std::min<uint32_t>(P.n_hist_blocks, (uint32_t)ctx->sms * 8u);
-    const uint32_t cgrid = std::min<uint32_t>(P.n_chunks, (uint32_t)ctx->sms * 4u);
     k_hist<GradT, true><<<hgrid, kThreads, 0, st>>>(L, 0, P.n_hist_blocks);
     mark(ctx, RTOPK_PHASE_ORDER, st);
     mark(ctx, RTOPK_PHASE_EXACT, st);
     if (P.any_select) {
-      for (int pass = 1; pass < 3; ++pass) k_hist<float, false><<<hgrid, kThreads, 0, st>>>(L, pass, P.n_hist_blocks);
-      k_collect<float, false, true><<<cgrid, kThreads, 0, st>>>(L, P.n_chunks);
+      rc = launch_exact(ctx, P, L, 1, st);
+      if (rc) return rc;
     }
   }
   return RTOPK_OK;
@@ -495,6 +506,10 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
     if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_bf16, k_stream<__nv_bfloat16>, kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>));
     if (e == cudaSuccess && (per_f32 < 1 || per_bf16 < 1)) e = cudaErrorLaunchOutOfResources;
     ctx->sms = sms;
+    int per_exact = 0;
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_exact, k_exact, kThreads, 0);
+    if (e == cudaSuccess && per_exact < 1) e = cudaErrorLaunchOutOfResources;
+    ctx->exact_blocks = sms * std::min(per_exact, 4);
     ctx->stream_blocks[0] = sms * per_f32;
     ctx->stream_blocks[1] = sms * per_bf16;
   }

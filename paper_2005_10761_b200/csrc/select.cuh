@@ -244,7 +244,7 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(Launch L) {
 // eq_quota keys == tau_lo in index order.  The candidate list keeps index order: inside a block by
 // ballot-free packed prefix sums, across blocks by the look-back on (count above, count equal).
 template <typename GradT, bool FUSE, bool TIES>
-__global__ void __launch_bounds__(kThreads) k_collect(Launch L, uint32_t total_tiles) {
+__device__ __forceinline__ void collect_body(const Launch& L, uint32_t total_tiles) {
   __shared__ uint32_t s_tile, s_wA[kWarps], s_wB[kWarps], s_ex[2];
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (!FUSE && !L.general_primary && L.s.tickets[3] == 0) return;   // no slice needs the exact path
@@ -259,7 +259,7 @@ __global__ void __launch_bounds__(kThreads) k_collect(Launch L, uint32_t total_t
   if (tile >= total_tiles) return;
   const uint32_t sl = find_slice(L.n_slices, tile, [&](uint32_t i) { return slices[i].chunk_begin; });
   const Slice S = slices[sl];
-  SelState* st = &L.s.state[sl];
+  volatile SelState* st = &L.s.state[sl];   // other blocks update it inside one launch: no L1
   if (!FUSE) {
     if (!((st->flags & FLAG_GENERAL) && st->stage == STAGE_COLLECT)) continue;
   }
@@ -363,7 +363,7 @@ __device__ __forceinline__ void finish_pass(const Launch& L, uint32_t sl, const 
     gh[b] = 0;
   }
   __syncthreads();
-  SelState* st = &L.s.state[sl];
+  volatile SelState* st = &L.s.state[sl];   // other blocks update it inside one launch: no L1
   const uint32_t need = st->need;
   uint32_t D, above;
   const bool ok = pick_digit(hist_s, 1 << bits, need, scratch, D, above);
@@ -401,7 +401,7 @@ __device__ __forceinline__ bool is_last_block(uint32_t* counter, uint32_t nblock
   return s_last != 0;
 }
 
-__device__ __forceinline__ bool first_pass_missed(const SelState* st, const Slice& S) {
+__device__ __forceinline__ bool first_pass_missed(const volatile SelState* st, const Slice& S) {
   return st->n_cand < S.r || st->n_cand > S.cand_cap;
 }
 
@@ -409,7 +409,7 @@ __device__ __forceinline__ bool first_pass_missed(const SelState* st, const Slic
 // add and the write-back; otherwise a is read from the residual buffer.  Pass p > 0 counts only keys
 // whose higher bits equal the resolved prefix.
 template <typename GradT, bool FUSE>
-__global__ void __launch_bounds__(kThreads) k_hist(Launch L, int pass, uint32_t total_blocks) {
+__device__ __forceinline__ void hist_body(const Launch& L, int pass, uint32_t total_blocks) {
   __shared__ uint32_t hist_s[kBins];
   __shared__ uint32_t scratch[kWarps + 2];
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -420,7 +420,7 @@ __global__ void __launch_bounds__(kThreads) k_hist(Launch L, int pass, uint32_t 
     __syncthreads();                                   // hist_s / scratch of the previous unit are free
     const uint32_t sl = find_slice(L.n_slices, unit, [&](uint32_t i) { return slices[i].hist_begin; });
     const Slice S = slices[sl];
-    SelState* st = &L.s.state[sl];
+    volatile SelState* st = &L.s.state[sl];   // other blocks update it inside one launch: no L1
     const uint32_t flags = st->flags;
     const bool fell_back = !(flags & FLAG_GENERAL) && !FUSE && pass == 0 && S.r < S.len && first_pass_missed(st, S);
     const bool counting = (flags & FLAG_GENERAL) ? st->stage == (uint32_t)pass : fell_back;
@@ -463,6 +463,48 @@ __global__ void __launch_bounds__(kThreads) k_hist(Launch L, int pass, uint32_t 
     const uint32_t nblocks = (nchunks + kHistChunks - 1) / kHistChunks;
     if (is_last_block(&L.s.done[sl], nblocks)) finish_pass(L, sl, S, pass, true, fell_back, hist_s, scratch);
   }
+}
+
+template <typename GradT, bool FUSE>
+__global__ void __launch_bounds__(kThreads) k_hist(Launch L, int pass, uint32_t total_blocks) {
+  hist_body<GradT, FUSE>(L, pass, total_blocks);
+}
+
+// Grid-wide barrier of a cooperative launch (all blocks resident).  `target` = blocks * barriers
+// passed so far.  Bounded: on expiry the error flag is raised and false is returned to every thread
+// of the block, which then leaves the kernel; the other blocks run into the same limit.
+constexpr int kGridSpinLimit = 1 << 22;
+__device__ __forceinline__ bool grid_barrier(uint32_t* counter, uint32_t target, uint32_t* error) {
+  __shared__ uint32_t s_ok;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(counter, 1u);
+    uint32_t ok = 1;
+    int spins = 0;
+    while (*reinterpret_cast<volatile uint32_t*>(counter) < target) {
+      if (++spins > kGridSpinLimit) { ok = 0; atomicOr(error, ERR_LOOKBACK_TIMEOUT); break; }
+      __nanosleep(100);
+    }
+    __threadfence();
+    s_ok = ok;
+  }
+  __syncthreads();
+  return s_ok != 0;
+}
+
+// The whole exact path in one cooperative launch: the remaining radix passes over the full vector
+// (each ends with the per-slice digit pick in the last block that finishes that slice), a grid
+// barrier after each, then the ordered collect.  When no slice needs the exact path -- the usual
+// case after the sampled pass -- every block returns at once, so the idle cost is one launch.
+__global__ void __launch_bounds__(kThreads) k_exact(Launch L, int first_pass, uint32_t n_hist_blocks, uint32_t n_chunks) {
+  if (!L.general_primary && L.s.tickets[3] == 0) return;
+  uint32_t passed = 0;
+  for (int pass = first_pass; pass < 3; ++pass) {
+    hist_body<float, false>(L, pass, n_hist_blocks);
+    if (!grid_barrier(&L.s.tickets[2], gridDim.x * (++passed), L.s.error)) return;
+  }
+  collect_body<float, false, true>(L, n_chunks);
 }
 
 // ----------------------------------------------------------------------------- finish
