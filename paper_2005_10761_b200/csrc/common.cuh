@@ -225,15 +225,14 @@ __device__ __forceinline__ bool pick_digit(const uint32_t* hist, int nbins, uint
   uint32_t incl = warp_incl_scan(mine);
   const uint32_t warp = threadIdx.x >> 5, nwarps = (nthreads + 31) >> 5;
   if (lane_id() == 31) scratch[warp] = incl;
-  __syncthreads();
   if (threadIdx.x == 0) {
-    uint32_t run = 0;
-    for (uint32_t w = 0; w < nwarps; ++w) { uint32_t v = scratch[w]; scratch[w] = run; run += v; }
     scratch[nwarps] = 0xFFFFFFFFu;      // result: digit
     scratch[nwarps + 1] = 0;            // result: above
   }
   __syncthreads();
-  incl += scratch[warp];
+  uint32_t woff = 0;
+  for (uint32_t w = 0; w < warp; ++w) woff += scratch[w];
+  incl += woff;
   const uint32_t excl = incl - mine;
   if (excl < need && need <= incl) {     // the crossing lies in this thread's bins
     uint32_t run = excl;

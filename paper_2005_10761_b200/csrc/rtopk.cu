@@ -53,7 +53,7 @@ struct rtopk_ctx {
   uint32_t last_n_slices = 0;
   // optional per-phase timing (RTOPK_OPT_PROFILE): events recorded on the caller's stream
   int sms = 0;
-  int finish_max_clusters[5] = {0, 0, 0, 0, 0};   // co-resident k_finish clusters of size 1, 2, 4, 8, 16
+  int finish_max_clusters[kMaxCluster + 1] = {};  // [cs]: co-resident k_finish clusters of size cs (1..16)
   int stream_blocks[2] = {0, 0};
   int exact_blocks = 0;               // cooperative grid of k_exact (all blocks resident)      // persistent grid of k_stream per gradient dtype
   // work that does not depend on the data (the k-of-r subset, clearing the dense update) runs on a
@@ -354,8 +354,8 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   if (P.any_select) {
     // the largest cluster size that still lets every slice's cluster be resident at once
     int cs = 1;
-    for (int i = 4; i >= 0; --i)
-      if ((int)L.n_slices <= ctx->finish_max_clusters[i]) { cs = 1 << i; break; }
+    for (int c = kMaxCluster; c >= 1; --c)
+      if ((int)L.n_slices <= ctx->finish_max_clusters[c]) { cs = c; break; }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)cs * L.n_slices, 1, 1);
     cfg.blockDim = dim3(kFinishThreads, 1, 1);
@@ -483,20 +483,20 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFinishSmemBytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-  for (int i = 0; i < 5 && e == cudaSuccess; ++i) {
+  for (int c = 1; c <= kMaxCluster && e == cudaSuccess; ++c) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(1u << i, 1, 1);
+    cfg.gridDim = dim3((unsigned)c, 1, 1);
     cfg.blockDim = dim3(kFinishThreads, 1, 1);
     cfg.dynamicSmemBytes = kFinishSmemBytes;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 1u << i; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[0].val.clusterDim.x = (unsigned)c; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, k_finish, &cfg) == cudaSuccess) ctx->finish_max_clusters[i] = n;
+    if (cudaOccupancyMaxActiveClusters(&n, k_finish, &cfg) == cudaSuccess) ctx->finish_max_clusters[c] = n;
     else cudaGetLastError();
   }
-  if (e == cudaSuccess && ctx->finish_max_clusters[0] < 1) e = cudaErrorLaunchOutOfResources;
+  if (e == cudaSuccess && ctx->finish_max_clusters[1] < 1) e = cudaErrorLaunchOutOfResources;
   if (e == cudaSuccess) {
     int sms = 0, per_f32 = 0, per_bf16 = 0;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);

@@ -525,6 +525,7 @@ constexpr int kFinishThreads = 1024;
 constexpr int kFinishWarps = kFinishThreads / 32;
 constexpr int kFinishCache = 46 * 1024;   // candidate values a CTA keeps in shared memory (184 KB)
 constexpr int kFinishBatch = 8;           // independent loads in flight per thread
+constexpr int kFinishList = 512;         // bucket population up to which the bucket is ranked directly
 constexpr int kFinishSelWords = 2048;     // bitmap words (64 Ki positions) a CTA keeps in shared memory
 
 struct alignas(16) FinishSmem {           // the value cache behind it is read as float4
@@ -535,6 +536,8 @@ struct alignas(16) FinishSmem {           // the value cache behind it is read a
   uint32_t scratch[kFinishWarps + 2];
   uint32_t counts[2 * kMaxCluster];    // (members above tau, equal to tau) of every CTA's share
   uint32_t warpA[kFinishWarps], warpB[kFinishWarps];
+  uint32_t list_pre[kMaxCluster + 1];  // list round: exclusive prefix of the CTAs' list lengths
+  uint32_t list_n, tau_out;            // list round: my list length; the key that was found
 };
 static_assert(sizeof(FinishSmem) % 16 == 0, "the value cache must start 16-byte aligned");
 constexpr size_t kFinishSmemBytes = sizeof(FinishSmem) + (size_t)kFinishCache * sizeof(float);
@@ -545,7 +548,7 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
   FinishSmem& sm = *reinterpret_cast<FinishSmem*>(finish_raw);
   float* cache = reinterpret_cast<float*>(finish_raw + sizeof(FinishSmem));
   cg::cluster_group cluster = cg::this_cluster();
-  const uint32_t CS = cluster.num_blocks();                    // 1, 2, 4, 8 or 16
+  const uint32_t CS = cluster.num_blocks();                    // 1 .. kMaxCluster
   const uint32_t q = cluster.block_rank();
   const uint32_t sl = blockIdx.x / CS;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -612,7 +615,57 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
     }
   };
 
+  // keys inside [lo_key, hi_key) over the whole cluster, when known
+  uint32_t bucket_n = (st->flags & FLAG_GENERAL) ? n_cand - n_gt : 0xFFFFFFFFu;
   for (int round = 0; (hi_key - lo_key > 1u || count_above) && round < 8; ++round) {
+    if (!count_above && bucket_n <= (uint32_t)kFinishList) {
+      // Few keys are left in the interval: instead of more histogram rounds, every CTA lists its own,
+      // reads the other CTAs' lists through distributed shared memory and ranks the union by counting.
+      if (tid == 0) sm.list_n = 0;
+      __syncthreads();
+      for_each_key([&](uint32_t key) {
+        if (key >= lo_key && key < hi_key) {
+          const uint32_t at = atomicAdd(&sm.list_n, 1u);
+          if (at < (uint32_t)kBins) sm.hist[at] = key;
+        }
+      });
+      cluster.sync();
+      if (warp == 0) {
+        const uint32_t n = lane < CS ? *cluster.map_shared_rank(&sm.list_n, lane) : 0u;
+        const uint32_t incl = warp_incl_scan(n);
+        if (lane < (uint32_t)kMaxCluster) sm.list_pre[lane + 1] = incl;
+        if (lane == 0) sm.list_pre[0] = 0;
+      }
+      __syncthreads();
+      const uint32_t total = sm.list_pre[CS];
+      if (total > (uint32_t)kFinishList || total < need) {       // the same on every CTA
+        if (q == 0 && tid == 0) { atomicOr(L.s.error, ERR_SELECT_INCONSISTENT); st->resolved = 32; }
+        cluster.sync();
+        return;
+      }
+      for (uint32_t t = tid; t < total; t += kFinishThreads) {
+        uint32_t rr = 0;
+        while (sm.list_pre[rr + 1] <= t) ++rr;
+        sm.red[t] = cluster.map_shared_rank(sm.hist, rr)[t - sm.list_pre[rr]];
+      }
+      __syncthreads();
+      if (tid < total) {
+        const uint32_t e = sm.red[tid];
+        uint32_t rank = 0;                                       // keys ranked before e (ties: list order)
+        for (uint32_t j = 0; j < total; ++j) {
+          const uint32_t o = sm.red[j];
+          rank += (o > e) || (o == e && j < tid);
+        }
+        if (rank == need - 1u) sm.tau_out = e;
+      }
+      __syncthreads();
+      const uint32_t found = sm.tau_out;
+      const uint32_t above = __syncthreads_count(tid < total && sm.red[tid] > found);
+      cluster.sync();                                            // all remote reads of the lists are done
+      n_gt += above; need -= above;
+      lo_key = found; hi_key = found + 1u;
+      break;
+    }
     const uint32_t width = hi_key - lo_key;                    // >= 1
     uint32_t sh = 0;
     while (((width - 1u) >> sh) >= (uint32_t)(kBins - 1)) ++sh;
@@ -643,6 +696,7 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
     __syncthreads();
     uint32_t D, above;
     pick_digit(sm.red, kBins, need, sm.scratch, D, above);
+    bucket_n = D < (uint32_t)kBins ? sm.red[D] : 0u;
     cluster.sync();                                            // all remote reads of sm.hist are done
     if (D == 0xFFFFFFFFu) {                                    // fewer keys than the rank asked for
       if (q == 0 && tid == 0) { atomicOr(L.s.error, ERR_SELECT_INCONSISTENT); st->resolved = 32; }
@@ -651,7 +705,7 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
     if (D == (uint32_t)(kBins - 1)) {
       // only possible while the keys above the interval were being counted: the sampled upper
       // estimate was too low and the target lies above it
-      lo_key = hi_key; hi_key = 0x80000000u;
+      lo_key = hi_key; hi_key = 0x80000000u;                    // bucket_n: the keys above, all still inside
     } else {
       n_gt += above; need -= above;
       lo_key += D << sh;
@@ -736,6 +790,11 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
     const uint32_t i0 = base + lane * 4u;
     float v[4];
     load4(i0, v);
+    // the four indices, fetched now so that no store below waits on a load (the list's capacity is a
+    // multiple of 32 entries, so the vector stays inside the slice's list)
+    uint4 ci = make_uint4(0u, 0u, 0u, 0u);
+    if (i0 < w_hi) ci = __ldg(reinterpret_cast<const uint4*>(cidx + lo + i0));
+    const uint32_t cj[4] = {ci.x, ci.y, ci.z, ci.w};
     uint32_t mA = 0, mB = 0;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -757,7 +816,7 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
           const uint32_t p = g + min(e, quota);
           uint32_t slot;
           if (p < S.r && selected(p, slot) && slot < S.k) {
-            const uint32_t idx = cidx[lo + i0 + j];
+            const uint32_t idx = cj[j];
             L.msg_idx[S.msg_off + slot] = S.idx_base + idx;
             L.msg_val[S.msg_off + slot] = v[j];
             L.residual[S.m_off + idx] = 0.0f;
