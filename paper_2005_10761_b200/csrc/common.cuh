@@ -15,8 +15,7 @@ constexpr int kIter = 4;                      // 4-element vectors per thread pe
 constexpr int kWarpSpan = 32 * kIter * 4;     // 512 consecutive elements per warp
 constexpr int kChunk = kWarps * kWarpSpan;    // 4096 elements per block of the collect kernels
 constexpr int kHistChunks = 16;               // chunks per block of the histogram kernels
-constexpr int kCandTile = 2048;               // candidates per block of the candidate kernels
-constexpr int kCandPer = kCandTile / kThreads;
+constexpr int kGroupsMax = 2048;              // chunk groups per slice (two per thread of k_finish)
 
 // radix digits of the 31-bit magnitude key, most significant first: 11 + 11 + 9 bits
 constexpr int kBins = 2048;
@@ -47,11 +46,11 @@ struct Slice {
   uint32_t cand_off, cand_cap;
   uint32_t chunk_begin; // first collect tile (all slices are numbered one after another)
   uint32_t hist_begin;  // first histogram block
-  uint32_t ctile_begin; // first candidate tile
+  uint32_t group_begin; // first entry of the slice in the chunk-group totals
   uint32_t samp_off;    // start in the draw buffer (k entries)
   uint32_t first_off;   // start in the first-occurrence table (r entries)
   uint32_t sel_off;     // start in the selection bitmap / its prefix counts (32-bit words)
-  uint32_t pad;
+  uint32_t gshift;      // a chunk group is 2^gshift consecutive chunks (at most kGroupsMax groups per slice)
 };
 
 // Selection state of one slice, advanced kernel by kernel.
@@ -75,14 +74,12 @@ struct Scratch {
   SelState* state;
   uint32_t* hist;         // [slices][kBins]
   uint32_t* done;         // [slices] block-completion counters
-  uint32_t* tickets;      // [0..2] dynamic tile counters; [3] slices whose sampled threshold missed
-  unsigned long long* look_a;   // look-back words of the first collect
-  unsigned long long* look_b;   // ... of the fallback collect
-  unsigned long long* look_e;   // ... of the emit pass
-  uint32_t* cursor;       // [slices] next free entry of the raw candidate buffer
+  uint32_t* tickets;      // [1] tile counter of the exact collect; [2] grid-barrier counter
+  unsigned long long* look_b;   // look-back words of the exact path's collect
+  uint32_t* cursor;       // [slices] next free entry of the raw candidate buffer (= candidates so far)
+  uint32_t* group_total;  // candidates per chunk group (summed by the stream pass)
   uint32_t* chunk_start;  // [chunks] where a chunk's run sits in the raw buffer ...
   uint32_t* chunk_count;  // ... its length ...
-  uint32_t* chunk_dst;    // ... and its place in chunk order
   uint32_t* raw_idx;      // candidates in reservation order
   float* raw_val;
   uint32_t* cand_idx;     // candidates in index order

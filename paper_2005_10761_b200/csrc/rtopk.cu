@@ -38,7 +38,7 @@ struct rtopk_ctx {
   float* d_cand_val = nullptr;
   uint32_t* d_raw_idx = nullptr;
   float* d_raw_val = nullptr;
-  uint32_t* d_chunk_tab = nullptr;   // chunk_start | chunk_count | chunk_dst
+  uint32_t* d_chunk_tab = nullptr;   // chunk_start | chunk_count
   size_t chunk_tab_entries = 0;
   size_t cand_entries = 0;
   uint32_t* d_draws = nullptr;
@@ -106,7 +106,7 @@ uint32_t cand_capacity(uint64_t len, uint64_t r) {
 // Layout of one call: the slice table plus every per-call scratch offset.
 struct Plan {
   std::vector<Slice> slices;
-  uint32_t n_chunks = 0, n_hist_blocks = 0, n_ctiles = 0;
+  uint32_t n_chunks = 0, n_hist_blocks = 0, n_groups = 0;
   size_t cand_entries = 0, draw_entries = 0, first_entries = 0, sel_words = 0;
   uint32_t k_draw_max = 0, words_all_max = 0, cap_max = 0, chunks_max = 0;
   bool any_select = false, any_sampler = false, any_all = false;
@@ -129,7 +129,7 @@ int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32
   P.K_row = (uint32_t)K;
   P.uniform = (S == 1);
   P.slices.resize((size_t)W * (size_t)S);
-  uint64_t chunks = 0, hblocks = 0, ctiles = 0, cand = 0, draws = 0, first = 0, selw = 0;
+  uint64_t chunks = 0, hblocks = 0, groups = 0, cand = 0, draws = 0, first = 0, selw = 0;
   for (int w = 0; w < W; ++w) {
     uint64_t msg_at = (uint64_t)w * K;
     for (int s = 0; s < S; ++s) {
@@ -153,13 +153,17 @@ int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32
       chunks += nchunks;
       if (nchunks > P.chunks_max) P.chunks_max = nchunks;
       hblocks += (nchunks + kHistChunks - 1) / kHistChunks;
-      sl.ctile_begin = (uint32_t)ctiles;
+      // chunk groups: the stream pass sums the candidates of 2^gshift consecutive chunks, which lets
+      // k_finish place every run without a pass over the whole chunk table
+      sl.gshift = 5;
+      while (((nchunks + (1u << sl.gshift) - 1) >> sl.gshift) > (uint32_t)kGroupsMax) ++sl.gshift;
+      sl.group_begin = (uint32_t)groups;
+      groups += (nchunks + (1u << sl.gshift) - 1) >> sl.gshift;
       sl.cand_off = (uint32_t)cand;
       if (sl.r < sl.len) {
         sl.cand_cap = cand_capacity(sl.len, sl.r);
         cand += sl.cand_cap;
         if (sl.cand_cap > P.cap_max) P.cap_max = sl.cand_cap;
-        ctiles += (sl.cand_cap + kCandTile - 1) / kCandTile;
         P.any_select = true;
       } else {
         sl.cand_cap = 0;
@@ -180,7 +184,7 @@ int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32
     }
   }
   if (chunks >= (1ull << 31) || cand >= (1ull << 32) || first >= (1ull << 32)) return RTOPK_ERR_INVALID_ARG;
-  P.n_chunks = (uint32_t)chunks; P.n_hist_blocks = (uint32_t)hblocks; P.n_ctiles = (uint32_t)ctiles;
+  P.n_chunks = (uint32_t)chunks; P.n_hist_blocks = (uint32_t)hblocks; P.n_groups = (uint32_t)groups;
   P.cand_entries = cand; P.draw_entries = draws; P.first_entries = first; P.sel_words = selw;
   return RTOPK_OK;
 }
@@ -194,17 +198,16 @@ size_t carve_zero(const rtopk_ctx* ctx, const Plan& P, Scratch& s) {
   s.done = (uint32_t*)take(P.slices.size() * sizeof(uint32_t));
   s.cursor = (uint32_t*)take(P.slices.size() * sizeof(uint32_t));
   s.hist = (uint32_t*)take(P.slices.size() * kBins * sizeof(uint32_t));
-  s.look_a = (unsigned long long*)take((size_t)P.n_chunks * 8);
+  s.group_total = (uint32_t*)take((size_t)P.n_groups * sizeof(uint32_t));
   s.look_b = (unsigned long long*)take((size_t)P.n_chunks * 8);
-  s.look_e = (unsigned long long*)take((size_t)P.n_ctiles * 8);
   s.sel = (uint32_t*)take(P.sel_words * sizeof(uint32_t));
   return at;
 }
 
-size_t zero_region_bytes(size_t slices, size_t chunks, size_t ctiles, size_t sel_words) {
+size_t zero_region_bytes(size_t slices, size_t chunks, size_t groups, size_t sel_words) {
   size_t at = 0;
   auto take = [&](size_t bytes) { at = align_up(at + bytes, 256); };
-  take(16); take(slices * 4); take(slices * 4); take(slices * kBins * 4); take(chunks * 8); take(chunks * 8); take(ctiles * 8);
+  take(16); take(slices * 4); take(slices * 4); take(slices * kBins * 4); take(groups * 4); take(chunks * 8);
   take(sel_words * 4);
   return at;
 }
@@ -249,10 +252,6 @@ int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t s
       const int blocks = ctx->stream_blocks[sizeof(GradT) == 4 ? 0 : 1];
       k_stream<GradT><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
       mark(ctx, RTOPK_PHASE_ORDER, st);
-      if (P.any_select) {
-        k_cand_scan<<<n, kOrderThreads, 0, st>>>(L);
-        k_cand_gather<<<(P.n_chunks + kWarps - 1) / kWarps, kThreads, 0, st>>>(L, P.n_chunks, uniform);
-      }
     }
     mark(ctx, RTOPK_PHASE_EXACT, st);
     if (P.any_select) {
@@ -321,7 +320,6 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   if ((size_t)P.n_chunks > ctx->chunk_tab_entries) return RTOPK_ERR_INVALID_ARG;
   L.s.chunk_start = ctx->d_chunk_tab;
   L.s.chunk_count = ctx->d_chunk_tab + ctx->chunk_tab_entries;
-  L.s.chunk_dst = ctx->d_chunk_tab + 2 * ctx->chunk_tab_entries;
   L.s.draws = ctx->d_draws; L.s.first = ctx->d_first; L.s.sel_pre = ctx->d_sel_pre;
   L.s.error = ctx->d_error;
   L.grad = grad; L.residual = residual; L.msg_idx = msg_idx; L.msg_val = msg_val;
@@ -452,11 +450,11 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   const size_t W = (size_t)W_max, S = (size_t)segments_max, slices = W * S;
   const size_t chunks = W * ((size_t)d_max / kChunk + 2 * S + 1);
   const size_t cand_row = std::min<size_t>((size_t)d_max, 2 * (size_t)r_max + 1024 * S) + 32 * S;
-  const size_t ctiles = W * (cand_row / kCandTile + 1 + S);
+  const size_t groups = W * ((size_t)d_max / kChunk / 32 + 2 * S + 1);
   ctx->cand_entries = W * cand_row;
   ctx->first_entries = W * (size_t)r_max;
   ctx->sel_words = W * ((size_t)r_max / 32 + S + 1);
-  ctx->zero_bytes = zero_region_bytes(slices, chunks, ctiles, ctx->sel_words);
+  ctx->zero_bytes = zero_region_bytes(slices, chunks, groups, ctx->sel_words);
   ctx->agg_start_entries = W * ((size_t)(d_max + kAggTile - 1) / kAggTile + 2);
   if (ctx->cand_entries >= (1ull << 32) || ctx->first_entries >= (1ull << 32)) { delete ctx; return RTOPK_ERR_INVALID_ARG; }
   cudaError_t e = cudaSuccess;
@@ -470,7 +468,7 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   alloc((void**)&ctx->d_raw_idx, ctx->cand_entries * sizeof(uint32_t));
   alloc((void**)&ctx->d_raw_val, ctx->cand_entries * sizeof(float));
   ctx->chunk_tab_entries = chunks;
-  alloc((void**)&ctx->d_chunk_tab, 3 * chunks * sizeof(uint32_t));
+  alloc((void**)&ctx->d_chunk_tab, 2 * chunks * sizeof(uint32_t));
   alloc((void**)&ctx->d_draws, W * (size_t)k_max * sizeof(uint32_t));
   alloc((void**)&ctx->d_sel_pre, ctx->sel_words * sizeof(uint32_t));
   alloc((void**)&ctx->d_error, 16);
@@ -752,7 +750,7 @@ __global__ void k_static_slice(Slice* slot, uint32_t r, uint32_t k, uint32_t seg
   Slice s;
   s.g_off = 0; s.m_off = 0; s.len = r; s.r = r; s.k = k; s.row = 0; s.segment = segment; s.idx_base = 0;
   s.head = 0; s.msg_off = 0; s.cand_off = 0; s.cand_cap = 0; s.chunk_begin = 0; s.hist_begin = 0;
-  s.ctile_begin = 0; s.samp_off = 0; s.first_off = 0; s.sel_off = 0; s.pad = 0;
+  s.group_begin = 0; s.samp_off = 0; s.first_off = 0; s.sel_off = 0; s.gshift = 5;
   *slot = s;
 }
 }  // namespace

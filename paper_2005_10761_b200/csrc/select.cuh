@@ -247,7 +247,6 @@ template <typename GradT, bool FUSE, bool TIES>
 __device__ __forceinline__ void collect_body(const Launch& L, uint32_t total_tiles) {
   __shared__ uint32_t s_tile, s_wA[kWarps], s_wB[kWarps], s_ex[2];
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (!FUSE && !L.general_primary && L.s.tickets[3] == 0) return;   // no slice needs the exact path
   const Slice* slices = L.s.slices;
   // persistent blocks; tiles are handed out by ticket so that the look-back only ever waits on
   // tiles whose blocks are already running
@@ -309,7 +308,7 @@ __device__ __forceinline__ void collect_body(const Launch& L, uint32_t total_til
 #pragma unroll
     for (int w = 0; w < kWarps; ++w) { bA += s_wA[w]; bB += s_wB[w]; }
     uint32_t exA, exB;
-    unsigned long long* words = (FUSE ? L.s.look_a : L.s.look_b) + S.chunk_begin;
+    unsigned long long* words = L.s.look_b + S.chunk_begin;
     lookback_exclusive(words, c, bA, bB, exA, exB, L.s.error);
     if (lane == 0) {
       s_ex[0] = exA; s_ex[1] = exB;
@@ -401,8 +400,10 @@ __device__ __forceinline__ bool is_last_block(uint32_t* counter, uint32_t nblock
   return s_last != 0;
 }
 
-__device__ __forceinline__ bool first_pass_missed(const volatile SelState* st, const Slice& S) {
-  return st->n_cand < S.r || st->n_cand > S.cand_cap;
+// Did the sampled pass gather too few or too many candidates for this slice?  (The slice's cursor
+// is the number of candidates the stream pass reserved room for.)
+__device__ __forceinline__ bool first_pass_missed(uint32_t n_gathered, const Slice& S) {
+  return S.r < S.len && (n_gathered < S.r || n_gathered > S.cand_cap);
 }
 
 // Histogram of one digit over the whole slice.  FUSE (pass 0 of the exact path) also performs the
@@ -413,7 +414,6 @@ __device__ __forceinline__ void hist_body(const Launch& L, int pass, uint32_t to
   __shared__ uint32_t hist_s[kBins];
   __shared__ uint32_t scratch[kWarps + 2];
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (!FUSE && !L.general_primary && L.s.tickets[3] == 0) return;   // no slice needs the exact path
   const Slice* slices = L.s.slices;
   const int bits = digit_bits(pass), shift = digit_shift(pass);
   for (uint32_t unit = blockIdx.x; unit < total_blocks; unit += gridDim.x) {
@@ -422,7 +422,7 @@ __device__ __forceinline__ void hist_body(const Launch& L, int pass, uint32_t to
     const Slice S = slices[sl];
     volatile SelState* st = &L.s.state[sl];   // other blocks update it inside one launch: no L1
     const uint32_t flags = st->flags;
-    const bool fell_back = !(flags & FLAG_GENERAL) && !FUSE && pass == 0 && S.r < S.len && first_pass_missed(st, S);
+    const bool fell_back = !(flags & FLAG_GENERAL) && !FUSE && pass == 0 && first_pass_missed(L.s.cursor[sl], S);
     const bool counting = (flags & FLAG_GENERAL) ? st->stage == (uint32_t)pass : fell_back;
     const bool add_only = FUSE && S.r == S.len;      // nothing to select, but a = g + m is still due
     if (!counting && !add_only) continue;
@@ -498,7 +498,12 @@ __device__ __forceinline__ bool grid_barrier(uint32_t* counter, uint32_t target,
 // barrier after each, then the ordered collect.  When no slice needs the exact path -- the usual
 // case after the sampled pass -- every block returns at once, so the idle cost is one launch.
 __global__ void __launch_bounds__(kThreads) k_exact(Launch L, int first_pass, uint32_t n_hist_blocks, uint32_t n_chunks) {
-  if (!L.general_primary && L.s.tickets[3] == 0) return;
+  if (!L.general_primary) {
+    bool missed = false;
+    for (uint32_t s = threadIdx.x; s < L.n_slices; s += kThreads)
+      missed |= first_pass_missed(L.s.cursor[s], L.s.slices[s]);
+    if (!__syncthreads_or(missed)) return;          // the same answer in every block
+  }
   uint32_t passed = 0;
   for (int pass = first_pass; pass < 3; ++pass) {
     hist_body<float, false>(L, pass, n_hist_blocks);
@@ -556,7 +561,8 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
   SelState* st = &L.s.state[sl];
   // every early exit below depends on the slice only, so a cluster leaves as a whole
   if (S.r == S.len) return;
-  const uint32_t n_cand = st->n_cand;
+  const bool general = (st->flags & FLAG_GENERAL) != 0;         // the list was built by the exact path
+  const uint32_t n_cand = general ? st->n_cand : L.s.cursor[sl];
   if (st->resolved > 31) return;                               // an earlier pass already failed
   if (n_cand < S.r || n_cand > S.cand_cap) {                   // cannot happen once the exact path ran
     if (q == 0 && tid == 0) atomicOr(L.s.error, ERR_CANDIDATE_OVERFLOW);
@@ -564,35 +570,154 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
   }
   uint32_t n_gt = st->n_gt, need = st->need, lo_key, hi_key;
   bool count_above;
-  if (st->flags & FLAG_GENERAL) {
+  if (general) {
     const uint32_t free_bits = 31u - st->resolved;
     lo_key = st->prefix << free_bits; hi_key = lo_key + (1u << free_bits); count_above = false;
   } else {
     lo_key = st->tau_lo; hi_key = st->tau_hi + 1u; count_above = true; n_gt = 0; need = S.r;
+    if (q == 0 && tid == 0) { st->n_cand = n_cand; st->n_cand_first = n_cand; }
   }
-  const uint32_t* cidx = L.s.cand_idx + S.cand_off;
-  const float* cval = L.s.cand_val + S.cand_off;
+  // the slice's candidate list in index order: complete already after the exact path; after the
+  // sampled pass this kernel builds its own part of it from the stream pass's runs
+  uint32_t* cidx = L.s.cand_idx + S.cand_off;
+  float* cval = L.s.cand_val + S.cand_off;
   const uint32_t per = ((n_cand + CS - 1) / CS + 31u) & ~31u;
   const uint32_t lo = min(n_cand, q * per), hi = min(n_cand, lo + per);
   const uint32_t n_mine = hi - lo;
   const uint32_t n_cached = min(n_mine, (uint32_t)kFinishCache);
 
-  // my share of the candidate values -> shared memory (the share starts 128-byte aligned)
-  {
+  if (general) {
+    // my share of the candidate values -> shared memory (the share starts 128-byte aligned)
     const float4* src = reinterpret_cast<const float4*>(cval + lo);
     float4* dst = reinterpret_cast<float4*>(cache);
     const uint32_t nv = n_cached >> 2;
     for (uint32_t base = tid; base < nv; base += kFinishThreads * 4) {
       float4 v[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) if (base + u * kFinishThreads < nv) v[u] = __ldg(src + base + u * kFinishThreads);
+      for (int u = 0; u < 4; ++u) if (base + u * kFinishThreads < nv) v[u] = src[base + u * kFinishThreads];
 #pragma unroll
       for (int u = 0; u < 4; ++u) if (base + u * kFinishThreads < nv) dst[base + u * kFinishThreads] = v[u];
     }
-    for (uint32_t i = (nv << 2) + tid; i < n_cached; i += kFinishThreads) cache[i] = __ldg(cval + lo + i);
+    for (uint32_t i = (nv << 2) + tid; i < n_cached; i += kFinishThreads) cache[i] = cval[lo + i];
+  } else {
+    // Runs -> my share.  The place of a run in index order is the number of candidates in earlier
+    // chunks: the prefix over the chunk groups (summed by the stream pass) plus a warp scan inside
+    // the group.  Places inside [lo, hi) are mine: the value goes to the shared-memory cache (to
+    // the global list beyond the cache's size), the index to the global list.
+    const uint32_t nchunks = slice_chunks(S), gsh = S.gshift;
+    const uint32_t ngroups = (nchunks + (1u << gsh) - 1u) >> gsh;
+    uint32_t* gpre = sm.hist;                                    // [ngroups + 1] exclusive prefix (hist + red)
+    {
+      static_assert(kGroupsMax == 2 * kFinishThreads && kGroupsMax + 1 <= 2 * kBins, "two groups per thread");
+      const uint32_t ga = 2u * tid, gb = 2u * tid + 1u;
+      const uint32_t ta = ga < ngroups ? L.s.group_total[S.group_begin + ga] : 0u;
+      const uint32_t tb = gb < ngroups ? L.s.group_total[S.group_begin + gb] : 0u;
+      const uint32_t incl = warp_incl_scan(ta + tb);
+      if (lane == 31) sm.warpA[warp] = incl;
+      __syncthreads();
+      uint32_t woff = 0;
+      for (uint32_t w = 0; w < warp; ++w) woff += sm.warpA[w];
+      if (ga < ngroups) gpre[ga + 1] = woff + incl - tb;
+      if (gb < ngroups) gpre[gb + 1] = woff + incl;
+      if (tid == 0) gpre[0] = 0;
+      __syncthreads();
+    }
+    const uint32_t* cstart = L.s.chunk_start + S.chunk_begin;
+    const uint32_t* ccount = L.s.chunk_count + S.chunk_begin;
+    const uint32_t* ridx = L.s.raw_idx + S.cand_off;
+    const float* rval = L.s.raw_val + S.cand_off;
+    auto put = [&](uint32_t at, uint32_t i, float v) {          // candidate (i, v) belongs at place `at`
+      cidx[at] = i;
+      if (at - lo < n_cached) cache[at - lo] = v; else cval[at] = v;
+    };
+    uint32_t g0 = 0;
+    if (n_mine > 0) {                                            // last group that starts at or before lo
+      uint32_t g1 = ngroups;
+      while (g1 - g0 > 1) { const uint32_t mid = (g0 + g1) >> 1; if (gpre[mid] <= lo) g0 = mid; else g1 = mid; }
+    }
+    if (n_mine > 0 && gsh == 5) {
+      // Windows of 32 groups = 1024 chunks.  Each warp places one group's 32 runs (first place and
+      // source of every run -> shared memory); then all threads copy the window's places that lie
+      // inside [lo, hi), kFinishBatch gathers in flight each.
+      uint32_t* dstTab = sm.sel;                                 // [1025] first place of each run of the window
+      uint32_t* srcTab = sm.sel_pre;                             // [1024] where the run sits in the raw buffer
+      for (uint32_t gw = g0; gw < ngroups && gpre[gw] < hi; gw += kFinishWarps) {
+        __syncthreads();                                         // the previous window's tables are free
+        const uint32_t g = gw + warp;
+        {
+          const uint32_t c = (g << 5) + lane;
+          const bool has = g < ngroups && c < nchunks;
+          const uint32_t cnt = has ? __ldg(ccount + c) : 0u;
+          const uint32_t src0 = has ? __ldg(cstart + c) : 0u;
+          const uint32_t incl = warp_incl_scan(cnt);
+          const uint32_t first = (g < ngroups ? gpre[g] : gpre[ngroups]) + incl - cnt;
+          dstTab[warp * 32u + lane] = first;
+          srcTab[warp * 32u + lane] = src0;
+          if (tid == kFinishThreads - 1) dstTab[kFinishThreads] = first + cnt;
+        }
+        __syncthreads();
+        const uint32_t r_lo = max(lo, dstTab[0]), r_hi = min(hi, dstTab[kFinishThreads]);
+        // neighbouring threads take neighbouring places (coalesced gathers and stores); each finds
+        // the run of its place by a 10-step search in the shared-memory table
+        for (uint32_t base = r_lo + tid; base < r_hi; base += kFinishThreads * kFinishBatch) {
+          uint32_t from[kFinishBatch];
+#pragma unroll
+          for (int u = 0; u < kFinishBatch; ++u) {
+            const uint32_t at = base + u * kFinishThreads;
+            from[u] = 0;
+            if (at < r_hi) {
+              uint32_t ci = 0, c1 = kFinishThreads;              // last run that starts at or before `at`
+#pragma unroll
+              for (int step = 0; step < 10; ++step) {
+                const uint32_t mid = (ci + c1) >> 1;
+                if (dstTab[mid] <= at) ci = mid; else c1 = mid;
+              }
+              from[u] = srcTab[ci] + (at - dstTab[ci]);
+            }
+          }
+          uint32_t ri[kFinishBatch];
+          float rv[kFinishBatch];
+#pragma unroll
+          for (int u = 0; u < kFinishBatch; ++u)
+            if (base + u * kFinishThreads < r_hi) { ri[u] = __ldg(ridx + from[u]); rv[u] = __ldg(rval + from[u]); }
+#pragma unroll
+          for (int u = 0; u < kFinishBatch; ++u)
+            if (base + u * kFinishThreads < r_hi) put(base + u * kFinishThreads, ri[u], rv[u]);
+        }
+      }
+    } else if (n_mine > 0) {
+      // very long slices (groups of more than 32 chunks): a warp walks one group at a time
+      for (uint32_t g = g0 + warp; g < ngroups && gpre[g] < hi; g += kFinishWarps) {
+        uint32_t running = gpre[g];
+        const uint32_t c_end = min(nchunks, (g + 1u) << gsh);
+        for (uint32_t c0 = g << gsh; c0 < c_end; c0 += 32u) {
+          const uint32_t c = c0 + lane;
+          const uint32_t cnt = c < c_end ? __ldg(ccount + c) : 0u;
+          const uint32_t src0 = c < c_end ? __ldg(cstart + c) : 0u;
+          const uint32_t incl = warp_incl_scan(cnt);
+          const uint32_t excl = incl - cnt;
+          const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+          if (running + tot > lo && running < hi) {
+            for (uint32_t base = 0; base < tot; base += 32u) {
+              const uint32_t e = base + lane;
+              uint32_t a = 0, b = 32;                            // the run that holds element e: last lane with excl <= e
+#pragma unroll
+              for (int step = 0; step < 5; ++step) {
+                const uint32_t mid = (a + b) >> 1;
+                if (__shfl_sync(0xFFFFFFFFu, excl, mid) <= e) a = mid; else b = mid;
+              }
+              const uint32_t from = __shfl_sync(0xFFFFFFFFu, src0, a) + (e - __shfl_sync(0xFFFFFFFFu, excl, a));
+              const uint32_t at = running + e;
+              if (e < tot && at >= lo && at < hi) put(at, __ldg(ridx + from), __ldg(rval + from));
+            }
+          }
+          running += tot;
+        }
+      }
+    }
   }
   __syncthreads();
-  auto value_at = [&](uint32_t i) -> float { return i < n_cached ? cache[i] : __ldg(cval + lo + i); };
+  auto value_at = [&](uint32_t i) -> float { return i < n_cached ? cache[i] : cval[lo + i]; };
   // visits every key of my share once (order is irrelevant to the callers)
   auto for_each_key = [&](auto&& f) {
     const float4* c4 = reinterpret_cast<const float4*>(cache);
@@ -607,7 +732,7 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
 #pragma unroll
       for (int u = 0; u < kFinishBatch; ++u) {
         const uint32_t i = base + u * kFinishThreads;
-        v[u] = i < n_mine ? __ldg(cval + lo + i) : 0.f;
+        v[u] = i < n_mine ? cval[lo + i] : 0.f;
       }
 #pragma unroll
       for (int u = 0; u < kFinishBatch; ++u)
@@ -616,7 +741,7 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
   };
 
   // keys inside [lo_key, hi_key) over the whole cluster, when known
-  uint32_t bucket_n = (st->flags & FLAG_GENERAL) ? n_cand - n_gt : 0xFFFFFFFFu;
+  uint32_t bucket_n = general ? n_cand - n_gt : 0xFFFFFFFFu;
   for (int round = 0; (hi_key - lo_key > 1u || count_above) && round < 8; ++round) {
     if (!count_above && bucket_n <= (uint32_t)kFinishList) {
       // Few keys are left in the interval: instead of more histogram rounds, every CTA lists its own,
@@ -729,7 +854,7 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
       const float4 x = *reinterpret_cast<const float4*>(cache + i);
       v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
     } else if (i >= n_cached && i + 4u <= n_mine) {
-      const float4 x = __ldg(reinterpret_cast<const float4*>(cval + lo + i));
+      const float4 x = *reinterpret_cast<const float4*>(cval + lo + i);
       v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
     } else {
 #pragma unroll
@@ -793,7 +918,7 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
     // the four indices, fetched now so that no store below waits on a load (the list's capacity is a
     // multiple of 32 entries, so the vector stays inside the slice's list)
     uint4 ci = make_uint4(0u, 0u, 0u, 0u);
-    if (i0 < w_hi) ci = __ldg(reinterpret_cast<const uint4*>(cidx + lo + i0));
+    if (i0 < w_hi) ci = *reinterpret_cast<const uint4*>(cidx + lo + i0);
     const uint32_t cj[4] = {ci.x, ci.y, ci.z, ci.w};
     uint32_t mA = 0, mB = 0;
 #pragma unroll

@@ -6,9 +6,10 @@
 // keeps loads in flight while the consumers work.  The consumers form a = g + m, store it back,
 // flag the keys >= the sampled threshold, and append them -- in index order inside the chunk
 // (packed prefix sums) -- to a run of the slice's raw candidate buffer reserved with one atomicAdd
-// per chunk.  The run's start and length go into a per-chunk table; k_cand_scan / k_cand_gather
-// then lay the runs out in chunk order, which makes the final list independent of the order in
-// which chunks happened to reserve their runs.  No block ever waits on another block.
+// per chunk.  The run's start and length go into a per-chunk table and its length is also added to
+// the total of its chunk group; k_finish then lays the runs out in chunk order, which makes the
+// final list independent of the order in which chunks happened to reserve their runs.  No block
+// ever waits on another block.
 //
 // The only waits are on the block's own mbarriers; they are bounded, and on expiry the error flag
 // is raised and the block leaves through a path every consumer takes together.
@@ -61,6 +62,16 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
   for (int i = 0; i < kWaitLimit; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
+}
+// L2 eviction policy of the candidate runs: they are small and k_finish reads them back, so they
+// should outlive the gradient / residual traffic (which is loaded and stored with streaming hints).
+__device__ __forceinline__ unsigned long long l2_policy_evict_last() {
+  unsigned long long p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void st_hint(uint32_t* ptr, uint32_t v, unsigned long long policy) {
+  asm volatile("st.global.L2::cache_hint.u32 [%0], %1, %2;" ::"l"(ptr), "r"(v), "l"(policy) : "memory");
 }
 // 1-D bulk async copy global -> shared (TMA); src, dst 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
@@ -143,6 +154,7 @@ __global__ void __launch_bounds__(kStreamThreads) k_stream(Launch L, uint32_t to
   }
 
   // -------------------------------------------------------------------- consumers
+  const unsigned long long keep = l2_policy_evict_last();
   uint32_t cur_slice = 0xFFFFFFFFu;
   Slice S;
   uint32_t tau = 0x80000000u;
@@ -208,7 +220,11 @@ __global__ void __launch_bounds__(kStreamThreads) k_stream(Launch L, uint32_t to
       uint32_t bA = 0;
 #pragma unroll
       for (int w = 0; w < kWarps; ++w) bA += sm.wA[buf][w];
-      const uint32_t start = bA ? atomicAdd(&L.s.cursor[cur_slice], bA) : 0u;
+      uint32_t start = 0;
+      if (bA) {
+        start = atomicAdd(&L.s.cursor[cur_slice], bA);
+        atomicAdd(&L.s.group_total[S.group_begin + (d.chunk >> S.gshift)], bA);
+      }
       const uint32_t tile = S.chunk_begin + d.chunk;
       L.s.chunk_start[tile] = start;
       L.s.chunk_count[tile] = bA;
@@ -229,77 +245,13 @@ __global__ void __launch_bounds__(kStreamThreads) k_stream(Launch L, uint32_t to
 #pragma unroll
           for (int j = 0; j < 4; ++j)
             if ((bits >> j) & 1u) {
-              if (pos < S.cand_cap) { cidx[pos] = e + j - head; cval[pos] = a[it][j]; }
+              if (pos < S.cand_cap) { st_hint(cidx + pos, e + j - head, keep); st_hint(reinterpret_cast<uint32_t*>(cval) + pos, __float_as_uint(a[it][j]), keep); }
               ++pos;
             }
         }
         before += (totA >> (it * 8)) & 0xFFu;
       }
     }
-  }
-}
-
-// Chunk-order layout of the raw runs, one block per slice: chunk_dst = exclusive prefix of the
-// chunk counts; the total is the slice's candidate count.
-constexpr int kOrderThreads = 1024;
-__global__ void __launch_bounds__(kOrderThreads) k_cand_scan(Launch L) {
-  __shared__ uint32_t s_warp[32];
-  __shared__ uint32_t s_carry, s_total;
-  const Slice S = L.s.slices[blockIdx.x];
-  if (S.r == S.len) return;
-  const uint32_t n = slice_chunks(S);
-  const uint32_t* cnt = L.s.chunk_count + S.chunk_begin;
-  uint32_t* dst = L.s.chunk_dst + S.chunk_begin;
-  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) s_carry = 0;
-  __syncthreads();
-  for (uint32_t base = 0; base < n; base += kOrderThreads) {
-    const uint32_t c = base + tid;
-    const uint32_t v = c < n ? cnt[c] : 0u;
-    const uint32_t incl = warp_incl_scan(v);
-    if (lane == 31) s_warp[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-      const uint32_t x = s_warp[lane];
-      const uint32_t xi = warp_incl_scan(x);
-      s_warp[lane] = xi - x;
-      if (lane == 31) s_total = xi;
-    }
-    __syncthreads();
-    const uint32_t carry = s_carry;
-    if (c < n) dst[c] = carry + s_warp[warp] + incl - v;
-    __syncthreads();
-    if (tid == 0) s_carry = carry + s_total;
-    __syncthreads();
-  }
-  if (tid == 0) {
-    SelState* st = &L.s.state[blockIdx.x];
-    const uint32_t total = s_carry;
-    st->n_cand = total;
-    st->n_cand_first = total;
-    if (total < S.r || total > S.cand_cap) atomicAdd(&L.s.tickets[3], 1u);   // wakes the exact path
-  }
-}
-
-// Copies every chunk's run to its place in chunk order (one warp per chunk).
-__global__ void __launch_bounds__(kThreads) k_cand_gather(Launch L, uint32_t total_tiles, uint32_t uniform_chunks) {
-  const uint32_t tile = blockIdx.x * kWarps + (threadIdx.x >> 5);
-  if (tile >= total_tiles) return;
-  const uint32_t lane = lane_id();
-  const Slice* slices = L.s.slices;
-  const uint32_t sl = uniform_chunks ? tile / uniform_chunks
-                                     : find_slice(L.n_slices, tile, [&](uint32_t s) { return slices[s].chunk_begin; });
-  const uint32_t count = L.s.chunk_count[tile];
-  if (count == 0) return;
-  const Slice* S = slices + sl;
-  const uint32_t cap = S->cand_cap, off = S->cand_off;
-  if (cap == 0) return;
-  const uint32_t n_cand = L.s.state[sl].n_cand;
-  if (n_cand > cap) return;                       // overflowed: the exact path rebuilds the list
-  const uint32_t src = L.s.chunk_start[tile], dst = L.s.chunk_dst[tile];
-  for (uint32_t i = lane; i < count; i += 32) {
-    L.s.cand_idx[off + dst + i] = L.s.raw_idx[off + src + i];
-    L.s.cand_val[off + dst + i] = L.s.raw_val[off + src + i];
   }
 }
 
