@@ -148,6 +148,18 @@ def test_c5_quarter_billion_coordinates(lib):
     _run_config(lib, cfg, 1, [2])
 
 
+def test_slice_longer_than_2_to_28_uses_wider_chunk_groups(lib):
+    # above 2^28 coordinates a slice has more than 2048 x 32 chunks and k_finish takes its
+    # group-walking layout path; properties only (the oracle's sort of such a row takes minutes)
+    free, _ = torch.cuda.mem_get_info()
+    if free < 16e9:
+        pytest.skip("not enough free device memory on this (shared) GPU")
+    import dataclasses
+    d = (1 << 28) + (1 << 26) + 6
+    cfg = dataclasses.replace(wl.configs()["c5_W1_r100_k10"], d=d, r=d // 1000, k=d // 10000, name="long_slice")
+    _run_config(lib, cfg, 1, [])
+
+
 def test_c5_limits_topk_and_randomk(lib):
     free, _ = torch.cuda.mem_get_info()
     if free < 16e9:
