@@ -356,11 +356,11 @@ def main():
         cpu = {"value": n_rows * d * gsz / sec / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
                "seconds": sec, "sample": f"1 step, {n_rows} of {W} worker rows, step-0 gradient, zero residual"}
 
-    # launches per step of this library's kernels (memsets and copies not counted)
-    if cfg.r == cfg.d:
-        per_step = 3 + 2 + 1 + 2          # subset (3), threshold + stream, emit_all, aggregate (2)
-    else:
-        per_step = (3 if cfg.k < cfg.r or seg else 0) + 2 + 4 + 3 + 1 + 2
+    # launches per step of this library's kernels (memsets and copies not counted):
+    # k_draw, k_resolve, k_sel_scan (unless k = r), k_sample, k_stream, then either k_exact + k_finish
+    # (r < d) or k_emit_all (r = d), then k_agg_starts and one aggregate kernel
+    subset = 3 if (seg or cfg.k < cfg.r) else 0
+    per_step = subset + 2 + (1 if cfg.r == cfg.d and not seg else 2) + 2
     if rank == 0:
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -48,7 +48,8 @@ struct Slice {
   uint32_t hist_begin;  // first histogram block
   uint32_t group_begin; // first entry of the slice in the chunk-group totals
   uint32_t samp_off;    // start in the draw buffer (k entries)
-  uint32_t first_off;   // start in the first-occurrence table (r entries)
+  uint32_t first_off;   // start in the first-occurrence table
+  uint32_t first_mask;  // 0: the table is dense (r entries); else it is a hash table of first_mask + 1 slots
   uint32_t sel_off;     // start in the selection bitmap / its prefix counts (32-bit words)
   uint32_t gshift;      // a chunk group is 2^gshift consecutive chunks (at most kGroupsMax groups per slice)
 };
@@ -88,6 +89,7 @@ struct Scratch {
   uint32_t* first;        // first-occurrence table F
   uint32_t* sel;          // selection bitmap over positions
   uint32_t* sel_pre;      // exclusive popcount prefix per bitmap word
+  uint32_t* sel_blk;      // selected positions per chunk of bitmap words (scan scratch)
   uint32_t* error;        // device error flags
 };
 

@@ -43,6 +43,8 @@ struct rtopk_ctx {
   size_t cand_entries = 0;
   uint32_t* d_draws = nullptr;
   uint32_t* d_sel_pre = nullptr;
+  uint32_t* d_sel_blk = nullptr;
+  size_t sel_blk_entries = 0;
   size_t sel_words = 0;
   uint32_t* d_error = nullptr;
   uint32_t* d_agg_starts = nullptr;
@@ -99,8 +101,18 @@ struct DeviceGuard {
 };
 
 uint32_t cand_capacity(uint64_t len, uint64_t r) {
-  const uint64_t c = 2 * r + 1024;
+  const uint64_t c = 3 * r + 4096;   // room for the sampled bracket's margin at small r / d
   return (uint32_t)(((c < len ? c : len) + 31u) & ~31ull);     // multiples of 32 keep every list 128-byte aligned
+}
+
+// First-occurrence table of the k-of-r subset: dense (r entries) while r <= 16 k, else a hash table of
+// at least 2 k slots (keys | firsts).  Returns the entries it takes and sets the slice's mask.
+uint64_t first_table_entries(Slice& sl) {
+  if ((uint64_t)sl.r <= 16ull * sl.k) { sl.first_mask = 0; return sl.r; }
+  uint32_t slots = 64;
+  while (slots < 2u * sl.k) slots <<= 1;
+  sl.first_mask = slots - 1;
+  return 2ull * slots;
 }
 
 // Layout of one call: the slice table plus every per-call scratch offset.
@@ -108,7 +120,7 @@ struct Plan {
   std::vector<Slice> slices;
   uint32_t n_chunks = 0, n_hist_blocks = 0, n_groups = 0;
   size_t cand_entries = 0, draw_entries = 0, first_entries = 0, sel_words = 0;
-  uint32_t k_draw_max = 0, words_all_max = 0, cap_max = 0, chunks_max = 0;
+  uint32_t k_draw_max = 0, words_all_max = 0, cap_max = 0, chunks_max = 0, sel_words_max = 0;
   bool any_select = false, any_sampler = false, any_all = false;
   bool uniform = false;               // every slice has the same number of chunks (plain calls)
   uint32_t K_row = 0;
@@ -176,8 +188,9 @@ int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32
       sl.sel_off = (uint32_t)selw;
       if (sl.k < sl.r) {
         draws += sl.k;
-        first += sl.r;
+        first += first_table_entries(sl);
         selw += (sl.r + 31) / 32;
+        if ((sl.r + 31) / 32 > P.sel_words_max) P.sel_words_max = (sl.r + 31) / 32;
         P.any_sampler = true;
         if (sl.k > P.k_draw_max) P.k_draw_max = sl.k;
       }
@@ -291,7 +304,10 @@ int run_sampler(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st)
   const dim3 grid((P.k_draw_max + kDrawThreads - 1) / kDrawThreads, n);
   k_draw<<<grid, kDrawThreads, 0, st>>>(L);
   k_resolve<<<grid, kDrawThreads, 0, st>>>(L);
-  k_sel_scan<<<n, kScanThreads, 0, st>>>(L);
+  const dim3 sgrid((P.sel_words_max + kSelChunk - 1) / kSelChunk, n);
+  if ((size_t)sgrid.x * n > ctx->sel_blk_entries) return RTOPK_ERR_INVALID_ARG;
+  k_sel_count<<<sgrid, kScanThreads, 0, st>>>(L);
+  k_sel_scan<<<sgrid, kScanThreads, 0, st>>>(L);
   return RTOPK_OK;
 }
 
@@ -320,7 +336,7 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   if ((size_t)P.n_chunks > ctx->chunk_tab_entries) return RTOPK_ERR_INVALID_ARG;
   L.s.chunk_start = ctx->d_chunk_tab;
   L.s.chunk_count = ctx->d_chunk_tab + ctx->chunk_tab_entries;
-  L.s.draws = ctx->d_draws; L.s.first = ctx->d_first; L.s.sel_pre = ctx->d_sel_pre;
+  L.s.draws = ctx->d_draws; L.s.first = ctx->d_first; L.s.sel_pre = ctx->d_sel_pre; L.s.sel_blk = ctx->d_sel_blk;
   L.s.error = ctx->d_error;
   L.grad = grad; L.residual = residual; L.msg_idx = msg_idx; L.msg_val = msg_val;
   L.n_slices = (uint32_t)P.slices.size();
@@ -449,10 +465,10 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   if (!guard.ok) { delete ctx; return RTOPK_ERR_CUDA; }
   const size_t W = (size_t)W_max, S = (size_t)segments_max, slices = W * S;
   const size_t chunks = W * ((size_t)d_max / kChunk + 2 * S + 1);
-  const size_t cand_row = std::min<size_t>((size_t)d_max, 2 * (size_t)r_max + 1024 * S) + 32 * S;
+  const size_t cand_row = std::min<size_t>((size_t)d_max, 3 * (size_t)r_max + 4096 * S) + 32 * S;
   const size_t groups = W * ((size_t)d_max / kChunk / 32 + 2 * S + 1);
   ctx->cand_entries = W * cand_row;
-  ctx->first_entries = W * (size_t)r_max;
+  ctx->first_entries = W * (std::min<size_t>((size_t)r_max, 16 * (size_t)k_max) + 128 * S);
   ctx->sel_words = W * ((size_t)r_max / 32 + S + 1);
   ctx->zero_bytes = zero_region_bytes(slices, chunks, groups, ctx->sel_words);
   ctx->agg_start_entries = W * ((size_t)(d_max + kAggTile - 1) / kAggTile + 2);
@@ -471,6 +487,8 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   alloc((void**)&ctx->d_chunk_tab, 2 * chunks * sizeof(uint32_t));
   alloc((void**)&ctx->d_draws, W * (size_t)k_max * sizeof(uint32_t));
   alloc((void**)&ctx->d_sel_pre, ctx->sel_words * sizeof(uint32_t));
+  ctx->sel_blk_entries = slices * ((size_t)r_max / 32 / kSelChunk + 2);
+  alloc((void**)&ctx->d_sel_blk, ctx->sel_blk_entries * sizeof(uint32_t));
   alloc((void**)&ctx->d_error, 16);
   alloc((void**)&ctx->d_agg_starts, ctx->agg_start_entries * sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_sample<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSampleSmemBytes);
@@ -528,7 +546,7 @@ int rtopk_destroy(rtopk_ctx* ctx) {
   DeviceGuard guard(ctx->device);
   void* ptrs[] = {ctx->d_slices, ctx->d_state, ctx->d_zero, ctx->d_first, ctx->d_cand_idx, ctx->d_cand_val,
                   ctx->d_raw_idx, ctx->d_raw_val, ctx->d_chunk_tab,
-                  ctx->d_draws, ctx->d_sel_pre, ctx->d_error, ctx->d_agg_starts, ctx->d_stage};
+                  ctx->d_draws, ctx->d_sel_pre, ctx->d_sel_blk, ctx->d_error, ctx->d_agg_starts, ctx->d_stage};
   for (void* p : ptrs) if (p) cudaFree(p);
   for (cudaEvent_t ev : ctx->ev) if (ev) cudaEventDestroy(ev);
   if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
@@ -652,14 +670,16 @@ int rtopk_sample_positions(rtopk_ctx* ctx, int64_t r, int64_t k, uint64_t seed, 
   sl.len = (uint32_t)r; sl.r = (uint32_t)r; sl.k = (uint32_t)k; sl.row = 0; sl.segment = segment;
   P.any_sampler = k < r;
   P.k_draw_max = (uint32_t)k;
-  P.first_entries = (size_t)r;
+  P.first_entries = k < r ? (size_t)first_table_entries(sl) : 0;
+  if (P.first_entries > ctx->first_entries) return RTOPK_ERR_INVALID_ARG;
   P.sel_words = ((size_t)r + 31) / 32;
+  P.sel_words_max = (uint32_t)P.sel_words;
   Launch L;
   std::memset(&L, 0, sizeof(L));
   const size_t zbytes = carve_zero(ctx, P, L.s);
   if (zbytes > ctx->zero_bytes) return RTOPK_ERR_INVALID_ARG;
   L.s.slices = ctx->d_slices; L.s.state = ctx->d_state; L.s.draws = ctx->d_draws; L.s.first = ctx->d_first;
-  L.s.sel_pre = ctx->d_sel_pre; L.s.error = ctx->d_error;
+  L.s.sel_pre = ctx->d_sel_pre; L.s.sel_blk = ctx->d_sel_blk; L.s.error = ctx->d_error;
   L.n_slices = 1; L.worker_base = worker; L.seed_lo = (uint32_t)seed; L.seed_hi = (uint32_t)(seed >> 32);
   L.step = step;
   int rc = upload_slices(ctx, P, st);
@@ -733,7 +753,8 @@ constexpr size_t kStaticDrawsOff = kStaticSliceBytes;
 constexpr size_t kStaticFirstOff = kStaticDrawsOff + kStaticR * 4;
 constexpr size_t kStaticSelOff = kStaticFirstOff + kStaticR * 4;
 constexpr size_t kStaticPreOff = kStaticSelOff + (kStaticR / 32 + 8) * 4;
-constexpr size_t kStaticBytes = kStaticPreOff + (kStaticR / 32 + 8) * 4;
+constexpr size_t kStaticBlkOff = kStaticPreOff + (kStaticR / 32 + 8) * 4;
+constexpr size_t kStaticBytes = kStaticBlkOff + 256;
 static_assert(sizeof(Slice) <= kStaticSliceBytes, "slice descriptor must fit its slot");
 }  // namespace
 
@@ -750,7 +771,7 @@ __global__ void k_static_slice(Slice* slot, uint32_t r, uint32_t k, uint32_t seg
   Slice s;
   s.g_off = 0; s.m_off = 0; s.len = r; s.r = r; s.k = k; s.row = 0; s.segment = segment; s.idx_base = 0;
   s.head = 0; s.msg_off = 0; s.cand_off = 0; s.cand_cap = 0; s.chunk_begin = 0; s.hist_begin = 0;
-  s.group_begin = 0; s.samp_off = 0; s.first_off = 0; s.sel_off = 0; s.gshift = 5;
+  s.group_begin = 0; s.samp_off = 0; s.first_off = 0; s.first_mask = 0; s.sel_off = 0; s.gshift = 5;
   *slot = s;
 }
 }  // namespace
@@ -780,6 +801,7 @@ int rtopk_sample_positions_static(int64_t r, int64_t k, uint64_t seed, uint32_t 
   L.s.first = reinterpret_cast<uint32_t*>(base + kStaticFirstOff);
   L.s.sel = reinterpret_cast<uint32_t*>(base + kStaticSelOff);
   L.s.sel_pre = reinterpret_cast<uint32_t*>(base + kStaticPreOff);
+  L.s.sel_blk = reinterpret_cast<uint32_t*>(base + kStaticBlkOff);
   L.n_slices = 1; L.worker_base = worker; L.seed_lo = (uint32_t)seed; L.seed_hi = (uint32_t)(seed >> 32);
   L.step = step;
   const uint32_t nwords = (uint32_t)((r + 31) / 32);
@@ -791,7 +813,9 @@ int rtopk_sample_positions_static(int64_t r, int64_t k, uint64_t seed, uint32_t 
     const dim3 grid(((uint32_t)k + kDrawThreads - 1) / kDrawThreads, 1);
     k_draw<<<grid, kDrawThreads, 0, st>>>(L);
     k_resolve<<<grid, kDrawThreads, 0, st>>>(L);
-    k_sel_scan<<<1, kScanThreads, 0, st>>>(L);
+    const dim3 sgrid((nwords + kSelChunk - 1) / kSelChunk, 1);   // at most 4 chunks at the largest r
+    k_sel_count<<<sgrid, kScanThreads, 0, st>>>(L);
+    k_sel_scan<<<sgrid, kScanThreads, 0, st>>>(L);
   }
   k_positions<<<(nwords + kThreads - 1) / kThreads, kThreads, 0, st>>>(L, pos);
   return cudaGetLastError() == cudaSuccess ? RTOPK_OK : RTOPK_ERR_CUDA;

@@ -111,7 +111,7 @@ __global__ void k_init_state(Launch L, uint32_t general) {
 // thread keeps only the maximum of each group of 4 sampled keys, and the rho-th largest of these
 // 8192 maxima is a lower bound of the rho-th largest key (there are at least rho keys that large;
 // with groups this small the bound is within a few per cent of the exact sample rank).  tau_lo is that bound at
-// rank expect + 6 sigma; tau_hi the same at rank (expect - 6 sigma) * 3/4, which as a sample rank
+// rank expect + 4.5 sigma; tau_hi the same at rank (expect - 4.5 sigma) * 3/4, which as a sample rank
 // stays clearly above the r-th largest.  Samples whose ranks exceed the thread count take a radix
 // select over all sample keys instead.
 constexpr int kSampleHold = 8;   // maxima a thread keeps (one per 4 sampled keys)
@@ -206,7 +206,7 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(Launch L) {
       }
     }
     const float expect = (float)n_s * ((float)S.r / (float)S.len);
-    const float margin = 6.0f * sqrtf(expect) + 8.0f;
+    const float margin = 4.5f * sqrtf(expect) + 4.0f;             // a miss (about 3e-6 per slice) costs one exact pass
     rho_lo = expect + margin >= (float)n_s ? n_s : (uint32_t)(expect + margin);
     rho_hi = expect - margin < 2.0f ? 1u : (uint32_t)((expect - margin) * 0.75f);
   }
