@@ -21,12 +21,33 @@ constexpr int kAggStage = 1024;   // entries of one output tile staged in shared
 constexpr int kAggSparseTile = 16384;   // output coordinates per block of the sparse kernel
 constexpr int kAggSparseStage = 2048;   // entries of one such tile staged in shared memory
 constexpr int kAggMaxW = 1024;    // workers the sparse kernel keeps run tables for
+constexpr int kAggSearchW = 64;   // up to this many workers the sparse kernel finds the runs itself
 
 __device__ __forceinline__ uint32_t lower_bound_u32(const uint32_t* a, uint32_t n, uint32_t key) {
   uint32_t lo = 0, hi = n;
   while (lo < hi) {
     const uint32_t mid = (lo + hi) >> 1;
     if (__ldg(a + mid) < key) lo = mid + 1; else hi = mid;
+  }
+  return lo;
+}
+
+// The same as a 16-way search by each half of a warp (lanes 0-15 share one key, lanes 16-31
+// another): every lane of a half returns that half's lower bound.  a is sorted ascending.
+__device__ __forceinline__ uint32_t half_warp_lower_bound(const uint32_t* a, uint32_t n, uint32_t key, uint32_t lane) {
+  const uint32_t l = lane & 15u, sh = lane & 16u;
+  uint32_t lo = 0, hi = n;                                   // the answer lies in [lo, hi]
+  // both halves run the same number of steps (the range shrinks 16-fold per step whatever the key)
+  for (uint32_t span = n; span > 0; span = span > 16u ? (span + 15u) / 16u - 1u : 0u) {
+    const uint32_t step = (hi - lo + 15u) / 16u;              // 0 once this half is done
+    const uint32_t probe = min(lo + (l + 1u) * step, hi) - 1u; // < hi; unused when step == 0
+    const bool less = step != 0u && __ldg(a + (step ? probe : 0u)) < key;
+    const uint32_t cnt = __popc((__ballot_sync(0xFFFFFFFFu, less) >> sh) & 0xFFFFu);
+    if (step != 0u) {
+      const uint32_t nlo = min(hi, lo + cnt * step);
+      hi = min(hi, lo + (cnt + 1u) * step - 1u);
+      lo = nlo;
+    }
   }
   return lo;
 }
@@ -135,7 +156,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(const uint32_t
                                                                   const uint32_t* __restrict__ starts, uint32_t d,
                                                                   uint32_t W, uint32_t K, int mean,
                                                                   float* __restrict__ out) {
-  __shared__ uint32_t s_beg[kAggMaxW], s_pre[kAggMaxW + 1];
+  __shared__ uint32_t s_beg[kAggMaxW], s_pre[kAggMaxW + 1], s_cnt[kAggSearchW];
   __shared__ uint32_t st_idx[kAggSparseStage];
   __shared__ float st_val[kAggSparseStage];
   __shared__ uint32_t s_warp[kAggThreads / 32];
@@ -145,14 +166,31 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(const uint32_t
   const uint32_t lo = blockIdx.x * (uint32_t)kAggSparseTile;
   if (tid == 0) s_carry = 0;
   __syncthreads();
+  if (starts == nullptr) {
+    // no table of run starts: a warp per worker finds the run of this tile in the worker's sorted
+    // row, half the warp searching for each end (16-way search: a few dependent loads)
+    for (uint32_t w = warp; w < W; w += kAggThreads / 32) {
+      const uint32_t* row = msg_idx + (size_t)w * K;
+      const uint32_t end = lo > 0xFFFFFFFFu - (uint32_t)kAggSparseTile ? 0xFFFFFFFFu : lo + (uint32_t)kAggSparseTile;
+      const uint32_t key = lane < 16 ? lo : end;                 // every index is below 2^32 - 1
+      const uint32_t at = half_warp_lower_bound(row, K, key, lane);
+      const uint32_t e = __shfl_sync(0xFFFFFFFFu, at, 16);
+      if (lane == 0) { s_beg[w] = at; s_cnt[w] = e - at; }
+    }
+    __syncthreads();
+  }
   for (uint32_t w0 = 0; w0 < W; w0 += kAggThreads) {
     const uint32_t w = w0 + tid;
     uint32_t cnt = 0;
     if (w < W) {
-      const uint32_t* st = starts + (size_t)w * (ntiles + 1) + blockIdx.x;
-      const uint32_t b = __ldg(st), e = __ldg(st + 1);
-      s_beg[w] = b;
-      cnt = e > b ? e - b : 0u;
+      if (starts != nullptr) {
+        const uint32_t* st = starts + (size_t)w * (ntiles + 1) + blockIdx.x;
+        const uint32_t b = __ldg(st), e = __ldg(st + 1);
+        s_beg[w] = b;
+        cnt = e > b ? e - b : 0u;
+      } else {
+        cnt = s_cnt[w];
+      }
     }
     const uint32_t incl = warp_incl_scan(cnt);
     if (lane == 31) s_warp[warp] = incl;

@@ -70,7 +70,7 @@ struct rtopk_ctx {
 namespace {
 
 constexpr int kVersion = 100;
-constexpr size_t kSampleSmemBytes = (size_t)(kSampleMax + kBins + 64) * sizeof(uint32_t);
+constexpr size_t kSampleSmemBytes = (size_t)(kSampleMax + 2 * kBins + 64) * sizeof(uint32_t);
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -411,13 +411,18 @@ int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val
   if ((size_t)W * (ntiles + 1) > ctx->agg_start_entries) return RTOPK_ERR_INVALID_ARG;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return RTOPK_ERR_CUDA;
-  const dim3 sgrid((ntiles + 1 + kAggThreads - 1) / kAggThreads, (uint32_t)W);
-  k_agg_starts<<<sgrid, kAggThreads, 0, st>>>(msg_idx, (uint32_t)W, (uint32_t)k, ntiles, tile, ctx->d_agg_starts);
+  // with few workers and tiles the sparse kernel finds every tile's runs itself (one launch fewer);
+  // otherwise a table of run starts is built first, all searches side by side
+  const bool own_search = sparse && W <= kAggSearchW && (uint64_t)ntiles * (uint64_t)((W + 7) / 8) <= 4096u;
+  if (!own_search) {
+    const dim3 sgrid((ntiles + 1 + kAggThreads - 1) / kAggThreads, (uint32_t)W);
+    k_agg_starts<<<sgrid, kAggThreads, 0, st>>>(msg_idx, (uint32_t)W, (uint32_t)k, ntiles, tile, ctx->d_agg_starts);
+  }
   const int mean = scale_mode == RTOPK_SCALE_MEAN ? 1 : 0;
   if (sparse) {
     // few coordinates are touched: clear the update, then compute only what was sent
     if (!out_cleared) RTOPK_CUDA(ctx, cudaMemsetAsync(out, 0, (size_t)d * sizeof(float), st));
-    k_aggregate_sparse<<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, ctx->d_agg_starts, (uint32_t)d,
+    k_aggregate_sparse<<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, own_search ? nullptr : ctx->d_agg_starts, (uint32_t)d,
                                                        (uint32_t)W, (uint32_t)k, mean, out);
   } else {
     k_aggregate<<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, ctx->d_agg_starts, (uint32_t)d, (uint32_t)W,

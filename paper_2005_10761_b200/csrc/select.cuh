@@ -116,34 +116,88 @@ __global__ void k_init_state(Launch L, uint32_t general) {
 // select over all sample keys instead.
 constexpr int kSampleHold = 8;   // maxima a thread keeps (one per 4 sampled keys)
 
-// rank-th largest (1-based) of the held keys of all threads: slot u of thread t is in use iff
-// t + u * blockDim.x < n_held.  Three radix passes of at most kSampleHold increments per thread.
-__device__ __forceinline__ uint32_t block_select_desc(const uint32_t (&key)[kSampleHold], uint32_t n_held,
-                                                      uint32_t rank, uint32_t* hist, uint32_t* scratch) {
-  uint32_t prefix = 0, need = rank;
-  for (int pass = 0; pass < 3; ++pass) {
-    const int bits = digit_bits(pass), shift = digit_shift(pass);
-    for (uint32_t b = threadIdx.x; b < (uint32_t)kBins; b += blockDim.x) hist[b] = 0;
-    __syncthreads();
-#pragma unroll
-    for (int u = 0; u < kSampleHold; ++u)
-      if (threadIdx.x + u * blockDim.x < n_held && (pass == 0 || (key[u] >> (shift + bits)) == prefix))
-        atomicAdd(&hist[(key[u] >> shift) & ((1u << bits) - 1u)], 1u);
-    __syncthreads();
-    uint32_t D, above;
-    pick_digit(hist, 1 << bits, need, scratch, D, above);
-    need -= above;
-    prefix = (prefix << bits) | D;
+// Two ranks at once in two histograms of kBins bins whose totals stay below 2^16 (ha == hb is
+// allowed): the counts travel packed, a's in the low and b's in the high half of a word, so one
+// block scan serves both.  For each: the digit D with count(> D) < need <= count(>= D), and
+// count(> D).  Called by all kSampleThreads threads; scratch holds 32 + 4 words.  A digit of
+// 0xFFFFFFFF means the histogram holds fewer than `need` keys.
+__device__ __forceinline__ void pick_two(const uint32_t* ha, const uint32_t* hb, uint32_t need_a, uint32_t need_b,
+                                         uint32_t* scratch, uint32_t& Da, uint32_t& above_a, uint32_t& Db, uint32_t& above_b) {
+  static_assert(kBins == 2 * kSampleThreads, "two bins per thread");
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  const int hi = kBins - 1 - 2 * (int)tid;                      // thread 0 holds the largest digits
+  const uint32_t p0 = ha[hi] | (hb[hi] << 16), p1 = ha[hi - 1] | (hb[hi - 1] << 16);
+  const uint32_t mine = p0 + p1;
+  uint32_t incl = warp_incl_scan(mine);
+  if (lane == 31) scratch[warp] = incl;
+  if (tid == 0) { scratch[32] = 0xFFFFFFFFu; scratch[33] = 0; scratch[34] = 0xFFFFFFFFu; scratch[35] = 0; }
+  __syncthreads();
+  {
+    const uint32_t wt = scratch[lane];
+    const uint32_t wincl = warp_incl_scan(wt);
+    incl += __shfl_sync(0xFFFFFFFFu, wincl - wt, warp);
   }
-  return prefix;
+  const uint32_t excl = incl - mine;
+  {
+    const uint32_t ex = excl & 0xFFFFu, in = incl & 0xFFFFu, h0 = p0 & 0xFFFFu;
+    if (ex < need_a && need_a <= in) {
+      if (ex + h0 >= need_a) { scratch[32] = (uint32_t)hi; scratch[33] = ex; }
+      else { scratch[32] = (uint32_t)(hi - 1); scratch[33] = ex + h0; }
+    }
+  }
+  {
+    const uint32_t ex = excl >> 16, in = incl >> 16, h0 = p0 >> 16;
+    if (ex < need_b && need_b <= in) {
+      if (ex + h0 >= need_b) { scratch[34] = (uint32_t)hi; scratch[35] = ex; }
+      else { scratch[34] = (uint32_t)(hi - 1); scratch[35] = ex + h0; }
+    }
+  }
+  __syncthreads();
+  Da = scratch[32]; above_a = scratch[33]; Db = scratch[34]; above_b = scratch[35];
+}
+
+// The rank_a-th and rank_b-th largest (1-based) of the held keys of all threads, to 22 of the 31
+// key bits: slot u of thread t is in use iff t + u * blockDim.x < n_held (fewer than 2^16 in all).
+// pa <= the rank_a-th largest key <= pa + 511, and the same for pb.  Two radix passes of at most
+// kSampleHold (then 2 * kSampleHold) shared-memory increments per thread; hist holds 2 * kBins words.
+__device__ __forceinline__ void block_select_two(const uint32_t (&key)[kSampleHold], uint32_t n_held,
+                                                 uint32_t rank_a, uint32_t rank_b, uint32_t* hist, uint32_t* scratch,
+                                                 uint32_t& pa, uint32_t& pb) {
+  const uint32_t tid = threadIdx.x;
+  uint32_t* ha = hist;
+  uint32_t* hb = hist + kBins;
+  for (uint32_t b = tid; b < 2u * kBins; b += blockDim.x) hist[b] = 0;
+  __syncthreads();
+#pragma unroll
+  for (int u = 0; u < kSampleHold; ++u)
+    if (tid + u * blockDim.x < n_held) atomicAdd(&ha[key[u] >> 20], 1u);
+  __syncthreads();
+  uint32_t Da, Db, above_a, above_b;
+  pick_two(ha, ha, rank_a, rank_b, scratch, Da, above_a, Db, above_b);
+  const uint32_t need_a = rank_a - above_a, need_b = rank_b - above_b;
+  __syncthreads();                                               // everyone has read pass 0's result
+  for (uint32_t b = tid; b < (uint32_t)kBins; b += blockDim.x) ha[b] = 0;
+  __syncthreads();
+#pragma unroll
+  for (int u = 0; u < kSampleHold; ++u)
+    if (tid + u * blockDim.x < n_held) {
+      const uint32_t top = key[u] >> 20, next = (key[u] >> 9) & 0x7FFu;
+      if (top == Da) atomicAdd(&ha[next], 1u);
+      if (top == Db) atomicAdd(&hb[next], 1u);
+    }
+  __syncthreads();
+  uint32_t Ea, Eb;
+  pick_two(ha, hb, need_a, need_b, scratch, Ea, above_a, Eb, above_b);
+  pa = Da == 0xFFFFFFFFu || Ea == 0xFFFFFFFFu ? 0u : ((Da << 11) | Ea) << 9;
+  pb = Db == 0xFFFFFFFFu || Eb == 0xFFFFFFFFu ? 0x7FFFFE00u : ((Db << 11) | Eb) << 9;
 }
 
 template <typename GradT>
 __global__ void __launch_bounds__(kSampleThreads) k_sample(Launch L) {
   extern __shared__ uint32_t smem[];
   uint32_t* keys = smem;                       // [kSampleMax]
-  uint32_t* hist = smem + kSampleMax;          // [kBins]
-  uint32_t* scratch = hist + kBins;            // [64]
+  uint32_t* hist = smem + kSampleMax;          // [2 * kBins]
+  uint32_t* scratch = hist + 2 * kBins;        // [64]
   const uint32_t sl = blockIdx.x;
   const Slice S = L.s.slices[sl];
   const uint32_t tid = threadIdx.x;
@@ -213,8 +267,9 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(Launch L) {
   __syncthreads();
   uint32_t tau_lo, tau_hi;
   if (rho_lo <= n_held) {
-    tau_lo = block_select_desc(mine, n_held, rho_lo, hist, scratch);
-    tau_hi = block_select_desc(mine, n_held, rho_hi, hist, scratch);
+    // 22 of the 31 key bits are enough for estimates: tau_lo rounds down, tau_hi up
+    block_select_two(mine, n_held, rho_lo, rho_hi, hist, scratch, tau_lo, tau_hi);
+    tau_hi |= 0x1FFu;
   } else {
     // radix select of the rho_lo-th largest over all sample keys; no upper estimate
     uint32_t prefix = 0, need = rho_lo;
@@ -530,7 +585,9 @@ constexpr int kFinishThreads = 1024;
 constexpr int kFinishWarps = kFinishThreads / 32;
 constexpr int kFinishCache = 46 * 1024;   // candidate values a CTA keeps in shared memory (184 KB)
 constexpr int kFinishBatch = 8;           // independent loads in flight per thread
-constexpr int kFinishList = 512;         // bucket population up to which the bucket is ranked directly
+constexpr int kRunBatch = 4;              // runs a lane group copies at a time
+constexpr int kFinishList = 512;          // bucket population up to which the bucket is ranked directly
+constexpr int kFinishListLong = 2048;     // ... when the CTAs' shares are long (must fit hist / red)
 constexpr int kFinishSelWords = 2048;     // bitmap words (64 Ki positions) a CTA keeps in shared memory
 
 struct alignas(16) FinishSmem {           // the value cache behind it is read as float4
@@ -609,6 +666,7 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
     uint32_t* gpre = sm.hist;                                    // [ngroups + 1] exclusive prefix (hist + red)
     {
       static_assert(kGroupsMax == 2 * kFinishThreads && kGroupsMax + 1 <= 2 * kBins, "two groups per thread");
+      static_assert(kFinishThreads == 1024 && kFinishWarps == 32, "a window is 1024 chunks, scanned by 32 warps");
       const uint32_t ga = 2u * tid, gb = 2u * tid + 1u;
       const uint32_t ta = ga < ngroups ? L.s.group_total[S.group_begin + ga] : 0u;
       const uint32_t tb = gb < ngroups ? L.s.group_total[S.group_begin + gb] : 0u;
@@ -635,83 +693,75 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
       uint32_t g1 = ngroups;
       while (g1 - g0 > 1) { const uint32_t mid = (g0 + g1) >> 1; if (gpre[mid] <= lo) g0 = mid; else g1 = mid; }
     }
-    if (n_mine > 0 && gsh == 5) {
-      // Windows of 32 groups = 1024 chunks.  Each warp places one group's 32 runs (first place and
-      // source of every run -> shared memory); then all threads copy the window's places that lie
-      // inside [lo, hi), kFinishBatch gathers in flight each.
+    if (n_mine > 0) {
+      // Windows of kFinishThreads chunks (a whole number of groups: a group has at most as many
+      // chunks as a window).  One thread per chunk: the first place and the source of its run go to
+      // shared memory (block scan on top of the group prefix); then all threads copy the window's
+      // places that lie inside [lo, hi), kFinishBatch gathers in flight each.
       uint32_t* dstTab = sm.sel;                                 // [1025] first place of each run of the window
       uint32_t* srcTab = sm.sel_pre;                             // [1024] where the run sits in the raw buffer
-      for (uint32_t gw = g0; gw < ngroups && gpre[gw] < hi; gw += kFinishWarps) {
+      const uint32_t gpw = 10u - gsh;                            // log2(groups per window)
+      const uint32_t G = n_cand / nchunks < 16u ? 8u : 32u;      // lanes per run
+      for (uint32_t wi = g0 >> gpw; (wi << 10) < nchunks && gpre[wi << gpw] < hi; ++wi) {
+        const uint32_t c = (wi << 10) + tid;
+        const bool has = c < nchunks;
+        const uint32_t cnt = has ? __ldg(ccount + c) : 0u;
+        const uint32_t src0 = has ? __ldg(cstart + c) : 0u;
+        const uint32_t incl = warp_incl_scan(cnt);
         __syncthreads();                                         // the previous window's tables are free
-        const uint32_t g = gw + warp;
+        if (lane == 31) sm.warpA[warp] = incl;
+        __syncthreads();
+        uint32_t first = gpre[wi << gpw] + incl - cnt;
         {
-          const uint32_t c = (g << 5) + lane;
-          const bool has = g < ngroups && c < nchunks;
-          const uint32_t cnt = has ? __ldg(ccount + c) : 0u;
-          const uint32_t src0 = has ? __ldg(cstart + c) : 0u;
-          const uint32_t incl = warp_incl_scan(cnt);
-          const uint32_t first = (g < ngroups ? gpre[g] : gpre[ngroups]) + incl - cnt;
-          dstTab[warp * 32u + lane] = first;
-          srcTab[warp * 32u + lane] = src0;
-          if (tid == kFinishThreads - 1) dstTab[kFinishThreads] = first + cnt;
+          const uint32_t wt = sm.warpA[lane];
+          const uint32_t wincl = warp_incl_scan(wt);
+          first += __shfl_sync(0xFFFFFFFFu, wincl - wt, warp);
         }
+        dstTab[tid] = first;
+        srcTab[tid] = src0;
+        if (tid == kFinishThreads - 1) dstTab[kFinishThreads] = first + cnt;
         __syncthreads();
         const uint32_t r_lo = max(lo, dstTab[0]), r_hi = min(hi, dstTab[kFinishThreads]);
-        // neighbouring threads take neighbouring places (coalesced gathers and stores); each finds
-        // the run of its place by a 10-step search in the shared-memory table
-        for (uint32_t base = r_lo + tid; base < r_hi; base += kFinishThreads * kFinishBatch) {
-          uint32_t from[kFinishBatch];
+        if (r_lo >= r_hi) continue;
+        // the window's runs that reach into [r_lo, r_hi): j_lo .. j_hi (block-uniform searches)
+        uint32_t j_lo = 0, j_hi = 0;
+        {
+          uint32_t c1 = kFinishThreads, d1 = kFinishThreads;
 #pragma unroll
-          for (int u = 0; u < kFinishBatch; ++u) {
-            const uint32_t at = base + u * kFinishThreads;
-            from[u] = 0;
-            if (at < r_hi) {
-              uint32_t ci = 0, c1 = kFinishThreads;              // last run that starts at or before `at`
-#pragma unroll
-              for (int step = 0; step < 10; ++step) {
-                const uint32_t mid = (ci + c1) >> 1;
-                if (dstTab[mid] <= at) ci = mid; else c1 = mid;
-              }
-              from[u] = srcTab[ci] + (at - dstTab[ci]);
-            }
+          for (int step = 0; step < 10; ++step) {
+            const uint32_t ma = (j_lo + c1) >> 1, mb = (j_hi + d1) >> 1;
+            if (dstTab[ma] <= r_lo) j_lo = ma; else c1 = ma;
+            if (dstTab[mb] < r_hi) j_hi = mb; else d1 = mb;
           }
-          uint32_t ri[kFinishBatch];
-          float rv[kFinishBatch];
-#pragma unroll
-          for (int u = 0; u < kFinishBatch; ++u)
-            if (base + u * kFinishThreads < r_hi) { ri[u] = __ldg(ridx + from[u]); rv[u] = __ldg(rval + from[u]); }
-#pragma unroll
-          for (int u = 0; u < kFinishBatch; ++u)
-            if (base + u * kFinishThreads < r_hi) put(base + u * kFinishThreads, ri[u], rv[u]);
+          ++j_hi;
         }
-      }
-    } else if (n_mine > 0) {
-      // very long slices (groups of more than 32 chunks): a warp walks one group at a time
-      for (uint32_t g = g0 + warp; g < ngroups && gpre[g] < hi; g += kFinishWarps) {
-        uint32_t running = gpre[g];
-        const uint32_t c_end = min(nchunks, (g + 1u) << gsh);
-        for (uint32_t c0 = g << gsh; c0 < c_end; c0 += 32u) {
-          const uint32_t c = c0 + lane;
-          const uint32_t cnt = c < c_end ? __ldg(ccount + c) : 0u;
-          const uint32_t src0 = c < c_end ? __ldg(cstart + c) : 0u;
-          const uint32_t incl = warp_incl_scan(cnt);
-          const uint32_t excl = incl - cnt;
-          const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
-          if (running + tot > lo && running < hi) {
-            for (uint32_t base = 0; base < tot; base += 32u) {
-              const uint32_t e = base + lane;
-              uint32_t a = 0, b = 32;                            // the run that holds element e: last lane with excl <= e
+        // A group of G lanes copies one run (G = 8 when runs are short, else a whole warp), kRunBatch
+        // runs at a time so that their gathers are in flight together; lanes of a group take
+        // neighbouring elements, neighbouring groups neighbouring runs.
+        const uint32_t gl = tid & (G - 1u), gi = tid / G, n_grp = (uint32_t)kFinishThreads / G;
+        for (uint32_t j = j_lo + gi; j < j_hi; j += n_grp * kRunBatch) {
+          uint32_t first[kRunBatch], cnt[kRunBatch], src[kRunBatch], longest = 0;
 #pragma unroll
-              for (int step = 0; step < 5; ++step) {
-                const uint32_t mid = (a + b) >> 1;
-                if (__shfl_sync(0xFFFFFFFFu, excl, mid) <= e) a = mid; else b = mid;
-              }
-              const uint32_t from = __shfl_sync(0xFFFFFFFFu, src0, a) + (e - __shfl_sync(0xFFFFFFFFu, excl, a));
-              const uint32_t at = running + e;
-              if (e < tot && at >= lo && at < hi) put(at, __ldg(ridx + from), __ldg(rval + from));
+          for (int u = 0; u < kRunBatch; ++u) {
+            const uint32_t jj = j + u * n_grp;
+            first[u] = 0; cnt[u] = 0; src[u] = 0;
+            if (jj < j_hi) { first[u] = dstTab[jj]; cnt[u] = dstTab[jj + 1] - first[u]; src[u] = srcTab[jj]; }
+            longest = max(longest, cnt[u]);
+          }
+          for (uint32_t e = gl; e < longest; e += G) {
+            uint32_t ri[kRunBatch];
+            float rv[kRunBatch];
+#pragma unroll
+            for (int u = 0; u < kRunBatch; ++u) {
+              const uint32_t at = first[u] + e;
+              if (e < cnt[u] && at >= r_lo && at < r_hi) { ri[u] = __ldg(ridx + src[u] + e); rv[u] = __ldg(rval + src[u] + e); }
+            }
+#pragma unroll
+            for (int u = 0; u < kRunBatch; ++u) {
+              const uint32_t at = first[u] + e;
+              if (e < cnt[u] && at >= r_lo && at < r_hi) put(at, ri[u], rv[u]);
             }
           }
-          running += tot;
         }
       }
     }
@@ -742,8 +792,11 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
 
   // keys inside [lo_key, hi_key) over the whole cluster, when known
   uint32_t bucket_n = general ? n_cand - n_gt : 0xFFFFFFFFu;
+  // ranking a list by counting is quadratic: worth more than 512 keys only when a pass over the
+  // share is long
+  const uint32_t list_max = n_mine > 32768u ? (uint32_t)kFinishListLong : (uint32_t)kFinishList;
   for (int round = 0; (hi_key - lo_key > 1u || count_above) && round < 8; ++round) {
-    if (!count_above && bucket_n <= (uint32_t)kFinishList) {
+    if (!count_above && bucket_n <= list_max) {
       // Few keys are left in the interval: instead of more histogram rounds, every CTA lists its own,
       // reads the other CTAs' lists through distributed shared memory and ranks the union by counting.
       if (tid == 0) sm.list_n = 0;
@@ -763,7 +816,7 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
       }
       __syncthreads();
       const uint32_t total = sm.list_pre[CS];
-      if (total > (uint32_t)kFinishList || total < need) {       // the same on every CTA
+      if (total > list_max || total < need) {       // the same on every CTA
         if (q == 0 && tid == 0) { atomicOr(L.s.error, ERR_SELECT_INCONSISTENT); st->resolved = 32; }
         cluster.sync();
         return;
@@ -774,18 +827,20 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
         sm.red[t] = cluster.map_shared_rank(sm.hist, rr)[t - sm.list_pre[rr]];
       }
       __syncthreads();
-      if (tid < total) {
-        const uint32_t e = sm.red[tid];
+      for (uint32_t t = tid; t < total; t += kFinishThreads) {
+        const uint32_t e = sm.red[t];
         uint32_t rank = 0;                                       // keys ranked before e (ties: list order)
         for (uint32_t j = 0; j < total; ++j) {
           const uint32_t o = sm.red[j];
-          rank += (o > e) || (o == e && j < tid);
+          rank += (o > e) || (o == e && j < t);
         }
         if (rank == need - 1u) sm.tau_out = e;
       }
       __syncthreads();
       const uint32_t found = sm.tau_out;
-      const uint32_t above = __syncthreads_count(tid < total && sm.red[tid] > found);
+      uint32_t above = 0;
+      for (uint32_t off = 0; off < total; off += kFinishThreads)
+        above += __syncthreads_count(off + tid < total && sm.red[off + tid] > found);
       cluster.sync();                                            // all remote reads of the lists are done
       n_gt += above; need -= above;
       lo_key = found; hi_key = found + 1u;

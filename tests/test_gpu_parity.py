@@ -242,6 +242,13 @@ def test_aggregate_sparse_path_many_workers_and_crowded_tiles(lib):
     d, W, k = 3_000_000, 16, 3000                      # identical supports: every coordinate shared by all
     same = np.sort(rng.choice(d, k, replace=False))
     cases.append((d, np.stack([same] * W)))
+    d, W, k = 2_000_003, 13, 777                       # a worker count that is no multiple of the warps per block
+    cases.append((d, np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)])))
+    d, W, k = 70_001, 3, 1                             # one entry per worker: the shortest sorted rows
+    cases.append((d, np.array([[70_000], [0], [16_384]])))
+    d, W, k = 1_000_000, 5, 40                         # runs that end exactly at tile borders
+    edge = np.sort(np.concatenate([np.arange(16_380, 16_400), np.arange(32_758, 32_778)]))
+    cases.append((d, np.stack([edge] * W)))
     for d, idx in cases:
         idx = idx.astype(np.uint32)
         W, k = idx.shape
