@@ -604,6 +604,13 @@ struct alignas(16) FinishSmem {           // the value cache behind it is read a
 static_assert(sizeof(FinishSmem) % 16 == 0, "the value cache must start 16-byte aligned");
 constexpr size_t kFinishSmemBytes = sizeof(FinishSmem) + (size_t)kFinishCache * sizeof(float);
 
+// 4-byte asynchronous copy global -> shared (no register holds the value in between) ...
+__device__ __forceinline__ void async_copy_4(void* smem_dst, const void* gmem_src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
+}
+// ... and the wait for all such copies of the calling thread.
+__device__ __forceinline__ void async_copy_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
   namespace cg = cooperative_groups;
   extern __shared__ __align__(16) unsigned char finish_raw[];
@@ -642,6 +649,10 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
   const uint32_t lo = min(n_cand, q * per), hi = min(n_cand, lo + per);
   const uint32_t n_mine = hi - lo;
   const uint32_t n_cached = min(n_mine, (uint32_t)kFinishCache);
+  // a share of at most half the cache keeps its indices in shared memory as well (never written to
+  // the global list); runs then reach the cache by asynchronous copies, all in flight at once
+  const bool idx_cached = !general && n_mine <= (uint32_t)(kFinishCache / 2);
+  uint32_t* cache_idx = reinterpret_cast<uint32_t*>(cache + kFinishCache / 2);
 
   if (general) {
     // my share of the candidate values -> shared memory (the share starts 128-byte aligned)
@@ -748,6 +759,19 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
             if (jj < j_hi) { first[u] = dstTab[jj]; cnt[u] = dstTab[jj + 1] - first[u]; src[u] = srcTab[jj]; }
             longest = max(longest, cnt[u]);
           }
+          if (idx_cached) {
+            for (uint32_t e = gl; e < longest; e += G) {
+#pragma unroll
+              for (int u = 0; u < kRunBatch; ++u) {
+                const uint32_t at = first[u] + e;
+                if (e < cnt[u] && at >= r_lo && at < r_hi) {
+                  async_copy_4(cache_idx + (at - lo), ridx + src[u] + e);
+                  async_copy_4(cache + (at - lo), rval + src[u] + e);
+                }
+              }
+            }
+            continue;
+          }
           for (uint32_t e = gl; e < longest; e += G) {
             uint32_t ri[kRunBatch];
             float rv[kRunBatch];
@@ -764,6 +788,7 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
           }
         }
       }
+      async_copy_wait_all();
     }
   }
   __syncthreads();
@@ -973,7 +998,8 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
     // the four indices, fetched now so that no store below waits on a load (the list's capacity is a
     // multiple of 32 entries, so the vector stays inside the slice's list)
     uint4 ci = make_uint4(0u, 0u, 0u, 0u);
-    if (i0 < w_hi) ci = *reinterpret_cast<const uint4*>(cidx + lo + i0);
+    if (i0 < w_hi) ci = idx_cached ? *reinterpret_cast<const uint4*>(cache_idx + i0)
+                                   : *reinterpret_cast<const uint4*>(cidx + lo + i0);
     const uint32_t cj[4] = {ci.x, ci.y, ci.z, ci.w};
     uint32_t mA = 0, mB = 0;
 #pragma unroll
