@@ -296,7 +296,9 @@ def main():
     sync_all()
     sampler = ClockSampler(local) if rank == 0 else None
     wall0 = time.time()
+    launches0 = ctx.launch_count()
     total_ms = timed(one_step, t_next, args.steps)
+    gpu_launches = ctx.launch_count() - launches0   # this library's kernels inside the timed region
     wall1 = time.time()
     t_next += args.steps
     clocks = sampler.stop(wall0, wall1) if sampler else None
@@ -352,15 +354,15 @@ def main():
         cores = os.cpu_count() or 1
         n_rows = cpu_sample_rows(cfg, cores)
         threads = min(cores, n_rows)
+        # one step to size the sample, then enough steps for roughly 12 s of CPU work
         sec = time_oracle(cfg, n_rows, threads)
+        n_cpu_steps = max(1, min(40, int(12.0 / max(sec, 1e-3))))
+        if n_cpu_steps > 1:
+            sec = time_oracle(cfg, n_rows, threads, steps=n_cpu_steps)
         cpu = {"value": n_rows * d * gsz / sec / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
-               "seconds": sec, "sample": f"1 step, {n_rows} of {W} worker rows, step-0 gradient, zero residual"}
+               "seconds": sec * n_cpu_steps,
+               "sample": f"{n_cpu_steps} steps, {n_rows} of {W} worker rows, step-0 gradient, residual carried"}
 
-    # launches per step of this library's kernels (memsets and copies not counted):
-    # k_draw, k_resolve, k_sel_scan (unless k = r), k_sample, k_stream, then either k_exact + k_finish
-    # (r < d) or k_emit_all (r = d), then k_agg_starts and one aggregate kernel
-    subset = 3 if (seg or cfg.k < cfg.r) else 0
-    per_step = subset + 2 + (1 if cfg.r == cfg.d and not seg else 2) + 2
     if rank == 0:
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -373,7 +375,7 @@ def main():
             "elements_per_s": W_total * d / (ms_per_step * 1e-3),
             "step_roofline_frac": step_frac, "step_algorithmic_bytes": step_bytes,
             "phases_ms": phases, "fallback_slices": fallbacks,
-            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": per_step * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": gpu_launches,
             "clocks": clocks,
         }))
     if world > 1:

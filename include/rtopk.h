@@ -223,6 +223,11 @@ int rtopk_get_phase_times(rtopk_ctx* ctx, float* ms, void* stream);
  * of the last sparsify call into *out (host). */
 int rtopk_get_stats(rtopk_ctx* ctx, int32_t slice, rtopk_stats* out, void* stream);
 
+/* Number of kernels this context has launched since rtopk_create (memsets and copies are not
+ * counted; neither are the launches of rtopk_sample_positions_static, which has no context).
+ * A bookkeeping call with no counterpart in the paper.  *out is host memory.  Errors: INVALID_ARG. */
+int rtopk_get_launch_count(const rtopk_ctx* ctx, uint64_t* out);
+
 #ifdef __cplusplus
 }
 #endif

@@ -46,6 +46,7 @@ EXPORTS = {
     "rtopk_poll_status": (_int, [_vp, _vp]),
     "rtopk_get_phase_times": (_int, [_vp, _vp, _vp]),
     "rtopk_get_stats": (_int, [_vp, _i32, _vp, _vp]),
+    "rtopk_get_launch_count": (_int, [_vp, _vp]),
 }
 
 _lib: Optional[C.CDLL] = None
@@ -210,6 +211,11 @@ class RTopK:
         ms = (C.c_float * len(PHASES))()
         self._check(self._lib.rtopk_get_phase_times(self._h, ms, _stream()), "rtopk_get_phase_times")
         return {name: float(ms[i]) for i, name in enumerate(PHASES)}
+
+    def launch_count(self) -> int:
+        n = C.c_uint64(0)
+        self._check(self._lib.rtopk_get_launch_count(self._h, C.byref(n)), "rtopk_get_launch_count")
+        return int(n.value)
 
     def stats(self, slice_index: int) -> dict:
         s = Stats()

@@ -55,6 +55,7 @@ struct rtopk_ctx {
   uint32_t last_n_slices = 0;
   // optional per-phase timing (RTOPK_OPT_PROFILE): events recorded on the caller's stream
   int sms = 0;
+  uint64_t launches = 0;                          // kernels launched by this context so far
   int finish_max_clusters[kMaxCluster + 1] = {};  // [cs]: co-resident k_finish clusters of size cs (1..16)
   int stream_blocks[2] = {0, 0};
   int exact_blocks = 0;               // cooperative grid of k_exact (all blocks resident)      // persistent grid of k_stream per gradient dtype
@@ -248,6 +249,7 @@ int launch_exact(rtopk_ctx* ctx, const Plan& P, const Launch& L, int first_pass,
   void* args[] = {&Lc, &fp, &nh, &nc};
   RTOPK_CUDA(ctx, cudaLaunchCooperativeKernel((const void*)k_exact, dim3((unsigned)ctx->exact_blocks), dim3(kThreads),
                                               args, 0, st));
+  ++ctx->launches;
   return RTOPK_OK;
 }
 
@@ -258,12 +260,14 @@ int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t s
   if (ctx->select_path == 0) {
     mark(ctx, RTOPK_PHASE_THRESHOLD, st);
     k_sample<GradT><<<n, kSampleThreads, kSampleSmemBytes, st>>>(L);
+    ++ctx->launches;
     mark(ctx, RTOPK_PHASE_STREAM, st);
     {
       const uint32_t per = (uint32_t)((P.slices[0].head + (uint64_t)P.slices[0].len + kChunk - 1) / kChunk);
       const uint32_t uniform = P.uniform ? per : 0u;
       const int blocks = ctx->stream_blocks[sizeof(GradT) == 4 ? 0 : 1];
       k_stream<GradT><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
+      ++ctx->launches;
       mark(ctx, RTOPK_PHASE_ORDER, st);
     }
     mark(ctx, RTOPK_PHASE_EXACT, st);
@@ -274,9 +278,11 @@ int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t s
   } else {
     mark(ctx, RTOPK_PHASE_THRESHOLD, st);
     k_init_state<<<(n + 127) / 128, 128, 0, st>>>(L, 1u);
+    ++ctx->launches;
     mark(ctx, RTOPK_PHASE_STREAM, st);
     const uint32_t hgrid = std::min<uint32_t>(P.n_hist_blocks, (uint32_t)ctx->sms * 8u);
     k_hist<GradT, true><<<hgrid, kThreads, 0, st>>>(L, 0, P.n_hist_blocks);
+    ++ctx->launches;
     mark(ctx, RTOPK_PHASE_ORDER, st);
     mark(ctx, RTOPK_PHASE_EXACT, st);
     if (P.any_select) {
@@ -303,11 +309,15 @@ int run_sampler(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st)
   RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_first, 0xFF, P.first_entries * sizeof(uint32_t), st));
   const dim3 grid((P.k_draw_max + kDrawThreads - 1) / kDrawThreads, n);
   k_draw<<<grid, kDrawThreads, 0, st>>>(L);
+  ++ctx->launches;
   k_resolve<<<grid, kDrawThreads, 0, st>>>(L);
+  ++ctx->launches;
   const dim3 sgrid((P.sel_words_max + kSelChunk - 1) / kSelChunk, n);
   if ((size_t)sgrid.x * n > ctx->sel_blk_entries) return RTOPK_ERR_INVALID_ARG;
   k_sel_count<<<sgrid, kScanThreads, 0, st>>>(L);
+  ++ctx->launches;
   k_sel_scan<<<sgrid, kScanThreads, 0, st>>>(L);
+  ++ctx->launches;
   return RTOPK_OK;
 }
 
@@ -380,10 +390,12 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
     attr[0].val.clusterDim.x = (unsigned)cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     RTOPK_CUDA(ctx, cudaLaunchKernelEx(&cfg, k_finish, L));
+    ++ctx->launches;
   }
   if (P.any_all) {
     const dim3 grid((P.words_all_max + kThreads - 1) / kThreads, L.n_slices);
     k_emit_all<<<grid, kThreads, 0, st>>>(L, P.words_all_max);
+    ++ctx->launches;
   }
   mark(ctx, RTOPK_PHASE_AGGREGATE, st);
   ctx->ev_valid[RTOPK_N_PHASES] = false;   // closed by the aggregate of a step call, if any
@@ -417,6 +429,7 @@ int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val
   if (!own_search) {
     const dim3 sgrid((ntiles + 1 + kAggThreads - 1) / kAggThreads, (uint32_t)W);
     k_agg_starts<<<sgrid, kAggThreads, 0, st>>>(msg_idx, (uint32_t)W, (uint32_t)k, ntiles, tile, ctx->d_agg_starts);
+    ++ctx->launches;
   }
   const int mean = scale_mode == RTOPK_SCALE_MEAN ? 1 : 0;
   if (sparse) {
@@ -424,9 +437,11 @@ int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val
     if (!out_cleared) RTOPK_CUDA(ctx, cudaMemsetAsync(out, 0, (size_t)d * sizeof(float), st));
     k_aggregate_sparse<<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, own_search ? nullptr : ctx->d_agg_starts, (uint32_t)d,
                                                        (uint32_t)W, (uint32_t)k, mean, out);
+    ++ctx->launches;
   } else {
     k_aggregate<<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, ctx->d_agg_starts, (uint32_t)d, (uint32_t)W,
                                                 (uint32_t)k, mean, out);
+    ++ctx->launches;
   }
   mark(ctx, RTOPK_N_PHASES, st);
   RTOPK_CUDA(ctx, cudaGetLastError());
@@ -694,6 +709,7 @@ int rtopk_sample_positions(rtopk_ctx* ctx, int64_t r, int64_t k, uint64_t seed, 
   if (rc) return rc;
   const uint32_t nwords = (uint32_t)((r + 31) / 32);
   k_positions<<<(nwords + kThreads - 1) / kThreads, kThreads, 0, st>>>(L, pos);
+  ++ctx->launches;
   RTOPK_CUDA(ctx, cudaGetLastError());
   return RTOPK_OK;
 }
@@ -743,6 +759,12 @@ int rtopk_get_stats(rtopk_ctx* ctx, int32_t slice, rtopk_stats* out, void* strea
   out->n_greater = s.n_gt;
   out->n_candidates = s.n_cand;
   out->used_fallback = (s.flags & FLAG_FELL_BACK) ? 1u : 0u;
+  return RTOPK_OK;
+}
+
+int rtopk_get_launch_count(const rtopk_ctx* ctx, uint64_t* out) {
+  if (!ctx || !out) return RTOPK_ERR_INVALID_ARG;
+  *out = ctx->launches;
   return RTOPK_OK;
 }
 
