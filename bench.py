@@ -31,7 +31,7 @@ sys.path.insert(0, ROOT)
 
 METRIC = "rtopk_step_gradient_input_bandwidth"
 UNIT = "GB/s"
-KERNEL_SOURCES = ["common.cuh", "select.cuh", "stream.cuh", "sampler.cuh", "aggregate.cuh", "rtopk.cu"]
+KERNEL_SOURCES = ["common.cuh", "element.cuh", "stream.cuh"]   # everything k_stream is compiled from
 
 
 def load_peak():

@@ -16,7 +16,7 @@
 #pragma once
 
 #include "common.cuh"
-#include "select.cuh"
+#include "element.cuh"
 
 namespace rtopk {
 
