@@ -7,6 +7,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
@@ -203,16 +204,18 @@ int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32
   return RTOPK_OK;
 }
 
-// Carves the per-call zeroed region.  Returns the bytes used.
-size_t carve_zero(const rtopk_ctx* ctx, const Plan& P, Scratch& s) {
+// Carves the per-call zeroed region.  Returns the bytes used; *early_bytes is the leading part that
+// holds the counters the sampling kernels clear themselves (the rest is cleared by a memset).
+size_t carve_zero(const rtopk_ctx* ctx, const Plan& P, Scratch& s, size_t* early_bytes = nullptr) {
   char* p = ctx->d_zero;
   size_t at = 0;
   auto take = [&](size_t bytes) { char* q = p + at; at = align_up(at + bytes, 256); return q; };
   s.tickets = (uint32_t*)take(4 * sizeof(uint32_t));
   s.done = (uint32_t*)take(P.slices.size() * sizeof(uint32_t));
   s.cursor = (uint32_t*)take(P.slices.size() * sizeof(uint32_t));
-  s.hist = (uint32_t*)take(P.slices.size() * kBins * sizeof(uint32_t));
   s.group_total = (uint32_t*)take((size_t)P.n_groups * sizeof(uint32_t));
+  if (early_bytes) *early_bytes = at;
+  s.hist = (uint32_t*)take(P.slices.size() * kBins * sizeof(uint32_t));
   s.look_b = (unsigned long long*)take((size_t)P.n_chunks * 8);
   s.sel = (uint32_t*)take(P.sel_words * sizeof(uint32_t));
   return at;
@@ -221,8 +224,8 @@ size_t carve_zero(const rtopk_ctx* ctx, const Plan& P, Scratch& s) {
 size_t zero_region_bytes(size_t slices, size_t chunks, size_t groups, size_t sel_words) {
   size_t at = 0;
   auto take = [&](size_t bytes) { at = align_up(at + bytes, 256); };
-  take(16); take(slices * 4); take(slices * 4); take(slices * kBins * 4); take(groups * 4); take(chunks * 8);
-  take(sel_words * 4);
+  take(16); take(slices * 4); take(slices * 4); take(groups * 4);
+  take(slices * kBins * 4); take(chunks * 8); take(sel_words * 4);
   return at;
 }
 
@@ -254,7 +257,7 @@ int launch_exact(rtopk_ctx* ctx, const Plan& P, const Launch& L, int first_pass,
 }
 
 template <typename GradT>
-int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st) {
+int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st, cudaEvent_t join) {
   const uint32_t n = (uint32_t)P.slices.size();
   int rc = RTOPK_OK;
   if (ctx->select_path == 0) {
@@ -271,6 +274,8 @@ int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t s
       mark(ctx, RTOPK_PHASE_ORDER, st);
     }
     mark(ctx, RTOPK_PHASE_EXACT, st);
+    // the exact path's histograms and look-back words are cleared on the side stream
+    if (join) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, join, 0));
     if (P.any_select) {
       rc = launch_exact(ctx, P, L, 0, st);
       if (rc) return rc;
@@ -338,7 +343,8 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   if (!guard.ok) return RTOPK_ERR_CUDA;
   Launch L;
   std::memset(&L, 0, sizeof(L));
-  const size_t zbytes = carve_zero(ctx, P, L.s);
+  size_t early_bytes = 0;
+  const size_t zbytes = carve_zero(ctx, P, L.s, &early_bytes);
   if (zbytes > ctx->zero_bytes) return RTOPK_ERR_INVALID_ARG;
   L.s.slices = ctx->d_slices; L.s.state = ctx->d_state;
   L.s.cand_idx = ctx->d_cand_idx; L.s.cand_val = ctx->d_cand_val;
@@ -359,19 +365,27 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   if (rc) return rc;
   ctx->last_n_slices = L.n_slices;
   mark(ctx, RTOPK_PHASE_SUBSET, st);
-  RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero, 0, zbytes, st));
+  // The sampling kernels clear the leading counters of the zeroed region themselves; the exact
+  // primary path has no such kernel.  The rest (exact-path histograms and look-back words, the
+  // selection bitmap) is first touched by the sampler and the exact path, both behind the fork.
+  const bool late_on_side = ctx->select_path == 0;
+  if (!late_on_side) RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero, 0, zbytes, st));
   const bool forked = P.any_sampler || clear_out != nullptr;
   if (forked) {
     // work that does not depend on the data runs beside the streaming pass: the k-of-r subset and,
     // for a step call, the clearing of the dense update
     RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_fork, st));
     RTOPK_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
+    if (late_on_side) RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero + early_bytes, 0, zbytes - early_bytes, ctx->side));
     rc = run_sampler(ctx, P, L, ctx->side);
     if (rc) return rc;
     if (clear_out) RTOPK_CUDA(ctx, cudaMemsetAsync(clear_out, 0, (size_t)d * sizeof(float), ctx->side));
     RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_join, ctx->side));
+  } else if (late_on_side) {
+    RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero + early_bytes, 0, zbytes - early_bytes, st));
   }
-  rc = grad_dtype == RTOPK_F32 ? launch_select<float>(ctx, P, L, st) : launch_select<__nv_bfloat16>(ctx, P, L, st);
+  cudaEvent_t join = forked ? ctx->ev_join : nullptr;
+  rc = grad_dtype == RTOPK_F32 ? launch_select<float>(ctx, P, L, st, join) : launch_select<__nv_bfloat16>(ctx, P, L, st, join);
   if (rc) return rc;
   if (forked) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0));
   mark(ctx, RTOPK_PHASE_FINISH, st);

@@ -22,6 +22,19 @@ __device__ __forceinline__ uint32_t slice_chunks(const Slice& S) {
   return (S.head + S.len + kChunk - 1) / kChunk;
 }
 
+// Clears the counters of slice `sl` that the streaming pass and the exact path expect to be zero
+// (run cursor, block counter, chunk-group totals; plus the launch-wide tickets).  The sampling
+// kernels do this instead of a memset node in front of them; `part` of `nparts` thread blocks of
+// blockDim.x threads share the work.
+__device__ __forceinline__ void clear_slice_counters(const Launch& L, uint32_t sl, const Slice& S, uint32_t part, uint32_t nparts) {
+  const uint32_t t = part * blockDim.x + threadIdx.x, nt = nparts * blockDim.x;
+  const uint32_t nchunks = slice_chunks(S);
+  const uint32_t ngroups = (nchunks + (1u << S.gshift) - 1u) >> S.gshift;
+  for (uint32_t g = t; g < ngroups; g += nt) L.s.group_total[S.group_begin + g] = 0;
+  if (t == 0) { L.s.cursor[sl] = 0; L.s.done[sl] = 0; }
+  if (sl == 0 && t < 4u) L.s.tickets[t] = 0;
+}
+
 // ----------------------------------------------------------------------------- state init
 __global__ void k_init_state(Launch L, uint32_t general) {
   const uint32_t s = blockIdx.x * blockDim.x + threadIdx.x;
@@ -138,6 +151,7 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(Launch L) {
   const uint32_t sl = blockIdx.x;
   const Slice S = L.s.slices[sl];
   const uint32_t tid = threadIdx.x;
+  clear_slice_counters(L, sl, S, 0, 1);
   SelState st;
   st.eq_quota = kNoQuota; st.prefix = 0; st.resolved = 0; st.n_gt = 0; st.need = S.r;
   st.n_cand = 0; st.n_cand_first = 0; st.stage = STAGE_PASS0; st.flags = 0; st.tau_hi = 0x7FFFFFFFu; st.pad = 0;
