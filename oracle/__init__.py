@@ -63,6 +63,8 @@ def lib() -> C.CDLL:
                                                 i64p, i64p, C.c_uint64, C.c_uint32, u32p, f32p]
         L.oracle_aggregate.argtypes = [u32p, f32p, C.c_int64, C.c_int32, C.c_int64, C.c_int,
                                        f64p, f32p]
+        L.oracle_apply_update.argtypes = [u32p, f32p, C.c_int64, C.c_int32, C.c_int64, C.c_int,
+                                          C.c_float, f32p]
         _lib = L
     return _lib
 
@@ -175,6 +177,18 @@ def aggregate(msg_idx: np.ndarray, msg_val: np.ndarray, d: int, scale_mode: int 
     _check(lib().oracle_aggregate(_p(idx, C.c_uint32), _p(val, C.c_float), d, W, k, scale_mode,
                                   _p(o64, C.c_double), _p(o32, C.c_float)), "aggregate")
     return o64, o32
+
+
+def apply_update(msg_idx: np.ndarray, msg_val: np.ndarray, d: int, eta: float, weights: np.ndarray,
+                 scale_mode: int = SCALE_MEAN) -> np.ndarray:
+    """Algorithm 1 master update w - eta * ghat on a copy of `weights` (float32 [d])."""
+    idx = np.ascontiguousarray(msg_idx, dtype=np.uint32)
+    val = np.ascontiguousarray(msg_val, dtype=np.float32)
+    W, k = idx.shape
+    w = np.array(weights, dtype=np.float32, copy=True)
+    _check(lib().oracle_apply_update(_p(idx, C.c_uint32), _p(val, C.c_float), d, W, k, scale_mode,
+                                     C.c_float(eta), _p(w, C.c_float)), "apply_update")
+    return w
 
 
 if __name__ == "__main__":

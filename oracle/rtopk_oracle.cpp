@@ -5,7 +5,7 @@
 // Estimation Approach to Distributed SGD"):
 //
 //   Algorithm 1, node body:   a = g + m ; ghat = rTop_k(a) ; m' = a - ghat ; send ghat
-//   Algorithm 1, master:      ghat = (1/n) * sum_i ghat_i
+//   Algorithm 1, master:      ghat = (1/n) * sum_i ghat_i ; w' = w - eta * ghat
 //   Definition 1 (top-r), Definition 2 (random-k), Definition 3 (rTop-k).
 //
 // Only the tests, the smoke check and the benchmark's cpu_baseline leg may call
@@ -27,7 +27,9 @@
 //   * IEEE 754 leaves the payload of a NaN result to the implementation, so a NaN sum is stored as
 //     the default quiet NaN (bit pattern 0x7FC00000);
 //   * m' is a bit copy of a outside the sent set and +0.0f inside it;
-//   * messages are listed by ascending index.
+//   * messages are listed by ascending index;
+//   * the master update rounds once: w' = fp32(double(w) - double(eta) * double(ghat)) with ghat
+//     the binary32 average (the product of two binary32 numbers is exact in binary64).
 //
 // Pins (tests/test_oracle_*.py): Philox against published known answers; the
 // draw scaling against big-integer arithmetic; Floyd against exhaustive
@@ -286,6 +288,20 @@ int oracle_aggregate(const uint32_t* msg_idx, const float* msg_val, int64_t d, i
     if (out64) out64[i] = v;
     if (out32) out32[i] = (float)v;
   }
+  return ORACLE_OK;
+}
+
+// Algorithm 1, master update: w <- w - eta * ghat with ghat the average (or sum) above, for every
+// coordinate.  eta >= 0 (with a negative eta a zero weight at an unsent coordinate would change
+// its sign, which the sparse restatements of this update never touch).
+int oracle_apply_update(const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
+                        int scale_mode, float eta, float* weights) {
+  if (!weights || !(eta >= 0.0f) || eta > 3.0e38f) return ORACLE_BAD_ARG;
+  std::vector<float> ghat((size_t)d);
+  const int rc = oracle_aggregate(msg_idx, msg_val, d, W, k, scale_mode, nullptr, ghat.data());
+  if (rc != ORACLE_OK) return rc;
+  for (int64_t i = 0; i < d; ++i)
+    weights[i] = (float)((double)weights[i] - (double)eta * (double)ghat[(size_t)i]);
   return ORACLE_OK;
 }
 

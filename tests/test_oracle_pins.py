@@ -377,6 +377,42 @@ def test_aggregate_against_numpy_and_special_cases():
     assert np.array_equal(o64[: W * k], val.ravel().astype(np.float64) / W)
 
 
+def test_master_update_worked_example_and_textbook_sgd():
+    # Algorithm 1, master update w <- w - eta * ghat.  d = 4, two workers as in the average's worked
+    # example: ghat = [0.5, 0, 3, 4]; with eta = 0.5 and w = [1, 1, 1, 1] the update is exact.
+    idx = np.array([[0, 2], [2, 3]], dtype=np.uint32)
+    val = np.array([[1, 2], [4, 8]], dtype=np.float32)
+    w = oracle.apply_update(idx, val, 4, 0.5, np.ones(4, dtype=np.float32))
+    assert w.tolist() == [0.75, 1.0, -0.5, -1.0]
+    # one worker, sum scaling: plain SGD on the sent coordinates, every other weight bit-unchanged
+    rng = np.random.default_rng(21)
+    d, k, eta = 3000, 200, np.float32(0.0371)
+    idx = np.sort(rng.choice(d, k, replace=False)).astype(np.uint32)[None, :]
+    val = (rng.standard_normal((1, k)) * np.exp(2 * rng.standard_normal((1, k)))).astype(np.float32)
+    w0 = rng.standard_normal(d).astype(np.float32)
+    w0[idx[0, 0]] = -0.0
+    w0[(idx[0, 0] + 1) % d if (idx[0, 0] + 1) % d not in idx[0] else idx[0, 0]] = -0.0
+    w1 = oracle.apply_update(idx, val, d, float(eta), w0, oracle.SCALE_SUM)
+    ref = w0.astype(np.float64)
+    ref[idx[0].astype(np.int64)] -= np.float64(eta) * val[0].astype(np.float64)
+    assert np.array_equal(w1.view(np.uint32), ref.astype(np.float32).view(np.uint32))
+    untouched = np.ones(d, dtype=bool)
+    untouched[idx[0].astype(np.int64)] = False
+    assert np.array_equal(w1.view(np.uint32)[untouched], w0.view(np.uint32)[untouched])
+    # eta = 0 changes no value (a sent -0.0 weight may become +0.0: -0 - (0 * negative) = -0 + 0), and
+    # no bit at unsent coordinates; the update agrees with the (separately pinned) average applied densely
+    z = oracle.apply_update(idx, val, d, 0.0, w0)
+    assert np.array_equal(z, w0) and np.array_equal(z.view(np.uint32)[untouched], w0.view(np.uint32)[untouched])
+    W = 4
+    idx4 = np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)]).astype(np.uint32)
+    val4 = rng.standard_normal((W, k)).astype(np.float32)
+    _, g32 = oracle.aggregate(idx4, val4, d)
+    dense = (w0.astype(np.float64) - np.float64(eta) * g32.astype(np.float64)).astype(np.float32)
+    assert np.array_equal(oracle.apply_update(idx4, val4, d, float(eta), w0).view(np.uint32), dense.view(np.uint32))
+    with pytest.raises(ValueError):
+        oracle.apply_update(idx4, val4, d, -1.0, w0)
+
+
 def test_bad_arguments_are_rejected():
     g = np.zeros((1, 8), dtype=np.float32)
     m = np.zeros((1, 8), dtype=np.float32)
