@@ -203,6 +203,8 @@ def main():
     ap.add_argument("--scale-d", type=int, default=0, help="run the workload's recipe at this vector length")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--apply", action="store_true",
+                    help="time rtopk_step_apply (master update fused into the aggregation; plain workloads, 1 GPU)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -246,7 +248,10 @@ def main():
     residual = wl.zero_residual(cfg, dev)
     idx = torch.zeros((W, K), dtype=torch.int32, device=dev)
     val = torch.zeros((W, K), dtype=torch.float32, device=dev)
-    out = torch.empty(wl.round_up(d, 4), dtype=torch.float32, device=dev)
+    # the dense update; with --apply the model weights that the update is applied to
+    out = torch.zeros(wl.round_up(d, 4), dtype=torch.float32, device=dev)
+    if args.apply and (seg or world > 1):
+        raise SystemExit("--apply covers the plain single-GPU workloads")
     base = rank * W
 
     def one_step(t: int):
@@ -254,6 +259,8 @@ def main():
         if world == 1:
             if seg:
                 ctx.step_segmented(g, residual, d, cfg.seg_off, cfg.seg_r, cfg.seg_k, cfg.seed, t, idx, val, out)
+            elif args.apply:
+                ctx.step_apply(g, residual, d, cfg.r, cfg.k, cfg.seed, t, 0.01, idx, val, out)
             else:
                 ctx.step(g, residual, d, cfg.r, cfg.k, cfg.seed, t, idx, val, out)
         else:
@@ -327,12 +334,13 @@ def main():
                 "frac": (achieved / peak) if achieved else None,
                 "traffic": recorded_traffic(cfg.name, stream_bytes),
                 "algorithmic_bytes_per_launch": stream_bytes, "kernel_ms": stream_ms}
-    step_bytes = W * d * (gsz + 8) + 4 * d + 16 * W * K
+    # with --apply the 4 d-byte dense update is not written: 8 bytes per sent coordinate instead
+    step_bytes = W * d * (gsz + 8) + (8 * W * K if args.apply else 4 * d) + 16 * W * K
     step_frac = step_bytes / (ms_per_step * 1e-3) / 1e9 / peak if world == 1 else None
 
     # end to end: host gradient in, host messages + update out, through rtopk_step_host
     e2e = None
-    if not args.no_e2e and world == 1 and not seg:
+    if not args.no_e2e and world == 1 and not seg and not args.apply:
         h_grad = grads[0].cpu().pin_memory()
         h_idx = torch.zeros((W, K), dtype=torch.int32).pin_memory()
         h_val = torch.zeros((W, K), dtype=torch.float32).pin_memory()
@@ -371,7 +379,8 @@ def main():
             "config": {"workload": cfg.name, "d": d, "W_per_gpu": W, "W_total": W_total, "r": cfg.r, "k": K,
                        "grad_dtype": cfg.grad_dtype, "recipe": cfg.recipe, "segments": len(cfg.seg_r) if seg else 1,
                        "gradient_batches_resident": n_batches, "residual": "carried across steps",
-                       "l2": "inputs larger than L2 (no flush)", "parallelism": f"workers sharded x{world}"},
+                       "l2": "inputs larger than L2 (no flush)", "parallelism": f"workers sharded x{world}",
+                       "variant": "rtopk_step_apply (fused master update)" if args.apply else "rtopk_step"},
             "elements_per_s": W_total * d / (ms_per_step * 1e-3),
             "step_roofline_frac": step_frac, "step_algorithmic_bytes": step_bytes,
             "phases_ms": phases, "fallback_slices": fallbacks,

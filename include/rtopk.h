@@ -135,6 +135,24 @@ int rtopk_sparsify(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_
 int rtopk_aggregate(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d,
                     int32_t W, int64_t k, int scale_mode, float* out, void* stream);
 
+/*
+ * Algorithm 1, master update w <- w - eta * ghat applied straight from the messages: ghat is the
+ * binary32 result rtopk_aggregate would write, and every coordinate that some worker sent receives
+ * fp32(double(w_i) - double(eta) * double(ghat_i)) (one rounding); all other weights are not touched
+ * (ghat_i = 0 there), so no dense vector is written.
+ *   weights [in/out]  d binary32, 16-byte aligned;   eta  finite, >= 0.
+ * Errors: INVALID_ARG (also for a negative or non-finite eta), CUDA.
+ */
+int rtopk_apply_update(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d,
+                       int32_t W, int64_t k, int scale_mode, float eta, float* weights, void* stream);
+
+/* rtopk_sparsify followed by rtopk_apply_update of the W messages it produced: one round of
+ * Algorithm 1 including the master's update of the model.  Arguments as in the two calls. */
+int rtopk_step_apply(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,
+                     int64_t ld_m, int64_t d, int32_t W, int32_t worker_base, int64_t r, int64_t k,
+                     uint64_t seed, uint32_t step, int scale_mode, float eta, uint32_t* msg_idx,
+                     float* msg_val, float* weights, void* stream);
+
 /* One round of Algorithm 1's communication path: rtopk_sparsify followed by rtopk_aggregate of
  * the W messages it produced.  Arguments as in the two calls. */
 int rtopk_step(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,

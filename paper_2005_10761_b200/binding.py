@@ -33,6 +33,9 @@ EXPORTS = {
     "rtopk_aggregate": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _int, _vp, _vp]),
     "rtopk_step": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _i64, _u64, _u32, _int,
                           _vp, _vp, _vp, _vp]),
+    "rtopk_apply_update": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _int, C.c_float, _vp, _vp]),
+    "rtopk_step_apply": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _i64, _u64, _u32, _int,
+                                C.c_float, _vp, _vp, _vp, _vp]),
     "rtopk_sparsify_segmented": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i32,
                                         C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64), _u64, _u32,
                                         _vp, _vp, _vp]),
@@ -170,6 +173,21 @@ class RTopK:
                                   residual.data_ptr(), residual.stride(0), d, W, worker_base, r, k, seed, step,
                                   scale_mode, msg_idx.data_ptr(), msg_val.data_ptr(), out.data_ptr(), _stream())
         self._check(rc, "rtopk_step")
+
+    def apply_update(self, msg_idx, msg_val, d, eta, weights, scale_mode=SCALE_MEAN) -> None:
+        W, k = msg_idx.shape
+        rc = self._lib.rtopk_apply_update(self._h, msg_idx.data_ptr(), msg_val.data_ptr(), d, W, k, scale_mode,
+                                          eta, weights.data_ptr(), _stream())
+        self._check(rc, "rtopk_apply_update")
+
+    def step_apply(self, grad, residual, d, r, k, seed, step, eta, msg_idx, msg_val, weights, worker_base=0,
+                   scale_mode=SCALE_MEAN) -> None:
+        W = grad.shape[0]
+        rc = self._lib.rtopk_step_apply(self._h, grad.data_ptr(), self._grad_dtype(grad), grad.stride(0),
+                                        residual.data_ptr(), residual.stride(0), d, W, worker_base, r, k, seed,
+                                        step, scale_mode, eta, msg_idx.data_ptr(), msg_val.data_ptr(),
+                                        weights.data_ptr(), _stream())
+        self._check(rc, "rtopk_step_apply")
 
     def sparsify_segmented(self, grad, residual, d, seg_off, seg_r, seg_k, seed, step, msg_idx, msg_val,
                            worker_base=0) -> None:

@@ -23,6 +23,13 @@ constexpr int kAggSparseStage = 2048;   // entries of one such tile staged in sh
 constexpr int kAggMaxW = 1024;    // workers the sparse kernel keeps run tables for
 constexpr int kAggSearchW = 64;   // up to this many workers the sparse kernel finds the runs itself
 
+// What a coordinate's slot receives: the average itself, or (Algorithm 1's master update
+// w <- w - eta * ghat, with eta < 0 meaning "store the average") the updated weight, rounded once
+// from double; the product of two binary32 numbers is exact in double.
+__device__ __forceinline__ float agg_result(float ghat, float old, float eta) {
+  return eta < 0.0f ? ghat : (float)((double)old - (double)eta * (double)ghat);
+}
+
 __device__ __forceinline__ uint32_t lower_bound_u32(const uint32_t* a, uint32_t n, uint32_t key) {
   uint32_t lo = 0, hi = n;
   while (lo < hi) {
@@ -67,7 +74,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(const uint32_t* __res
                                                            const float* __restrict__ msg_val,
                                                            const uint32_t* __restrict__ starts, uint32_t d,
                                                            uint32_t W, uint32_t K, int mean,
-                                                           float* __restrict__ out) {
+                                                           float eta, float* __restrict__ out) {
   __shared__ double acc[kAggTile];
   __shared__ uint32_t s_beg[kAggThreads], s_pre[kAggThreads + 1];
   __shared__ uint32_t st_idx[kAggStage];
@@ -140,11 +147,18 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(const uint32_t* __res
       o.y = (float)(mean && a1 != 0.0 ? a1 / inv : a1);
       o.z = (float)(mean && a2 != 0.0 ? a2 / inv : a2);
       o.w = (float)(mean && a3 != 0.0 ? a3 / inv : a3);
+      if (eta >= 0.0f) {                                   // master update: out holds the weights
+        const float4 w4 = *reinterpret_cast<const float4*>(out + lo + i);
+        o.x = agg_result(o.x, w4.x, eta); o.y = agg_result(o.y, w4.y, eta);
+        o.z = agg_result(o.z, w4.z, eta); o.w = agg_result(o.w, w4.w, eta);
+      }
       __stcs(reinterpret_cast<float4*>(out + lo + i), o);
     }
   } else {
-    for (uint32_t i = tid; i < hi - lo; i += kAggThreads)
-      out[lo + i] = (float)(mean ? acc[i] / inv : acc[i]);
+    for (uint32_t i = tid; i < hi - lo; i += kAggThreads) {
+      const float ghat = (float)(mean ? acc[i] / inv : acc[i]);
+      out[lo + i] = agg_result(ghat, eta >= 0.0f ? out[lo + i] : 0.0f, eta);
+    }
   }
 }
 
@@ -155,7 +169,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(const uint32_t
                                                                   const float* __restrict__ msg_val,
                                                                   const uint32_t* __restrict__ starts, uint32_t d,
                                                                   uint32_t W, uint32_t K, int mean,
-                                                                  float* __restrict__ out) {
+                                                                  float eta, float* __restrict__ out) {
   __shared__ uint32_t s_beg[kAggMaxW], s_pre[kAggMaxW + 1], s_cnt[kAggSearchW];
   __shared__ uint32_t st_idx[kAggSparseStage];
   __shared__ float st_val[kAggSparseStage];
@@ -248,7 +262,8 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(const uint32_t
       if (local >= (uint32_t)kAggSparseTile || idx >= d) continue;    // malformed row: ignore
       if (!((s_shared[local >> 5] >> (local & 31u)) & 1u)) {    // sole sender: the sum is the value
         const double v = (double)st_val[q];
-        out[idx] = (float)(mean ? v / (double)W : v);
+        const float ghat = (float)(mean ? v / (double)W : v);
+        out[idx] = agg_result(ghat, eta >= 0.0f ? out[idx] : 0.0f, eta);
         continue;
       }
     }
@@ -267,7 +282,10 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(const uint32_t
         sum += (double)val_at(x, a);
       }
     }
-    if (owner) out[idx] = (float)(mean ? sum / (double)W : sum);
+    if (owner) {
+      const float ghat = (float)(mean ? sum / (double)W : sum);
+      out[idx] = agg_result(ghat, eta >= 0.0f ? out[idx] : 0.0f, eta);
+    }
   }
 }
 

@@ -424,8 +424,10 @@ bool aggregate_is_sparse(int64_t d, int32_t W, int64_t k) {
 
 // `out_cleared`: the caller has already zeroed `out` in stream order (the step calls do it beside
 // the streaming pass).
+// eta < 0: `out` receives the average.  eta >= 0: `out` holds weights and receives w - eta * average
+// (only the coordinates some worker sent change, so nothing is cleared).
 int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
-                   int scale_mode, float* out, cudaStream_t st, bool out_cleared = false) {
+                   int scale_mode, float* out, cudaStream_t st, bool out_cleared = false, float eta = -1.0f) {
   if (!ctx || !msg_idx || !msg_val || !out) return RTOPK_ERR_INVALID_ARG;
   if (d < 1 || d > ctx->d_max || W < 1 || W > ctx->W_max || k < 1 || k > d) return RTOPK_ERR_INVALID_ARG;
   if (scale_mode != RTOPK_SCALE_MEAN && scale_mode != RTOPK_SCALE_SUM) return RTOPK_ERR_INVALID_ARG;
@@ -448,13 +450,13 @@ int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val
   const int mean = scale_mode == RTOPK_SCALE_MEAN ? 1 : 0;
   if (sparse) {
     // few coordinates are touched: clear the update, then compute only what was sent
-    if (!out_cleared) RTOPK_CUDA(ctx, cudaMemsetAsync(out, 0, (size_t)d * sizeof(float), st));
+    if (!out_cleared && eta < 0.0f) RTOPK_CUDA(ctx, cudaMemsetAsync(out, 0, (size_t)d * sizeof(float), st));
     k_aggregate_sparse<<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, own_search ? nullptr : ctx->d_agg_starts, (uint32_t)d,
-                                                       (uint32_t)W, (uint32_t)k, mean, out);
+                                                       (uint32_t)W, (uint32_t)k, mean, eta, out);
     ++ctx->launches;
   } else {
     k_aggregate<<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, ctx->d_agg_starts, (uint32_t)d, (uint32_t)W,
-                                                (uint32_t)k, mean, out);
+                                                (uint32_t)k, mean, eta, out);
     ++ctx->launches;
   }
   mark(ctx, RTOPK_N_PHASES, st);
@@ -620,6 +622,27 @@ int rtopk_sparsify_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, i
 int rtopk_aggregate(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
                     int scale_mode, float* out, void* stream) {
   return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, out, (cudaStream_t)stream);
+}
+
+int rtopk_apply_update(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W,
+                       int64_t k, int scale_mode, float eta, float* weights, void* stream) {
+  if (!(eta >= 0.0f) || eta > 3.0e38f) return RTOPK_ERR_INVALID_ARG;
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, false, eta);
+}
+
+int rtopk_step_apply(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
+                     int64_t d, int32_t W, int32_t worker_base, int64_t r, int64_t k, uint64_t seed,
+                     uint32_t step, int scale_mode, float eta, uint32_t* msg_idx, float* msg_val, float* weights,
+                     void* stream) {
+  if (!weights || ((uintptr_t)weights & 15u) || (scale_mode != RTOPK_SCALE_MEAN && scale_mode != RTOPK_SCALE_SUM))
+    return RTOPK_ERR_INVALID_ARG;
+  if (!(eta >= 0.0f) || eta > 3.0e38f) return RTOPK_ERR_INVALID_ARG;
+  if (!ctx || d < 1 || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
+  const int64_t off[2] = {0, d};
+  const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed,
+                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, nullptr);
+  if (rc) return rc;
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, false, eta);
 }
 
 int rtopk_step(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,

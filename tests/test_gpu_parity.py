@@ -263,6 +263,66 @@ def test_aggregate_sparse_path_many_workers_and_crowded_tiles(lib):
         ctx.close()
 
 
+def test_master_update_against_oracle(lib):
+    """Algorithm 1's w <- w - eta * ghat straight from the messages: bit-equal to the oracle on the
+    sparse path (few entries per tile), the dense path, shared coordinates and -0.0 weights."""
+    rng = np.random.default_rng(123)
+    cases = []
+    d, W, k = 2_000_003, 8, 900                        # sparse path, own run search
+    cases.append((d, np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)])))
+    d, W, k = 3_000_017, 70, 400                       # sparse path behind the table of run starts
+    cases.append((d, np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)])))
+    d, W, k = 100_003, 6, 20_000                       # dense path, ragged last tile
+    cases.append((d, np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)])))
+    d, W, k = 1_000_000, 5, 3000                       # identical supports: every coordinate shared by all
+    same = np.sort(rng.choice(d, k, replace=False))
+    cases.append((d, np.stack([same] * W)))
+    for d, idx in cases:
+        idx = idx.astype(np.uint32)
+        W, k = idx.shape
+        val = (rng.standard_normal((W, k)) * np.exp(2 * rng.standard_normal((W, k)))).astype(np.float32)
+        w0 = rng.standard_normal(wl.round_up(d, 4)).astype(np.float32)
+        w0[idx[0, :5].astype(np.int64)] = -0.0
+        w0[::1001] = -0.0
+        ctx = _ctx(lib, d, W, k, k)
+        for mode, eta in ((lib.SCALE_MEAN, 0.05), (lib.SCALE_SUM, 1.0), (lib.SCALE_MEAN, 0.0)):
+            w = torch.from_numpy(w0.copy()).cuda()
+            ctx.apply_update(torch.from_numpy(idx.view(np.int32)).cuda(), torch.from_numpy(val).cuda(), d, eta, w,
+                             scale_mode=mode)
+            want = oracle.apply_update(idx, val, d, eta, w0[:d], mode)
+            got = w.cpu().numpy()
+            assert np.array_equal(_bits(got[:d]), _bits(want))
+            assert np.array_equal(_bits(got[d:]), _bits(w0[d:]))          # padding is never touched
+        with pytest.raises(RuntimeError):
+            ctx.apply_update(torch.from_numpy(idx.view(np.int32)).cuda(), torch.from_numpy(val).cuda(), d, -0.1,
+                             torch.from_numpy(w0.copy()).cuda())
+        ctx.close()
+
+
+def test_step_apply_is_sparsify_then_update(lib):
+    cfg = wl.scaled(wl.configs()["c1"], d=300_007, W=4)
+    ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
+    rng = np.random.default_rng(5)
+    w0 = rng.standard_normal(cfg.ld).astype(np.float32)
+    w = torch.from_numpy(w0.copy()).cuda()
+    m = wl.zero_residual(cfg, "cuda")
+    m_ref = np.zeros((cfg.W, cfg.ld), dtype=np.float32)
+    idx = torch.zeros((cfg.W, cfg.k), dtype=torch.int32, device="cuda")
+    val = torch.zeros((cfg.W, cfg.k), dtype=torch.float32, device="cuda")
+    want = w0[:cfg.d].copy()
+    for t in range(3):
+        g = wl.gradient(cfg, t, "cuda")
+        ctx.step_apply(g, m, cfg.d, cfg.r, cfg.k, cfg.seed, t, 0.1, idx, val, w)
+        o_idx, o_val = oracle.sparsify(g.cpu().numpy(), m_ref, cfg.d, cfg.r, cfg.k, cfg.seed, t)
+        want = oracle.apply_update(o_idx, o_val, cfg.d, 0.1, want)
+        assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx)
+        assert np.array_equal(_bits(val.cpu().numpy()), _bits(o_val))
+        assert np.array_equal(_bits(m.cpu().numpy()), _bits(m_ref))
+        assert np.array_equal(_bits(w.cpu().numpy()[:cfg.d]), _bits(want))
+    ctx.poll_status()
+    ctx.close()
+
+
 def test_step_is_sparsify_then_aggregate(lib):
     cfg = wl.configs()["c1"]
     ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
