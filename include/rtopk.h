@@ -55,8 +55,16 @@ typedef enum {
 /* gradient element type; residual, message values and the update are always binary32 */
 enum { RTOPK_F32 = 0, RTOPK_BF16 = 1 };
 
-/* scaling of the aggregated update: 1/W as in Algorithm 1's master step, or the plain sum */
-enum { RTOPK_SCALE_MEAN = 0, RTOPK_SCALE_SUM = 1 };
+/* Scaling of the aggregated update (S_i = sum over the workers that sent coordinate i, in double):
+ *   MEAN      S_i / W                 Algorithm 1's master step;
+ *   SUM       S_i;
+ *   UNBIASED  S_i * r / (W * k)       the estimator in the proof of Theorem 1, (1/n) sum_w X_w / S with
+ *                                     subsampling fraction S = k / r (needs r: rtopk_step, rtopk_step_apply,
+ *                                     rtopk_aggregate_unbiased; the segmented step returns UNSUPPORTED);
+ *   COUNT     S_i / c_i               c_i = number of workers that sent i (the average over the updates a
+ *                                     coordinate received, a second reading of the master step; W <= 65535).
+ * All four are rounded to binary32 once. */
+enum { RTOPK_SCALE_MEAN = 0, RTOPK_SCALE_SUM = 1, RTOPK_SCALE_UNBIASED = 2, RTOPK_SCALE_COUNT = 3 };
 
 /* rtopk_set_option keys */
 enum {
@@ -126,7 +134,8 @@ int rtopk_sparsify(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_
                    uint64_t seed, uint32_t step, uint32_t* msg_idx, float* msg_val, void* stream);
 
 /*
- * Algorithm 1, master step: out_i = scale * sum_w [i in U_w] val_{w,i}, scale = 1/W or 1.
+ * Algorithm 1, master step: out_i = scale * sum_w [i in U_w] val_{w,i}; scale_mode MEAN, SUM or
+ * COUNT (UNBIASED: rtopk_aggregate_unbiased).
  * Sums run in double precision in worker order and are rounded once, so the result does not depend
  * on scheduling.  msg_idx rows must be ascending (as rtopk_sparsify writes them) with entries < d.
  *   msg_idx, msg_val [in]  W x k;   out [out]  d binary32, fully overwritten.
@@ -134,6 +143,11 @@ int rtopk_sparsify(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_
  */
 int rtopk_aggregate(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d,
                     int32_t W, int64_t k, int scale_mode, float* out, void* stream);
+
+/* rtopk_aggregate with the UNBIASED scaling, which needs the r the messages were drawn from
+ * (k <= r <= d).  Errors: INVALID_ARG, CUDA. */
+int rtopk_aggregate_unbiased(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d,
+                             int32_t W, int64_t k, int64_t r, float* out, void* stream);
 
 /*
  * Algorithm 1, master update w <- w - eta * ghat applied straight from the messages: ghat is the

@@ -23,7 +23,7 @@ _SRC = os.path.join(_HERE, "rtopk_oracle.cpp")
 _LIB = os.path.join(_HERE, "librtopk_oracle.so")
 
 GRAD_F32, GRAD_BF16 = 0, 1
-SCALE_MEAN, SCALE_SUM = 0, 1
+SCALE_MEAN, SCALE_SUM, SCALE_UNBIASED, SCALE_COUNT = 0, 1, 2, 3
 
 _lib = None
 
@@ -63,8 +63,10 @@ def lib() -> C.CDLL:
                                                 i64p, i64p, C.c_uint64, C.c_uint32, u32p, f32p]
         L.oracle_aggregate.argtypes = [u32p, f32p, C.c_int64, C.c_int32, C.c_int64, C.c_int,
                                        f64p, f32p]
+        L.oracle_aggregate_scaled.argtypes = [u32p, f32p, C.c_int64, C.c_int32, C.c_int64, C.c_int,
+                                              C.c_int64, f64p, f32p]
         L.oracle_apply_update.argtypes = [u32p, f32p, C.c_int64, C.c_int32, C.c_int64, C.c_int,
-                                          C.c_float, f32p]
+                                          C.c_int64, C.c_float, f32p]
         _lib = L
     return _lib
 
@@ -167,26 +169,27 @@ def sparsify_segmented(grad: np.ndarray, residual: np.ndarray, d: int, seg_off, 
     return idx, val
 
 
-def aggregate(msg_idx: np.ndarray, msg_val: np.ndarray, d: int, scale_mode: int = SCALE_MEAN):
-    """Algorithm 1 master average.  Returns (out64 float64 [d], out32 float32 [d])."""
+def aggregate(msg_idx: np.ndarray, msg_val: np.ndarray, d: int, scale_mode: int = SCALE_MEAN, r: int = 0):
+    """Algorithm 1 master average (``r`` only for SCALE_UNBIASED).
+    Returns (out64 float64 [d], out32 float32 [d])."""
     idx = np.ascontiguousarray(msg_idx, dtype=np.uint32)
     val = np.ascontiguousarray(msg_val, dtype=np.float32)
     W, k = idx.shape
     o64 = np.zeros(d, dtype=np.float64)
     o32 = np.zeros(d, dtype=np.float32)
-    _check(lib().oracle_aggregate(_p(idx, C.c_uint32), _p(val, C.c_float), d, W, k, scale_mode,
-                                  _p(o64, C.c_double), _p(o32, C.c_float)), "aggregate")
+    _check(lib().oracle_aggregate_scaled(_p(idx, C.c_uint32), _p(val, C.c_float), d, W, k, scale_mode, r,
+                                         _p(o64, C.c_double), _p(o32, C.c_float)), "aggregate")
     return o64, o32
 
 
 def apply_update(msg_idx: np.ndarray, msg_val: np.ndarray, d: int, eta: float, weights: np.ndarray,
-                 scale_mode: int = SCALE_MEAN) -> np.ndarray:
+                 scale_mode: int = SCALE_MEAN, r: int = 0) -> np.ndarray:
     """Algorithm 1 master update w - eta * ghat on a copy of `weights` (float32 [d])."""
     idx = np.ascontiguousarray(msg_idx, dtype=np.uint32)
     val = np.ascontiguousarray(msg_val, dtype=np.float32)
     W, k = idx.shape
     w = np.array(weights, dtype=np.float32, copy=True)
-    _check(lib().oracle_apply_update(_p(idx, C.c_uint32), _p(val, C.c_float), d, W, k, scale_mode,
+    _check(lib().oracle_apply_update(_p(idx, C.c_uint32), _p(val, C.c_float), d, W, k, scale_mode, r,
                                      C.c_float(eta), _p(w, C.c_float)), "apply_update")
     return w
 

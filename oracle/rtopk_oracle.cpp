@@ -47,7 +47,7 @@ namespace {
 
 enum { ORACLE_OK = 0, ORACLE_BAD_ARG = 1 };
 enum { GRAD_F32 = 0, GRAD_BF16 = 1 };
-enum { SCALE_MEAN = 0, SCALE_SUM = 1 };
+enum { SCALE_MEAN = 0, SCALE_SUM = 1, SCALE_UNBIASED = 2, SCALE_COUNT = 3 };
 
 int g_threads = 1;
 
@@ -272,33 +272,51 @@ int oracle_sparsify_segmented(const void* grad, int grad_dtype, int64_t ld_g, fl
 // Algorithm 1, master: dense sum of the W sparse messages in double precision,
 // workers in order, scaled by 1/W (mean) or 1 (sum).  out64 (optional) receives
 // the double result; out32 (optional) the same rounded once to binary32.
-int oracle_aggregate(const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
-                     int scale_mode, double* out64, float* out32) {
+// Algorithm 1, master step, with the scalings of the library's contract: S_i = sum of the values
+// the workers sent for coordinate i (double, worker order), c_i = how many sent it;
+//   MEAN S_i / W;  SUM S_i;  UNBIASED S_i * r / (W k) (the estimator in the proof of Theorem 1 with
+//   subsampling fraction k / r);  COUNT S_i / c_i (0 where nobody sent i).
+int oracle_aggregate_scaled(const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
+                            int scale_mode, int64_t r, double* out64, float* out32) {
   if (!msg_idx || !msg_val || d < 1 || W < 1 || k < 1) return ORACLE_BAD_ARG;
-  if (scale_mode != SCALE_MEAN && scale_mode != SCALE_SUM) return ORACLE_BAD_ARG;
+  if (scale_mode != SCALE_MEAN && scale_mode != SCALE_SUM && scale_mode != SCALE_UNBIASED && scale_mode != SCALE_COUNT)
+    return ORACLE_BAD_ARG;
+  if (scale_mode == SCALE_UNBIASED && (r < k || r > d)) return ORACLE_BAD_ARG;
   std::vector<double> acc((size_t)d, 0.0);
+  std::vector<uint32_t> senders((size_t)d, 0u);
   for (int32_t w = 0; w < W; ++w)
     for (int64_t q = 0; q < k; ++q) {
       const uint32_t i = msg_idx[(size_t)w * (size_t)k + (size_t)q];
       if ((int64_t)i >= d) return ORACLE_BAD_ARG;
       acc[i] += (double)msg_val[(size_t)w * (size_t)k + (size_t)q];
+      senders[i] += 1u;
     }
   for (int64_t i = 0; i < d; ++i) {
-    const double v = scale_mode == SCALE_MEAN ? acc[(size_t)i] / (double)W : acc[(size_t)i];
+    const double s = acc[(size_t)i];
+    double v = s;
+    if (scale_mode == SCALE_MEAN) v = s / (double)W;
+    else if (scale_mode == SCALE_UNBIASED) v = (s * (double)r) / ((double)W * (double)k);
+    else if (scale_mode == SCALE_COUNT) v = senders[(size_t)i] ? s / (double)senders[(size_t)i] : 0.0;
     if (out64) out64[i] = v;
     if (out32) out32[i] = (float)v;
   }
   return ORACLE_OK;
 }
 
+int oracle_aggregate(const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
+                     int scale_mode, double* out64, float* out32) {
+  if (scale_mode != SCALE_MEAN && scale_mode != SCALE_SUM && scale_mode != SCALE_COUNT) return ORACLE_BAD_ARG;
+  return oracle_aggregate_scaled(msg_idx, msg_val, d, W, k, scale_mode, 0, out64, out32);
+}
+
 // Algorithm 1, master update: w <- w - eta * ghat with ghat the average (or sum) above, for every
 // coordinate.  eta >= 0 (with a negative eta a zero weight at an unsent coordinate would change
 // its sign, which the sparse restatements of this update never touch).
 int oracle_apply_update(const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
-                        int scale_mode, float eta, float* weights) {
+                        int scale_mode, int64_t r, float eta, float* weights) {
   if (!weights || !(eta >= 0.0f) || eta > 3.0e38f) return ORACLE_BAD_ARG;
   std::vector<float> ghat((size_t)d);
-  const int rc = oracle_aggregate(msg_idx, msg_val, d, W, k, scale_mode, nullptr, ghat.data());
+  const int rc = oracle_aggregate_scaled(msg_idx, msg_val, d, W, k, scale_mode, r, nullptr, ghat.data());
   if (rc != ORACLE_OK) return rc;
   for (int64_t i = 0; i < d; ++i)
     weights[i] = (float)((double)weights[i] - (double)eta * (double)ghat[(size_t)i]);

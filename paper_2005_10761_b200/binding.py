@@ -14,7 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "librtopk.so")
 
 GRAD_F32, GRAD_BF16 = 0, 1
-SCALE_MEAN, SCALE_SUM = 0, 1
+SCALE_MEAN, SCALE_SUM, SCALE_UNBIASED, SCALE_COUNT = 0, 1, 2, 3
 OPT_SELECT_PATH, OPT_PROFILE = 0, 1
 PHASES = ("subset", "threshold", "stream", "order", "exact", "finish", "aggregate")
 
@@ -33,6 +33,7 @@ EXPORTS = {
     "rtopk_aggregate": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _int, _vp, _vp]),
     "rtopk_step": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _i64, _u64, _u32, _int,
                           _vp, _vp, _vp, _vp]),
+    "rtopk_aggregate_unbiased": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _i64, _vp, _vp]),
     "rtopk_apply_update": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _int, C.c_float, _vp, _vp]),
     "rtopk_step_apply": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _i64, _u64, _u32, _int,
                                 C.c_float, _vp, _vp, _vp, _vp]),
@@ -173,6 +174,12 @@ class RTopK:
                                   residual.data_ptr(), residual.stride(0), d, W, worker_base, r, k, seed, step,
                                   scale_mode, msg_idx.data_ptr(), msg_val.data_ptr(), out.data_ptr(), _stream())
         self._check(rc, "rtopk_step")
+
+    def aggregate_unbiased(self, msg_idx, msg_val, d, r, out) -> None:
+        W, k = msg_idx.shape
+        rc = self._lib.rtopk_aggregate_unbiased(self._h, msg_idx.data_ptr(), msg_val.data_ptr(), d, W, k, r,
+                                                out.data_ptr(), _stream())
+        self._check(rc, "rtopk_aggregate_unbiased")
 
     def apply_update(self, msg_idx, msg_val, d, eta, weights, scale_mode=SCALE_MEAN) -> None:
         W, k = msg_idx.shape

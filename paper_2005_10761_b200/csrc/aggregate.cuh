@@ -23,6 +23,15 @@ constexpr int kAggSparseStage = 2048;   // entries of one such tile staged in sh
 constexpr int kAggMaxW = 1024;    // workers the sparse kernel keeps run tables for
 constexpr int kAggSearchW = 64;   // up to this many workers the sparse kernel finds the runs itself
 
+// How a coordinate's double-precision sum becomes the update: sum * num / den (Algorithm 1's 1/W:
+// num = 1, den = W; the plain sum: 1, 1; the unbiased estimator's r / (W k): r, W k), or, with
+// by_count, the sum divided by the number of workers that sent the coordinate.
+struct AggScale { double num, den; int by_count; };
+__device__ __forceinline__ double agg_scaled(double sum, uint32_t senders, const AggScale& sc) {
+  if (sc.by_count) return senders ? sum / (double)senders : 0.0;
+  return (sum * sc.num) / sc.den;
+}
+
 // What a coordinate's slot receives: the average itself, or (Algorithm 1's master update
 // w <- w - eta * ghat, with eta < 0 meaning "store the average") the updated weight, rounded once
 // from double; the product of two binary32 numbers is exact in double.
@@ -70,21 +79,24 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_starts(const uint32_t* __re
   starts[(size_t)w * (ntiles + 1) + t] = t == ntiles ? K : lower_bound_u32(row, K, t * tile_size);
 }
 
+template <bool COUNT>   // COUNT: also keep the number of senders per coordinate (smaller stage to make room)
 __global__ void __launch_bounds__(kAggThreads) k_aggregate(const uint32_t* __restrict__ msg_idx,
                                                            const float* __restrict__ msg_val,
                                                            const uint32_t* __restrict__ starts, uint32_t d,
-                                                           uint32_t W, uint32_t K, int mean,
+                                                           uint32_t W, uint32_t K, AggScale sc,
                                                            float eta, float* __restrict__ out) {
+  constexpr int kStage = COUNT ? kAggStage / 2 : kAggStage;
   __shared__ double acc[kAggTile];
+  __shared__ uint16_t senders[COUNT ? kAggTile : 1];    // at most 65535 workers (checked by the host)
   __shared__ uint32_t s_beg[kAggThreads], s_pre[kAggThreads + 1];
-  __shared__ uint32_t st_idx[kAggStage];
-  __shared__ float st_val[kAggStage];
+  __shared__ uint32_t st_idx[kStage];
+  __shared__ float st_val[kStage];
   __shared__ uint32_t s_warp[kAggThreads / 32];
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t ntiles = gridDim.x;
   const uint32_t lo = blockIdx.x * (uint32_t)kAggTile;
   const uint32_t hi = min(d, lo + (uint32_t)kAggTile);
-  for (uint32_t i = tid; i < (uint32_t)kAggTile; i += kAggThreads) acc[i] = 0.0;
+  for (uint32_t i = tid; i < (uint32_t)kAggTile; i += kAggThreads) { acc[i] = 0.0; if (COUNT) senders[i] = 0; }
   for (uint32_t w0 = 0; w0 < W; w0 += kAggThreads) {
     const uint32_t nw = min((uint32_t)kAggThreads, W - w0);
     __syncthreads();
@@ -105,7 +117,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(const uint32_t* __res
     if (tid == kAggThreads - 1) s_pre[kAggThreads] = woff + incl;
     __syncthreads();
     const uint32_t total = s_pre[kAggThreads];
-    if (total <= (uint32_t)kAggStage) {
+    if (total <= (uint32_t)kStage) {
       // stage every entry of the tile with one round of loads, then add worker by worker
       for (uint32_t q = tid; q < total; q += kAggThreads) {
         uint32_t a = 0, b = nw;                       // last worker with s_pre[w] <= q
@@ -120,7 +132,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(const uint32_t* __res
         if (e > b) {                                   // block-uniform
           for (uint32_t q = b + tid; q < e; q += kAggThreads) {
             const uint32_t i = st_idx[q] - lo;        // the unsigned check keeps a malformed row inside the tile
-            if (i < (uint32_t)kAggTile) acc[i] += (double)st_val[q];
+            if (i < (uint32_t)kAggTile) { acc[i] += (double)st_val[q]; if (COUNT) ++senders[i]; }
           }
           __syncthreads();
         }
@@ -131,22 +143,21 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(const uint32_t* __res
         const size_t row = (size_t)(w0 + w) * K;
         for (uint32_t q = tid; q < n; q += kAggThreads) {
           const uint32_t i = __ldg(msg_idx + row + b + q) - lo;
-          if (i < (uint32_t)kAggTile) acc[i] += (double)__ldg(msg_val + row + b + q);
+          if (i < (uint32_t)kAggTile) { acc[i] += (double)__ldg(msg_val + row + b + q); if (COUNT) ++senders[i]; }
         }
         __syncthreads();
       }
     }
   }
   __syncthreads();
-  const double inv = (double)W;
+  auto scaled = [&](uint32_t i) -> float {                 // most entries are zero: skip their division
+    const double a = acc[i];
+    return (float)(a != 0.0 ? agg_scaled(a, COUNT ? (uint32_t)senders[i] : 0u, sc) : a);
+  };
   if (hi - lo == (uint32_t)kAggTile) {
     for (uint32_t i = tid * 4; i < (uint32_t)kAggTile; i += kAggThreads * 4) {
-      const double a0 = acc[i + 0], a1 = acc[i + 1], a2 = acc[i + 2], a3 = acc[i + 3];
       float4 o;
-      o.x = (float)(mean && a0 != 0.0 ? a0 / inv : a0);   // most entries are zero: skip their division
-      o.y = (float)(mean && a1 != 0.0 ? a1 / inv : a1);
-      o.z = (float)(mean && a2 != 0.0 ? a2 / inv : a2);
-      o.w = (float)(mean && a3 != 0.0 ? a3 / inv : a3);
+      o.x = scaled(i + 0); o.y = scaled(i + 1); o.z = scaled(i + 2); o.w = scaled(i + 3);
       if (eta >= 0.0f) {                                   // master update: out holds the weights
         const float4 w4 = *reinterpret_cast<const float4*>(out + lo + i);
         o.x = agg_result(o.x, w4.x, eta); o.y = agg_result(o.y, w4.y, eta);
@@ -156,8 +167,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(const uint32_t* __res
     }
   } else {
     for (uint32_t i = tid; i < hi - lo; i += kAggThreads) {
-      const float ghat = (float)(mean ? acc[i] / inv : acc[i]);
-      out[lo + i] = agg_result(ghat, eta >= 0.0f ? out[lo + i] : 0.0f, eta);
+      out[lo + i] = agg_result(scaled(i), eta >= 0.0f ? out[lo + i] : 0.0f, eta);
     }
   }
 }
@@ -168,7 +178,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(const uint32_t* __res
 __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(const uint32_t* __restrict__ msg_idx,
                                                                   const float* __restrict__ msg_val,
                                                                   const uint32_t* __restrict__ starts, uint32_t d,
-                                                                  uint32_t W, uint32_t K, int mean,
+                                                                  uint32_t W, uint32_t K, AggScale sc,
                                                                   float eta, float* __restrict__ out) {
   __shared__ uint32_t s_beg[kAggMaxW], s_pre[kAggMaxW + 1], s_cnt[kAggSearchW];
   __shared__ uint32_t st_idx[kAggSparseStage];
@@ -262,8 +272,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(const uint32_t
       if (local >= (uint32_t)kAggSparseTile || idx >= d) continue;    // malformed row: ignore
       if (!((s_shared[local >> 5] >> (local & 31u)) & 1u)) {    // sole sender: the sum is the value
         const double v = (double)st_val[q];
-        const float ghat = (float)(mean ? v / (double)W : v);
-        out[idx] = agg_result(ghat, eta >= 0.0f ? out[idx] : 0.0f, eta);
+        out[idx] = agg_result((float)agg_scaled(v, 1u, sc), eta >= 0.0f ? out[idx] : 0.0f, eta);
         continue;
       }
     }
@@ -271,20 +280,21 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(const uint32_t
     const uint32_t idx = idx_at(w, q - s_pre[w]);
     if (idx - lo >= (uint32_t)kAggSparseTile || idx >= d) continue;   // malformed row: ignore
     double sum = 0.0;
+    uint32_t senders = 0;
     bool owner = true;
     for (uint32_t x = 0; x < W; ++x) {
-      if (x == w) { sum += (double)val_at(w, q - s_pre[w]); continue; }
+      if (x == w) { sum += (double)val_at(w, q - s_pre[w]); ++senders; continue; }
       const uint32_t n = s_pre[x + 1] - s_pre[x];
       uint32_t a = 0, b = n;
       while (a < b) { const uint32_t mid = (a + b) >> 1; if (idx_at(x, mid) < idx) a = mid + 1; else b = mid; }
       if (a < n && idx_at(x, a) == idx) {
         if (x < w) { owner = false; break; }          // a lower worker owns this coordinate
         sum += (double)val_at(x, a);
+        ++senders;
       }
     }
     if (owner) {
-      const float ghat = (float)(mean ? sum / (double)W : sum);
-      out[idx] = agg_result(ghat, eta >= 0.0f ? out[idx] : 0.0f, eta);
+      out[idx] = agg_result((float)agg_scaled(sum, senders, sc), eta >= 0.0f ? out[idx] : 0.0f, eta);
     }
   }
 }

@@ -418,6 +418,10 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   return RTOPK_OK;
 }
 
+bool scale_mode_known(int m) {
+  return m == RTOPK_SCALE_MEAN || m == RTOPK_SCALE_SUM || m == RTOPK_SCALE_UNBIASED || m == RTOPK_SCALE_COUNT;
+}
+
 bool aggregate_is_sparse(int64_t d, int32_t W, int64_t k) {
   return W <= kAggMaxW && (uint64_t)W * (uint64_t)k * 16ull <= (uint64_t)d;   // <= 1024 entries per tile on average
 }
@@ -427,10 +431,13 @@ bool aggregate_is_sparse(int64_t d, int32_t W, int64_t k) {
 // eta < 0: `out` receives the average.  eta >= 0: `out` holds weights and receives w - eta * average
 // (only the coordinates some worker sent change, so nothing is cleared).
 int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
-                   int scale_mode, float* out, cudaStream_t st, bool out_cleared = false, float eta = -1.0f) {
+                   int scale_mode, float* out, cudaStream_t st, bool out_cleared = false, float eta = -1.0f,
+                   int64_t r = 0) {
   if (!ctx || !msg_idx || !msg_val || !out) return RTOPK_ERR_INVALID_ARG;
   if (d < 1 || d > ctx->d_max || W < 1 || W > ctx->W_max || k < 1 || k > d) return RTOPK_ERR_INVALID_ARG;
-  if (scale_mode != RTOPK_SCALE_MEAN && scale_mode != RTOPK_SCALE_SUM) return RTOPK_ERR_INVALID_ARG;
+  if (!scale_mode_known(scale_mode)) return RTOPK_ERR_INVALID_ARG;
+  if (scale_mode == RTOPK_SCALE_UNBIASED && (r < k || r > d)) return RTOPK_ERR_INVALID_ARG;   // needs the call's r
+  if (scale_mode == RTOPK_SCALE_COUNT && W > 65535) return RTOPK_ERR_UNSUPPORTED;
   if (((uintptr_t)out & 15u) || ((uintptr_t)msg_idx & 3u) || ((uintptr_t)msg_val & 3u)) return RTOPK_ERR_INVALID_ARG;
   if ((uint64_t)k * (uint64_t)W >= (1ull << 32)) return RTOPK_ERR_INVALID_ARG;
   const bool sparse = aggregate_is_sparse(d, W, k);
@@ -447,16 +454,23 @@ int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val
     k_agg_starts<<<sgrid, kAggThreads, 0, st>>>(msg_idx, (uint32_t)W, (uint32_t)k, ntiles, tile, ctx->d_agg_starts);
     ++ctx->launches;
   }
-  const int mean = scale_mode == RTOPK_SCALE_MEAN ? 1 : 0;
+  AggScale sc = {1.0, 1.0, 0};
+  if (scale_mode == RTOPK_SCALE_MEAN) sc.den = (double)W;
+  else if (scale_mode == RTOPK_SCALE_UNBIASED) { sc.num = (double)r; sc.den = (double)W * (double)k; }
+  else if (scale_mode == RTOPK_SCALE_COUNT) sc.by_count = 1;
   if (sparse) {
     // few coordinates are touched: clear the update, then compute only what was sent
     if (!out_cleared && eta < 0.0f) RTOPK_CUDA(ctx, cudaMemsetAsync(out, 0, (size_t)d * sizeof(float), st));
     k_aggregate_sparse<<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, own_search ? nullptr : ctx->d_agg_starts, (uint32_t)d,
-                                                       (uint32_t)W, (uint32_t)k, mean, eta, out);
+                                                       (uint32_t)W, (uint32_t)k, sc, eta, out);
     ++ctx->launches;
   } else {
-    k_aggregate<<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, ctx->d_agg_starts, (uint32_t)d, (uint32_t)W,
-                                                (uint32_t)k, mean, eta, out);
+    if (sc.by_count)
+      k_aggregate<true><<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, ctx->d_agg_starts, (uint32_t)d, (uint32_t)W,
+                                                        (uint32_t)k, sc, eta, out);
+    else
+      k_aggregate<false><<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, ctx->d_agg_starts, (uint32_t)d, (uint32_t)W,
+                                                         (uint32_t)k, sc, eta, out);
     ++ctx->launches;
   }
   mark(ctx, RTOPK_N_PHASES, st);
@@ -624,6 +638,11 @@ int rtopk_aggregate(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_va
   return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, out, (cudaStream_t)stream);
 }
 
+int rtopk_aggregate_unbiased(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W,
+                             int64_t k, int64_t r, float* out, void* stream) {
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, RTOPK_SCALE_UNBIASED, out, (cudaStream_t)stream, false, -1.0f, r);
+}
+
 int rtopk_apply_update(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W,
                        int64_t k, int scale_mode, float eta, float* weights, void* stream) {
   if (!(eta >= 0.0f) || eta > 3.0e38f) return RTOPK_ERR_INVALID_ARG;
@@ -634,37 +653,35 @@ int rtopk_step_apply(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t l
                      int64_t d, int32_t W, int32_t worker_base, int64_t r, int64_t k, uint64_t seed,
                      uint32_t step, int scale_mode, float eta, uint32_t* msg_idx, float* msg_val, float* weights,
                      void* stream) {
-  if (!weights || ((uintptr_t)weights & 15u) || (scale_mode != RTOPK_SCALE_MEAN && scale_mode != RTOPK_SCALE_SUM))
-    return RTOPK_ERR_INVALID_ARG;
+  if (!weights || ((uintptr_t)weights & 15u) || !scale_mode_known(scale_mode)) return RTOPK_ERR_INVALID_ARG;
   if (!(eta >= 0.0f) || eta > 3.0e38f) return RTOPK_ERR_INVALID_ARG;
   if (!ctx || d < 1 || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
   const int64_t off[2] = {0, d};
   const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed,
                                step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, nullptr);
   if (rc) return rc;
-  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, false, eta);
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, false, eta, r);
 }
 
 int rtopk_step(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
                int64_t d, int32_t W, int32_t worker_base, int64_t r, int64_t k, uint64_t seed, uint32_t step,
                int scale_mode, uint32_t* msg_idx, float* msg_val, float* out, void* stream) {
-  if (!out || ((uintptr_t)out & 15u) || (scale_mode != RTOPK_SCALE_MEAN && scale_mode != RTOPK_SCALE_SUM))
-    return RTOPK_ERR_INVALID_ARG;
+  if (!out || ((uintptr_t)out & 15u) || !scale_mode_known(scale_mode)) return RTOPK_ERR_INVALID_ARG;
   if (!ctx || d < 1 || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
   const bool sparse = W >= 1 && k >= 1 && aggregate_is_sparse(d, W, k);
   const int64_t off[2] = {0, d};
   const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed,
                                step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, sparse ? out : nullptr);
   if (rc) return rc;
-  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, out, (cudaStream_t)stream, sparse);
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, out, (cudaStream_t)stream, sparse, -1.0f, r);
 }
 
 int rtopk_step_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,
                          int64_t ld_m, int64_t d, int32_t W, int32_t worker_base, int32_t S, const int64_t* seg_off,
                          const int64_t* seg_r, const int64_t* seg_k, uint64_t seed, uint32_t step, int scale_mode,
                          uint32_t* msg_idx, float* msg_val, float* out, void* stream) {
-  if (!out || ((uintptr_t)out & 15u) || (scale_mode != RTOPK_SCALE_MEAN && scale_mode != RTOPK_SCALE_SUM))
-    return RTOPK_ERR_INVALID_ARG;
+  if (!out || ((uintptr_t)out & 15u) || !scale_mode_known(scale_mode)) return RTOPK_ERR_INVALID_ARG;
+  if (scale_mode == RTOPK_SCALE_UNBIASED) return RTOPK_ERR_UNSUPPORTED;   // r / k differs from tensor to tensor
   if (!ctx || d < 1 || d > ctx->d_max || S < 1 || S > ctx->S_max || !seg_k) return RTOPK_ERR_INVALID_ARG;
   int64_t Ksum = 0;
   for (int s = 0; s < S; ++s) Ksum += seg_k[s] > 0 ? seg_k[s] : 0;

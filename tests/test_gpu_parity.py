@@ -263,6 +263,70 @@ def test_aggregate_sparse_path_many_workers_and_crowded_tiles(lib):
         ctx.close()
 
 
+def test_aggregate_scalings_against_oracle(lib):
+    """UNBIASED (r / (W k), the estimator in the proof of Theorem 1) and COUNT (sum over senders /
+    number of senders) on the sparse path, the dense path and with shared coordinates."""
+    rng = np.random.default_rng(77)
+    cases = []
+    d, W, k = 2_000_003, 8, 900
+    cases.append((d, np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)])))
+    d, W, k = 100_003, 6, 20_000
+    cases.append((d, np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)])))
+    d, W, k = 50_000, 300, 2_000                       # dense path, more workers than one block batch
+    cases.append((d, np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)])))
+    d, W, k = 1_000_000, 5, 3000
+    same = np.sort(rng.choice(d, k, replace=False))
+    cases.append((d, np.stack([same] * W)))
+    for d, idx in cases:
+        idx = idx.astype(np.uint32)
+        W, k = idx.shape
+        val = (rng.standard_normal((W, k)) * np.exp(2 * rng.standard_normal((W, k)))).astype(np.float32)
+        ctx = _ctx(lib, d, W, k, k)
+        t_idx, t_val = torch.from_numpy(idx.view(np.int32)).cuda(), torch.from_numpy(val).cuda()
+        out = torch.full((wl.round_up(d, 4),), float("nan"), dtype=torch.float32, device="cuda")
+        r = min(d, 7 * k + 3)
+        ctx.aggregate_unbiased(t_idx, t_val, d, r, out)
+        _, want = oracle.aggregate(idx, val, d, oracle.SCALE_UNBIASED, r=r)
+        assert np.array_equal(_bits(out.cpu().numpy()[:d]), _bits(want))
+        out.fill_(float("nan"))
+        ctx.aggregate(t_idx, t_val, d, out, scale_mode=lib.SCALE_COUNT)
+        _, want = oracle.aggregate(idx, val, d, oracle.SCALE_COUNT)
+        assert np.array_equal(_bits(out.cpu().numpy()[:d]), _bits(want))
+        # the update with by-count scaling
+        w0 = rng.standard_normal(wl.round_up(d, 4)).astype(np.float32)
+        w = torch.from_numpy(w0.copy()).cuda()
+        ctx.apply_update(t_idx, t_val, d, 0.25, w, scale_mode=lib.SCALE_COUNT)
+        want = oracle.apply_update(idx, val, d, 0.25, w0[:d], oracle.SCALE_COUNT)
+        assert np.array_equal(_bits(w.cpu().numpy()[:d]), _bits(want))
+        with pytest.raises(RuntimeError):                # UNBIASED needs r
+            ctx.aggregate(t_idx, t_val, d, out, scale_mode=lib.SCALE_UNBIASED)
+        ctx.close()
+
+
+def test_step_with_unbiased_scaling(lib):
+    cfg = wl.scaled(wl.configs()["c1"], d=300_007, W=4)
+    ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
+    g = wl.gradient(cfg, 0, "cuda")
+    m = wl.zero_residual(cfg, "cuda")
+    m_ref = np.zeros((cfg.W, cfg.ld), dtype=np.float32)
+    idx = torch.zeros((cfg.W, cfg.k), dtype=torch.int32, device="cuda")
+    val = torch.zeros((cfg.W, cfg.k), dtype=torch.float32, device="cuda")
+    out = torch.full((cfg.ld,), float("nan"), dtype=torch.float32, device="cuda")
+    ctx.step(g, m, cfg.d, cfg.r, cfg.k, cfg.seed, 0, idx, val, out, scale_mode=lib.SCALE_UNBIASED)
+    o_idx, o_val = oracle.sparsify(g.cpu().numpy(), m_ref, cfg.d, cfg.r, cfg.k, cfg.seed, 0)
+    _, want = oracle.aggregate(o_idx, o_val, cfg.d, oracle.SCALE_UNBIASED, r=cfg.r)
+    assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx)
+    assert np.array_equal(_bits(out.cpu().numpy()[:cfg.d]), _bits(want))
+    w0 = np.linspace(-1, 1, cfg.ld).astype(np.float32)
+    w = torch.from_numpy(w0.copy()).cuda()
+    ctx.step_apply(g, m, cfg.d, cfg.r, cfg.k, cfg.seed, 1, 0.5, idx, val, w, scale_mode=lib.SCALE_UNBIASED)
+    o_idx, o_val = oracle.sparsify(g.cpu().numpy(), m_ref, cfg.d, cfg.r, cfg.k, cfg.seed, 1)
+    want = oracle.apply_update(o_idx, o_val, cfg.d, 0.5, w0[:cfg.d], oracle.SCALE_UNBIASED, r=cfg.r)
+    assert np.array_equal(_bits(w.cpu().numpy()[:cfg.d]), _bits(want))
+    ctx.poll_status()
+    ctx.close()
+
+
 def test_master_update_against_oracle(lib):
     """Algorithm 1's w <- w - eta * ghat straight from the messages: bit-equal to the oracle on the
     sparse path (few entries per tile), the dense path, shared coordinates and -0.0 weights."""

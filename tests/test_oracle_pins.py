@@ -413,6 +413,53 @@ def test_master_update_worked_example_and_textbook_sgd():
         oracle.apply_update(idx4, val4, d, -1.0, w0)
 
 
+def test_aggregate_scalings_unbiased_and_by_count():
+    # the worked example again: S = [1, 0, 6, 8], senders c = [1, 0, 2, 1], W = 2, k = 2
+    idx = np.array([[0, 2], [2, 3]], dtype=np.uint32)
+    val = np.array([[1, 2], [4, 8]], dtype=np.float32)
+    u64, _ = oracle.aggregate(idx, val, 4, oracle.SCALE_UNBIASED, r=3)       # S * 3 / 4
+    assert u64.tolist() == [0.75, 0.0, 4.5, 6.0]
+    c64, _ = oracle.aggregate(idx, val, 4, oracle.SCALE_COUNT)               # S / c
+    assert c64.tolist() == [1.0, 0.0, 3.0, 8.0]
+    # k = r: the unbiased scaling is the mean; disjoint supports: by-count is the sum; identical
+    # supports: by-count is the mean
+    rng = np.random.default_rng(8)
+    d, W, k = 4000, 6, 300
+    idx = np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)]).astype(np.uint32)
+    val = rng.standard_normal((W, k)).astype(np.float32)
+    m64, _ = oracle.aggregate(idx, val, d)
+    u64, _ = oracle.aggregate(idx, val, d, oracle.SCALE_UNBIASED, r=k)
+    assert np.allclose(u64, m64, rtol=1e-15, atol=0)
+    u64, _ = oracle.aggregate(idx, val, d, oracle.SCALE_UNBIASED, r=4 * k)   # r / k = 4: exact scaling
+    assert np.array_equal(u64, 4.0 * m64) or np.allclose(u64, 4.0 * m64, rtol=1e-15, atol=0)
+    idx_d = np.arange(W * k, dtype=np.uint32).reshape(W, k)
+    c64, _ = oracle.aggregate(idx_d, val, d, oracle.SCALE_COUNT)
+    s64, _ = oracle.aggregate(idx_d, val, d, oracle.SCALE_SUM)
+    assert np.array_equal(c64, s64)
+    same = np.stack([idx[0]] * W)
+    c64, _ = oracle.aggregate(same, val, d, oracle.SCALE_COUNT)
+    m64, _ = oracle.aggregate(same, val, d)
+    assert np.array_equal(c64, m64)
+    # by-count against numpy: sums and sender counts by np.add.at
+    ref, cnt = np.zeros(d), np.zeros(d)
+    np.add.at(ref, idx.ravel().astype(np.int64), val.ravel().astype(np.float64))
+    np.add.at(cnt, idx.ravel().astype(np.int64), 1.0)
+    c64, c32 = oracle.aggregate(idx, val, d, oracle.SCALE_COUNT)
+    want = np.divide(ref, cnt, out=np.zeros(d), where=cnt > 0)
+    assert np.allclose(c64, want, rtol=1e-14, atol=0) and np.array_equal(c32, c64.astype(np.float32))
+    # unbiasedness (Definition 3 + the estimator's 1/S): averaged over many subsets of a fixed top-r
+    # list, (r/k) * message converges to the list itself
+    r, k2, trials = 12, 3, 6000
+    vals = np.arange(1, r + 1, dtype=np.float64)
+    acc = np.zeros(r)
+    for t in range(trials):
+        pos = oracle.sample_positions(r, k2, seed=99, worker=0, segment=0, step=t)
+        acc[pos] += vals[pos] * r / k2
+    assert np.allclose(acc / trials, vals, rtol=0.08)
+    with pytest.raises(ValueError):
+        oracle.aggregate(idx, val, d, oracle.SCALE_UNBIASED, r=k - 1)
+
+
 def test_bad_arguments_are_rejected():
     g = np.zeros((1, 8), dtype=np.float32)
     m = np.zeros((1, 8), dtype=np.float32)
