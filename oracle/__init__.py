@@ -67,6 +67,12 @@ def lib() -> C.CDLL:
                                               C.c_int64, f64p, f32p]
         L.oracle_apply_update.argtypes = [u32p, f32p, C.c_int64, C.c_int32, C.c_int64, C.c_int,
                                           C.c_int64, C.c_float, f32p]
+        u16p = C.POINTER(C.c_uint16)
+        L.oracle_index_bits.argtypes = [C.c_int64]
+        L.oracle_bf16_rne.argtypes = [C.c_float]
+        L.oracle_bf16_rne.restype = C.c_uint16
+        L.oracle_encode_row.argtypes = [u32p, f32p, C.c_int64, C.c_int64, u32p, u16p, f32p]
+        L.oracle_decode_row.argtypes = [u32p, u16p, C.c_int64, C.c_int64, u32p, f32p]
         _lib = L
     return _lib
 
@@ -192,6 +198,46 @@ def apply_update(msg_idx: np.ndarray, msg_val: np.ndarray, d: int, eta: float, w
     _check(lib().oracle_apply_update(_p(idx, C.c_uint32), _p(val, C.c_float), d, W, k, scale_mode, r,
                                      C.c_float(eta), _p(w, C.c_float)), "apply_update")
     return w
+
+
+def index_bits(d: int) -> int:
+    return int(lib().oracle_index_bits(d))
+
+
+def bf16_rne(x: float) -> int:
+    return int(lib().oracle_bf16_rne(C.c_float(x)))
+
+
+def packed_words(d: int, k: int) -> int:
+    return (k * index_bits(d) + 31) // 32
+
+
+def encode(msg_idx: np.ndarray, msg_val: np.ndarray, d: int, residual: np.ndarray | None = None):
+    """Packed form of W rows of k (index, value) pairs: (uint32 [W, words], uint16 [W, k]).  When
+    ``residual`` (float32 [W, ld]) is given, the bfloat16 rounding error is written to the sent
+    coordinates' slots in place."""
+    idx = np.ascontiguousarray(msg_idx, dtype=np.uint32)
+    val = np.ascontiguousarray(msg_val, dtype=np.float32)
+    W, k = idx.shape
+    pi = np.zeros((W, packed_words(d, k)), dtype=np.uint32)
+    pv = np.zeros((W, k), dtype=np.uint16)
+    for w in range(W):
+        res = None if residual is None else residual[w].ctypes.data_as(C.POINTER(C.c_float))
+        _check(lib().oracle_encode_row(_p(idx[w], C.c_uint32), _p(val[w], C.c_float), k, d, _p(pi[w], C.c_uint32),
+                                       _p(pv[w], C.c_uint16), res), "encode_row")
+    return pi, pv
+
+
+def decode(packed_idx: np.ndarray, packed_val: np.ndarray, d: int, k: int):
+    pi = np.ascontiguousarray(packed_idx, dtype=np.uint32)
+    pv = np.ascontiguousarray(packed_val, dtype=np.uint16)
+    W = pi.shape[0]
+    idx = np.zeros((W, k), dtype=np.uint32)
+    val = np.zeros((W, k), dtype=np.float32)
+    for w in range(W):
+        _check(lib().oracle_decode_row(_p(pi[w], C.c_uint32), _p(pv[w], C.c_uint16), k, d, _p(idx[w], C.c_uint32),
+                                       _p(val[w], C.c_float)), "decode_row")
+    return idx, val
 
 
 if __name__ == "__main__":

@@ -38,6 +38,7 @@
 // Proposition 1 and the limits k = r (Def. 1) and r = d (Def. 2).
 
 #include <algorithm>
+#include <cmath>
 #include <cstdint>
 #include <cstring>
 #include <thread>
@@ -320,6 +321,77 @@ int oracle_apply_update(const uint32_t* msg_idx, const float* msg_val, int64_t d
   if (rc != ORACLE_OK) return rc;
   for (int64_t i = 0; i < d; ++i)
     weights[i] = (float)((double)weights[i] - (double)eta * (double)ghat[(size_t)i]);
+  return ORACLE_OK;
+}
+
+// ----------------------------------------------------------------------------- message codec
+// Section III notes that an index costs log d bits and a value a constant number of bits.  The
+// library's packed message format states one such encoding:
+//   * indices: b = ceil(log2 d) bits each (1 when d <= 2), entry j at bits [j b, (j + 1) b) of the
+//     row's bit stream; bit p of the stream is bit (p mod 32) of 32-bit word p / 32;
+//   * values: bfloat16 = the upper 16 bits of the binary32 value rounded to nearest, ties to even
+//     (a NaN becomes 0x7FC0);
+//   * error feedback of the rounding (Algorithm 1: m = a - ghat with ghat what is sent): the
+//     residual slot of a sent coordinate receives a - widen(q(a)), one binary32 subtraction, or
+//     +0.0f when widen(q(a)) is not finite.
+int oracle_index_bits(int64_t d) {
+  int b = 1;
+  while (b < 63 && ((int64_t)1 << b) < d) ++b;
+  return b;
+}
+
+uint16_t oracle_bf16_rne(float x) {
+  uint32_t u;
+  std::memcpy(&u, &x, 4);
+  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return 0x7FC0u;          // NaN
+  const uint32_t lsb = (u >> 16) & 1u;
+  u += 0x7FFFu + lsb;                                            // round to nearest, ties to even
+  return (uint16_t)(u >> 16);
+}
+
+// One row: k ascending (index, value) pairs -> packed_idx (ceil(k b / 32) words, zero-filled first)
+// and packed_val (k halves); residual (may be null) gets the rounding error at the sent coordinates.
+int oracle_encode_row(const uint32_t* idx, const float* val, int64_t k, int64_t d, uint32_t* packed_idx,
+                      uint16_t* packed_val, float* residual) {
+  if (!idx || !val || !packed_idx || !packed_val || k < 1 || d < 1) return ORACLE_BAD_ARG;
+  const int b = oracle_index_bits(d);
+  if (b > 32) return ORACLE_BAD_ARG;
+  const int64_t nwords = (k * b + 31) / 32;
+  for (int64_t w = 0; w < nwords; ++w) packed_idx[w] = 0;
+  for (int64_t j = 0; j < k; ++j) {
+    if ((int64_t)idx[j] >= d) return ORACLE_BAD_ARG;
+    for (int bit = 0; bit < b; ++bit)
+      if ((idx[j] >> bit) & 1u) {
+        const int64_t p = j * b + bit;
+        packed_idx[p / 32] |= 1u << (p % 32);
+      }
+    const uint16_t q = oracle_bf16_rne(val[j]);
+    packed_val[j] = q;
+    if (residual) {
+      const uint32_t wide = (uint32_t)q << 16;
+      float back;
+      std::memcpy(&back, &wide, 4);
+      residual[idx[j]] = std::isfinite(back) ? val[j] - back : 0.0f;
+    }
+  }
+  return ORACLE_OK;
+}
+
+int oracle_decode_row(const uint32_t* packed_idx, const uint16_t* packed_val, int64_t k, int64_t d, uint32_t* idx,
+                      float* val) {
+  if (!idx || !val || !packed_idx || !packed_val || k < 1 || d < 1) return ORACLE_BAD_ARG;
+  const int b = oracle_index_bits(d);
+  if (b > 32) return ORACLE_BAD_ARG;
+  for (int64_t j = 0; j < k; ++j) {
+    uint32_t v = 0;
+    for (int bit = 0; bit < b; ++bit) {
+      const int64_t p = j * b + bit;
+      v |= ((packed_idx[p / 32] >> (p % 32)) & 1u) << bit;
+    }
+    idx[j] = v;
+    const uint32_t wide = (uint32_t)packed_val[j] << 16;
+    std::memcpy(&val[j], &wide, 4);
+  }
   return ORACLE_OK;
 }
 

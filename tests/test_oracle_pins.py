@@ -466,3 +466,80 @@ def test_bad_arguments_are_rejected():
     for d, r, k in [(8, 4, 5), (8, 9, 1), (8, 4, 0), (9, 4, 1)]:
         with pytest.raises(ValueError):
             oracle.sparsify(g, m, d, r, k, seed=0, step=0)
+
+
+# ----------------------------------------------------------------------------- message codec
+def test_codec_index_bits_and_hand_packed_words():
+    # Section III: an index costs log d bits.  b = ceil(log2 d), at least 1.
+    for d, b in [(1, 1), (2, 1), (3, 2), (4, 2), (5, 3), (1000, 10), (1024, 10), (1025, 11), (2**31, 31), (2**32 - 1, 32)]:
+        assert oracle.index_bits(d) == b
+    # d = 1000 (b = 10), indices 1, 2, 1023 -> not allowed (>= d); use 999: the bit stream is the
+    # little-endian integer sum idx_j << (10 j): written out by hand for three entries
+    idx = np.array([[1, 2, 999, 512]], dtype=np.uint32)
+    val = np.array([[1.0, -2.0, 0.5, 3.0]], dtype=np.float32)
+    pi, pv = oracle.encode(idx, val, 1000)
+    stream = 1 | (2 << 10) | (999 << 20) | (512 << 30)             # 40 bits
+    assert pi.shape == (1, 2) and int(pi[0, 0]) == stream & 0xFFFFFFFF and int(pi[0, 1]) == stream >> 32
+    assert pv[0].tolist() == [0x3F80, 0xC000, 0x3F00, 0x4040]
+
+
+def test_codec_bit_stream_against_big_integers_and_round_trip():
+    rng = np.random.default_rng(31)
+    for d, k in [(2, 5), (37, 64), (1000, 333), (1 << 20, 1000), ((1 << 24) + 1, 257), (2**32 - 1, 50)]:
+        b = oracle.index_bits(d)
+        idx = np.sort(rng.choice(min(d, 1 << 40), size=min(k, d), replace=False) if d <= (1 << 26)
+                      else np.unique(rng.integers(0, d, size=4 * k))[:k]).astype(np.uint32)[None, :]
+        kk = idx.shape[1]
+        val = rng.standard_normal((1, kk)).astype(np.float32)
+        pi, pv = oracle.encode(idx, val, d)
+        big = 0
+        for j, v in enumerate(idx[0].tolist()):
+            big |= v << (j * b)
+        words = [(big >> (32 * w)) & 0xFFFFFFFF for w in range(pi.shape[1])]
+        assert pi[0].tolist() == words and pi.shape[1] == (kk * b + 31) // 32
+        i2, v2 = oracle.decode(pi, pv, d, kk)
+        assert np.array_equal(i2, idx)
+        assert np.array_equal(v2.view(np.uint32), pv.astype(np.uint32) << 16)
+
+
+def test_codec_bfloat16_rounding_against_torch_and_rules():
+    import torch
+    rng = np.random.default_rng(32)
+    x = np.concatenate([
+        (rng.standard_normal(20000) * np.exp(8 * rng.standard_normal(20000))).astype(np.float32),
+        rng.integers(0, 2**32, size=20000, dtype=np.uint64).astype(np.uint32).view(np.float32),
+        np.array([0.0, -0.0, 1.0, np.inf, -np.inf, 3.3895314e38, 3.4028235e38, 1e-45, 1.17549435e-38], dtype=np.float32),
+        np.array([0x3F808000, 0x3F818000, 0x3F807FFF, 0x3F808001, 0x7F7F8000], dtype=np.uint32).view(np.float32),
+    ])
+    x = x[~np.isnan(x)]
+    ours = np.array([oracle.bf16_rne(float(v)) for v in x], dtype=np.uint16)
+    theirs = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(ours, theirs)
+    # the rules spelled out: exact halves go to the even neighbour, NaN is the default quiet NaN
+    assert oracle.bf16_rne(float(np.array([0x3F808000], dtype=np.uint32).view(np.float32)[0])) == 0x3F80   # tie -> even (down)
+    assert oracle.bf16_rne(float(np.array([0x3F818000], dtype=np.uint32).view(np.float32)[0])) == 0x3F82   # tie -> even (up)
+    assert oracle.bf16_rne(float("nan")) == 0x7FC0
+    assert oracle.bf16_rne(3.4028235e38) == 0x7F80                                                    # rounds to +inf
+
+
+def test_codec_rounding_error_goes_to_the_residual():
+    # Algorithm 1: m = a - ghat, with ghat the value that is sent.  The decoded value plus the
+    # residual slot gives back a exactly (the rounding error of bfloat16 is a binary32 number).
+    rng = np.random.default_rng(33)
+    d, k = 5000, 400
+    idx = np.sort(rng.choice(d, k, replace=False)).astype(np.uint32)[None, :]
+    val = (rng.standard_normal((1, k)) * np.exp(3 * rng.standard_normal((1, k)))).astype(np.float32)
+    val[0, 0] = 3.4e38          # rounds to +inf: no finite error to keep
+    val[0, 1] = 1.0             # exact in bfloat16: the slot stays +0.0
+    m = rng.standard_normal((1, d)).astype(np.float32)
+    m[0, idx[0].astype(np.int64)] = 0.0
+    m0 = m.copy()
+    pi, pv = oracle.encode(idx, val, d, residual=m)
+    _, back = oracle.decode(pi, pv, d, k)
+    sent = idx[0].astype(np.int64)
+    ok = np.isfinite(back[0])
+    assert np.array_equal((back[0][ok].astype(np.float64) + m[0, sent][ok].astype(np.float64)), val[0][ok].astype(np.float64))
+    assert m[0, sent[0]] == 0.0 and m[0, sent[1]] == 0.0 and not np.signbit(m[0, sent[1]])
+    untouched = np.ones(d, dtype=bool); untouched[sent] = False
+    assert np.array_equal(m[0, untouched].view(np.uint32), m0[0, untouched].view(np.uint32))
+    assert np.all(np.abs(m[0, sent][ok]) <= np.abs(val[0][ok]) * 2.0**-8)
