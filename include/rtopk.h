@@ -150,6 +150,37 @@ int rtopk_aggregate_unbiased(rtopk_ctx* ctx, const uint32_t* msg_idx, const floa
                              int32_t W, int64_t k, int64_t r, float* out, void* stream);
 
 /*
+ * Packed message format.  Section III counts log d bits per index and a constant number of bits per
+ * value; this format spends exactly b = ceil(log2 d) bits (at least 1) per index and 16 per value:
+ *   packed_idx  W rows of ld_words 32-bit words: entry j of a row occupies bits [j b, (j + 1) b) of
+ *               the row's bit stream, bit p of the stream being bit (p mod 32) of word p / 32;
+ *   packed_val  W rows of ld_halves bfloat16 values (binary32 rounded to nearest, ties to even,
+ *               upper 16 bits; NaN -> 0x7FC0).
+ * rtopk_packed_layout (host only, no GPU work) returns b and the smallest accepted row strides
+ * (ld_words a multiple of 4, ld_halves a multiple of 8); any of the three outputs may be null.
+ * Errors: INVALID_ARG (d < 1, d >= 2^32, k < 1 or k > d).
+ */
+int rtopk_packed_layout(int64_t d, int64_t k, int32_t* index_bits, int64_t* ld_words, int64_t* ld_halves);
+
+/*
+ * Encodes W rows of k (index, value) pairs (as rtopk_sparsify writes them) into the packed format.
+ * Algorithm 1 keeps m = a - ghat with ghat what is sent: when `residual` (W x ld_m, the buffer the
+ * sparsify call updated) is not null, the slot of every sent coordinate receives the rounding error
+ * a - widen(bfloat16(a)) (one binary32 subtraction; +0.0f when the rounded value is not finite).
+ * Row padding of the outputs is written as zero.  All pointers are device pointers; packed_idx and
+ * packed_val 16-byte aligned.  Errors: INVALID_ARG, CUDA.
+ */
+int rtopk_encode(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W,
+                 int64_t k, float* residual, int64_t ld_m, uint32_t* packed_idx, int64_t ld_words,
+                 uint16_t* packed_val, int64_t ld_halves, void* stream);
+
+/* rtopk_aggregate reading the packed format directly (the decoder is fused into the aggregation
+ * kernels).  scale_mode MEAN, SUM or COUNT.  Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+int rtopk_aggregate_packed(rtopk_ctx* ctx, const uint32_t* packed_idx, int64_t ld_words,
+                           const uint16_t* packed_val, int64_t ld_halves, int64_t d, int32_t W,
+                           int64_t k, int scale_mode, float* out, void* stream);
+
+/*
  * Algorithm 1, master update w <- w - eta * ghat applied straight from the messages: ghat is the
  * binary32 result rtopk_aggregate would write, and every coordinate that some worker sent receives
  * fp32(double(w_i) - double(eta) * double(ghat_i)) (one rounding); all other weights are not touched

@@ -34,6 +34,9 @@ EXPORTS = {
     "rtopk_step": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _i64, _u64, _u32, _int,
                           _vp, _vp, _vp, _vp]),
     "rtopk_aggregate_unbiased": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _i64, _vp, _vp]),
+    "rtopk_packed_layout": (_int, [_i64, _i64, C.POINTER(_i32), C.POINTER(_i64), C.POINTER(_i64)]),
+    "rtopk_encode": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _vp]),
+    "rtopk_aggregate_packed": (_int, [_vp, _vp, _i64, _vp, _i64, _i64, _i32, _i64, _int, _vp, _vp]),
     "rtopk_apply_update": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _int, C.c_float, _vp, _vp]),
     "rtopk_step_apply": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _i64, _u64, _u32, _int,
                                 C.c_float, _vp, _vp, _vp, _vp]),
@@ -60,6 +63,15 @@ class RTopKError(RuntimeError):
     def __init__(self, status: int, what: str, detail: str = ""):
         self.status = status
         super().__init__(f"{what}: status {status} ({detail})")
+
+
+def packed_layout(d: int, k: int):
+    """(index bits, row stride in 32-bit words, row stride in 16-bit halves) of the packed format."""
+    bits, lw, lh = _i32(0), _i64(0), _i64(0)
+    rc = load_library().rtopk_packed_layout(d, k, C.byref(bits), C.byref(lw), C.byref(lh))
+    if rc != 0:
+        raise RTopKError(rc, "rtopk_packed_layout", "invalid argument")
+    return int(bits.value), int(lw.value), int(lh.value)
 
 
 def library_path() -> str:
@@ -180,6 +192,24 @@ class RTopK:
         rc = self._lib.rtopk_aggregate_unbiased(self._h, msg_idx.data_ptr(), msg_val.data_ptr(), d, W, k, r,
                                                 out.data_ptr(), _stream())
         self._check(rc, "rtopk_aggregate_unbiased")
+
+    def encode(self, msg_idx, msg_val, d, packed_idx, packed_val, residual=None) -> None:
+        """msg -> packed rows (int32 [W, ld_words], int16 [W, ld_halves]); with `residual` the
+        bfloat16 rounding error goes back into the sent coordinates' slots."""
+        W, k = msg_idx.shape
+        rc = self._lib.rtopk_encode(self._h, msg_idx.data_ptr(), msg_val.data_ptr(), d, W, k,
+                                    residual.data_ptr() if residual is not None else None,
+                                    residual.stride(0) if residual is not None else 0,
+                                    packed_idx.data_ptr(), packed_idx.stride(0), packed_val.data_ptr(),
+                                    packed_val.stride(0), _stream())
+        self._check(rc, "rtopk_encode")
+
+    def aggregate_packed(self, packed_idx, packed_val, d, k, out, scale_mode=SCALE_MEAN) -> None:
+        W = packed_idx.shape[0]
+        rc = self._lib.rtopk_aggregate_packed(self._h, packed_idx.data_ptr(), packed_idx.stride(0),
+                                              packed_val.data_ptr(), packed_val.stride(0), d, W, k, scale_mode,
+                                              out.data_ptr(), _stream())
+        self._check(rc, "rtopk_aggregate_packed")
 
     def apply_update(self, msg_idx, msg_val, d, eta, weights, scale_mode=SCALE_MEAN) -> None:
         W, k = msg_idx.shape

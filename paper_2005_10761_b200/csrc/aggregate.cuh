@@ -39,25 +39,56 @@ __device__ __forceinline__ float agg_result(float ghat, float old, float eta) {
   return eta < 0.0f ? ghat : (float)((double)old - (double)eta * (double)ghat);
 }
 
-__device__ __forceinline__ uint32_t lower_bound_u32(const uint32_t* a, uint32_t n, uint32_t key) {
+// The W x K messages as the kernels read them: plain (u32 index, f32 value) rows, or the packed
+// format (Section III: an index costs log d bits, a value a constant number): `bits` = ceil(log2 d)
+// bits per index, entry j at bits [j * bits, (j + 1) * bits) of the row's little-endian stream of
+// 32-bit words, and bfloat16 values (the upper half of the binary32 pattern).
+struct PlainMsgs {
+  const uint32_t* idx;
+  const float* val;
+  uint32_t K;
+  __device__ __forceinline__ uint32_t index(uint32_t w, uint32_t j) const { return __ldg(idx + (size_t)w * K + j); }
+  __device__ __forceinline__ float value(uint32_t w, uint32_t j) const { return __ldg(val + (size_t)w * K + j); }
+};
+struct PackedMsgs {
+  const uint32_t* words;
+  const uint16_t* halves;
+  uint32_t ld_words, ld_halves, bits;
+  __device__ __forceinline__ uint32_t index(uint32_t w, uint32_t j) const {
+    const uint32_t* row = words + (size_t)w * ld_words;
+    const uint64_t p = (uint64_t)j * bits;
+    const uint32_t wi = (uint32_t)(p >> 5), sh = (uint32_t)p & 31u;
+    uint32_t v = __ldg(row + wi) >> sh;
+    if (sh + bits > 32u) v |= __ldg(row + wi + 1) << (32u - sh);
+    return bits >= 32u ? v : v & ((1u << bits) - 1u);
+  }
+  __device__ __forceinline__ float value(uint32_t w, uint32_t j) const {
+    return __uint_as_float((uint32_t)__ldg(halves + (size_t)w * ld_halves + j) << 16);
+  }
+};
+
+// first entry of worker w's ascending row (n entries) whose index is >= key
+template <typename M>
+__device__ __forceinline__ uint32_t lower_bound_row(const M& msgs, uint32_t w, uint32_t n, uint32_t key) {
   uint32_t lo = 0, hi = n;
   while (lo < hi) {
     const uint32_t mid = (lo + hi) >> 1;
-    if (__ldg(a + mid) < key) lo = mid + 1; else hi = mid;
+    if (msgs.index(w, mid) < key) lo = mid + 1; else hi = mid;
   }
   return lo;
 }
 
 // The same as a 16-way search by each half of a warp (lanes 0-15 share one key, lanes 16-31
-// another): every lane of a half returns that half's lower bound.  a is sorted ascending.
-__device__ __forceinline__ uint32_t half_warp_lower_bound(const uint32_t* a, uint32_t n, uint32_t key, uint32_t lane) {
+// another): every lane of a half returns that half's lower bound in worker w's ascending row.
+template <typename M>
+__device__ __forceinline__ uint32_t half_warp_lower_bound(const M& msgs, uint32_t w, uint32_t n, uint32_t key, uint32_t lane) {
   const uint32_t l = lane & 15u, sh = lane & 16u;
   uint32_t lo = 0, hi = n;                                   // the answer lies in [lo, hi]
   // both halves run the same number of steps (the range shrinks 16-fold per step whatever the key)
   for (uint32_t span = n; span > 0; span = span > 16u ? (span + 15u) / 16u - 1u : 0u) {
     const uint32_t step = (hi - lo + 15u) / 16u;              // 0 once this half is done
     const uint32_t probe = min(lo + (l + 1u) * step, hi) - 1u; // < hi; unused when step == 0
-    const bool less = step != 0u && __ldg(a + (step ? probe : 0u)) < key;
+    const bool less = step != 0u && msgs.index(w, step ? probe : 0u) < key;
     const uint32_t cnt = __popc((__ballot_sync(0xFFFFFFFFu, less) >> sh) & 0xFFFFu);
     if (step != 0u) {
       const uint32_t nlo = min(hi, lo + cnt * step);
@@ -69,20 +100,17 @@ __device__ __forceinline__ uint32_t half_warp_lower_bound(const uint32_t* a, uin
 }
 
 // starts[w * (ntiles + 1) + t] = first entry of worker w with index >= t * tile_size (K for t = ntiles)
-__global__ void __launch_bounds__(kAggThreads) k_agg_starts(const uint32_t* __restrict__ msg_idx, uint32_t W,
-                                                            uint32_t K, uint32_t ntiles, uint32_t tile_size,
-                                                            uint32_t* __restrict__ starts) {
+template <typename M>
+__global__ void __launch_bounds__(kAggThreads) k_agg_starts(M msgs, uint32_t W, uint32_t K, uint32_t ntiles,
+                                                            uint32_t tile_size, uint32_t* __restrict__ starts) {
   const uint32_t t = blockIdx.x * kAggThreads + threadIdx.x;
   const uint32_t w = blockIdx.y;
   if (t > ntiles || w >= W) return;
-  const uint32_t* row = msg_idx + (size_t)w * K;
-  starts[(size_t)w * (ntiles + 1) + t] = t == ntiles ? K : lower_bound_u32(row, K, t * tile_size);
+  starts[(size_t)w * (ntiles + 1) + t] = t == ntiles ? K : lower_bound_row(msgs, w, K, t * tile_size);
 }
 
-template <bool COUNT>   // COUNT: also keep the number of senders per coordinate (smaller stage to make room)
-__global__ void __launch_bounds__(kAggThreads) k_aggregate(const uint32_t* __restrict__ msg_idx,
-                                                           const float* __restrict__ msg_val,
-                                                           const uint32_t* __restrict__ starts, uint32_t d,
+template <typename M, bool COUNT>   // COUNT: also keep the number of senders per coordinate (smaller stage to make room)
+__global__ void __launch_bounds__(kAggThreads) k_aggregate(M msgs, const uint32_t* __restrict__ starts, uint32_t d,
                                                            uint32_t W, uint32_t K, AggScale sc,
                                                            float eta, float* __restrict__ out) {
   constexpr int kStage = COUNT ? kAggStage / 2 : kAggStage;
@@ -122,9 +150,9 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(const uint32_t* __res
       for (uint32_t q = tid; q < total; q += kAggThreads) {
         uint32_t a = 0, b = nw;                       // last worker with s_pre[w] <= q
         while (b - a > 1) { const uint32_t mid = (a + b) >> 1; if (s_pre[mid] <= q) a = mid; else b = mid; }
-        const size_t at = (size_t)(w0 + a) * K + s_beg[a] + (q - s_pre[a]);
-        st_idx[q] = __ldg(msg_idx + at);
-        st_val[q] = __ldg(msg_val + at);
+        const uint32_t j = s_beg[a] + (q - s_pre[a]);
+        st_idx[q] = msgs.index(w0 + a, j);
+        st_val[q] = msgs.value(w0 + a, j);
       }
       __syncthreads();
       for (uint32_t w = 0; w < nw; ++w) {
@@ -140,10 +168,9 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(const uint32_t* __res
     } else {
       for (uint32_t w = 0; w < nw; ++w) {
         const uint32_t b = s_beg[w], n = s_pre[w + 1] - s_pre[w];
-        const size_t row = (size_t)(w0 + w) * K;
         for (uint32_t q = tid; q < n; q += kAggThreads) {
-          const uint32_t i = __ldg(msg_idx + row + b + q) - lo;
-          if (i < (uint32_t)kAggTile) { acc[i] += (double)__ldg(msg_val + row + b + q); if (COUNT) ++senders[i]; }
+          const uint32_t i = msgs.index(w0 + w, b + q) - lo;
+          if (i < (uint32_t)kAggTile) { acc[i] += (double)msgs.value(w0 + w, b + q); if (COUNT) ++senders[i]; }
         }
         __syncthreads();
       }
@@ -175,9 +202,8 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(const uint32_t* __res
 // A block stages the entries of its tile (all workers' runs, in worker order); the entry of the
 // lowest worker that holds a coordinate owns it and sums that coordinate over the workers in
 // ascending order (binary search in each staged run): the same fixed-order sum as k_aggregate.
-__global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(const uint32_t* __restrict__ msg_idx,
-                                                                  const float* __restrict__ msg_val,
-                                                                  const uint32_t* __restrict__ starts, uint32_t d,
+template <typename M>
+__global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const uint32_t* __restrict__ starts, uint32_t d,
                                                                   uint32_t W, uint32_t K, AggScale sc,
                                                                   float eta, float* __restrict__ out) {
   __shared__ uint32_t s_beg[kAggMaxW], s_pre[kAggMaxW + 1], s_cnt[kAggSearchW];
@@ -194,10 +220,9 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(const uint32_t
     // no table of run starts: a warp per worker finds the run of this tile in the worker's sorted
     // row, half the warp searching for each end (16-way search: a few dependent loads)
     for (uint32_t w = warp; w < W; w += kAggThreads / 32) {
-      const uint32_t* row = msg_idx + (size_t)w * K;
       const uint32_t end = lo > 0xFFFFFFFFu - (uint32_t)kAggSparseTile ? 0xFFFFFFFFu : lo + (uint32_t)kAggSparseTile;
       const uint32_t key = lane < 16 ? lo : end;                 // every index is below 2^32 - 1
-      const uint32_t at = half_warp_lower_bound(row, K, key, lane);
+      const uint32_t at = half_warp_lower_bound(msgs, w, K, key, lane);
       const uint32_t e = __shfl_sync(0xFFFFFFFFu, at, 16);
       if (lane == 0) { s_beg[w] = at; s_cnt[w] = e - at; }
     }
@@ -239,17 +264,17 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(const uint32_t
   if (staged) {
     for (uint32_t q = tid; q < total; q += kAggThreads) {
       const uint32_t a = worker_of(q);
-      const size_t at = (size_t)a * K + s_beg[a] + (q - s_pre[a]);
-      st_idx[q] = __ldg(msg_idx + at);
-      st_val[q] = __ldg(msg_val + at);
+      const uint32_t j = s_beg[a] + (q - s_pre[a]);
+      st_idx[q] = msgs.index(a, j);
+      st_val[q] = msgs.value(a, j);
     }
     __syncthreads();
   }
   auto idx_at = [&](uint32_t w, uint32_t j) {        // j-th entry of worker w's run in this tile
-    return staged ? st_idx[s_pre[w] + j] : __ldg(msg_idx + (size_t)w * K + s_beg[w] + j);
+    return staged ? st_idx[s_pre[w] + j] : msgs.index(w, s_beg[w] + j);
   };
   auto val_at = [&](uint32_t w, uint32_t j) {
-    return staged ? st_val[s_pre[w] + j] : __ldg(msg_val + (size_t)w * K + s_beg[w] + j);
+    return staged ? st_val[s_pre[w] + j] : msgs.value(w, s_beg[w] + j);
   };
   // Most coordinates are sent by a single worker.  Two bitmaps over the tile find the ones that are
   // not: the second entry that sets a coordinate's "seen" bit also sets its "shared" bit.

@@ -15,6 +15,7 @@
 #include <vector>
 
 #include "aggregate.cuh"
+#include "codec.cuh"
 #include "common.cuh"
 #include "sampler.cuh"
 #include "select.cuh"
@@ -430,15 +431,15 @@ bool aggregate_is_sparse(int64_t d, int32_t W, int64_t k) {
 // the streaming pass).
 // eta < 0: `out` receives the average.  eta >= 0: `out` holds weights and receives w - eta * average
 // (only the coordinates some worker sent change, so nothing is cleared).
-int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
-                   int scale_mode, float* out, cudaStream_t st, bool out_cleared = false, float eta = -1.0f,
-                   int64_t r = 0) {
-  if (!ctx || !msg_idx || !msg_val || !out) return RTOPK_ERR_INVALID_ARG;
+template <typename M>
+int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_t k, int scale_mode, float* out,
+                     cudaStream_t st, bool out_cleared, float eta, int64_t r) {
+  if (!ctx || !out) return RTOPK_ERR_INVALID_ARG;
   if (d < 1 || d > ctx->d_max || W < 1 || W > ctx->W_max || k < 1 || k > d) return RTOPK_ERR_INVALID_ARG;
   if (!scale_mode_known(scale_mode)) return RTOPK_ERR_INVALID_ARG;
   if (scale_mode == RTOPK_SCALE_UNBIASED && (r < k || r > d)) return RTOPK_ERR_INVALID_ARG;   // needs the call's r
   if (scale_mode == RTOPK_SCALE_COUNT && W > 65535) return RTOPK_ERR_UNSUPPORTED;
-  if (((uintptr_t)out & 15u) || ((uintptr_t)msg_idx & 3u) || ((uintptr_t)msg_val & 3u)) return RTOPK_ERR_INVALID_ARG;
+  if ((uintptr_t)out & 15u) return RTOPK_ERR_INVALID_ARG;
   if ((uint64_t)k * (uint64_t)W >= (1ull << 32)) return RTOPK_ERR_INVALID_ARG;
   const bool sparse = aggregate_is_sparse(d, W, k);
   const uint32_t tile = sparse ? (uint32_t)kAggSparseTile : (uint32_t)kAggTile;
@@ -451,7 +452,7 @@ int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val
   const bool own_search = sparse && W <= kAggSearchW && (uint64_t)ntiles * (uint64_t)((W + 7) / 8) <= 4096u;
   if (!own_search) {
     const dim3 sgrid((ntiles + 1 + kAggThreads - 1) / kAggThreads, (uint32_t)W);
-    k_agg_starts<<<sgrid, kAggThreads, 0, st>>>(msg_idx, (uint32_t)W, (uint32_t)k, ntiles, tile, ctx->d_agg_starts);
+    k_agg_starts<M><<<sgrid, kAggThreads, 0, st>>>(msgs, (uint32_t)W, (uint32_t)k, ntiles, tile, ctx->d_agg_starts);
     ++ctx->launches;
   }
   AggScale sc = {1.0, 1.0, 0};
@@ -461,20 +462,41 @@ int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val
   if (sparse) {
     // few coordinates are touched: clear the update, then compute only what was sent
     if (!out_cleared && eta < 0.0f) RTOPK_CUDA(ctx, cudaMemsetAsync(out, 0, (size_t)d * sizeof(float), st));
-    k_aggregate_sparse<<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, own_search ? nullptr : ctx->d_agg_starts, (uint32_t)d,
-                                                       (uint32_t)W, (uint32_t)k, sc, eta, out);
+    k_aggregate_sparse<M><<<ntiles, kAggThreads, 0, st>>>(msgs, own_search ? nullptr : ctx->d_agg_starts, (uint32_t)d,
+                                                          (uint32_t)W, (uint32_t)k, sc, eta, out);
     ++ctx->launches;
   } else {
     if (sc.by_count)
-      k_aggregate<true><<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, ctx->d_agg_starts, (uint32_t)d, (uint32_t)W,
-                                                        (uint32_t)k, sc, eta, out);
+      k_aggregate<M, true><<<ntiles, kAggThreads, 0, st>>>(msgs, ctx->d_agg_starts, (uint32_t)d, (uint32_t)W,
+                                                           (uint32_t)k, sc, eta, out);
     else
-      k_aggregate<false><<<ntiles, kAggThreads, 0, st>>>(msg_idx, msg_val, ctx->d_agg_starts, (uint32_t)d, (uint32_t)W,
-                                                         (uint32_t)k, sc, eta, out);
+      k_aggregate<M, false><<<ntiles, kAggThreads, 0, st>>>(msgs, ctx->d_agg_starts, (uint32_t)d, (uint32_t)W,
+                                                            (uint32_t)k, sc, eta, out);
     ++ctx->launches;
   }
   mark(ctx, RTOPK_N_PHASES, st);
   RTOPK_CUDA(ctx, cudaGetLastError());
+  return RTOPK_OK;
+}
+
+int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
+                   int scale_mode, float* out, cudaStream_t st, bool out_cleared = false, float eta = -1.0f,
+                   int64_t r = 0) {
+  if (!msg_idx || !msg_val || ((uintptr_t)msg_idx & 3u) || ((uintptr_t)msg_val & 3u)) return RTOPK_ERR_INVALID_ARG;
+  if (k < 1 || k > 0xFFFFFFFFll) return RTOPK_ERR_INVALID_ARG;
+  const PlainMsgs msgs = {msg_idx, msg_val, (uint32_t)k};
+  return aggregate_launch(ctx, msgs, d, W, k, scale_mode, out, st, out_cleared, eta, r);
+}
+
+// ceil(log2 d) index bits (at least 1) and the smallest row strides of the packed format: index
+// words rounded up to 4 (16 bytes), value halves rounded up to 8 (16 bytes).
+int packed_layout(int64_t d, int64_t k, int32_t* bits, int64_t* ld_words, int64_t* ld_halves) {
+  if (d < 1 || d > 0xFFFFFFFFll || k < 1 || k > d) return RTOPK_ERR_INVALID_ARG;
+  int b = 1;
+  while (((int64_t)1 << b) < d) ++b;
+  if (bits) *bits = b;
+  if (ld_words) *ld_words = (((k * b + 31) / 32) + 3) / 4 * 4;
+  if (ld_halves) *ld_halves = (k + 7) / 8 * 8;
   return RTOPK_OK;
 }
 
@@ -641,6 +663,51 @@ int rtopk_aggregate(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_va
 int rtopk_aggregate_unbiased(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W,
                              int64_t k, int64_t r, float* out, void* stream) {
   return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, RTOPK_SCALE_UNBIASED, out, (cudaStream_t)stream, false, -1.0f, r);
+}
+
+int rtopk_packed_layout(int64_t d, int64_t k, int32_t* index_bits, int64_t* ld_words, int64_t* ld_halves) {
+  return packed_layout(d, k, index_bits, ld_words, ld_halves);
+}
+
+int rtopk_encode(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
+                 float* residual, int64_t ld_m, uint32_t* packed_idx, int64_t ld_words, uint16_t* packed_val,
+                 int64_t ld_halves, void* stream) {
+  if (!ctx || !msg_idx || !msg_val || !packed_idx || !packed_val) return RTOPK_ERR_INVALID_ARG;
+  if (W < 1 || W > ctx->W_max || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
+  int32_t bits = 0;
+  int64_t min_words = 0, min_halves = 0;
+  if (packed_layout(d, k, &bits, &min_words, &min_halves)) return RTOPK_ERR_INVALID_ARG;
+  if (ld_words < min_words || ld_halves < min_halves || ld_words > 0xFFFFFFFFll || ld_halves > 0xFFFFFFFFll ||
+      (ld_words % 4) || (ld_halves % 8))
+    return RTOPK_ERR_INVALID_ARG;
+  if (((uintptr_t)msg_idx & 3u) || ((uintptr_t)msg_val & 3u) || ((uintptr_t)packed_idx & 15u) || ((uintptr_t)packed_val & 15u))
+    return RTOPK_ERR_INVALID_ARG;
+  if (residual && (ld_m < d || ((uintptr_t)residual & 3u))) return RTOPK_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return RTOPK_ERR_CUDA;
+  const uint32_t span = (uint32_t)std::max(ld_words, ld_halves);
+  const dim3 grid((span + kCodecThreads - 1) / kCodecThreads, (uint32_t)W);
+  k_encode<<<grid, kCodecThreads, 0, (cudaStream_t)stream>>>(msg_idx, msg_val, (uint32_t)k, (uint32_t)bits, residual, ld_m,
+                                                             packed_idx, (uint32_t)ld_words, packed_val,
+                                                             (uint32_t)ld_halves);
+  ++ctx->launches;
+  RTOPK_CUDA(ctx, cudaGetLastError());
+  return RTOPK_OK;
+}
+
+int rtopk_aggregate_packed(rtopk_ctx* ctx, const uint32_t* packed_idx, int64_t ld_words, const uint16_t* packed_val,
+                           int64_t ld_halves, int64_t d, int32_t W, int64_t k, int scale_mode, float* out,
+                           void* stream) {
+  if (!packed_idx || !packed_val || ((uintptr_t)packed_idx & 3u) || ((uintptr_t)packed_val & 1u))
+    return RTOPK_ERR_INVALID_ARG;
+  int32_t bits = 0;
+  int64_t min_words = 0, min_halves = 0;
+  if (packed_layout(d, k, &bits, &min_words, &min_halves)) return RTOPK_ERR_INVALID_ARG;
+  if (ld_words < (k * bits + 31) / 32 || ld_halves < k || ld_words > 0xFFFFFFFFll || ld_halves > 0xFFFFFFFFll)
+    return RTOPK_ERR_INVALID_ARG;
+  if (scale_mode == RTOPK_SCALE_UNBIASED) return RTOPK_ERR_INVALID_ARG;   // needs r: scale the result by r / k instead
+  const PackedMsgs msgs = {packed_idx, packed_val, (uint32_t)ld_words, (uint32_t)ld_halves, (uint32_t)bits};
+  return aggregate_launch(ctx, msgs, d, W, k, scale_mode, out, (cudaStream_t)stream, false, -1.0f, 0);
 }
 
 int rtopk_apply_update(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W,

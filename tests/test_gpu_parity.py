@@ -263,6 +263,47 @@ def test_aggregate_sparse_path_many_workers_and_crowded_tiles(lib):
         ctx.close()
 
 
+def test_packed_messages_against_oracle(lib):
+    """Encoder (bit-packed indices, bfloat16 values, rounding error into the residual) and the
+    aggregation that decodes on the fly: bit-equal to the oracle's encoder and to the oracle's
+    aggregate of the decoded messages."""
+    rng = np.random.default_rng(2024)
+    cases = [(2_000_003, 8, 900), (100_003, 6, 20_000), (1 << 20, 3, 4097), (37, 2, 37), (5, 70, 3)]
+    for d, W, k in cases:
+        idx = np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)]).astype(np.uint32)
+        val = (rng.standard_normal((W, k)) * np.exp(3 * rng.standard_normal((W, k)))).astype(np.float32)
+        val[0, 0] = 3.4e38                      # rounds to +inf in bfloat16
+        val[W - 1, k - 1] = np.float32(np.nan)
+        bits, lw, lh = lib.packed_layout(d, k)
+        assert bits == oracle.index_bits(d) and lw >= oracle.packed_words(d, k) and lw % 4 == 0 and lh >= k and lh % 8 == 0
+        ld = wl.round_up(d, 4)
+        m0 = rng.standard_normal((W, ld)).astype(np.float32)
+        for w in range(W):
+            m0[w, idx[w].astype(np.int64)] = 0.0
+        m_ref = m0.copy()
+        o_pi, o_pv = oracle.encode(idx, val, d, residual=m_ref)
+        ctx = _ctx(lib, d, W, k, k)
+        t_idx, t_val = torch.from_numpy(idx.view(np.int32)).cuda(), torch.from_numpy(val).cuda()
+        m = torch.from_numpy(m0.copy()).cuda()
+        pi = torch.full((W, lw), -1, dtype=torch.int32, device="cuda")
+        pv = torch.full((W, lh), -1, dtype=torch.int16, device="cuda")
+        ctx.encode(t_idx, t_val, d, pi, pv, residual=m)
+        got_pi = pi.cpu().numpy().view(np.uint32)
+        got_pv = pv.cpu().numpy().view(np.uint16)
+        nw = o_pi.shape[1]
+        assert np.array_equal(got_pi[:, :nw], o_pi) and not got_pi[:, nw:].any()
+        assert np.array_equal(got_pv[:, :k], o_pv) and not got_pv[:, k:].any()
+        assert np.array_equal(_bits(m.cpu().numpy()), _bits(m_ref))
+        d_idx, d_val = oracle.decode(o_pi, o_pv, d, k)
+        assert np.array_equal(d_idx, idx)
+        out = torch.full((ld,), float("nan"), dtype=torch.float32, device="cuda")
+        for mode, omode in ((lib.SCALE_MEAN, oracle.SCALE_MEAN), (lib.SCALE_COUNT, oracle.SCALE_COUNT)):
+            ctx.aggregate_packed(pi, pv, d, k, out, scale_mode=mode)
+            _, want = oracle.aggregate(d_idx, d_val, d, omode)
+            assert np.array_equal(_bits(out.cpu().numpy()[:d]), _bits(want))
+        ctx.close()
+
+
 def test_aggregate_scalings_against_oracle(lib):
     """UNBIASED (r / (W k), the estimator in the proof of Theorem 1) and COUNT (sum over senders /
     number of senders) on the sparse path, the dense path and with shared coordinates."""
