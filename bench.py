@@ -205,6 +205,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--apply", action="store_true",
                     help="time rtopk_step_apply (master update fused into the aggregation; plain workloads, 1 GPU)")
+    ap.add_argument("--reuse-threshold", type=int, default=1, choices=[0, 1],
+                    help="1 (default): the rounds of the loop predict their first threshold from the previous "
+                         "rounds (RTOPK_OPT_REUSE_THRESHOLD; results are the same); 0: every round samples")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -238,6 +241,10 @@ def main():
     seg = cfg.seg_off is not None
     ctx = rt.RTopK(d_max=d, W_max=W_total, r_max=cfg.r, k_max=K, segments_max=len(cfg.seg_r) if seg else 1,
                    device=local)
+
+    if args.reuse_threshold:
+        from paper_2005_10761_b200.binding import OPT_REUSE_THRESHOLD
+        ctx.set_option(OPT_REUSE_THRESHOLD, 1)
 
     # gradient batches resident in HBM before timing; the residual is carried across all steps
     batch_bytes = W * ld * gsz
@@ -312,7 +319,9 @@ def main():
     ctx.poll_status()
     ms_per_step = total_ms / args.steps
     value = W_total * d * gsz / (ms_per_step * 1e-3) / 1e9
-    fallbacks = sum(ctx.stats(s)["used_fallback"] for s in range(W * (len(cfg.seg_r) if seg else 1)))
+    n_slices = W * (len(cfg.seg_r) if seg else 1)
+    fallbacks = sum(ctx.stats(s)["used_fallback"] for s in range(n_slices))     # of the last timed step
+    predicted = 0
 
     # the streaming kernel's own duration: same steps again with events between the phases
     ctx.set_option(OPT_PROFILE, 1)
@@ -323,6 +332,9 @@ def main():
             if ms >= 0:
                 phase_sum[name] = phase_sum.get(name, 0.0) + ms
         n_prof += 1
+        stats = [ctx.stats(s) for s in range(n_slices)]                         # ... and of every profiled step
+        fallbacks += sum(s["used_fallback"] for s in stats)
+        predicted += sum(s["bracket_predicted"] for s in stats)
     ctx.set_option(OPT_PROFILE, 0)
     phases = {k: v / n_prof for k, v in phase_sum.items()}
     peak, peak_src = load_peak()
@@ -380,10 +392,12 @@ def main():
                        "grad_dtype": cfg.grad_dtype, "recipe": cfg.recipe, "segments": len(cfg.seg_r) if seg else 1,
                        "gradient_batches_resident": n_batches, "residual": "carried across steps",
                        "l2": "inputs larger than L2 (no flush)", "parallelism": f"workers sharded x{world}",
-                       "variant": "rtopk_step_apply (fused master update)" if args.apply else "rtopk_step"},
+                       "variant": "rtopk_step_apply (fused master update)" if args.apply else "rtopk_step",
+                       "reuse_threshold": bool(args.reuse_threshold)},
             "elements_per_s": W_total * d / (ms_per_step * 1e-3),
             "step_roofline_frac": step_frac, "step_algorithmic_bytes": step_bytes,
             "phases_ms": phases, "fallback_slices": fallbacks,
+            "predicted_brackets": {"slices": predicted, "of": n_slices * n_prof},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": gpu_launches,
             "clocks": clocks,
         }))

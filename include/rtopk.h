@@ -70,8 +70,13 @@ enum { RTOPK_SCALE_MEAN = 0, RTOPK_SCALE_SUM = 1, RTOPK_SCALE_UNBIASED = 2, RTOP
 enum {
   RTOPK_OPT_SELECT_PATH = 0, /* 0 = automatic (sampled threshold with exact fallback),
                                 1 = always the multi-pass radix select over the full vector */
-  RTOPK_OPT_PROFILE = 1      /* 1 = record CUDA events between the phases of each call on the
+  RTOPK_OPT_PROFILE = 1,     /* 1 = record CUDA events between the phases of each call on the
                                 caller's stream (read with rtopk_get_phase_times); 0 = off */
+  RTOPK_OPT_REUSE_THRESHOLD = 2 /* 1 = consecutive calls of one shape on one residual buffer predict the
+                                first threshold from the exact thresholds of the last calls instead
+                                of sampling (a = g + m drifts slowly from round to round); a
+                                prediction that misses is repaired by the exact path and the next
+                                call samples again.  Results never depend on it.  0 = off (default) */
 };
 
 /* Phases of one call, in stream order.  STREAM is the single pass over the full vectors that
@@ -95,7 +100,8 @@ typedef struct {
   uint32_t n_greater;   /* coordinates with a strictly larger magnitude */
   uint32_t n_candidates;/* coordinates that survived the first threshold */
   uint32_t used_fallback; /* 1 if the sampled threshold missed and the full radix select ran */
-  uint32_t reserved[3];
+  uint32_t bracket_predicted; /* 1 if the first threshold came from the slice's history, not from a sample */
+  uint32_t reserved[2];
 } rtopk_stats;
 
 int rtopk_version(void);

@@ -67,8 +67,13 @@ struct SelState {
   uint32_t flags;
   uint32_t n_cand_first;// candidates of the sampled-threshold pass (statistics)
   uint32_t tau_hi;      // sampled upper estimate of the r-th largest key (0x7FFFFFFF = none)
-  uint32_t pad;
+  uint32_t pred;        // predicted r-th largest key when the bracket came from the history (0: from the sample)
 };
+
+// What a slice remembers from call to call when thresholds are reused: the exact r-th largest keys
+// of the last two calls, a running bound of the relative prediction error, and how many of the two
+// keys may be used (0: the next call samples).
+struct TauHistory { uint32_t tau1, tau2; float err; uint32_t valid; };
 
 struct Scratch {
   Slice* slices;
@@ -91,6 +96,7 @@ struct Scratch {
   uint32_t* sel_pre;      // exclusive popcount prefix per bitmap word
   uint32_t* sel_blk;      // selected positions per chunk of bitmap words (scan scratch)
   uint32_t* error;        // device error flags
+  TauHistory* history;    // [slices] threshold history across calls
 };
 
 struct Launch {
@@ -104,6 +110,7 @@ struct Launch {
   uint32_t seed_lo, seed_hi;
   uint32_t step;
   uint32_t general_primary;   // 1: the full-vector radix select is the main path, not a fallback
+  uint32_t reuse;             // 1: brackets may be predicted from the slices' threshold history
 };
 
 // ----------------------------------------------------------------------------- small helpers

@@ -49,6 +49,10 @@ struct rtopk_ctx {
   size_t sel_blk_entries = 0;
   size_t sel_words = 0;
   uint32_t* d_error = nullptr;
+  TauHistory* d_history = nullptr;   // per-slice threshold history (RTOPK_OPT_REUSE_THRESHOLD)
+  int reuse = 0;
+  bool history_stale = true;         // cleared before the next call that may use it
+  const float* history_residual = nullptr;
   uint32_t* d_agg_starts = nullptr;
   size_t agg_start_entries = 0;
   void* d_stage = nullptr;       // host-call staging: gradient, messages, update
@@ -306,6 +310,7 @@ int upload_slices(rtopk_ctx* ctx, const Plan& P, cudaStream_t st) {
     return RTOPK_OK;
   RTOPK_CUDA(ctx, cudaMemcpyAsync(ctx->d_slices, P.slices.data(), bytes, cudaMemcpyHostToDevice, st));
   ctx->cached_slices = P.slices;
+  ctx->history_stale = true;          // other slices: what was learnt about the old ones does not apply
   return RTOPK_OK;
 }
 
@@ -365,6 +370,18 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   rc = upload_slices(ctx, P, st);
   if (rc) return rc;
   ctx->last_n_slices = L.n_slices;
+  L.s.history = ctx->d_history;
+  L.reuse = (ctx->reuse && ctx->select_path == 0) ? 1u : 0u;
+  if (L.reuse) {
+    // the history follows one residual buffer through consecutive calls of one shape
+    if (ctx->history_stale || ctx->history_residual != residual) {
+      RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_history, 0, P.slices.size() * sizeof(TauHistory), st));
+      ctx->history_stale = false;
+      ctx->history_residual = residual;
+    }
+  } else {
+    ctx->history_stale = true;
+  }
   mark(ctx, RTOPK_PHASE_SUBSET, st);
   // The sampling kernels clear the leading counters of the zeroed region themselves; the exact
   // primary path has no such kernel.  The rest (exact-path histograms and look-back words, the
@@ -562,6 +579,7 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   ctx->sel_blk_entries = slices * ((size_t)r_max / 32 / kSelChunk + 2);
   alloc((void**)&ctx->d_sel_blk, ctx->sel_blk_entries * sizeof(uint32_t));
   alloc((void**)&ctx->d_error, 16);
+  alloc((void**)&ctx->d_history, slices * sizeof(TauHistory));
   alloc((void**)&ctx->d_agg_starts, ctx->agg_start_entries * sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_sample<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSampleSmemBytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_sample<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSampleSmemBytes);
@@ -618,7 +636,7 @@ int rtopk_destroy(rtopk_ctx* ctx) {
   DeviceGuard guard(ctx->device);
   void* ptrs[] = {ctx->d_slices, ctx->d_state, ctx->d_zero, ctx->d_first, ctx->d_cand_idx, ctx->d_cand_val,
                   ctx->d_raw_idx, ctx->d_raw_val, ctx->d_chunk_tab,
-                  ctx->d_draws, ctx->d_sel_pre, ctx->d_sel_blk, ctx->d_error, ctx->d_agg_starts, ctx->d_stage};
+                  ctx->d_draws, ctx->d_sel_pre, ctx->d_sel_blk, ctx->d_error, ctx->d_agg_starts, ctx->d_stage, ctx->d_history};
   for (void* p : ptrs) if (p) cudaFree(p);
   for (cudaEvent_t ev : ctx->ev) if (ev) cudaEventDestroy(ev);
   if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
@@ -631,6 +649,11 @@ int rtopk_destroy(rtopk_ctx* ctx) {
 int rtopk_set_option(rtopk_ctx* ctx, int option, int64_t value) {
   if (!ctx) return RTOPK_ERR_INVALID_ARG;
   if (option == RTOPK_OPT_SELECT_PATH && (value == 0 || value == 1)) { ctx->select_path = (int)value; return RTOPK_OK; }
+  if (option == RTOPK_OPT_REUSE_THRESHOLD && (value == 0 || value == 1)) {
+    ctx->reuse = (int)value;
+    ctx->history_stale = true;
+    return RTOPK_OK;
+  }
   if (option == RTOPK_OPT_PROFILE && (value == 0 || value == 1)) {
     ctx->profile = (int)value;
     for (bool& v : ctx->ev_valid) v = false;
@@ -880,6 +903,7 @@ int rtopk_get_stats(rtopk_ctx* ctx, int32_t slice, rtopk_stats* out, void* strea
   out->n_greater = s.n_gt;
   out->n_candidates = s.n_cand;
   out->used_fallback = (s.flags & FLAG_FELL_BACK) ? 1u : 0u;
+  out->bracket_predicted = s.pred != 0 ? 1u : 0u;
   return RTOPK_OK;
 }
 

@@ -44,7 +44,7 @@ __global__ void k_init_state(Launch L, uint32_t general) {
   st.tau_lo = 0x80000000u;           // above every key: nothing is a candidate
   st.eq_quota = kNoQuota;
   st.prefix = 0; st.n_gt = 0; st.need = S.r; st.n_cand = 0; st.n_cand_first = 0;
-  st.tau_hi = 0x7FFFFFFFu; st.pad = 0;
+  st.tau_hi = 0x7FFFFFFFu; st.pred = 0;
   if (S.r == S.len) { st.resolved = 31; st.stage = STAGE_DONE; st.flags = 0; }   // top-r is everything
   else { st.resolved = 0; st.stage = STAGE_PASS0; st.flags = general ? FLAG_GENERAL : 0u; }
   L.s.state[s] = st;
@@ -154,11 +154,31 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(Launch L) {
   clear_slice_counters(L, sl, S, 0, 1);
   SelState st;
   st.eq_quota = kNoQuota; st.prefix = 0; st.resolved = 0; st.n_gt = 0; st.need = S.r;
-  st.n_cand = 0; st.n_cand_first = 0; st.stage = STAGE_PASS0; st.flags = 0; st.tau_hi = 0x7FFFFFFFu; st.pad = 0;
+  st.n_cand = 0; st.n_cand_first = 0; st.stage = STAGE_PASS0; st.flags = 0; st.tau_hi = 0x7FFFFFFFu; st.pred = 0;
   if (S.r == S.len) {
     st.tau_lo = 0x80000000u; st.resolved = 31; st.stage = STAGE_DONE;
     if (tid == 0) L.s.state[sl] = st;
     return;
+  }
+  if (L.reuse) {
+    // Step-to-step reuse: a = g + m changes slowly from one round to the next, so the last exact
+    // thresholds predict this one (geometric extrapolation of the last two); the bracket is the
+    // prediction widened by a few times the error the predictions have shown so far.  A bracket
+    // that misses is repaired by the exact path and makes the next call sample again.
+    const TauHistory h = L.s.history[sl];                       // the same for every thread
+    if (h.valid >= 1 && h.tau1 > 0x00800000u && h.tau1 < 0x7E800000u) {
+      const float t1 = __uint_as_float(h.tau1);
+      float ratio = 1.0f;
+      if (h.valid >= 2 && h.tau2 > 0x00800000u && h.tau2 < 0x7E800000u)
+        ratio = fminf(fmaxf(t1 / __uint_as_float(h.tau2), 0.5f), 2.0f);
+      const float p = t1 * ratio;
+      const float delta = fminf(fmaxf(3.0f * h.err + 0.01f, 0.02f), 0.15f);
+      st.tau_lo = mag_key(p * (1.0f - delta));
+      st.tau_hi = max(mag_key(p * (1.0f + delta)), st.tau_lo);
+      st.pred = mag_key(p);
+      if (tid == 0) L.s.state[sl] = st;
+      return;
+    }
   }
   const float* m = L.residual;
   uint32_t n_s, rho_lo, rho_hi, n_held;
@@ -874,7 +894,28 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
     return;
   }
   const uint32_t tau = lo_key, quota = need;
-  if (q == 0 && tid == 0) { st->prefix = tau; st->resolved = 31; st->n_gt = n_gt; st->need = need; }
+  if (q == 0 && tid == 0) {
+    st->prefix = tau; st->resolved = 31; st->n_gt = n_gt; st->need = need;
+    if (L.reuse) {
+      TauHistory h = L.s.history[sl];
+      const uint32_t pred = st->pred;
+      if (pred != 0 && (st->flags & FLAG_FELL_BACK)) {        // the predicted bracket missed: sample next time
+        h.err = fminf(fmaxf(2.0f * h.err, 0.05f), 0.2f);
+        h.tau1 = tau; h.tau2 = 0; h.valid = 0;
+      } else {
+        if (pred != 0) {
+          const float rel = fabsf(__uint_as_float(tau) / __uint_as_float(pred) - 1.0f);
+          h.err = rel == rel ? fmaxf(rel, 0.7f * h.err) : 0.2f;
+        } else if (h.valid == 0 && h.err == 0.0f) {
+          h.err = 0.03f;                                         // nothing known yet about this slice
+        }
+        h.tau2 = h.valid >= 1 ? h.tau1 : 0u;
+        h.tau1 = tau;
+        h.valid = min(h.valid + 1u, 2u);
+      }
+      L.s.history[sl] = h;
+    }
+  }
 
   // Members of my share (keys above tau, keys equal to tau), per warp: warp w owns the w-th
   // contiguous part of the share, so that the walk below needs no block-wide barrier.

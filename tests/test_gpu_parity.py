@@ -428,6 +428,44 @@ def test_step_apply_is_sparsify_then_update(lib):
     ctx.close()
 
 
+def test_threshold_reuse_changes_nothing_but_the_path(lib):
+    """RTOPK_OPT_REUSE_THRESHOLD: consecutive rounds predict the first threshold from the last exact
+    ones.  Messages, residual and update stay bit-equal to the oracle; the brackets are predicted
+    from the second round on; an abrupt collapse of the magnitudes is repaired by the exact path and
+    the next round samples again."""
+    from paper_2005_10761_b200.binding import OPT_REUSE_THRESHOLD
+    cfg = wl.scaled(wl.configs()["c2"], d=400_003, W=3)
+    ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
+    ctx.set_option(OPT_REUSE_THRESHOLD, 1)
+    m = wl.zero_residual(cfg, "cuda")
+    m_ref = np.zeros((cfg.W, cfg.ld), dtype=np.float32)
+    idx = torch.zeros((cfg.W, cfg.k), dtype=torch.int32, device="cuda")
+    val = torch.zeros((cfg.W, cfg.k), dtype=torch.float32, device="cuda")
+    out = torch.empty(cfg.ld, dtype=torch.float32, device="cuda")
+    scale = [1.0] * 12 + [None, 1.0, 1.0]
+    predicted, fell = [], []
+    for t, sc in enumerate(scale):
+        g = wl.gradient(cfg, t, "cuda")
+        if sc is None:
+            g = g * 1e-4 - m                    # a = g + m collapses to a thousandth of its size: every prediction misses
+        ctx.step(g, m, cfg.d, cfg.r, cfg.k, cfg.seed, t, idx, val, out)
+        o_idx, o_val = oracle.sparsify(g.cpu().numpy(), m_ref, cfg.d, cfg.r, cfg.k, cfg.seed, t)
+        _, o_out = oracle.aggregate(o_idx, o_val, cfg.d)
+        assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx), t
+        assert np.array_equal(_bits(val.cpu().numpy()), _bits(o_val)), t
+        assert np.array_equal(_bits(m.cpu().numpy()), _bits(m_ref)), t
+        assert np.array_equal(_bits(out.cpu().numpy()[:cfg.d]), _bits(o_out)), t
+        st = [ctx.stats(w) for w in range(cfg.W)]
+        predicted.append(all(s["bracket_predicted"] for s in st))
+        fell.append(any(s["used_fallback"] for s in st))
+    ctx.poll_status()
+    assert not predicted[0] and predicted[1]                  # the first round samples, the second predicts
+    assert sum(predicted[1:12]) >= 8                          # early rounds may miss while the residual builds up
+    assert predicted[10] and predicted[11] and not fell[10] and not fell[11]   # steady state: predictions hold
+    assert predicted[12] and fell[12] and not predicted[13]   # the collapse is missed, repaired, and sampled after
+    ctx.close()
+
+
 def test_step_is_sparsify_then_aggregate(lib):
     cfg = wl.configs()["c1"]
     ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
