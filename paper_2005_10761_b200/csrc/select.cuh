@@ -1,14 +1,18 @@
 // Top-r selection kernels (Definition 1 with the lower-index tie rule), fused with the
 // error-feedback add of Algorithm 1 (a = g + m, written back into the residual buffer).
 //
-//   k_sample        estimates a threshold from a strided sample of a = g + m
-//   k_collect       one streaming pass: a = g + m -> residual, keys above the threshold are appended
-//                   to an index-ordered candidate list (ballot/prefix compaction + look-back)
-//   k_hist          full-vector radix histogram pass (exact path and fallback)
-//   k_finish        one cluster per slice: exact r-th largest key among the candidates, then a walk
-//                   over the candidates in index order that numbers the members of the top-r set and
-//                   writes the ones the k-of-r sampler chose as (index, value) messages, zeroing
-//                   their residual slots (m' = a - ghat)
+//   k_sample        brackets the r-th largest key of every slice from a strided sample of a = g + m
+//                   (or, with threshold reuse, from the slice's last exact thresholds) and clears
+//                   the counters of the streaming pass (k_stream, stream.cuh)
+//   k_exact         the exact path, one cooperative launch: three radix histogram passes over the
+//                   full vector (hist_body) and an index-ordered collect (collect_body, ballot-free
+//                   prefix compaction + bounded look-back); runs only for slices whose bracket
+//                   missed, or as the main path behind k_hist (fused add in pass 0)
+//   k_finish        one cluster per slice: candidate runs -> index order, exact r-th largest key
+//                   among the candidates, then a walk over the candidates in index order that
+//                   numbers the members of the top-r set and writes the ones the k-of-r sampler
+//                   chose as (index, value) messages, zeroing their residual slots (m' = a - ghat)
+//   k_emit_all      r = d (Definition 2): positions are indices, no selection
 #pragma once
 
 #include <cooperative_groups.h>
