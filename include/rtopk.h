@@ -156,6 +156,16 @@ int rtopk_aggregate_unbiased(rtopk_ctx* ctx, const uint32_t* msg_idx, const floa
                              int32_t W, int64_t k, int64_t r, float* out, void* stream);
 
 /*
+ * Sizes for round `step` under the schedule of Section IV: the sparsity grows exponentially over
+ * the warm-up period and k / r = 1 / n throughout.  Host only, no GPU work.
+ *   density(step) = initial * (final / initial)^(step / warmup_steps) for step < warmup_steps,
+ *                   final afterwards;   k = clamp(floor(density * d), 1, d);   r = min(d, n * k).
+ *   0 < final_density <= initial_density <= 1.   *r, *k [out] host.   Errors: INVALID_ARG.
+ */
+int rtopk_warmup_sizes(int64_t d, int32_t n_workers, double initial_density, double final_density,
+                       int64_t warmup_steps, int64_t step, int64_t* r, int64_t* k);
+
+/*
  * Packed message format.  Section III counts log d bits per index and a constant number of bits per
  * value; this format spends exactly b = ceil(log2 d) bits (at least 1) per index and 16 per value:
  *   packed_idx  W rows of ld_words 32-bit words: entry j of a row occupies bits [j b, (j + 1) b) of

@@ -67,6 +67,8 @@ def lib() -> C.CDLL:
                                               C.c_int64, f64p, f32p]
         L.oracle_apply_update.argtypes = [u32p, f32p, C.c_int64, C.c_int32, C.c_int64, C.c_int,
                                           C.c_int64, C.c_float, f32p]
+        L.oracle_warmup_sizes.argtypes = [C.c_int64, C.c_int32, C.c_double, C.c_double, C.c_int64, C.c_int64,
+                                          i64p, i64p]
         u16p = C.POINTER(C.c_uint16)
         L.oracle_index_bits.argtypes = [C.c_int64]
         L.oracle_bf16_rne.argtypes = [C.c_float]
@@ -198,6 +200,12 @@ def apply_update(msg_idx: np.ndarray, msg_val: np.ndarray, d: int, eta: float, w
     _check(lib().oracle_apply_update(_p(idx, C.c_uint32), _p(val, C.c_float), d, W, k, scale_mode, r,
                                      C.c_float(eta), _p(w, C.c_float)), "apply_update")
     return w
+
+
+def warmup_sizes(d: int, n: int, initial: float, final: float, warmup_steps: int, step: int):
+    r, k = C.c_int64(0), C.c_int64(0)
+    _check(lib().oracle_warmup_sizes(d, n, initial, final, warmup_steps, step, C.byref(r), C.byref(k)), "warmup_sizes")
+    return int(r.value), int(k.value)
 
 
 def index_bits(d: int) -> int:

@@ -324,6 +324,22 @@ int oracle_apply_update(const uint32_t* msg_idx, const float* msg_val, int64_t d
   return ORACLE_OK;
 }
 
+// ----------------------------------------------------------------------------- warm-up schedule
+// Section IV: sparsity is increased exponentially during the warm-up period, and k / r = 1 / n.
+// density(t) = initial * (final / initial)^(t / T) for t < T, final afterwards;
+// k = clamp(floor(density d), 1, d), r = min(d, n k).
+int oracle_warmup_sizes(int64_t d, int32_t n, double initial, double final_, int64_t T, int64_t t, int64_t* r,
+                        int64_t* k) {
+  if (d < 1 || n < 1 || t < 0 || T < 0 || !r || !k || !(final_ > 0.0) || !(initial >= final_) || !(initial <= 1.0))
+    return ORACLE_BAD_ARG;
+  const double density = t < T ? initial * std::exp(std::log(final_ / initial) * ((double)t / (double)T)) : final_;
+  int64_t kk = (int64_t)(density * (double)d);
+  kk = std::max<int64_t>(1, std::min<int64_t>(d, kk));
+  *k = kk;
+  *r = (int64_t)std::min<double>((double)d, (double)kk * (double)n);
+  return ORACLE_OK;
+}
+
 // ----------------------------------------------------------------------------- message codec
 // Section III notes that an index costs log d bits and a value a constant number of bits.  The
 // library's packed message format states one such encoding:

@@ -34,6 +34,7 @@ EXPORTS = {
     "rtopk_step": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _i64, _u64, _u32, _int,
                           _vp, _vp, _vp, _vp]),
     "rtopk_aggregate_unbiased": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _i64, _vp, _vp]),
+    "rtopk_warmup_sizes": (_int, [_i64, _i32, C.c_double, C.c_double, _i64, _i64, C.POINTER(_i64), C.POINTER(_i64)]),
     "rtopk_packed_layout": (_int, [_i64, _i64, C.POINTER(_i32), C.POINTER(_i64), C.POINTER(_i64)]),
     "rtopk_encode": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _vp]),
     "rtopk_aggregate_packed": (_int, [_vp, _vp, _i64, _vp, _i64, _i64, _i32, _i64, _int, _vp, _vp]),
@@ -63,6 +64,17 @@ class RTopKError(RuntimeError):
     def __init__(self, status: int, what: str, detail: str = ""):
         self.status = status
         super().__init__(f"{what}: status {status} ({detail})")
+
+
+def warmup_sizes(d: int, n_workers: int, initial_density: float, final_density: float, warmup_steps: int,
+                 step: int):
+    """(r, k) of round `step` under the exponential warm-up schedule with k / r = 1 / n."""
+    r, k = _i64(0), _i64(0)
+    rc = load_library().rtopk_warmup_sizes(d, n_workers, initial_density, final_density, warmup_steps, step,
+                                           C.byref(r), C.byref(k))
+    if rc != 0:
+        raise RTopKError(rc, "rtopk_warmup_sizes", "invalid argument")
+    return int(r.value), int(k.value)
 
 
 def packed_layout(d: int, k: int):

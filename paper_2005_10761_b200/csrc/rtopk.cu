@@ -688,6 +688,22 @@ int rtopk_aggregate_unbiased(rtopk_ctx* ctx, const uint32_t* msg_idx, const floa
   return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, RTOPK_SCALE_UNBIASED, out, (cudaStream_t)stream, false, -1.0f, r);
 }
 
+int rtopk_warmup_sizes(int64_t d, int32_t n_workers, double initial_density, double final_density,
+                       int64_t warmup_steps, int64_t step, int64_t* r, int64_t* k) {
+  if (d < 1 || n_workers < 1 || step < 0 || warmup_steps < 0 || !r || !k) return RTOPK_ERR_INVALID_ARG;
+  if (!(final_density > 0.0) || !(initial_density >= final_density) || !(initial_density <= 1.0))
+    return RTOPK_ERR_INVALID_ARG;
+  double density = final_density;
+  if (step < warmup_steps)
+    density = initial_density * std::pow(final_density / initial_density, (double)step / (double)warmup_steps);
+  int64_t kk = (int64_t)std::floor(density * (double)d);
+  if (kk < 1) kk = 1;
+  if (kk > d) kk = d;
+  *k = kk;
+  *r = kk > d / n_workers ? d : kk * (int64_t)n_workers;        // k / r = 1 / n, capped at d
+  return RTOPK_OK;
+}
+
 int rtopk_packed_layout(int64_t d, int64_t k, int32_t* index_bits, int64_t* ld_words, int64_t* ld_halves) {
   return packed_layout(d, k, index_bits, ld_words, ld_halves);
 }

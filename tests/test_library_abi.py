@@ -54,3 +54,21 @@ def test_product_package_does_not_import_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 src = open(os.path.join(dirpath, f)).read()
                 assert "import oracle" not in src and "from oracle" not in src and "oracle/" not in src, f
+
+
+def test_warmup_sizes_host_function_matches_the_oracle():
+    """rtopk_warmup_sizes is host-only arithmetic: callable without a GPU.  exp/log in the oracle and
+    pow in the library may differ in the last bit, so k may differ by one where density * d is
+    within rounding of an integer; the exact-power cases agree exactly."""
+    import oracle
+    import paper_2005_10761_b200 as rt
+    d, n = 1 << 20, 8
+    for t in range(7):
+        assert rt.warmup_sizes(d, n, 0.25, 1.0 / 1024, 4, t) == oracle.warmup_sizes(d, n, 0.25, 1.0 / 1024, 4, t)
+    for t in range(0, 70, 3):
+        r1, k1 = rt.warmup_sizes(11_173_962, 5, 0.3, 0.001, 50, t)
+        r2, k2 = oracle.warmup_sizes(11_173_962, 5, 0.3, 0.001, 50, t)
+        assert abs(k1 - k2) <= 1 and r1 == min(11_173_962, 5 * k1)
+    import pytest
+    with pytest.raises(rt.RTopKError):
+        rt.warmup_sizes(100, 4, 0.001, 0.01, 5, 0)

@@ -543,3 +543,26 @@ def test_codec_rounding_error_goes_to_the_residual():
     untouched = np.ones(d, dtype=bool); untouched[sent] = False
     assert np.array_equal(m[0, untouched].view(np.uint32), m0[0, untouched].view(np.uint32))
     assert np.all(np.abs(m[0, sent][ok]) <= np.abs(val[0][ok]) * 2.0**-8)
+
+
+# ----------------------------------------------------------------------------- warm-up schedule
+def test_warmup_schedule_geometric_sequence_and_limits():
+    # Section IV: sparsity grows exponentially over the warm-up, k / r = 1 / n.  With density going
+    # from 1/4 to 1/1024 in 4 steps every step divides the density by 4 (exact powers of two).
+    d, n = 1 << 20, 8
+    ks = [oracle.warmup_sizes(d, n, 0.25, 1.0 / 1024, 4, t)[1] for t in range(7)]
+    assert ks == [d // 4, d // 16, d // 64, d // 256, d // 1024, d // 1024, d // 1024]
+    for t in range(7):
+        r, k = oracle.warmup_sizes(d, n, 0.25, 1.0 / 1024, 4, t)
+        assert r == min(d, n * k) and 1 <= k <= r <= d
+    # monotone, ends at floor(final d), never below one coordinate, r capped at d
+    seq = [oracle.warmup_sizes(11_173_962, 5, 0.3, 0.001, 50, t) for t in range(60)]
+    assert all(a[1] >= b[1] for a, b in zip(seq, seq[1:])) and seq[50][1] == 11_173
+    assert seq[0] == (11_173_962, int(0.3 * 11_173_962))
+    assert oracle.warmup_sizes(100, 4, 0.001, 0.001, 0, 3) == (4, 1)
+    # against numpy's power on a grid (floor may differ by one where density * d is an integer)
+    for t in range(0, 50, 7):
+        want = int(np.floor(0.3 * np.power(0.001 / 0.3, t / 50) * 11_173_962))
+        assert abs(seq[t][1] - want) <= 1
+    with pytest.raises(ValueError):
+        oracle.warmup_sizes(100, 4, 0.001, 0.01, 5, 0)
