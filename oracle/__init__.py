@@ -75,6 +75,11 @@ def lib() -> C.CDLL:
         L.oracle_bf16_rne.restype = C.c_uint16
         L.oracle_encode_row.argtypes = [u32p, f32p, C.c_int64, C.c_int64, u32p, u16p, f32p]
         L.oracle_decode_row.argtypes = [u32p, u16p, C.c_int64, C.c_int64, u32p, f32p]
+        L.oracle_sparsify_threshold.argtypes = [C.c_void_p, C.c_int, C.c_int64, f32p, C.c_int64, C.c_int64,
+                                                C.c_int32, C.c_int32, C.c_float, C.c_int64, C.c_uint64,
+                                                C.c_uint32, u32p, f32p, u32p, u32p]
+        L.oracle_aggregate_threshold.argtypes = [u32p, f32p, u32p, u32p, C.c_int64, C.c_int32, C.c_int64,
+                                                 f64p, f32p]
         _lib = L
     return _lib
 
@@ -250,3 +255,37 @@ def decode(packed_idx: np.ndarray, packed_val: np.ndarray, d: int, k: int):
 
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv))
+
+
+def sparsify_threshold(grad: np.ndarray, residual: np.ndarray, d: int, theta: float, k: int, seed: int,
+                       step: int, worker_base: int = 0):
+    """Threshold-then-subsample encoder (proof of Theorem 1) on W rows; ``residual`` is updated in place.
+    Returns (msg_idx [W,k] uint32, msg_val [W,k] float32, count [W] uint32, ones [W] uint32)."""
+    dt = _grad_args(grad)
+    assert residual.dtype == np.float32 and residual.ndim == 2 and residual.flags.c_contiguous
+    W = grad.shape[0]
+    assert residual.shape[0] == W
+    idx = np.zeros((W, k), dtype=np.uint32)
+    val = np.zeros((W, k), dtype=np.float32)
+    count = np.zeros(W, dtype=np.uint32)
+    ones = np.zeros(W, dtype=np.uint32)
+    _check(lib().oracle_sparsify_threshold(grad.ctypes.data, dt, grad.shape[1], _p(residual, C.c_float),
+                                           residual.shape[1], d, W, worker_base, theta, k, seed, step,
+                                           _p(idx, C.c_uint32), _p(val, C.c_float), _p(count, C.c_uint32),
+                                           _p(ones, C.c_uint32)), "sparsify_threshold")
+    return idx, val, count, ones
+
+
+def aggregate_threshold(msg_idx: np.ndarray, msg_val: np.ndarray, count: np.ndarray, ones: np.ndarray, d: int):
+    """Estimator of the proof of Theorem 1: (1/n) sum_w kept_w / S_w.  Returns (out64, out32)."""
+    idx = np.ascontiguousarray(msg_idx, dtype=np.uint32)
+    val = np.ascontiguousarray(msg_val, dtype=np.float32)
+    cnt = np.ascontiguousarray(count, dtype=np.uint32)
+    one = np.ascontiguousarray(ones, dtype=np.uint32)
+    W, k = idx.shape
+    o64 = np.zeros(d, dtype=np.float64)
+    o32 = np.zeros(d, dtype=np.float32)
+    _check(lib().oracle_aggregate_threshold(_p(idx, C.c_uint32), _p(val, C.c_float), _p(cnt, C.c_uint32),
+                                            _p(one, C.c_uint32), d, W, k, _p(o64, C.c_double),
+                                            _p(o32, C.c_float)), "aggregate_threshold")
+    return o64, o32

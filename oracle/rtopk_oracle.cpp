@@ -35,7 +35,10 @@
 // draw scaling against big-integer arithmetic; Floyd against exhaustive
 // enumeration (every k-subset equally often); top-r against brute force and
 // library sorts; the whole operator against the closed form in the proof of
-// Proposition 1 and the limits k = r (Def. 1) and r = d (Def. 2).
+// Proposition 1 and the limits k = r (Def. 1) and r = d (Def. 2); the
+// threshold-then-subsample encoder (proof of Theorem 1) against a library
+// comparison of magnitudes, exhaustive enumeration of the kept subsets, the
+// exact unbiasedness of its estimator and the identity sum(X~ / S) = ||X||_1.
 
 #include <algorithm>
 #include <cmath>
@@ -407,6 +410,98 @@ int oracle_decode_row(const uint32_t* packed_idx, const uint16_t* packed_val, in
     idx[j] = v;
     const uint32_t wide = (uint32_t)packed_val[j] << 16;
     std::memcpy(&val[j], &wide, 4);
+  }
+  return ORACLE_OK;
+}
+
+// ----------------------------------------------------------------------------- threshold, then subsample
+// The scheme in the proof of Theorem 1, applied to real-valued vectors as Section II describes for
+// continuous observations (quantise by magnitude at a threshold first, then subsample):
+//   * X_w marks the coordinates of a = g + m whose magnitude exceeds theta ("1"), the rest are "0";
+//     ones_w = ||X_w||_1 travels with the message;
+//   * if ones_w > k, k of those coordinates are kept uniformly at random (the same Floyd / Philox
+//     subset as Definition 3, over the marked coordinates numbered by ascending index), otherwise
+//     all of them; count_w = min(ones_w, k) entries are sent, the subsampling fraction is
+//     S_w = count_w / ones_w;
+//   * the estimator is (1/n) sum_w Xtilde_w / S_w.
+// Readings: a kept coordinate carries its value a_i (as in Definition 3), "exceeds" is the strict
+// comparison of the magnitude bit patterns (so a NaN counts as marked), the node keeps m' = a - ghat
+// as in Algorithm 1, unused message slots hold index 0xFFFFFFFF and value +0, and one term of the
+// estimator is double(value) * (double(ones_w) / double(count_w)), summed in worker order and
+// divided by n once.
+int oracle_sparsify_threshold(const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
+                              int64_t d, int32_t W, int32_t worker_base, float theta, int64_t k, uint64_t seed,
+                              uint32_t step, uint32_t* msg_idx, float* msg_val, uint32_t* msg_count,
+                              uint32_t* msg_ones) {
+  if (!grad || !residual || !msg_idx || !msg_val || !msg_count || !msg_ones) return ORACLE_BAD_ARG;
+  if (d < 1 || d > 0x7FFFFFFF || W < 1 || k < 1 || k > d || ld_g < d || ld_m < d) return ORACLE_BAD_ARG;
+  if (grad_dtype != GRAD_F32 && grad_dtype != GRAD_BF16) return ORACLE_BAD_ARG;
+  if (!(theta >= 0.0f) || std::isinf(theta)) return ORACLE_BAD_ARG;
+  const size_t gsz = grad_dtype == GRAD_F32 ? 4 : 2;
+  const uint32_t theta_key = magnitude_key(theta);
+  for_each_row(W, [&](int w) {
+    const char* g = (const char*)grad + (size_t)w * (size_t)ld_g * gsz;
+    float* a = residual + (size_t)w * (size_t)ld_m;
+    uint32_t* out_idx = msg_idx + (size_t)w * (size_t)k;
+    float* out_val = msg_val + (size_t)w * (size_t)k;
+    // a = g + m
+    for (int64_t i = 0; i < d; ++i) {
+      float s = widen_grad(g, grad_dtype, i) + a[i];
+      if (s != s) s = bits_float(0x7FC00000u);
+      a[i] = s;
+    }
+    // X: the marked coordinates, ascending
+    std::vector<uint32_t> marked;
+    for (int64_t i = 0; i < d; ++i)
+      if (magnitude_key(a[i]) > theta_key) marked.push_back((uint32_t)i);
+    const int64_t ones = (int64_t)marked.size();
+    // Xtilde: all of them, or k drawn uniformly
+    std::vector<uint32_t> kept;
+    if (ones > k) {
+      std::vector<uint32_t> pos((size_t)k);
+      sample_positions(ones, k, seed, step, (uint32_t)(worker_base + w), 0u, pos.data());
+      for (int64_t q = 0; q < k; ++q) kept.push_back(marked[pos[(size_t)q]]);
+    } else {
+      kept = marked;
+    }
+    msg_ones[w] = (uint32_t)ones;
+    msg_count[w] = (uint32_t)kept.size();
+    for (int64_t q = 0; q < k; ++q) {
+      if (q < (int64_t)kept.size()) {
+        const uint32_t i = kept[(size_t)q];
+        out_idx[q] = i;
+        out_val[q] = a[i];
+        a[i] = 0.0f;                                    // m' = a - ghat
+      } else {
+        out_idx[q] = 0xFFFFFFFFu;
+        out_val[q] = 0.0f;
+      }
+    }
+  });
+  return ORACLE_OK;
+}
+
+// The estimator of the same proof: out_i = (1/n) sum_w [i kept by w] value_{w,i} / S_w.
+int oracle_aggregate_threshold(const uint32_t* msg_idx, const float* msg_val, const uint32_t* msg_count,
+                               const uint32_t* msg_ones, int64_t d, int32_t W, int64_t k, double* out64,
+                               float* out32) {
+  if (!msg_idx || !msg_val || !msg_count || !msg_ones || d < 1 || W < 1 || k < 1) return ORACLE_BAD_ARG;
+  std::vector<double> acc((size_t)d, 0.0);
+  for (int32_t w = 0; w < W; ++w) {
+    const int64_t count = msg_count[w], ones = msg_ones[w];
+    if (count > k || count > ones || (ones > k && count != k)) return ORACLE_BAD_ARG;
+    if (count == 0) continue;
+    const double inv_S = (double)ones / (double)count;
+    for (int64_t q = 0; q < count; ++q) {
+      const uint32_t i = msg_idx[(size_t)w * (size_t)k + (size_t)q];
+      if ((int64_t)i >= d) return ORACLE_BAD_ARG;
+      acc[i] += (double)msg_val[(size_t)w * (size_t)k + (size_t)q] * inv_S;
+    }
+  }
+  for (int64_t i = 0; i < d; ++i) {
+    const double v = acc[(size_t)i] / (double)W;
+    if (out64) out64[i] = v;
+    if (out32) out32[i] = (float)v;
   }
   return ORACLE_OK;
 }
