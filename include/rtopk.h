@@ -241,6 +241,48 @@ int rtopk_step_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64
                          uint32_t* msg_idx, float* msg_val, float* out, void* stream);
 
 /*
+ * Threshold-then-subsample encoder: the scheme in the proof of Theorem 1 (Section V), applied to
+ * real-valued vectors the way Section II describes it for continuous observations: a coordinate of
+ * a = g + m is marked ("1") when its magnitude exceeds theta, ||X_w||_1 = ones_w of worker w's
+ * coordinates are; if ones_w > k, k of them are kept uniformly at random (Floyd / Philox as in
+ * rtopk_sparsify, over the marked coordinates listed by ascending index, segment 0), otherwise all.
+ * The message carries ones_w, count_w = min(ones_w, k) and the kept (index, value = a_i) pairs,
+ * ascending; the node keeps m' = a - ghat (Algorithm 1).  "Exceeds" compares the magnitude bit
+ * patterns strictly, so a NaN sum counts as marked.
+ *   theta               finite, >= 0.
+ *   k                   message capacity (the proof's k'), 1 <= k <= min(d, the context's k_max).
+ *   msg_idx, msg_val [out]  W x k; row w: count_w pairs, then padding (index 0xFFFFFFFF, value +0.0f).
+ *   msg_count, msg_ones [out]  W 32-bit words each (device).
+ * The scratch holds at most min(d, the context's r_max) marked coordinates per worker.  A worker
+ * that marks more sends nothing in this call (count_w = 0, ones_w still reported, all of a stays in
+ * its residual) and rtopk_poll_status reports RTOPK_ERR_INTERNAL: raise theta or create the context
+ * with a larger r_max.
+ * Errors: INVALID_ARG, UNSUPPORTED (RTOPK_OPT_SELECT_PATH = 1), CUDA.
+ */
+int rtopk_sparsify_threshold(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,
+                             int64_t ld_m, int64_t d, int32_t W, int32_t worker_base, float theta, int64_t k,
+                             uint64_t seed, uint32_t step, uint32_t* msg_idx, float* msg_val, uint32_t* msg_count,
+                             uint32_t* msg_ones, void* stream);
+
+/*
+ * The estimator of the same proof: out_i = (1/W) sum_w [i kept by w] val_{w,i} / S_w with the
+ * subsampling fraction S_w = count_w / ones_w.  One term is double(val) * (double(ones_w) /
+ * double(count_w)); terms are summed in double in worker order, divided by W and rounded once.
+ *   msg_* [in] as rtopk_sparsify_threshold writes them (rows of several GPUs may be concatenated);
+ *   out [out] d binary32, fully overwritten.
+ * Errors: INVALID_ARG, CUDA.
+ */
+int rtopk_aggregate_threshold(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val,
+                              const uint32_t* msg_count, const uint32_t* msg_ones, int64_t d, int32_t W, int64_t k,
+                              float* out, void* stream);
+
+/* rtopk_sparsify_threshold followed by rtopk_aggregate_threshold of the messages it produced. */
+int rtopk_step_threshold(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,
+                         int64_t ld_m, int64_t d, int32_t W, int32_t worker_base, float theta, int64_t k,
+                         uint64_t seed, uint32_t step, uint32_t* msg_idx, float* msg_val, uint32_t* msg_count,
+                         uint32_t* msg_ones, float* out, void* stream);
+
+/*
  * rtopk_step with HOST gradient and HOST results: copies h_grad (W x ld_g, ideally pinned) to a
  * device staging buffer owned by the context (allocated on first use), runs the step against the
  * DEVICE residual, and copies the messages and the dense update back to h_msg_idx, h_msg_val

@@ -49,6 +49,11 @@ EXPORTS = {
                                     _vp, _vp, _vp, _vp]),
     "rtopk_step_host": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _i64, _u64, _u32,
                                _int, _vp, _vp, _vp, _vp]),
+    "rtopk_sparsify_threshold": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, C.c_float, _i64, _u64, _u32,
+                                        _vp, _vp, _vp, _vp, _vp]),
+    "rtopk_aggregate_threshold": (_int, [_vp, _vp, _vp, _vp, _vp, _i64, _i32, _i64, _vp, _vp]),
+    "rtopk_step_threshold": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, C.c_float, _i64, _u64, _u32,
+                                    _vp, _vp, _vp, _vp, _vp, _vp]),
     "rtopk_sample_positions": (_int, [_vp, _i64, _i64, _u64, _u32, _u32, _u32, _vp, _vp]),
     "rtopk_sample_positions_static": (_int, [_i64, _i64, _u64, _u32, _u32, _u32, _vp, _vp]),
     "rtopk_poll_status": (_int, [_vp, _vp]),
@@ -265,6 +270,32 @@ class RTopK:
                                        step, scale_mode, h_msg_idx.data_ptr(), h_msg_val.data_ptr(),
                                        h_out.data_ptr(), _stream())
         self._check(rc, "rtopk_step_host")
+
+    def sparsify_threshold(self, grad, residual, d, theta, k, seed, step, msg_idx, msg_val, msg_count, msg_ones,
+                           worker_base=0) -> None:
+        """Threshold-then-subsample encoder: msg_count / msg_ones are int32 [W] device tensors."""
+        W = grad.shape[0]
+        rc = self._lib.rtopk_sparsify_threshold(self._h, grad.data_ptr(), self._grad_dtype(grad), grad.stride(0),
+                                                residual.data_ptr(), residual.stride(0), d, W, worker_base, theta, k,
+                                                seed, step, msg_idx.data_ptr(), msg_val.data_ptr(),
+                                                msg_count.data_ptr(), msg_ones.data_ptr(), _stream())
+        self._check(rc, "rtopk_sparsify_threshold")
+
+    def aggregate_threshold(self, msg_idx, msg_val, msg_count, msg_ones, d, out) -> None:
+        W, k = msg_idx.shape
+        rc = self._lib.rtopk_aggregate_threshold(self._h, msg_idx.data_ptr(), msg_val.data_ptr(),
+                                                 msg_count.data_ptr(), msg_ones.data_ptr(), d, W, k, out.data_ptr(),
+                                                 _stream())
+        self._check(rc, "rtopk_aggregate_threshold")
+
+    def step_threshold(self, grad, residual, d, theta, k, seed, step, msg_idx, msg_val, msg_count, msg_ones, out,
+                       worker_base=0) -> None:
+        W = grad.shape[0]
+        rc = self._lib.rtopk_step_threshold(self._h, grad.data_ptr(), self._grad_dtype(grad), grad.stride(0),
+                                            residual.data_ptr(), residual.stride(0), d, W, worker_base, theta, k,
+                                            seed, step, msg_idx.data_ptr(), msg_val.data_ptr(),
+                                            msg_count.data_ptr(), msg_ones.data_ptr(), out.data_ptr(), _stream())
+        self._check(rc, "rtopk_step_threshold")
 
     def sample_positions(self, r, k, seed, step, worker, segment, pos) -> None:
         rc = self._lib.rtopk_sample_positions(self._h, r, k, seed, step, worker, segment, pos.data_ptr(),

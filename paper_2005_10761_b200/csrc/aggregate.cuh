@@ -49,6 +49,10 @@ struct PlainMsgs {
   uint32_t K;
   __device__ __forceinline__ uint32_t index(uint32_t w, uint32_t j) const { return __ldg(idx + (size_t)w * K + j); }
   __device__ __forceinline__ float value(uint32_t w, uint32_t j) const { return __ldg(val + (size_t)w * K + j); }
+  // what worker w's value v adds to a coordinate's double-precision sum
+  static constexpr bool kPerWorker = false;   // the term does not depend on the worker
+  static constexpr bool kPadded = false;      // every row holds K valid entries
+  __device__ __forceinline__ double term(uint32_t, float v) const { return (double)v; }
 };
 struct PackedMsgs {
   const uint32_t* words;
@@ -64,6 +68,27 @@ struct PackedMsgs {
   }
   __device__ __forceinline__ float value(uint32_t w, uint32_t j) const {
     return __uint_as_float((uint32_t)__ldg(halves + (size_t)w * ld_halves + j) << 16);
+  }
+  static constexpr bool kPerWorker = false;
+  static constexpr bool kPadded = false;
+  __device__ __forceinline__ double term(uint32_t, float v) const { return (double)v; }
+};
+// Messages of the threshold-then-subsample encoder (proof of Theorem 1): row w holds count[w] valid
+// entries followed by padding (index 0xFFFFFFFF, which lies beyond every coordinate and keeps the row
+// ascending), and a value enters the estimator divided by the worker's subsampling fraction
+// S_w = count[w] / ones[w]: one division and one multiplication in double, each rounded to nearest.
+struct ThresholdMsgs {
+  const uint32_t* idx;
+  const float* val;
+  uint32_t K;
+  const uint32_t* count;
+  const uint32_t* ones;
+  __device__ __forceinline__ uint32_t index(uint32_t w, uint32_t j) const { return __ldg(idx + (size_t)w * K + j); }
+  __device__ __forceinline__ float value(uint32_t w, uint32_t j) const { return __ldg(val + (size_t)w * K + j); }
+  static constexpr bool kPerWorker = true;
+  static constexpr bool kPadded = true;
+  __device__ __forceinline__ double term(uint32_t w, float v) const {
+    return __dmul_rn((double)v, __ddiv_rn((double)__ldg(ones + w), (double)__ldg(count + w)));
   }
 };
 
@@ -106,7 +131,9 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_starts(M msgs, uint32_t W, 
   const uint32_t t = blockIdx.x * kAggThreads + threadIdx.x;
   const uint32_t w = blockIdx.y;
   if (t > ntiles || w >= W) return;
-  starts[(size_t)w * (ntiles + 1) + t] = t == ntiles ? K : lower_bound_row(msgs, w, K, t * tile_size);
+  // padded rows end their last run at the first padding entry (padding indices exceed every tile bound)
+  const uint32_t bound = t == ntiles ? 0xFFFFFFFFu : t * tile_size;
+  starts[(size_t)w * (ntiles + 1) + t] = (t == ntiles && !M::kPadded) ? K : lower_bound_row(msgs, w, K, bound);
 }
 
 template <typename M, bool COUNT>   // COUNT: also keep the number of senders per coordinate (smaller stage to make room)
@@ -160,7 +187,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(M msgs, const uint32_
         if (e > b) {                                   // block-uniform
           for (uint32_t q = b + tid; q < e; q += kAggThreads) {
             const uint32_t i = st_idx[q] - lo;        // the unsigned check keeps a malformed row inside the tile
-            if (i < (uint32_t)kAggTile) { acc[i] += (double)st_val[q]; if (COUNT) ++senders[i]; }
+            if (i < (uint32_t)kAggTile) { acc[i] += msgs.term(w0 + w, st_val[q]); if (COUNT) ++senders[i]; }
           }
           __syncthreads();
         }
@@ -170,7 +197,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(M msgs, const uint32_
         const uint32_t b = s_beg[w], n = s_pre[w + 1] - s_pre[w];
         for (uint32_t q = tid; q < n; q += kAggThreads) {
           const uint32_t i = msgs.index(w0 + w, b + q) - lo;
-          if (i < (uint32_t)kAggTile) { acc[i] += (double)msgs.value(w0 + w, b + q); if (COUNT) ++senders[i]; }
+          if (i < (uint32_t)kAggTile) { acc[i] += msgs.term(w0 + w, msgs.value(w0 + w, b + q)); if (COUNT) ++senders[i]; }
         }
         __syncthreads();
       }
@@ -296,7 +323,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
       const uint32_t idx = st_idx[q], local = idx - lo;
       if (local >= (uint32_t)kAggSparseTile || idx >= d) continue;    // malformed row: ignore
       if (!((s_shared[local >> 5] >> (local & 31u)) & 1u)) {    // sole sender: the sum is the value
-        const double v = (double)st_val[q];
+        const double v = msgs.term(M::kPerWorker ? worker_of(q) : 0u, st_val[q]);
         out[idx] = agg_result((float)agg_scaled(v, 1u, sc), eta >= 0.0f ? out[idx] : 0.0f, eta);
         continue;
       }
@@ -308,13 +335,13 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     uint32_t senders = 0;
     bool owner = true;
     for (uint32_t x = 0; x < W; ++x) {
-      if (x == w) { sum += (double)val_at(w, q - s_pre[w]); ++senders; continue; }
+      if (x == w) { sum += msgs.term(w, val_at(w, q - s_pre[w])); ++senders; continue; }
       const uint32_t n = s_pre[x + 1] - s_pre[x];
       uint32_t a = 0, b = n;
       while (a < b) { const uint32_t mid = (a + b) >> 1; if (idx_at(x, mid) < idx) a = mid + 1; else b = mid; }
       if (a < n && idx_at(x, a) == idx) {
         if (x < w) { owner = false; break; }          // a lower worker owns this coordinate
-        sum += (double)val_at(x, a);
+        sum += msgs.term(x, val_at(x, a));
         ++senders;
       }
     }

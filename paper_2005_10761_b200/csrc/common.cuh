@@ -86,6 +86,7 @@ struct Scratch {
   uint32_t* group_total;  // candidates per chunk group (summed by the stream pass)
   uint32_t* chunk_start;  // [chunks] where a chunk's run sits in the raw buffer ...
   uint32_t* chunk_count;  // ... its length ...
+  uint32_t* chunk_pre;    // ... and (threshold encoder) how many marked coordinates precede it in the slice
   uint32_t* raw_idx;      // candidates in reservation order
   float* raw_val;
   uint32_t* cand_idx;     // candidates in index order

@@ -20,6 +20,7 @@
 #include "sampler.cuh"
 #include "select.cuh"
 #include "stream.cuh"
+#include "threshold.cuh"
 
 using namespace rtopk;
 
@@ -40,7 +41,7 @@ struct rtopk_ctx {
   float* d_cand_val = nullptr;
   uint32_t* d_raw_idx = nullptr;
   float* d_raw_val = nullptr;
-  uint32_t* d_chunk_tab = nullptr;   // chunk_start | chunk_count
+  uint32_t* d_chunk_tab = nullptr;   // chunk_start | chunk_count | chunk_pre
   size_t chunk_tab_entries = 0;
   size_t cand_entries = 0;
   uint32_t* d_draws = nullptr;
@@ -69,6 +70,7 @@ struct rtopk_ctx {
   // side stream next to the streaming pass
   cudaStream_t side = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  cudaEvent_t ev_streamed = nullptr, ev_cleared = nullptr;   // the dense update is cleared beside the finishing kernels
   int profile = 0;
   cudaEvent_t ev[RTOPK_N_PHASES + 1] = {};
   bool ev_valid[RTOPK_N_PHASES + 1] = {};
@@ -133,8 +135,11 @@ struct Plan {
   uint32_t K_row = 0;
 };
 
+// `always_gather`: every slice gets a candidate list, also when r equals its length (the threshold
+// encoder's r is only an upper bound of the marked set).
 int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32_t W, int32_t S,
-              const int64_t* seg_off, const int64_t* seg_r, const int64_t* seg_k, Plan& P) {
+              const int64_t* seg_off, const int64_t* seg_r, const int64_t* seg_k, Plan& P,
+              bool always_gather = false) {
   uint64_t K = 0, R = 0;
   for (int s = 0; s < S; ++s) {
     const int64_t len = seg_off[s + 1] - seg_off[s];
@@ -179,7 +184,7 @@ int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32
       sl.group_begin = (uint32_t)groups;
       groups += (nchunks + (1u << sl.gshift) - 1) >> sl.gshift;
       sl.cand_off = (uint32_t)cand;
-      if (sl.r < sl.len) {
+      if (sl.r < sl.len || always_gather) {
         sl.cand_cap = cand_capacity(sl.len, sl.r);
         cand += sl.cand_cap;
         if (sl.cand_cap > P.cap_max) P.cap_max = sl.cand_cap;
@@ -262,7 +267,8 @@ int launch_exact(rtopk_ctx* ctx, const Plan& P, const Launch& L, int first_pass,
 }
 
 template <typename GradT>
-int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st, cudaEvent_t join) {
+int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st, cudaEvent_t join,
+                  float* clear_out, size_t clear_bytes) {
   const uint32_t n = (uint32_t)P.slices.size();
   int rc = RTOPK_OK;
   if (ctx->select_path == 0) {
@@ -276,6 +282,14 @@ int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t s
       const int blocks = ctx->stream_blocks[sizeof(GradT) == 4 ? 0 : 1];
       k_stream<GradT><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
       ++ctx->launches;
+      if (clear_out) {
+        // the streaming pass saturates the memory system and the kernels after it do not: the dense
+        // update is cleared on the side stream once the pass has ended
+        RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_streamed, st));
+        RTOPK_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_streamed, 0));
+        RTOPK_CUDA(ctx, cudaMemsetAsync(clear_out, 0, clear_bytes, ctx->side));
+        RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_cleared, ctx->side));
+      }
       mark(ctx, RTOPK_PHASE_ORDER, st);
     }
     mark(ctx, RTOPK_PHASE_EXACT, st);
@@ -314,10 +328,10 @@ int upload_slices(rtopk_ctx* ctx, const Plan& P, cudaStream_t st) {
   return RTOPK_OK;
 }
 
-int run_sampler(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st) {
+int run_sampler(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st, bool clear_first = true) {
   if (!P.any_sampler) return RTOPK_OK;
   const uint32_t n = (uint32_t)P.slices.size();
-  RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_first, 0xFF, P.first_entries * sizeof(uint32_t), st));
+  if (clear_first) RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_first, 0xFF, P.first_entries * sizeof(uint32_t), st));
   const dim3 grid((P.k_draw_max + kDrawThreads - 1) / kDrawThreads, n);
   k_draw<<<grid, kDrawThreads, 0, st>>>(L);
   ++ctx->launches;
@@ -329,6 +343,30 @@ int run_sampler(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st)
   ++ctx->launches;
   k_sel_scan<<<sgrid, kScanThreads, 0, st>>>(L);
   ++ctx->launches;
+  return RTOPK_OK;
+}
+
+// Points a launch descriptor at the context's scratch for plan P and fills in the call's arguments.
+int bind_launch(rtopk_ctx* ctx, const Plan& P, const void* grad, float* residual, int32_t worker_base, uint64_t seed,
+                uint32_t step, uint32_t* msg_idx, float* msg_val, Launch& L, size_t* early_bytes, size_t* zbytes) {
+  std::memset(&L, 0, sizeof(L));
+  *zbytes = carve_zero(ctx, P, L.s, early_bytes);
+  if (*zbytes > ctx->zero_bytes) return RTOPK_ERR_INVALID_ARG;
+  L.s.slices = ctx->d_slices; L.s.state = ctx->d_state;
+  L.s.cand_idx = ctx->d_cand_idx; L.s.cand_val = ctx->d_cand_val;
+  L.s.raw_idx = ctx->d_raw_idx; L.s.raw_val = ctx->d_raw_val;
+  if ((size_t)P.n_chunks > ctx->chunk_tab_entries) return RTOPK_ERR_INVALID_ARG;
+  L.s.chunk_start = ctx->d_chunk_tab;
+  L.s.chunk_count = ctx->d_chunk_tab + ctx->chunk_tab_entries;
+  L.s.chunk_pre = ctx->d_chunk_tab + 2 * ctx->chunk_tab_entries;
+  L.s.draws = ctx->d_draws; L.s.first = ctx->d_first; L.s.sel_pre = ctx->d_sel_pre; L.s.sel_blk = ctx->d_sel_blk;
+  L.s.error = ctx->d_error;
+  L.grad = grad; L.residual = residual; L.msg_idx = msg_idx; L.msg_val = msg_val;
+  L.n_slices = (uint32_t)P.slices.size();
+  L.worker_base = (uint32_t)worker_base;
+  L.seed_lo = (uint32_t)seed; L.seed_hi = (uint32_t)(seed >> 32);
+  L.step = step;
+  L.general_primary = ctx->select_path == 1 ? 1u : 0u;
   return RTOPK_OK;
 }
 
@@ -348,24 +386,9 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return RTOPK_ERR_CUDA;
   Launch L;
-  std::memset(&L, 0, sizeof(L));
-  size_t early_bytes = 0;
-  const size_t zbytes = carve_zero(ctx, P, L.s, &early_bytes);
-  if (zbytes > ctx->zero_bytes) return RTOPK_ERR_INVALID_ARG;
-  L.s.slices = ctx->d_slices; L.s.state = ctx->d_state;
-  L.s.cand_idx = ctx->d_cand_idx; L.s.cand_val = ctx->d_cand_val;
-  L.s.raw_idx = ctx->d_raw_idx; L.s.raw_val = ctx->d_raw_val;
-  if ((size_t)P.n_chunks > ctx->chunk_tab_entries) return RTOPK_ERR_INVALID_ARG;
-  L.s.chunk_start = ctx->d_chunk_tab;
-  L.s.chunk_count = ctx->d_chunk_tab + ctx->chunk_tab_entries;
-  L.s.draws = ctx->d_draws; L.s.first = ctx->d_first; L.s.sel_pre = ctx->d_sel_pre; L.s.sel_blk = ctx->d_sel_blk;
-  L.s.error = ctx->d_error;
-  L.grad = grad; L.residual = residual; L.msg_idx = msg_idx; L.msg_val = msg_val;
-  L.n_slices = (uint32_t)P.slices.size();
-  L.worker_base = (uint32_t)worker_base;
-  L.seed_lo = (uint32_t)seed; L.seed_hi = (uint32_t)(seed >> 32);
-  L.step = step;
-  L.general_primary = ctx->select_path == 1 ? 1u : 0u;
+  size_t early_bytes = 0, zbytes = 0;
+  rc = bind_launch(ctx, P, grad, residual, worker_base, seed, step, msg_idx, msg_val, L, &early_bytes, &zbytes);
+  if (rc) return rc;
 
   rc = upload_slices(ctx, P, st);
   if (rc) return rc;
@@ -397,13 +420,17 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
     if (late_on_side) RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero + early_bytes, 0, zbytes - early_bytes, ctx->side));
     rc = run_sampler(ctx, P, L, ctx->side);
     if (rc) return rc;
-    if (clear_out) RTOPK_CUDA(ctx, cudaMemsetAsync(clear_out, 0, (size_t)d * sizeof(float), ctx->side));
+    const bool clear_now = clear_out && !late_on_side;
+    if (clear_now) RTOPK_CUDA(ctx, cudaMemsetAsync(clear_out, 0, (size_t)d * sizeof(float), ctx->side));
     RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_join, ctx->side));
   } else if (late_on_side) {
     RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero + early_bytes, 0, zbytes - early_bytes, st));
   }
   cudaEvent_t join = forked ? ctx->ev_join : nullptr;
-  rc = grad_dtype == RTOPK_F32 ? launch_select<float>(ctx, P, L, st, join) : launch_select<__nv_bfloat16>(ctx, P, L, st, join);
+  float* clear_late = late_on_side ? clear_out : nullptr;
+  const size_t clear_bytes = (size_t)d * sizeof(float);
+  rc = grad_dtype == RTOPK_F32 ? launch_select<float>(ctx, P, L, st, join, clear_late, clear_bytes)
+                               : launch_select<__nv_bfloat16>(ctx, P, L, st, join, clear_late, clear_bytes);
   if (rc) return rc;
   if (forked) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0));
   mark(ctx, RTOPK_PHASE_FINISH, st);
@@ -429,12 +456,96 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
     k_emit_all<<<grid, kThreads, 0, st>>>(L, P.words_all_max);
     ++ctx->launches;
   }
+  if (clear_late) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_cleared, 0));
   mark(ctx, RTOPK_PHASE_AGGREGATE, st);
   ctx->ev_valid[RTOPK_N_PHASES] = false;   // closed by the aggregate of a step call, if any
   RTOPK_CUDA(ctx, cudaGetLastError());
   if (K_out) *K_out = P.K_row;
   return RTOPK_OK;
 }
+
+
+// The threshold-then-subsample encoder (proof of Theorem 1) for W rows: the streaming pass gathers
+// the coordinates above theta, then the sizes, the subset and the messages follow on the device.
+// `clear_out`: a dense update to clear beside the kernels that follow the streaming pass.
+int threshold_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
+                   int64_t d, int32_t W, int32_t worker_base, float theta, int64_t k, uint64_t seed, uint32_t step,
+                   uint32_t* msg_idx, float* msg_val, uint32_t* msg_count, uint32_t* msg_ones, cudaStream_t st,
+                   float* clear_out) {
+  int rc = check_common(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, msg_idx, msg_val);
+  if (rc) return rc;
+  if (!msg_count || !msg_ones || ((uintptr_t)msg_count & 3u) || ((uintptr_t)msg_ones & 3u)) return RTOPK_ERR_INVALID_ARG;
+  if (!(theta >= 0.0f) || theta > 3.4028234e38f) return RTOPK_ERR_INVALID_ARG;        // finite, not NaN
+  if (k < 1 || k > d || k > ctx->k_max) return RTOPK_ERR_INVALID_ARG;
+  if (ctx->select_path != 0) return RTOPK_ERR_UNSUPPORTED;
+  const int64_t limit = std::min<int64_t>(ctx->r_max, d);      // the largest marked set the scratch holds
+  if (k > limit) return RTOPK_ERR_INVALID_ARG;
+  const int64_t off[2] = {0, d};
+  Plan P;
+  rc = make_plan(ctx, ld_g, ld_m, d, W, 1, off, &limit, &k, P, true);
+  if (rc) return rc;
+  if (P.cand_entries > ctx->cand_entries || P.first_entries > ctx->first_entries || P.sel_words > ctx->sel_words)
+    return RTOPK_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return RTOPK_ERR_CUDA;
+  Launch L;
+  size_t early_bytes = 0, zbytes = 0;
+  rc = bind_launch(ctx, P, grad, residual, worker_base, seed, step, msg_idx, msg_val, L, &early_bytes, &zbytes);
+  if (rc) return rc;
+  rc = upload_slices(ctx, P, st);
+  if (rc) return rc;
+  // k_thr_sizes rewrites (r, k) of the device table: the next call uploads its slices afresh
+  ctx->cached_slices.clear();
+  ctx->history_stale = true;
+  ctx->last_n_slices = L.n_slices;
+  L.s.history = ctx->d_history;
+  uint32_t theta_key;
+  std::memcpy(&theta_key, &theta, 4);
+  theta_key &= 0x7FFFFFFFu;
+  mark(ctx, RTOPK_PHASE_SUBSET, st);
+  mark(ctx, RTOPK_PHASE_THRESHOLD, st);
+  k_thr_init<<<L.n_slices, kThrThreads, 0, st>>>(L, theta_key + 1u);
+  ++ctx->launches;
+  // the subset's tables are cleared beside the streaming pass
+  RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_fork, st));
+  RTOPK_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
+  RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero + early_bytes, 0, zbytes - early_bytes, ctx->side));
+  if (P.any_sampler) RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_first, 0xFF, P.first_entries * sizeof(uint32_t), ctx->side));
+  RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_join, ctx->side));
+  mark(ctx, RTOPK_PHASE_STREAM, st);
+  const uint32_t per = (uint32_t)((P.slices[0].head + (uint64_t)P.slices[0].len + kChunk - 1) / kChunk);
+  if (grad_dtype == RTOPK_F32)
+    k_stream<float><<<ctx->stream_blocks[0], kStreamThreads, sizeof(StreamSmem<float>), st>>>(L, P.n_chunks, per);
+  else
+    k_stream<__nv_bfloat16><<<ctx->stream_blocks[1], kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>), st>>>(L, P.n_chunks, per);
+  ++ctx->launches;
+  if (clear_out) {
+    RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_streamed, st));
+    RTOPK_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_streamed, 0));
+    RTOPK_CUDA(ctx, cudaMemsetAsync(clear_out, 0, (size_t)d * sizeof(float), ctx->side));
+    RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_cleared, ctx->side));
+  }
+  mark(ctx, RTOPK_PHASE_ORDER, st);
+  k_thr_sizes<<<L.n_slices, kThrSizeThreads, 0, st>>>(L, (uint32_t)limit, (uint32_t)k, msg_count, msg_ones);
+  ++ctx->launches;
+  mark(ctx, RTOPK_PHASE_EXACT, st);
+  RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0));
+  rc = run_sampler(ctx, P, L, st, false);
+  if (rc) return rc;
+  mark(ctx, RTOPK_PHASE_FINISH, st);
+  const dim3 egrid((P.chunks_max + kThrThreads / 32 - 1) / (kThrThreads / 32), L.n_slices);
+  k_thr_emit<<<egrid, kThrThreads, 0, st>>>(L);
+  ++ctx->launches;
+  if (clear_out) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_cleared, 0));
+  mark(ctx, RTOPK_PHASE_AGGREGATE, st);
+  ctx->ev_valid[RTOPK_N_PHASES] = false;
+  RTOPK_CUDA(ctx, cudaGetLastError());
+  return RTOPK_OK;
+}
+
+int aggregate_threshold_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, const uint32_t* msg_count,
+                             const uint32_t* msg_ones, int64_t d, int32_t W, int64_t k, float* out, cudaStream_t st,
+                             bool out_cleared);
 
 bool scale_mode_known(int m) {
   return m == RTOPK_SCALE_MEAN || m == RTOPK_SCALE_SUM || m == RTOPK_SCALE_UNBIASED || m == RTOPK_SCALE_COUNT;
@@ -505,6 +616,17 @@ int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val
   return aggregate_launch(ctx, msgs, d, W, k, scale_mode, out, st, out_cleared, eta, r);
 }
 
+int aggregate_threshold_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, const uint32_t* msg_count,
+                             const uint32_t* msg_ones, int64_t d, int32_t W, int64_t k, float* out, cudaStream_t st,
+                             bool out_cleared) {
+  if (!msg_idx || !msg_val || !msg_count || !msg_ones) return RTOPK_ERR_INVALID_ARG;
+  if (((uintptr_t)msg_idx & 3u) || ((uintptr_t)msg_val & 3u) || ((uintptr_t)msg_count & 3u) || ((uintptr_t)msg_ones & 3u))
+    return RTOPK_ERR_INVALID_ARG;
+  if (k < 1 || k > 0xFFFFFFFFll) return RTOPK_ERR_INVALID_ARG;
+  const ThresholdMsgs msgs = {msg_idx, msg_val, (uint32_t)k, msg_count, msg_ones};
+  return aggregate_launch(ctx, msgs, d, W, k, RTOPK_SCALE_MEAN, out, st, out_cleared, -1.0f, 0);
+}
+
 // ceil(log2 d) index bits (at least 1) and the smallest row strides of the packed format: index
 // words rounded up to 4 (16 bytes), value halves rounded up to 8 (16 bytes).
 int packed_layout(int64_t d, int64_t k, int32_t* bits, int64_t* ld_words, int64_t* ld_halves) {
@@ -573,7 +695,7 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   alloc((void**)&ctx->d_raw_idx, ctx->cand_entries * sizeof(uint32_t));
   alloc((void**)&ctx->d_raw_val, ctx->cand_entries * sizeof(float));
   ctx->chunk_tab_entries = chunks;
-  alloc((void**)&ctx->d_chunk_tab, 2 * chunks * sizeof(uint32_t));
+  alloc((void**)&ctx->d_chunk_tab, 3 * chunks * sizeof(uint32_t));
   alloc((void**)&ctx->d_draws, W * (size_t)k_max * sizeof(uint32_t));
   alloc((void**)&ctx->d_sel_pre, ctx->sel_words * sizeof(uint32_t));
   ctx->sel_blk_entries = slices * ((size_t)r_max / 32 / kSelChunk + 2);
@@ -587,6 +709,8 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_streamed, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_cleared, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFinishSmemBytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
   for (int c = 1; c <= kMaxCluster && e == cudaSuccess; ++c) {
@@ -641,6 +765,8 @@ int rtopk_destroy(rtopk_ctx* ctx) {
   for (cudaEvent_t ev : ctx->ev) if (ev) cudaEventDestroy(ev);
   if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
   if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+  if (ctx->ev_streamed) cudaEventDestroy(ctx->ev_streamed);
+  if (ctx->ev_cleared) cudaEventDestroy(ctx->ev_cleared);
   if (ctx->side) cudaStreamDestroy(ctx->side);
   delete ctx;
   return RTOPK_OK;
@@ -797,6 +923,32 @@ int rtopk_step_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64
                                seg_k, seed, step, msg_idx, msg_val, (cudaStream_t)stream, &K, sparse ? out : nullptr);
   if (rc) return rc;
   return aggregate_impl(ctx, msg_idx, msg_val, d, W, K, scale_mode, out, (cudaStream_t)stream, sparse);
+}
+
+int rtopk_sparsify_threshold(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,
+                             int64_t ld_m, int64_t d, int32_t W, int32_t worker_base, float theta, int64_t k,
+                             uint64_t seed, uint32_t step, uint32_t* msg_idx, float* msg_val, uint32_t* msg_count,
+                             uint32_t* msg_ones, void* stream) {
+  return threshold_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, theta, k, seed, step, msg_idx,
+                        msg_val, msg_count, msg_ones, (cudaStream_t)stream, nullptr);
+}
+
+int rtopk_aggregate_threshold(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, const uint32_t* msg_count,
+                              const uint32_t* msg_ones, int64_t d, int32_t W, int64_t k, float* out, void* stream) {
+  return aggregate_threshold_impl(ctx, msg_idx, msg_val, msg_count, msg_ones, d, W, k, out, (cudaStream_t)stream, false);
+}
+
+int rtopk_step_threshold(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
+                         int64_t d, int32_t W, int32_t worker_base, float theta, int64_t k, uint64_t seed,
+                         uint32_t step, uint32_t* msg_idx, float* msg_val, uint32_t* msg_count, uint32_t* msg_ones,
+                         float* out, void* stream) {
+  if (!out || ((uintptr_t)out & 15u)) return RTOPK_ERR_INVALID_ARG;
+  if (!ctx || d < 1 || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
+  const bool sparse = W >= 1 && k >= 1 && aggregate_is_sparse(d, W, k);
+  const int rc = threshold_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, theta, k, seed, step,
+                                msg_idx, msg_val, msg_count, msg_ones, (cudaStream_t)stream, sparse ? out : nullptr);
+  if (rc) return rc;
+  return aggregate_threshold_impl(ctx, msg_idx, msg_val, msg_count, msg_ones, d, W, k, out, (cudaStream_t)stream, sparse);
 }
 
 int rtopk_step_host(rtopk_ctx* ctx, const void* h_grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
