@@ -205,6 +205,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--apply", action="store_true",
                     help="time rtopk_step_apply (master update fused into the aggregation; plain workloads, 1 GPU)")
+    ap.add_argument("--threshold", type=float, default=None,
+                    help="time rtopk_step_threshold (the threshold-then-subsample encoder) with this theta "
+                         "instead of rtopk_step (plain workloads, 1 GPU; message capacity = the workload's k)")
     ap.add_argument("--reuse-threshold", type=int, default=1, choices=[0, 1],
                     help="1 (default): the rounds of the loop predict their first threshold from the previous "
                          "rounds (RTOPK_OPT_REUSE_THRESHOLD; results are the same); 0: every round samples")
@@ -239,8 +242,9 @@ def main():
     gsz = 4 if cfg.grad_dtype == "f32" else 2
     K = cfg.k_total
     seg = cfg.seg_off is not None
-    ctx = rt.RTopK(d_max=d, W_max=W_total, r_max=cfg.r, k_max=K, segments_max=len(cfg.seg_r) if seg else 1,
-                   device=local)
+    thr = args.threshold is not None
+    ctx = rt.RTopK(d_max=d, W_max=W_total, r_max=min(d, 4 * cfg.r) if thr else cfg.r, k_max=K,
+                   segments_max=len(cfg.seg_r) if seg else 1, device=local)
 
     if args.reuse_threshold:
         from paper_2005_10761_b200.binding import OPT_REUSE_THRESHOLD
@@ -257,8 +261,10 @@ def main():
     val = torch.zeros((W, K), dtype=torch.float32, device=dev)
     # the dense update; with --apply the model weights that the update is applied to
     out = torch.zeros(wl.round_up(d, 4), dtype=torch.float32, device=dev)
-    if args.apply and (seg or world > 1):
-        raise SystemExit("--apply covers the plain single-GPU workloads")
+    if (args.apply or thr) and (seg or world > 1):
+        raise SystemExit("--apply and --threshold cover the plain single-GPU workloads")
+    cnt = torch.zeros(W, dtype=torch.int32, device=dev)
+    ones = torch.zeros(W, dtype=torch.int32, device=dev)
     base = rank * W
 
     def one_step(t: int):
@@ -266,6 +272,8 @@ def main():
         if world == 1:
             if seg:
                 ctx.step_segmented(g, residual, d, cfg.seg_off, cfg.seg_r, cfg.seg_k, cfg.seed, t, idx, val, out)
+            elif thr:
+                ctx.step_threshold(g, residual, d, args.threshold, cfg.k, cfg.seed, t, idx, val, cnt, ones, out)
             elif args.apply:
                 ctx.step_apply(g, residual, d, cfg.r, cfg.k, cfg.seed, t, 0.01, idx, val, out)
             else:
@@ -352,7 +360,7 @@ def main():
 
     # end to end: host gradient in, host messages + update out, through rtopk_step_host
     e2e = None
-    if not args.no_e2e and world == 1 and not seg and not args.apply:
+    if not args.no_e2e and world == 1 and not seg and not args.apply and not thr:
         h_grad = grads[0].cpu().pin_memory()
         h_idx = torch.zeros((W, K), dtype=torch.int32).pin_memory()
         h_val = torch.zeros((W, K), dtype=torch.float32).pin_memory()
@@ -392,11 +400,14 @@ def main():
                        "grad_dtype": cfg.grad_dtype, "recipe": cfg.recipe, "segments": len(cfg.seg_r) if seg else 1,
                        "gradient_batches_resident": n_batches, "residual": "carried across steps",
                        "l2": "inputs larger than L2 (no flush)", "parallelism": f"workers sharded x{world}",
-                       "variant": "rtopk_step_apply (fused master update)" if args.apply else "rtopk_step",
+                       "variant": ("rtopk_step_apply (fused master update)" if args.apply else
+                                   f"rtopk_step_threshold (theta = {args.threshold})" if thr else "rtopk_step"),
                        "reuse_threshold": bool(args.reuse_threshold)},
             "elements_per_s": W_total * d / (ms_per_step * 1e-3),
             "step_roofline_frac": step_frac, "step_algorithmic_bytes": step_bytes,
             "phases_ms": phases, "fallback_slices": fallbacks,
+            **({"marked_per_worker_last_step": float(ones.float().mean().item()),
+                "sent_per_worker_last_step": float(cnt.float().mean().item())} if thr else {}),
             "predicted_brackets": {"slices": predicted, "of": n_slices * n_prof},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": gpu_launches,
             "clocks": clocks,

@@ -170,3 +170,35 @@ def test_bad_arguments(lib):
         assert e.value.status == 1
     torch.cuda.synchronize()
     assert (idx == 5).all()
+
+
+@pytest.mark.parametrize("name,theta,k", [("c2", 0.5, 11173), ("c3_bf16", 150.0, 25557)])
+def test_full_size_all_rows(lib, name, theta, k):
+    # The encoder's oracle needs no sort, so every row of the full-size workloads is compared bit for bit,
+    # through rtopk_step_threshold, over two rounds with the residual carried.
+    cfg = wl.configs()[name]
+    oracle.set_threads(8)
+    ctx = lib.RTopK(d_max=cfg.d, W_max=cfg.W, r_max=cfg.r * 4, k_max=k)
+    tm = wl.zero_residual(cfg, "cuda")
+    m_or = np.zeros((cfg.W, cfg.ld), dtype=np.float32)
+    idx = torch.zeros((cfg.W, k), dtype=torch.int32, device="cuda")
+    val = torch.zeros((cfg.W, k), dtype=torch.float32, device="cuda")
+    cnt = torch.zeros(cfg.W, dtype=torch.int32, device="cuda")
+    ones = torch.zeros(cfg.W, dtype=torch.int32, device="cuda")
+    out = torch.zeros(wl.round_up(cfg.d, 4), dtype=torch.float32, device="cuda")
+    for t in range(2):
+        g = wl.gradient(cfg, t, "cuda")
+        ctx.step_threshold(g, tm, cfg.d, theta, k, cfg.seed, t, idx, val, cnt, ones, out)
+        ctx.poll_status()
+        g_or = g.cpu().view(torch.int16).numpy().view(np.uint16) if cfg.grad_dtype == "bf16" else g.cpu().numpy()
+        o_idx, o_val, o_cnt, o_ones = oracle.sparsify_threshold(np.ascontiguousarray(g_or), m_or, cfg.d, theta, k,
+                                                                cfg.seed, t)
+        _, o32 = oracle.aggregate_threshold(o_idx, o_val, o_cnt, o_ones, cfg.d)
+        assert np.array_equal(ones.cpu().numpy().view(np.uint32), o_ones)
+        assert np.array_equal(cnt.cpu().numpy().view(np.uint32), o_cnt)
+        assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx)
+        assert np.array_equal(_bits(val.cpu().numpy()), _bits(o_val))
+        assert np.array_equal(_bits(tm.cpu().numpy()), _bits(m_or))
+        assert np.array_equal(_bits(out.cpu().numpy()[:cfg.d]), _bits(o32))
+        assert (o_ones > k).any()                      # some rows subsample
+    oracle.set_threads(1)
