@@ -80,7 +80,7 @@ struct Scratch {
   SelState* state;
   uint32_t* hist;         // [slices][kBins]
   uint32_t* done;         // [slices] block-completion counters
-  uint32_t* tickets;      // [1] tile counter of the exact collect; [2] grid-barrier counter
+  uint32_t* tickets;      // [0], [1] tile counters of the exact collect; [2] grid-barrier counter; [3] chunk counter of k_stream
   unsigned long long* look_b;   // look-back words of the exact path's collect
   uint32_t* cursor;       // [slices] next free entry of the raw candidate buffer (= candidates so far)
   uint32_t* group_total;  // candidates per chunk group (summed by the stream pass)

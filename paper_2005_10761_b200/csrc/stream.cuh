@@ -1,7 +1,8 @@
 // k_stream: the one pass over the W x d gradient and residual matrices (Algorithm 1's g + m).
 //
 // Persistent blocks; each has one producer warp and eight consumer warps.  The producer takes chunk
-// tickets from a global counter and stages the chunk's residual and gradient bytes into shared
+// tickets from a global counter (blocks run at different speeds: a fixed assignment ends with the
+// slowest block's share) and stages the chunk's residual and gradient bytes into shared
 // memory with 1-D bulk async copies (TMA) that complete on an mbarrier; a ring of kStages buffers
 // keeps loads in flight while the consumers work.  The consumers form a = g + m, store it back,
 // flag the keys >= the sampled threshold, and append them -- in index order inside the chunk
@@ -128,9 +129,13 @@ __global__ void __launch_bounds__(kStreamThreads) k_stream(Launch L, uint32_t to
     // ------------------------------------------------------------------ producer (one lane)
     if (lane != 0) return;
     const char* grad = static_cast<const char*>(L.grad);
+    // The first chunk of a block is its own number; the following ones are tickets drawn from a
+    // global counter, so that blocks that run ahead take more chunks and all blocks end together.
+    // The next ticket is drawn while the current stage is still in use (its latency is hidden).
+    uint32_t tile = blockIdx.x;
     for (uint32_t i = 0;; ++i) {
       const uint32_t stage = i % kStages, phase = (i / kStages) & 1u;
-      const uint32_t tile = blockIdx.x + i * gridDim.x;
+      const uint32_t next_tile = tile < total_tiles ? gridDim.x + atomicAdd(&L.s.tickets[3], 1u) : tile;
       if (!mbar_wait(&sm.empty[stage], phase ^ 1u)) { atomicOr(L.s.error, ERR_LOOKBACK_TIMEOUT); return; }
       if (tile >= total_tiles) {
         sm.desc[stage].valid = 0;
@@ -150,6 +155,7 @@ __global__ void __launch_bounds__(kStreamThreads) k_stream(Launch L, uint32_t to
       mbar_arrive_expect_tx(&sm.full[stage], bytes_m + bytes_g);
       bulk_load(sm.m[stage], L.residual + (S->m_off - head) + e0, bytes_m, &sm.full[stage]);
       bulk_load(sm.g[stage], grad + ((S->g_off - head) + (int64_t)e0) * (int64_t)sizeof(GradT), bytes_g, &sm.full[stage]);
+      tile = next_tile;
     }
   }
 
