@@ -560,7 +560,6 @@ constexpr int kFinishThreads = 1024;
 constexpr int kFinishWarps = kFinishThreads / 32;
 constexpr int kFinishCache = 46 * 1024;   // candidate values a CTA keeps in shared memory (184 KB)
 constexpr int kFinishBatch = 8;           // independent loads in flight per thread
-constexpr int kRunBatch = 4;              // runs a lane group copies at a time
 constexpr int kFinishList = 512;          // bucket population up to which the bucket is ranked directly
 constexpr int kFinishListLong = 2048;     // ... when the CTAs' shares are long (must fit hist / red)
 constexpr int kFinishSelWords = 2048;     // bitmap words (64 Ki positions) a CTA keeps in shared memory
@@ -687,7 +686,6 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
       uint32_t* dstTab = sm.sel;                                 // [1025] first place of each run of the window
       uint32_t* srcTab = sm.sel_pre;                             // [1024] where the run sits in the raw buffer
       const uint32_t gpw = 10u - gsh;                            // log2(groups per window)
-      const uint32_t G = n_cand / nchunks < 16u ? 8u : 32u;      // lanes per run
       for (uint32_t wi = g0 >> gpw; (wi << 10) < nchunks && gpre[wi << gpw] < hi; ++wi) {
         const uint32_t c = (wi << 10) + tid;
         const bool has = c < nchunks;
@@ -721,45 +719,56 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
           }
           ++j_hi;
         }
-        // A group of G lanes copies one run (G = 8 when runs are short, else a whole warp), kRunBatch
-        // runs at a time so that their gathers are in flight together; lanes of a group take
-        // neighbouring elements, neighbouring groups neighbouring runs.
-        const uint32_t gl = tid & (G - 1u), gi = tid / G, n_grp = (uint32_t)kFinishThreads / G;
-        for (uint32_t j = j_lo + gi; j < j_hi; j += n_grp * kRunBatch) {
-          uint32_t first[kRunBatch], cnt[kRunBatch], src[kRunBatch], longest = 0;
+        // Copy the window's places inside [r_lo, r_hi): a warp takes 256 consecutive places at a time,
+        // lane l the places l, l + 32, ... of them (neighbouring lanes read neighbouring entries of a
+        // run and write neighbouring places).  The run of a lane's first place comes from a binary
+        // search in the window's table, the following ones by stepping forward; the 8 gathers of a
+        // lane are all in flight before the first is stored.
+        if (idx_cached) {
+          // everything goes to shared memory by asynchronous copies (no register holds a value), so a
+          // lane keeps 16 places in flight
+          for (uint32_t wb = r_lo + warp * 512u; wb < r_hi; wb += (uint32_t)kFinishWarps * 512u) {
+            const uint32_t at0 = wb + lane;
+            uint32_t j = j_lo;
+            if (at0 < r_hi) {                                      // last run that starts at or before at0
+              uint32_t hi_j = j_hi;
+              while (hi_j - j > 1u) { const uint32_t mid = (j + hi_j) >> 1; if (dstTab[mid] <= at0) j = mid; else hi_j = mid; }
+            }
 #pragma unroll
-          for (int u = 0; u < kRunBatch; ++u) {
-            const uint32_t jj = j + u * n_grp;
-            first[u] = 0; cnt[u] = 0; src[u] = 0;
-            if (jj < j_hi) { first[u] = dstTab[jj]; cnt[u] = dstTab[jj + 1] - first[u]; src[u] = srcTab[jj]; }
-            longest = max(longest, cnt[u]);
-          }
-          if (idx_cached) {
-            for (uint32_t e = gl; e < longest; e += G) {
-#pragma unroll
-              for (int u = 0; u < kRunBatch; ++u) {
-                const uint32_t at = first[u] + e;
-                if (e < cnt[u] && at >= r_lo && at < r_hi) {
-                  async_copy_4(cache_idx + (at - lo), ridx + src[u] + e);
-                  async_copy_4(cache + (at - lo), rval + src[u] + e);
-                }
+            for (int u = 0; u < 16; ++u) {
+              const uint32_t at = at0 + 32u * u;
+              if (at < r_hi) {
+                while (dstTab[j + 1] <= at) ++j;                   // dstTab[j_hi] >= r_hi > at ends it
+                const uint32_t src = srcTab[j] + (at - dstTab[j]);
+                async_copy_4(cache_idx + (at - lo), ridx + src);
+                async_copy_4(cache + (at - lo), rval + src);
               }
             }
-            continue;
           }
-          for (uint32_t e = gl; e < longest; e += G) {
-            uint32_t ri[kRunBatch];
-            float rv[kRunBatch];
+          continue;
+        }
+        for (uint32_t wb = r_lo + warp * 256u; wb < r_hi; wb += (uint32_t)kFinishWarps * 256u) {
+          const uint32_t at0 = wb + lane;
+          uint32_t j = j_lo;
+          if (at0 < r_hi) {
+            uint32_t hi_j = j_hi;
+            while (hi_j - j > 1u) { const uint32_t mid = (j + hi_j) >> 1; if (dstTab[mid] <= at0) j = mid; else hi_j = mid; }
+          }
+          uint32_t ri[kFinishBatch];
+          float rv[kFinishBatch];
 #pragma unroll
-            for (int u = 0; u < kRunBatch; ++u) {
-              const uint32_t at = first[u] + e;
-              if (e < cnt[u] && at >= r_lo && at < r_hi) { ri[u] = __ldg(ridx + src[u] + e); rv[u] = __ldg(rval + src[u] + e); }
+          for (int u = 0; u < kFinishBatch; ++u) {
+            const uint32_t at = at0 + 32u * u;
+            if (at < r_hi) {
+              while (dstTab[j + 1] <= at) ++j;
+              const uint32_t src = srcTab[j] + (at - dstTab[j]);
+              ri[u] = __ldg(ridx + src); rv[u] = __ldg(rval + src);
             }
+          }
 #pragma unroll
-            for (int u = 0; u < kRunBatch; ++u) {
-              const uint32_t at = first[u] + e;
-              if (e < cnt[u] && at >= r_lo && at < r_hi) put(at, ri[u], rv[u]);
-            }
+          for (int u = 0; u < kFinishBatch; ++u) {
+            const uint32_t at = at0 + 32u * u;
+            if (at < r_hi) put(at, ri[u], rv[u]);
           }
         }
       }
@@ -975,28 +984,47 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
       sm.sel_pre[w] = L.s.sel_pre[S.sel_off + word0 + w];
     }
   __syncthreads();
-  auto selected = [&](uint32_t p, uint32_t& slot) -> bool {
-    if (sel_all) { slot = p; return true; }
-    const uint32_t wi = p >> 5;
-    const uint32_t word = sel_cached ? sm.sel[wi - word0] : L.s.sel[S.sel_off + wi];
-    if (!((word >> (p & 31u)) & 1u)) return false;
-    const uint32_t pre = sel_cached ? sm.sel_pre[wi - word0] : L.s.sel_pre[S.sel_off + wi];
-    slot = pre + __popc(word & ((1u << (p & 31u)) - 1u));
-    return true;
+  // Bitmap words of a walk step: the members met in one step of 128 candidates take consecutive
+  // positions first_pos, first_pos + 1, ..., so they fall into at most 5 consecutive bitmap words.
+  // Lane l < 5 fetches word (first_pos / 32) + l and its running popcount; the walk reads them by shuffle.
+  const uint32_t sel_words_all = (S.r + 31u) >> 5;
+  auto fetch_sel = [&](uint32_t first_pos, uint32_t& word, uint32_t& pre) {
+    word = 0; pre = 0;
+    const uint32_t wi = (first_pos >> 5) + lane;
+    if (!sel_all && lane < 5u && wi < sel_words_all) {
+      if (sel_cached) {
+        if (wi - word0 < nwords) { word = sm.sel[wi - word0]; pre = sm.sel_pre[wi - word0]; }
+      } else {
+        word = L.s.sel[S.sel_off + wi];
+        pre = L.s.sel_pre[S.sel_off + wi];
+      }
+    }
   };
-
-  // walk my warp's part in index order: 4 consecutive candidates per lane, 128 per step
-  for (uint32_t w = 0; w < warp; ++w) { gt_before += sm.warpA[w]; eq_before += sm.warpB[w]; }
-  for (uint32_t base = w_lo; base < w_hi; base += 128u) {
+  // values and indices of a walk step (4 consecutive candidates per lane, 128 per step); the index
+  // list's capacity is a multiple of 32 entries, so the vector stays inside the slice's list
+  auto fetch_step = [&](uint32_t base, float (&v)[4], uint4& ci) {
     const uint32_t i0 = base + lane * 4u;
-    float v[4];
     load4(i0, v);
-    // the four indices, fetched now so that no store below waits on a load (the list's capacity is a
-    // multiple of 32 entries, so the vector stays inside the slice's list)
-    uint4 ci = make_uint4(0u, 0u, 0u, 0u);
+    ci = make_uint4(0u, 0u, 0u, 0u);
     if (i0 < w_hi) ci = idx_cached ? *reinterpret_cast<const uint4*>(cache_idx + i0)
                                    : *reinterpret_cast<const uint4*>(cidx + lo + i0);
-    const uint32_t cj[4] = {ci.x, ci.y, ci.z, ci.w};
+  };
+
+  // Walk my warp's part in index order.  Everything a step loads is requested one step ahead (the
+  // next step's candidates, and -- as soon as this step's member count is known -- the next step's
+  // bitmap words), so that no store of the current step waits behind a load.
+  for (uint32_t w = 0; w < warp; ++w) { gt_before += sm.warpA[w]; eq_before += sm.warpB[w]; }
+  float v_next[4] = {0.f, 0.f, 0.f, 0.f};
+  uint4 ci_next = make_uint4(0u, 0u, 0u, 0u);
+  uint32_t sw_next, sp_next;
+  if (w_lo < w_hi) fetch_step(w_lo, v_next, ci_next);
+  fetch_sel(gt_before + min(eq_before, quota), sw_next, sp_next);
+  for (uint32_t base = w_lo; base < w_hi; base += 128u) {
+    const uint32_t i0 = base + lane * 4u;
+    const float v[4] = {v_next[0], v_next[1], v_next[2], v_next[3]};
+    const uint32_t cj[4] = {ci_next.x, ci_next.y, ci_next.z, ci_next.w};
+    const uint32_t sw = sw_next, sp = sp_next;
+    if (base + 128u < w_hi) fetch_step(base + 128u, v_next, ci_next);
     uint32_t mA = 0, mB = 0;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -1009,25 +1037,32 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
     const uint32_t incl = warp_incl_scan(pack);
     const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
     const uint32_t excl = incl - pack;
+    const uint32_t first_pos = gt_before + min(eq_before, quota);
+    const uint32_t gt_after = gt_before + (tot & 0xFFFFu), eq_after = eq_before + (tot >> 16);
+    fetch_sel(gt_after + min(eq_after, quota), sw_next, sp_next);
     uint32_t g = gt_before + (excl & 0xFFFFu), e = eq_before + (excl >> 16);
-    if (mA | mB) {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const bool isA = (mA >> j) & 1u, isB = (mB >> j) & 1u;
-        if (isA || (isB && e < quota)) {
-          const uint32_t p = g + min(e, quota);
-          uint32_t slot;
-          if (p < S.r && selected(p, slot) && slot < S.k) {
-            const uint32_t idx = cj[j];
-            L.msg_idx[S.msg_off + slot] = S.idx_base + idx;
-            L.msg_val[S.msg_off + slot] = v[j];
-            L.residual[S.m_off + idx] = 0.0f;
-          }
+    for (int j = 0; j < 4; ++j) {
+      const bool isA = (mA >> j) & 1u, isB = (mB >> j) & 1u;
+      const bool member = isA || (isB && e < quota);
+      const uint32_t p = g + min(e, quota);
+      const uint32_t rel = member ? (p >> 5) - (first_pos >> 5) : 0u;       // 0 .. 4
+      const uint32_t word = __shfl_sync(0xFFFFFFFFu, sw, rel);
+      const uint32_t pre = __shfl_sync(0xFFFFFFFFu, sp, rel);
+      if (member && p < S.r) {
+        const uint32_t bit = p & 31u;
+        const bool take = sel_all || ((word >> bit) & 1u);
+        const uint32_t slot = sel_all ? p : pre + __popc(word & ((1u << bit) - 1u));
+        if (take && slot < S.k) {
+          const uint32_t idx = cj[j];
+          L.msg_idx[S.msg_off + slot] = S.idx_base + idx;
+          L.msg_val[S.msg_off + slot] = v[j];
+          L.residual[S.m_off + idx] = 0.0f;
         }
-        g += isA; e += isB;
       }
+      g += isA; e += isB;
     }
-    gt_before += tot & 0xFFFFu; eq_before += tot >> 16;
+    gt_before = gt_after; eq_before = eq_after;
   }
 }
 
