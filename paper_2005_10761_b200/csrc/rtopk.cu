@@ -432,7 +432,9 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   rc = grad_dtype == RTOPK_F32 ? launch_select<float>(ctx, P, L, st, join, clear_late, clear_bytes)
                                : launch_select<__nv_bfloat16>(ctx, P, L, st, join, clear_late, clear_bytes);
   if (rc) return rc;
-  if (forked) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0));
+  // (on the sampled path the exact kernel's launch has already waited for the side stream)
+  const bool joined = forked && ctx->select_path == 0;
+  if (forked && !joined) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0));
   mark(ctx, RTOPK_PHASE_FINISH, st);
   if (P.any_select) {
     // the largest cluster size that still lets every slice's cluster be resident at once

@@ -986,12 +986,12 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
   __syncthreads();
   // Bitmap words of a walk step: the members met in one step of 128 candidates take consecutive
   // positions first_pos, first_pos + 1, ..., so they fall into at most 5 consecutive bitmap words.
-  // Lane l < 5 fetches word (first_pos / 32) + l and its running popcount; the walk reads them by shuffle.
+  // Lane l < 6 fetches word (first_pos / 32) + l and its running popcount; the walk reads them by shuffle.
   const uint32_t sel_words_all = (S.r + 31u) >> 5;
   auto fetch_sel = [&](uint32_t first_pos, uint32_t& word, uint32_t& pre) {
     word = 0; pre = 0;
     const uint32_t wi = (first_pos >> 5) + lane;
-    if (!sel_all && lane < 5u && wi < sel_words_all) {
+    if (!sel_all && lane < 6u && wi < sel_words_all) {
       if (sel_cached) {
         if (wi - word0 < nwords) { word = sm.sel[wi - word0]; pre = sm.sel_pre[wi - word0]; }
       } else {
@@ -1040,27 +1040,45 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
     const uint32_t first_pos = gt_before + min(eq_before, quota);
     const uint32_t gt_after = gt_before + (tot & 0xFFFFu), eq_after = eq_before + (tot >> 16);
     fetch_sel(gt_after + min(eq_after, quota), sw_next, sp_next);
-    uint32_t g = gt_before + (excl & 0xFFFFu), e = eq_before + (excl >> 16);
+    // A lane's members take consecutive positions p0, p0 + 1, ... (at most four): their bitmap bits are
+    // one funnel shift of two neighbouring words, and the slot of the first is the word's running
+    // popcount plus the selected positions below p0 inside the word.
+    const uint32_t g0 = gt_before + (excl & 0xFFFFu), e0 = eq_before + (excl >> 16);
+    const uint32_t p0 = g0 + min(e0, quota);
+    uint32_t members = mA;                                                   // bit j: candidate j is in the top-r set
+    {
+      uint32_t e = e0;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const bool isA = (mA >> j) & 1u, isB = (mB >> j) & 1u;
-      const bool member = isA || (isB && e < quota);
-      const uint32_t p = g + min(e, quota);
-      const uint32_t rel = member ? (p >> 5) - (first_pos >> 5) : 0u;       // 0 .. 4
-      const uint32_t word = __shfl_sync(0xFFFFFFFFu, sw, rel);
-      const uint32_t pre = __shfl_sync(0xFFFFFFFFu, sp, rel);
-      if (member && p < S.r) {
-        const uint32_t bit = p & 31u;
-        const bool take = sel_all || ((word >> bit) & 1u);
-        const uint32_t slot = sel_all ? p : pre + __popc(word & ((1u << bit) - 1u));
-        if (take && slot < S.k) {
-          const uint32_t idx = cj[j];
-          L.msg_idx[S.msg_off + slot] = S.idx_base + idx;
-          L.msg_val[S.msg_off + slot] = v[j];
-          L.residual[S.m_off + idx] = 0.0f;
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t isB = (mB >> j) & 1u;
+        members |= (isB & (uint32_t)(e < quota)) << j;
+        e += isB;
+      }
+    }
+    const uint32_t rel = members ? (p0 >> 5) - (first_pos >> 5) : 0u;       // 0 .. 4
+    const uint32_t w0 = __shfl_sync(0xFFFFFFFFu, sw, rel);
+    const uint32_t w1 = __shfl_sync(0xFFFFFFFFu, sw, rel + 1u);
+    const uint32_t pre = __shfl_sync(0xFFFFFFFFu, sp, rel);
+    if (members) {
+      const uint32_t sh = p0 & 31u;
+      const uint32_t bits = sel_all ? 0xFu : __funnelshift_r(w0, w1, sh);    // bit o: the o-th member of the lane is chosen
+      const uint32_t slot0 = sel_all ? p0 : pre + __popc(w0 & ((1u << sh) - 1u));
+      uint32_t o = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if ((members >> j) & 1u) {
+          if (((bits >> o) & 1u) && p0 + o < S.r) {
+            const uint32_t slot = slot0 + __popc(bits & ((1u << o) - 1u));
+            if (slot < S.k) {
+              const uint32_t idx = cj[j];
+              L.msg_idx[S.msg_off + slot] = S.idx_base + idx;
+              L.msg_val[S.msg_off + slot] = v[j];
+              L.residual[S.m_off + idx] = 0.0f;
+            }
+          }
+          ++o;
         }
       }
-      g += isA; e += isB;
     }
     gt_before = gt_after; eq_before = eq_after;
   }

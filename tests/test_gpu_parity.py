@@ -584,3 +584,34 @@ def test_bad_arguments_return_invalid_arg_and_write_nothing(lib):
     assert bool((m == 1).all())
     ctx.poll_status()
     ctx.close()
+
+
+def test_step_can_be_captured_in_a_cuda_graph_and_replayed(lib):
+    # The call only enqueues work (its side stream forks from and rejoins the caller's stream), so a
+    # caller may capture it; the replay must give what the oracle gives for the captured (seed, step).
+    cfg = wl.scaled(wl.configs()["c2"], d=400003, W=3)
+    ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
+    g = wl.gradient(cfg, 0, "cuda")
+    m = wl.zero_residual(cfg, "cuda")
+    idx = torch.zeros((cfg.W, cfg.k), dtype=torch.int32, device="cuda")
+    val = torch.zeros((cfg.W, cfg.k), dtype=torch.float32, device="cuda")
+    out = torch.zeros(wl.round_up(cfg.d, 4), dtype=torch.float32, device="cuda")
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        ctx.step(g, m, cfg.d, cfg.r, cfg.k, cfg.seed, 0, idx, val, out)      # first call outside the capture
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=s):
+            ctx.step(g, m, cfg.d, cfg.r, cfg.k, cfg.seed, 1, idx, val, out)
+        m.zero_()
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        ctx.poll_status()
+    m_or = np.zeros((cfg.W, cfg.ld), dtype=np.float32)
+    o_idx, o_val = oracle.sparsify(g.cpu().numpy(), m_or, cfg.d, cfg.r, cfg.k, cfg.seed, 1)
+    _, o32 = oracle.aggregate(o_idx, o_val, cfg.d)
+    assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx)
+    assert np.array_equal(_bits(val.cpu().numpy()), _bits(o_val))
+    assert np.array_equal(_bits(m.cpu().numpy()), _bits(m_or))
+    assert np.array_equal(_bits(out.cpu().numpy()[:cfg.d]), _bits(o32))
