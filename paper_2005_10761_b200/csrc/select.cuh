@@ -560,8 +560,7 @@ constexpr int kFinishThreads = 1024;
 constexpr int kFinishWarps = kFinishThreads / 32;
 constexpr int kFinishCache = 46 * 1024;   // candidate values a CTA keeps in shared memory (184 KB)
 constexpr int kFinishBatch = 8;           // independent loads in flight per thread
-constexpr int kFinishList = 512;          // bucket population up to which the bucket is ranked directly
-constexpr int kFinishListLong = 2048;     // ... when the CTAs' shares are long (must fit hist / red)
+constexpr int kFinishList = 2048;         // bucket population up to which the CTAs gather the bucket and finish on the list (fits hist / red)
 constexpr int kFinishSelWords = 2048;     // bitmap words (64 Ki positions) a CTA keeps in shared memory
 
 struct alignas(16) FinishSmem {           // the value cache behind it is read as float4
@@ -803,11 +802,11 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
   uint32_t bucket_n = general ? n_cand - n_gt : 0xFFFFFFFFu;
   // ranking a list by counting is quadratic: worth more than 512 keys only when a pass over the
   // share is long
-  const uint32_t list_max = n_mine > 32768u ? (uint32_t)kFinishListLong : (uint32_t)kFinishList;
+  const uint32_t list_max = (uint32_t)kFinishList;
   for (int round = 0; (hi_key - lo_key > 1u || count_above) && round < 8; ++round) {
     if (!count_above && bucket_n <= list_max) {
       // Few keys are left in the interval: instead of more histogram rounds, every CTA lists its own,
-      // reads the other CTAs' lists through distributed shared memory and ranks the union by counting.
+      // reads the other CTAs' lists through distributed shared memory and finishes on the union alone.
       if (tid == 0) sm.list_n = 0;
       __syncthreads();
       for_each_key([&](uint32_t key) {
@@ -835,22 +834,33 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
         while (sm.list_pre[rr + 1] <= t) ++rr;
         sm.red[t] = cluster.map_shared_rank(sm.hist, rr)[t - sm.list_pre[rr]];
       }
-      __syncthreads();
-      for (uint32_t t = tid; t < total; t += kFinishThreads) {
-        const uint32_t e = sm.red[t];
-        uint32_t rank = 0;                                       // keys ranked before e (ties: list order)
-        for (uint32_t j = 0; j < total; ++j) {
-          const uint32_t o = sm.red[j];
-          rank += (o > e) || (o == e && j < t);
-        }
-        if (rank == need - 1u) sm.tau_out = e;
-      }
-      __syncthreads();
-      const uint32_t found = sm.tau_out;
-      uint32_t above = 0;
-      for (uint32_t off = 0; off < total; off += kFinishThreads)
-        above += __syncthreads_count(off + tid < total && sm.red[off + tid] > found);
       cluster.sync();                                            // all remote reads of the lists are done
+      // Every CTA now holds the whole list and finishes alone: histogram rounds over the list only
+      // (equal buckets over what is left of the interval; one round when it spans at most 2048 keys).
+      uint32_t found = lo_key, end = hi_key, above = 0, rank = need;
+      bool ok = true;
+      while (end - found > 1u) {
+        const uint32_t w = end - found;
+        uint32_t s2 = 0;
+        while (((w - 1u) >> s2) >= (uint32_t)kBins) ++s2;
+        for (uint32_t bkt = tid; bkt < (uint32_t)kBins; bkt += kFinishThreads) sm.hist[bkt] = 0;
+        __syncthreads();
+        for (uint32_t t = tid; t < total; t += kFinishThreads) {
+          const uint32_t key = sm.red[t];
+          if (key >= found && key < end) atomicAdd(&sm.hist[(key - found) >> s2], 1u);
+        }
+        __syncthreads();
+        uint32_t D, ab;
+        ok = pick_digit(sm.hist, kBins, rank, sm.scratch, D, ab);
+        if (!ok) break;                                          // the same on every thread
+        above += ab; rank -= ab;
+        found += D << s2;
+        end = min(end, found + (1u << s2));
+      }
+      if (!ok) {
+        if (q == 0 && tid == 0) { atomicOr(L.s.error, ERR_SELECT_INCONSISTENT); st->resolved = 32; }
+        return;                                                  // every CTA of the cluster takes this exit
+      }
       n_gt += above; need -= above;
       lo_key = found; hi_key = found + 1u;
       break;
