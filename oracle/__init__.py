@@ -77,7 +77,7 @@ def lib() -> C.CDLL:
         L.oracle_decode_row.argtypes = [u32p, u16p, C.c_int64, C.c_int64, u32p, f32p]
         L.oracle_sparsify_threshold.argtypes = [C.c_void_p, C.c_int, C.c_int64, f32p, C.c_int64, C.c_int64,
                                                 C.c_int32, C.c_int32, C.c_float, C.c_int64, C.c_uint64,
-                                                C.c_uint32, u32p, f32p, u32p, u32p]
+                                                C.c_uint32, C.c_int, u32p, f32p, u32p, u32p]
         L.oracle_aggregate_threshold.argtypes = [u32p, f32p, u32p, u32p, C.c_int64, C.c_int32, C.c_int64,
                                                  f64p, f32p]
         _lib = L
@@ -258,8 +258,9 @@ if __name__ == "__main__":
 
 
 def sparsify_threshold(grad: np.ndarray, residual: np.ndarray, d: int, theta: float, k: int, seed: int,
-                       step: int, worker_base: int = 0):
+                       step: int, worker_base: int = 0, signs: bool = False):
     """Threshold-then-subsample encoder (proof of Theorem 1) on W rows; ``residual`` is updated in place.
+    ``signs``: a kept coordinate carries sign(a_i) * 2 theta instead of a_i.
     Returns (msg_idx [W,k] uint32, msg_val [W,k] float32, count [W] uint32, ones [W] uint32)."""
     dt = _grad_args(grad)
     assert residual.dtype == np.float32 and residual.ndim == 2 and residual.flags.c_contiguous
@@ -271,7 +272,7 @@ def sparsify_threshold(grad: np.ndarray, residual: np.ndarray, d: int, theta: fl
     ones = np.zeros(W, dtype=np.uint32)
     _check(lib().oracle_sparsify_threshold(grad.ctypes.data, dt, grad.shape[1], _p(residual, C.c_float),
                                            residual.shape[1], d, W, worker_base, theta, k, seed, step,
-                                           _p(idx, C.c_uint32), _p(val, C.c_float), _p(count, C.c_uint32),
+                                           1 if signs else 0, _p(idx, C.c_uint32), _p(val, C.c_float), _p(count, C.c_uint32),
                                            _p(ones, C.c_uint32)), "sparsify_threshold")
     return idx, val, count, ones
 

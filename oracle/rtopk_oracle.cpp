@@ -429,14 +429,20 @@ int oracle_decode_row(const uint32_t* packed_idx, const uint16_t* packed_val, in
 // as in Algorithm 1, unused message slots hold index 0xFFFFFFFF and value +0, and one term of the
 // estimator is double(value) * (double(ones_w) / double(count_w)), summed in worker order and
 // divided by n once.
+// `signs` != 0 is the scheme as Section II states it for signed, scaled observations: after the
+// quantisation a coordinate is 0 or +-M with M = 2 theta, so a kept coordinate carries sign(a_i) * M
+// (one bit on the wire) and the node keeps a_i - sign(a_i) * M there (one binary32 subtraction; a NaN
+// difference is stored as the default quiet NaN, like a NaN sum).
 int oracle_sparsify_threshold(const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
                               int64_t d, int32_t W, int32_t worker_base, float theta, int64_t k, uint64_t seed,
-                              uint32_t step, uint32_t* msg_idx, float* msg_val, uint32_t* msg_count,
+                              uint32_t step, int signs, uint32_t* msg_idx, float* msg_val, uint32_t* msg_count,
                               uint32_t* msg_ones) {
   if (!grad || !residual || !msg_idx || !msg_val || !msg_count || !msg_ones) return ORACLE_BAD_ARG;
   if (d < 1 || d > 0x7FFFFFFF || W < 1 || k < 1 || k > d || ld_g < d || ld_m < d) return ORACLE_BAD_ARG;
   if (grad_dtype != GRAD_F32 && grad_dtype != GRAD_BF16) return ORACLE_BAD_ARG;
   if (!(theta >= 0.0f) || std::isinf(theta)) return ORACLE_BAD_ARG;
+  const float M = theta + theta;
+  if (signs && std::isinf(M)) return ORACLE_BAD_ARG;
   const size_t gsz = grad_dtype == GRAD_F32 ? 4 : 2;
   const uint32_t theta_key = magnitude_key(theta);
   for_each_row(W, [&](int w) {
@@ -470,8 +476,16 @@ int oracle_sparsify_threshold(const void* grad, int grad_dtype, int64_t ld_g, fl
       if (q < (int64_t)kept.size()) {
         const uint32_t i = kept[(size_t)q];
         out_idx[q] = i;
-        out_val[q] = a[i];
-        a[i] = 0.0f;                                    // m' = a - ghat
+        if (!signs) {
+          out_val[q] = a[i];
+          a[i] = 0.0f;                                  // m' = a - ghat
+        } else {
+          const float sent = bits_float((float_bits(a[i]) & 0x80000000u) | float_bits(M));   // sign(a_i) * M
+          float rest = a[i] - sent;
+          if (rest != rest) rest = bits_float(0x7FC00000u);
+          out_val[q] = sent;
+          a[i] = rest;
+        }
       } else {
         out_idx[q] = 0xFFFFFFFFu;
         out_val[q] = 0.0f;

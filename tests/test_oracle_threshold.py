@@ -149,3 +149,40 @@ def test_estimator_mean_over_seeds_approaches_the_thresholded_vector():
     sd = np.sqrt(np.maximum(sq / n - mean * mean, 0) / n)
     assert (np.abs(mean - target) <= 5 * sd + 1e-12).all()
     assert (ones > k).all()                                               # the case really subsamples
+
+
+def test_sign_mode_sends_plus_minus_two_theta_and_keeps_the_difference():
+    rng = np.random.default_rng(21)
+    d, W, k, theta = 3000, 3, 50, 0.25
+    g = _spiky(rng, W, d, frac=0.05)
+    m0 = (_spiky(rng, W, d, frac=0.05) * 0.5).astype(np.float32)
+    a = g + m0
+    m_v, m_s = m0.copy(), m0.copy()
+    idx_v, val_v, cnt_v, ones_v = oracle.sparsify_threshold(g, m_v, d, theta, k, seed=4, step=2)
+    idx_s, val_s, cnt_s, ones_s = oracle.sparsify_threshold(g, m_s, d, theta, k, seed=4, step=2, signs=True)
+    assert np.array_equal(idx_v, idx_s) and np.array_equal(cnt_v, cnt_s) and np.array_equal(ones_v, ones_s)
+    M = np.float32(2 * theta)
+    for w in range(W):
+        n = int(cnt_s[w])
+        sent = idx_s[w, :n].astype(np.int64)
+        assert np.array_equal(val_s[w, :n], np.copysign(M, a[w][sent]))          # library copysign
+        want = a[w].copy()
+        want[sent] = a[w][sent] - np.copysign(M, a[w][sent])                      # numpy binary32 subtraction
+        assert np.array_equal(m_s[w].view(np.uint32), want.view(np.uint32))
+    with pytest.raises(ValueError):
+        oracle.sparsify_threshold(g, m0.copy(), d, 3e38, k, seed=4, step=2, signs=True)   # 2 theta overflows
+
+
+def test_sign_mode_on_the_scaled_signed_bernoulli_model_is_lossless_at_kept_coordinates():
+    # X in {0, +-M}^d, threshold M / 2: a kept coordinate is reproduced exactly and leaves nothing behind,
+    # and the estimate of n identical workers that keep everything is X itself.
+    rng = np.random.default_rng(8)
+    d, W, M = 400, 4, np.float32(0.75)
+    X = (np.where(rng.random(d) < 0.05, 1.0, 0.0) * np.where(rng.random(d) < 0.5, -1.0, 1.0)).astype(np.float32) * M
+    g = np.tile(X, (W, 1))
+    m = np.zeros_like(g)
+    n_ones = int(np.count_nonzero(X))
+    idx, val, cnt, ones = oracle.sparsify_threshold(g, m, d, float(M) / 2, n_ones, seed=1, step=0, signs=True)
+    assert (ones == n_ones).all() and (cnt == n_ones).all() and not m.any()
+    o64, o32 = oracle.aggregate_threshold(idx, val, cnt, ones, d)
+    assert np.array_equal(o32, X)
