@@ -72,11 +72,16 @@ enum {
                                 1 = always the multi-pass radix select over the full vector */
   RTOPK_OPT_PROFILE = 1,     /* 1 = record CUDA events between the phases of each call on the
                                 caller's stream (read with rtopk_get_phase_times); 0 = off */
-  RTOPK_OPT_REUSE_THRESHOLD = 2 /* 1 = consecutive calls of one shape on one residual buffer predict the
+  RTOPK_OPT_REUSE_THRESHOLD = 2, /* 1 = consecutive calls of one shape on one residual buffer predict the
                                 first threshold from the exact thresholds of the last calls instead
                                 of sampling (a = g + m drifts slowly from round to round); a
                                 prediction that misses is repaired by the exact path and the next
                                 call samples again.  Results never depend on it.  0 = off (default) */
+  RTOPK_OPT_THRESHOLD_SIGNS = 3 /* what rtopk_sparsify_threshold sends for a kept coordinate: 0 (default) its
+                                value a_i; 1 = sign(a_i) * M with M = 2 theta, the quantised observation of
+                                Section II (after the pre-processing step a coordinate is 0 or +-M, so one bit
+                                per kept coordinate describes it); the node then keeps a_i - sign(a_i) * M in
+                                that residual slot (one binary32 subtraction), m' = a - ghat as before */
 };
 
 /* Phases of one call, in stream order.  STREAM is the single pass over the full vectors that
@@ -249,7 +254,7 @@ int rtopk_step_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64
  * The message carries ones_w, count_w = min(ones_w, k) and the kept (index, value = a_i) pairs,
  * ascending; the node keeps m' = a - ghat (Algorithm 1).  "Exceeds" compares the magnitude bit
  * patterns strictly, so a NaN sum counts as marked.
- *   theta               finite, >= 0.
+ *   theta               finite, >= 0 (2 theta finite too with RTOPK_OPT_THRESHOLD_SIGNS).
  *   k                   message capacity (the proof's k'), 1 <= k <= min(d, the context's k_max).
  *   msg_idx, msg_val [out]  W x k; row w: count_w pairs, then padding (index 0xFFFFFFFF, value +0.0f).
  *   msg_count, msg_ones [out]  W 32-bit words each (device).

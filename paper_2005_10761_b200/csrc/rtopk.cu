@@ -52,6 +52,7 @@ struct rtopk_ctx {
   uint32_t* d_error = nullptr;
   TauHistory* d_history = nullptr;   // per-slice threshold history (RTOPK_OPT_REUSE_THRESHOLD)
   int reuse = 0;
+  int threshold_signs = 0;            // RTOPK_OPT_THRESHOLD_SIGNS
   bool history_stale = true;         // cleared before the next call that may use it
   const float* history_residual = nullptr;
   uint32_t* d_agg_starts = nullptr;
@@ -478,6 +479,8 @@ int threshold_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_
   if (rc) return rc;
   if (!msg_count || !msg_ones || ((uintptr_t)msg_count & 3u) || ((uintptr_t)msg_ones & 3u)) return RTOPK_ERR_INVALID_ARG;
   if (!(theta >= 0.0f) || theta > 3.4028234e38f) return RTOPK_ERR_INVALID_ARG;        // finite, not NaN
+  const float M = theta + theta;                                                       // the model's scale
+  if (ctx->threshold_signs && M > 3.4028234e38f) return RTOPK_ERR_INVALID_ARG;
   if (k < 1 || k > d || k > ctx->k_max) return RTOPK_ERR_INVALID_ARG;
   if (ctx->select_path != 0) return RTOPK_ERR_UNSUPPORTED;
   const int64_t limit = std::min<int64_t>(ctx->r_max, d);      // the largest marked set the scratch holds
@@ -536,7 +539,7 @@ int threshold_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_
   if (rc) return rc;
   mark(ctx, RTOPK_PHASE_FINISH, st);
   const dim3 egrid((P.chunks_max + kThrThreads / 32 - 1) / (kThrThreads / 32), L.n_slices);
-  k_thr_emit<<<egrid, kThrThreads, 0, st>>>(L);
+  k_thr_emit<<<egrid, kThrThreads, 0, st>>>(L, ctx->threshold_signs ? 1u : 0u, M);
   ++ctx->launches;
   if (clear_out) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_cleared, 0));
   mark(ctx, RTOPK_PHASE_AGGREGATE, st);
@@ -782,6 +785,7 @@ int rtopk_set_option(rtopk_ctx* ctx, int option, int64_t value) {
     ctx->history_stale = true;
     return RTOPK_OK;
   }
+  if (option == RTOPK_OPT_THRESHOLD_SIGNS && (value == 0 || value == 1)) { ctx->threshold_signs = (int)value; return RTOPK_OK; }
   if (option == RTOPK_OPT_PROFILE && (value == 0 || value == 1)) {
     ctx->profile = (int)value;
     for (bool& v : ctx->ev_valid) v = false;

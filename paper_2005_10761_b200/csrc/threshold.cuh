@@ -86,7 +86,10 @@ __global__ void __launch_bounds__(kThrSizeThreads) k_thr_sizes(Launch L, uint32_
 }
 
 // grid: (ceil(most chunks of a slice / warps per block), n_slices); one warp per chunk.
-__global__ void __launch_bounds__(kThrThreads) k_thr_emit(Launch L) {
+// signs != 0: a kept coordinate carries sign(a) * M (Section II: after the quantisation an observation
+// is 0 or +-M) and its residual slot keeps a - sign(a) * M, one binary32 subtraction (a NaN difference
+// is stored as the default quiet NaN, like a NaN sum).
+__global__ void __launch_bounds__(kThrThreads) k_thr_emit(Launch L, uint32_t signs, float M) {
   const uint32_t sl = blockIdx.y;
   const Slice S = L.s.slices[sl];
   const uint32_t lane = threadIdx.x & 31u;
@@ -110,9 +113,16 @@ __global__ void __launch_bounds__(kThrThreads) k_thr_emit(Launch L) {
     }
     if (slot >= S.k) continue;
     const uint32_t idx = ridx[e];
+    const float a = rval[e];
+    float sent = a, rest = 0.0f;
+    if (signs) {
+      sent = __uint_as_float((__float_as_uint(a) & 0x80000000u) | __float_as_uint(M));
+      rest = __fsub_rn(a, sent);
+      if (rest != rest) rest = __uint_as_float(0x7FC00000u);
+    }
     L.msg_idx[S.msg_off + slot] = S.idx_base + idx;
-    L.msg_val[S.msg_off + slot] = rval[e];
-    L.residual[S.m_off + idx] = 0.0f;
+    L.msg_val[S.msg_off + slot] = sent;
+    L.residual[S.m_off + idx] = rest;
   }
 }
 

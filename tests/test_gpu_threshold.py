@@ -41,9 +41,11 @@ def _spiky(rng, W, d, p=0.02):
     return np.where(m, rng.standard_normal((W, d)), x).astype(np.float32)
 
 
-def run_both(lib, g, m0, d, theta, k, r_max, seed=3, step=0, worker_base=0, bf16=False, ctx=None, use_step=False):
+def run_both(lib, g, m0, d, theta, k, r_max, seed=3, step=0, worker_base=0, bf16=False, ctx=None, use_step=False,
+             signs=False):
     W = g.shape[0]
     ctx = ctx or lib.RTopK(d_max=d, W_max=W, r_max=r_max, k_max=k)
+    ctx.set_option(3, 1 if signs else 0)
     tg = torch.from_numpy(g).cuda()
     g_or = g
     if bf16:
@@ -62,7 +64,7 @@ def run_both(lib, g, m0, d, theta, k, r_max, seed=3, step=0, worker_base=0, bf16
         ctx.aggregate_threshold(idx, val, cnt, ones, d, out)
     ctx.poll_status()
     m_or = m0.copy()
-    o_idx, o_val, o_cnt, o_ones = oracle.sparsify_threshold(g_or, m_or, d, theta, k, seed, step, worker_base)
+    o_idx, o_val, o_cnt, o_ones = oracle.sparsify_threshold(g_or, m_or, d, theta, k, seed, step, worker_base, signs)
     o64, o32 = oracle.aggregate_threshold(o_idx, o_val, o_cnt, o_ones, d)
     assert np.array_equal(ones.cpu().numpy().view(np.uint32), o_ones)
     assert np.array_equal(cnt.cpu().numpy().view(np.uint32), o_cnt)
@@ -71,7 +73,8 @@ def run_both(lib, g, m0, d, theta, k, r_max, seed=3, step=0, worker_base=0, bf16
     assert np.array_equal(_bits(tm.cpu().numpy()[:, :d]), _bits(m_or[:, :d]))
     got = out.cpu().numpy()[:d]
     assert np.array_equal(_bits(got), _bits(o32))
-    scale = float(np.abs(g[:, :d]).max()) or 1.0
+    finite = g[:, :d][np.isfinite(g[:, :d])]
+    scale = (float(np.abs(finite).max()) if finite.size else 0.0) or 1.0
     assert np.abs(got.astype(np.float64) - o64).max() <= 1e-6 * scale * max(1.0, float((o_ones / np.maximum(o_cnt, 1)).max()))
     return o_cnt, o_ones, tm, ctx
 
@@ -84,6 +87,18 @@ def test_small_and_ragged_sizes(lib, d, k, theta):
     g = _pad(_spiky(rng, W, d, p=0.05))
     m0 = _pad(_spiky(rng, W, d, p=0.05) * 0.5)
     run_both(lib, g, m0, d, theta, k, r_max=d, worker_base=4)
+
+
+@pytest.mark.parametrize("d,k,theta", [(5, 2, 0.0), (4097, 41, 0.1), (100003, 300, 0.3), (100003, 3000, 0.3)])
+def test_sign_mode(lib, d, k, theta):
+    rng = np.random.default_rng(d + 3 * k)
+    W = 3
+    g = _pad(_spiky(rng, W, d, p=0.05))
+    g[0, d // 2] = np.nan
+    g[1, 0] = np.inf
+    m0 = _pad(_spiky(rng, W, d, p=0.05) * 0.5)
+    run_both(lib, g, m0, d, theta, k, r_max=d, worker_base=2, signs=True)
+    run_both(lib, g, m0, d, theta, k, r_max=d, worker_base=2, signs=True, bf16=True, use_step=True)
 
 
 def test_subsampled_kept_all_and_empty_rows_in_one_call(lib):
