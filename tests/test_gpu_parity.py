@@ -615,3 +615,23 @@ def test_step_can_be_captured_in_a_cuda_graph_and_replayed(lib):
     assert np.array_equal(_bits(val.cpu().numpy()), _bits(o_val))
     assert np.array_equal(_bits(m.cpu().numpy()), _bits(m_or))
     assert np.array_equal(_bits(out.cpu().numpy()[:cfg.d]), _bits(o32))
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_random_shapes_values_and_paths(lib, case):
+    # Seeded random draws of everything a caller chooses: length, workers, r, k, first worker id, step,
+    # gradient type, selection path, and how heavy the ties are (values quantised to a few levels).
+    rng = np.random.default_rng(1000 + case)
+    d = int(rng.choice([rng.integers(1, 64), rng.integers(64, 5000), rng.integers(5000, 200000)]))
+    W = int(rng.integers(1, 6))
+    r = int(rng.integers(1, d + 1)) if rng.random() < 0.3 else int(max(1, d * rng.choice([0.001, 0.01, 0.05, 0.3])))
+    k = int(rng.integers(1, r + 1)) if rng.random() < 0.5 else max(1, r // int(rng.choice([2, 4, 10])))
+    g = _spiky(rng, W, d, p=float(rng.choice([0.0, 0.01, 0.2])))
+    m0 = _spiky(rng, W, d) * 0.5
+    levels = int(rng.choice([0, 0, 3, 17]))
+    if levels:                                   # many equal magnitudes, some across the threshold
+        g = (np.round(g * levels) / levels).astype(np.float32)
+        m0 = (np.round(m0 * levels) / levels).astype(np.float32)
+    check_against_oracle(lib, _pad(g), _pad(m0), d, r, k, seed=int(rng.integers(0, 2**40)), step=int(rng.integers(0, 1000)),
+                         worker_base=int(rng.integers(0, 50)), path=int(rng.choice([AUTO, EXACT])),
+                         bf16=bool(rng.random() < 0.3))
