@@ -288,10 +288,15 @@ int rtopk_step_threshold(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64
                          uint32_t* msg_ones, float* out, void* stream);
 
 /*
- * rtopk_step with HOST gradient and HOST results: copies h_grad (W x ld_g, ideally pinned) to a
- * device staging buffer owned by the context (allocated on first use), runs the step against the
- * DEVICE residual, and copies the messages and the dense update back to h_msg_idx, h_msg_val
- * (W x k) and h_out (d).  All copies are enqueued on `stream`; the call returns without waiting.
+ * rtopk_step with HOST gradient and HOST results.  h_grad (W x ld_g, ideally pinned, and complete when
+ * the call is made) is copied to one of two device staging buffers owned by the context (allocated
+ * on first use), the step runs on `stream` against the DEVICE residual, and the messages and the
+ * dense update are copied back to h_msg_idx, h_msg_val (W x k) and h_out (d).  The copies run on two
+ * streams of the context's own: the upload does not wait for `stream`, so in a sequence of calls it
+ * overlaps the previous call's step and download; `stream` waits for the download, so work enqueued on
+ * it afterwards, or a synchronisation of it, sees the results.  The call itself returns without
+ * waiting.  h_grad must stay unchanged until the step that reads it has started (synchronise `stream`,
+ * or make two further calls), the result buffers until `stream` has passed this call.
  */
 int rtopk_step_host(rtopk_ctx* ctx, const void* h_grad, int grad_dtype, int64_t ld_g,
                     float* residual, int64_t ld_m, int64_t d, int32_t W, int32_t worker_base,

@@ -57,8 +57,16 @@ struct rtopk_ctx {
   const float* history_residual = nullptr;
   uint32_t* d_agg_starts = nullptr;
   size_t agg_start_entries = 0;
-  void* d_stage = nullptr;       // host-call staging: gradient, messages, update
+  void* d_stage = nullptr;       // host-call staging: two gradient buffers, messages, update
   size_t stage_bytes = 0;
+  // rtopk_step_host moves data on two copy streams of its own, so that the upload of the next call's
+  // gradient and the download of the last call's results overlap the step between them
+  cudaStream_t copy_in = nullptr, copy_out = nullptr;
+  cudaEvent_t ev_uploaded[2] = {nullptr, nullptr};   // gradient buffer b holds this call's gradient
+  cudaEvent_t ev_consumed[2] = {nullptr, nullptr};   // the step that read gradient buffer b has ended
+  bool consumed_valid[2] = {false, false};
+  cudaEvent_t ev_downloaded = nullptr;               // the results of the last call are in host memory
+  int stage_next = 0;
   std::vector<Slice> cached_slices;   // what d_slices currently holds
   uint32_t last_n_slices = 0;
   // optional per-phase timing (RTOPK_OPT_PROFILE): events recorded on the caller's stream
@@ -773,6 +781,13 @@ int rtopk_destroy(rtopk_ctx* ctx) {
   if (ctx->ev_streamed) cudaEventDestroy(ctx->ev_streamed);
   if (ctx->ev_cleared) cudaEventDestroy(ctx->ev_cleared);
   if (ctx->side) cudaStreamDestroy(ctx->side);
+  if (ctx->copy_in) { cudaStreamSynchronize(ctx->copy_in); cudaStreamDestroy(ctx->copy_in); }
+  if (ctx->copy_out) { cudaStreamSynchronize(ctx->copy_out); cudaStreamDestroy(ctx->copy_out); }
+  for (int b = 0; b < 2; ++b) {
+    if (ctx->ev_uploaded[b]) cudaEventDestroy(ctx->ev_uploaded[b]);
+    if (ctx->ev_consumed[b]) cudaEventDestroy(ctx->ev_consumed[b]);
+  }
+  if (ctx->ev_downloaded) cudaEventDestroy(ctx->ev_downloaded);
   delete ctx;
   return RTOPK_OK;
 }
@@ -971,27 +986,55 @@ int rtopk_step_host(rtopk_ctx* ctx, const void* h_grad, int grad_dtype, int64_t 
   const size_t g_bytes = align_up((size_t)W * (size_t)ld_g * gsz, 256);
   const size_t mi_bytes = align_up((size_t)W * (size_t)k * 4, 256);
   const size_t out_bytes = align_up((size_t)d * 4, 256);
-  const size_t total = g_bytes + 2 * mi_bytes + out_bytes;
+  const size_t total = 2 * g_bytes + 2 * mi_bytes + out_bytes;
+  if (!ctx->copy_in) {
+    // first use: the copy streams and their events
+    RTOPK_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking));
+    RTOPK_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking));
+    for (int b = 0; b < 2; ++b) {
+      RTOPK_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_uploaded[b], cudaEventDisableTiming));
+      RTOPK_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_consumed[b], cudaEventDisableTiming));
+    }
+    RTOPK_CUDA(ctx, cudaEventCreateWithFlags(&ctx->ev_downloaded, cudaEventDisableTiming));
+  }
   if (total > ctx->stage_bytes) {
     // first use (or a larger shape): the one place a call allocates, and therefore waits
     RTOPK_CUDA(ctx, cudaStreamSynchronize(st));
+    RTOPK_CUDA(ctx, cudaStreamSynchronize(ctx->copy_in));
+    RTOPK_CUDA(ctx, cudaStreamSynchronize(ctx->copy_out));
     if (ctx->d_stage) { cudaFree(ctx->d_stage); ctx->d_stage = nullptr; ctx->stage_bytes = 0; }
     const cudaError_t e = cudaMalloc(&ctx->d_stage, total);
     if (e != cudaSuccess) { cudaGetLastError(); ctx->last_cuda_error = (int)e; return RTOPK_ERR_ALLOC; }
     ctx->stage_bytes = total;
+    ctx->consumed_valid[0] = ctx->consumed_valid[1] = false;
   }
+  const int b = ctx->stage_next;
+  ctx->stage_next ^= 1;
   char* base = (char*)ctx->d_stage;
-  void* d_grad = base;
-  uint32_t* d_idx = (uint32_t*)(base + g_bytes);
-  float* d_val = (float*)(base + g_bytes + mi_bytes);
-  float* d_out = (float*)(base + g_bytes + 2 * mi_bytes);
-  RTOPK_CUDA(ctx, cudaMemcpyAsync(d_grad, h_grad, (size_t)W * (size_t)ld_g * gsz, cudaMemcpyHostToDevice, st));
+  void* d_grad = base + (size_t)b * g_bytes;
+  uint32_t* d_idx = (uint32_t*)(base + 2 * g_bytes);
+  float* d_val = (float*)(base + 2 * g_bytes + mi_bytes);
+  float* d_out = (float*)(base + 2 * g_bytes + 2 * mi_bytes);
+  // upload: as soon as the step that last read this gradient buffer (two calls ago) has ended -- it does
+  // not wait for the caller's stream, so it runs beside the previous call's step and download
+  if (ctx->consumed_valid[b]) RTOPK_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_in, ctx->ev_consumed[b], 0));
+  RTOPK_CUDA(ctx, cudaMemcpyAsync(d_grad, h_grad, (size_t)W * (size_t)ld_g * gsz, cudaMemcpyHostToDevice, ctx->copy_in));
+  RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_uploaded[b], ctx->copy_in));
+  // step: on the caller's stream, once the gradient is there
+  RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_uploaded[b], 0));
   const int rc = rtopk_step(ctx, d_grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, r, k, seed, step,
                             scale_mode, d_idx, d_val, d_out, stream);
   if (rc) return rc;
-  RTOPK_CUDA(ctx, cudaMemcpyAsync(h_msg_idx, d_idx, (size_t)W * (size_t)k * 4, cudaMemcpyDeviceToHost, st));
-  RTOPK_CUDA(ctx, cudaMemcpyAsync(h_msg_val, d_val, (size_t)W * (size_t)k * 4, cudaMemcpyDeviceToHost, st));
-  RTOPK_CUDA(ctx, cudaMemcpyAsync(h_out, d_out, (size_t)d * 4, cudaMemcpyDeviceToHost, st));
+  RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_consumed[b], st));
+  ctx->consumed_valid[b] = true;
+  // download: behind the step; the caller's stream waits for it, so that whatever follows on that
+  // stream (or a synchronisation of it) sees the results, and the next step does not overwrite them early
+  RTOPK_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_out, ctx->ev_consumed[b], 0));
+  RTOPK_CUDA(ctx, cudaMemcpyAsync(h_msg_idx, d_idx, (size_t)W * (size_t)k * 4, cudaMemcpyDeviceToHost, ctx->copy_out));
+  RTOPK_CUDA(ctx, cudaMemcpyAsync(h_msg_val, d_val, (size_t)W * (size_t)k * 4, cudaMemcpyDeviceToHost, ctx->copy_out));
+  RTOPK_CUDA(ctx, cudaMemcpyAsync(h_out, d_out, (size_t)d * 4, cudaMemcpyDeviceToHost, ctx->copy_out));
+  RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_downloaded, ctx->copy_out));
+  RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_downloaded, 0));
   return RTOPK_OK;
 }
 

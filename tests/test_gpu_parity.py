@@ -511,6 +511,36 @@ def test_step_host_matches_device_call(lib):
     ctx.close()
 
 
+def test_step_host_sequence_without_waiting_in_between(lib):
+    # Five calls in a row on one stream, each with its own gradient and result buffers and no wait between
+    # them: uploads, steps and downloads of neighbouring calls overlap inside the library, and every
+    # call must still give what the device call gives on the same data (residual carried).
+    cfg = wl.scaled(wl.configs()["c2"], d=600011, W=4)
+    ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
+    n = 5
+    gs = [wl.gradient(cfg, t, "cpu").pin_memory() for t in range(n)]
+    idx_h = [torch.zeros((cfg.W, cfg.k), dtype=torch.int32).pin_memory() for _ in range(n)]
+    val_h = [torch.zeros((cfg.W, cfg.k), dtype=torch.float32).pin_memory() for _ in range(n)]
+    out_h = [torch.zeros(cfg.d, dtype=torch.float32).pin_memory() for _ in range(n)]
+    m_h = wl.zero_residual(cfg, "cuda")
+    for t in range(n):
+        ctx.step_host(gs[t], m_h, cfg.d, cfg.r, cfg.k, cfg.seed, t, idx_h[t], val_h[t], out_h[t])
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    ctx2 = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
+    m_d = wl.zero_residual(cfg, "cuda")
+    idx_d = torch.zeros((cfg.W, cfg.k), dtype=torch.int32, device="cuda")
+    val_d = torch.zeros((cfg.W, cfg.k), dtype=torch.float32, device="cuda")
+    out_d = torch.empty(cfg.ld, dtype=torch.float32, device="cuda")
+    for t in range(n):
+        ctx2.step(gs[t].cuda(), m_d, cfg.d, cfg.r, cfg.k, cfg.seed, t, idx_d, val_d, out_d)
+        torch.cuda.synchronize()
+        assert torch.equal(idx_h[t], idx_d.cpu()), t
+        assert torch.equal(val_h[t].view(torch.int32), val_d.cpu().view(torch.int32)), t
+        assert torch.equal(out_h[t].view(torch.int32), out_d.cpu()[: cfg.d].view(torch.int32)), t
+    assert torch.equal(m_h.view(torch.int32), m_d.view(torch.int32))
+
+
 @pytest.mark.parametrize("r,k", [(1, 1), (2, 1), (7, 3), (64, 64), (1000, 1), (1000, 999), (16384, 1024),
                                  (111739, 11173), (2684354, 671088)])
 def test_sampler_positions_against_oracle(lib, r, k):
