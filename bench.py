@@ -118,14 +118,15 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def pick_workload(name: str, scale_d: int = 0):
+def pick_workload(name: str, scale_d: int = 0, workers: int = 0):
     from paper_2005_10761_b200 import workloads as wl
     cfgs = wl.configs()
     if name not in cfgs:
         raise SystemExit(f"unknown workload {name!r}; choose from {sorted(cfgs)}")
     cfg = cfgs[name]
-    if scale_d:          # same recipe and ratios at another length (small profiling captures)
-        cfg = wl.scaled(cfg, d=scale_d)
+    if scale_d or workers:   # same recipe and ratios at another length / row count (small profiling captures)
+        cfg = wl.scaled(cfg, d=scale_d or cfg.d, W=workers or cfg.W,
+                        name=cfg.name + (f"_d{scale_d}" if scale_d else "") + (f"_W{workers}" if workers else ""))
     return cfg
 
 
@@ -173,7 +174,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    cfg = pick_workload(args.workload, args.scale_d)
+    cfg = pick_workload(args.workload, args.scale_d, args.workers)
     cores = os.cpu_count() or 1
     rows = cpu_sample_rows(cfg, cores)
     threads = min(cores, rows)
@@ -201,6 +202,8 @@ def main():
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--scale-d", type=int, default=0, help="run the workload's recipe at this vector length")
+    ap.add_argument("--workers", type=int, default=0,
+                    help="run the workload's recipe with this many worker rows per GPU (plain workloads)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--apply", action="store_true",
@@ -236,7 +239,7 @@ def main():
     if world > 1:
         dist.barrier()
 
-    cfg = pick_workload(args.workload, args.scale_d)
+    cfg = pick_workload(args.workload, args.scale_d, args.workers)
     W, d, ld = cfg.W, cfg.d, cfg.ld
     W_total = W * world                      # weak scaling: W workers per GPU
     gsz = 4 if cfg.grad_dtype == "f32" else 2

@@ -572,7 +572,7 @@ struct alignas(16) FinishSmem {           // the value cache behind it is read a
   uint32_t counts[2 * kMaxCluster];    // (members above tau, equal to tau) of every CTA's share
   uint32_t warpA[kFinishWarps], warpB[kFinishWarps];
   uint32_t list_pre[kMaxCluster + 1];  // list round: exclusive prefix of the CTAs' list lengths
-  uint32_t list_n, tau_out;            // list round: my list length; the key that was found
+  uint32_t list_n, pad_;               // list round: my list length
 };
 static_assert(sizeof(FinishSmem) % 16 == 0, "the value cache must start 16-byte aligned");
 constexpr size_t kFinishSmemBytes = sizeof(FinishSmem) + (size_t)kFinishCache * sizeof(float);
@@ -800,8 +800,7 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
 
   // keys inside [lo_key, hi_key) over the whole cluster, when known
   uint32_t bucket_n = general ? n_cand - n_gt : 0xFFFFFFFFu;
-  // ranking a list by counting is quadratic: worth more than 512 keys only when a pass over the
-  // share is long
+  // a bucket of up to kFinishList keys is gathered by every CTA and resolved there without further passes over the shares
   const uint32_t list_max = (uint32_t)kFinishList;
   for (int round = 0; (hi_key - lo_key > 1u || count_above) && round < 8; ++round) {
     if (!count_above && bucket_n <= list_max) {
