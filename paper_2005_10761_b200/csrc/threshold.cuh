@@ -12,7 +12,9 @@
 //                 when ||X||_1 <= k'), numbers the chunks' runs in index order and pads the message;
 //   k_thr_emit    walks the runs: a marked coordinate's position in index order is its run's first
 //                 position plus its place in the run; the ones the subset holds become (index,
-//                 value) messages and their residual slots are zeroed (Algorithm 1's m' = a - ghat).
+//                 value) messages -- the value a_i, or sign(a_i) * 2 theta in sign mode -- and their
+//                 residual slots keep what was not sent (Algorithm 1's m' = a - ghat: zero, or the
+//                 difference in sign mode).
 #pragma once
 
 #include "common.cuh"
