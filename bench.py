@@ -12,6 +12,9 @@ time of a step, inputs resident in HBM); `e2e` is the same through rtopk_step_ho
 buffers (host<->device copies inside the timed region); `roofline` is the fused streaming kernel's
 algorithmic bytes over its own event-timed duration against the measured HBM copy bandwidth;
 `cpu_baseline` is the CPU oracle timed on a bounded sample of the same workload.
+On one GPU the timed rounds are replays of a CUDA graph that holds one round per resident gradient
+batch (`--graph 0` launches them on the stream instead); the kernels and their work are the same, the
+round number that enters the Philox counter lives in a device word that every round advances.
 """
 from __future__ import annotations
 
@@ -211,6 +214,10 @@ def main():
     ap.add_argument("--threshold", type=float, default=None,
                     help="time rtopk_step_threshold (the threshold-then-subsample encoder) with this theta "
                          "instead of rtopk_step (plain workloads, 1 GPU; message capacity = the workload's k)")
+    ap.add_argument("--graph", type=int, default=1, choices=[0, 1],
+                    help="1 (default): the timed rounds are replays of a CUDA graph that holds one round per resident "
+                         "gradient batch (the round counter lives on the device, RTOPK_OPT_DEVICE_STEP, so every "
+                         "replayed round still draws its own subset); 1 GPU")
     ap.add_argument("--reuse-threshold", type=int, default=1, choices=[0, 1],
                     help="1 (default): the rounds of the loop predict their first threshold from the previous "
                          "rounds (RTOPK_OPT_REUSE_THRESHOLD; results are the same); 0: every round samples")
@@ -322,8 +329,41 @@ def main():
     sampler = ClockSampler(local) if rank == 0 else None
     wall0 = time.time()
     launches0 = ctx.launch_count()
-    total_ms = timed(one_step, t_next, args.steps)
-    gpu_launches = ctx.launch_count() - launches0   # this library's kernels inside the timed region
+    graphed = bool(args.graph) and world == 1
+    if graphed:
+        from paper_2005_10761_b200.binding import OPT_DEVICE_STEP
+        ctx.set_option(OPT_DEVICE_STEP, 1)
+        ctx.set_device_step(t_next)
+        reps, rem = divmod(args.steps, n_batches)
+        launches_per_graph = 0
+        if reps:
+            try:
+                cap_stream = torch.cuda.Stream()
+                graph = torch.cuda.CUDAGraph()
+                torch.cuda.synchronize()
+                l0 = ctx.launch_count()
+                with torch.cuda.graph(graph, stream=cap_stream):
+                    for b in range(n_batches):
+                        one_step(b)
+                launches_per_graph = ctx.launch_count() - l0
+                torch.cuda.synchronize()
+            except Exception as ex:        # no capture on this machine: the rounds are launched one by one
+                print(f"bench: CUDA graph capture failed ({ex!r}); launching on the stream", file=sys.stderr)
+                torch.cuda.synchronize()
+                reps, rem, graphed = 0, args.steps, False
+
+        def graph_rounds(i: int):          # called once per timed "step" index; replays at the batch boundaries
+            if i < reps * n_batches:
+                if i % n_batches == 0:
+                    graph.replay()
+            else:
+                one_step(i)
+        launches0 = ctx.launch_count()
+        total_ms = timed(graph_rounds, 0, args.steps)
+        gpu_launches = ctx.launch_count() - launches0 + reps * launches_per_graph
+    else:
+        total_ms = timed(one_step, t_next, args.steps)
+        gpu_launches = ctx.launch_count() - launches0   # this library's kernels inside the timed region
     wall1 = time.time()
     t_next += args.steps
     clocks = sampler.stop(wall0, wall1) if sampler else None
@@ -405,6 +445,7 @@ def main():
                        "l2": "inputs larger than L2 (no flush)", "parallelism": f"workers sharded x{world}",
                        "variant": ("rtopk_step_apply (fused master update)" if args.apply else
                                    f"rtopk_step_threshold (theta = {args.threshold})" if thr else "rtopk_step"),
+                       "launch": "cuda graph replay" if (graphed and reps) else "stream launches",
                        "reuse_threshold": bool(args.reuse_threshold)},
             "elements_per_s": W_total * d / (ms_per_step * 1e-3),
             "step_roofline_frac": step_frac, "step_algorithmic_bytes": step_bytes,

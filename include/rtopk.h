@@ -77,11 +77,17 @@ enum {
                                 of sampling (a = g + m drifts slowly from round to round); a
                                 prediction that misses is repaired by the exact path and the next
                                 call samples again.  Results never depend on it.  0 = off (default) */
-  RTOPK_OPT_THRESHOLD_SIGNS = 3 /* what rtopk_sparsify_threshold sends for a kept coordinate: 0 (default) its
+  RTOPK_OPT_THRESHOLD_SIGNS = 3, /* what rtopk_sparsify_threshold sends for a kept coordinate: 0 (default) its
                                 value a_i; 1 = sign(a_i) * M with M = 2 theta, the quantised observation of
                                 Section II (after the pre-processing step a coordinate is 0 or +-M, so one bit
                                 per kept coordinate describes it); the node then keeps a_i - sign(a_i) * M in
                                 that residual slot (one binary32 subtraction), m' = a - ghat as before */
+  RTOPK_OPT_DEVICE_STEP = 4     /* 1 = the round number t that enters the Philox counter is kept in a word on
+                                the device: the sparsify / step calls (plain, segmented, threshold) ignore
+                                their `step` argument, read the word, and add one to it at their end (set it
+                                with rtopk_set_device_step; it starts at 0).  A caller that captures one round
+                                in a CUDA graph can then replay the graph round after round and still draw a
+                                fresh subset each time.  0 = off (default): `step` is the argument */
 };
 
 /* Phases of one call, in stream order.  STREAM is the single pass over the full vectors that
@@ -341,6 +347,10 @@ int rtopk_sample_positions(rtopk_ctx* ctx, int64_t r, int64_t k, uint64_t seed, 
 #define RTOPK_STATIC_MAX_R (1 << 20)
 int rtopk_sample_positions_static(int64_t r, int64_t k, uint64_t seed, uint32_t step, uint32_t worker,
                                   uint32_t segment, uint32_t* pos, void* stream);
+
+/* Sets the context's round counter (RTOPK_OPT_DEVICE_STEP) to `step`, in stream order.  A bookkeeping
+ * call with no counterpart in the paper beyond Algorithm 1's loop variable t.  Errors: INVALID_ARG, CUDA. */
+int rtopk_set_device_step(rtopk_ctx* ctx, uint32_t step, void* stream);
 
 /* Waits for `stream` and returns RTOPK_ERR_INTERNAL if any kernel of this context has raised the
  * device-side error flag since the last poll (the flag is then cleared), else RTOPK_OK. */

@@ -15,7 +15,7 @@ _LIB_PATH = os.path.join(_HERE, "librtopk.so")
 
 GRAD_F32, GRAD_BF16 = 0, 1
 SCALE_MEAN, SCALE_SUM, SCALE_UNBIASED, SCALE_COUNT = 0, 1, 2, 3
-OPT_SELECT_PATH, OPT_PROFILE, OPT_REUSE_THRESHOLD, OPT_THRESHOLD_SIGNS = 0, 1, 2, 3
+OPT_SELECT_PATH, OPT_PROFILE, OPT_REUSE_THRESHOLD, OPT_THRESHOLD_SIGNS, OPT_DEVICE_STEP = 0, 1, 2, 3, 4
 PHASES = ("subset", "threshold", "stream", "order", "exact", "finish", "aggregate")
 
 _vp, _i32, _i64, _u32, _u64, _int = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_uint64, C.c_int
@@ -56,6 +56,7 @@ EXPORTS = {
                                     _vp, _vp, _vp, _vp, _vp, _vp]),
     "rtopk_sample_positions": (_int, [_vp, _i64, _i64, _u64, _u32, _u32, _u32, _vp, _vp]),
     "rtopk_sample_positions_static": (_int, [_i64, _i64, _u64, _u32, _u32, _u32, _vp, _vp]),
+    "rtopk_set_device_step": (_int, [_vp, _u32, _vp]),
     "rtopk_poll_status": (_int, [_vp, _vp]),
     "rtopk_get_phase_times": (_int, [_vp, _vp, _vp]),
     "rtopk_get_stats": (_int, [_vp, _i32, _vp, _vp]),
@@ -301,6 +302,9 @@ class RTopK:
         rc = self._lib.rtopk_sample_positions(self._h, r, k, seed, step, worker, segment, pos.data_ptr(),
                                               _stream())
         self._check(rc, "rtopk_sample_positions")
+
+    def set_device_step(self, step: int) -> None:
+        self._check(self._lib.rtopk_set_device_step(self._h, step, _stream()), "rtopk_set_device_step")
 
     def poll_status(self) -> None:
         self._check(self._lib.rtopk_poll_status(self._h, _stream()), "rtopk_poll_status")

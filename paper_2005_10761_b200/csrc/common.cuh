@@ -110,6 +110,7 @@ struct Launch {
   uint32_t worker_base;
   uint32_t seed_lo, seed_hi;
   uint32_t step;
+  const uint32_t* step_ptr;   // not null: the round number is read from this device word instead of `step`
   uint32_t general_primary;   // 1: the full-vector radix select is the main path, not a fallback
   uint32_t reuse;             // 1: brackets may be predicted from the slices' threshold history
 };

@@ -53,6 +53,8 @@ struct rtopk_ctx {
   TauHistory* d_history = nullptr;   // per-slice threshold history (RTOPK_OPT_REUSE_THRESHOLD)
   int reuse = 0;
   int threshold_signs = 0;            // RTOPK_OPT_THRESHOLD_SIGNS
+  int device_step = 0;                // RTOPK_OPT_DEVICE_STEP
+  uint32_t* d_step = nullptr;         // the round counter on the device
   bool history_stale = true;         // cleared before the next call that may use it
   const float* history_residual = nullptr;
   uint32_t* d_agg_starts = nullptr;
@@ -376,6 +378,7 @@ int bind_launch(rtopk_ctx* ctx, const Plan& P, const void* grad, float* residual
   L.seed_lo = (uint32_t)seed; L.seed_hi = (uint32_t)(seed >> 32);
   L.step = step;
   L.general_primary = ctx->select_path == 1 ? 1u : 0u;
+  L.step_ptr = ctx->device_step ? ctx->d_step : nullptr;
   return RTOPK_OK;
 }
 
@@ -468,6 +471,7 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
     ++ctx->launches;
   }
   if (clear_late) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_cleared, 0));
+  if (ctx->device_step) { k_step_bump<<<1, 32, 0, st>>>(ctx->d_step); ++ctx->launches; }
   mark(ctx, RTOPK_PHASE_AGGREGATE, st);
   ctx->ev_valid[RTOPK_N_PHASES] = false;   // closed by the aggregate of a step call, if any
   RTOPK_CUDA(ctx, cudaGetLastError());
@@ -550,6 +554,7 @@ int threshold_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_
   k_thr_emit<<<egrid, kThrThreads, 0, st>>>(L, ctx->threshold_signs ? 1u : 0u, M);
   ++ctx->launches;
   if (clear_out) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_cleared, 0));
+  if (ctx->device_step) { k_step_bump<<<1, 32, 0, st>>>(ctx->d_step); ++ctx->launches; }
   mark(ctx, RTOPK_PHASE_AGGREGATE, st);
   ctx->ev_valid[RTOPK_N_PHASES] = false;
   RTOPK_CUDA(ctx, cudaGetLastError());
@@ -714,6 +719,7 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   ctx->sel_blk_entries = slices * ((size_t)r_max / 32 / kSelChunk + 2);
   alloc((void**)&ctx->d_sel_blk, ctx->sel_blk_entries * sizeof(uint32_t));
   alloc((void**)&ctx->d_error, 16);
+  alloc((void**)&ctx->d_step, 16);
   alloc((void**)&ctx->d_history, slices * sizeof(TauHistory));
   alloc((void**)&ctx->d_agg_starts, ctx->agg_start_entries * sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_sample<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSampleSmemBytes);
@@ -757,6 +763,7 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
     ctx->stream_blocks[1] = sms * per_bf16;
   }
   if (e == cudaSuccess) e = cudaMemset(ctx->d_error, 0, 16);
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_step, 0, 16);
   if (e == cudaSuccess) e = cudaMemset(ctx->d_state, 0, slices * sizeof(SelState));
   if (e != cudaSuccess) {
     const int rc = e == cudaErrorMemoryAllocation ? RTOPK_ERR_ALLOC : RTOPK_ERR_CUDA;
@@ -773,7 +780,8 @@ int rtopk_destroy(rtopk_ctx* ctx) {
   DeviceGuard guard(ctx->device);
   void* ptrs[] = {ctx->d_slices, ctx->d_state, ctx->d_zero, ctx->d_first, ctx->d_cand_idx, ctx->d_cand_val,
                   ctx->d_raw_idx, ctx->d_raw_val, ctx->d_chunk_tab,
-                  ctx->d_draws, ctx->d_sel_pre, ctx->d_sel_blk, ctx->d_error, ctx->d_agg_starts, ctx->d_stage, ctx->d_history};
+                  ctx->d_draws, ctx->d_sel_pre, ctx->d_sel_blk, ctx->d_error, ctx->d_agg_starts, ctx->d_stage, ctx->d_history,
+                  ctx->d_step};
   for (void* p : ptrs) if (p) cudaFree(p);
   for (cudaEvent_t ev : ctx->ev) if (ev) cudaEventDestroy(ev);
   if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
@@ -800,6 +808,7 @@ int rtopk_set_option(rtopk_ctx* ctx, int option, int64_t value) {
     ctx->history_stale = true;
     return RTOPK_OK;
   }
+  if (option == RTOPK_OPT_DEVICE_STEP && (value == 0 || value == 1)) { ctx->device_step = (int)value; return RTOPK_OK; }
   if (option == RTOPK_OPT_THRESHOLD_SIGNS && (value == 0 || value == 1)) { ctx->threshold_signs = (int)value; return RTOPK_OK; }
   if (option == RTOPK_OPT_PROFILE && (value == 0 || value == 1)) {
     ctx->profile = (int)value;
@@ -1070,6 +1079,16 @@ int rtopk_sample_positions(rtopk_ctx* ctx, int64_t r, int64_t k, uint64_t seed, 
   if (rc) return rc;
   const uint32_t nwords = (uint32_t)((r + 31) / 32);
   k_positions<<<(nwords + kThreads - 1) / kThreads, kThreads, 0, st>>>(L, pos);
+  ++ctx->launches;
+  RTOPK_CUDA(ctx, cudaGetLastError());
+  return RTOPK_OK;
+}
+
+int rtopk_set_device_step(rtopk_ctx* ctx, uint32_t step, void* stream) {
+  if (!ctx) return RTOPK_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return RTOPK_ERR_CUDA;
+  k_step_set<<<1, 32, 0, (cudaStream_t)stream>>>(ctx->d_step, step);
   ++ctx->launches;
   RTOPK_CUDA(ctx, cudaGetLastError());
   return RTOPK_OK;

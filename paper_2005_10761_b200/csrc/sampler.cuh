@@ -52,7 +52,8 @@ __global__ void __launch_bounds__(kDrawThreads) k_draw(Launch L) {
   const uint32_t i = blockIdx.x * kDrawThreads + threadIdx.x;
   if (i >= S.k) return;
   const uint32_t j = S.r - S.k + i;
-  const uint32_t t = floyd_draw(j, L.worker_base + S.row, S.segment, L.step, L.seed_lo, L.seed_hi);
+  const uint32_t step = L.step_ptr ? __ldg(L.step_ptr) : L.step;
+  const uint32_t t = floyd_draw(j, L.worker_base + S.row, S.segment, step, L.seed_lo, L.seed_hi);
   L.s.draws[S.samp_off + i] = t;
   first_note(L.s.first + S.first_off, S.first_mask, t, j);
 }
@@ -145,6 +146,10 @@ __global__ void __launch_bounds__(kScanThreads) k_sel_scan(Launch L) {
     run += cnt[u];
   }
 }
+
+// The context's round counter (RTOPK_OPT_DEVICE_STEP): set, and advanced by one at the end of a call.
+__global__ void k_step_set(uint32_t* word, uint32_t value) { if (blockIdx.x == 0 && threadIdx.x == 0) *word = value; }
+__global__ void k_step_bump(uint32_t* word) { if (blockIdx.x == 0 && threadIdx.x == 0) *word += 1u; }
 
 // Expands one slice's bitmap into the ascending list of chosen positions.
 __global__ void __launch_bounds__(kThreads) k_positions(Launch L, uint32_t* pos) {

@@ -665,3 +665,52 @@ def test_random_shapes_values_and_paths(lib, case):
     check_against_oracle(lib, _pad(g), _pad(m0), d, r, k, seed=int(rng.integers(0, 2**40)), step=int(rng.integers(0, 1000)),
                          worker_base=int(rng.integers(0, 50)), path=int(rng.choice([AUTO, EXACT])),
                          bf16=bool(rng.random() < 0.3))
+
+
+def test_device_round_counter_and_graph_replay_draw_fresh_subsets(lib):
+    # With the round counter on the device the `step` argument is ignored and every call advances the
+    # counter, so a captured round can be replayed and still follows Algorithm 1's t = 0, 1, 2, ...:
+    # eager calls with explicit steps, eager calls on the counter and graph replays must agree bit for bit.
+    cfg = wl.scaled(wl.configs()["c2"], d=300007, W=3)
+    g = wl.gradient(cfg, 0, "cuda")
+    n, first = 4, 7
+
+    def buffers():
+        return (wl.zero_residual(cfg, "cuda"), torch.zeros((cfg.W, cfg.k), dtype=torch.int32, device="cuda"),
+                torch.zeros((cfg.W, cfg.k), dtype=torch.float32, device="cuda"),
+                torch.zeros(wl.round_up(cfg.d, 4), dtype=torch.float32, device="cuda"))
+
+    want = []
+    ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
+    m, idx, val, out = buffers()
+    for t in range(first, first + n):
+        ctx.step(g, m, cfg.d, cfg.r, cfg.k, cfg.seed, t, idx, val, out)
+        want.append((idx.clone(), val.clone(), out.clone(), m.clone()))
+    ctx.close()
+
+    ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
+    ctx.set_option(4, 1)
+    ctx.set_device_step(first)
+    m, idx, val, out = buffers()
+    for i in range(n):
+        ctx.step(g, m, cfg.d, cfg.r, cfg.k, cfg.seed, 12345, idx, val, out)       # the argument is ignored
+        for got, ref in zip((idx, val, out, m), want[i]):
+            assert torch.equal(got.view(torch.int32), ref.view(torch.int32)), i
+    ctx.poll_status()
+
+    # the same rounds as replays of one captured call
+    m, idx, val, out = buffers()
+    ctx.set_device_step(first)
+    s = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=s):
+            ctx.step(g, m, cfg.d, cfg.r, cfg.k, cfg.seed, 0, idx, val, out)
+        for i in range(n):
+            graph.replay()
+            torch.cuda.synchronize()
+            for got, ref in zip((idx, val, out, m), want[i]):
+                assert torch.equal(got.view(torch.int32), ref.view(torch.int32)), i
+    ctx.poll_status()
+    ctx.close()
