@@ -432,6 +432,8 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
     if (late_on_side) RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero + early_bytes, 0, zbytes - early_bytes, ctx->side));
     rc = run_sampler(ctx, P, L, ctx->side);
     if (rc) return rc;
+    // the subset kernels are the only readers of the round counter: it advances right behind them
+    if (ctx->device_step) { k_step_bump<<<1, 32, 0, ctx->side>>>(ctx->d_step); ++ctx->launches; }
     const bool clear_now = clear_out && !late_on_side;
     if (clear_now) RTOPK_CUDA(ctx, cudaMemsetAsync(clear_out, 0, (size_t)d * sizeof(float), ctx->side));
     RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_join, ctx->side));
@@ -471,7 +473,7 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
     ++ctx->launches;
   }
   if (clear_late) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_cleared, 0));
-  if (ctx->device_step) { k_step_bump<<<1, 32, 0, st>>>(ctx->d_step); ++ctx->launches; }
+  if (ctx->device_step && !forked) { k_step_bump<<<1, 32, 0, st>>>(ctx->d_step); ++ctx->launches; }
   mark(ctx, RTOPK_PHASE_AGGREGATE, st);
   ctx->ev_valid[RTOPK_N_PHASES] = false;   // closed by the aggregate of a step call, if any
   RTOPK_CUDA(ctx, cudaGetLastError());
