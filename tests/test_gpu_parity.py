@@ -714,3 +714,46 @@ def test_device_round_counter_and_graph_replay_draw_fresh_subsets(lib):
                 assert torch.equal(got.view(torch.int32), ref.view(torch.int32)), i
     ctx.poll_status()
     ctx.close()
+
+
+def test_device_round_counter_in_segmented_threshold_and_limit_calls(lib):
+    # every sparsify-type call reads and advances the counter: per-tensor, threshold encoder, r = d (no
+    # selection kernel) and k = r (no subset kernels); each must match the oracle at the counter's value
+    rng = np.random.default_rng(31)
+    W, d = 2, 50021
+    g = _pad(_spiky(rng, W, d))
+    tg = torch.from_numpy(g).cuda()
+    ctx = lib.RTopK(d_max=d, W_max=W, r_max=d, k_max=600, segments_max=2)
+    ctx.set_option(4, 1)
+    ctx.set_device_step(40)
+    tm = torch.zeros(g.shape, device="cuda")
+    m_or = np.zeros_like(g)
+    out = torch.empty(wl.round_up(d, 4), dtype=torch.float32, device="cuda")
+
+    def msgs(k):
+        return (torch.zeros((W, k), dtype=torch.int32, device="cuda"), torch.zeros((W, k), dtype=torch.float32, device="cuda"))
+
+    # round 40: per-tensor
+    off, seg_r, seg_k = [0, 20003, d], [300, 500], [30, 50]
+    idx, val = msgs(80)
+    ctx.step_segmented(tg, tm, d, off, seg_r, seg_k, 9, 999, idx, val, out)
+    o_idx, o_val = oracle.sparsify_segmented(g, m_or, d, off, seg_r, seg_k, seed=9, step=40)
+    assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx) and np.array_equal(_bits(val.cpu().numpy()), _bits(o_val))
+    # round 41: threshold encoder
+    idx, val = msgs(60)
+    cnt = torch.zeros(W, dtype=torch.int32, device="cuda")
+    ones = torch.zeros(W, dtype=torch.int32, device="cuda")
+    ctx.step_threshold(tg, tm, d, 0.3, 60, 9, 999, idx, val, cnt, ones, out)
+    o_idx, o_val, o_cnt, o_ones = oracle.sparsify_threshold(g, m_or, d, 0.3, 60, 9, 41)
+    assert (o_ones > 60).all()
+    assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx) and np.array_equal(_bits(val.cpu().numpy()), _bits(o_val))
+    # round 42: r = d (random-k), round 43: k = r (top-k, draws nothing), round 44: plain again
+    for r, k, t in ((d, 100, 42), (400, 400, 43), (600, 60, 44)):
+        idx, val = msgs(k)
+        ctx.step(tg, tm, d, r, k, 9, 999, idx, val, out)
+        o_idx, o_val = oracle.sparsify(g, m_or, d, r, k, 9, t)
+        assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx), (r, k)
+        assert np.array_equal(_bits(val.cpu().numpy()), _bits(o_val)), (r, k)
+    assert np.array_equal(_bits(tm.cpu().numpy()), _bits(m_or))
+    ctx.poll_status()
+    ctx.close()
