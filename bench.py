@@ -329,12 +329,13 @@ def main():
     sampler = ClockSampler(local) if rank == 0 else None
     wall0 = time.time()
     launches0 = ctx.launch_count()
-    graphed = bool(args.graph) and world == 1
+    graphed = bool(args.graph) and world == 1 and not thr   # (the threshold call re-uploads its slice table)
     if graphed:
         from paper_2005_10761_b200.binding import OPT_DEVICE_STEP
         ctx.set_option(OPT_DEVICE_STEP, 1)
         ctx.set_device_step(t_next)
-        reps, rem = divmod(args.steps, n_batches)
+        graph_len = min(n_batches, args.steps)     # rounds held by the graph
+        reps, rem = divmod(args.steps, graph_len)
         launches_per_graph = 0
         if reps:
             try:
@@ -343,9 +344,10 @@ def main():
                 torch.cuda.synchronize()
                 l0 = ctx.launch_count()
                 with torch.cuda.graph(graph, stream=cap_stream):
-                    for b in range(n_batches):
+                    for b in range(graph_len):
                         one_step(b)
                 launches_per_graph = ctx.launch_count() - l0
+                graph.replay()             # untimed: the first launch of a graph also uploads it
                 torch.cuda.synchronize()
             except Exception as ex:        # no capture on this machine: the rounds are launched one by one
                 print(f"bench: CUDA graph capture failed ({ex!r}); launching on the stream", file=sys.stderr)
@@ -353,8 +355,8 @@ def main():
                 reps, rem, graphed = 0, args.steps, False
 
         def graph_rounds(i: int):          # called once per timed "step" index; replays at the batch boundaries
-            if i < reps * n_batches:
-                if i % n_batches == 0:
+            if i < reps * graph_len:
+                if i % graph_len == 0:
                     graph.replay()
             else:
                 one_step(i)
