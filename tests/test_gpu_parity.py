@@ -757,3 +757,42 @@ def test_device_round_counter_in_segmented_threshold_and_limit_calls(lib):
     assert np.array_equal(_bits(tm.cpu().numpy()), _bits(m_or))
     ctx.poll_status()
     ctx.close()
+
+
+def test_checkpoint_and_resume_with_a_new_context(lib):
+    # The only state of Algorithm 1's node loop is the residual and the round number: ten rounds in one go
+    # equal five rounds, a checkpoint of the residual on the host, a new context, and five more rounds.
+    cfg = wl.scaled(wl.configs()["c2"], d=250003, W=3)
+    gs = [wl.gradient(cfg, t, "cuda") for t in range(10)]
+
+    def run(ctx, m, t0, t1, keep):
+        idx = torch.zeros((cfg.W, cfg.k), dtype=torch.int32, device="cuda")
+        val = torch.zeros((cfg.W, cfg.k), dtype=torch.float32, device="cuda")
+        out = torch.zeros(wl.round_up(cfg.d, 4), dtype=torch.float32, device="cuda")
+        for t in range(t0, t1):
+            ctx.step(gs[t], m, cfg.d, cfg.r, cfg.k, cfg.seed, t, idx, val, out)
+            keep.append((idx.cpu().clone(), val.cpu().clone(), out.cpu().clone()))
+        ctx.poll_status()
+
+    straight, resumed = [], []
+    ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
+    ctx.set_option(2, 1)                                  # threshold reuse: its history is not part of the state
+    m = wl.zero_residual(cfg, "cuda")
+    run(ctx, m, 0, 10, straight)
+    m_straight = m.cpu().clone()
+    ctx.close()
+
+    ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
+    ctx.set_option(2, 1)
+    m = wl.zero_residual(cfg, "cuda")
+    run(ctx, m, 0, 5, resumed)
+    checkpoint = m.cpu().clone()
+    ctx.close()
+    del m
+    ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)           # a fresh context and a fresh residual buffer
+    m = checkpoint.cuda()
+    run(ctx, m, 5, 10, resumed)
+    for a, b in zip(straight, resumed):
+        for x, y in zip(a, b):
+            assert torch.equal(x.view(torch.int32), y.view(torch.int32))
+    assert torch.equal(m.cpu().view(torch.int32), m_straight.view(torch.int32))
