@@ -733,13 +733,13 @@ def test_device_round_counter_in_segmented_threshold_and_limit_calls(lib):
     def msgs(k):
         return (torch.zeros((W, k), dtype=torch.int32, device="cuda"), torch.zeros((W, k), dtype=torch.float32, device="cuda"))
 
-    # round 40: per-tensor
+    # t = 40: per-tensor
     off, seg_r, seg_k = [0, 20003, d], [300, 500], [30, 50]
     idx, val = msgs(80)
     ctx.step_segmented(tg, tm, d, off, seg_r, seg_k, 9, 999, idx, val, out)
     o_idx, o_val = oracle.sparsify_segmented(g, m_or, d, off, seg_r, seg_k, seed=9, step=40)
     assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx) and np.array_equal(_bits(val.cpu().numpy()), _bits(o_val))
-    # round 41: threshold encoder
+    # t = 41: threshold encoder
     idx, val = msgs(60)
     cnt = torch.zeros(W, dtype=torch.int32, device="cuda")
     ones = torch.zeros(W, dtype=torch.int32, device="cuda")
@@ -747,7 +747,7 @@ def test_device_round_counter_in_segmented_threshold_and_limit_calls(lib):
     o_idx, o_val, o_cnt, o_ones = oracle.sparsify_threshold(g, m_or, d, 0.3, 60, 9, 41)
     assert (o_ones > 60).all()
     assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx) and np.array_equal(_bits(val.cpu().numpy()), _bits(o_val))
-    # round 42: r = d (random-k), round 43: k = r (top-k, draws nothing), round 44: plain again
+    # t = 42: r = d (random-k), t = 43: k = r (top-k, draws nothing), t = 44: plain again
     for r, k, t in ((d, 100, 42), (400, 400, 43), (600, 60, 44)):
         idx, val = msgs(k)
         ctx.step(tg, tm, d, r, k, 9, 999, idx, val, out)
