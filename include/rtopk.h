@@ -73,10 +73,11 @@ enum {
   RTOPK_OPT_PROFILE = 1,     /* 1 = record CUDA events between the phases of each call on the
                                 caller's stream (read with rtopk_get_phase_times); 0 = off */
   RTOPK_OPT_REUSE_THRESHOLD = 2, /* 1 = consecutive calls of one shape on one residual buffer predict the
-                                first threshold from the exact thresholds of the last calls instead
-                                of sampling (a = g + m drifts slowly from round to round); a
-                                prediction that misses is repaired by the exact path and the next
-                                call samples again.  Results never depend on it.  0 = off (default) */
+                                first threshold from the exact thresholds of the last two calls instead
+                                of sampling, once those two are within 25 % of each other (a = g + m
+                                drifts slowly from round to round); a prediction that misses is
+                                repaired by the exact path and the next two calls sample again.
+                                Results never depend on it.  0 = off (default) */
   RTOPK_OPT_THRESHOLD_SIGNS = 3, /* what rtopk_sparsify_threshold sends for a kept coordinate: 0 (default) its
                                 value a_i; 1 = sign(a_i) * M with M = 2 theta, the quantised observation of
                                 Section II (after the pre-processing step a coordinate is 0 or +-M, so one bit

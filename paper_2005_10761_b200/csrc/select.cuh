@@ -165,23 +165,28 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(Launch L) {
     return;
   }
   if (L.reuse) {
-    // Step-to-step reuse: a = g + m changes slowly from one round to the next, so the last exact
-    // thresholds predict this one (geometric extrapolation of the last two); the bracket is the
-    // prediction widened by a few times the error the predictions have shown so far.  A bracket
-    // that misses is repaired by the exact path and makes the next call sample again.
+    // Step-to-step reuse: a = g + m changes slowly from one round to the next, so the last two exact
+    // thresholds predict this one.  Only a smooth history is trusted (two thresholds within 25 % of
+    // each other: while a fresh residual builds up the threshold still jumps, and sampling costs far
+    // less than a miss); a ratio beyond 5 % is damped to its square root, because a threshold that
+    // moves that fast is slowing down, and a prediction that is too low only adds candidates whereas
+    // one that is too high misses.  The bracket is the prediction widened by a few times the error
+    // the predictions have shown so far.  A bracket that misses is repaired by the exact path and
+    // makes the next two calls sample again.
     const TauHistory h = L.s.history[sl];                       // the same for every thread
-    if (h.valid >= 1 && h.tau1 > 0x00800000u && h.tau1 < 0x7E800000u) {
+    if (h.valid >= 2 && h.tau1 > 0x00800000u && h.tau1 < 0x7E800000u && h.tau2 > 0x00800000u && h.tau2 < 0x7E800000u) {
       const float t1 = __uint_as_float(h.tau1);
-      float ratio = 1.0f;
-      if (h.valid >= 2 && h.tau2 > 0x00800000u && h.tau2 < 0x7E800000u)
-        ratio = fminf(fmaxf(t1 / __uint_as_float(h.tau2), 0.5f), 2.0f);
-      const float p = t1 * ratio;
-      const float delta = fminf(fmaxf(3.0f * h.err + 0.01f, 0.02f), 0.15f);
-      st.tau_lo = mag_key(p * (1.0f - delta));
-      st.tau_hi = max(mag_key(p * (1.0f + delta)), st.tau_lo);
-      st.pred = mag_key(p);
-      if (tid == 0) L.s.state[sl] = st;
-      return;
+      float ratio = t1 / __uint_as_float(h.tau2);
+      if (ratio >= 0.8f && ratio <= 1.25f) {
+        if (ratio < 0.95f || ratio > 1.05f) ratio = sqrtf(ratio);
+        const float p = t1 * ratio;
+        const float delta = fminf(fmaxf(3.0f * h.err + 0.01f, 0.02f), 0.15f);
+        st.tau_lo = mag_key(p * (1.0f - delta));
+        st.tau_hi = max(mag_key(p * (1.0f + delta)), st.tau_lo);
+        st.pred = mag_key(p);
+        if (tid == 0) L.s.state[sl] = st;
+        return;
+      }
     }
   }
   const float* m = L.residual;
