@@ -75,8 +75,8 @@ struct rtopk_ctx {
   int sms = 0;
   uint64_t launches = 0;                          // kernels launched by this context so far
   int finish_max_clusters[kMaxCluster + 1] = {};  // [cs]: co-resident k_finish clusters of size cs (1..16)
-  int stream_blocks[2] = {0, 0};
-  int exact_blocks = 0;               // cooperative grid of k_exact (all blocks resident)      // persistent grid of k_stream per gradient dtype
+  int stream_blocks[2] = {0, 0};      // persistent grid of k_stream per gradient dtype
+  int exact_blocks = 0;               // cooperative grid of k_exact (all blocks resident)
   // work that does not depend on the data (the k-of-r subset, clearing the dense update) runs on a
   // side stream next to the streaming pass
   cudaStream_t side = nullptr;
@@ -304,12 +304,9 @@ int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t s
       mark(ctx, RTOPK_PHASE_ORDER, st);
     }
     mark(ctx, RTOPK_PHASE_EXACT, st);
-    // the exact path's histograms and look-back words are cleared on the side stream
+    // k_finish needs the subset (side stream); a slice whose bracket missed is selected exactly inside
+    // its k_finish cluster, so no kernel of the exact path is launched here
     if (join) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, join, 0));
-    if (P.any_select) {
-      rc = launch_exact(ctx, P, L, 0, st);
-      if (rc) return rc;
-    }
   } else {
     mark(ctx, RTOPK_PHASE_THRESHOLD, st);
     k_init_state<<<(n + 127) / 128, 128, 0, st>>>(L, 1u);

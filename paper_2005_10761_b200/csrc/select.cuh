@@ -589,6 +589,101 @@ __device__ __forceinline__ void async_copy_4(void* smem_dst, const void* gmem_sr
 // ... and the wait for all such copies of the calling thread.
 __device__ __forceinline__ void async_copy_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 
+// The exact path inside the finishing cluster, for a slice whose first bracket missed (too few
+// candidates gathered, or more than the list holds).  This is rare -- a sampled bracket misses about
+// once in 10^5 slices, a predicted one after an abrupt change of the data -- so it is written for
+// clarity, not speed: three radix passes over the slice's a = g + m (already materialised in the
+// residual buffer by the streaming pass), each CTA histogramming its range of chunks and all CTAs
+// summing the histograms through distributed shared memory, give the r-th largest key tau, the count
+// n_gt of larger keys and the quota of keys equal to tau; an ordered sweep then writes exactly the
+// top-r set (keys above tau, and the first `quota` keys equal to it) into the candidate list in index
+// order.  Called by every thread of every CTA of the cluster; returns false (to all of them) if the
+// slice holds fewer than r keys, which cannot happen for a valid slice.
+template <typename Cluster>
+__device__ __forceinline__ bool cluster_exact_collect(const Launch& L, const Slice& S, Cluster& cluster, FinishSmem& sm,
+                                                      uint32_t CS, uint32_t q, uint32_t& tau_out, uint32_t& n_gt_out,
+                                                      uint32_t& quota_out) {
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t nchunks = slice_chunks(S);
+  const uint32_t cpc = (nchunks + CS - 1) / CS;                       // chunks per CTA
+  const uint32_t span = S.head + S.len;
+  const uint32_t e_lo = max(S.head, min(span, q * cpc * (uint32_t)kChunk));
+  const uint32_t e_hi = max(e_lo, min(span, (q + 1u) * cpc * (uint32_t)kChunk));
+  const float* a = L.residual + (S.m_off - S.head);                   // element e of the slice's grid
+  uint32_t prefix = 0, need = S.r, n_gt = 0;
+  for (int pass = 0; pass < 3; ++pass) {
+    const int bits = digit_bits(pass), shift = digit_shift(pass);
+    for (uint32_t b = tid; b < (uint32_t)kBins; b += kFinishThreads) sm.hist[b] = 0;
+    __syncthreads();
+    for (uint32_t e = e_lo + tid; e < e_hi; e += kFinishThreads) {
+      const uint32_t key = mag_key(a[e]);
+      if (pass == 0 || (key >> (shift + bits)) == prefix) atomicAdd(&sm.hist[(key >> shift) & ((1u << bits) - 1u)], 1u);
+    }
+    cluster.sync();
+    for (uint32_t b = tid; b < (uint32_t)kBins; b += kFinishThreads) {
+      uint32_t sum = 0;
+      for (uint32_t rr = 0; rr < CS; ++rr) sum += cluster.map_shared_rank(sm.hist, rr)[b];
+      sm.red[b] = sum;
+    }
+    __syncthreads();
+    uint32_t D, above;
+    const bool ok = pick_digit(sm.red, 1 << bits, need, sm.scratch, D, above);
+    cluster.sync();                                                    // all remote reads of sm.hist are done
+    if (!ok) return false;                                             // the same in every CTA
+    n_gt += above; need -= above;
+    prefix = (prefix << bits) | D;
+  }
+  const uint32_t tau = prefix, quota = need;
+  // members of my range: keys above tau (A) and keys equal to tau (B)
+  uint32_t cA = 0, cB = 0;
+  for (uint32_t e = e_lo + tid; e < e_hi; e += kFinishThreads) {
+    const uint32_t key = mag_key(a[e]);
+    cA += key > tau; cB += key == tau;
+  }
+  cA = warp_sum(cA); cB = warp_sum(cB);
+  if (lane == 0) { sm.warpA[warp] = cA; sm.warpB[warp] = cB; }
+  __syncthreads();
+  if (tid < CS) {
+    uint32_t tA = 0, tB = 0;
+    for (int w = 0; w < kFinishWarps; ++w) { tA += sm.warpA[w]; tB += sm.warpB[w]; }
+    uint32_t* c = cluster.map_shared_rank(sm.counts, tid);             // my counts, into CTA `tid`
+    c[2 * q] = tA; c[2 * q + 1] = tB;
+  }
+  cluster.sync();
+  uint32_t runA = 0, runB = 0;                                         // members before my range
+  for (uint32_t p = 0; p < q; ++p) { runA += sm.counts[2 * p]; runB += sm.counts[2 * p + 1]; }
+  // ordered sweep, 1024 consecutive elements at a time
+  uint32_t* cidx = L.s.cand_idx + S.cand_off;
+  float* cval = L.s.cand_val + S.cand_off;
+  for (uint32_t base = e_lo; base < e_hi; base += kFinishThreads) {
+    const uint32_t e = base + tid;
+    const bool in = e < e_hi;
+    const float v = in ? a[e] : 0.f;
+    const uint32_t key = mag_key(v);
+    const bool isA = in && key > tau, isB = in && key == tau;
+    const uint32_t mA = __ballot_sync(0xFFFFFFFFu, isA), mB = __ballot_sync(0xFFFFFFFFu, isB);
+    __syncthreads();                                                   // the previous tile's warp totals are consumed
+    if (lane == 0) { sm.warpA[warp] = __popc(mA); sm.warpB[warp] = __popc(mB); }
+    __syncthreads();
+    uint32_t gA = runA + __popc(mA & ((1u << lane) - 1u)), gB = runB + __popc(mB & ((1u << lane) - 1u));
+    uint32_t tA = 0, tB = 0;
+    for (uint32_t w = 0; w < (uint32_t)kFinishWarps; ++w) {
+      const uint32_t wa = sm.warpA[w], wb = sm.warpB[w];
+      if (w < warp) { gA += wa; gB += wb; }
+      tA += wa; tB += wb;
+    }
+    if (isA || (isB && gB < quota)) {
+      const uint32_t pos = gA + min(gB, quota);
+      if (pos < S.cand_cap) { cidx[pos] = e - S.head; cval[pos] = v; }
+    }
+    runA += tA; runB += tB;
+  }
+  __threadfence();
+  cluster.sync();                                                      // the whole list is written and visible
+  tau_out = tau; n_gt_out = n_gt; quota_out = quota;
+  return true;
+}
+
 __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
   namespace cg = cooperative_groups;
   extern __shared__ __align__(16) unsigned char finish_raw[];
@@ -603,16 +698,26 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
   SelState* st = &L.s.state[sl];
   // every early exit below depends on the slice only, so a cluster leaves as a whole
   if (S.r == S.len) return;
-  const bool general = (st->flags & FLAG_GENERAL) != 0;         // the list was built by the exact path
-  const uint32_t n_cand = general ? st->n_cand : L.s.cursor[sl];
+  bool general = (st->flags & FLAG_GENERAL) != 0;               // the list was built by the exact path
+  uint32_t n_cand = general ? st->n_cand : L.s.cursor[sl];
   if (st->resolved > 31) return;                               // an earlier pass already failed
-  if (n_cand < S.r || n_cand > S.cand_cap) {                   // cannot happen once the exact path ran
-    if (q == 0 && tid == 0) atomicOr(L.s.error, ERR_CANDIDATE_OVERFLOW);
-    return;
-  }
   uint32_t n_gt = st->n_gt, need = st->need, lo_key, hi_key;
   bool count_above;
-  if (general) {
+  if (n_cand < S.r || n_cand > S.cand_cap) {
+    // the first bracket missed (and no exact pass has repaired it): select exactly, here
+    if (general) {                                             // cannot happen after an exact pass
+      if (q == 0 && tid == 0) atomicOr(L.s.error, ERR_CANDIDATE_OVERFLOW);
+      return;
+    }
+    uint32_t tau_x, gt_x, quota_x;
+    if (!cluster_exact_collect(L, S, cluster, sm, CS, q, tau_x, gt_x, quota_x)) {
+      if (q == 0 && tid == 0) { atomicOr(L.s.error, ERR_SELECT_INCONSISTENT); st->resolved = 32; }
+      return;
+    }
+    if (q == 0 && tid == 0) { st->flags |= FLAG_GENERAL | FLAG_FELL_BACK; st->n_cand_first = n_cand; st->n_cand = S.r; }
+    general = true; n_cand = S.r;
+    n_gt = gt_x; need = quota_x; lo_key = tau_x; hi_key = tau_x + 1u; count_above = false;
+  } else if (general) {
     const uint32_t free_bits = 31u - st->resolved;
     lo_key = st->prefix << free_bits; hi_key = lo_key + (1u << free_bits); count_above = false;
   } else {
