@@ -796,3 +796,39 @@ def test_checkpoint_and_resume_with_a_new_context(lib):
         for x, y in zip(a, b):
             assert torch.equal(x.view(torch.int32), y.view(torch.int32))
     assert torch.equal(m.cpu().view(torch.int32), m_straight.view(torch.int32))
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_exact_selection_inside_the_finishing_cluster(lib, bf16):
+    # Every slice is made to miss its first bracket (threshold reuse, then a collapse of the magnitudes), with
+    # many workers (small clusters), long rows (several CTAs and chunks per slice) and values quantised to a
+    # few levels, so that ties straddle the r-th largest magnitude and the tie quota decides.
+    from paper_2005_10761_b200.binding import OPT_REUSE_THRESHOLD
+    rng = np.random.default_rng(77)
+    W, d, r, k = 12, 150001, 3000, 300
+    ctx = _ctx(lib, d, W, r, k)
+    ctx.set_option(OPT_REUSE_THRESHOLD, 1)
+    tm = torch.zeros((W, wl.round_up(d, 8)), dtype=torch.float32, device="cuda")
+    m_or = np.zeros((W, wl.round_up(d, 8)), dtype=np.float32)
+    idx = torch.zeros((W, k), dtype=torch.int32, device="cuda")
+    val = torch.zeros((W, k), dtype=torch.float32, device="cuda")
+    fell = []
+    for t in range(8):
+        g = _pad(_spiky(rng, W, d, p=0.05))
+        if t >= 5:
+            g = (np.round(g * 4) / 4).astype(np.float32) * (1e-3 if t == 5 else 1.0)   # few levels; t = 5 collapses
+            g = g - (m_or if t == 5 else 0)
+        tg = torch.from_numpy(g).cuda()
+        g_or = g
+        if bf16:
+            tg = tg.to(torch.bfloat16)
+            g_or = tg.view(torch.int16).cpu().numpy().view(np.uint16).copy()
+        ctx.sparsify(tg, tm, d, r, k, 5, t, idx, val)
+        ctx.poll_status()
+        o_idx, o_val = oracle.sparsify(g_or, m_or, d, r, k, 5, t)
+        assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx), t
+        assert np.array_equal(_bits(val.cpu().numpy()), _bits(o_val)), t
+        assert np.array_equal(_bits(tm.cpu().numpy()), _bits(m_or)), t
+        fell.append(sum(ctx.stats(w)["used_fallback"] for w in range(W)))
+    assert max(fell) == W                      # in some round every slice took the exact path
+    ctx.close()
