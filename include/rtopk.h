@@ -98,8 +98,9 @@ enum {
   RTOPK_PHASE_THRESHOLD = 1, /* sampled bracket of the r-th largest magnitude */
   RTOPK_PHASE_STREAM = 2,    /* the one kernel over W x d elements: add, write-back, candidate gathering */
   RTOPK_PHASE_ORDER = 3,     /* candidate runs laid out in index order; count check */
-  RTOPK_PHASE_EXACT = 4,     /* full-vector radix passes (fallback; near-empty launches otherwise) */
-  RTOPK_PHASE_FINISH = 5,    /* exact threshold among the candidates, messages, residual zeroing */
+  RTOPK_PHASE_EXACT = 4,     /* full-vector radix passes (RTOPK_OPT_SELECT_PATH = 1 only; empty otherwise) */
+  RTOPK_PHASE_FINISH = 5,    /* exact threshold among the candidates (over the whole slice where the first
+                                threshold missed), messages, residual zeroing */
   RTOPK_PHASE_AGGREGATE = 6, /* master average (step calls only) */
   RTOPK_N_PHASES = 7
 };

@@ -4,14 +4,16 @@
 //   k_sample        brackets the r-th largest key of every slice from a strided sample of a = g + m
 //                   (or, with threshold reuse, from the slice's last exact thresholds) and clears
 //                   the counters of the streaming pass (k_stream, stream.cuh)
-//   k_exact         the exact path, one cooperative launch: three radix histogram passes over the
-//                   full vector (hist_body) and an index-ordered collect (collect_body, ballot-free
-//                   prefix compaction + bounded look-back); runs only for slices whose bracket
-//                   missed, or as the main path behind k_hist (fused add in pass 0)
+//   k_exact         the exact path over the full vector, one cooperative launch: three radix histogram
+//                   passes (hist_body) and an index-ordered collect (collect_body, ballot-free
+//                   prefix compaction + bounded look-back); the main path behind k_hist (fused add in
+//                   pass 0) when the caller asks for it
 //   k_finish        one cluster per slice: candidate runs -> index order, exact r-th largest key
 //                   among the candidates, then a walk over the candidates in index order that
 //                   numbers the members of the top-r set and writes the ones the k-of-r sampler
-//                   chose as (index, value) messages, zeroing their residual slots (m' = a - ghat)
+//                   chose as (index, value) messages, zeroing their residual slots (m' = a - ghat);
+//                   a slice whose bracket missed is first selected exactly over all of its a = g + m
+//                   inside the cluster (cluster_exact_collect)
 //   k_emit_all      r = d (Definition 2): positions are indices, no selection
 #pragma once
 
