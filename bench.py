@@ -5,16 +5,20 @@ A step = rtopk_step over one batch: for W workers, a = g + m, top-r, random k-of
 residual update, then the master's average into a dense vector.  Inputs are synthetic (see
 paper_2005_10761_b200/workloads.py); the residual is carried from step to step.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3_f32] [--impl ours|reference]
 
 Prints one JSON line.  `value` is GB/s of gradient input (W*d*sizeof(g) per step over the device
-time of a step, inputs resident in HBM); `e2e` is the same through rtopk_step_host with pinned host
-buffers (host<->device copies inside the timed region); `roofline` is the fused streaming kernel's
-algorithmic bytes over its own event-timed duration against the measured HBM copy bandwidth;
-`cpu_baseline` is the CPU oracle timed on a bounded sample of the same workload.
-On one GPU the timed rounds are replays of a CUDA graph that holds one round per resident gradient
-batch (`--graph 0` launches them on the stream instead); the kernels and their work are the same, the
-round number that enters the Philox counter lives in a device word that every round advances.
+time of a step, inputs resident in HBM); the timed region of K steps is repeated (`repeats`) and
+`ms_per_step` is the median over the repeats, `ms_per_step_min` the fastest; `e2e` is the same
+metric through rtopk_step_host with pinned host buffers (host<->device copies inside the timed
+region); `roofline` is the dominant kernel's algorithmic bytes over its own event-timed duration
+against the measured HBM copy bandwidth; `cpu_baseline` is the CPU oracle timed on a bounded sample
+of the same workload; `sweep` holds short runs of the other configurations (the metric is defined
+"vs d, W, r, k").  On one GPU the timed rounds are replays of a CUDA graph that holds one round per
+resident gradient batch (`--graph 0` launches them on the stream instead); the kernels and their
+work are the same, the round number that enters the Philox counter lives in a device word that every
+round advances.  With --gpus N > 1 and no launcher in the environment the script starts N ranks
+itself (one per GPU, NCCL).
 """
 from __future__ import annotations
 
@@ -23,6 +27,7 @@ import dataclasses
 import hashlib
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -34,7 +39,10 @@ sys.path.insert(0, ROOT)
 
 METRIC = "rtopk_step_gradient_input_bandwidth"
 UNIT = "GB/s"
-KERNEL_SOURCES = ["common.cuh", "element.cuh", "stream.cuh"]   # everything k_stream is compiled from
+NOMINAL_HBM_GBS = 8000.0
+# everything the dominant kernel is compiled from (a change voids the recorded DRAM traffic)
+KERNEL_SOURCES = ["common.cuh", "element.cuh", "stream.cuh"]
+L2_BYTES = 126 * 1024 * 1024
 
 
 def load_peak():
@@ -54,7 +62,7 @@ def kernel_source_hash() -> str:
     return h.hexdigest()[:16]
 
 
-def recorded_traffic(workload: str, launch_bytes: float):
+def recorded_traffic(launch_bytes: float):
     """DRAM bytes per launch of the streaming kernel from the committed ncu summary, scaled by the
     algorithmic bytes when the capture was taken on a smaller case; None if there is no summary or
     the kernel sources changed since."""
@@ -133,6 +141,27 @@ def pick_workload(name: str, scale_d: int = 0, workers: int = 0):
     return cfg
 
 
+def resident_batches(cfg, steps: int, warmup: int) -> int:
+    gsz = 4 if cfg.grad_dtype == "f32" else 2
+    return max(1, min(cfg.steps, int(24e9 // (cfg.W * cfg.ld * gsz)), steps + warmup))
+
+
+def config_dict(cfg, args, world: int) -> dict:
+    """What both arms (ours and --impl reference) print as `config`: the workload and how it is run."""
+    seg = cfg.seg_off is not None
+    return {"workload": cfg.name, "d": cfg.d, "W_per_gpu": cfg.W, "W_total": cfg.W * world, "r": cfg.r,
+            "k": cfg.k_total, "grad_dtype": cfg.grad_dtype, "recipe": cfg.recipe,
+            "segments": len(cfg.seg_r) if seg else 1,
+            "gradient_batches_resident": resident_batches(cfg, args.steps, args.warmup),
+            "residual": "carried across steps", "l2": "inputs larger than L2 (no flush)",
+            "parallelism": f"workers sharded x{world}",
+            "variant": ("rtopk_step_apply (fused master update)" if args.apply else
+                        f"rtopk_step_threshold (theta = {args.threshold})" if args.threshold is not None
+                        else "rtopk_step"),
+            "select_path": args.select_path, "reuse_threshold": bool(args.reuse_threshold)}
+
+
+# ------------------------------------------------------------------------------------ CPU oracle legs
 def oracle_sample(cfg, rows: int):
     """Host inputs of the bounded CPU-baseline sample: `rows` workers of step 0, zero residual."""
     import numpy as np
@@ -181,20 +210,293 @@ def run_reference(args):
     cores = os.cpu_count() or 1
     rows = cpu_sample_rows(cfg, cores)
     threads = min(cores, rows)
-    sec = time_oracle(cfg, rows, threads, steps=args.steps, warmup=args.warmup)
+    # every step is one bounded sample; the whole run stays within a few minutes
+    per_step = max(0.05, cfg.d * 1.3e-7) * ((rows + threads - 1) // threads) * 1.3
+    steps = max(1, min(args.steps, int(120.0 / per_step)))
+    warmup = min(args.warmup, max(0, int(30.0 / per_step)))
+    sec = time_oracle(cfg, rows, threads, steps=steps, warmup=warmup)
     gsz = 4 if cfg.grad_dtype == "f32" else 2
     value = rows * cfg.d * gsz / sec / 1e9
-    sample = f"{rows} of {cfg.W} worker rows per step, step-0 gradient, residual carried"
+    sample = (f"{rows} of {cfg.W} worker rows per step, step-0 gradient, residual carried; "
+              f"{steps} timed steps after {warmup} warm-up steps (bounded to a few minutes of CPU work)")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": cfg.name, "d": cfg.d, "W": rows, "r": cfg.r, "k": cfg.k_total,
-                   "grad_dtype": cfg.grad_dtype},
+        "config": config_dict(cfg, args, max(1, args.gpus)),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
+
+
+# ------------------------------------------------------------------------------------ the GPU arm
+class Round:
+    """Buffers and the step call of one workload on this rank's GPU."""
+
+    def __init__(self, cfg, args, dev, world=1, rank=0, grads=None, n_batches=None):
+        import torch
+        import paper_2005_10761_b200 as rt
+        from paper_2005_10761_b200 import workloads as wl
+        from paper_2005_10761_b200 import binding as B
+        self.cfg, self.args, self.dev, self.world, self.rank = cfg, args, dev, world, rank
+        self.W, self.d, self.ld = cfg.W, cfg.d, cfg.ld
+        self.W_total = cfg.W * world
+        self.gsz = 4 if cfg.grad_dtype == "f32" else 2
+        self.K = cfg.k_total
+        self.seg = cfg.seg_off is not None
+        self.thr = args.threshold is not None
+        self.ctx = rt.RTopK(d_max=self.d, W_max=self.W_total, r_max=min(self.d, 4 * cfg.r) if self.thr else cfg.r,
+                            k_max=self.K, segments_max=len(cfg.seg_r) if self.seg else 1, device=dev.index)
+        if args.reuse_threshold and args.select_path == "sampled":
+            self.ctx.set_option(B.OPT_REUSE_THRESHOLD, 1)
+        if args.select_path == "exact":
+            self.ctx.set_option(B.OPT_SELECT_PATH, 1)
+        if grads is None:
+            n_batches = n_batches or resident_batches(cfg, args.steps, args.warmup)
+            shard_cfg = cfg if world == 1 else dataclasses.replace(cfg, W=self.W_total)
+            rows = range(rank * self.W, rank * self.W + self.W)
+            grads = [wl.gradient(shard_cfg, t, dev, workers=rows) for t in range(n_batches)]
+        self.grads = grads
+        self.n_batches = len(grads)
+        self.residual = wl.zero_residual(cfg, dev)
+        self.idx = torch.zeros((self.W, self.K), dtype=torch.int32, device=dev)
+        self.val = torch.zeros((self.W, self.K), dtype=torch.float32, device=dev)
+        # the dense update; with --apply the model weights that the update is applied to
+        self.out = torch.zeros(wl.round_up(self.d, 4), dtype=torch.float32, device=dev)
+        self.cnt = torch.zeros(self.W, dtype=torch.int32, device=dev)
+        self.ones = torch.zeros(self.W, dtype=torch.int32, device=dev)
+        self.t_next = 0
+
+    @property
+    def n_slices(self):
+        return self.W * (len(self.cfg.seg_r) if self.seg else 1)
+
+    def step(self, t: int):
+        cfg, ctx, args = self.cfg, self.ctx, self.args
+        g = self.grads[t % self.n_batches]
+        if self.world == 1:
+            if self.seg:
+                ctx.step_segmented(g, self.residual, self.d, cfg.seg_off, cfg.seg_r, cfg.seg_k, cfg.seed, t,
+                                   self.idx, self.val, self.out)
+            elif self.thr:
+                ctx.step_threshold(g, self.residual, self.d, args.threshold, cfg.k, cfg.seed, t, self.idx, self.val,
+                                   self.cnt, self.ones, self.out)
+            elif args.apply:
+                ctx.step_apply(g, self.residual, self.d, cfg.r, cfg.k, cfg.seed, t, 0.01, self.idx, self.val, self.out)
+            else:
+                ctx.step(g, self.residual, self.d, cfg.r, cfg.k, cfg.seed, t, self.idx, self.val, self.out)
+        else:
+            from paper_2005_10761_b200 import sharded
+
+            def sp(gl, ml, wb):
+                if self.seg:
+                    ctx.sparsify_segmented(gl, ml, self.d, cfg.seg_off, cfg.seg_r, cfg.seg_k, cfg.seed, t, self.idx,
+                                           self.val, worker_base=wb)
+                else:
+                    ctx.sparsify(gl, ml, self.d, cfg.r, cfg.k, cfg.seed, t, self.idx, self.val, worker_base=wb)
+                return self.idx, self.val
+
+            def ag(ia, va):
+                ctx.aggregate(ia, va, self.d, self.out)
+                return self.out
+            sharded.sharded_round(sp, ag, g, self.residual, self.W_total, self.world, self.rank)
+
+    def sync_all(self):
+        import torch
+        torch.cuda.synchronize()
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(self, fn, t_first: int, n: int) -> float:
+        """Device time in ms of n consecutive steps (max over ranks)."""
+        import torch
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        self.sync_all()
+        e0.record()
+        for t in range(t_first, t_first + n):
+            fn(t)
+        e1.record()
+        self.sync_all()
+        ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=self.dev)
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item())
+
+    def measure(self, steps: int, warmup: int, repeats: int, graph: bool):
+        """Warm-up, then `repeats` timed regions of `steps` steps each.  Returns (ms per step of each
+        region, kernels launched per region, launch mode)."""
+        import torch
+        from paper_2005_10761_b200 import binding as B
+        ctx = self.ctx
+        for _ in range(warmup):
+            self.step(self.t_next); self.t_next += 1
+        self.sync_all()
+        graphed = graph and self.world == 1 and not self.thr   # (the threshold call re-uploads its slice table)
+        per_region, launches = [], 0
+        if graphed:
+            ctx.set_option(B.OPT_DEVICE_STEP, 1)
+            ctx.set_device_step(self.t_next)
+            graph_len = min(self.n_batches, steps)     # rounds held by the graph
+            reps, rem = divmod(steps, graph_len)
+            launches_per_graph = 0
+            try:
+                cap_stream = torch.cuda.Stream()
+                g = torch.cuda.CUDAGraph()
+                torch.cuda.synchronize()
+                l0 = ctx.launch_count()
+                with torch.cuda.graph(g, stream=cap_stream):
+                    for b in range(graph_len):
+                        self.step(b)
+                launches_per_graph = ctx.launch_count() - l0
+                g.replay()                 # untimed: the first launch of a graph also uploads it
+                torch.cuda.synchronize()
+            except Exception as ex:        # no capture on this box: the rounds are launched one by one
+                print(f"bench: CUDA graph capture failed ({ex!r}); launching on the stream", file=sys.stderr)
+                torch.cuda.synchronize()
+                graphed = False
+                ctx.set_option(B.OPT_DEVICE_STEP, 0)
+        if graphed:
+            def graph_rounds(i: int):      # called once per timed step index; replays at the batch boundaries
+                if i < reps * graph_len:
+                    if i % graph_len == 0:
+                        g.replay()
+                else:
+                    self.step(i)
+            for _ in range(repeats):
+                l0 = ctx.launch_count()
+                per_region.append(self.timed(graph_rounds, 0, steps) / steps)
+                launches = ctx.launch_count() - l0 + reps * launches_per_graph
+            ctx.set_option(B.OPT_DEVICE_STEP, 0)
+            self.t_next += steps * repeats + graph_len
+        else:
+            for _ in range(repeats):
+                l0 = ctx.launch_count()
+                per_region.append(self.timed(self.step, self.t_next, steps) / steps)
+                launches = ctx.launch_count() - l0
+                self.t_next += steps
+        ctx.poll_status()
+        return per_region, launches, ("cuda graph replay" if graphed else "stream launches")
+
+    def profile_phases(self, n: int):
+        """Phase durations (events between the phases of a call), averaged over n more steps, plus how many
+        slices fell back to the exact selection and how many brackets were predicted."""
+        from paper_2005_10761_b200 import binding as B
+        ctx = self.ctx
+        ctx.set_option(B.OPT_PROFILE, 1)
+        phase_sum, fallbacks, predicted = {}, 0, 0
+        for _ in range(n):
+            self.step(self.t_next); self.t_next += 1
+            for name, ms in ctx.phase_times().items():
+                if ms >= 0:
+                    phase_sum[name] = phase_sum.get(name, 0.0) + ms
+            stats = [ctx.stats(s) for s in range(self.n_slices)]
+            fallbacks += sum(s["used_fallback"] for s in stats)
+            predicted += sum(s["bracket_predicted"] for s in stats)
+        ctx.set_option(B.OPT_PROFILE, 0)
+        return {k: v / n for k, v in phase_sum.items()}, fallbacks, predicted
+
+    def step_bytes(self) -> int:
+        """Algorithmic bytes of one step: g and m read, m' written, the dense update, messages written and read."""
+        upd = 8 * self.W * self.K if self.args.apply else 4 * self.d   # --apply touches only the sent coordinates
+        return self.W * self.d * (self.gsz + 8) + upd + 16 * self.W * self.K
+
+    def stream_bytes(self) -> int:
+        return self.W * self.d * (self.gsz + 8)
+
+    def close(self):
+        self.ctx.close()
+
+
+def sweep_point(name, args, dev, peak, grads=None, steps=10, warmup=5, repeats=3, select_path=None, cold_l2=False):
+    """One short run of another configuration: the metric "vs d, W, r, k"."""
+    import torch
+    cfg = pick_workload(name)
+    a = argparse.Namespace(**vars(args))
+    a.apply, a.threshold = False, None
+    a.select_path = select_path or "sampled"
+    a.steps, a.warmup = steps, warmup
+    try:
+        rd = Round(cfg, a, dev, grads=grads)
+    except Exception as ex:
+        return {"workload": name, "skipped": repr(ex)[:160]}
+    try:
+        regions, _, mode = rd.measure(steps, warmup, repeats, bool(args.graph))
+        phases, fallbacks, _ = rd.profile_phases(5)
+        ms = statistics.median(regions)
+        e = {"workload": name, "d": cfg.d, "W": cfg.W, "r": cfg.r, "k": cfg.k_total, "dtype": cfg.grad_dtype,
+             "select_path": a.select_path, "ms_per_step": ms, "ms_per_step_min": min(regions),
+             "gbs_gradient_in": cfg.W * cfg.d * rd.gsz / (ms * 1e-3) / 1e9,
+             "step_roofline_frac": rd.step_bytes() / (ms * 1e-3) / 1e9 / peak,
+             "kstream_frac": (rd.stream_bytes() / (phases["stream"] * 1e-3) / 1e9 / peak) if phases.get("stream") else None,
+             "phases_ms": {k: round(v, 4) for k, v in phases.items()}, "fallback_slices": fallbacks, "launch": mode}
+        if cold_l2:
+            # every step behind a write of a buffer larger than L2, timed on its own
+            flush = torch.empty(2 * L2_BYTES // 4, dtype=torch.float32, device=dev)
+            ts = []
+            for _ in range(20):
+                flush.fill_(1.0)
+                ts.append(rd.timed(rd.step, rd.t_next, 1)); rd.t_next += 1
+            e["ms_per_step_cold_l2"] = statistics.median(ts)
+            del flush
+        return e
+    except Exception as ex:
+        return {"workload": name, "skipped": repr(ex)[:160]}
+    finally:
+        rd.close()
+        del rd
+        torch.cuda.empty_cache()
+
+
+def run_sweep(args, dev, peak):
+    import torch
+    from paper_2005_10761_b200 import workloads as wl
+    out = []
+    out.append(sweep_point("c1", args, dev, peak, steps=50, warmup=10, cold_l2=True))
+    for name in ("c2", "c2_n5", "c3_f32", "c3_bf16", "c4"):
+        if name != args.workload:
+            out.append(sweep_point(name, args, dev, peak, steps=20, warmup=10))
+    for name in ("c2", "c3_f32"):
+        out.append(sweep_point(name, args, dev, peak, steps=10, warmup=3, select_path="exact"))
+    # c5: d = 2^28; one gradient batch of the largest row count is generated once and shared (every
+    # point reads rows 0..W-1 of it; the vector is 8x the L2 already at W = 1)
+    free_b, _ = torch.cuda.mem_get_info()
+    d5 = 1 << 28
+    W_fit = int((free_b - 12e9) // (d5 * 4 * 2 * 1.08))
+    W_all = [W for W in (1, 4, 16, 32) if W <= W_fit]
+    if not W_all:
+        out.append({"workload": "c5", "skipped": f"free memory {free_b / 1e9:.0f} GB holds no c5 row"})
+        return out
+    Wg = max(W_all)
+    g5 = wl.gradient(dataclasses.replace(wl.configs()["c5_W32_r100_k10"], W=Wg), 0, dev)
+    for W in W_all:
+        names = [f"c5_W{W}_r{rd}_k{kd}" for rd in (100, 1000) for kd in (10, 4)] + [f"c5_W{W}_topk", f"c5_W{W}_randk"]
+        for name in names:
+            st = 3 if W >= 16 else 6
+            out.append(sweep_point(name, args, dev, peak, grads=[g5[:W]], steps=st, warmup=3, repeats=3))
+    if Wg < 32:
+        out.append({"workload": "c5_W32_*", "skipped": f"free memory {free_b / 1e9:.0f} GB: W limited to {Wg}"})
+    del g5
+    torch.cuda.empty_cache()
+    return out
+
+
+def spawn_ranks(args) -> int:
+    """--gpus N > 1 without a launcher: start N ranks of this script, one per GPU."""
+    import torch
+    have = torch.cuda.device_count()
+    if have < args.gpus:
+        print(f"bench: --gpus {args.gpus} but {have} CUDA devices are visible", file=sys.stderr)
+        return 2
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
@@ -202,13 +504,18 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--repeats", type=int, default=5, help="how many times the timed region of --steps steps is run")
+    ap.add_argument("--workload", default="c3_f32")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--scale-d", type=int, default=0, help="run the workload's recipe at this vector length")
     ap.add_argument("--workers", type=int, default=0,
                     help="run the workload's recipe with this many worker rows per GPU (plain workloads)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sweep", type=int, default=1, choices=[0, 1],
+                    help="1 (default, one GPU): also run the other configurations briefly and print them as `sweep`")
+    ap.add_argument("--select-path", default="sampled", choices=["sampled", "exact"],
+                    help="exact: the multi-pass radix select over the full vector (RTOPK_OPT_SELECT_PATH = 1)")
     ap.add_argument("--apply", action="store_true",
                     help="time rtopk_step_apply (master update fused into the aggregation; plain workloads, 1 GPU)")
     ap.add_argument("--threshold", type=float, default=None,
@@ -225,18 +532,20 @@ def main():
     if args.impl == "reference":
         run_reference(args)
         return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
 
     import torch
     import torch.distributed as dist
-    import paper_2005_10761_b200 as rt
-    from paper_2005_10761_b200 import build, sharded, workloads as wl
-    from paper_2005_10761_b200.binding import OPT_PROFILE
+    from paper_2005_10761_b200 import build
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for the product path)")
+    if local >= torch.cuda.device_count():
+        raise SystemExit(f"rank {rank}: no CUDA device {local} ({torch.cuda.device_count()} visible)")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     if world > 1:
@@ -247,180 +556,65 @@ def main():
         dist.barrier()
 
     cfg = pick_workload(args.workload, args.scale_d, args.workers)
-    W, d, ld = cfg.W, cfg.d, cfg.ld
-    W_total = W * world                      # weak scaling: W workers per GPU
-    gsz = 4 if cfg.grad_dtype == "f32" else 2
-    K = cfg.k_total
     seg = cfg.seg_off is not None
     thr = args.threshold is not None
-    ctx = rt.RTopK(d_max=d, W_max=W_total, r_max=min(d, 4 * cfg.r) if thr else cfg.r, k_max=K,
-                   segments_max=len(cfg.seg_r) if seg else 1, device=local)
-
-    if args.reuse_threshold:
-        from paper_2005_10761_b200.binding import OPT_REUSE_THRESHOLD
-        ctx.set_option(OPT_REUSE_THRESHOLD, 1)
-
-    # gradient batches resident in HBM before timing; the residual is carried across all steps
-    batch_bytes = W * ld * gsz
-    n_batches = max(1, min(cfg.steps, int(24e9 // batch_bytes), args.steps + args.warmup))
-    shard_cfg = cfg if world == 1 else dataclasses.replace(cfg, W=W_total)
-    rows = range(rank * W, rank * W + W)
-    grads = [wl.gradient(shard_cfg, t, dev, workers=rows) for t in range(n_batches)]
-    residual = wl.zero_residual(cfg, dev)
-    idx = torch.zeros((W, K), dtype=torch.int32, device=dev)
-    val = torch.zeros((W, K), dtype=torch.float32, device=dev)
-    # the dense update; with --apply the model weights that the update is applied to
-    out = torch.zeros(wl.round_up(d, 4), dtype=torch.float32, device=dev)
     if (args.apply or thr) and (seg or world > 1):
         raise SystemExit("--apply and --threshold cover the plain single-GPU workloads")
-    cnt = torch.zeros(W, dtype=torch.int32, device=dev)
-    ones = torch.zeros(W, dtype=torch.int32, device=dev)
-    base = rank * W
+    if args.select_path == "exact" and thr:
+        raise SystemExit("--threshold runs on the sampled path only")
+    rd = Round(cfg, args, dev, world, rank)
+    W, d, K, gsz = rd.W, rd.d, rd.K, rd.gsz
 
-    def one_step(t: int):
-        g = grads[t % n_batches]
-        if world == 1:
-            if seg:
-                ctx.step_segmented(g, residual, d, cfg.seg_off, cfg.seg_r, cfg.seg_k, cfg.seed, t, idx, val, out)
-            elif thr:
-                ctx.step_threshold(g, residual, d, args.threshold, cfg.k, cfg.seed, t, idx, val, cnt, ones, out)
-            elif args.apply:
-                ctx.step_apply(g, residual, d, cfg.r, cfg.k, cfg.seed, t, 0.01, idx, val, out)
-            else:
-                ctx.step(g, residual, d, cfg.r, cfg.k, cfg.seed, t, idx, val, out)
-        else:
-            def sp(gl, ml, wb):
-                if seg:
-                    ctx.sparsify_segmented(gl, ml, d, cfg.seg_off, cfg.seg_r, cfg.seg_k, cfg.seed, t, idx, val,
-                                           worker_base=wb)
-                else:
-                    ctx.sparsify(gl, ml, d, cfg.r, cfg.k, cfg.seed, t, idx, val, worker_base=wb)
-                return idx, val
-
-            def ag(ia, va):
-                ctx.aggregate(ia, va, d, out)
-                return out
-            sharded.sharded_round(sp, ag, g, residual, W_total, world, rank)
-
-    def sync_all():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-            torch.cuda.synchronize()
-
-    def timed(fn, t_first: int, n: int) -> float:
-        """Device time in ms of n consecutive steps (max over ranks)."""
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        sync_all()
-        e0.record()
-        for t in range(t_first, t_first + n):
-            fn(t)
-        e1.record()
-        sync_all()
-        ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item())
-
-    t_next = 0
-    for _ in range(args.warmup):
-        one_step(t_next); t_next += 1
-    sync_all()
     sampler = ClockSampler(local) if rank == 0 else None
     wall0 = time.time()
-    launches0 = ctx.launch_count()
-    graphed = bool(args.graph) and world == 1 and not thr   # (the threshold call re-uploads its slice table)
-    if graphed:
-        from paper_2005_10761_b200.binding import OPT_DEVICE_STEP
-        ctx.set_option(OPT_DEVICE_STEP, 1)
-        ctx.set_device_step(t_next)
-        graph_len = min(n_batches, args.steps)     # rounds held by the graph
-        reps, rem = divmod(args.steps, graph_len)
-        launches_per_graph = 0
-        if reps:
-            try:
-                cap_stream = torch.cuda.Stream()
-                graph = torch.cuda.CUDAGraph()
-                torch.cuda.synchronize()
-                l0 = ctx.launch_count()
-                with torch.cuda.graph(graph, stream=cap_stream):
-                    for b in range(graph_len):
-                        one_step(b)
-                launches_per_graph = ctx.launch_count() - l0
-                graph.replay()             # untimed: the first launch of a graph also uploads it
-                torch.cuda.synchronize()
-            except Exception as ex:        # no capture on this box: the rounds are launched one by one
-                print(f"bench: CUDA graph capture failed ({ex!r}); launching on the stream", file=sys.stderr)
-                torch.cuda.synchronize()
-                reps, rem, graphed = 0, args.steps, False
-
-        def graph_rounds(i: int):          # called once per timed "step" index; replays at the batch boundaries
-            if i < reps * graph_len:
-                if i % graph_len == 0:
-                    graph.replay()
-            else:
-                one_step(i)
-        launches0 = ctx.launch_count()
-        total_ms = timed(graph_rounds, 0, args.steps)
-        gpu_launches = ctx.launch_count() - launches0 + reps * launches_per_graph
-    else:
-        total_ms = timed(one_step, t_next, args.steps)
-        gpu_launches = ctx.launch_count() - launches0   # this library's kernels inside the timed region
+    regions, gpu_launches, launch_mode = rd.measure(args.steps, args.warmup, max(1, args.repeats), bool(args.graph))
     wall1 = time.time()
-    t_next += args.steps
     clocks = sampler.stop(wall0, wall1) if sampler else None
-    ctx.poll_status()
-    ms_per_step = total_ms / args.steps
-    value = W_total * d * gsz / (ms_per_step * 1e-3) / 1e9
-    n_slices = W * (len(cfg.seg_r) if seg else 1)
-    fallbacks = sum(ctx.stats(s)["used_fallback"] for s in range(n_slices))     # of the last timed step
-    predicted = 0
+    ms_per_step = statistics.median(regions)
+    value = rd.W_total * d * gsz / (ms_per_step * 1e-3) / 1e9
 
-    # the streaming kernel's own duration: same steps again with events between the phases
-    ctx.set_option(OPT_PROFILE, 1)
-    phase_sum, n_prof = {}, 0
-    for _ in range(min(args.steps, 20)):
-        one_step(t_next); t_next += 1
-        for name, ms in ctx.phase_times().items():
-            if ms >= 0:
-                phase_sum[name] = phase_sum.get(name, 0.0) + ms
-        n_prof += 1
-        stats = [ctx.stats(s) for s in range(n_slices)]                         # ... and of every profiled step
-        fallbacks += sum(s["used_fallback"] for s in stats)
-        predicted += sum(s["bracket_predicted"] for s in stats)
-    ctx.set_option(OPT_PROFILE, 0)
-    phases = {k: v / n_prof for k, v in phase_sum.items()}
+    # the dominant kernel's own duration: more steps with events between the phases
+    phases, fallbacks, predicted = rd.profile_phases(min(args.steps, 20))
+    n_prof = min(args.steps, 20)
     peak, peak_src = load_peak()
-    stream_bytes = W * d * (gsz + 8)
+    stream_bytes = rd.stream_bytes()
     stream_ms = phases.get("stream")
     achieved = stream_bytes / (stream_ms * 1e-3) / 1e9 if stream_ms else None
     roofline = {"bound": "hbm", "kernel": "k_stream (fused add + write-back + candidate gather)",
                 "achieved": achieved, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None,
-                "traffic": recorded_traffic(cfg.name, stream_bytes),
+                "traffic": recorded_traffic(stream_bytes),
                 "algorithmic_bytes_per_launch": stream_bytes, "kernel_ms": stream_ms}
-    # with --apply the 4 d-byte dense update is not written: 8 bytes per sent coordinate instead
-    step_bytes = W * d * (gsz + 8) + (8 * W * K if args.apply else 4 * d) + 16 * W * K
-    step_frac = step_bytes / (ms_per_step * 1e-3) / 1e9 / peak if world == 1 else None
+    step_bytes = rd.step_bytes()
+    step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
+    step_frac = step_gbs / peak if world == 1 else None
 
     # end to end: host gradient in, host messages + update out, through rtopk_step_host
     e2e = None
     if not args.no_e2e and world == 1 and not seg and not args.apply and not thr:
-        h_grad = grads[0].cpu().pin_memory()
+        h_grad = rd.grads[0].cpu().pin_memory()
         h_idx = torch.zeros((W, K), dtype=torch.int32).pin_memory()
         h_val = torch.zeros((W, K), dtype=torch.float32).pin_memory()
         h_out = torch.zeros(d, dtype=torch.float32).pin_memory()
 
         def host_step(t: int):
-            ctx.step_host(h_grad, residual, d, cfg.r, cfg.k, cfg.seed, t, h_idx, h_val, h_out)
-        for _ in range(2):
-            host_step(t_next); t_next += 1
+            rd.ctx.step_host(h_grad, rd.residual, d, cfg.r, cfg.k, cfg.seed, t, h_idx, h_val, h_out)
+        for _ in range(3):
+            host_step(rd.t_next); rd.t_next += 1
         n_e2e = max(3, min(args.steps, 10))
-        ms = timed(host_step, t_next, n_e2e) / n_e2e
-        t_next += n_e2e
+        ms = rd.timed(host_step, rd.t_next, n_e2e) / n_e2e
+        rd.t_next += n_e2e
         e2e = {"value": W * d * gsz / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms,
-               "h2d_bytes_per_step": W * ld * gsz, "d2h_bytes_per_step": 8 * W * K + 4 * d}
-    ctx.poll_status()
+               "h2d_bytes_per_step": W * rd.ld * gsz, "d2h_bytes_per_step": 8 * W * K + 4 * d}
+        del h_grad, h_idx, h_val, h_out
+    rd.ctx.poll_status()
+    rd.close()
+    del rd
+    torch.cuda.empty_cache()
+
+    sweep = None
+    if args.sweep and world == 1 and rank == 0 and not (args.apply or thr or args.scale_d or args.workers):
+        sweep = run_sweep(args, dev, peak)
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -439,28 +633,22 @@ def main():
     if rank == 0:
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "repeats": len(regions), "ms_per_step": ms_per_step,
+            "ms_per_step_min": min(regions), "ms_per_step_regions": regions,
+            "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": cfg.name, "d": d, "W_per_gpu": W, "W_total": W_total, "r": cfg.r, "k": K,
-                       "grad_dtype": cfg.grad_dtype, "recipe": cfg.recipe, "segments": len(cfg.seg_r) if seg else 1,
-                       "gradient_batches_resident": n_batches, "residual": "carried across steps",
-                       "l2": "inputs larger than L2 (no flush)", "parallelism": f"workers sharded x{world}",
-                       "variant": ("rtopk_step_apply (fused master update)" if args.apply else
-                                   f"rtopk_step_threshold (theta = {args.threshold})" if thr else "rtopk_step"),
-                       "launch": "cuda graph replay" if (graphed and reps) else "stream launches",
-                       "reuse_threshold": bool(args.reuse_threshold)},
-            "elements_per_s": W_total * d / (ms_per_step * 1e-3),
-            "step_roofline_frac": step_frac, "step_algorithmic_bytes": step_bytes,
+            "config": config_dict(cfg, args, world),
+            "launch": launch_mode,
+            "elements_per_s": W * world * d / (ms_per_step * 1e-3),
+            "step_roofline_frac": step_frac, "step_roofline_frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS if world == 1 else None,
+            "step_algorithmic_bytes": step_bytes,
             "phases_ms": phases, "fallback_slices": fallbacks,
-            **({"marked_per_worker_last_step": float(ones.float().mean().item()),
-                "sent_per_worker_last_step": float(cnt.float().mean().item())} if thr else {}),
-            "predicted_brackets": {"slices": predicted, "of": n_slices * n_prof},
+            "predicted_brackets": {"slices": predicted, "of": W * (len(cfg.seg_r) if seg else 1) * n_prof},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": gpu_launches,
-            "clocks": clocks,
+            "clocks": clocks, "sweep": sweep,
         }))
     if world > 1:
         dist.destroy_process_group()
-    ctx.close()
 
 
 if __name__ == "__main__":

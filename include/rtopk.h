@@ -305,6 +305,10 @@ int rtopk_step_threshold(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64
  * it afterwards, or a synchronisation of it, sees the results.  The call itself returns without
  * waiting.  h_grad must stay unchanged until the step that reads it has started (synchronise `stream`,
  * or make two further calls), the result buffers until `stream` has passed this call.
+ * A call whose shape (W, ld_g, k or grad_dtype) differs from the previous host call's waits on the host
+ * for the work of the earlier calls (`stream` and both copy streams) before it re-divides the staging
+ * buffers, and a call that needs larger buffers than any before it also reallocates them (cudaFree /
+ * cudaMalloc): keep the shape fixed inside a loop that must not stall.
  */
 int rtopk_step_host(rtopk_ctx* ctx, const void* h_grad, int grad_dtype, int64_t ld_g,
                     float* residual, int64_t ld_m, int64_t d, int32_t W, int32_t worker_base,

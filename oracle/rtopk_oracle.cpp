@@ -149,19 +149,19 @@ inline float widen_grad(const void* grad, int dtype, int64_t i) {
 void sparsify_slice(const void* grad, int dtype, float* residual, int64_t d, int64_t r, int64_t k,
                     uint64_t seed, uint32_t step, uint32_t worker, uint32_t segment,
                     uint32_t idx_base, uint32_t* msg_idx, float* msg_val) {
-  // a = g + m   (materialised in the residual buffer)
+  // the error-compensated vector (Algorithm 1), kept in the residual buffer from here on
   for (int64_t i = 0; i < d; ++i) {
     float s = widen_grad(grad, dtype, i) + residual[i];   // one binary32 add
     if (s != s) s = bits_float(0x7FC00000u);              // NaN payloads are not portable: store the default NaN
     residual[i] = s;
   }
-  // I <- indices of the r largest-magnitude components
+  // Definition 1: full sort by (magnitude descending, index ascending), first r, listed by ascending index
   std::vector<uint32_t> L((size_t)r);
   top_r_indices(residual, d, r, L.data());
-  // I <- random k-subset of I
+  // Definition 3: k positions of that list, by the sequential Floyd loop on Philox draws
   std::vector<uint32_t> pos((size_t)k);
   sample_positions(r, k, seed, step, worker, segment, pos.data());
-  // ghat <- a restricted to I ;  m' <- a - ghat
+  // the chosen coordinates are sent with their values; what is sent leaves the residual (+0.0f there)
   for (int64_t q = 0; q < k; ++q) {
     const uint32_t i = L[pos[(size_t)q]];
     msg_idx[q] = idx_base + i;
@@ -335,7 +335,7 @@ int oracle_warmup_sizes(int64_t d, int32_t n, double initial, double final_, int
                         int64_t* k) {
   if (d < 1 || n < 1 || t < 0 || T < 0 || !r || !k || !(final_ > 0.0) || !(initial >= final_) || !(initial <= 1.0))
     return ORACLE_BAD_ARG;
-  const double density = t < T ? initial * std::exp(std::log(final_ / initial) * ((double)t / (double)T)) : final_;
+  const double density = t < T ? initial * std::pow(final_ / initial, (double)t / (double)T) : final_;
   int64_t kk = (int64_t)(density * (double)d);
   kk = std::max<int64_t>(1, std::min<int64_t>(d, kk));
   *k = kk;

@@ -61,6 +61,7 @@ struct rtopk_ctx {
   size_t agg_start_entries = 0;
   void* d_stage = nullptr;       // host-call staging: two gradient buffers, messages, update
   size_t stage_bytes = 0;
+  size_t stage_g_bytes = 0, stage_mi_bytes = 0;   // the layout the staging buffer is currently carved with
   // rtopk_step_host moves data on two copy streams of its own, so that the upload of the next call's
   // gradient and the download of the last call's results overlap the step between them
   cudaStream_t copy_in = nullptr, copy_out = nullptr;
@@ -1014,6 +1015,15 @@ int rtopk_step_host(rtopk_ctx* ctx, const void* h_grad, int grad_dtype, int64_t 
     const cudaError_t e = cudaMalloc(&ctx->d_stage, total);
     if (e != cudaSuccess) { cudaGetLastError(); ctx->last_cuda_error = (int)e; return RTOPK_ERR_ALLOC; }
     ctx->stage_bytes = total;
+    ctx->stage_g_bytes = g_bytes; ctx->stage_mi_bytes = mi_bytes;
+    ctx->consumed_valid[0] = ctx->consumed_valid[1] = false;
+  } else if (g_bytes != ctx->stage_g_bytes || mi_bytes != ctx->stage_mi_bytes) {
+    // another shape carves the same allocation differently: the earlier calls' steps and copies may
+    // still be using the old offsets, so everything in flight ends before the new ones are used
+    RTOPK_CUDA(ctx, cudaStreamSynchronize(st));
+    RTOPK_CUDA(ctx, cudaStreamSynchronize(ctx->copy_in));
+    RTOPK_CUDA(ctx, cudaStreamSynchronize(ctx->copy_out));
+    ctx->stage_g_bytes = g_bytes; ctx->stage_mi_bytes = mi_bytes;
     ctx->consumed_valid[0] = ctx->consumed_valid[1] = false;
   }
   const int b = ctx->stage_next;

@@ -11,6 +11,8 @@ The oracle's full sort is too slow for every row at these sizes, so per configur
   * the dense update is compared with the oracle's aggregate of the very messages the GPU produced
     (all W rows), bit for bit, which also meets the 1e-6 * max|g| bar.
 """
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import pytest
 import torch
@@ -90,15 +92,21 @@ def _run_config(lib, cfg, steps, sample_rows, path=0):
         ctx.poll_status()
         _check_rows_on_gpu(cfg, ctx, g, m_prev, m, idx, val, seg)
         del m_prev
-        # sampled rows against the oracle (each row is an independent worker: worker_base = its id)
+        # sampled rows against the oracle (each row is an independent worker: worker_base = its id);
+        # the rows' full sorts run side by side on host threads (the oracle call releases the GIL)
         idx_h, val_h = idx.cpu().numpy().view(np.uint32), val.cpu().numpy()
-        for n, w in enumerate(sample_rows):
+
+        def follow(n_w):
+            n, w = n_w
             g_h = _host_grad(cfg, g[w:w + 1])
             if seg:
-                o_idx, o_val = oracle.sparsify_segmented(g_h, m_or[n:n + 1], cfg.d, cfg.seg_off, cfg.seg_r, cfg.seg_k,
-                                                         cfg.seed, t, worker_base=w)
-            else:
-                o_idx, o_val = oracle.sparsify(g_h, m_or[n:n + 1], cfg.d, cfg.r, cfg.k, cfg.seed, t, worker_base=w)
+                return oracle.sparsify_segmented(g_h, m_or[n:n + 1], cfg.d, cfg.seg_off, cfg.seg_r, cfg.seg_k,
+                                                 cfg.seed, t, worker_base=w)
+            return oracle.sparsify(g_h, m_or[n:n + 1], cfg.d, cfg.r, cfg.k, cfg.seed, t, worker_base=w)
+        with ThreadPoolExecutor(max_workers=max(1, min(4, len(sample_rows)))) as pool:
+            followed = list(pool.map(follow, enumerate(sample_rows)))
+        for n, w in enumerate(sample_rows):
+            o_idx, o_val = followed[n]
             assert np.array_equal(idx_h[w], o_idx[0]), f"{cfg.name} step {t} worker {w}: indices"
             assert np.array_equal(val_h[w].view(np.uint32), o_val[0].view(np.uint32)), f"{cfg.name} step {t} worker {w}: values"
             assert np.array_equal(m[w].cpu().numpy().view(np.uint32), m_or[n].view(np.uint32)), f"{cfg.name} step {t} worker {w}: residual"
@@ -146,6 +154,19 @@ def test_c5_quarter_billion_coordinates(lib):
     if free < 24e9:
         pytest.skip("not enough free device memory on this (shared) GPU")
     _run_config(lib, cfg, 1, [2])
+
+
+@pytest.mark.parametrize("name,rows", [("c5_W16_r1000_k4", [0, 5, 10, 15]), ("c5_W32_r100_k10", [1, 12, 23, 31]),
+                                       ("c5_W4_r1000_k10", [0, 3]), ("c5_W4_r100_k4", [1])])
+def test_c5_sweep_points_many_workers(lib, name, rows):
+    # the remaining corners of the d = 2^28 sweep: W in {16, 32}, r / d = 0.1 %, k / r = 1 / 4.  Properties on
+    # every row, the oracle on four sampled rows, the update against the oracle's aggregate of all messages.
+    cfg = wl.configs()[name]
+    free, _ = torch.cuda.mem_get_info()
+    need = cfg.W * cfg.ld * 4 * 3.2 + 8e9            # g, m, the copy of m the checks keep, scratch, temporaries
+    if free < need:
+        pytest.skip(f"not enough free device memory on this (shared) GPU: {free / 1e9:.0f} GB of {need / 1e9:.0f} GB")
+    _run_config(lib, cfg, 1, rows)
 
 
 def test_slice_longer_than_2_to_28_uses_wider_chunk_groups(lib):

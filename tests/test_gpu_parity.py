@@ -541,6 +541,39 @@ def test_step_host_sequence_without_waiting_in_between(lib):
     assert torch.equal(m_h.view(torch.int32), m_d.view(torch.int32))
 
 
+def test_step_host_calls_of_changing_shape(lib):
+    # W = 8, then W = 4, then W = 8 again through one context with no wait in between: the smaller call
+    # divides the staging buffers differently, which must not disturb the call before it (whose step may
+    # still be reading its gradient) nor the call after it.
+    base = wl.scaled(wl.configs()["c2"], d=400009, W=8)
+    shapes = [base, wl.scaled(wl.configs()["c2"], d=400009, W=4), base]
+    ctx = _ctx(lib, base.d, 8, base.r, base.k)
+    gs, res, m_h = [], [], []
+    for t, cfg in enumerate(shapes):
+        gs.append(wl.gradient(cfg, t, "cpu").pin_memory())
+        res.append((torch.zeros((cfg.W, cfg.k), dtype=torch.int32).pin_memory(),
+                    torch.zeros((cfg.W, cfg.k), dtype=torch.float32).pin_memory(),
+                    torch.zeros(cfg.d, dtype=torch.float32).pin_memory()))
+        m_h.append(wl.zero_residual(cfg, "cuda"))
+    for t, cfg in enumerate(shapes):
+        ctx.step_host(gs[t], m_h[t], cfg.d, cfg.r, cfg.k, cfg.seed, t, *res[t])
+    torch.cuda.synchronize()
+    ctx.poll_status()
+    ctx2 = _ctx(lib, base.d, 8, base.r, base.k)
+    for t, cfg in enumerate(shapes):
+        m_d = wl.zero_residual(cfg, "cuda")
+        idx_d = torch.zeros((cfg.W, cfg.k), dtype=torch.int32, device="cuda")
+        val_d = torch.zeros((cfg.W, cfg.k), dtype=torch.float32, device="cuda")
+        out_d = torch.empty(cfg.ld, dtype=torch.float32, device="cuda")
+        ctx2.step(gs[t].cuda(), m_d, cfg.d, cfg.r, cfg.k, cfg.seed, t, idx_d, val_d, out_d)
+        torch.cuda.synchronize()
+        assert torch.equal(res[t][0], idx_d.cpu()), t
+        assert torch.equal(res[t][1].view(torch.int32), val_d.cpu().view(torch.int32)), t
+        assert torch.equal(res[t][2].view(torch.int32), out_d.cpu()[: cfg.d].view(torch.int32)), t
+        assert torch.equal(m_h[t].view(torch.int32), m_d.view(torch.int32)), t
+    ctx.close(); ctx2.close()
+
+
 @pytest.mark.parametrize("r,k", [(1, 1), (2, 1), (7, 3), (64, 64), (1000, 1), (1000, 999), (16384, 1024),
                                  (111739, 11173), (2684354, 671088)])
 def test_sampler_positions_against_oracle(lib, r, k):

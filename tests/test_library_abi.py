@@ -57,18 +57,19 @@ def test_product_package_does_not_import_the_oracle():
 
 
 def test_warmup_sizes_host_function_matches_the_oracle():
-    """rtopk_warmup_sizes is host-only arithmetic: callable without a GPU.  exp/log in the oracle and
-    pow in the library may differ in the last bit, so k may differ by one where density * d is
-    within rounding of an integer; the exact-power cases agree exactly."""
+    """rtopk_warmup_sizes is host-only arithmetic: callable without a GPU.  The contract is one formula in
+    binary64, k = max(1, min(d, floor(d * initial * pow(final / initial, t / T)))) for t < T, evaluated in
+    that order with the C library's pow, and r = min(d, n k): integer outputs, so both sides must agree
+    exactly."""
     import oracle
     import paper_2005_10761_b200 as rt
     d, n = 1 << 20, 8
     for t in range(7):
         assert rt.warmup_sizes(d, n, 0.25, 1.0 / 1024, 4, t) == oracle.warmup_sizes(d, n, 0.25, 1.0 / 1024, 4, t)
-    for t in range(0, 70, 3):
-        r1, k1 = rt.warmup_sizes(11_173_962, 5, 0.3, 0.001, 50, t)
-        r2, k2 = oracle.warmup_sizes(11_173_962, 5, 0.3, 0.001, 50, t)
-        assert abs(k1 - k2) <= 1 and r1 == min(11_173_962, 5 * k1)
+    for (dd, nn, hi, lo, T) in [(11_173_962, 5, 0.3, 0.001, 50), (25_557_032, 16, 1.0, 0.001, 97),
+                                (1 << 28, 32, 0.25, 0.0001, 1000), (1000, 3, 0.5, 0.01, 7)]:
+        for t in range(0, T + 20, max(1, T // 40)):
+            assert rt.warmup_sizes(dd, nn, hi, lo, T, t) == oracle.warmup_sizes(dd, nn, hi, lo, T, t), (dd, t)
     import pytest
     with pytest.raises(rt.RTopKError):
         rt.warmup_sizes(100, 4, 0.001, 0.01, 5, 0)

@@ -5,12 +5,15 @@ memory through its own allocator, or they sit in a latency-critical loop where t
 of an allocation is not acceptable.  A context allocates, so they get one entry point that keeps its
 scratch in a fixed array inside the library.  This test calls it through the C ABI twice in a row
 (the second call meets the first call's leftovers in the shared array) and compares the positions,
-bit for bit, with the context-based entry point; positions are integers, so the tolerance is zero.
+bit for bit, with the context-based entry point and with the CPU oracle's sequential Floyd loop;
+positions are integers, so the tolerance is zero.
 The file name makes pytest collect it after every other test.
 """
 import numpy as np
 import pytest
 import torch
+
+import oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -56,6 +59,7 @@ def test_static_scratch_call_matches_context_call_twice_in_a_row(lib):
             torch.cuda.synchronize()
             assert torch.cuda.mem_get_info()[0] == free_before      # the call took no device memory
         assert np.array_equal(pos.cpu().numpy(), w), f"r={r} k={k}"
+        assert np.array_equal(pos.cpu().numpy().view(np.uint32), oracle.sample_positions(*c)), f"r={r} k={k} (oracle)"
 
 
 def test_static_scratch_call_rejects_sizes_beyond_its_array(lib):
