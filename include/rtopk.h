@@ -83,12 +83,20 @@ enum {
                                 Section II (after the pre-processing step a coordinate is 0 or +-M, so one bit
                                 per kept coordinate describes it); the node then keeps a_i - sign(a_i) * M in
                                 that residual slot (one binary32 subtraction), m' = a - ghat as before */
-  RTOPK_OPT_DEVICE_STEP = 4     /* 1 = the round number t that enters the Philox counter is kept in a word on
+  RTOPK_OPT_DEVICE_STEP = 4,    /* 1 = the round number t that enters the Philox counter is kept in a word on
                                 the device: the sparsify / step calls (plain, segmented, threshold) ignore
                                 their `step` argument, read the word, and add one to it at their end (set it
                                 with rtopk_set_device_step; it starts at 0).  A caller that captures one round
                                 in a CUDA graph can then replay the graph round after round and still draw a
                                 fresh subset each time.  0 = off (default): `step` is the argument */
+  RTOPK_OPT_FINISH_PATH = 5     /* how the sampled path turns the candidates of the streaming pass into messages
+                                (the result is the same): 1 = one thread-block cluster per slice, which lays
+                                the candidate runs out in index order first; 2 = three grid-wide launches over
+                                all slices that work on the runs as they are (a histogram over the bracket, a
+                                count, the emission), with the cluster kernel behind them for what they leave
+                                (a missed bracket, heavy ties); 0 (default) = 2 for slices of 2^26 coordinates
+                                or more, where the runs no longer fit one cluster's shared memory and the L2,
+                                else 1 */
 };
 
 /* Phases of one call, in stream order.  STREAM is the single pass over the full vectors that

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librtopk.so")
 SOURCES = ["rtopk.cu"]
-HEADERS = ["common.cuh", "element.cuh", "select.cuh", "stream.cuh", "sampler.cuh", "aggregate.cuh", "codec.cuh", "threshold.cuh"]
+HEADERS = ["common.cuh", "element.cuh", "select.cuh", "stream.cuh", "sampler.cuh", "aggregate.cuh", "codec.cuh", "threshold.cuh", "finish.cuh"]
 
 
 def nvcc() -> str:

@@ -29,7 +29,7 @@ constexpr int kSampleThreads = 1024;
 
 // stage of the full-vector radix select of one slice
 enum : uint32_t { STAGE_PASS0 = 0, STAGE_PASS1 = 1, STAGE_PASS2 = 2, STAGE_COLLECT = 3, STAGE_DONE = 4 };
-enum : uint32_t { FLAG_GENERAL = 1u, FLAG_FELL_BACK = 2u };
+enum : uint32_t { FLAG_GENERAL = 1u, FLAG_FELL_BACK = 2u, FLAG_FINISHED = 4u /* finished by the run kernels (finish.cuh) */ };
 enum : uint32_t { ERR_LOOKBACK_TIMEOUT = 1u, ERR_CANDIDATE_OVERFLOW = 2u, ERR_SELECT_INCONSISTENT = 4u };
 
 // One slice: a worker row, or one tensor of a worker row.  Offsets are in elements.
@@ -52,6 +52,7 @@ struct Slice {
   uint32_t first_mask;  // 0: the table is dense (r entries); else it is a hash table of first_mask + 1 slots
   uint32_t sel_off;     // start in the selection bitmap / its prefix counts (32-bit words)
   uint32_t gshift;      // a chunk group is 2^gshift consecutive chunks (at most kGroupsMax groups per slice)
+  uint32_t part_begin;  // first entry of the slice in the per-block member totals of the run kernels
 };
 
 // Selection state of one slice, advanced kernel by kernel.
@@ -74,6 +75,16 @@ struct SelState {
 // of the last two calls, a running bound of the relative prediction error, and how many of the two
 // keys may be used (0: the next call samples).
 struct TauHistory { uint32_t tau1, tau2; float err; uint32_t valid; };
+
+// Where the run kernels (finish.cuh) stand with one slice.
+constexpr int kListMax = 2048;        // the histogram bucket that holds the r-th largest key is resolved on a list of up to this many candidates
+struct alignas(32) Fin {
+  uint32_t tau, cut;         // the exact r-th largest key; a key equal to it is a member up to this index
+  uint32_t ok;
+  uint32_t list_n;           // entries of the slice's short list
+  uint32_t done2;            // chunk groups k_run_count has completed
+  uint32_t pad[3];
+};
 
 struct Scratch {
   Slice* slices;
@@ -98,6 +109,9 @@ struct Scratch {
   uint32_t* sel_blk;      // selected positions per chunk of bitmap words (scan scratch)
   uint32_t* error;        // device error flags
   TauHistory* history;    // [slices] threshold history across calls
+  Fin* fin;               // [slices] state of the run kernels
+  uint32_t* list;         // [slices][2 * kListMax]: keys, then indices, of the candidates inside the bucket
+  uint32_t* part_tot;     // members per block of k_run_count (Slice::part_begin), then their exclusive prefix
 };
 
 struct Launch {
@@ -132,6 +146,14 @@ __device__ __forceinline__ uint32_t warp_sum(uint32_t v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
   return v;
+}
+
+// Bucket width (log2) of the histogram over a bracket [tau_lo, tau_hi] of the r-th largest key: 2047
+// equal buckets hold the bracket, the last one the keys above it.
+__device__ __forceinline__ uint32_t bracket_shift(uint32_t tau_lo, uint32_t tau_hi) {
+  uint32_t sh = 0;
+  while (((tau_hi - tau_lo) >> sh) >= (uint32_t)(kBins - 1)) ++sh;
+  return sh;
 }
 
 // index of the slice that owns global tile `t`: the last s with begin(s) <= t

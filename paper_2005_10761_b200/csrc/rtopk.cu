@@ -17,6 +17,7 @@
 #include "aggregate.cuh"
 #include "codec.cuh"
 #include "common.cuh"
+#include "finish.cuh"
 #include "sampler.cuh"
 #include "select.cuh"
 #include "stream.cuh"
@@ -29,6 +30,7 @@ struct rtopk_ctx {
   int64_t d_max = 0, r_max = 0, k_max = 0;
   int32_t W_max = 0, S_max = 0;
   int select_path = 0;
+  int finish_path = 0;                // RTOPK_OPT_FINISH_PATH
   int last_cuda_error = 0;
   // device scratch (one allocation each)
   Slice* d_slices = nullptr;
@@ -50,6 +52,10 @@ struct rtopk_ctx {
   size_t sel_blk_entries = 0;
   size_t sel_words = 0;
   uint32_t* d_error = nullptr;
+  Fin* d_fin = nullptr;              // per-slice state of the run kernels
+  uint32_t* d_list = nullptr;        // per-slice short lists (keys, indices)
+  uint32_t* d_part_tot = nullptr;    // per-block member totals of the run kernels
+  size_t part_entries = 0;
   TauHistory* d_history = nullptr;   // per-slice threshold history (RTOPK_OPT_REUSE_THRESHOLD)
   int reuse = 0;
   int threshold_signs = 0;            // RTOPK_OPT_THRESHOLD_SIGNS
@@ -139,7 +145,7 @@ uint64_t first_table_entries(Slice& sl) {
 // Layout of one call: the slice table plus every per-call scratch offset.
 struct Plan {
   std::vector<Slice> slices;
-  uint32_t n_chunks = 0, n_hist_blocks = 0, n_groups = 0;
+  uint32_t n_chunks = 0, n_hist_blocks = 0, n_groups = 0, n_parts = 0;
   size_t cand_entries = 0, draw_entries = 0, first_entries = 0, sel_words = 0;
   uint32_t k_draw_max = 0, words_all_max = 0, cap_max = 0, chunks_max = 0, sel_words_max = 0;
   bool any_select = false, any_sampler = false, any_all = false;
@@ -165,7 +171,7 @@ int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32
   P.K_row = (uint32_t)K;
   P.uniform = (S == 1);
   P.slices.resize((size_t)W * (size_t)S);
-  uint64_t chunks = 0, hblocks = 0, groups = 0, cand = 0, draws = 0, first = 0, selw = 0;
+  uint64_t chunks = 0, hblocks = 0, groups = 0, cand = 0, draws = 0, first = 0, selw = 0, parts = 0;
   for (int w = 0; w < W; ++w) {
     uint64_t msg_at = (uint64_t)w * K;
     for (int s = 0; s < S; ++s) {
@@ -195,6 +201,8 @@ int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32
       while (((nchunks + (1u << sl.gshift) - 1) >> sl.gshift) > (uint32_t)kGroupsMax) ++sl.gshift;
       sl.group_begin = (uint32_t)groups;
       groups += (nchunks + (1u << sl.gshift) - 1) >> sl.gshift;
+      sl.part_begin = (uint32_t)parts;
+      parts += (nchunks + kRunChunks - 1) / kRunChunks;
       sl.cand_off = (uint32_t)cand;
       if (sl.r < sl.len || always_gather) {
         sl.cand_cap = cand_capacity(sl.len, sl.r);
@@ -222,6 +230,7 @@ int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32
   }
   if (chunks >= (1ull << 31) || cand >= (1ull << 32) || first >= (1ull << 32)) return RTOPK_ERR_INVALID_ARG;
   P.n_chunks = (uint32_t)chunks; P.n_hist_blocks = (uint32_t)hblocks; P.n_groups = (uint32_t)groups;
+  P.n_parts = (uint32_t)parts;
   P.cand_entries = cand; P.draw_entries = draws; P.first_entries = first; P.sel_words = selw;
   return RTOPK_OK;
 }
@@ -292,7 +301,7 @@ int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t s
       const uint32_t per = (uint32_t)((P.slices[0].head + (uint64_t)P.slices[0].len + kChunk - 1) / kChunk);
       const uint32_t uniform = P.uniform ? per : 0u;
       const int blocks = ctx->stream_blocks[sizeof(GradT) == 4 ? 0 : 1];
-      k_stream<GradT><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
+      k_stream<GradT, false><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
       ++ctx->launches;
       if (clear_out) {
         // the streaming pass saturates the memory system and the kernels after it do not: the dense
@@ -370,6 +379,8 @@ int bind_launch(rtopk_ctx* ctx, const Plan& P, const void* grad, float* residual
   L.s.chunk_pre = ctx->d_chunk_tab + 2 * ctx->chunk_tab_entries;
   L.s.draws = ctx->d_draws; L.s.first = ctx->d_first; L.s.sel_pre = ctx->d_sel_pre; L.s.sel_blk = ctx->d_sel_blk;
   L.s.error = ctx->d_error;
+  if ((size_t)P.n_parts > ctx->part_entries) return RTOPK_ERR_INVALID_ARG;
+  L.s.fin = ctx->d_fin; L.s.list = ctx->d_list; L.s.part_tot = ctx->d_part_tot;
   L.grad = grad; L.residual = residual; L.msg_idx = msg_idx; L.msg_val = msg_val;
   L.n_slices = (uint32_t)P.slices.size();
   L.worker_base = (uint32_t)worker_base;
@@ -448,6 +459,21 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   const bool joined = forked && ctx->select_path == 0;
   if (forked && !joined) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0));
   mark(ctx, RTOPK_PHASE_FINISH, st);
+  const bool from_runs = ctx->finish_path == 2 || (ctx->finish_path == 0 && P.chunks_max >= (1u << 14));
+  if (P.any_select && ctx->select_path == 0 && from_runs && L.n_slices <= 65535u) {
+    // the usual case is finished straight from the streaming pass's runs, all slices side by side; what
+    // these kernels leave (a missed bracket, heavy ties) is flagged for k_finish
+    // about one wave of blocks over all slices together (8 blocks of 256 threads per SM)
+    const uint32_t per_slice = std::max<uint32_t>(1u, ((uint32_t)ctx->sms * 8u + L.n_slices - 1u) / L.n_slices);
+    const uint32_t tiles = (P.cap_max + kRunThreads * kHistPer - 1) / (kRunThreads * kHistPer);
+    const dim3 hgrid(std::min(tiles, per_slice), L.n_slices);
+    k_run_hist<<<hgrid, kRunThreads, 0, st>>>(L);
+    const uint32_t groups = (P.chunks_max + kRunChunks - 1) / kRunChunks;
+    const dim3 rgrid((groups + kRunBlockGroups - 1) / kRunBlockGroups, L.n_slices);
+    k_run_count<<<rgrid, kRunThreads, 0, st>>>(L);
+    k_run_emit<<<rgrid, kRunThreads, 0, st>>>(L);
+    ctx->launches += 3;
+  }
   if (P.any_select) {
     // the largest cluster size that still lets every slice's cluster be resident at once
     int cs = 1;
@@ -532,9 +558,9 @@ int threshold_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_
   mark(ctx, RTOPK_PHASE_STREAM, st);
   const uint32_t per = (uint32_t)((P.slices[0].head + (uint64_t)P.slices[0].len + kChunk - 1) / kChunk);
   if (grad_dtype == RTOPK_F32)
-    k_stream<float><<<ctx->stream_blocks[0], kStreamThreads, sizeof(StreamSmem<float>), st>>>(L, P.n_chunks, per);
+    k_stream<float, false><<<ctx->stream_blocks[0], kStreamThreads, sizeof(StreamSmem<float>), st>>>(L, P.n_chunks, per);
   else
-    k_stream<__nv_bfloat16><<<ctx->stream_blocks[1], kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>), st>>>(L, P.n_chunks, per);
+    k_stream<__nv_bfloat16, false><<<ctx->stream_blocks[1], kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>), st>>>(L, P.n_chunks, per);
   ++ctx->launches;
   if (clear_out) {
     RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_streamed, st));
@@ -719,6 +745,10 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   ctx->sel_blk_entries = slices * ((size_t)r_max / 32 / kSelChunk + 2);
   alloc((void**)&ctx->d_sel_blk, ctx->sel_blk_entries * sizeof(uint32_t));
   alloc((void**)&ctx->d_error, 16);
+  alloc((void**)&ctx->d_fin, slices * sizeof(Fin));
+  alloc((void**)&ctx->d_list, slices * 2 * kListMax * sizeof(uint32_t));
+  ctx->part_entries = chunks / kRunChunks + slices + 1;
+  alloc((void**)&ctx->d_part_tot, ctx->part_entries * sizeof(uint32_t));
   alloc((void**)&ctx->d_step, 16);
   alloc((void**)&ctx->d_history, slices * sizeof(TauHistory));
   alloc((void**)&ctx->d_agg_starts, ctx->agg_start_entries * sizeof(uint32_t));
@@ -749,10 +779,12 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   if (e == cudaSuccess) {
     int sms = 0, per_f32 = 0, per_bf16 = 0;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<float>));
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<__nv_bfloat16>));
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_f32, k_stream<float>, kStreamThreads, sizeof(StreamSmem<float>));
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_bf16, k_stream<__nv_bfloat16>, kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<float>));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<float>));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<__nv_bfloat16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<__nv_bfloat16>));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<__nv_bfloat16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<__nv_bfloat16>));
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_f32, k_stream<float, true>, kStreamThreads, sizeof(StreamSmem<float>));
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_bf16, k_stream<__nv_bfloat16, true>, kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>));
     if (e == cudaSuccess && (per_f32 < 1 || per_bf16 < 1)) e = cudaErrorLaunchOutOfResources;
     ctx->sms = sms;
     int per_exact = 0;
@@ -781,7 +813,7 @@ int rtopk_destroy(rtopk_ctx* ctx) {
   void* ptrs[] = {ctx->d_slices, ctx->d_state, ctx->d_zero, ctx->d_first, ctx->d_cand_idx, ctx->d_cand_val,
                   ctx->d_raw_idx, ctx->d_raw_val, ctx->d_chunk_tab,
                   ctx->d_draws, ctx->d_sel_pre, ctx->d_sel_blk, ctx->d_error, ctx->d_agg_starts, ctx->d_stage, ctx->d_history,
-                  ctx->d_step};
+                  ctx->d_step, ctx->d_fin, ctx->d_list, ctx->d_part_tot};
   for (void* p : ptrs) if (p) cudaFree(p);
   for (cudaEvent_t ev : ctx->ev) if (ev) cudaEventDestroy(ev);
   if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
@@ -809,6 +841,7 @@ int rtopk_set_option(rtopk_ctx* ctx, int option, int64_t value) {
     return RTOPK_OK;
   }
   if (option == RTOPK_OPT_DEVICE_STEP && (value == 0 || value == 1)) { ctx->device_step = (int)value; return RTOPK_OK; }
+  if (option == RTOPK_OPT_FINISH_PATH && value >= 0 && value <= 2) { ctx->finish_path = (int)value; return RTOPK_OK; }
   if (option == RTOPK_OPT_THRESHOLD_SIGNS && (value == 0 || value == 1)) { ctx->threshold_signs = (int)value; return RTOPK_OK; }
   if (option == RTOPK_OPT_PROFILE && (value == 0 || value == 1)) {
     ctx->profile = (int)value;

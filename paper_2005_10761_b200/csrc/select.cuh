@@ -28,8 +28,8 @@ __device__ __forceinline__ uint32_t slice_chunks(const Slice& S) {
   return (S.head + S.len + kChunk - 1) / kChunk;
 }
 
-// Clears the counters of slice `sl` that the streaming pass and the exact path expect to be zero
-// (run cursor, block counter, chunk-group totals; plus the launch-wide tickets).  The sampling
+// Clears the counters of slice `sl` that the streaming pass, the run kernels and the exact path expect
+// to be zero (run cursor, block counter, list length, chunk-group totals; plus the launch-wide tickets).  The sampling
 // kernels do this instead of a memset node in front of them; `part` of `nparts` thread blocks of
 // blockDim.x threads share the work.
 __device__ __forceinline__ void clear_slice_counters(const Launch& L, uint32_t sl, const Slice& S, uint32_t part, uint32_t nparts) {
@@ -37,7 +37,7 @@ __device__ __forceinline__ void clear_slice_counters(const Launch& L, uint32_t s
   const uint32_t nchunks = slice_chunks(S);
   const uint32_t ngroups = (nchunks + (1u << S.gshift) - 1u) >> S.gshift;
   for (uint32_t g = t; g < ngroups; g += nt) L.s.group_total[S.group_begin + g] = 0;
-  if (t == 0) { L.s.cursor[sl] = 0; L.s.done[sl] = 0; }
+  if (t == 0) { L.s.cursor[sl] = 0; L.s.done[sl] = 0; L.s.fin[sl].list_n = 0; L.s.fin[sl].done2 = 0; }
   if (sl == 0 && t < 4u) L.s.tickets[t] = 0;
 }
 
@@ -700,6 +700,7 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
   SelState* st = &L.s.state[sl];
   // every early exit below depends on the slice only, so a cluster leaves as a whole
   if (S.r == S.len) return;
+  if (st->flags & FLAG_FINISHED) return;                       // the run kernels have finished this slice
   bool general = (st->flags & FLAG_GENERAL) != 0;               // the list was built by the exact path
   uint32_t n_cand = general ? st->n_cand : L.s.cursor[sl];
   if (st->resolved > 31) return;                               // an earlier pass already failed

@@ -13,7 +13,10 @@ from paper_2005_10761_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
-AUTO, EXACT = 0, 1
+# how a context selects: the sampled bracket finished by the cluster kernel (what AUTO takes at these
+# sizes), the full-vector radix select, or the sampled bracket finished from the runs by the three
+# grid-wide kernels (what AUTO takes for slices of 2^26 coordinates or more)
+AUTO, EXACT, RUNS = 0, 1, 2
 
 
 @pytest.fixture(scope="module")
@@ -26,7 +29,8 @@ def lib():
 
 def _ctx(lib, d, W, r, k, S=1, path=AUTO):
     ctx = lib.RTopK(d_max=d, W_max=W, r_max=r, k_max=k, segments_max=S)
-    ctx.set_option(0, path)
+    ctx.set_option(0, EXACT if path == EXACT else AUTO)          # RTOPK_OPT_SELECT_PATH
+    ctx.set_option(5, 2 if path == RUNS else 0)                  # RTOPK_OPT_FINISH_PATH
     return ctx
 
 
@@ -94,7 +98,7 @@ SMALL = [(1, 1, 1), (2, 2, 1), (3, 2, 2), (5, 3, 2), (31, 7, 3), (33, 33, 4), (1
          (4098, 4098, 17), (5003, 1, 1), (12289, 900, 90), (40001, 400, 40)]
 
 
-@pytest.mark.parametrize("path", [AUTO, EXACT])
+@pytest.mark.parametrize("path", [AUTO, EXACT, RUNS])
 @pytest.mark.parametrize("d,r,k", SMALL)
 def test_small_and_ragged_sizes(lib, d, r, k, path):
     rng = np.random.default_rng(d * 7 + r)
@@ -104,7 +108,7 @@ def test_small_and_ragged_sizes(lib, d, r, k, path):
     check_against_oracle(lib, g, m0, d, r, k, seed=d, step=3, worker_base=5, path=path)
 
 
-@pytest.mark.parametrize("path", [AUTO, EXACT])
+@pytest.mark.parametrize("path", [AUTO, EXACT, RUNS])
 def test_heavy_ties(lib, path):
     rng = np.random.default_rng(2)
     W, d = 2, 70001
@@ -123,7 +127,7 @@ def test_heavy_ties(lib, path):
             assert stats is not None, name
 
 
-@pytest.mark.parametrize("path", [AUTO, EXACT])
+@pytest.mark.parametrize("path", [AUTO, EXACT, RUNS])
 def test_non_finite_and_denormal_values(lib, path):
     rng = np.random.default_rng(3)
     W, d = 2, 9001
@@ -140,7 +144,7 @@ def test_multi_tile_many_workers_and_worker_base(lib):
     W, d, r, k = 7, 300007, 3000, 300
     g = _pad(_spiky(rng, W, d, p=0.01))
     m0 = _pad(_spiky(rng, W, d, p=0.01) * 0.3)
-    for path in (AUTO, EXACT):
+    for path in (AUTO, EXACT, RUNS):
         check_against_oracle(lib, g, m0, d, r, k, seed=0xDEADBEEF12345, step=77, worker_base=1000, path=path)
 
 
@@ -149,7 +153,7 @@ def test_limits_topk_and_randomk(lib):
     W, d = 2, 50000
     g = _pad(_spiky(rng, W, d))
     m0 = np.zeros_like(g)
-    for path in (AUTO, EXACT):
+    for path in (AUTO, EXACT, RUNS):
         check_against_oracle(lib, g, m0, d, 500, 500, seed=1, step=2, path=path)      # k = r: Definition 1
         check_against_oracle(lib, g, m0, d, d, 50, seed=1, step=2, path=path)         # r = d: Definition 2
         check_against_oracle(lib, g, m0, d, d, d, seed=1, step=2, path=path)          # everything is sent
@@ -160,7 +164,7 @@ def test_bf16_gradient(lib):
     W, d, r, k = 3, 100003, 1000, 100
     g = _pad(_spiky(rng, W, d))
     m0 = _pad(_spiky(rng, W, d) * 0.25)
-    for path in (AUTO, EXACT):
+    for path in (AUTO, EXACT, RUNS):
         check_against_oracle(lib, g, m0, d, r, k, seed=6, step=6, path=path, bf16=True)
 
 
@@ -196,7 +200,7 @@ def test_segmented_per_tensor_selection(lib):
     m0 = _pad(_spiky(rng, W, d) * 0.5)
     m_or = m0.copy()
     o_idx, o_val = oracle.sparsify_segmented(g, m_or, d, off, seg_r, seg_k, seed=8, step=5, worker_base=2)
-    for path in (AUTO, EXACT):
+    for path in (AUTO, EXACT, RUNS):
         ctx = _ctx(lib, d, W, sum(seg_r), K, S=len(sizes), path=path)
         tg, tm = torch.from_numpy(g).cuda(), torch.from_numpy(m0.copy()).cuda()
         idx = torch.zeros((W, K), dtype=torch.int32, device="cuda")
@@ -696,7 +700,7 @@ def test_random_shapes_values_and_paths(lib, case):
         g = (np.round(g * levels) / levels).astype(np.float32)
         m0 = (np.round(m0 * levels) / levels).astype(np.float32)
     check_against_oracle(lib, _pad(g), _pad(m0), d, r, k, seed=int(rng.integers(0, 2**40)), step=int(rng.integers(0, 1000)),
-                         worker_base=int(rng.integers(0, 50)), path=int(rng.choice([AUTO, EXACT])),
+                         worker_base=int(rng.integers(0, 50)), path=int(rng.choice([AUTO, EXACT, RUNS])),
                          bf16=bool(rng.random() < 0.3))
 
 
