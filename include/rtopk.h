@@ -135,6 +135,10 @@ int rtopk_last_cuda_error(const rtopk_ctx* ctx);
  * vectors of at most d_max elements, W_max rows, r_max / k_max per slice summed over a row's
  * slices (for the plain calls: r and k), segments_max slices per row (1 for the plain calls).
  * The context owns its scratch (cudaMalloc) until rtopk_destroy.  d_max < 2^31.
+ * A context with r_max = d_max whose candidate lists would take 2^30 entries or more (W_max * d_max, about)
+ * is taken to be made for Definition 2's r = d (random-k), which needs no lists: it also serves calls
+ * with r < d, but only up to about r = d_max / 32 per row (a call beyond what the lists hold returns
+ * INVALID_ARG, as every call beyond the context's maxima does).
  * Errors: INVALID_ARG, ALLOC, CUDA.
  */
 int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int64_t r_max,

@@ -289,45 +289,120 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     return a;
   };
   if (staged) {
+    // ---- the usual case: the tile's entries fit the stage
+    __shared__ uint16_t st_w[kAggSparseStage];                       // worker of every staged entry
+    __shared__ uint32_t s_seen[kAggSparseTile / 32], s_shared[kAggSparseTile / 32];
+    __shared__ uint16_t s_pool[kAggSparseStage];
+    // (the run tables are not needed once the entries are staged with their workers, nor is the "seen"
+    // bitmap once the shared coordinates are marked: the slot tables take their place)
+    static_assert(kAggSparseStage / 2 <= kAggMaxW, "the slot tables fit the run tables");
+    uint32_t* const s_off = s_pre;                                    // [kAggSparseStage / 2 + 1]
+    uint32_t* const s_cur = s_beg;                                    // [kAggSparseStage / 2]
+    uint32_t* const s_slot = s_seen;                                  // [kAggSparseTile / 32]
     for (uint32_t q = tid; q < total; q += kAggThreads) {
       const uint32_t a = worker_of(q);
       const uint32_t j = s_beg[a] + (q - s_pre[a]);
       st_idx[q] = msgs.index(a, j);
       st_val[q] = msgs.value(a, j);
+      st_w[q] = (uint16_t)a;
     }
-    __syncthreads();
-  }
-  auto idx_at = [&](uint32_t w, uint32_t j) {        // j-th entry of worker w's run in this tile
-    return staged ? st_idx[s_pre[w] + j] : msgs.index(w, s_beg[w] + j);
-  };
-  auto val_at = [&](uint32_t w, uint32_t j) {
-    return staged ? st_val[s_pre[w] + j] : msgs.value(w, s_beg[w] + j);
-  };
-  // Most coordinates are sent by a single worker.  Two bitmaps over the tile find the ones that are
-  // not: the second entry that sets a coordinate's "seen" bit also sets its "shared" bit.
-  __shared__ uint32_t s_seen[kAggSparseTile / 32], s_shared[kAggSparseTile / 32];
-  if (staged) {
+    // Most coordinates are sent by a single worker.  Two bitmaps over the tile find the ones that are
+    // not: the second entry that sets a coordinate's "seen" bit also sets its "shared" bit.
     for (uint32_t i = tid; i < (uint32_t)(kAggSparseTile / 32); i += kAggThreads) { s_seen[i] = 0; s_shared[i] = 0; }
     __syncthreads();
+    bool any_shared = false;
     for (uint32_t q = tid; q < total; q += kAggThreads) {
       const uint32_t local = st_idx[q] - lo;
       if (local < (uint32_t)kAggSparseTile) {
         const uint32_t bit = 1u << (local & 31u);
-        if (atomicOr(&s_seen[local >> 5], bit) & bit) atomicOr(&s_shared[local >> 5], bit);
+        if (atomicOr(&s_seen[local >> 5], bit) & bit) { atomicOr(&s_shared[local >> 5], bit); any_shared = true; }
+      }
+    }
+    any_shared = __syncthreads_or(any_shared);
+    // a sole sender's coordinate: the sum is the value
+    for (uint32_t q = tid; q < total; q += kAggThreads) {
+      const uint32_t idx = st_idx[q], local = idx - lo;
+      if (local >= (uint32_t)kAggSparseTile || idx >= d) continue;   // malformed row: ignore
+      if (!((s_shared[local >> 5] >> (local & 31u)) & 1u)) {
+        const double v = msgs.term(st_w[q], st_val[q]);
+        out[idx] = agg_result((float)agg_scaled(v, 1u, sc), eta >= 0.0f ? out[idx] : 0.0f, eta);
+      }
+    }
+    if (!any_shared) return;                                          // (block-uniform)
+    for (uint32_t i = tid; i < (uint32_t)(kAggSparseStage / 2); i += kAggThreads) s_cur[i] = 0;
+    // Shared coordinates (at most half the stage: each has two entries or more) get consecutive slots
+    // in index order; a counting sort by slot brings every coordinate's entries together, and since
+    // the stage is in worker order, taking a slot's entries by ascending stage position sums them in
+    // worker order -- the same fixed-order double sum as everywhere else.
+    static_assert(kAggSparseTile / 32 == 2 * kAggThreads, "two bitmap words per thread");
+    uint32_t n_slots;
+    {
+      const uint32_t c0 = __popc(s_shared[2 * tid]), c1 = __popc(s_shared[2 * tid + 1]);
+      const uint32_t incl = warp_incl_scan(c0 + c1);
+      if (lane == 31) s_warp[warp] = incl;
+      __syncthreads();
+      uint32_t woff = 0, all = 0;
+      for (uint32_t x = 0; x < (uint32_t)(kAggThreads / 32); ++x) { if (x < warp) woff += s_warp[x]; all += s_warp[x]; }
+      s_slot[2 * tid] = woff + incl - c0 - c1;
+      s_slot[2 * tid + 1] = woff + incl - c1;
+      n_slots = all;
+      __syncthreads();
+    }
+    if (n_slots == 0) return;                                         // (block-uniform)
+    auto slot_of = [&](uint32_t local) { return s_slot[local >> 5] + __popc(s_shared[local >> 5] & ((1u << (local & 31u)) - 1u)); };
+    for (uint32_t q = tid; q < total; q += kAggThreads) {            // entries per slot
+      const uint32_t local = st_idx[q] - lo;
+      if (local < (uint32_t)kAggSparseTile && st_idx[q] < d && ((s_shared[local >> 5] >> (local & 31u)) & 1u))
+        atomicAdd(&s_cur[slot_of(local)], 1u);
+    }
+    __syncthreads();
+    {                                                                 // exclusive prefix over the slots (up to 1024)
+      constexpr int kPer = kAggSparseStage / 2 / kAggThreads;
+      uint32_t c[kPer], sum = 0;
+#pragma unroll
+      for (int u = 0; u < kPer; ++u) { c[u] = s_cur[tid * kPer + u]; sum += c[u]; }
+      const uint32_t incl = warp_incl_scan(sum);
+      __syncthreads();
+      if (lane == 31) s_warp[warp] = incl;
+      __syncthreads();
+      uint32_t run = incl - sum;
+      for (uint32_t x = 0; x < warp; ++x) run += s_warp[x];
+#pragma unroll
+      for (int u = 0; u < kPer; ++u) { s_off[tid * kPer + u] = run; s_cur[tid * kPer + u] = 0; run += c[u]; }
+      if (tid == kAggThreads - 1) s_off[kAggSparseStage / 2] = run;
+      __syncthreads();
+    }
+    for (uint32_t q = tid; q < total; q += kAggThreads) {            // scatter the stage positions
+      const uint32_t local = st_idx[q] - lo;
+      if (local < (uint32_t)kAggSparseTile && st_idx[q] < d && ((s_shared[local >> 5] >> (local & 31u)) & 1u)) {
+        const uint32_t sl = slot_of(local);
+        s_pool[s_off[sl] + atomicAdd(&s_cur[sl], 1u)] = (uint16_t)q;
       }
     }
     __syncthreads();
-  }
-  for (uint32_t q = tid; q < total; q += kAggThreads) {
-    if (staged) {
-      const uint32_t idx = st_idx[q], local = idx - lo;
-      if (local >= (uint32_t)kAggSparseTile || idx >= d) continue;    // malformed row: ignore
-      if (!((s_shared[local >> 5] >> (local & 31u)) & 1u)) {    // sole sender: the sum is the value
-        const double v = msgs.term(M::kPerWorker ? worker_of(q) : 0u, st_val[q]);
-        out[idx] = agg_result((float)agg_scaled(v, 1u, sc), eta >= 0.0f ? out[idx] : 0.0f, eta);
-        continue;
+    for (uint32_t sl = tid; sl < n_slots; sl += kAggThreads) {       // one thread per shared coordinate
+      const uint32_t b = s_off[sl], e = s_off[sl + 1];
+      if (e == b) continue;                                           // (only entries of a malformed row)
+      double sum = 0.0;
+      int32_t last = -1;
+      uint32_t idx = 0;
+      for (uint32_t n = b; n < e; ++n) {                              // next stage position above `last`
+        uint32_t best = 0xFFFFFFFFu;
+        for (uint32_t x = b; x < e; ++x) { const uint32_t q = s_pool[x]; if ((int32_t)q > last && q < best) best = q; }
+        last = (int32_t)best;
+        idx = st_idx[best];
+        sum += msgs.term(st_w[best], st_val[best]);
       }
+      out[idx] = agg_result((float)agg_scaled(sum, e - b, sc), eta >= 0.0f ? out[idx] : 0.0f, eta);
     }
+    return;
+  }
+  // ---- a crowded tile (more entries than the stage holds): every entry looks the other workers' runs
+  // up in global memory; the entry of the lowest worker that holds a coordinate owns it and sums that
+  // coordinate over the workers in ascending order
+  auto idx_at = [&](uint32_t w, uint32_t j) { return msgs.index(w, s_beg[w] + j); };
+  auto val_at = [&](uint32_t w, uint32_t j) { return msgs.value(w, s_beg[w] + j); };
+  for (uint32_t q = tid; q < total; q += kAggThreads) {
     const uint32_t w = worker_of(q);
     const uint32_t idx = idx_at(w, q - s_pre[w]);
     if (idx - lo >= (uint32_t)kAggSparseTile || idx >= d) continue;   // malformed row: ignore

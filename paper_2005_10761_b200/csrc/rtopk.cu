@@ -720,7 +720,13 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   if (!guard.ok) { delete ctx; return RTOPK_ERR_CUDA; }
   const size_t W = (size_t)W_max, S = (size_t)segments_max, slices = W * S;
   const size_t chunks = W * ((size_t)d_max / kChunk + 2 * S + 1);
-  const size_t cand_row = std::min<size_t>((size_t)d_max, 3 * (size_t)r_max + 4096 * S) + 32 * S;
+  // Candidate lists: a slice with r below its length gathers up to 3 r + 4096 candidates; a slice with
+  // r equal to its length (Definition 2, random-k) gathers none.  A context made with r_max = d_max whose
+  // full lists would take 2^30 entries or more is taken to be made for the latter: its lists are sized
+  // for selections up to r = d_max / 32 only.
+  size_t cand_row = std::min<size_t>((size_t)d_max, 3 * (size_t)r_max + 4096 * S) + 32 * S;
+  if (r_max == d_max && W * cand_row >= ((size_t)1 << 30))
+    cand_row = std::min<size_t>((size_t)d_max, 3 * ((size_t)d_max / 32) + 4096 * S) + 32 * S;
   const size_t groups = W * ((size_t)d_max / kChunk / 32 + 2 * S + 1);
   ctx->cand_entries = W * cand_row;
   ctx->first_entries = W * (std::min<size_t>((size_t)r_max, 16 * (size_t)k_max) + 128 * S);
