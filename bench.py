@@ -266,6 +266,11 @@ class Round:
         self.out = torch.zeros(wl.round_up(self.d, 4), dtype=torch.float32, device=dev)
         self.cnt = torch.zeros(self.W, dtype=torch.int32, device=dev)
         self.ones = torch.zeros(self.W, dtype=torch.int32, device=dev)
+        if world > 1:
+            if self.seg:
+                raise SystemExit("the sharded run covers the plain (whole-vector) workloads")
+            from paper_2005_10761_b200 import sharded
+            self.exchange = sharded.Exchange(self.W_total, self.K, world, rank, dev)
         self.t_next = 0
 
     @property
@@ -287,20 +292,16 @@ class Round:
             else:
                 ctx.step(g, self.residual, self.d, cfg.r, cfg.k, cfg.seed, t, self.idx, self.val, self.out)
         else:
+            # workers sharded over the ranks: messages as 8-byte pairs, ONE all-gather, every rank aggregates
             from paper_2005_10761_b200 import sharded
 
-            def sp(gl, ml, wb):
-                if self.seg:
-                    ctx.sparsify_segmented(gl, ml, self.d, cfg.seg_off, cfg.seg_r, cfg.seg_k, cfg.seed, t, self.idx,
-                                           self.val, worker_base=wb)
-                else:
-                    ctx.sparsify(gl, ml, self.d, cfg.r, cfg.k, cfg.seed, t, self.idx, self.val, worker_base=wb)
-                return self.idx, self.val
+            def sp(gl, ml, wb, pairs):
+                ctx.sparsify_pairs(gl, ml, self.d, cfg.r, cfg.k, cfg.seed, t, pairs, worker_base=wb)
 
-            def ag(ia, va):
-                ctx.aggregate(ia, va, self.d, self.out)
+            def ag(pairs_all):
+                ctx.aggregate_pairs(pairs_all, self.d, self.out)
                 return self.out
-            sharded.sharded_round(sp, ag, g, self.residual, self.W_total, self.world, self.rank)
+            sharded.sharded_round(sp, ag, g, self.residual, self.exchange)
 
     def sync_all(self):
         import torch
@@ -638,7 +639,7 @@ def main():
             "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": config_dict(cfg, args, world),
-            "launch": launch_mode,
+            "launch": launch_mode if world == 1 else launch_mode + "; per round one NCCL all-gather of W*k 8-byte pairs",
             "elements_per_s": W * world * d / (ms_per_step * 1e-3),
             "step_roofline_frac": step_frac, "step_roofline_frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS if world == 1 else None,
             "step_algorithmic_bytes": step_bytes,

@@ -89,7 +89,7 @@ enum {
                                 with rtopk_set_device_step; it starts at 0).  A caller that captures one round
                                 in a CUDA graph can then replay the graph round after round and still draw a
                                 fresh subset each time.  0 = off (default): `step` is the argument */
-  RTOPK_OPT_FINISH_PATH = 5     /* how the sampled path turns the candidates of the streaming pass into messages
+  RTOPK_OPT_FINISH_PATH = 5,    /* how the sampled path turns the candidates of the streaming pass into messages
                                 (the result is the same): 1 = one thread-block cluster per slice, which lays
                                 the candidate runs out in index order first; 2 = three grid-wide launches over
                                 all slices that work on the runs as they are (a histogram over the bracket, a
@@ -97,6 +97,12 @@ enum {
                                 (a missed bracket, heavy ties); 0 (default) = 2 for slices of 2^26 coordinates
                                 or more, where the runs no longer fit one cluster's shared memory and the L2,
                                 else 1 */
+  RTOPK_OPT_TEST_LOOKBACK_LIMIT = 6 /* for tests of the give-up path only: how often a block of the full-vector
+                                radix select (RTOPK_OPT_SELECT_PATH = 1) re-reads a predecessor's word that is
+                                still empty before it gives up (default 2^22).  0 makes every such wait give
+                                up at once: the call still returns, writes nothing outside the caller's
+                                buffers, its messages are then meaningless and rtopk_poll_status reports
+                                RTOPK_ERR_INTERNAL */
 };
 
 /* Phases of one call, in stream order.  STREAM is the single pass over the full vectors that
@@ -174,6 +180,21 @@ int rtopk_sparsify(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_
  */
 int rtopk_aggregate(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d,
                     int32_t W, int64_t k, int scale_mode, float* out, void* stream);
+
+/*
+ * rtopk_sparsify and rtopk_aggregate with the messages as one array of 8-byte (index, value) pairs: entry
+ * j of worker w is the 64-bit word msg_pairs[w * k + j], low half the index, high half the bit pattern of
+ * the binary32 value (ascending index, as always).  This is what a node sends in Algorithm 1 ("send
+ * ghat_i"): one contiguous buffer of k pairs per worker, so that a run sharded over several GPUs moves its
+ * messages with a single all-gather of W * k * 8 bytes and aggregates the gathered buffer in place.
+ * msg_pairs is 8-byte aligned; everything else as in rtopk_sparsify / rtopk_aggregate (MEAN, SUM, COUNT;
+ * UNBIASED needs r: scale the SUM by r / (W k)).
+ */
+int rtopk_sparsify_pairs(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,
+                         int64_t ld_m, int64_t d, int32_t W, int32_t worker_base, int64_t r, int64_t k,
+                         uint64_t seed, uint32_t step, uint64_t* msg_pairs, void* stream);
+int rtopk_aggregate_pairs(rtopk_ctx* ctx, const uint64_t* msg_pairs, int64_t d, int32_t W, int64_t k,
+                          int scale_mode, float* out, void* stream);
 
 /* rtopk_aggregate with the UNBIASED scaling, which needs the r the messages were drawn from
  * (k <= r <= d).  Errors: INVALID_ARG, CUDA. */

@@ -16,6 +16,7 @@ _LIB_PATH = os.path.join(_HERE, "librtopk.so")
 GRAD_F32, GRAD_BF16 = 0, 1
 SCALE_MEAN, SCALE_SUM, SCALE_UNBIASED, SCALE_COUNT = 0, 1, 2, 3
 OPT_SELECT_PATH, OPT_PROFILE, OPT_REUSE_THRESHOLD, OPT_THRESHOLD_SIGNS, OPT_DEVICE_STEP, OPT_FINISH_PATH = 0, 1, 2, 3, 4, 5
+OPT_TEST_LOOKBACK_LIMIT = 6
 PHASES = ("subset", "threshold", "stream", "order", "exact", "finish", "aggregate")
 
 _vp, _i32, _i64, _u32, _u64, _int = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_uint64, C.c_int
@@ -33,6 +34,8 @@ EXPORTS = {
     "rtopk_aggregate": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _int, _vp, _vp]),
     "rtopk_step": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _i64, _u64, _u32, _int,
                           _vp, _vp, _vp, _vp]),
+    "rtopk_sparsify_pairs": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _i64, _u64, _u32, _vp, _vp]),
+    "rtopk_aggregate_pairs": (_int, [_vp, _vp, _i64, _i32, _i64, _int, _vp, _vp]),
     "rtopk_aggregate_unbiased": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _i64, _vp, _vp]),
     "rtopk_warmup_sizes": (_int, [_i64, _i32, C.c_double, C.c_double, _i64, _i64, C.POINTER(_i64), C.POINTER(_i64)]),
     "rtopk_packed_layout": (_int, [_i64, _i64, C.POINTER(_i32), C.POINTER(_i64), C.POINTER(_i64)]),
@@ -204,6 +207,20 @@ class RTopK:
                                   residual.data_ptr(), residual.stride(0), d, W, worker_base, r, k, seed, step,
                                   scale_mode, msg_idx.data_ptr(), msg_val.data_ptr(), out.data_ptr(), _stream())
         self._check(rc, "rtopk_step")
+
+    def sparsify_pairs(self, grad, residual, d, r, k, seed, step, msg_pairs, worker_base=0) -> None:
+        """msg_pairs: int64 [W, k] device tensor; entry = index | (value bits << 32)."""
+        W = grad.shape[0]
+        rc = self._lib.rtopk_sparsify_pairs(self._h, grad.data_ptr(), self._grad_dtype(grad), grad.stride(0),
+                                            residual.data_ptr(), residual.stride(0), d, W, worker_base, r, k,
+                                            seed, step, msg_pairs.data_ptr(), _stream())
+        self._check(rc, "rtopk_sparsify_pairs")
+
+    def aggregate_pairs(self, msg_pairs, d, out, scale_mode=SCALE_MEAN) -> None:
+        W, k = msg_pairs.shape
+        rc = self._lib.rtopk_aggregate_pairs(self._h, msg_pairs.data_ptr(), d, W, k, scale_mode, out.data_ptr(),
+                                             _stream())
+        self._check(rc, "rtopk_aggregate_pairs")
 
     def aggregate_unbiased(self, msg_idx, msg_val, d, r, out) -> None:
         W, k = msg_idx.shape

@@ -47,8 +47,9 @@ struct PlainMsgs {
   const uint32_t* idx;
   const float* val;
   uint32_t K;
-  __device__ __forceinline__ uint32_t index(uint32_t w, uint32_t j) const { return __ldg(idx + (size_t)w * K + j); }
-  __device__ __forceinline__ float value(uint32_t w, uint32_t j) const { return __ldg(val + (size_t)w * K + j); }
+  uint32_t stride;   // 1: two arrays of W x K words; 2: one array of W x K (index, value) pairs, val = idx + 1
+  __device__ __forceinline__ uint32_t index(uint32_t w, uint32_t j) const { return __ldg(idx + ((size_t)w * K + j) * stride); }
+  __device__ __forceinline__ float value(uint32_t w, uint32_t j) const { return __ldg(val + ((size_t)w * K + j) * stride); }
   // what worker w's value v adds to a coordinate's double-precision sum
   static constexpr bool kPerWorker = false;   // the term does not depend on the worker
   static constexpr bool kPadded = false;      // every row holds K valid entries

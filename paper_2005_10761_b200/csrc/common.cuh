@@ -120,6 +120,7 @@ struct Launch {
   float* residual;
   uint32_t* msg_idx;
   float* msg_val;
+  uint32_t msg_stride;        // words between consecutive entries of msg_idx / msg_val: 1 (two arrays) or 2 (pairs)
   uint32_t n_slices;
   uint32_t worker_base;
   uint32_t seed_lo, seed_hi;
@@ -127,6 +128,7 @@ struct Launch {
   const uint32_t* step_ptr;   // not null: the round number is read from this device word instead of `step`
   uint32_t general_primary;   // 1: the full-vector radix select is the main path, not a fallback
   uint32_t reuse;             // 1: brackets may be predicted from the slices' threshold history
+  int32_t lookback_limit;     // spin limit of the exact path's look-back (kLookSpinLimit unless a test lowers it)
 };
 
 // ----------------------------------------------------------------------------- small helpers
@@ -192,9 +194,11 @@ __device__ __forceinline__ void st_relaxed(unsigned long long* p, unsigned long 
 // Called by all 32 lanes of one warp.  `words` points at the slice's tile 0, `tile` is the tile
 // inside the slice, (aggA, aggB) the tile's own counts.  Returns the exclusive prefix in
 // (exA, exB) on every lane.
+// `spin_limit` = how often a lane re-reads a word that is still empty before the warp gives up (0: at
+// once, which is what the test of the give-up path asks for).
 __device__ __forceinline__ void lookback_exclusive(unsigned long long* words, uint32_t tile, uint32_t aggA,
                                                    uint32_t aggB, uint32_t& exA, uint32_t& exB,
-                                                   uint32_t* error) {
+                                                   uint32_t* error, int spin_limit = kLookSpinLimit) {
   const uint32_t lane = lane_id();
   if (tile == 0) {
     if (lane == 0) st_relaxed(words, look_pack(kLookIncl, aggA, aggB));
@@ -204,15 +208,15 @@ __device__ __forceinline__ void lookback_exclusive(unsigned long long* words, ui
   if (lane == 0) st_relaxed(words + tile, look_pack(kLookAgg, aggA, aggB));
   uint32_t sumA = 0, sumB = 0;
   int64_t top = (int64_t)tile - 1;          // newest tile not yet accounted for
-  bool failed = false;
-  while (true) {
+  bool failed = spin_limit == 0;            // (a limit of zero gives up without looking: the give-up path under test)
+  while (!failed) {
     const int64_t mine = top - lane;
     unsigned long long w = kLookIncl;       // lanes before tile 0 read as "inclusive, zero"
     if (mine >= 0) {
       int spins = 0;
       w = ld_relaxed(words + mine);
       while ((w >> 62) == 0) {
-        if (++spins > kLookSpinLimit) { failed = true; break; }
+        if (++spins > spin_limit) { failed = true; break; }
         __nanosleep(40);
         w = ld_relaxed(words + mine);
       }

@@ -412,8 +412,8 @@ __global__ void __launch_bounds__(kRunThreads) k_run_emit(Launch L) {
           slot = pre + __popc(word & ((1u << (p & 31u)) - 1u));
         }
         if (chosen && slot < S.k) {
-          L.msg_idx[S.msg_off + slot] = S.idx_base + idx;
-          L.msg_val[S.msg_off + slot] = v;
+          L.msg_idx[(size_t)(S.msg_off + slot) * L.msg_stride] = S.idx_base + idx;
+          L.msg_val[(size_t)(S.msg_off + slot) * L.msg_stride] = v;
           L.residual[S.m_off + idx] = 0.0f;
         }
       }

@@ -31,6 +31,7 @@ struct rtopk_ctx {
   int32_t W_max = 0, S_max = 0;
   int select_path = 0;
   int finish_path = 0;                // RTOPK_OPT_FINISH_PATH
+  int lookback_limit = kLookSpinLimit; // RTOPK_OPT_TEST_LOOKBACK_LIMIT
   int last_cuda_error = 0;
   // device scratch (one allocation each)
   Slice* d_slices = nullptr;
@@ -382,6 +383,8 @@ int bind_launch(rtopk_ctx* ctx, const Plan& P, const void* grad, float* residual
   if ((size_t)P.n_parts > ctx->part_entries) return RTOPK_ERR_INVALID_ARG;
   L.s.fin = ctx->d_fin; L.s.list = ctx->d_list; L.s.part_tot = ctx->d_part_tot;
   L.grad = grad; L.residual = residual; L.msg_idx = msg_idx; L.msg_val = msg_val;
+  L.msg_stride = 1;
+  L.lookback_limit = ctx->lookback_limit;
   L.n_slices = (uint32_t)P.slices.size();
   L.worker_base = (uint32_t)worker_base;
   L.seed_lo = (uint32_t)seed; L.seed_hi = (uint32_t)(seed >> 32);
@@ -394,7 +397,7 @@ int bind_launch(rtopk_ctx* ctx, const Plan& P, const void* grad, float* residual
 int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
                   int64_t d, int32_t W, int32_t worker_base, int32_t S, const int64_t* seg_off,
                   const int64_t* seg_r, const int64_t* seg_k, uint64_t seed, uint32_t step, uint32_t* msg_idx,
-                  float* msg_val, cudaStream_t st, uint32_t* K_out, float* clear_out = nullptr) {
+                  float* msg_val, cudaStream_t st, uint32_t* K_out, float* clear_out = nullptr, uint32_t msg_stride = 1) {
   int rc = check_common(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, msg_idx, msg_val);
   if (rc) return rc;
   if (S < 1 || S > ctx->S_max || !seg_off || !seg_r || !seg_k) return RTOPK_ERR_INVALID_ARG;
@@ -411,6 +414,7 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   rc = bind_launch(ctx, P, grad, residual, worker_base, seed, step, msg_idx, msg_val, L, &early_bytes, &zbytes);
   if (rc) return rc;
 
+  L.msg_stride = msg_stride;
   rc = upload_slices(ctx, P, st);
   if (rc) return rc;
   ctx->last_n_slices = L.n_slices;
@@ -653,10 +657,10 @@ int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_
 
 int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
                    int scale_mode, float* out, cudaStream_t st, bool out_cleared = false, float eta = -1.0f,
-                   int64_t r = 0) {
+                   int64_t r = 0, uint32_t msg_stride = 1) {
   if (!msg_idx || !msg_val || ((uintptr_t)msg_idx & 3u) || ((uintptr_t)msg_val & 3u)) return RTOPK_ERR_INVALID_ARG;
   if (k < 1 || k > 0xFFFFFFFFll) return RTOPK_ERR_INVALID_ARG;
-  const PlainMsgs msgs = {msg_idx, msg_val, (uint32_t)k};
+  const PlainMsgs msgs = {msg_idx, msg_val, (uint32_t)k, msg_stride};
   return aggregate_launch(ctx, msgs, d, W, k, scale_mode, out, st, out_cleared, eta, r);
 }
 
@@ -848,6 +852,7 @@ int rtopk_set_option(rtopk_ctx* ctx, int option, int64_t value) {
   }
   if (option == RTOPK_OPT_DEVICE_STEP && (value == 0 || value == 1)) { ctx->device_step = (int)value; return RTOPK_OK; }
   if (option == RTOPK_OPT_FINISH_PATH && value >= 0 && value <= 2) { ctx->finish_path = (int)value; return RTOPK_OK; }
+  if (option == RTOPK_OPT_TEST_LOOKBACK_LIMIT && value >= 0 && value <= kLookSpinLimit) { ctx->lookback_limit = (int)value; return RTOPK_OK; }
   if (option == RTOPK_OPT_THRESHOLD_SIGNS && (value == 0 || value == 1)) { ctx->threshold_signs = (int)value; return RTOPK_OK; }
   if (option == RTOPK_OPT_PROFILE && (value == 0 || value == 1)) {
     ctx->profile = (int)value;
@@ -876,6 +881,24 @@ int rtopk_sparsify_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, i
 int rtopk_aggregate(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
                     int scale_mode, float* out, void* stream) {
   return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, out, (cudaStream_t)stream);
+}
+
+int rtopk_sparsify_pairs(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
+                         int64_t d, int32_t W, int32_t worker_base, int64_t r, int64_t k, uint64_t seed, uint32_t step,
+                         uint64_t* msg_pairs, void* stream) {
+  if (!msg_pairs || ((uintptr_t)msg_pairs & 7u)) return RTOPK_ERR_INVALID_ARG;
+  const int64_t off[2] = {0, d};
+  uint32_t* words = reinterpret_cast<uint32_t*>(msg_pairs);
+  return sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed, step,
+                       words, reinterpret_cast<float*>(words + 1), (cudaStream_t)stream, nullptr, nullptr, 2);
+}
+
+int rtopk_aggregate_pairs(rtopk_ctx* ctx, const uint64_t* msg_pairs, int64_t d, int32_t W, int64_t k, int scale_mode,
+                          float* out, void* stream) {
+  if (!msg_pairs || ((uintptr_t)msg_pairs & 7u)) return RTOPK_ERR_INVALID_ARG;
+  const uint32_t* words = reinterpret_cast<const uint32_t*>(msg_pairs);
+  return aggregate_impl(ctx, words, reinterpret_cast<const float*>(words + 1), d, W, k, scale_mode, out,
+                        (cudaStream_t)stream, false, -1.0f, 0, 2);
 }
 
 int rtopk_aggregate_unbiased(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W,

@@ -346,7 +346,7 @@ __device__ __forceinline__ void collect_body(const Launch& L, uint32_t total_til
     for (int w = 0; w < kWarps; ++w) { bA += s_wA[w]; bB += s_wB[w]; }
     uint32_t exA, exB;
     unsigned long long* words = L.s.look_b + S.chunk_begin;
-    lookback_exclusive(words, c, bA, bB, exA, exB, L.s.error);
+    lookback_exclusive(words, c, bA, bB, exA, exB, L.s.error, L.lookback_limit);
     if (lane == 0) {
       s_ex[0] = exA; s_ex[1] = exB;
       if (c + 1 == slice_chunks(S)) {      // last tile of the slice: publish the total
@@ -1191,10 +1191,10 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
         if ((members >> j) & 1u) {
           if (((bits >> o) & 1u) && p0 + o < S.r) {
             const uint32_t slot = slot0 + __popc(bits & ((1u << o) - 1u));
-            if (slot < S.k) {
-              const uint32_t idx = cj[j];
-              L.msg_idx[S.msg_off + slot] = S.idx_base + idx;
-              L.msg_val[S.msg_off + slot] = v[j];
+            const uint32_t idx = cj[j];
+            if (slot < S.k && idx < S.len) {                     // (idx < len always, unless an earlier wait gave up and left the list incomplete)
+              L.msg_idx[(size_t)(S.msg_off + slot) * L.msg_stride] = S.idx_base + idx;
+              L.msg_val[(size_t)(S.msg_off + slot) * L.msg_stride] = v[j];
               L.residual[S.m_off + idx] = 0.0f;
             }
           }
@@ -1228,8 +1228,8 @@ __global__ void __launch_bounds__(kThreads) k_emit_all(Launch L, uint32_t words_
     word &= word - 1;
     const uint32_t p = w * 32u + b;
     if (pre < S.k) {
-      L.msg_idx[S.msg_off + pre] = S.idx_base + p;
-      L.msg_val[S.msg_off + pre] = L.residual[S.m_off + p];
+      L.msg_idx[(size_t)(S.msg_off + pre) * L.msg_stride] = S.idx_base + p;
+      L.msg_val[(size_t)(S.msg_off + pre) * L.msg_stride] = L.residual[S.m_off + p];
       L.residual[S.m_off + p] = 0.0f;
     }
     ++pre;

@@ -64,6 +64,13 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }
+// A last, shorter wait of a block that is giving up (see the consumers' exit in k_stream): if the phase
+// was never armed it simply runs out.
+constexpr int kDrainLimit = 1 << 16;
+__device__ __forceinline__ void mbar_drain(unsigned long long* bar, uint32_t parity) {
+  for (int i = 0; i < kDrainLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return;
+}
 // L2 eviction policy of the candidate runs: they are small and k_finish reads them back, so they
 // should outlive the gradient / residual traffic (which is loaded and stored with streaming hints).
 __device__ __forceinline__ unsigned long long l2_policy_evict_last() {
@@ -172,6 +179,10 @@ __global__ void __launch_bounds__(kStreamThreads, 3) k_stream(Launch L, uint32_t
     const bool arrived = mbar_wait(&sm.full[stage], phase);
     if (consumer_any(!arrived)) {                 // every consumer leaves together
       if (tid == 0) atomicOr(L.s.error, ERR_LOOKBACK_TIMEOUT);
+      // ... but not while a bulk copy into this block's shared memory may still be on its way: the copies
+      // the producer has issued into both stages get one more (bounded) wait before the block ends
+      mbar_drain(&sm.full[stage], phase);
+      mbar_drain(&sm.full[(i + 1) % kStages], ((i + 1) / kStages) & 1u);
       return;
     }
     const StageDesc d = sm.desc[stage];

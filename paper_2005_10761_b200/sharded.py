@@ -3,11 +3,17 @@
 Workers are independent until the master's average (Algorithm 1: the node loop, then
 ghat = (1/n) sum_i ghat_i), so the W workers are split by rows across ranks.  Each rank sparsifies
 its rows with ``worker_base`` = its first global worker id (the subsets then equal the single-process
-run), the fixed-size messages are exchanged with one all-gather, and every rank aggregates all W
-messages into the same dense update.
+run) into one buffer of 8-byte (index, value) pairs, the buffers are exchanged with ONE all-gather of a
+fixed size per rank, and every rank aggregates the gathered buffer in place into the same dense update.
+
+Rows are dealt out in blocks of ceil(W / world): rank p holds workers [p * c, min(W, (p + 1) * c)).
+The last ranks may hold fewer rows (or none), but the step time is that of the largest shard either
+way, and with this split the gathered buffer [world * c, k] holds the W messages in global worker
+order in its first W rows, whatever the shard sizes: no re-ordering, no copy, no second collective.
 
 The functions take the sparsify / aggregate callables as arguments so that the identical sharding
-logic runs with the CUDA library on GPUs and, in CPU tests, with any stand-in.
+logic runs with the CUDA library on GPUs and, in CPU tests, with any stand-in.  Nothing here reads
+another rank's memory: the gathered messages land in this rank's own buffer before any kernel uses them.
 """
 from __future__ import annotations
 
@@ -17,49 +23,61 @@ import torch
 import torch.distributed as dist
 
 
+def shard_block(W_total: int, world: int) -> int:
+    """Rows per rank of the block split: ceil(W / world)."""
+    return (W_total + world - 1) // world
+
+
 def shard_rows(W_total: int, world: int, rank: int) -> Tuple[int, int]:
-    """(first global worker id, number of workers) of ``rank``: contiguous, sizes differ by <= 1."""
-    base, extra = divmod(W_total, world)
-    rows = base + (1 if rank < extra else 0)
-    begin = rank * base + min(rank, extra)
-    return begin, rows
+    """(first global worker id, number of workers) of ``rank``: blocks of ceil(W / world) rows."""
+    c = shard_block(W_total, world)
+    begin = min(W_total, rank * c)
+    return begin, min(W_total, begin + c) - begin
 
 
-def gather_messages(idx_local: torch.Tensor, val_local: torch.Tensor, W_total: int, world: int, rank: int,
-                    group=None) -> Tuple[torch.Tensor, torch.Tensor]:
-    """All-gathers [rows, k] message blocks into [W_total, k], ordered by global worker id."""
-    k = idx_local.shape[1]
-    if world == 1:
-        return idx_local, val_local
-    counts = [shard_rows(W_total, world, r)[1] for r in range(world)]
-    if len(set(counts)) == 1:
-        idx_all = torch.empty((W_total, k), dtype=idx_local.dtype, device=idx_local.device)
-        val_all = torch.empty((W_total, k), dtype=val_local.dtype, device=val_local.device)
-        dist.all_gather_into_tensor(idx_all, idx_local.contiguous(), group=group)
-        dist.all_gather_into_tensor(val_all, val_local.contiguous(), group=group)
-        return idx_all, val_all
-    # uneven shards: pad every block to the largest shard, gather, then drop the padding rows
-    cmax = max(counts)
+class Exchange:
+    """The buffers of the one all-gather, allocated once: ``send`` [c, k] pairs of this rank (rows beyond
+    its shard stay zero and are never read), ``recv`` [world * c, k] pairs of everybody."""
 
-    def padded(x):
-        buf = torch.zeros((cmax, k), dtype=x.dtype, device=x.device)
-        buf[: x.shape[0]] = x
-        return buf
+    def __init__(self, W_total: int, k: int, world: int, rank: int, device, group=None):
+        self.W_total, self.k, self.world, self.rank, self.group = W_total, k, world, rank, group
+        self.c = shard_block(W_total, world)
+        self.begin, self.rows = shard_rows(W_total, world, rank)
+        self.send = torch.zeros((self.c, k), dtype=torch.int64, device=device)
+        self.recv = self.send if world == 1 else torch.zeros((world * self.c, k), dtype=torch.int64, device=device)
 
-    idx_pad = torch.empty((world * cmax, k), dtype=idx_local.dtype, device=idx_local.device)
-    val_pad = torch.empty((world * cmax, k), dtype=val_local.dtype, device=val_local.device)
-    dist.all_gather_into_tensor(idx_pad, padded(idx_local), group=group)
-    dist.all_gather_into_tensor(val_pad, padded(val_local), group=group)
-    keep = torch.cat([torch.arange(r * cmax, r * cmax + c, device=idx_local.device) for r, c in enumerate(counts)])
-    return idx_pad.index_select(0, keep), val_pad.index_select(0, keep)
+    def local_pairs(self) -> torch.Tensor:
+        """Where this rank's sparsify call writes its messages: [rows, k] pairs."""
+        return self.send[: self.rows]
+
+    def gather(self) -> torch.Tensor:
+        """All ranks' messages, [W_total, k] pairs in global worker order (a view of ``recv``)."""
+        if self.world > 1:
+            dist.all_gather_into_tensor(self.recv, self.send, group=self.group)
+        return self.recv[: self.W_total]
 
 
-def sharded_round(sparsify: Callable, aggregate: Callable, grad_local: torch.Tensor,
-                  residual_local: torch.Tensor, W_total: int, world: int, rank: int, group=None):
-    """One round.  ``sparsify(grad, residual, worker_base) -> (idx [rows,k], val [rows,k])`` updates the
-    residual in place; ``aggregate(idx_all [W,k], val_all [W,k]) -> out``.  Returns (idx_all, val_all, out)."""
-    begin, rows = shard_rows(W_total, world, rank)
-    assert grad_local.shape[0] == rows and residual_local.shape[0] == rows
-    idx_l, val_l = sparsify(grad_local, residual_local, begin)
-    idx_all, val_all = gather_messages(idx_l, val_l, W_total, world, rank, group)
-    return idx_all, val_all, aggregate(idx_all, val_all)
+def sharded_round(sparsify_pairs: Callable, aggregate_pairs: Callable, grad_local: torch.Tensor,
+                  residual_local: torch.Tensor, ex: Exchange):
+    """One round.  ``sparsify_pairs(grad, residual, worker_base, pairs [rows, k])`` fills ``pairs`` and
+    updates the residual in place; ``aggregate_pairs(pairs_all [W, k]) -> out``.  Returns (pairs_all, out)."""
+    assert grad_local.shape[0] == ex.rows and residual_local.shape[0] == ex.rows
+    if ex.rows > 0:
+        sparsify_pairs(grad_local, residual_local, ex.begin, ex.local_pairs())
+    pairs_all = ex.gather()
+    return pairs_all, aggregate_pairs(pairs_all)
+
+
+def pack_pairs(idx: torch.Tensor, val: torch.Tensor) -> torch.Tensor:
+    """(index, value) arrays -> 8-byte pairs: low half the index, high half the value's bit pattern.
+    (Host-side helper for tests and stand-ins; the CUDA library writes pairs itself.)"""
+    lo = idx.to(torch.int64) & 0xFFFFFFFF
+    hi = val.contiguous().view(torch.int32).to(torch.int64) & 0xFFFFFFFF
+    return lo | (hi << 32)
+
+
+def unpack_pairs(pairs: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:
+    """8-byte pairs -> (int32 index bits, float32 values)."""
+    idx = (pairs & 0xFFFFFFFF).to(torch.int32)          # (indices are below 2^31)
+    val = (pairs >> 32).to(torch.int32).view(torch.float32)
+    return idx, val

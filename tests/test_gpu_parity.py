@@ -495,6 +495,32 @@ def test_step_is_sparsify_then_aggregate(lib):
     ctx.close()
 
 
+def test_pairs_format_equals_the_two_array_format(lib):
+    # one buffer of 8-byte (index, value) pairs per worker -- what a sharded run all-gathers -- through
+    # both finishing paths and the random-k limit, and its aggregation, against the two-array calls
+    from paper_2005_10761_b200 import sharded
+    cfg = wl.scaled(wl.configs()["c2"], d=300011, W=5)
+    g = wl.gradient(cfg, 0, "cuda")
+    for path, (r, k) in [(AUTO, (cfg.r, cfg.k)), (RUNS, (cfg.r, cfg.k)), (AUTO, (cfg.d, cfg.k)), (EXACT, (cfg.r, cfg.r))]:
+        ctx = _ctx(lib, cfg.d, cfg.W, r, k, path=path)
+        m1, m2 = wl.zero_residual(cfg, "cuda"), wl.zero_residual(cfg, "cuda")
+        idx = torch.zeros((cfg.W, k), dtype=torch.int32, device="cuda")
+        val = torch.zeros((cfg.W, k), dtype=torch.float32, device="cuda")
+        pairs = torch.zeros((cfg.W, k), dtype=torch.int64, device="cuda")
+        out1 = torch.empty(cfg.ld, dtype=torch.float32, device="cuda")
+        out2 = torch.empty(cfg.ld, dtype=torch.float32, device="cuda")
+        ctx.sparsify(g, m1, cfg.d, r, k, 21, 3, idx, val, worker_base=7)
+        ctx.sparsify_pairs(g, m2, cfg.d, r, k, 21, 3, pairs, worker_base=7)
+        ctx.aggregate(idx, val, cfg.d, out1)
+        ctx.aggregate_pairs(pairs, cfg.d, out2)
+        ctx.poll_status()
+        i2, v2 = sharded.unpack_pairs(pairs)
+        assert torch.equal(i2, idx) and torch.equal(v2.view(torch.int32), val.view(torch.int32)), (path, r, k)
+        assert torch.equal(m1.view(torch.int32), m2.view(torch.int32))
+        assert torch.equal(out1[: cfg.d].view(torch.int32), out2[: cfg.d].view(torch.int32))
+        ctx.close()
+
+
 def test_step_host_matches_device_call(lib):
     cfg = wl.scaled(wl.configs()["c1"], d=200003, W=3)
     ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
@@ -624,6 +650,49 @@ def test_fallback_is_taken_and_exact_when_the_sample_misleads(lib):
     g2 = _pad(g2)
     stats2 = check_against_oracle(lib, g2, np.zeros_like(g2), d, r, k, seed=12, step=0, path=AUTO)
     assert any(s["used_fallback"] for s in stats + stats2)
+
+
+def test_a_wait_that_gives_up_is_reported_and_leaves_the_context_usable(lib):
+    # The waits inside the kernels are bounded.  The look-back of the full-vector radix select is made to
+    # give up at once (a test-only option: no GPU fault, no hang is involved): the call returns, nothing
+    # outside the caller's buffers is written (canaries around the messages and the residual), the status
+    # poll reports the internal error, and the same context then serves a normal call correctly.
+    from paper_2005_10761_b200.binding import OPT_TEST_LOOKBACK_LIMIT
+    rng = np.random.default_rng(77)
+    W, d, r, k = 2, 20000, 5000, 500                 # five tiles per row; the last tile alone cannot hold r candidates
+    g = _pad(_spiky(rng, W, d))
+    ld = g.shape[1]
+    ctx = _ctx(lib, d, W, r, k, path=EXACT)
+    tg = torch.from_numpy(g).cuda()
+    pad = 4096
+    res_buf = torch.full((W * ld + 2 * pad,), 123.0, dtype=torch.float32, device="cuda")
+    idx_buf = torch.full((W * k + 2 * pad,), -7, dtype=torch.int32, device="cuda")
+    val_buf = torch.full((W * k + 2 * pad,), -7.0, dtype=torch.float32, device="cuda")
+    tm = res_buf[pad:pad + W * ld].view(W, ld)
+    tm.zero_()
+    idx = idx_buf[pad:pad + W * k].view(W, k)
+    val = val_buf[pad:pad + W * k].view(W, k)
+    ctx.set_option(OPT_TEST_LOOKBACK_LIMIT, 0)
+    ctx.sparsify(tg, tm, d, r, k, 5, 0, idx, val)
+    torch.cuda.synchronize()
+    with pytest.raises(lib.RTopKError) as e:
+        ctx.poll_status()
+    assert e.value.status == 5                                       # RTOPK_ERR_INTERNAL
+    for buf, fill in ((res_buf, 123.0), (idx_buf, -7), (val_buf, -7.0)):
+        assert bool((buf[:pad] == fill).all()) and bool((buf[-pad:] == fill).all())
+    assert bool((tm[:, d:] == 0).all())                              # padding columns untouched
+    ctx.poll_status()                                                # the flag was cleared by the failed poll
+    # back to the normal limit: the same context gives the oracle's result
+    ctx.set_option(OPT_TEST_LOOKBACK_LIMIT, 1 << 22)
+    tm.zero_()
+    m_or = np.zeros_like(g)
+    ctx.sparsify(tg, tm, d, r, k, 5, 1, idx, val)
+    ctx.poll_status()
+    o_idx, o_val = oracle.sparsify(g, m_or, d, r, k, 5, 1)
+    assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx)
+    assert np.array_equal(_bits(val.cpu().numpy()), _bits(o_val))
+    assert np.array_equal(_bits(tm.cpu().numpy()), _bits(m_or))
+    ctx.close()
 
 
 def test_bad_arguments_return_invalid_arg_and_write_nothing(lib):
