@@ -31,6 +31,13 @@
  * Conditions only the device can detect (an internal bounded wait that gave up) are reported by
  * rtopk_poll_status.  A context serialises its scratch memory: calls that share a context must be
  * ordered on one stream (or otherwise not overlap on the GPU).
+ *
+ * A call that only enqueues work may be captured into a CUDA graph (it forks onto a stream of the
+ * context and joins again, which capture follows).  The context keeps the table of the call's
+ * slices on the device and re-sends it only when the shape of the call changes (d, W, segments,
+ * r, k, leading dimensions, worker-independent); a captured graph holds either no such copy or one
+ * from a buffer of the context.  So between the capture and the last replay of the graph make no
+ * call of another shape on that context, or capture again after it.
  */
 #ifndef RTOPK_H_
 #define RTOPK_H_
@@ -92,11 +99,11 @@ enum {
   RTOPK_OPT_FINISH_PATH = 5,    /* how the sampled path turns the candidates of the streaming pass into messages
                                 (the result is the same): 1 = one thread-block cluster per slice, which lays
                                 the candidate runs out in index order first; 2 = three grid-wide launches over
-                                all slices that work on the runs as they are (a histogram over the bracket, a
-                                count, the emission), with the cluster kernel behind them for what they leave
-                                (a missed bracket, heavy ties); 0 (default) = 2 for slices of 2^26 coordinates
-                                or more, where the runs no longer fit one cluster's shared memory and the L2,
-                                else 1 */
+                                all slices that walk the candidate list as the streaming pass left it (a
+                                histogram over the bracket, a count, the emission), with the cluster kernel
+                                behind them for what they leave (a missed bracket, heavy ties); 0 (default) =
+                                2 for calls over 2^27 coordinates or more in all (rows x slice lengths), where
+                                the clusters' serial steps no longer hide behind one another, else 1 */
   RTOPK_OPT_TEST_LOOKBACK_LIMIT = 6 /* for tests of the give-up path only: how often a block of the full-vector
                                 radix select (RTOPK_OPT_SELECT_PATH = 1) re-reads a predecessor's word that is
                                 still empty before it gives up (default 2^22).  0 makes every such wait give

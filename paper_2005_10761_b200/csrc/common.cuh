@@ -52,7 +52,6 @@ struct Slice {
   uint32_t first_mask;  // 0: the table is dense (r entries); else it is a hash table of first_mask + 1 slots
   uint32_t sel_off;     // start in the selection bitmap / its prefix counts (32-bit words)
   uint32_t gshift;      // a chunk group is 2^gshift consecutive chunks (at most kGroupsMax groups per slice)
-  uint32_t part_begin;  // first entry of the slice in the per-block member totals of the run kernels
 };
 
 // Selection state of one slice, advanced kernel by kernel.
@@ -78,12 +77,17 @@ struct TauHistory { uint32_t tau1, tau2; float err; uint32_t valid; };
 
 // Where the run kernels (finish.cuh) stand with one slice.
 constexpr int kListMax = 2048;        // the histogram bucket that holds the r-th largest key is resolved on a list of up to this many candidates
-struct alignas(32) Fin {
+struct alignas(64) Fin {
   uint32_t tau, cut;         // the exact r-th largest key; a key equal to it is a member up to this index
   uint32_t ok;
   uint32_t list_n;           // entries of the slice's short list
-  uint32_t done2;            // chunk groups k_run_count has completed
-  uint32_t pad[3];
+  uint32_t done1, done2;     // blocks of k_run_hist / k_run_count that have completed
+  // the bucket of the bracket's histogram that holds the r-th largest key (k_run_hist's last block):
+  uint32_t b_lo, b_hi;       // keys lo <= key < hi
+  uint32_t b_above;          // candidates above it
+  uint32_t b_n;              // candidates inside it
+  uint32_t b_ok;             // 0: the run kernels do not go on with this slice
+  uint32_t pad[5];
 };
 
 struct Scratch {
@@ -97,7 +101,7 @@ struct Scratch {
   uint32_t* group_total;  // candidates per chunk group (summed by the stream pass)
   uint32_t* chunk_start;  // [chunks] where a chunk's run sits in the raw buffer ...
   uint32_t* chunk_count;  // ... its length ...
-  uint32_t* chunk_pre;    // ... and (threshold encoder) how many marked coordinates precede it in the slice
+  uint32_t* chunk_pre;    // ... and how many marked coordinates (threshold encoder) or members of the top-r set (run kernels) precede it in the slice
   uint32_t* raw_idx;      // candidates in reservation order
   float* raw_val;
   uint32_t* cand_idx;     // candidates in index order
@@ -111,7 +115,6 @@ struct Scratch {
   TauHistory* history;    // [slices] threshold history across calls
   Fin* fin;               // [slices] state of the run kernels
   uint32_t* list;         // [slices][2 * kListMax]: keys, then indices, of the candidates inside the bucket
-  uint32_t* part_tot;     // members per block of k_run_count (Slice::part_begin), then their exclusive prefix
 };
 
 struct Launch {

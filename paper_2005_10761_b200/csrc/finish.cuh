@@ -1,31 +1,32 @@
 // Finishing a slice straight from the runs of the streaming pass (Definition 1's top-r set, then the
 // members Definition 3's subset chose), without laying the candidates out in index order first.
 //
-// The streaming pass leaves, per chunk of 4096 coordinates, a run of candidates (index, value) in
-// index order, and the sampled or predicted bracket [tau_lo, tau_hi] of the r-th largest key.  A
-// histogram of the candidates over the bracket -- 2047 equal buckets plus one for the keys above --
-// gives the bucket that holds the r-th largest key, and that bucket splits the candidates: those above
-// it are members of the top-r set for sure, those below it are not, and the few dozen inside it are
-// decided exactly.  Three grid-wide launches over all slices at once, each about one wave of blocks:
+// The streaming pass leaves the candidates of a slice in one dense list: per chunk of 4096 coordinates
+// a run of (index, value) entries in index order, the runs one behind the other in the order in which
+// the chunks were finished, and per chunk where its run starts.  It also leaves the sampled or predicted
+// bracket [tau_lo, tau_hi] of the r-th largest key.  A histogram of the candidates over the bracket --
+// 2047 equal buckets plus one for the keys above -- gives the bucket that holds the r-th largest key, and
+// that bucket splits the candidates: those above it are members of the top-r set for sure, those below
+// it are not, and the few dozen inside it are decided exactly.  Three grid-wide launches over all slices
+// at once; each walks the LIST in tiles of 2048 entries, eight consecutive entries per thread, so the
+// work is spread evenly however unevenly the candidates are spread over the chunks:
 //
-//   k_run_hist    the histogram (block-local first, the keys above the bracket counted in registers).
-//   k_run_count   every block picks the bucket for itself (8 KB of histogram and one block scan cost
-//                 less than a launch of its own).  Then eight lanes per chunk walk the chunk's run: the
-//                 sure members are counted, the candidates inside the bucket go to a short list with
-//                 their indices.  The last block of a slice finds the r-th element of the whole order --
-//                 larger magnitude first, then lower index -- on the list: its key is the exact
+//   k_run_hist    the histogram (block-local first, the keys above the bracket counted in registers);
+//                 clears the chunks' member counts; the last block of a slice picks the bucket.
+//   k_run_count   the sure members are counted per chunk (a thread adds its eight entries to their
+//                 chunks' counts, one addition per chunk it meets), the candidates inside the bucket go
+//                 to a short list.  The last block of a slice finds the r-th element of the whole order
+//                 -- larger magnitude first, then lower index -- on the list: its key is the exact
 //                 threshold tau, its index the last one at which a key equal to tau still is a member.
-//                 It adds the listed members to their chunks' counts and turns the totals of the chunk
-//                 groups into a prefix.
-//   k_run_emit    eight lanes per chunk again: the position of a member in index order is the number of
-//                 members before it (groups before, chunks before, rank in its run), so the members of a
-//                 run take consecutive positions and their bits lie in two or three words of the
-//                 subset's bitmap, fetched once per run; the chosen ones become messages and their
-//                 residual slots are zeroed.
-// A run holds about 1 % of a chunk, 40 to 50 candidates.  Eight lanes read it one 32-byte sector at a
-// time, four runs per warp: a whole warp per run leaves a third of the lanes idle and costs several
-// times the instructions (these kernels are bound by instruction issue, not by bytes), a thread per run
-// scatters every load over 32 sectors.
+//                 It adds the listed members to their chunks' counts and turns the counts into an
+//                 exclusive prefix over the chunks.
+//   k_run_emit    the position of a member in index order is the number of members before it: those of
+//                 the chunks before (the prefix) plus those before it in its own run (a segmented prefix
+//                 over the tile; for the one run that may reach back into earlier tiles, at most 4095
+//                 entries, the block counts the members among them again).  The members the subset
+//                 chose become messages and their residual slots are zeroed.
+// A block walks several tiles and fetches the next one while it works on the current one: these kernels
+// are chains of dependent memory round trips, and one wave of blocks pays the slice's set-up once.
 //
 // Whatever does not fit this scheme -- the first bracket missed (too few or too many candidates), the
 // r-th largest key lies above the bracket, or more than kListMax candidates share the bucket (heavy
@@ -39,10 +40,10 @@ namespace rtopk {
 
 constexpr int kRunThreads = 256;
 constexpr int kRunWarps = kRunThreads / 32;
-constexpr int kRunChunks = 4;                                // chunks per group (one warp step): members are totalled per group, then per slice
-constexpr int kRunBlockGroups = 32;                          // groups per block (four per warp)
+constexpr int kRunPer = 8;                                   // consecutive list entries per thread
+constexpr int kRunTile = kRunThreads * kRunPer;              // list entries per tile
 constexpr int kHistPer = 8;                                  // candidates per thread and tile of k_run_hist
-constexpr int kRunBatch = 8;                                 // entries of a run a thread reads at a time
+constexpr int kScanPer = 16;                                 // loads in flight per thread of the prefix over the chunks
 constexpr int kRankMax = 512;                                // lists up to this length are ranked by counting
 
 // Exclusive prefix of v over the block's threads, and the block's total.  `s` holds kRunWarps words.
@@ -91,14 +92,21 @@ __device__ __forceinline__ void run_pick(const uint32_t* hist, uint32_t need, ui
 // grid: (blocks per slice, n_slices); a block takes tile after tile of kRunThreads * kHistPer candidates
 __global__ void __launch_bounds__(kRunThreads) k_run_hist(Launch L) {
   __shared__ uint32_t hist[kBins];
+  __shared__ uint32_t s[16];
   const uint32_t sl = blockIdx.y, tid = threadIdx.x, lane = tid & 31u;
   const Slice S = L.s.slices[sl];
-  if (S.r == S.len) return;
   const uint32_t n_cand = L.s.cursor[sl];
-  if (n_cand < S.r || n_cand > S.cand_cap) return;               // the bracket missed: left to k_finish
-  constexpr uint32_t kTile = kRunThreads * kHistPer;
-  if (blockIdx.x * kTile >= n_cand) return;
   const uint32_t tau_lo = L.s.state[sl].tau_lo, tau_hi = max(tau_lo, L.s.state[sl].tau_hi);
+  if (S.r == S.len) return;
+  if (n_cand < S.r || n_cand > S.cand_cap) return;               // the bracket missed: left to k_finish
+  {
+    uint32_t* cm = L.s.chunk_pre + S.chunk_begin;                  // members per chunk: counted by k_run_count
+    const uint32_t nchunks = slice_chunks(S);
+    for (uint32_t c = blockIdx.x * kRunThreads + tid; c < nchunks; c += gridDim.x * kRunThreads) cm[c] = 0;
+  }
+  constexpr uint32_t kTile = kRunThreads * kHistPer;
+  const uint32_t nblocks = min(gridDim.x, (n_cand + kTile - 1u) / kTile);
+  if (blockIdx.x >= nblocks) return;
   const uint32_t sh = bracket_shift(tau_lo, tau_hi);
   for (uint32_t b = tid; b < (uint32_t)kBins; b += kRunThreads) hist[b] = 0;
   __syncthreads();
@@ -122,102 +130,97 @@ __global__ void __launch_bounds__(kRunThreads) k_run_hist(Launch L) {
   __syncthreads();
   uint32_t* gh = L.s.hist + (size_t)sl * kBins;
   for (uint32_t b = tid; b < (uint32_t)kBins; b += kRunThreads) { const uint32_t c = hist[b]; if (c) atomicAdd(gh + b, c); }
-}
-
-// The bucket of the bracket's histogram that holds the r-th largest key.  `ok` is false where the run
-// kernels do not go on.
-struct Bucket { uint32_t lo, hi, above, n; bool ok; };
-__device__ __forceinline__ Bucket run_bucket(const Launch& L, uint32_t sl, const Slice& S, uint32_t* hist, uint32_t* s) {
-  const uint32_t tid = threadIdx.x;
-  const uint32_t n_cand = L.s.cursor[sl];
-  const uint32_t tau_lo = L.s.state[sl].tau_lo, tau_hi = max(tau_lo, L.s.state[sl].tau_hi);
-  const uint32_t* gh = L.s.hist + (size_t)sl * kBins;
+  // the last block of the slice picks the bucket that holds the r-th largest key
+  Fin* F = L.s.fin + sl;
+  __syncthreads();
+  if (tid == 0) {
+    __threadfence();
+    s[15] = atomicAdd(&F->done1, 1u) == nblocks - 1u;
+    if (s[15]) __threadfence();
+  }
+  __syncthreads();
+  if (!s[15]) return;
 #pragma unroll
-  for (int i = 0; i < kBins / kRunThreads; ++i) hist[tid + i * kRunThreads] = gh[tid + i * kRunThreads];
+  for (int i = 0; i < kBins / kRunThreads; ++i) hist[tid + i * kRunThreads] = __ldcg(gh + tid + i * kRunThreads);
   __syncthreads();
   uint32_t D, above;
   run_pick(hist, S.r, s, D, above);
-  const uint32_t sh = bracket_shift(tau_lo, tau_hi);
-  Bucket b;
-  b.ok = n_cand >= S.r && n_cand <= S.cand_cap && D < (uint32_t)(kBins - 1);   // else: missed, or above the bracket
-  b.n = b.ok ? hist[D] : 0u;
-  b.ok = b.ok && b.n <= (uint32_t)kListMax;                                    // else: heavy ties
-  b.lo = tau_lo + (D << sh);
-  b.hi = min(tau_hi + 1u, b.lo + (1u << sh));
-  b.above = above;
-  return b;
+  if (tid != 0) return;
+  const bool in_bracket = D < (uint32_t)(kBins - 1);              // else: the r-th largest key lies above the bracket
+  const uint32_t n = in_bracket ? hist[D] : 0u;
+  const uint32_t lo = tau_lo + (D << sh);
+  F->b_lo = lo;
+  F->b_hi = min(tau_hi + 1u, lo + (1u << sh));
+  F->b_above = above;
+  F->b_n = n;
+  F->b_ok = in_bracket && n <= (uint32_t)kListMax;                // else: heavy ties
 }
 
-// Sum over the four octets' leaders / over an octet (8 neighbouring lanes).
-__device__ __forceinline__ uint32_t octet_sum(uint32_t v) {
-  v += __shfl_xor_sync(0xFFFFFFFFu, v, 4); v += __shfl_xor_sync(0xFFFFFFFFu, v, 2); v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
-  return v;
-}
-__device__ __forceinline__ uint32_t octets_max(uint32_t v) {     // v is the same on the lanes of an octet
-  v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, 8)); v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, 16));
-  return v;
+// Eight consecutive entries of a slice's candidate list, starting at entry i0 (a multiple of 8; the
+// lists start on 128-byte boundaries and their capacities are multiples of 32 entries).
+__device__ __forceinline__ void run_load8(const float* rv, const uint32_t* ri, uint32_t i0, uint32_t n_cand,
+                                          float (&v)[kRunPer], uint32_t (&ix)[kRunPer]) {
+  static_assert(kRunPer == 8, "two 16-byte vectors per array");
+  if (i0 < n_cand) {
+    const float4 a = *reinterpret_cast<const float4*>(rv + i0), b = *reinterpret_cast<const float4*>(rv + i0 + 4);
+    const uint4 c = *reinterpret_cast<const uint4*>(ri + i0), e = *reinterpret_cast<const uint4*>(ri + i0 + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    ix[0] = c.x; ix[1] = c.y; ix[2] = c.z; ix[3] = c.w; ix[4] = e.x; ix[5] = e.y; ix[6] = e.z; ix[7] = e.w;
+  } else {
+#pragma unroll
+    for (int u = 0; u < kRunPer; ++u) { v[u] = 0.f; ix[u] = 0u; }
+  }
 }
 
-// grid: (ceil(most groups of a slice / kRunBlockGroups), n_slices); a warp step is one group of four
-// chunks, eight lanes per chunk
-__global__ void __launch_bounds__(kRunThreads) k_run_count(Launch L) {
+constexpr uint32_t kNoChunk = 0xFFFFFFFFu;
+
+// grid: (blocks per slice, n_slices); a block takes tile after tile of the slice's list
+__global__ void __launch_bounds__(kRunThreads, 4) k_run_count(Launch L) {
+  __shared__ uint32_t hist[kBins];                                 // (last block: rounds over the list)
   __shared__ uint32_t keys[kListMax];
   __shared__ uint32_t idxs[kListMax];
-  __shared__ uint32_t hist[kBins];
   __shared__ uint32_t s[16];
-  const uint32_t sl = blockIdx.y, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  const uint32_t sl = blockIdx.y, tid = threadIdx.x;
   const Slice S = L.s.slices[sl];
-  if (S.r == S.len) return;
-  const uint32_t nchunks = slice_chunks(S);
-  const uint32_t ngroups = (nchunks + kRunChunks - 1) / kRunChunks;
-  const uint32_t nblocks = (ngroups + kRunBlockGroups - 1) / kRunBlockGroups;
-  if (blockIdx.x >= nblocks) return;
-  const Bucket b = run_bucket(L, sl, S, hist, s);
-  if (!b.ok) return;                                             // (the same in every block of the slice)
+  const uint32_t n_cand = L.s.cursor[sl];
   Fin* F = L.s.fin + sl;
-  const uint32_t* cs = L.s.chunk_start + S.chunk_begin;
-  const uint32_t* cc = L.s.chunk_count + S.chunk_begin;
+  const uint32_t b_ok = F->b_ok, b_lo = F->b_lo, b_hi = F->b_hi, b_above = F->b_above, b_n = F->b_n;
+  if (S.r == S.len || !b_ok) return;                               // (the same in every block of the slice)
+  const uint32_t n_tiles = (n_cand + kRunTile - 1) / kRunTile;
+  const uint32_t nblocks = min(gridDim.x, n_tiles);
+  if (blockIdx.x >= nblocks) return;
   uint32_t* cm = L.s.chunk_pre + S.chunk_begin;
   const float* rv = L.s.raw_val + S.cand_off;
   const uint32_t* ri = L.s.raw_idx + S.cand_off;
   uint32_t* lkey = L.s.list + (size_t)sl * 2 * kListMax;
   uint32_t* lidx = lkey + kListMax;
-  uint32_t* pt = L.s.part_tot + S.part_begin;
-  const uint32_t width = b.hi - b.lo;
-  const uint32_t oct = lane >> 3, sub = lane & 7u;
-  const uint32_t g_end = min(ngroups, (blockIdx.x + 1u) * (uint32_t)kRunBlockGroups);
-  uint32_t g = blockIdx.x * (uint32_t)kRunBlockGroups + warp;
-  // the place of the next run is fetched while the current one is walked
-  uint32_t c = g * (uint32_t)kRunChunks + oct;
-  uint32_t start = g < g_end && c < nchunks ? cs[c] : 0u, cnt = g < g_end && c < nchunks ? cc[c] : 0u;
-  for (; g < g_end; g += kRunWarps) {
-    const uint32_t start_c = start, cnt_c = cnt, c_c = c;
-    c = (g + kRunWarps) * (uint32_t)kRunChunks + oct;
-    const bool more = g + kRunWarps < g_end && c < nchunks;
-    start = more ? cs[c] : 0u;
-    cnt = more ? cc[c] : 0u;
-    const uint32_t steps = (octets_max(cnt_c) + 7u) >> 3;
-    uint32_t sure = 0;
-    for (uint32_t st = 0; st < steps; st += 2) {                   // two sectors per lane in flight
-      const uint32_t j0 = st * 8u + sub, j1 = j0 + 8u;
-      const bool in0 = j0 < cnt_c, in1 = j1 < cnt_c;
-      const float x0 = in0 ? rv[start_c + j0] : 0.f, x1 = in1 ? rv[start_c + j1] : 0.f;
-      const uint32_t k0 = mag_key(x0), k1 = mag_key(x1);
-      sure += (in0 && k0 >= b.hi) + (in1 && k1 >= b.hi);
-      if (in0 && k0 - b.lo < width) {                              // inside the bucket: a few dozen per slice
-        const uint32_t at = atomicAdd(&F->list_n, 1u);
-        if (at < (uint32_t)kListMax) { lkey[at] = k0; lidx[at] = ri[start_c + j0]; }
+  const uint32_t width = b_hi - b_lo;
+  float v[kRunPer], vn[kRunPer];
+  uint32_t ix[kRunPer], ixn[kRunPer];
+  run_load8(rv, ri, blockIdx.x * (uint32_t)kRunTile + tid * (uint32_t)kRunPer, n_cand, v, ix);
+  for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    const uint32_t i0 = tile * (uint32_t)kRunTile + tid * (uint32_t)kRunPer;
+    const uint32_t nx = tile + gridDim.x;                          // the next tile is under way while this one is counted
+    run_load8(rv, ri, nx < n_tiles ? nx * (uint32_t)kRunTile + tid * (uint32_t)kRunPer : n_cand, n_cand, vn, ixn);
+    uint32_t cur = kNoChunk, acc = 0;
+#pragma unroll
+    for (int u = 0; u < kRunPer; ++u) {
+      const bool in = i0 + u < n_cand;
+      const uint32_t key = mag_key(v[u]);
+      const uint32_t chunk = in ? (ix[u] + S.head) / (uint32_t)kChunk : kNoChunk;
+      if (chunk != cur) {
+        if (acc) atomicAdd(cm + cur, acc);                         // (acc is zero while cur is no chunk)
+        cur = chunk; acc = 0;
       }
-      if (in1 && k1 - b.lo < width) {
+      acc += in && key >= b_hi;
+      if (in && key - b_lo < width) {                              // inside the bucket: a few dozen per slice
         const uint32_t at = atomicAdd(&F->list_n, 1u);
-        if (at < (uint32_t)kListMax) { lkey[at] = k1; lidx[at] = ri[start_c + j1]; }
+        if (at < (uint32_t)kListMax) { lkey[at] = key; lidx[at] = ix[u]; }
       }
     }
-    sure = octet_sum(sure);
-    if (sub == 0 && c_c < nchunks) cm[c_c] = sure;
-    uint32_t tot = sure;                                           // over the four octets
-    tot += __shfl_xor_sync(0xFFFFFFFFu, tot, 8); tot += __shfl_xor_sync(0xFFFFFFFFu, tot, 16);
-    if (lane == 0) pt[g] = tot;
+    if (acc) atomicAdd(cm + cur, acc);
+#pragma unroll
+    for (int u = 0; u < kRunPer; ++u) { v[u] = vn[u]; ix[u] = ixn[u]; }
   }
   __syncthreads();
   if (tid == 0) {
@@ -230,11 +233,11 @@ __global__ void __launch_bounds__(kRunThreads) k_run_count(Launch L) {
 
   // ---- the last block of the slice: the r-th element on the list, the listed members, the prefix
   SelState* st = &L.s.state[sl];
-  const uint32_t n = __ldcg(&F->list_n), need = S.r - b.above;   // rank of the target inside the bucket, from the top
+  const uint32_t n = __ldcg(&F->list_n), need = S.r - b_above;   // rank of the target inside the bucket, from the top
   auto fail = [&]() {
     if (tid == 0) { atomicOr(L.s.error, ERR_SELECT_INCONSISTENT); st->resolved = 32; }
   };
-  if (n != b.n || n < need) { fail(); return; }                   // cannot happen: the bucket was counted
+  if (n != b_n || n < need) { fail(); return; }                   // cannot happen: the bucket was counted
   for (uint32_t t = tid; t < n; t += kRunThreads) { keys[t] = __ldcg(lkey + t); idxs[t] = __ldcg(lidx + t); }
   __syncthreads();
   if (tid == 0) { s[10] = 0; s[11] = 0; s[12] = 0; s[13] = 0xFFFFFFFFu; }
@@ -252,7 +255,7 @@ __global__ void __launch_bounds__(kRunThreads) k_run_count(Launch L) {
     tau = s[10]; cut = s[11];
   } else {
     // histogram rounds over the list alone (equal buckets over what is left of the interval) ...
-    uint32_t found = b.lo, end = b.hi, rank = need;
+    uint32_t found = b_lo, end = b_hi, rank = need;
     bool ok = true;
     while (end - found > 1u) {
       const uint32_t w = end - found;
@@ -293,34 +296,48 @@ __global__ void __launch_bounds__(kRunThreads) k_run_count(Launch L) {
     __syncthreads();
     cut = s[13];
   }
-  // the listed members join their chunks' and groups' counts
+  // the listed members join their chunks' counts
   uint32_t n_above = 0;
   for (uint32_t t = tid; t < n; t += kRunThreads) {
     n_above += keys[t] > tau;
-    if (keys[t] > tau || (keys[t] == tau && idxs[t] <= cut)) {
-      const uint32_t chunk = (idxs[t] + S.head) / (uint32_t)kChunk;
-      atomicAdd(cm + chunk, 1u);
-      atomicAdd(pt + chunk / (uint32_t)kRunChunks, 1u);
-    }
+    if (keys[t] > tau || (keys[t] == tau && idxs[t] <= cut)) atomicAdd(cm + (idxs[t] + S.head) / (uint32_t)kChunk, 1u);
   }
-  uint32_t dummy;
-  (void)run_block_scan(n_above, s, dummy);
-  const uint32_t n_gt = b.above + dummy, quota = need - dummy;    // keys above tau; keys equal to tau inside the top-r set
+  uint32_t listed_above;
+  (void)run_block_scan(n_above, s, listed_above);
+  const uint32_t n_gt = b_above + listed_above, quota = need - listed_above;   // keys above tau; keys equal to tau inside the top-r set
   __threadfence();
   __syncthreads();
-  // exclusive prefix over the groups' totals, a window of 8 per thread at a time
-  uint32_t carry = 0;
-  for (uint32_t p0 = 0; p0 < ngroups; p0 += 8u * kRunThreads) {
-    uint32_t mine[8], sum = 0;
+  // Exclusive prefix over the chunks' member counts.  A warp takes a contiguous span, 32 chunks at a time
+  // (one line per load: a thread-contiguous split costs 32 memory transactions per load, and this one
+  // block works alone): the spans' totals first, then the prefix inside each span.
+  const uint32_t nchunks = slice_chunks(S);
+  const uint32_t lane = tid & 31u, warp = tid >> 5;
+  const uint32_t span = ((nchunks + kRunWarps * 32u - 1u) / (kRunWarps * 32u)) * 32u;
+  const uint32_t w_lo = min(nchunks, warp * span), w_hi = min(nchunks, w_lo + span);
+  uint32_t sum = 0;
+  for (uint32_t c0 = w_lo; c0 < w_hi; c0 += 32u * kScanPer) {
 #pragma unroll
-    for (int u = 0; u < 8; ++u) { const uint32_t p = p0 + tid * 8u + u; mine[u] = p < ngroups ? __ldcg(pt + p) : 0u; sum += mine[u]; }
-    uint32_t total;
-    uint32_t ex = carry + run_block_scan(sum, s, total);
-#pragma unroll
-    for (int u = 0; u < 8; ++u) { const uint32_t p = p0 + tid * 8u + u; if (p < ngroups) pt[p] = ex; ex += mine[u]; }
-    carry += total;
+    for (int u = 0; u < kScanPer; ++u) { const uint32_t c = c0 + u * 32u + lane; sum += c < w_hi ? __ldcg(cm + c) : 0u; }
   }
-  if (carry != S.r) { fail(); return; }                           // (block-uniform)
+  sum = warp_sum(sum);
+  __syncthreads();
+  if (lane == 0) s[warp] = sum;
+  __syncthreads();
+  uint32_t off = 0, total = 0;
+#pragma unroll
+  for (uint32_t w = 0; w < (uint32_t)kRunWarps; ++w) { const uint32_t x = s[w]; if (w < warp) off += x; total += x; }
+  if (total != S.r) { fail(); return; }                           // (block-uniform)
+  for (uint32_t c0 = w_lo; c0 < w_hi; c0 += 32u * kScanPer) {
+    uint32_t x[kScanPer];
+#pragma unroll
+    for (int u = 0; u < kScanPer; ++u) { const uint32_t c = c0 + u * 32u + lane; x[u] = c < w_hi ? __ldcg(cm + c) : 0u; }
+#pragma unroll
+    for (int u = 0; u < kScanPer; ++u) {
+      const uint32_t c = c0 + u * 32u + lane, incl = warp_incl_scan(x[u]);
+      if (c < w_hi) cm[c] = off + incl - x[u];
+      off += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    }
+  }
   if (tid != 0) return;
   Fin f;
   f.tau = tau; f.cut = cut; f.ok = 1; f.list_n = 0; f.done2 = 0;
@@ -344,80 +361,137 @@ __global__ void __launch_bounds__(kRunThreads) k_run_count(Launch L) {
   }
 }
 
-// grid: as k_run_count
-__global__ void __launch_bounds__(kRunThreads) k_run_emit(Launch L) {
+// Inclusive segmented sum over the block's threads: every thread brings the count of its last segment
+// (`val`) and whether a segment starts inside it (`flag`); returns, for the thread, the count carried
+// into its first entry from the threads before -- the entries since the last segment start there.
+// `s` holds kRunWarps words.  Counts stay below 2^31 (bit 31 carries the flag).
+__device__ __forceinline__ uint32_t run_segmented_carry(uint32_t val, bool flag, uint32_t* s) {
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  uint32_t x = val | (flag ? 0x80000000u : 0u);
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o);
+    if (lane >= (uint32_t)o) x = (x & 0x80000000u) ? x : ((x + (y & 0x7FFFFFFFu)) | (y & 0x80000000u));
+  }
+  __syncthreads();
+  if (lane == 31) s[warp] = x;
+  __syncthreads();
+  uint32_t carry = 0;                                             // from the warps before
+  for (uint32_t w = 0; w < warp; ++w) { const uint32_t y = s[w]; carry = (y & 0x80000000u) ? (y & 0x7FFFFFFFu) : carry + y; }
+  uint32_t ex = __shfl_up_sync(0xFFFFFFFFu, x, 1);                // from the lanes before
+  if (lane == 0) ex = 0;
+  return (ex & 0x80000000u) ? (ex & 0x7FFFFFFFu) : carry + ex;
+}
+
+// grid: (blocks per slice, n_slices); a block takes tile after tile of the slice's list
+__global__ void __launch_bounds__(kRunThreads, 5) k_run_emit(Launch L) {
+  __shared__ uint32_t s[16];
+  __shared__ uint32_t q_idx[kRunWarps][32 * kRunPer];              // per warp: the chosen members of its part of the tile
+  __shared__ float q_val[kRunWarps][32 * kRunPer];
+  __shared__ uint32_t q_pos[kRunWarps][32 * kRunPer];
   const uint32_t sl = blockIdx.y, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   const Slice S = L.s.slices[sl];
-  if (S.r == S.len) return;
-  if (!(L.s.state[sl].flags & FLAG_FINISHED)) return;            // left to k_finish
-  const uint32_t nchunks = slice_chunks(S);
-  const uint32_t ngroups = (nchunks + kRunChunks - 1) / kRunChunks;
-  if (blockIdx.x * (uint32_t)kRunBlockGroups >= ngroups) return;
+  const uint32_t n_cand = L.s.cursor[sl];
+  const uint32_t flags = L.s.state[sl].flags;
   const uint32_t tau = L.s.fin[sl].tau, cut = L.s.fin[sl].cut;
-  const uint32_t* cs = L.s.chunk_start + S.chunk_begin;
-  const uint32_t* cc = L.s.chunk_count + S.chunk_begin;
-  const uint32_t* cm = L.s.chunk_pre + S.chunk_begin;
+  if (S.r == S.len) return;
+  if (!(flags & FLAG_FINISHED)) return;                          // left to k_finish
+  const uint32_t n_tiles = (n_cand + kRunTile - 1) / kRunTile;
+  if (blockIdx.x >= n_tiles) return;
+  const uint32_t* cm = L.s.chunk_pre + S.chunk_begin;              // members in the chunks before
   const uint32_t* ri = L.s.raw_idx + S.cand_off;
   const float* rv = L.s.raw_val + S.cand_off;
   const uint32_t* sel = L.s.sel + S.sel_off;
   const uint32_t* sel_pre = L.s.sel_pre + S.sel_off;
-  const uint32_t* pt = L.s.part_tot + S.part_begin;
   const bool sel_all = S.k == S.r;
-  const uint32_t sel_words = (S.r + 31u) >> 5;
-  const uint32_t oct = lane >> 3, sub = lane & 7u, below = (1u << sub) - 1u;
-  const uint32_t g_end = min(ngroups, (blockIdx.x + 1u) * (uint32_t)kRunBlockGroups);
-  uint32_t g = blockIdx.x * (uint32_t)kRunBlockGroups + warp;
-  // the place and the member counts of the next group are fetched while the current one is walked
-  uint32_t c = g * (uint32_t)kRunChunks + oct;
-  bool has = g < g_end && c < nchunks;
-  uint32_t start = has ? cs[c] : 0u, cnt = has ? cc[c] : 0u, mem = has ? cm[c] : 0u, gbase = g < g_end ? pt[g] : 0u;
-  for (; g < g_end; g += kRunWarps) {
-    const uint32_t start_c = start, cnt_c = cnt, mem_c = mem, gbase_c = gbase;
-    c = (g + kRunWarps) * (uint32_t)kRunChunks + oct;
-    has = g + kRunWarps < g_end && c < nchunks;
-    start = has ? cs[c] : 0u; cnt = has ? cc[c] : 0u; mem = has ? cm[c] : 0u;
-    gbase = g + kRunWarps < g_end ? pt[g + kRunWarps] : 0u;
-    // members before this run: the groups before, then the octets before it in the group
-    const uint32_t m0 = __shfl_sync(0xFFFFFFFFu, mem_c, 0), m1 = __shfl_sync(0xFFFFFFFFu, mem_c, 8),
-                   m2 = __shfl_sync(0xFFFFFFFFu, mem_c, 16);
-    uint32_t p_run = gbase_c + (oct > 0 ? m0 : 0u) + (oct > 1 ? m1 : 0u) + (oct > 2 ? m2 : 0u);
-    // The run's members take positions p_run, p_run + 1, ...: lanes 0..3 of the octet hold the bitmap words
-    // that cover the first of them, lanes 4..7 those words' running popcounts (longer runs read on demand).
-    const uint32_t w0 = p_run >> 5;
-    uint32_t held = 0;
-    if (!sel_all && mem_c) {
-      const uint32_t w = w0 + (sub & 3u);
-      if (w < sel_words) held = sub < 4u ? sel[w] : sel_pre[w];
+  const uint32_t below = (1u << lane) - 1u;
+  auto member = [&](uint32_t key, uint32_t idx) { return key > tau || (key == tau && idx <= cut); };
+  for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    const uint32_t base = tile * (uint32_t)kRunTile, i0 = base + tid * (uint32_t)kRunPer;
+    // Besides its eight entries a thread fetches the entry in front of them (is its first entry the start
+    // of a run?) and one of the 256 entries in front of the tile (the tile's first run may begin there).
+    float v[kRunPer];
+    uint32_t ix[kRunPer];
+    run_load8(rv, ri, i0, n_cand, v, ix);
+    const uint32_t prev = lane == 0 && tid != 0 && i0 < n_cand ? ri[i0 - 1] : 0u;
+    const bool back = base > tid;
+    const float bv = back ? rv[base - 1u - tid] : 0.f;
+    const uint32_t bi = back ? ri[base - 1u - tid] : 0u;
+    // segments: the runs' parts inside the tile.  The tile's first entry starts no segment here.
+    uint32_t bits = 0, heads = 0, chunk_prev = 0;
+#pragma unroll
+    for (int u = 0; u < kRunPer; ++u) {
+      const bool in = i0 + u < n_cand;
+      const uint32_t chunk = in ? (ix[u] + S.head) / (uint32_t)kChunk : kNoChunk;
+      if (in && member(mag_key(v[u]), ix[u])) bits |= 1u << u;
+      if (u > 0 && chunk != chunk_prev) heads |= 1u << u;
+      if (u == 0) {
+        if (tid == 0) s[12] = chunk;
+      }
+      chunk_prev = chunk;
     }
-    const uint32_t steps = (octets_max(cnt_c) + 7u) >> 3;
-    for (uint32_t st = 0; st < steps; ++st) {
-      const uint32_t j = st * 8u + sub;
-      const bool in = j < cnt_c;
-      const float v = in ? rv[start_c + j] : 0.f;
-      const uint32_t idx = in ? ri[start_c + j] : 0u;
-      const uint32_t key = mag_key(v);
-      const bool member = in && (key > tau || (key == tau && idx <= cut));
-      const uint32_t bal = (__ballot_sync(0xFFFFFFFFu, member) >> (oct * 8u)) & 0xFFu;
-      const uint32_t p = p_run + __popc(bal & below);
-      p_run += __popc(bal);
-      const uint32_t k = (p >> 5) - w0;                            // which of the held words (if below 4)
-      uint32_t word = __shfl_sync(0xFFFFFFFFu, held, (oct << 3) + (k & 3u));
-      uint32_t pre = __shfl_sync(0xFFFFFFFFu, held, (oct << 3) + 4u + (k & 3u));
-      if (member && p < S.r) {
-        uint32_t slot = p;
-        bool chosen = true;
-        if (!sel_all) {
-          if (k >= 4u) { word = sel[p >> 5]; pre = sel_pre[p >> 5]; }
-          chosen = (word >> (p & 31u)) & 1u;
-          slot = pre + __popc(word & ((1u << (p & 31u)) - 1u));
-        }
-        if (chosen && slot < S.k) {
-          L.msg_idx[(size_t)(S.msg_off + slot) * L.msg_stride] = S.idx_base + idx;
-          L.msg_val[(size_t)(S.msg_off + slot) * L.msg_stride] = v;
-          L.residual[S.m_off + idx] = 0.0f;
-        }
+    {
+      uint32_t before = __shfl_up_sync(0xFFFFFFFFu, chunk_prev, 1);   // the last chunk of the thread in front
+      if (lane == 0) before = (prev + S.head) / (uint32_t)kChunk;
+      const uint32_t first = i0 < n_cand ? (ix[0] + S.head) / (uint32_t)kChunk : kNoChunk;
+      if (tid != 0 && first != before) heads |= 1u;
+    }
+    // the members of the chunks before, for every member (neighbours ask for the same word)
+    uint32_t p[kRunPer];
+#pragma unroll
+    for (int u = 0; u < kRunPer; ++u) p[u] = (bits >> u) & 1u ? cm[(ix[u] + S.head) / (uint32_t)kChunk] : 0u;
+    // members of the thread's last segment, and the count carried in from the threads before
+    const uint32_t last = heads ? 31u - (uint32_t)__clz(heads) : 0u;
+    const uint32_t carry = run_segmented_carry((uint32_t)__popc(bits >> last), heads != 0u, s);
+    // the tile's first run in front of the tile: its members are counted again.  Its entries there are the
+    // ones next to the tile that lie in the same chunk; a run longer than the 256 fetched is walked on.
+    const uint32_t c_first = s[12];
+    const bool same = back && (bi + S.head) / (uint32_t)kChunk == c_first;
+    uint32_t before = (uint32_t)__syncthreads_count(same && member(mag_key(bv), bi));
+    uint32_t reach = (uint32_t)__syncthreads_count(same);
+    for (uint32_t off = kRunThreads; reach == off && off < (uint32_t)kChunk; off += kRunThreads) {
+      const bool in = base > off + tid;
+      const uint32_t idx = in ? ri[base - 1u - off - tid] : 0u;
+      const bool more = in && (idx + S.head) / (uint32_t)kChunk == c_first;
+      before += (uint32_t)__syncthreads_count(more && member(mag_key(rv[base - 1u - off - tid]), idx));
+      reach += (uint32_t)__syncthreads_count(more);
+    }
+    // positions, then which of them the subset chose
+    uint32_t rank = carry, words[kRunPer];
+#pragma unroll
+    for (int u = 0; u < kRunPer; ++u) {
+      if ((heads >> u) & 1u) rank = 0;
+      if ((bits >> u) & 1u) {
+        p[u] += rank + ((ix[u] + S.head) / (uint32_t)kChunk == c_first ? before : 0u);
+        ++rank;
+        if (p[u] >= S.r) bits &= ~(1u << u);                       // (cannot happen: exactly r members)
       }
     }
+#pragma unroll
+    for (int u = 0; u < kRunPer; ++u) words[u] = !sel_all && ((bits >> u) & 1u) ? sel[p[u] >> 5] : 0xFFFFFFFFu;
+    uint32_t qn = 0;
+#pragma unroll
+    for (int u = 0; u < kRunPer; ++u) {
+      const bool chosen = ((bits >> u) & 1u) && ((words[u] >> (p[u] & 31u)) & 1u);
+      const uint32_t bal = __ballot_sync(0xFFFFFFFFu, chosen);
+      if (chosen) {
+        const uint32_t at = qn + (uint32_t)__popc(bal & below);
+        q_idx[warp][at] = ix[u]; q_val[warp][at] = v[u]; q_pos[warp][at] = p[u];
+      }
+      qn += (uint32_t)__popc(bal);
+    }
+    __syncwarp();
+    for (uint32_t q = lane; q < qn; q += 32u) {
+      const uint32_t pos = q_pos[warp][q], idx = q_idx[warp][q];
+      uint32_t slot = pos;
+      if (!sel_all) slot = sel_pre[pos >> 5] + (uint32_t)__popc(sel[pos >> 5] & ((1u << (pos & 31u)) - 1u));
+      if (slot < S.k) {
+        L.msg_idx[(size_t)(S.msg_off + slot) * L.msg_stride] = S.idx_base + idx;
+        L.msg_val[(size_t)(S.msg_off + slot) * L.msg_stride] = q_val[warp][q];
+        L.residual[S.m_off + idx] = 0.0f;
+      }
+    }
+    __syncwarp();
   }
 }
 

@@ -55,8 +55,6 @@ struct rtopk_ctx {
   uint32_t* d_error = nullptr;
   Fin* d_fin = nullptr;              // per-slice state of the run kernels
   uint32_t* d_list = nullptr;        // per-slice short lists (keys, indices)
-  uint32_t* d_part_tot = nullptr;    // per-block member totals of the run kernels
-  size_t part_entries = 0;
   TauHistory* d_history = nullptr;   // per-slice threshold history (RTOPK_OPT_REUSE_THRESHOLD)
   int reuse = 0;
   int threshold_signs = 0;            // RTOPK_OPT_THRESHOLD_SIGNS
@@ -78,6 +76,8 @@ struct rtopk_ctx {
   cudaEvent_t ev_downloaded = nullptr;               // the results of the last call are in host memory
   int stage_next = 0;
   std::vector<Slice> cached_slices;   // what d_slices currently holds
+  Slice* h_slices = nullptr;          // pinned copy of the table: the source of an upload that is captured into a graph
+  size_t slices_max = 0;
   uint32_t last_n_slices = 0;
   // optional per-phase timing (RTOPK_OPT_PROFILE): events recorded on the caller's stream
   int sms = 0;
@@ -146,7 +146,7 @@ uint64_t first_table_entries(Slice& sl) {
 // Layout of one call: the slice table plus every per-call scratch offset.
 struct Plan {
   std::vector<Slice> slices;
-  uint32_t n_chunks = 0, n_hist_blocks = 0, n_groups = 0, n_parts = 0;
+  uint32_t n_chunks = 0, n_hist_blocks = 0, n_groups = 0;
   size_t cand_entries = 0, draw_entries = 0, first_entries = 0, sel_words = 0;
   uint32_t k_draw_max = 0, words_all_max = 0, cap_max = 0, chunks_max = 0, sel_words_max = 0;
   bool any_select = false, any_sampler = false, any_all = false;
@@ -172,7 +172,7 @@ int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32
   P.K_row = (uint32_t)K;
   P.uniform = (S == 1);
   P.slices.resize((size_t)W * (size_t)S);
-  uint64_t chunks = 0, hblocks = 0, groups = 0, cand = 0, draws = 0, first = 0, selw = 0, parts = 0;
+  uint64_t chunks = 0, hblocks = 0, groups = 0, cand = 0, draws = 0, first = 0, selw = 0;
   for (int w = 0; w < W; ++w) {
     uint64_t msg_at = (uint64_t)w * K;
     for (int s = 0; s < S; ++s) {
@@ -202,8 +202,6 @@ int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32
       while (((nchunks + (1u << sl.gshift) - 1) >> sl.gshift) > (uint32_t)kGroupsMax) ++sl.gshift;
       sl.group_begin = (uint32_t)groups;
       groups += (nchunks + (1u << sl.gshift) - 1) >> sl.gshift;
-      sl.part_begin = (uint32_t)parts;
-      parts += (nchunks + kRunChunks - 1) / kRunChunks;
       sl.cand_off = (uint32_t)cand;
       if (sl.r < sl.len || always_gather) {
         sl.cand_cap = cand_capacity(sl.len, sl.r);
@@ -231,7 +229,6 @@ int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32
   }
   if (chunks >= (1ull << 31) || cand >= (1ull << 32) || first >= (1ull << 32)) return RTOPK_ERR_INVALID_ARG;
   P.n_chunks = (uint32_t)chunks; P.n_hist_blocks = (uint32_t)hblocks; P.n_groups = (uint32_t)groups;
-  P.n_parts = (uint32_t)parts;
   P.cand_entries = cand; P.draw_entries = draws; P.first_entries = first; P.sel_words = selw;
   return RTOPK_OK;
 }
@@ -341,7 +338,17 @@ int upload_slices(rtopk_ctx* ctx, const Plan& P, cudaStream_t st) {
   if (ctx->cached_slices.size() == P.slices.size() &&
       std::memcmp(ctx->cached_slices.data(), P.slices.data(), bytes) == 0)
     return RTOPK_OK;
-  RTOPK_CUDA(ctx, cudaMemcpyAsync(ctx->d_slices, P.slices.data(), bytes, cudaMemcpyHostToDevice, st));
+  // An eager copy from pageable memory has left the source when the call returns; a captured one reads
+  // its source at every replay, so it gets a buffer that lives as long as the context.
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (st != nullptr) RTOPK_CUDA(ctx, cudaStreamIsCapturing(st, &cap));
+  const Slice* src = P.slices.data();
+  if (cap != cudaStreamCaptureStatusNone) {
+    if (P.slices.size() > ctx->slices_max) return RTOPK_ERR_INVALID_ARG;
+    std::memcpy(ctx->h_slices, P.slices.data(), bytes);
+    src = ctx->h_slices;
+  }
+  RTOPK_CUDA(ctx, cudaMemcpyAsync(ctx->d_slices, src, bytes, cudaMemcpyHostToDevice, st));
   ctx->cached_slices = P.slices;
   ctx->history_stale = true;          // other slices: what was learnt about the old ones does not apply
   return RTOPK_OK;
@@ -380,8 +387,7 @@ int bind_launch(rtopk_ctx* ctx, const Plan& P, const void* grad, float* residual
   L.s.chunk_pre = ctx->d_chunk_tab + 2 * ctx->chunk_tab_entries;
   L.s.draws = ctx->d_draws; L.s.first = ctx->d_first; L.s.sel_pre = ctx->d_sel_pre; L.s.sel_blk = ctx->d_sel_blk;
   L.s.error = ctx->d_error;
-  if ((size_t)P.n_parts > ctx->part_entries) return RTOPK_ERR_INVALID_ARG;
-  L.s.fin = ctx->d_fin; L.s.list = ctx->d_list; L.s.part_tot = ctx->d_part_tot;
+  L.s.fin = ctx->d_fin; L.s.list = ctx->d_list;
   L.grad = grad; L.residual = residual; L.msg_idx = msg_idx; L.msg_val = msg_val;
   L.msg_stride = 1;
   L.lookback_limit = ctx->lookback_limit;
@@ -459,11 +465,11 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   rc = grad_dtype == RTOPK_F32 ? launch_select<float>(ctx, P, L, st, join, clear_late, clear_bytes)
                                : launch_select<__nv_bfloat16>(ctx, P, L, st, join, clear_late, clear_bytes);
   if (rc) return rc;
-  // (on the sampled path the exact kernel's launch has already waited for the side stream)
+  // (on the sampled path launch_select has made the stream wait for the side stream before its last kernel)
   const bool joined = forked && ctx->select_path == 0;
   if (forked && !joined) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0));
   mark(ctx, RTOPK_PHASE_FINISH, st);
-  const bool from_runs = ctx->finish_path == 2 || (ctx->finish_path == 0 && P.chunks_max >= (1u << 14));
+  const bool from_runs = ctx->finish_path == 2 || (ctx->finish_path == 0 && P.n_chunks >= (1u << 15));
   if (P.any_select && ctx->select_path == 0 && from_runs && L.n_slices <= 65535u) {
     // the usual case is finished straight from the streaming pass's runs, all slices side by side; what
     // these kernels leave (a missed bracket, heavy ties) is flagged for k_finish
@@ -472,10 +478,12 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
     const uint32_t tiles = (P.cap_max + kRunThreads * kHistPer - 1) / (kRunThreads * kHistPer);
     const dim3 hgrid(std::min(tiles, per_slice), L.n_slices);
     k_run_hist<<<hgrid, kRunThreads, 0, st>>>(L);
-    const uint32_t groups = (P.chunks_max + kRunChunks - 1) / kRunChunks;
-    const dim3 rgrid((groups + kRunBlockGroups - 1) / kRunBlockGroups, L.n_slices);
+    const uint32_t per_slice_run = std::max<uint32_t>(1u, ((uint32_t)ctx->sms * 4u + L.n_slices - 1u) / L.n_slices);
+    const dim3 rgrid(std::min((P.cap_max + kRunTile - 1) / (uint32_t)kRunTile, per_slice_run), L.n_slices);
     k_run_count<<<rgrid, kRunThreads, 0, st>>>(L);
-    k_run_emit<<<rgrid, kRunThreads, 0, st>>>(L);
+    const uint32_t per_slice_emit = std::max<uint32_t>(1u, ((uint32_t)ctx->sms * 5u + L.n_slices - 1u) / L.n_slices);
+    const dim3 egrid(std::min((P.cap_max + kRunTile - 1) / (uint32_t)kRunTile, per_slice_emit), L.n_slices);
+    k_run_emit<<<egrid, kRunThreads, 0, st>>>(L);
     ctx->launches += 3;
   }
   if (P.any_select) {
@@ -741,6 +749,8 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   cudaError_t e = cudaSuccess;
   auto alloc = [&](void** p, size_t bytes) { if (e == cudaSuccess) e = cudaMalloc(p, bytes ? bytes : 16); };
   alloc((void**)&ctx->d_slices, slices * sizeof(Slice));
+  ctx->slices_max = slices;
+  if (e == cudaSuccess) e = cudaMallocHost((void**)&ctx->h_slices, slices * sizeof(Slice));
   alloc((void**)&ctx->d_state, slices * sizeof(SelState));
   alloc((void**)&ctx->d_zero, ctx->zero_bytes);
   alloc((void**)&ctx->d_first, ctx->first_entries * sizeof(uint32_t));
@@ -757,8 +767,6 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   alloc((void**)&ctx->d_error, 16);
   alloc((void**)&ctx->d_fin, slices * sizeof(Fin));
   alloc((void**)&ctx->d_list, slices * 2 * kListMax * sizeof(uint32_t));
-  ctx->part_entries = chunks / kRunChunks + slices + 1;
-  alloc((void**)&ctx->d_part_tot, ctx->part_entries * sizeof(uint32_t));
   alloc((void**)&ctx->d_step, 16);
   alloc((void**)&ctx->d_history, slices * sizeof(TauHistory));
   alloc((void**)&ctx->d_agg_starts, ctx->agg_start_entries * sizeof(uint32_t));
@@ -823,8 +831,9 @@ int rtopk_destroy(rtopk_ctx* ctx) {
   void* ptrs[] = {ctx->d_slices, ctx->d_state, ctx->d_zero, ctx->d_first, ctx->d_cand_idx, ctx->d_cand_val,
                   ctx->d_raw_idx, ctx->d_raw_val, ctx->d_chunk_tab,
                   ctx->d_draws, ctx->d_sel_pre, ctx->d_sel_blk, ctx->d_error, ctx->d_agg_starts, ctx->d_stage, ctx->d_history,
-                  ctx->d_step, ctx->d_fin, ctx->d_list, ctx->d_part_tot};
+                  ctx->d_step, ctx->d_fin, ctx->d_list};
   for (void* p : ptrs) if (p) cudaFree(p);
+  if (ctx->h_slices) cudaFreeHost(ctx->h_slices);
   for (cudaEvent_t ev : ctx->ev) if (ev) cudaEventDestroy(ev);
   if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
   if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);

@@ -37,7 +37,7 @@ __device__ __forceinline__ void clear_slice_counters(const Launch& L, uint32_t s
   const uint32_t nchunks = slice_chunks(S);
   const uint32_t ngroups = (nchunks + (1u << S.gshift) - 1u) >> S.gshift;
   for (uint32_t g = t; g < ngroups; g += nt) L.s.group_total[S.group_begin + g] = 0;
-  if (t == 0) { L.s.cursor[sl] = 0; L.s.done[sl] = 0; L.s.fin[sl].list_n = 0; L.s.fin[sl].done2 = 0; }
+  if (t == 0) { L.s.cursor[sl] = 0; L.s.done[sl] = 0; L.s.fin[sl].list_n = 0; L.s.fin[sl].done1 = 0; L.s.fin[sl].done2 = 0; L.s.fin[sl].b_ok = 0; }
   if (sl == 0 && t < 4u) L.s.tickets[t] = 0;
 }
 

@@ -753,6 +753,39 @@ def test_step_can_be_captured_in_a_cuda_graph_and_replayed(lib):
     assert np.array_equal(_bits(out.cpu().numpy()[:cfg.d]), _bits(o32))
 
 
+def test_a_captured_first_call_sends_its_slice_table_from_the_context(lib):
+    # The first call of a shape sends the table of its slices to the device.  When that call is captured, the
+    # copy in the graph reads a buffer of the context (not one of the call), so replays long after the call
+    # has returned still send the right table.
+    cfg = wl.scaled(wl.configs()["c2"], d=300017, W=2)
+    ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
+    g = wl.gradient(cfg, 0, "cuda")
+    m = wl.zero_residual(cfg, "cuda")
+    idx = torch.zeros((cfg.W, cfg.k), dtype=torch.int32, device="cuda")
+    val = torch.zeros((cfg.W, cfg.k), dtype=torch.float32, device="cuda")
+    out = torch.zeros(wl.round_up(cfg.d, 4), dtype=torch.float32, device="cuda")
+    s = torch.cuda.Stream()
+    m_or = np.zeros((cfg.W, cfg.ld), dtype=np.float32)
+    with torch.cuda.stream(s):
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=s):
+            ctx.step(g, m, cfg.d, cfg.r, cfg.k, cfg.seed, 3, idx, val, out)   # the context's very first call
+        junk = [torch.empty(1 << 20, dtype=torch.uint8).random_() for _ in range(8)]   # host allocations come and go
+        del junk
+        for _ in range(2):                                                   # same step both times: residual carried
+            graph.replay()
+            torch.cuda.synchronize()
+            ctx.poll_status()
+            o_idx, o_val = oracle.sparsify(g.cpu().numpy(), m_or, cfg.d, cfg.r, cfg.k, cfg.seed, 3)
+            _, o32 = oracle.aggregate(o_idx, o_val, cfg.d)
+            assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx)
+            assert np.array_equal(_bits(val.cpu().numpy()), _bits(o_val))
+            assert np.array_equal(_bits(m.cpu().numpy()), _bits(m_or))
+            assert np.array_equal(_bits(out.cpu().numpy()[:cfg.d]), _bits(o32))
+    ctx.close()
+
+
 @pytest.mark.parametrize("case", range(24))
 def test_random_shapes_values_and_paths(lib, case):
     # Seeded random draws of everything a caller chooses: length, workers, r, k, first worker id, step,
