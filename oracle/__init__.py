@@ -44,6 +44,7 @@ def lib() -> C.CDLL:
         L = C.CDLL(_LIB)
         u32p, f32p, f64p, i64p = (C.POINTER(C.c_uint32), C.POINTER(C.c_float),
                                   C.POINTER(C.c_double), C.POINTER(C.c_int64))
+        u16p = C.POINTER(C.c_uint16)
         L.oracle_set_threads.argtypes = [C.c_int]
         L.oracle_get_threads.restype = C.c_int
         L.oracle_philox4x32_10.argtypes = [u32p, u32p, u32p]
@@ -67,9 +68,14 @@ def lib() -> C.CDLL:
                                               C.c_int64, f64p, f32p]
         L.oracle_apply_update.argtypes = [u32p, f32p, C.c_int64, C.c_int32, C.c_int64, C.c_int,
                                           C.c_int64, C.c_float, f32p]
+        L.oracle_apply_momentum.argtypes = [u32p, f32p, C.c_int64, C.c_int32, C.c_int64, C.c_int, C.c_int64,
+                                            C.c_float, C.c_float, f32p, f32p]
+        L.oracle_tiled_spans.argtypes = [C.c_int64]
+        L.oracle_tiled_spans.restype = C.c_int64
+        L.oracle_encode_tiled_row.argtypes = [u32p, f32p, C.c_int64, C.c_int64, u32p, u16p, u16p, f32p]
+        L.oracle_decode_tiled_row.argtypes = [u32p, u16p, u16p, C.c_int64, C.c_int64, u32p, f32p]
         L.oracle_warmup_sizes.argtypes = [C.c_int64, C.c_int32, C.c_double, C.c_double, C.c_int64, C.c_int64,
                                           i64p, i64p]
-        u16p = C.POINTER(C.c_uint16)
         L.oracle_index_bits.argtypes = [C.c_int64]
         L.oracle_bf16_rne.argtypes = [C.c_float]
         L.oracle_bf16_rne.restype = C.c_uint16
@@ -207,6 +213,21 @@ def apply_update(msg_idx: np.ndarray, msg_val: np.ndarray, d: int, eta: float, w
     return w
 
 
+def apply_momentum(msg_idx: np.ndarray, msg_val: np.ndarray, d: int, eta: float, mu: float, velocity: np.ndarray,
+                   weights: np.ndarray, scale_mode: int = SCALE_MEAN, r: int = 0):
+    """Heavy-ball master update v <- mu v + ghat, w <- w - eta v on copies of `velocity` and `weights`
+    (float32 [d]); returns (velocity, weights)."""
+    idx = np.ascontiguousarray(msg_idx, dtype=np.uint32)
+    val = np.ascontiguousarray(msg_val, dtype=np.float32)
+    W, k = idx.shape
+    v = np.array(velocity, dtype=np.float32, copy=True)
+    w = np.array(weights, dtype=np.float32, copy=True)
+    _check(lib().oracle_apply_momentum(_p(idx, C.c_uint32), _p(val, C.c_float), d, W, k, scale_mode, r,
+                                       C.c_float(eta), C.c_float(mu), _p(v, C.c_float), _p(w, C.c_float)),
+           "apply_momentum")
+    return v, w
+
+
 def warmup_sizes(d: int, n: int, initial: float, final: float, warmup_steps: int, step: int):
     r, k = C.c_int64(0), C.c_int64(0)
     _check(lib().oracle_warmup_sizes(d, n, initial, final, warmup_steps, step, C.byref(r), C.byref(k)), "warmup_sizes")
@@ -250,6 +271,41 @@ def decode(packed_idx: np.ndarray, packed_val: np.ndarray, d: int, k: int):
     for w in range(W):
         _check(lib().oracle_decode_row(_p(pi[w], C.c_uint32), _p(pv[w], C.c_uint16), k, d, _p(idx[w], C.c_uint32),
                                        _p(val[w], C.c_float)), "decode_row")
+    return idx, val
+
+
+def tiled_spans(d: int) -> int:
+    return int(lib().oracle_tiled_spans(d))
+
+
+def encode_tiled(msg_idx: np.ndarray, msg_val: np.ndarray, d: int, residual: np.ndarray | None = None):
+    """Span-table form of W ascending rows of k (index, value) pairs: (uint32 [W, T + 1] table,
+    uint16 [W, k] low index bits, uint16 [W, k] bfloat16 values).  When ``residual`` (float32 [W, ld]) is
+    given, the bfloat16 rounding error is written to the sent coordinates' slots in place."""
+    idx = np.ascontiguousarray(msg_idx, dtype=np.uint32)
+    val = np.ascontiguousarray(msg_val, dtype=np.float32)
+    W, k = idx.shape
+    T = tiled_spans(d)
+    tab = np.zeros((W, T + 1), dtype=np.uint32)
+    low = np.zeros((W, k), dtype=np.uint16)
+    qv = np.zeros((W, k), dtype=np.uint16)
+    for w in range(W):
+        res = None if residual is None else residual[w].ctypes.data_as(C.POINTER(C.c_float))
+        _check(lib().oracle_encode_tiled_row(_p(idx[w], C.c_uint32), _p(val[w], C.c_float), k, d, _p(tab[w], C.c_uint32),
+                                             _p(low[w], C.c_uint16), _p(qv[w], C.c_uint16), res), "encode_tiled_row")
+    return tab, low, qv
+
+
+def decode_tiled(tab: np.ndarray, low: np.ndarray, qval: np.ndarray, d: int, k: int):
+    tab = np.ascontiguousarray(tab, dtype=np.uint32)
+    low = np.ascontiguousarray(low, dtype=np.uint16)
+    qv = np.ascontiguousarray(qval, dtype=np.uint16)
+    W = tab.shape[0]
+    idx = np.zeros((W, k), dtype=np.uint32)
+    val = np.zeros((W, k), dtype=np.float32)
+    for w in range(W):
+        _check(lib().oracle_decode_tiled_row(_p(tab[w], C.c_uint32), _p(low[w], C.c_uint16), _p(qv[w], C.c_uint16), k, d,
+                                             _p(idx[w], C.c_uint32), _p(val[w], C.c_float)), "decode_tiled_row")
     return idx, val
 
 

@@ -38,7 +38,11 @@
 // Proposition 1 and the limits k = r (Def. 1) and r = d (Def. 2); the
 // threshold-then-subsample encoder (proof of Theorem 1) against a library
 // comparison of magnitudes, exhaustive enumeration of the kept subsets, the
-// exact unbiasedness of its estimator and the identity sum(X~ / S) = ||X||_1.
+// exact unbiasedness of its estimator and the identity sum(X~ / S) = ||X||_1;
+// the momentum form of the master update against worked steps in exact binary
+// fractions, its mu = 0 limit, a library optimizer run in binary64 and the
+// geometric series; the span-table message format against a hand-worked row, a
+// library lower-bound search, the bit-packed format and bfloat16 of a library.
 
 #include <algorithm>
 #include <cmath>
@@ -327,6 +331,27 @@ int oracle_apply_update(const uint32_t* msg_idx, const float* msg_val, int64_t d
   return ORACLE_OK;
 }
 
+// Section IV trains with momentum SGD.  The paper prints no formula for it; the reading taken is the
+// heavy-ball form on the master, applied to the average of Algorithm 1:
+//     v <- mu * v + ghat ;   w <- w - eta * v        for every coordinate, sent or not
+// (with mu = 0 it is the master update above).  Each of the two lines rounds once from binary64:
+// v' = fp32(double(mu) * double(v) + double(ghat)) -- the product is exact in binary64, the sum is
+// rounded to binary64 and then to binary32 -- and w' = fp32(double(w) - double(eta) * double(v')).
+// 0 <= mu < 1, eta >= 0.
+int oracle_apply_momentum(const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
+                          int scale_mode, int64_t r, float eta, float mu, float* velocity, float* weights) {
+  if (!weights || !velocity || !(eta >= 0.0f) || eta > 3.0e38f || !(mu >= 0.0f) || !(mu < 1.0f)) return ORACLE_BAD_ARG;
+  std::vector<float> ghat((size_t)d);
+  const int rc = oracle_aggregate_scaled(msg_idx, msg_val, d, W, k, scale_mode, r, nullptr, ghat.data());
+  if (rc != ORACLE_OK) return rc;
+  for (int64_t i = 0; i < d; ++i) {
+    const float v = (float)((double)mu * (double)velocity[i] + (double)ghat[(size_t)i]);
+    velocity[i] = v;
+    weights[i] = (float)((double)weights[i] - (double)eta * (double)v);
+  }
+  return ORACLE_OK;
+}
+
 // ----------------------------------------------------------------------------- warm-up schedule
 // Section IV: sparsity is increased exponentially during the warm-up period, and k / r = 1 / n.
 // density(t) = initial * (final / initial)^(t / T) for t < T, final afterwards;
@@ -410,6 +435,64 @@ int oracle_decode_row(const uint32_t* packed_idx, const uint16_t* packed_val, in
     idx[j] = v;
     const uint32_t wide = (uint32_t)packed_val[j] << 16;
     std::memcpy(&val[j], &wide, 4);
+  }
+  return ORACLE_OK;
+}
+
+// A second format, for rows in ascending index order (which every message here is): Section III's
+// log d bits per index are what an index costs on its own, but a sorted row can say the high bits of
+// its indices once per stretch.  The coordinates are cut into spans of 2^14 = 16384; a row states
+//   * tab[t], t = 0 .. T with T = ceil(d / 16384): how many of its entries have an index below
+//     t * 16384 (so tab[0] = 0, tab[T] = k, and the entries of span t are tab[t] .. tab[t + 1] - 1);
+//   * low[j] = idx[j] mod 16384 for every entry (16 bits, the upper two zero);
+//   * the values as bfloat16, with the same error feedback as above.
+// 32 (T + 1) + 32 k bits per row instead of (ceil(log2 d) + 16) k.
+constexpr int64_t TILED_SPAN = 16384;
+
+int64_t oracle_tiled_spans(int64_t d) { return d < 1 ? 0 : (d + TILED_SPAN - 1) / TILED_SPAN; }
+
+// One row: k (index, value) pairs in strictly ascending index order -> tab (T + 1 words), low (k halves),
+// qval (k halves); residual (may be null) gets the rounding error at the sent coordinates.
+int oracle_encode_tiled_row(const uint32_t* idx, const float* val, int64_t k, int64_t d, uint32_t* tab,
+                            uint16_t* low, uint16_t* qval, float* residual) {
+  if (!idx || !val || !tab || !low || !qval || k < 1 || d < 1 || d > 0xFFFFFFFFll) return ORACLE_BAD_ARG;
+  for (int64_t j = 0; j < k; ++j) {
+    if ((int64_t)idx[j] >= d) return ORACLE_BAD_ARG;
+    if (j > 0 && idx[j] <= idx[j - 1]) return ORACLE_BAD_ARG;
+  }
+  const int64_t T = oracle_tiled_spans(d);
+  for (int64_t t = 0; t <= T; ++t) {
+    int64_t below = 0;
+    for (int64_t j = 0; j < k; ++j)
+      if ((int64_t)idx[j] < t * TILED_SPAN) ++below;
+    tab[t] = (uint32_t)below;
+  }
+  for (int64_t j = 0; j < k; ++j) {
+    low[j] = (uint16_t)(idx[j] % TILED_SPAN);
+    const uint16_t q = oracle_bf16_rne(val[j]);
+    qval[j] = q;
+    if (residual) {
+      const uint32_t wide = (uint32_t)q << 16;
+      float back;
+      std::memcpy(&back, &wide, 4);
+      residual[idx[j]] = std::isfinite(back) ? val[j] - back : 0.0f;
+    }
+  }
+  return ORACLE_OK;
+}
+
+int oracle_decode_tiled_row(const uint32_t* tab, const uint16_t* low, const uint16_t* qval, int64_t k, int64_t d,
+                            uint32_t* idx, float* val) {
+  if (!idx || !val || !tab || !low || !qval || k < 1 || d < 1) return ORACLE_BAD_ARG;
+  const int64_t T = oracle_tiled_spans(d);
+  if (tab[0] != 0 || (int64_t)tab[T] != k) return ORACLE_BAD_ARG;
+  for (int64_t t = 0; t < T; ++t) {
+    if (tab[t + 1] < tab[t]) return ORACLE_BAD_ARG;
+    for (int64_t j = tab[t]; j < (int64_t)tab[t + 1]; ++j) {
+      idx[j] = (uint32_t)(t * TILED_SPAN + low[j]);
+      const uint32_t wide = (uint32_t)qval[j] << 16;
+      std::memcpy(&val[j], &wide, 4);
+    }
   }
   return ORACLE_OK;
 }

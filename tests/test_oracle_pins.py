@@ -413,6 +413,60 @@ def test_master_update_worked_example_and_textbook_sgd():
         oracle.apply_update(idx4, val4, d, -1.0, w0)
 
 
+def test_momentum_update_worked_example_limits_and_library_optimizer():
+    # Section IV trains with momentum SGD; reading: heavy ball on the master, v <- mu v + ghat, w <- w - eta v.
+    # Worked example with exact binary fractions: ghat = [0.5, 0, 3, 4] (the average's worked example),
+    # v0 = [1, 2, 0, -8], mu = 0.5, eta = 0.25, w0 = 1:  v1 = [1, 1, 3, 0],  w1 = [0.75, 0.75, 0.25, 1].
+    idx = np.array([[0, 2], [2, 3]], dtype=np.uint32)
+    val = np.array([[1, 2], [4, 8]], dtype=np.float32)
+    v1, w1 = oracle.apply_momentum(idx, val, 4, 0.25, 0.5, np.array([1, 2, 0, -8], dtype=np.float32), np.ones(4, dtype=np.float32))
+    assert v1.tolist() == [1.0, 1.0, 3.0, 0.0] and w1.tolist() == [0.75, 0.75, 0.25, 1.0]
+    # a second step with the same messages: v2 = 0.5 v1 + ghat = [1, 0.5, 4.5, 4], w2 = w1 - 0.25 v2
+    v2, w2 = oracle.apply_momentum(idx, val, 4, 0.25, 0.5, v1, w1)
+    assert v2.tolist() == [1.0, 0.5, 4.5, 4.0] and w2.tolist() == [0.5, 0.625, -0.875, 0.0]
+    rng = np.random.default_rng(41)
+    d, k, W, eta, mu = 4000, 300, 3, 0.05, 0.9
+    w0 = rng.standard_normal(d).astype(np.float32)
+    msgs = []
+    for _ in range(6):
+        i = np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)]).astype(np.uint32)
+        msgs.append((i, rng.standard_normal((W, k)).astype(np.float32)))
+    # mu = 0 is the (separately pinned) master update, bit for bit, and v is then the average itself
+    v, w = oracle.apply_momentum(msgs[0][0], msgs[0][1], d, eta, 0.0, rng.standard_normal(d).astype(np.float32), w0)
+    assert np.array_equal(w.view(np.uint32), oracle.apply_update(msgs[0][0], msgs[0][1], d, eta, w0).view(np.uint32))
+    assert np.array_equal(v, oracle.aggregate(msgs[0][0], msgs[0][1], d)[1])
+    # against the library optimizer (torch.optim.SGD with momentum, dampening 0, no Nesterov) run in float64 on
+    # the same averages: the oracle rounds to binary32 twice per step and coordinate, so the two stay within a
+    # few binary32 roundings of each other over six steps
+    p = torch.nn.Parameter(torch.from_numpy(w0.astype(np.float64)))
+    opt = torch.optim.SGD([p], lr=eta, momentum=mu)
+    v, w = np.zeros(d, dtype=np.float32), w0.copy()
+    for i, x in msgs:
+        v, w = oracle.apply_momentum(i, x, d, eta, mu, v, w)
+        p.grad = torch.from_numpy(oracle.aggregate(i, x, d)[1].astype(np.float64))
+        opt.step()
+    ref = p.detach().numpy()
+    assert np.max(np.abs(w.astype(np.float64) - ref)) <= 6 * 2.0**-23 * max(1.0, float(np.max(np.abs(ref))))
+    # a constant average g: v_n = g (1 - mu^n) / (1 - mu), the geometric series
+    gi = np.arange(0, d, 7, dtype=np.uint32)[None, :]
+    gv = rng.standard_normal((1, gi.shape[1])).astype(np.float32)
+    v, w = np.zeros(d, dtype=np.float32), w0.copy()
+    n = 12
+    for _ in range(n):
+        v, w = oracle.apply_momentum(gi, gv, d, eta, mu, v, w)
+    g = np.zeros(d); g[gi[0].astype(np.int64)] = gv[0].astype(np.float64)
+    assert np.allclose(v, g * (1 - mu**n) / (1 - mu), rtol=1e-5, atol=1e-7)
+    # unsent coordinates: v decays by mu per step there and the weight keeps moving along it
+    quiet = np.ones(d, dtype=bool); quiet[gi[0].astype(np.int64)] = False
+    v0 = rng.standard_normal(d).astype(np.float32)
+    v1, w1 = oracle.apply_momentum(gi, gv, d, eta, mu, v0, w0)
+    assert np.array_equal(v1[quiet], (np.float64(np.float32(mu)) * v0[quiet].astype(np.float64)).astype(np.float32))
+    assert np.array_equal(w1[quiet], (w0[quiet].astype(np.float64) - np.float64(np.float32(eta)) * v1[quiet].astype(np.float64)).astype(np.float32))
+    for bad in [dict(eta=-1.0, mu=0.5), dict(eta=0.1, mu=1.0), dict(eta=0.1, mu=-0.1), dict(eta=0.1, mu=float("nan"))]:
+        with pytest.raises(ValueError):
+            oracle.apply_momentum(gi, gv, d, bad["eta"], bad["mu"], v0, w0)
+
+
 def test_aggregate_scalings_unbiased_and_by_count():
     # the worked example again: S = [1, 0, 6, 8], senders c = [1, 0, 2, 1], W = 2, k = 2
     idx = np.array([[0, 2], [2, 3]], dtype=np.uint32)
@@ -543,6 +597,76 @@ def test_codec_rounding_error_goes_to_the_residual():
     untouched = np.ones(d, dtype=bool); untouched[sent] = False
     assert np.array_equal(m[0, untouched].view(np.uint32), m0[0, untouched].view(np.uint32))
     assert np.all(np.abs(m[0, sent][ok]) <= np.abs(val[0][ok]) * 2.0**-8)
+
+
+def test_tiled_codec_hand_example():
+    # Spans of 16384 coordinates; d = 40000 has T = 3 of them: [0, 16384), [16384, 32768), [32768, 40000).
+    # Row 3, 16383 | 16384, 16390 | 39999: two entries below 16384, four below 32768, five in all.
+    idx = np.array([[3, 16383, 16384, 16390, 39999]], dtype=np.uint32)
+    val = np.array([[1.0, -2.0, 0.5, 3.0, -0.15625]], dtype=np.float32)
+    assert oracle.tiled_spans(40000) == 3 and oracle.tiled_spans(16384) == 1 and oracle.tiled_spans(16385) == 2
+    tab, low, qv = oracle.encode_tiled(idx, val, 40000)
+    assert tab.tolist() == [[0, 2, 4, 5]]
+    assert low.tolist() == [[3, 16383, 0, 6, 39999 - 32768]]
+    assert qv.tolist() == [[0x3F80, 0xC000, 0x3F00, 0x4040, 0xBE20]]
+    i2, v2 = oracle.decode_tiled(tab, low, qv, 40000, 5)
+    assert np.array_equal(i2, idx) and np.array_equal(v2, val)
+    # a row that skips spans: the table repeats itself over the empty ones
+    tab, low, _ = oracle.encode_tiled(np.array([[5, 70000]], dtype=np.uint32), np.ones((1, 2), dtype=np.float32), 100000)
+    assert tab.tolist() == [[0, 1, 1, 1, 1, 2, 2, 2]] and low.tolist() == [[5, 70000 - 4 * 16384]]
+    for bad in [np.array([[5, 5]]), np.array([[9, 3]]), np.array([[1, 100000]])]:       # not ascending / out of range
+        with pytest.raises(ValueError):
+            oracle.encode_tiled(bad.astype(np.uint32), np.ones((1, 2), dtype=np.float32), 100000)
+
+
+def test_tiled_codec_against_library_search_round_trip_and_size():
+    rng = np.random.default_rng(51)
+    for d, k in [(1, 1), (16384, 16384), (16385, 9), (100003, 1000), (1 << 20, 5000), ((1 << 22) + 17, 300)]:
+        idx = np.sort(rng.choice(d, size=k, replace=False)).astype(np.uint32)[None, :]
+        val = (rng.standard_normal((1, k)) * np.exp(3 * rng.standard_normal((1, k)))).astype(np.float32)
+        tab, low, qv = oracle.encode_tiled(idx, val, d)
+        T = (d + 16383) // 16384
+        # the table is a lower-bound search of the span boundaries in the sorted row (library routine)
+        assert tab.shape == (1, T + 1)
+        assert np.array_equal(tab[0], np.searchsorted(idx[0], np.arange(T + 1, dtype=np.int64) * 16384, side="left"))
+        assert np.array_equal(low[0], idx[0] & 16383) and int(low.max()) < 16384
+        # values: the bfloat16 rounding pinned above, here against torch once more
+        assert np.array_equal(qv[0], torch.from_numpy(val[0]).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16))
+        i2, v2 = oracle.decode_tiled(tab, low, qv, d, k)
+        assert np.array_equal(i2, idx)
+        assert np.array_equal(v2.view(np.uint32), qv.astype(np.uint32) << 16)
+        # both codecs carry the same message
+        pi, pv = oracle.encode(idx, val, d)
+        i3, v3 = oracle.decode(pi, pv, d, k)
+        assert np.array_equal(i3, i2) and np.array_equal(v3.view(np.uint32), v2.view(np.uint32))
+    # size at the paper's scale (ResNet-18, 0.1 % of 11.17 M coordinates): 32 (T + 1) + 32 k bits against
+    # (24 + 16) k for the bit-packed indices and 64 k for plain pairs
+    d, k = 11173962, 11173
+    T = oracle.tiled_spans(d)
+    assert T == 683 and 32 * (T + 1) + 32 * k < (oracle.index_bits(d) + 16) * k < 64 * k
+
+
+def test_tiled_codec_rounding_error_goes_to_the_residual():
+    # the same error feedback as the bit-packed format: decoded value + residual slot = a exactly
+    rng = np.random.default_rng(52)
+    d, k = 50000, 700
+    idx = np.sort(rng.choice(d, k, replace=False)).astype(np.uint32)[None, :]
+    val = (rng.standard_normal((1, k)) * np.exp(3 * rng.standard_normal((1, k)))).astype(np.float32)
+    val[0, 0] = 3.4e38
+    val[0, 1] = 1.0
+    m = rng.standard_normal((1, d)).astype(np.float32)
+    m[0, idx[0].astype(np.int64)] = 0.0
+    m0, m_packed = m.copy(), m.copy()
+    tab, low, qv = oracle.encode_tiled(idx, val, d, residual=m)
+    oracle.encode(idx, val, d, residual=m_packed)
+    assert np.array_equal(m.view(np.uint32), m_packed.view(np.uint32))
+    _, back = oracle.decode_tiled(tab, low, qv, d, k)
+    sent = idx[0].astype(np.int64)
+    ok = np.isfinite(back[0])
+    assert np.array_equal(back[0][ok].astype(np.float64) + m[0, sent][ok].astype(np.float64), val[0][ok].astype(np.float64))
+    assert m[0, sent[0]] == 0.0 and m[0, sent[1]] == 0.0 and not np.signbit(m[0, sent[1]])
+    untouched = np.ones(d, dtype=bool); untouched[sent] = False
+    assert np.array_equal(m[0, untouched].view(np.uint32), m0[0, untouched].view(np.uint32))
 
 
 # ----------------------------------------------------------------------------- warm-up schedule
