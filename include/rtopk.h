@@ -250,6 +250,41 @@ int rtopk_aggregate_packed(rtopk_ctx* ctx, const uint32_t* packed_idx, int64_t l
                            int64_t k, int scale_mode, float* out, void* stream);
 
 /*
+ * Span-table message format, for rows in ascending index order (every message of this library is).
+ * Section III's log d bits are what an index costs on its own; a sorted row can state the high bits of
+ * its indices once per stretch.  The coordinates are cut into spans of 16384; per row
+ *   span_tab   spans + 1 32-bit words, spans = ceil(d / 16384): span_tab[t] = how many of the row's
+ *              entries have an index below t * 16384 (span_tab[0] = 0, span_tab[spans] = k); rows follow
+ *              one another without padding (row stride spans + 1);
+ *   low_idx    W rows of ld_low 16-bit words: index mod 16384 of every entry;
+ *   packed_val W rows of ld_halves bfloat16 values, as in the packed format.
+ * 32 (spans + 1) + 32 k bits per row (4.2 bytes per entry at d = 25.6 M, k = d / 1000; the packed format
+ * takes 5.1, plain pairs 8), and the table is also what the aggregation needs to find every worker's
+ * entries of an output tile, so rtopk_aggregate_tiled searches nothing.
+ * rtopk_tiled_layout (host only, no GPU work) returns spans and the smallest accepted row strides
+ * (multiples of 8); any output may be null.  Errors: INVALID_ARG (d < 1, d >= 2^32, k < 1 or k > d).
+ */
+int rtopk_tiled_layout(int64_t d, int64_t k, int64_t* spans, int64_t* ld_low, int64_t* ld_halves);
+
+/*
+ * Encodes W rows of k (index, value) pairs in strictly ascending index order (as rtopk_sparsify writes
+ * them) into the span-table format; `residual` as in rtopk_encode (the rounding error of the values is
+ * fed back).  Row padding of low_idx and packed_val is written as zero.  Device pointers; span_tab
+ * 4-byte, low_idx and packed_val 16-byte aligned.  Rows that are not ascending give a table that does
+ * not describe them (nothing is written out of bounds).  Errors: INVALID_ARG, CUDA.
+ */
+int rtopk_encode_tiled(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W,
+                       int64_t k, float* residual, int64_t ld_m, uint32_t* span_tab, uint16_t* low_idx,
+                       int64_t ld_low, uint16_t* packed_val, int64_t ld_halves, void* stream);
+
+/* rtopk_aggregate reading the span-table format directly (decoder fused into the aggregation kernels;
+ * table entries beyond k are read as k).  scale_mode MEAN, SUM or COUNT.  Errors: INVALID_ARG,
+ * UNSUPPORTED, CUDA. */
+int rtopk_aggregate_tiled(rtopk_ctx* ctx, const uint32_t* span_tab, const uint16_t* low_idx, int64_t ld_low,
+                          const uint16_t* packed_val, int64_t ld_halves, int64_t d, int32_t W, int64_t k,
+                          int scale_mode, float* out, void* stream);
+
+/*
  * Algorithm 1, master update w <- w - eta * ghat applied straight from the messages: ghat is the
  * binary32 result rtopk_aggregate would write, and every coordinate that some worker sent receives
  * fp32(double(w_i) - double(eta) * double(ghat_i)) (one rounding); all other weights are not touched
@@ -266,6 +301,27 @@ int rtopk_step_apply(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t l
                      int64_t ld_m, int64_t d, int32_t W, int32_t worker_base, int64_t r, int64_t k,
                      uint64_t seed, uint32_t step, int scale_mode, float eta, uint32_t* msg_idx,
                      float* msg_val, float* weights, void* stream);
+
+/*
+ * The master update with momentum.  Section IV trains with momentum SGD and prints no formula; this is
+ * the heavy-ball form applied to Algorithm 1's average ghat (the binary32 result rtopk_aggregate would
+ * write), for EVERY coordinate i, sent or not:
+ *     v_i <- fp32(double(mu) * double(v_i) + double(ghat_i));   w_i <- fp32(double(w_i) - double(eta) * double(v_i))
+ * (one rounding per line; with mu = 0 the weights receive what rtopk_apply_update gives them).
+ *   velocity, weights [in/out]  d binary32 each, 16-byte aligned, not overlapping;
+ *   eta  finite, >= 0;   0 <= mu < 1;   r  only read with RTOPK_SCALE_UNBIASED (k <= r <= d).
+ * Errors: INVALID_ARG, UNSUPPORTED (COUNT with more than 65535 workers), CUDA.
+ */
+int rtopk_apply_momentum(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W,
+                         int64_t k, int scale_mode, int64_t r, float eta, float mu, float* velocity,
+                         float* weights, void* stream);
+
+/* rtopk_sparsify followed by rtopk_apply_momentum of the W messages it produced.  Arguments as in the
+ * two calls. */
+int rtopk_step_momentum(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,
+                        int64_t ld_m, int64_t d, int32_t W, int32_t worker_base, int64_t r, int64_t k,
+                        uint64_t seed, uint32_t step, int scale_mode, float eta, float mu, uint32_t* msg_idx,
+                        float* msg_val, float* velocity, float* weights, void* stream);
 
 /* One round of Algorithm 1's communication path: rtopk_sparsify followed by rtopk_aggregate of
  * the W messages it produced.  Arguments as in the two calls. */

@@ -5,8 +5,8 @@ marshals arguments (torch tensors -> device pointers, the current CUDA stream). 
 fallback: using the binding without the built library or without a CUDA device raises.
 """
 from .workloads import Workload, configs, gradient, zero_residual  # noqa: F401
-from .binding import (RTopK, RTopKError, library_path, load_library, packed_layout, warmup_sizes, GRAD_F32, GRAD_BF16,  # noqa: F401
+from .binding import (RTopK, RTopKError, library_path, load_library, packed_layout, tiled_layout, warmup_sizes, GRAD_F32, GRAD_BF16,  # noqa: F401
                       SCALE_MEAN, SCALE_SUM, SCALE_UNBIASED, SCALE_COUNT, EXPORTS)
 
-__all__ = ["RTopK", "RTopKError", "library_path", "load_library", "packed_layout", "warmup_sizes", "Workload", "configs", "gradient",
+__all__ = ["RTopK", "RTopKError", "library_path", "load_library", "packed_layout", "tiled_layout", "warmup_sizes", "Workload", "configs", "gradient",
            "zero_residual", "GRAD_F32", "GRAD_BF16", "SCALE_MEAN", "SCALE_SUM", "SCALE_UNBIASED", "SCALE_COUNT", "EXPORTS"]

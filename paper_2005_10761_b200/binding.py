@@ -41,6 +41,12 @@ EXPORTS = {
     "rtopk_packed_layout": (_int, [_i64, _i64, C.POINTER(_i32), C.POINTER(_i64), C.POINTER(_i64)]),
     "rtopk_encode": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _vp, _i64, _vp, _i64, _vp, _i64, _vp]),
     "rtopk_aggregate_packed": (_int, [_vp, _vp, _i64, _vp, _i64, _i64, _i32, _i64, _int, _vp, _vp]),
+    "rtopk_tiled_layout": (_int, [_i64, _i64, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64)]),
+    "rtopk_encode_tiled": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _vp, _i64, _vp, _vp, _i64, _vp, _i64, _vp]),
+    "rtopk_aggregate_tiled": (_int, [_vp, _vp, _vp, _i64, _vp, _i64, _i64, _i32, _i64, _int, _vp, _vp]),
+    "rtopk_apply_momentum": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _int, _i64, C.c_float, C.c_float, _vp, _vp, _vp]),
+    "rtopk_step_momentum": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _i64, _u64, _u32, _int,
+                                   C.c_float, C.c_float, _vp, _vp, _vp, _vp, _vp]),
     "rtopk_apply_update": (_int, [_vp, _vp, _vp, _i64, _i32, _i64, _int, C.c_float, _vp, _vp]),
     "rtopk_step_apply": (_int, [_vp, _vp, _int, _i64, _vp, _i64, _i64, _i32, _i32, _i64, _i64, _u64, _u32, _int,
                                 C.c_float, _vp, _vp, _vp, _vp]),
@@ -93,6 +99,16 @@ def packed_layout(d: int, k: int):
     if rc != 0:
         raise RTopKError(rc, "rtopk_packed_layout", "invalid argument")
     return int(bits.value), int(lw.value), int(lh.value)
+
+
+def tiled_layout(d: int, k: int):
+    """(spans, row stride of the low index halves, row stride of the value halves) of the span-table format;
+    the table itself has spans + 1 words per row."""
+    sp, ll, lh = _i64(0), _i64(0), _i64(0)
+    rc = load_library().rtopk_tiled_layout(d, k, C.byref(sp), C.byref(ll), C.byref(lh))
+    if rc != 0:
+        raise RTopKError(rc, "rtopk_tiled_layout", "invalid argument")
+    return int(sp.value), int(ll.value), int(lh.value)
 
 
 def library_path() -> str:
@@ -245,6 +261,40 @@ class RTopK:
                                               packed_val.data_ptr(), packed_val.stride(0), d, W, k, scale_mode,
                                               out.data_ptr(), _stream())
         self._check(rc, "rtopk_aggregate_packed")
+
+    def encode_tiled(self, msg_idx, msg_val, d, span_tab, low_idx, packed_val, residual=None) -> None:
+        """msg -> span-table rows (int32 [W, spans + 1] contiguous, int16 [W, ld_low], int16 [W, ld_halves])."""
+        W, k = msg_idx.shape
+        assert span_tab.is_contiguous()
+        rc = self._lib.rtopk_encode_tiled(self._h, msg_idx.data_ptr(), msg_val.data_ptr(), d, W, k,
+                                          residual.data_ptr() if residual is not None else None,
+                                          residual.stride(0) if residual is not None else 0,
+                                          span_tab.data_ptr(), low_idx.data_ptr(), low_idx.stride(0),
+                                          packed_val.data_ptr(), packed_val.stride(0), _stream())
+        self._check(rc, "rtopk_encode_tiled")
+
+    def aggregate_tiled(self, span_tab, low_idx, packed_val, d, k, out, scale_mode=SCALE_MEAN) -> None:
+        W = low_idx.shape[0]
+        assert span_tab.is_contiguous()
+        rc = self._lib.rtopk_aggregate_tiled(self._h, span_tab.data_ptr(), low_idx.data_ptr(), low_idx.stride(0),
+                                             packed_val.data_ptr(), packed_val.stride(0), d, W, k, scale_mode,
+                                             out.data_ptr(), _stream())
+        self._check(rc, "rtopk_aggregate_tiled")
+
+    def apply_momentum(self, msg_idx, msg_val, d, eta, mu, velocity, weights, scale_mode=SCALE_MEAN, r=0) -> None:
+        W, k = msg_idx.shape
+        rc = self._lib.rtopk_apply_momentum(self._h, msg_idx.data_ptr(), msg_val.data_ptr(), d, W, k, scale_mode, r,
+                                            eta, mu, velocity.data_ptr(), weights.data_ptr(), _stream())
+        self._check(rc, "rtopk_apply_momentum")
+
+    def step_momentum(self, grad, residual, d, r, k, seed, step, eta, mu, msg_idx, msg_val, velocity, weights,
+                      worker_base=0, scale_mode=SCALE_MEAN) -> None:
+        W = grad.shape[0]
+        rc = self._lib.rtopk_step_momentum(self._h, grad.data_ptr(), self._grad_dtype(grad), grad.stride(0),
+                                           residual.data_ptr(), residual.stride(0), d, W, worker_base, r, k, seed,
+                                           step, scale_mode, eta, mu, msg_idx.data_ptr(), msg_val.data_ptr(),
+                                           velocity.data_ptr(), weights.data_ptr(), _stream())
+        self._check(rc, "rtopk_step_momentum")
 
     def apply_update(self, msg_idx, msg_val, d, eta, weights, scale_mode=SCALE_MEAN) -> None:
         W, k = msg_idx.shape

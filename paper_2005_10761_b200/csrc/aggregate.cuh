@@ -39,10 +39,25 @@ __device__ __forceinline__ float agg_result(float ghat, float old, float eta) {
   return eta < 0.0f ? ghat : (float)((double)old - (double)eta * (double)ghat);
 }
 
+// first entry of worker w's ascending row (n entries) whose index is >= key
+template <typename M>
+__device__ __forceinline__ uint32_t lower_bound_row(const M& msgs, uint32_t w, uint32_t n, uint32_t key) {
+  uint32_t lo = 0, hi = n;
+  while (lo < hi) {
+    const uint32_t mid = (lo + hi) >> 1;
+    if (msgs.index(w, mid) < key) lo = mid + 1; else hi = mid;
+  }
+  return lo;
+}
+
 // The W x K messages as the kernels read them: plain (u32 index, f32 value) rows, or the packed
 // format (Section III: an index costs log d bits, a value a constant number): `bits` = ceil(log2 d)
 // bits per index, entry j at bits [j * bits, (j + 1) * bits) of the row's little-endian stream of
 // 32-bit words, and bfloat16 values (the upper half of the binary32 pattern).
+// Every format offers index(w, j); index_in(w, j, base) for an entry known to lie in the span of
+// kTiledSpan coordinates that starts at `base`; lower_bound(w, n, key) = the first of the row's n
+// entries with an index >= key.
+constexpr uint32_t kTiledSpan = 16384;
 struct PlainMsgs {
   const uint32_t* idx;
   const float* val;
@@ -50,6 +65,8 @@ struct PlainMsgs {
   uint32_t stride;   // 1: two arrays of W x K words; 2: one array of W x K (index, value) pairs, val = idx + 1
   __device__ __forceinline__ uint32_t index(uint32_t w, uint32_t j) const { return __ldg(idx + ((size_t)w * K + j) * stride); }
   __device__ __forceinline__ float value(uint32_t w, uint32_t j) const { return __ldg(val + ((size_t)w * K + j) * stride); }
+  __device__ __forceinline__ uint32_t index_in(uint32_t w, uint32_t j, uint32_t) const { return index(w, j); }
+  __device__ __forceinline__ uint32_t lower_bound(uint32_t w, uint32_t n, uint32_t key) const { return lower_bound_row(*this, w, n, key); }
   // what worker w's value v adds to a coordinate's double-precision sum
   static constexpr bool kPerWorker = false;   // the term does not depend on the worker
   static constexpr bool kPadded = false;      // every row holds K valid entries
@@ -70,6 +87,42 @@ struct PackedMsgs {
   __device__ __forceinline__ float value(uint32_t w, uint32_t j) const {
     return __uint_as_float((uint32_t)__ldg(halves + (size_t)w * ld_halves + j) << 16);
   }
+  __device__ __forceinline__ uint32_t index_in(uint32_t w, uint32_t j, uint32_t) const { return index(w, j); }
+  __device__ __forceinline__ uint32_t lower_bound(uint32_t w, uint32_t n, uint32_t key) const { return lower_bound_row(*this, w, n, key); }
+  static constexpr bool kPerWorker = false;
+  static constexpr bool kPadded = false;
+  __device__ __forceinline__ double term(uint32_t, float v) const { return (double)v; }
+};
+// The span-table format for ascending rows: the coordinates are cut into spans of kTiledSpan; a row says
+// how many of its entries lie below every span boundary (tab[t], t = 0 .. spans: the entries of span t are
+// tab[t] .. tab[t + 1] - 1) and keeps only the 14 low bits of each index; values are bfloat16.  The table
+// is at the same time the table of run starts the sparse kernel works from.
+struct TiledMsgs {
+  const uint32_t* tab;      // [W][spans + 1]
+  const uint16_t* low;      // [W][ld_low]
+  const uint16_t* halves;   // [W][ld_halves]
+  uint32_t spans, ld_low, ld_halves;
+  __device__ __forceinline__ uint32_t index(uint32_t w, uint32_t j) const {     // the span of entry j: the last t with tab[t] <= j
+    const uint32_t* row = tab + (size_t)w * (spans + 1);
+    uint32_t a = 0, b = spans;
+    while (b - a > 1) { const uint32_t mid = (a + b) >> 1; if (__ldg(row + mid) <= j) a = mid; else b = mid; }
+    return a * kTiledSpan + __ldg(low + (size_t)w * ld_low + j);
+  }
+  __device__ __forceinline__ uint32_t index_in(uint32_t w, uint32_t j, uint32_t base) const {
+    return base + __ldg(low + (size_t)w * ld_low + j);
+  }
+  __device__ __forceinline__ float value(uint32_t w, uint32_t j) const {
+    return __uint_as_float((uint32_t)__ldg(halves + (size_t)w * ld_halves + j) << 16);
+  }
+  __device__ __forceinline__ uint32_t lower_bound(uint32_t w, uint32_t n, uint32_t key) const {
+    const uint32_t t = key / kTiledSpan, rem = key % kTiledSpan;
+    if (t >= spans) return n;
+    const uint32_t* row = tab + (size_t)w * (spans + 1);
+    uint32_t lo = min(n, __ldg(row + t)), hi = min(n, __ldg(row + t + 1));      // (a malformed table stays inside the row)
+    const uint16_t* l = low + (size_t)w * ld_low;
+    while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (__ldg(l + mid) < rem) lo = mid + 1; else hi = mid; }
+    return lo;
+  }
   static constexpr bool kPerWorker = false;
   static constexpr bool kPadded = false;
   __device__ __forceinline__ double term(uint32_t, float v) const { return (double)v; }
@@ -86,23 +139,14 @@ struct ThresholdMsgs {
   const uint32_t* ones;
   __device__ __forceinline__ uint32_t index(uint32_t w, uint32_t j) const { return __ldg(idx + (size_t)w * K + j); }
   __device__ __forceinline__ float value(uint32_t w, uint32_t j) const { return __ldg(val + (size_t)w * K + j); }
+  __device__ __forceinline__ uint32_t index_in(uint32_t w, uint32_t j, uint32_t) const { return index(w, j); }
+  __device__ __forceinline__ uint32_t lower_bound(uint32_t w, uint32_t n, uint32_t key) const { return lower_bound_row(*this, w, n, key); }
   static constexpr bool kPerWorker = true;
   static constexpr bool kPadded = true;
   __device__ __forceinline__ double term(uint32_t w, float v) const {
     return __dmul_rn((double)v, __ddiv_rn((double)__ldg(ones + w), (double)__ldg(count + w)));
   }
 };
-
-// first entry of worker w's ascending row (n entries) whose index is >= key
-template <typename M>
-__device__ __forceinline__ uint32_t lower_bound_row(const M& msgs, uint32_t w, uint32_t n, uint32_t key) {
-  uint32_t lo = 0, hi = n;
-  while (lo < hi) {
-    const uint32_t mid = (lo + hi) >> 1;
-    if (msgs.index(w, mid) < key) lo = mid + 1; else hi = mid;
-  }
-  return lo;
-}
 
 // The same as a 16-way search by each half of a warp (lanes 0-15 share one key, lanes 16-31
 // another): every lane of a half returns that half's lower bound in worker w's ascending row.
@@ -134,13 +178,15 @@ __global__ void __launch_bounds__(kAggThreads) k_agg_starts(M msgs, uint32_t W, 
   if (t > ntiles || w >= W) return;
   // padded rows end their last run at the first padding entry (padding indices exceed every tile bound)
   const uint32_t bound = t == ntiles ? 0xFFFFFFFFu : t * tile_size;
-  starts[(size_t)w * (ntiles + 1) + t] = (t == ntiles && !M::kPadded) ? K : lower_bound_row(msgs, w, K, bound);
+  starts[(size_t)w * (ntiles + 1) + t] = (t == ntiles && !M::kPadded) ? K : msgs.lower_bound(w, K, bound);
 }
 
 template <typename M, bool COUNT>   // COUNT: also keep the number of senders per coordinate (smaller stage to make room)
 __global__ void __launch_bounds__(kAggThreads) k_aggregate(M msgs, const uint32_t* __restrict__ starts, uint32_t d,
                                                            uint32_t W, uint32_t K, AggScale sc,
-                                                           float eta, float* __restrict__ out) {
+                                                           float eta, float* __restrict__ out, float mu,
+                                                           float* __restrict__ velocity) {
+  static_assert(kTiledSpan % kAggTile == 0, "a tile lies inside one span");
   constexpr int kStage = COUNT ? kAggStage / 2 : kAggStage;
   __shared__ double acc[kAggTile];
   __shared__ uint16_t senders[COUNT ? kAggTile : 1];    // at most 65535 workers (checked by the host)
@@ -152,6 +198,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(M msgs, const uint32_
   const uint32_t ntiles = gridDim.x;
   const uint32_t lo = blockIdx.x * (uint32_t)kAggTile;
   const uint32_t hi = min(d, lo + (uint32_t)kAggTile);
+  const uint32_t span_lo = lo - lo % kTiledSpan;
   for (uint32_t i = tid; i < (uint32_t)kAggTile; i += kAggThreads) { acc[i] = 0.0; if (COUNT) senders[i] = 0; }
   for (uint32_t w0 = 0; w0 < W; w0 += kAggThreads) {
     const uint32_t nw = min((uint32_t)kAggThreads, W - w0);
@@ -160,7 +207,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(M msgs, const uint32_
     uint32_t cnt = 0;
     if (tid < nw) {
       const uint32_t* st = starts + (size_t)(w0 + tid) * (ntiles + 1) + blockIdx.x;
-      const uint32_t b = __ldg(st), e = __ldg(st + 1);
+      const uint32_t b = min(K, __ldg(st)), e = min(K, __ldg(st + 1));
       s_beg[tid] = b;
       cnt = e > b ? e - b : 0u;
     }
@@ -179,7 +226,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(M msgs, const uint32_
         uint32_t a = 0, b = nw;                       // last worker with s_pre[w] <= q
         while (b - a > 1) { const uint32_t mid = (a + b) >> 1; if (s_pre[mid] <= q) a = mid; else b = mid; }
         const uint32_t j = s_beg[a] + (q - s_pre[a]);
-        st_idx[q] = msgs.index(w0 + a, j);
+        st_idx[q] = msgs.index_in(w0 + a, j, span_lo);
         st_val[q] = msgs.value(w0 + a, j);
       }
       __syncthreads();
@@ -197,7 +244,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(M msgs, const uint32_
       for (uint32_t w = 0; w < nw; ++w) {
         const uint32_t b = s_beg[w], n = s_pre[w + 1] - s_pre[w];
         for (uint32_t q = tid; q < n; q += kAggThreads) {
-          const uint32_t i = msgs.index(w0 + w, b + q) - lo;
+          const uint32_t i = msgs.index_in(w0 + w, b + q, span_lo) - lo;
           if (i < (uint32_t)kAggTile) { acc[i] += msgs.term(w0 + w, msgs.value(w0 + w, b + q)); if (COUNT) ++senders[i]; }
         }
         __syncthreads();
@@ -209,6 +256,16 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(M msgs, const uint32_
     const double a = acc[i];
     return (float)(a != 0.0 ? agg_scaled(a, COUNT ? (uint32_t)senders[i] : 0u, sc) : a);
   };
+  if (velocity != nullptr) {
+    // heavy-ball momentum on the master: v <- mu v + ghat, w <- w - eta v, every coordinate, each line
+    // rounded once from double (the products are exact in double)
+    for (uint32_t i = tid; i < hi - lo; i += kAggThreads) {
+      const float v = (float)((double)mu * (double)velocity[lo + i] + (double)scaled(i));
+      velocity[lo + i] = v;
+      out[lo + i] = (float)((double)out[lo + i] - (double)eta * (double)v);
+    }
+    return;
+  }
   if (hi - lo == (uint32_t)kAggTile) {
     for (uint32_t i = tid * 4; i < (uint32_t)kAggTile; i += kAggThreads * 4) {
       float4 o;
@@ -241,7 +298,9 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
   __shared__ uint32_t s_carry;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t ntiles = gridDim.x;
+  static_assert(kTiledSpan % kAggSparseTile == 0, "a tile lies inside one span");
   const uint32_t lo = blockIdx.x * (uint32_t)kAggSparseTile;
+  const uint32_t span_lo = lo - lo % kTiledSpan;
   if (tid == 0) s_carry = 0;
   __syncthreads();
   if (starts == nullptr) {
@@ -262,7 +321,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     if (w < W) {
       if (starts != nullptr) {
         const uint32_t* st = starts + (size_t)w * (ntiles + 1) + blockIdx.x;
-        const uint32_t b = __ldg(st), e = __ldg(st + 1);
+        const uint32_t b = min(K, __ldg(st)), e = min(K, __ldg(st + 1));
         s_beg[w] = b;
         cnt = e > b ? e - b : 0u;
       } else {
@@ -303,7 +362,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     for (uint32_t q = tid; q < total; q += kAggThreads) {
       const uint32_t a = worker_of(q);
       const uint32_t j = s_beg[a] + (q - s_pre[a]);
-      st_idx[q] = msgs.index(a, j);
+      st_idx[q] = msgs.index_in(a, j, span_lo);
       st_val[q] = msgs.value(a, j);
       st_w[q] = (uint16_t)a;
     }
@@ -401,7 +460,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
   // ---- a crowded tile (more entries than the stage holds): every entry looks the other workers' runs
   // up in global memory; the entry of the lowest worker that holds a coordinate owns it and sums that
   // coordinate over the workers in ascending order
-  auto idx_at = [&](uint32_t w, uint32_t j) { return msgs.index(w, s_beg[w] + j); };
+  auto idx_at = [&](uint32_t w, uint32_t j) { return msgs.index_in(w, s_beg[w] + j, span_lo); };
   auto val_at = [&](uint32_t w, uint32_t j) { return msgs.value(w, s_beg[w] + j); };
   for (uint32_t q = tid; q < total; q += kAggThreads) {
     const uint32_t w = worker_of(q);

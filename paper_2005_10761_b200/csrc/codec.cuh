@@ -2,7 +2,8 @@
 // bits): ceil(log2 d)-bit indices in a little-endian bit stream of 32-bit words, bfloat16 values
 // rounded to nearest even.  Algorithm 1 keeps m = a - ghat with ghat what is sent, so the rounding
 // error of a sent value goes back into its residual slot.  The decoder lives in the aggregation
-// kernels (PackedMsgs in aggregate.cuh).
+// kernels (PackedMsgs in aggregate.cuh).  A second format for ascending rows (a table of entry counts
+// per span of coordinates plus 14 low bits per index) is encoded at the end of this file.
 #pragma once
 
 #include "common.cuh"
@@ -53,6 +54,42 @@ __global__ void __launch_bounds__(kCodecThreads) k_encode(const uint32_t* __rest
     }
     halves[(size_t)w * ld_halves + t] = q;
   }
+}
+
+// The span-table format (TiledMsgs in aggregate.cuh).  grid (blocks over max(ld_low, ld_halves), W).  A thread
+// takes one entry: its 14 low index bits, its value, and the table words of the spans that begin between
+// the entry before it and itself (each word is written by exactly one thread; the last entry also writes
+// the words behind it).  `span` = coordinates per span.
+__global__ void __launch_bounds__(kCodecThreads) k_encode_tiled(const uint32_t* __restrict__ msg_idx,
+                                                                const float* __restrict__ msg_val, uint32_t K,
+                                                                uint32_t d, uint32_t span, uint32_t spans, float* residual,
+                                                                int64_t ld_m, uint32_t* __restrict__ tab,
+                                                                uint16_t* __restrict__ low, uint32_t ld_low,
+                                                                uint16_t* __restrict__ halves, uint32_t ld_halves) {
+  const uint32_t w = blockIdx.y;
+  const uint32_t t = blockIdx.x * kCodecThreads + threadIdx.x;
+  const uint32_t* idx = msg_idx + (size_t)w * K;
+  const float* val = msg_val + (size_t)w * K;
+  uint16_t l = 0, q = 0;
+  if (t < K) {
+    const uint32_t i = __ldg(idx + t);
+    uint32_t* row = tab + (size_t)w * (spans + 1);
+    const uint32_t mine = min(i / span, spans);                      // (an index beyond d stays inside the table)
+    const uint32_t from = t == 0 ? 0u : min(__ldg(idx + t - 1) / span, spans) + 1u;
+    for (uint32_t s = from; s <= mine; ++s) row[s] = t;              // spans that begin at or before this entry
+    if (t == K - 1)
+      for (uint32_t s = mine + 1u; s <= spans; ++s) row[s] = K;
+    l = (uint16_t)(i % span);
+    const float a = __ldg(val + t);
+    q = bf16_round(a);
+    if (residual && i < d) {
+      const float back = __uint_as_float((uint32_t)q << 16);
+      const bool finite = (__float_as_uint(back) & 0x7F800000u) != 0x7F800000u;
+      residual[(size_t)w * (size_t)ld_m + i] = finite ? __fsub_rn(a, back) : 0.0f;
+    }
+  }
+  if (t < ld_low) low[(size_t)w * ld_low + t] = l;
+  if (t < ld_halves) halves[(size_t)w * ld_halves + t] = q;
 }
 
 }  // namespace rtopk

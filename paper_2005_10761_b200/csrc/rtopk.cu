@@ -12,6 +12,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <type_traits>
 #include <vector>
 
 #include "aggregate.cuh"
@@ -615,9 +616,11 @@ bool aggregate_is_sparse(int64_t d, int32_t W, int64_t k) {
 // the streaming pass).
 // eta < 0: `out` receives the average.  eta >= 0: `out` holds weights and receives w - eta * average
 // (only the coordinates some worker sent change, so nothing is cleared).
+// `velocity` not null: heavy-ball momentum, `out` holds the weights (eta >= 0), every coordinate changes.
 template <typename M>
 int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_t k, int scale_mode, float* out,
-                     cudaStream_t st, bool out_cleared, float eta, int64_t r) {
+                     cudaStream_t st, bool out_cleared, float eta, int64_t r, float mu = 0.0f,
+                     float* velocity = nullptr) {
   if (!ctx || !out) return RTOPK_ERR_INVALID_ARG;
   if (d < 1 || d > ctx->d_max || W < 1 || W > ctx->W_max || k < 1 || k > d) return RTOPK_ERR_INVALID_ARG;
   if (!scale_mode_known(scale_mode)) return RTOPK_ERR_INVALID_ARG;
@@ -625,16 +628,23 @@ int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_
   if (scale_mode == RTOPK_SCALE_COUNT && W > 65535) return RTOPK_ERR_UNSUPPORTED;
   if ((uintptr_t)out & 15u) return RTOPK_ERR_INVALID_ARG;
   if ((uint64_t)k * (uint64_t)W >= (1ull << 32)) return RTOPK_ERR_INVALID_ARG;
-  const bool sparse = aggregate_is_sparse(d, W, k);
+  const bool sparse = aggregate_is_sparse(d, W, k) && velocity == nullptr;
   const uint32_t tile = sparse ? (uint32_t)kAggSparseTile : (uint32_t)kAggTile;
   const uint32_t ntiles = (uint32_t)((d + tile - 1) / tile);
-  if ((size_t)W * (ntiles + 1) > ctx->agg_start_entries) return RTOPK_ERR_INVALID_ARG;
+  // the span-table format brings the sparse kernel's table of run starts along
+  static_assert(kAggSparseTile == (int)kTiledSpan, "the spans of the format are the sparse kernel's tiles");
+  const uint32_t* starts = ctx->d_agg_starts;
+  bool have_starts = false;
+  if constexpr (std::is_same<M, TiledMsgs>::value) {
+    if (sparse) { starts = msgs.tab; have_starts = true; }
+  }
+  if (!have_starts && (size_t)W * (ntiles + 1) > ctx->agg_start_entries) return RTOPK_ERR_INVALID_ARG;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return RTOPK_ERR_CUDA;
   // with few workers and tiles the sparse kernel finds every tile's runs itself (one launch fewer);
   // otherwise a table of run starts is built first, all searches side by side
-  const bool own_search = sparse && W <= kAggSearchW && (uint64_t)ntiles * (uint64_t)((W + 7) / 8) <= 4096u;
-  if (!own_search) {
+  const bool own_search = !have_starts && sparse && W <= kAggSearchW && (uint64_t)ntiles * (uint64_t)((W + 7) / 8) <= 4096u;
+  if (!own_search && !have_starts) {
     const dim3 sgrid((ntiles + 1 + kAggThreads - 1) / kAggThreads, (uint32_t)W);
     k_agg_starts<M><<<sgrid, kAggThreads, 0, st>>>(msgs, (uint32_t)W, (uint32_t)k, ntiles, tile, ctx->d_agg_starts);
     ++ctx->launches;
@@ -646,16 +656,16 @@ int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_
   if (sparse) {
     // few coordinates are touched: clear the update, then compute only what was sent
     if (!out_cleared && eta < 0.0f) RTOPK_CUDA(ctx, cudaMemsetAsync(out, 0, (size_t)d * sizeof(float), st));
-    k_aggregate_sparse<M><<<ntiles, kAggThreads, 0, st>>>(msgs, own_search ? nullptr : ctx->d_agg_starts, (uint32_t)d,
+    k_aggregate_sparse<M><<<ntiles, kAggThreads, 0, st>>>(msgs, own_search ? nullptr : starts, (uint32_t)d,
                                                           (uint32_t)W, (uint32_t)k, sc, eta, out);
     ++ctx->launches;
   } else {
     if (sc.by_count)
       k_aggregate<M, true><<<ntiles, kAggThreads, 0, st>>>(msgs, ctx->d_agg_starts, (uint32_t)d, (uint32_t)W,
-                                                           (uint32_t)k, sc, eta, out);
+                                                           (uint32_t)k, sc, eta, out, mu, velocity);
     else
       k_aggregate<M, false><<<ntiles, kAggThreads, 0, st>>>(msgs, ctx->d_agg_starts, (uint32_t)d, (uint32_t)W,
-                                                            (uint32_t)k, sc, eta, out);
+                                                            (uint32_t)k, sc, eta, out, mu, velocity);
     ++ctx->launches;
   }
   mark(ctx, RTOPK_N_PHASES, st);
@@ -665,11 +675,11 @@ int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_
 
 int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
                    int scale_mode, float* out, cudaStream_t st, bool out_cleared = false, float eta = -1.0f,
-                   int64_t r = 0, uint32_t msg_stride = 1) {
+                   int64_t r = 0, uint32_t msg_stride = 1, float mu = 0.0f, float* velocity = nullptr) {
   if (!msg_idx || !msg_val || ((uintptr_t)msg_idx & 3u) || ((uintptr_t)msg_val & 3u)) return RTOPK_ERR_INVALID_ARG;
   if (k < 1 || k > 0xFFFFFFFFll) return RTOPK_ERR_INVALID_ARG;
   const PlainMsgs msgs = {msg_idx, msg_val, (uint32_t)k, msg_stride};
-  return aggregate_launch(ctx, msgs, d, W, k, scale_mode, out, st, out_cleared, eta, r);
+  return aggregate_launch(ctx, msgs, d, W, k, scale_mode, out, st, out_cleared, eta, r, mu, velocity);
 }
 
 int aggregate_threshold_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, const uint32_t* msg_count,
@@ -974,6 +984,83 @@ int rtopk_aggregate_packed(rtopk_ctx* ctx, const uint32_t* packed_idx, int64_t l
   if (scale_mode == RTOPK_SCALE_UNBIASED) return RTOPK_ERR_INVALID_ARG;   // needs r: scale the result by r / k instead
   const PackedMsgs msgs = {packed_idx, packed_val, (uint32_t)ld_words, (uint32_t)ld_halves, (uint32_t)bits};
   return aggregate_launch(ctx, msgs, d, W, k, scale_mode, out, (cudaStream_t)stream, false, -1.0f, 0);
+}
+
+int rtopk_tiled_layout(int64_t d, int64_t k, int64_t* spans, int64_t* ld_low, int64_t* ld_halves) {
+  if (d < 1 || d > 0xFFFFFFFFll || k < 1 || k > d) return RTOPK_ERR_INVALID_ARG;
+  if (spans) *spans = (d + kTiledSpan - 1) / kTiledSpan;
+  if (ld_low) *ld_low = (k + 7) / 8 * 8;
+  if (ld_halves) *ld_halves = (k + 7) / 8 * 8;
+  return RTOPK_OK;
+}
+
+int rtopk_encode_tiled(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
+                       float* residual, int64_t ld_m, uint32_t* span_tab, uint16_t* low_idx, int64_t ld_low,
+                       uint16_t* packed_val, int64_t ld_halves, void* stream) {
+  if (!ctx || !msg_idx || !msg_val || !span_tab || !low_idx || !packed_val) return RTOPK_ERR_INVALID_ARG;
+  if (W < 1 || W > ctx->W_max || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
+  int64_t spans = 0, min_low = 0, min_halves = 0;
+  if (rtopk_tiled_layout(d, k, &spans, &min_low, &min_halves)) return RTOPK_ERR_INVALID_ARG;
+  if (ld_low < min_low || ld_halves < min_halves || ld_low > 0xFFFFFFFFll || ld_halves > 0xFFFFFFFFll || (ld_low % 8) ||
+      (ld_halves % 8))
+    return RTOPK_ERR_INVALID_ARG;
+  if (((uintptr_t)msg_idx & 3u) || ((uintptr_t)msg_val & 3u) || ((uintptr_t)span_tab & 3u) || ((uintptr_t)low_idx & 15u) ||
+      ((uintptr_t)packed_val & 15u))
+    return RTOPK_ERR_INVALID_ARG;
+  if (residual && (ld_m < d || ((uintptr_t)residual & 3u))) return RTOPK_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return RTOPK_ERR_CUDA;
+  const uint32_t span = (uint32_t)std::max(ld_low, ld_halves);
+  const dim3 grid((span + kCodecThreads - 1) / kCodecThreads, (uint32_t)W);
+  k_encode_tiled<<<grid, kCodecThreads, 0, (cudaStream_t)stream>>>(msg_idx, msg_val, (uint32_t)k, (uint32_t)d, kTiledSpan,
+                                                                   (uint32_t)spans, residual, ld_m, span_tab, low_idx,
+                                                                   (uint32_t)ld_low, packed_val, (uint32_t)ld_halves);
+  ++ctx->launches;
+  RTOPK_CUDA(ctx, cudaGetLastError());
+  return RTOPK_OK;
+}
+
+int rtopk_aggregate_tiled(rtopk_ctx* ctx, const uint32_t* span_tab, const uint16_t* low_idx, int64_t ld_low,
+                          const uint16_t* packed_val, int64_t ld_halves, int64_t d, int32_t W, int64_t k,
+                          int scale_mode, float* out, void* stream) {
+  if (!span_tab || !low_idx || !packed_val || ((uintptr_t)span_tab & 3u) || ((uintptr_t)low_idx & 1u) ||
+      ((uintptr_t)packed_val & 1u))
+    return RTOPK_ERR_INVALID_ARG;
+  int64_t spans = 0;
+  if (rtopk_tiled_layout(d, k, &spans, nullptr, nullptr)) return RTOPK_ERR_INVALID_ARG;
+  if (ld_low < k || ld_halves < k || ld_low > 0xFFFFFFFFll || ld_halves > 0xFFFFFFFFll) return RTOPK_ERR_INVALID_ARG;
+  if (scale_mode == RTOPK_SCALE_UNBIASED) return RTOPK_ERR_INVALID_ARG;   // needs r: scale the result by r / k instead
+  const TiledMsgs msgs = {span_tab, low_idx, packed_val, (uint32_t)spans, (uint32_t)ld_low, (uint32_t)ld_halves};
+  return aggregate_launch(ctx, msgs, d, W, k, scale_mode, out, (cudaStream_t)stream, false, -1.0f, 0);
+}
+
+namespace {
+bool momentum_args_ok(float eta, float mu, const float* velocity, const float* weights) {
+  return (eta >= 0.0f) && eta <= 3.0e38f && (mu >= 0.0f) && (mu < 1.0f) && velocity && weights &&
+         !((uintptr_t)velocity & 15u) && !((uintptr_t)weights & 15u) && velocity != weights;
+}
+}  // namespace
+
+int rtopk_apply_momentum(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W,
+                         int64_t k, int scale_mode, int64_t r, float eta, float mu, float* velocity, float* weights,
+                         void* stream) {
+  if (!momentum_args_ok(eta, mu, velocity, weights)) return RTOPK_ERR_INVALID_ARG;
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, false, eta, r, 1, mu,
+                        velocity);
+}
+
+int rtopk_step_momentum(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
+                        int64_t d, int32_t W, int32_t worker_base, int64_t r, int64_t k, uint64_t seed, uint32_t step,
+                        int scale_mode, float eta, float mu, uint32_t* msg_idx, float* msg_val, float* velocity,
+                        float* weights, void* stream) {
+  if (!momentum_args_ok(eta, mu, velocity, weights) || !scale_mode_known(scale_mode)) return RTOPK_ERR_INVALID_ARG;
+  if (!ctx || d < 1 || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
+  const int64_t off[2] = {0, d};
+  const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed,
+                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, nullptr);
+  if (rc) return rc;
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, false, eta, r, 1, mu,
+                        velocity);
 }
 
 int rtopk_apply_update(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W,

@@ -432,6 +432,114 @@ def test_step_apply_is_sparsify_then_update(lib):
     ctx.close()
 
 
+def test_span_table_messages_against_oracle(lib):
+    """Encoder of the span-table format (entry counts per span of 16384 coordinates, 14 low index bits,
+    bfloat16 values, rounding error into the residual) and the aggregation that decodes on the fly:
+    bit-equal to the oracle's encoder and to the oracle's aggregate of the decoded messages.  Cases: few
+    entries per tile (sparse kernel, the table serves as its run starts), many (dense kernel), one span,
+    a ragged last span, rows that leave spans empty, more workers than one block's pass."""
+    rng = np.random.default_rng(2025)
+    cases = [(2_000_003, 8, 900), (100_003, 6, 20_000), (1 << 20, 3, 4097), (37, 2, 37), (16384, 5, 16384),
+             (16385, 4, 3), (5_000_000, 2, 40), (300_000, 300, 50)]
+    for d, W, k in cases:
+        idx = np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)]).astype(np.uint32)
+        val = (rng.standard_normal((W, k)) * np.exp(3 * rng.standard_normal((W, k)))).astype(np.float32)
+        val[0, 0] = 3.4e38                      # rounds to +inf in bfloat16
+        val[W - 1, k - 1] = np.float32(np.nan)
+        spans, ll, lh = lib.tiled_layout(d, k)
+        assert spans == oracle.tiled_spans(d) and ll >= k and ll % 8 == 0 and lh >= k and lh % 8 == 0
+        ld = wl.round_up(d, 4)
+        m0 = rng.standard_normal((W, ld)).astype(np.float32)
+        for w in range(W):
+            m0[w, idx[w].astype(np.int64)] = 0.0
+        m_ref = m0.copy()
+        o_tab, o_low, o_qv = oracle.encode_tiled(idx, val, d, residual=m_ref)
+        ctx = _ctx(lib, d, W, k, k)
+        t_idx, t_val = torch.from_numpy(idx.view(np.int32)).cuda(), torch.from_numpy(val).cuda()
+        m = torch.from_numpy(m0.copy()).cuda()
+        tab = torch.full((W, spans + 1), -1, dtype=torch.int32, device="cuda")
+        low = torch.full((W, ll), -1, dtype=torch.int16, device="cuda")
+        qv = torch.full((W, lh), -1, dtype=torch.int16, device="cuda")
+        ctx.encode_tiled(t_idx, t_val, d, tab, low, qv, residual=m)
+        assert np.array_equal(tab.cpu().numpy().view(np.uint32), o_tab)
+        got_low, got_qv = low.cpu().numpy().view(np.uint16), qv.cpu().numpy().view(np.uint16)
+        assert np.array_equal(got_low[:, :k], o_low) and not got_low[:, k:].any()
+        assert np.array_equal(got_qv[:, :k], o_qv) and not got_qv[:, k:].any()
+        assert np.array_equal(_bits(m.cpu().numpy()), _bits(m_ref))
+        d_idx, d_val = oracle.decode_tiled(o_tab, o_low, o_qv, d, k)
+        assert np.array_equal(d_idx, idx)
+        out = torch.full((ld,), float("nan"), dtype=torch.float32, device="cuda")
+        for mode, omode in ((lib.SCALE_MEAN, oracle.SCALE_MEAN), (lib.SCALE_SUM, oracle.SCALE_SUM),
+                            (lib.SCALE_COUNT, oracle.SCALE_COUNT)):
+            ctx.aggregate_tiled(tab, low, qv, d, k, out, scale_mode=mode)
+            _, want = oracle.aggregate(d_idx, d_val, d, omode)
+            assert np.array_equal(_bits(out.cpu().numpy()[:d]), _bits(want)), (d, W, k, mode)
+        # a table that claims more entries than the row holds is read as ending at k (nothing out of bounds)
+        bad = tab.clone()
+        bad[:, -1] = 2**31 - 1
+        ctx.aggregate_tiled(bad, low, qv, d, k, out)
+        torch.cuda.synchronize()
+        with pytest.raises(lib.RTopKError):
+            ctx.aggregate_tiled(tab, low, qv, d, k, out, scale_mode=lib.SCALE_UNBIASED)    # needs r
+        ctx.poll_status()
+        ctx.close()
+
+
+def test_momentum_update_against_oracle(lib):
+    """Heavy-ball master update: every coordinate's velocity and weight, bit for bit, over several rounds,
+    from given messages (all scalings) and fused behind the sparsifier."""
+    rng = np.random.default_rng(77)
+    for d, W, k in [(300_007, 4, 300), (5000, 3, 2500), (4096, 2, 1), (70_001, 70, 20)]:
+        ctx = _ctx(lib, d, W, k, k)
+        ld = wl.round_up(d, 4)
+        w0 = rng.standard_normal(ld).astype(np.float32)
+        v0 = (rng.standard_normal(ld) * 0.1).astype(np.float32)
+        for mode, omode, r in ((lib.SCALE_MEAN, oracle.SCALE_MEAN, 0), (lib.SCALE_COUNT, oracle.SCALE_COUNT, 0),
+                               (lib.SCALE_UNBIASED, oracle.SCALE_UNBIASED, min(d, 3 * k))):
+            w, v = torch.from_numpy(w0.copy()).cuda(), torch.from_numpy(v0.copy()).cuda()
+            want_v, want_w = v0[:d].copy(), w0[:d].copy()
+            for t in range(3):
+                idx = np.stack([np.sort(rng.choice(d, k, replace=False)) for _ in range(W)]).astype(np.uint32)
+                val = (rng.standard_normal((W, k)) * np.exp(rng.standard_normal((W, k)))).astype(np.float32)
+                ctx.apply_momentum(torch.from_numpy(idx.view(np.int32)).cuda(), torch.from_numpy(val).cuda(), d, 0.05,
+                                   0.9, v, w, scale_mode=mode, r=r)
+                want_v, want_w = oracle.apply_momentum(idx, val, d, 0.05, 0.9, want_v, want_w, omode, r)
+                assert np.array_equal(_bits(v.cpu().numpy()[:d]), _bits(want_v)), (d, W, k, mode, t)
+                assert np.array_equal(_bits(w.cpu().numpy()[:d]), _bits(want_w)), (d, W, k, mode, t)
+            assert np.array_equal(_bits(w.cpu().numpy()[d:]), _bits(w0[d:]))       # the padding is not touched
+        idx_t = torch.zeros((W, k), dtype=torch.int32, device="cuda")
+        val_t = torch.zeros((W, k), dtype=torch.float32, device="cuda")
+        w, v = torch.from_numpy(w0.copy()).cuda(), torch.from_numpy(v0.copy()).cuda()
+        for bad in (dict(eta=-0.1, mu=0.5), dict(eta=0.1, mu=1.0), dict(eta=0.1, mu=float("nan"))):
+            with pytest.raises(lib.RTopKError):
+                ctx.apply_momentum(idx_t, val_t, d, bad["eta"], bad["mu"], v, w)
+        with pytest.raises(lib.RTopKError):
+            ctx.apply_momentum(idx_t, val_t, d, 0.1, 0.5, w, w)
+        ctx.close()
+    # fused behind the sparsifier: three rounds of Algorithm 1 with the momentum master
+    cfg = wl.scaled(wl.configs()["c1"], d=300_007, W=4)
+    ctx = _ctx(lib, cfg.d, cfg.W, cfg.r, cfg.k)
+    w0 = rng.standard_normal(cfg.ld).astype(np.float32)
+    w = torch.from_numpy(w0.copy()).cuda()
+    v = torch.zeros(cfg.ld, dtype=torch.float32, device="cuda")
+    m = wl.zero_residual(cfg, "cuda")
+    m_ref = np.zeros((cfg.W, cfg.ld), dtype=np.float32)
+    idx = torch.zeros((cfg.W, cfg.k), dtype=torch.int32, device="cuda")
+    val = torch.zeros((cfg.W, cfg.k), dtype=torch.float32, device="cuda")
+    want_w, want_v = w0[:cfg.d].copy(), np.zeros(cfg.d, dtype=np.float32)
+    for t in range(3):
+        g = wl.gradient(cfg, t, "cuda")
+        ctx.step_momentum(g, m, cfg.d, cfg.r, cfg.k, cfg.seed, t, 0.1, 0.9, idx, val, v, w)
+        o_idx, o_val = oracle.sparsify(g.cpu().numpy(), m_ref, cfg.d, cfg.r, cfg.k, cfg.seed, t)
+        want_v, want_w = oracle.apply_momentum(o_idx, o_val, cfg.d, 0.1, 0.9, want_v, want_w)
+        assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx)
+        assert np.array_equal(_bits(m.cpu().numpy()), _bits(m_ref))
+        assert np.array_equal(_bits(v.cpu().numpy()[:cfg.d]), _bits(want_v))
+        assert np.array_equal(_bits(w.cpu().numpy()[:cfg.d]), _bits(want_w))
+    ctx.poll_status()
+    ctx.close()
+
+
 def test_threshold_reuse_changes_nothing_but_the_path(lib):
     """RTOPK_OPT_REUSE_THRESHOLD: consecutive rounds predict the first threshold from the last exact
     ones.  Messages, residual and update stay bit-equal to the oracle; the brackets are predicted
