@@ -452,6 +452,66 @@ def sweep_point(name, args, dev, peak, grads=None, steps=10, warmup=5, repeats=3
         torch.cuda.empty_cache()
 
 
+def message_and_master_point(name, args, dev):
+    """Times what follows the sparsifier on one configuration: the three message formats (encode, and the
+    aggregation with the decoder fused in) and the three master updates.  Device time per call in
+    microseconds, median of 20 calls behind a flush of L2 (the messages are a few MB)."""
+    import torch
+    import paper_2005_10761_b200 as rt
+    cfg = pick_workload(name)
+    a = argparse.Namespace(**vars(args))
+    a.apply, a.threshold, a.select_path, a.steps, a.warmup = False, None, "sampled", 2, 2
+    try:
+        rd = Round(cfg, a, dev, n_batches=1)
+    except Exception as ex:
+        return {"workload": name, "skipped": repr(ex)[:160]}
+    try:
+        ctx, d, W, k = rd.ctx, cfg.d, cfg.W, cfg.k
+        for t in range(2):
+            rd.step(t)
+        bits, lw, lh = rt.packed_layout(d, k)
+        spans, ll, lh2 = rt.tiled_layout(d, k)
+        pi = torch.zeros((W, lw), dtype=torch.int32, device=dev)
+        pv = torch.zeros((W, lh), dtype=torch.int16, device=dev)
+        tab = torch.zeros((W, spans + 1), dtype=torch.int32, device=dev)
+        low = torch.zeros((W, ll), dtype=torch.int16, device=dev)
+        qv = torch.zeros((W, lh2), dtype=torch.int16, device=dev)
+        weights = torch.zeros_like(rd.out)
+        velocity = torch.zeros_like(rd.out)
+        flush = torch.empty(2 * L2_BYTES // 4, dtype=torch.float32, device=dev)
+        calls = {
+            "encode_packed": lambda: ctx.encode(rd.idx, rd.val, d, pi, pv),
+            "encode_span_table": lambda: ctx.encode_tiled(rd.idx, rd.val, d, tab, low, qv),
+            "aggregate_plain": lambda: ctx.aggregate(rd.idx, rd.val, d, rd.out),
+            "aggregate_packed": lambda: ctx.aggregate_packed(pi, pv, d, k, rd.out),
+            "aggregate_span_table": lambda: ctx.aggregate_tiled(tab, low, qv, d, k, rd.out),
+            "apply_update": lambda: ctx.apply_update(rd.idx, rd.val, d, 0.01, weights),
+            "apply_momentum": lambda: ctx.apply_momentum(rd.idx, rd.val, d, 0.01, 0.9, velocity, weights),
+        }
+        us = {}
+        for label, fn in calls.items():
+            fn()
+            ts = []
+            for _ in range(20):
+                flush.fill_(1.0)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); fn(); e1.record()
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1) * 1e3)
+            us[label] = round(statistics.median(ts), 2)
+        ctx.poll_status()
+        return {"workload": name, "kind": "messages_and_master", "d": d, "W": W, "k": k, "us_per_call": us,
+                "bytes_per_entry": {"plain": 8.0, "packed": (bits + 16) / 8.0,
+                                    "span_table": (4.0 * (spans + 1) + 4.0 * k) / k},
+                "momentum_algorithmic_bytes": 16 * d, "l2": "flushed before every call"}
+    except Exception as ex:
+        return {"workload": name, "skipped": repr(ex)[:160]}
+    finally:
+        rd.close()
+        del rd
+        torch.cuda.empty_cache()
+
+
 def run_sweep(args, dev, peak):
     import torch
     from paper_2005_10761_b200 import workloads as wl
@@ -462,6 +522,8 @@ def run_sweep(args, dev, peak):
             out.append(sweep_point(name, args, dev, peak, steps=20, warmup=10))
     for name in ("c2", "c3_f32"):
         out.append(sweep_point(name, args, dev, peak, steps=10, warmup=3, select_path="exact"))
+    for name in ("c2", "c3_f32"):
+        out.append(message_and_master_point(name, args, dev))
     # c5: d = 2^28; one gradient batch of the largest row count is generated once and shared (every
     # point reads rows 0..W-1 of it; the vector is 8x the L2 already at W = 1)
     free_b, _ = torch.cuda.mem_get_info()

@@ -50,6 +50,54 @@ __device__ __forceinline__ uint32_t lower_bound_row(const M& msgs, uint32_t w, u
   return lo;
 }
 
+// Where the sparse kernel puts a coordinate's average: into the update (or, eta >= 0, into the weight), or --
+// heavy-ball momentum -- into velocity and weight, v <- mu v + ghat, w <- w - eta v, each rounded once from
+// double; it then marks the coordinate in `sent` (one bit per coordinate), and k_momentum_rest takes the others.
+struct AggOut {
+  float* out;
+  float eta, mu;
+  float* velocity;
+  uint32_t* sent;
+  __device__ __forceinline__ void store(uint32_t idx, float ghat) const {
+    if (velocity != nullptr) {
+      const float v = (float)((double)mu * (double)velocity[idx] + (double)ghat);
+      velocity[idx] = v;
+      out[idx] = (float)((double)out[idx] - (double)eta * (double)v);
+      atomicOr(sent + (idx >> 5), 1u << (idx & 31u));
+    } else {
+      out[idx] = agg_result(ghat, eta >= 0.0f ? out[idx] : 0.0f, eta);
+    }
+  }
+};
+
+// The coordinates no worker sent, under momentum: ghat is +0 there, so v <- fp32(mu v + 0), w <- fp32(w - eta v).
+// grid-stride over groups of four coordinates (velocity and weights are 16-byte aligned).
+__global__ void __launch_bounds__(256) k_momentum_rest(uint32_t d, float mu, float eta, const uint32_t* __restrict__ sent,
+                                                        float* __restrict__ velocity, float* __restrict__ weights) {
+  const uint32_t groups = (d + 3u) / 4u;
+  auto one = [&](float& v, float& w) {
+    v = (float)((double)mu * (double)v + 0.0);
+    w = (float)((double)w - (double)eta * (double)v);
+  };
+  for (uint32_t g = blockIdx.x * blockDim.x + threadIdx.x; g < groups; g += gridDim.x * blockDim.x) {
+    const uint32_t i = g * 4u;
+    const uint32_t nib = (__ldg(sent + (i >> 5)) >> (i & 31u)) & 0xFu;
+    if (i + 4u <= d) {
+      if (nib == 0xFu) continue;
+      float4 v = *reinterpret_cast<const float4*>(velocity + i), w = *reinterpret_cast<const float4*>(weights + i);
+      if (!(nib & 1u)) one(v.x, w.x);
+      if (!(nib & 2u)) one(v.y, w.y);
+      if (!(nib & 4u)) one(v.z, w.z);
+      if (!(nib & 8u)) one(v.w, w.w);
+      *reinterpret_cast<float4*>(velocity + i) = v;
+      *reinterpret_cast<float4*>(weights + i) = w;
+    } else {
+      for (uint32_t j = i; j < d; ++j)
+        if (!((nib >> (j - i)) & 1u)) { float v = velocity[j], w = weights[j]; one(v, w); velocity[j] = v; weights[j] = w; }
+    }
+  }
+}
+
 // The W x K messages as the kernels read them: plain (u32 index, f32 value) rows, or the packed
 // format (Section III: an index costs log d bits, a value a constant number): `bits` = ceil(log2 d)
 // bits per index, entry j at bits [j * bits, (j + 1) * bits) of the row's little-endian stream of
@@ -290,7 +338,9 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(M msgs, const uint32_
 template <typename M>
 __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const uint32_t* __restrict__ starts, uint32_t d,
                                                                   uint32_t W, uint32_t K, AggScale sc,
-                                                                  float eta, float* __restrict__ out) {
+                                                                  float eta, float* __restrict__ out, float mu,
+                                                                  float* __restrict__ velocity, uint32_t* __restrict__ sent) {
+  const AggOut dst = {out, eta, mu, velocity, sent};
   __shared__ uint32_t s_beg[kAggMaxW], s_pre[kAggMaxW + 1], s_cnt[kAggSearchW];
   __shared__ uint32_t st_idx[kAggSparseStage];
   __shared__ float st_val[kAggSparseStage];
@@ -385,7 +435,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
       if (local >= (uint32_t)kAggSparseTile || idx >= d) continue;   // malformed row: ignore
       if (!((s_shared[local >> 5] >> (local & 31u)) & 1u)) {
         const double v = msgs.term(st_w[q], st_val[q]);
-        out[idx] = agg_result((float)agg_scaled(v, 1u, sc), eta >= 0.0f ? out[idx] : 0.0f, eta);
+        dst.store(idx, (float)agg_scaled(v, 1u, sc));
       }
     }
     if (!any_shared) return;                                          // (block-uniform)
@@ -453,7 +503,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
         idx = st_idx[best];
         sum += msgs.term(st_w[best], st_val[best]);
       }
-      out[idx] = agg_result((float)agg_scaled(sum, e - b, sc), eta >= 0.0f ? out[idx] : 0.0f, eta);
+      dst.store(idx, (float)agg_scaled(sum, e - b, sc));
     }
     return;
   }
@@ -481,7 +531,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
       }
     }
     if (owner) {
-      out[idx] = agg_result((float)agg_scaled(sum, senders, sc), eta >= 0.0f ? out[idx] : 0.0f, eta);
+      dst.store(idx, (float)agg_scaled(sum, senders, sc));
     }
   }
 }

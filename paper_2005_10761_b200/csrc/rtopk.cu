@@ -45,6 +45,7 @@ struct rtopk_ctx {
   float* d_cand_val = nullptr;
   uint32_t* d_raw_idx = nullptr;
   float* d_raw_val = nullptr;
+  uint32_t* d_sent = nullptr;        // one bit per coordinate: updated by the sparse aggregation under momentum
   uint32_t* d_chunk_tab = nullptr;   // chunk_start | chunk_count | chunk_pre
   size_t chunk_tab_entries = 0;
   size_t cand_entries = 0;
@@ -628,7 +629,7 @@ int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_
   if (scale_mode == RTOPK_SCALE_COUNT && W > 65535) return RTOPK_ERR_UNSUPPORTED;
   if ((uintptr_t)out & 15u) return RTOPK_ERR_INVALID_ARG;
   if ((uint64_t)k * (uint64_t)W >= (1ull << 32)) return RTOPK_ERR_INVALID_ARG;
-  const bool sparse = aggregate_is_sparse(d, W, k) && velocity == nullptr;
+  const bool sparse = aggregate_is_sparse(d, W, k);
   const uint32_t tile = sparse ? (uint32_t)kAggSparseTile : (uint32_t)kAggTile;
   const uint32_t ntiles = (uint32_t)((d + tile - 1) / tile);
   // the span-table format brings the sparse kernel's table of run starts along
@@ -656,9 +657,18 @@ int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_
   if (sparse) {
     // few coordinates are touched: clear the update, then compute only what was sent
     if (!out_cleared && eta < 0.0f) RTOPK_CUDA(ctx, cudaMemsetAsync(out, 0, (size_t)d * sizeof(float), st));
+    // momentum: the sent coordinates are updated here and marked, the others by a plain pass behind it
+    if (velocity) RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_sent, 0, ((size_t)d + 31) / 32 * sizeof(uint32_t), st));
     k_aggregate_sparse<M><<<ntiles, kAggThreads, 0, st>>>(msgs, own_search ? nullptr : starts, (uint32_t)d,
-                                                          (uint32_t)W, (uint32_t)k, sc, eta, out);
+                                                          (uint32_t)W, (uint32_t)k, sc, eta, out, mu, velocity,
+                                                          ctx->d_sent);
     ++ctx->launches;
+    if (velocity) {
+      const uint32_t groups = (uint32_t)((d + 3) / 4);
+      const uint32_t blocks = std::min<uint32_t>((groups + 255u) / 256u, (uint32_t)ctx->sms * 16u);
+      k_momentum_rest<<<blocks, 256, 0, st>>>((uint32_t)d, mu, eta, ctx->d_sent, velocity, out);
+      ++ctx->launches;
+    }
   } else {
     if (sc.by_count)
       k_aggregate<M, true><<<ntiles, kAggThreads, 0, st>>>(msgs, ctx->d_agg_starts, (uint32_t)d, (uint32_t)W,
@@ -780,6 +790,7 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   alloc((void**)&ctx->d_step, 16);
   alloc((void**)&ctx->d_history, slices * sizeof(TauHistory));
   alloc((void**)&ctx->d_agg_starts, ctx->agg_start_entries * sizeof(uint32_t));
+  alloc((void**)&ctx->d_sent, ((size_t)d_max + 31) / 32 * sizeof(uint32_t) + 16);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_sample<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSampleSmemBytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_sample<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSampleSmemBytes);
   for (int i = 0; i <= RTOPK_N_PHASES && e == cudaSuccess; ++i) e = cudaEventCreate(&ctx->ev[i]);
@@ -841,7 +852,7 @@ int rtopk_destroy(rtopk_ctx* ctx) {
   void* ptrs[] = {ctx->d_slices, ctx->d_state, ctx->d_zero, ctx->d_first, ctx->d_cand_idx, ctx->d_cand_val,
                   ctx->d_raw_idx, ctx->d_raw_val, ctx->d_chunk_tab,
                   ctx->d_draws, ctx->d_sel_pre, ctx->d_sel_blk, ctx->d_error, ctx->d_agg_starts, ctx->d_stage, ctx->d_history,
-                  ctx->d_step, ctx->d_fin, ctx->d_list};
+                  ctx->d_step, ctx->d_fin, ctx->d_list, ctx->d_sent};
   for (void* p : ptrs) if (p) cudaFree(p);
   if (ctx->h_slices) cudaFreeHost(ctx->h_slices);
   for (cudaEvent_t ev : ctx->ev) if (ev) cudaEventDestroy(ev);
