@@ -75,8 +75,11 @@ enum { RTOPK_SCALE_MEAN = 0, RTOPK_SCALE_SUM = 1, RTOPK_SCALE_UNBIASED = 2, RTOP
 
 /* rtopk_set_option keys */
 enum {
-  RTOPK_OPT_SELECT_PATH = 0, /* 0 = automatic (sampled threshold with exact fallback),
-                                1 = always the multi-pass radix select over the full vector */
+  RTOPK_OPT_SELECT_PATH = 0, /* where the first bracket of the r-th largest magnitude comes from (the result
+                                is the same): 0 = from a sample of the slice, or from the slice's last
+                                thresholds with RTOPK_OPT_REUSE_THRESHOLD (a bracket that misses is repaired
+                                exactly); 1 = from an exact histogram of the 11 leading bits of every
+                                magnitude, one more pass that reads g and m: no sample, no statistics */
   RTOPK_OPT_PROFILE = 1,     /* 1 = record CUDA events between the phases of each call on the
                                 caller's stream (read with rtopk_get_phase_times); 0 = off */
   RTOPK_OPT_REUSE_THRESHOLD = 2, /* 1 = consecutive calls of one shape on one residual buffer predict the
@@ -104,22 +107,22 @@ enum {
                                 behind them for what they leave (a missed bracket, heavy ties); 0 (default) =
                                 2 for calls over 2^27 coordinates or more in all (rows x slice lengths), where
                                 the clusters' serial steps no longer hide behind one another, else 1 */
-  RTOPK_OPT_TEST_LOOKBACK_LIMIT = 6 /* for tests of the give-up path only: how often a block of the full-vector
-                                radix select (RTOPK_OPT_SELECT_PATH = 1) re-reads a predecessor's word that is
-                                still empty before it gives up (default 2^22).  0 makes every such wait give
-                                up at once: the call still returns, writes nothing outside the caller's
-                                buffers, its messages are then meaningless and rtopk_poll_status reports
-                                RTOPK_ERR_INTERNAL */
+  RTOPK_OPT_TEST_STREAM_GIVEUP = 6 /* for tests of the give-up path only: 1 = every block of the streaming pass
+                                behaves as if its first bounded wait had run out (consumers at once, the
+                                producer after a short wait for them).  The call still returns, all copies in
+                                flight are waited for, nothing outside the caller's buffers is written, the
+                                messages of that call are meaningless, and rtopk_poll_status reports
+                                RTOPK_ERR_INTERNAL.  0 = off (default) */
 };
 
 /* Phases of one call, in stream order.  STREAM is the single pass over the full vectors that
  * performs a = g + m, writes it back and gathers the coordinates above the threshold. */
 enum {
   RTOPK_PHASE_SUBSET = 0,    /* scratch clearing; the k-of-r subset itself runs beside the stream pass */
-  RTOPK_PHASE_THRESHOLD = 1, /* sampled bracket of the r-th largest magnitude */
+  RTOPK_PHASE_THRESHOLD = 1, /* first bracket of the r-th largest magnitude (sample, history or histogram pass) */
   RTOPK_PHASE_STREAM = 2,    /* the one kernel over W x d elements: add, write-back, candidate gathering */
   RTOPK_PHASE_ORDER = 3,     /* candidate runs laid out in index order; count check */
-  RTOPK_PHASE_EXACT = 4,     /* full-vector radix passes (RTOPK_OPT_SELECT_PATH = 1 only; empty otherwise) */
+  RTOPK_PHASE_EXACT = 4,     /* empty (kept so that the phase numbers stay what they were) */
   RTOPK_PHASE_FINISH = 5,    /* exact threshold among the candidates (over the whole slice where the first
                                 threshold missed), messages, residual zeroing */
   RTOPK_PHASE_AGGREGATE = 6, /* master average (step calls only) */
@@ -133,7 +136,7 @@ typedef struct {
   uint32_t tie_quota;   /* how many coordinates with exactly that magnitude are inside the top-r set */
   uint32_t n_greater;   /* coordinates with a strictly larger magnitude */
   uint32_t n_candidates;/* coordinates that survived the first threshold */
-  uint32_t used_fallback; /* 1 if the sampled threshold missed and the full radix select ran */
+  uint32_t used_fallback; /* 1 if the first bracket missed and the slice was selected over all its coordinates */
   uint32_t bracket_predicted; /* 1 if the first threshold came from the slice's history, not from a sample */
   uint32_t reserved[2];
 } rtopk_stats;

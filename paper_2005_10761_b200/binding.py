@@ -16,7 +16,7 @@ _LIB_PATH = os.path.join(_HERE, "librtopk.so")
 GRAD_F32, GRAD_BF16 = 0, 1
 SCALE_MEAN, SCALE_SUM, SCALE_UNBIASED, SCALE_COUNT = 0, 1, 2, 3
 OPT_SELECT_PATH, OPT_PROFILE, OPT_REUSE_THRESHOLD, OPT_THRESHOLD_SIGNS, OPT_DEVICE_STEP, OPT_FINISH_PATH = 0, 1, 2, 3, 4, 5
-OPT_TEST_LOOKBACK_LIMIT = 6
+OPT_TEST_STREAM_GIVEUP = 6
 PHASES = ("subset", "threshold", "stream", "order", "exact", "finish", "aggregate")
 
 _vp, _i32, _i64, _u32, _u64, _int = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_uint64, C.c_int

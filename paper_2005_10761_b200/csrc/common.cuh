@@ -1,5 +1,5 @@
 // Shared device-side definitions of the rTop-k library: slice descriptors, selection state,
-// scans, the bounded decoupled look-back and Philox4x32-10.
+// scans and Philox4x32-10.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -30,7 +30,7 @@ constexpr int kSampleThreads = 1024;
 // stage of the full-vector radix select of one slice
 enum : uint32_t { STAGE_PASS0 = 0, STAGE_PASS1 = 1, STAGE_PASS2 = 2, STAGE_COLLECT = 3, STAGE_DONE = 4 };
 enum : uint32_t { FLAG_GENERAL = 1u, FLAG_FELL_BACK = 2u, FLAG_FINISHED = 4u /* finished by the run kernels (finish.cuh) */ };
-enum : uint32_t { ERR_LOOKBACK_TIMEOUT = 1u, ERR_CANDIDATE_OVERFLOW = 2u, ERR_SELECT_INCONSISTENT = 4u };
+enum : uint32_t { ERR_WAIT_TIMEOUT = 1u, ERR_CANDIDATE_OVERFLOW = 2u, ERR_SELECT_INCONSISTENT = 4u };
 
 // One slice: a worker row, or one tensor of a worker row.  Offsets are in elements.
 struct Slice {
@@ -95,8 +95,7 @@ struct Scratch {
   SelState* state;
   uint32_t* hist;         // [slices][kBins]
   uint32_t* done;         // [slices] block-completion counters
-  uint32_t* tickets;      // [0], [1] tile counters of the exact collect; [2] grid-barrier counter; [3] chunk counter of k_stream
-  unsigned long long* look_b;   // look-back words of the exact path's collect
+  uint32_t* tickets;      // [3] chunk counter of k_stream ([0..2] unused)
   uint32_t* cursor;       // [slices] next free entry of the raw candidate buffer (= candidates so far)
   uint32_t* group_total;  // candidates per chunk group (summed by the stream pass)
   uint32_t* chunk_start;  // [chunks] where a chunk's run sits in the raw buffer ...
@@ -129,9 +128,7 @@ struct Launch {
   uint32_t seed_lo, seed_hi;
   uint32_t step;
   const uint32_t* step_ptr;   // not null: the round number is read from this device word instead of `step`
-  uint32_t general_primary;   // 1: the full-vector radix select is the main path, not a fallback
   uint32_t reuse;             // 1: brackets may be predicted from the slices' threshold history
-  int32_t lookback_limit;     // spin limit of the exact path's look-back (kLookSpinLimit unless a test lowers it)
 };
 
 // ----------------------------------------------------------------------------- small helpers
@@ -170,75 +167,6 @@ __device__ __forceinline__ uint32_t find_slice(uint32_t n, uint32_t t, F begin) 
     if (begin(mid) <= t) lo = mid; else hi = mid;
   }
   return lo;
-}
-
-// ----------------------------------------------------------------------------- look-back
-// Decoupled look-back over tiles of one slice, carrying two 31-bit counters.  Word layout:
-// bits 63..62 = 0 empty / 1 tile aggregate / 2 inclusive prefix; bits 61..31 = A; bits 30..0 = B.
-// Tiles are handed out by a ticket counter, so every predecessor of a waiting tile is already
-// running and publishes its aggregate before it waits itself.  Waits are bounded: on expiry the
-// error flag is raised and a zero prefix is returned (all later writes stay bounds-checked).
-constexpr unsigned long long kLookAgg = 1ull << 62, kLookIncl = 2ull << 62;
-constexpr uint32_t kLookMask31 = 0x7FFFFFFFu;
-constexpr int kLookSpinLimit = 1 << 22;
-
-__device__ __forceinline__ unsigned long long look_pack(unsigned long long flag, uint32_t a, uint32_t b) {
-  return flag | ((unsigned long long)(a & kLookMask31) << 31) | (unsigned long long)(b & kLookMask31);
-}
-__device__ __forceinline__ unsigned long long ld_relaxed(const unsigned long long* p) {
-  unsigned long long v;
-  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void st_relaxed(unsigned long long* p, unsigned long long v) {
-  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-
-// Called by all 32 lanes of one warp.  `words` points at the slice's tile 0, `tile` is the tile
-// inside the slice, (aggA, aggB) the tile's own counts.  Returns the exclusive prefix in
-// (exA, exB) on every lane.
-// `spin_limit` = how often a lane re-reads a word that is still empty before the warp gives up (0: at
-// once, which is what the test of the give-up path asks for).
-__device__ __forceinline__ void lookback_exclusive(unsigned long long* words, uint32_t tile, uint32_t aggA,
-                                                   uint32_t aggB, uint32_t& exA, uint32_t& exB,
-                                                   uint32_t* error, int spin_limit = kLookSpinLimit) {
-  const uint32_t lane = lane_id();
-  if (tile == 0) {
-    if (lane == 0) st_relaxed(words, look_pack(kLookIncl, aggA, aggB));
-    exA = 0; exB = 0;
-    return;
-  }
-  if (lane == 0) st_relaxed(words + tile, look_pack(kLookAgg, aggA, aggB));
-  uint32_t sumA = 0, sumB = 0;
-  int64_t top = (int64_t)tile - 1;          // newest tile not yet accounted for
-  bool failed = spin_limit == 0;            // (a limit of zero gives up without looking: the give-up path under test)
-  while (!failed) {
-    const int64_t mine = top - lane;
-    unsigned long long w = kLookIncl;       // lanes before tile 0 read as "inclusive, zero"
-    if (mine >= 0) {
-      int spins = 0;
-      w = ld_relaxed(words + mine);
-      while ((w >> 62) == 0) {
-        if (++spins > spin_limit) { failed = true; break; }
-        __nanosleep(40);
-        w = ld_relaxed(words + mine);
-      }
-    }
-    if (__any_sync(0xFFFFFFFFu, failed)) { failed = true; break; }
-    const uint32_t incl_mask = __ballot_sync(0xFFFFFFFFu, (w >> 62) == 2);
-    const uint32_t stop = incl_mask ? (uint32_t)(__ffs(incl_mask) - 1) : 32u;   // first inclusive lane
-    const bool use = lane <= stop;
-    sumA += warp_sum(use ? (uint32_t)((w >> 31) & kLookMask31) : 0u);
-    sumB += warp_sum(use ? (uint32_t)(w & kLookMask31) : 0u);
-    if (incl_mask) break;
-    top -= 32;
-  }
-  if (failed) {
-    if (lane == 0) atomicOr(error, ERR_LOOKBACK_TIMEOUT);
-    sumA = 0; sumB = 0;
-  }
-  if (lane == 0) st_relaxed(words + tile, look_pack(kLookIncl, sumA + aggA, sumB + aggB));
-  exA = sumA; exB = sumB;
 }
 
 // ----------------------------------------------------------------------------- digit pick

@@ -38,8 +38,8 @@ __device__ __forceinline__ float ef_add(float g, float m) {
 
 // Loads the 4 elements e..e+3 of the slice's aligned element grid (element `head` is the slice's
 // first coordinate, `span` = head + len is one past its last), forms a = g + m when FUSE and
-// stores it back, and returns the values with a 4-bit validity mask.
-template <typename GradT, bool FUSE>
+// stores it back when STORE, and returns the values with a 4-bit validity mask.
+template <typename GradT, bool FUSE, bool STORE = FUSE>
 __device__ __forceinline__ uint32_t load_vec(const void* grad, float* residual, int64_t base_g, int64_t base_m,
                                              uint32_t e, uint32_t head, uint32_t span, float (&a)[4]) {
   if (e >= span) { a[0] = a[1] = a[2] = a[3] = 0.f; return 0u; }
@@ -50,7 +50,7 @@ __device__ __forceinline__ uint32_t load_vec(const void* grad, float* residual, 
       const float4 g4 = Grad<GradT>::ld4(grad, base_g + e);
       m4.x = ef_add(g4.x, m4.x); m4.y = ef_add(g4.y, m4.y);
       m4.z = ef_add(g4.z, m4.z); m4.w = ef_add(g4.w, m4.w);
-      __stcs(reinterpret_cast<float4*>(residual + base_m + e), m4);
+      if (STORE) __stcs(reinterpret_cast<float4*>(residual + base_m + e), m4);
     }
     a[0] = m4.x; a[1] = m4.y; a[2] = m4.z; a[3] = m4.w;
     return 0xFu;
@@ -62,7 +62,7 @@ __device__ __forceinline__ uint32_t load_vec(const void* grad, float* residual, 
     a[j] = 0.f;
     if (ee >= head && ee < span) {
       float v = residual[base_m + ee];
-      if (FUSE) { v = ef_add(Grad<GradT>::ld1(grad, base_g + ee), v); residual[base_m + ee] = v; }
+      if (FUSE) { v = ef_add(Grad<GradT>::ld1(grad, base_g + ee), v); if (STORE) residual[base_m + ee] = v; }
       a[j] = v;
       valid |= 1u << j;
     }

@@ -32,12 +32,12 @@ struct rtopk_ctx {
   int32_t W_max = 0, S_max = 0;
   int select_path = 0;
   int finish_path = 0;                // RTOPK_OPT_FINISH_PATH
-  int lookback_limit = kLookSpinLimit; // RTOPK_OPT_TEST_LOOKBACK_LIMIT
+  int test_giveup = 0;                // RTOPK_OPT_TEST_STREAM_GIVEUP
   int last_cuda_error = 0;
   // device scratch (one allocation each)
   Slice* d_slices = nullptr;
   SelState* d_state = nullptr;
-  char* d_zero = nullptr;        // counters, histograms, look-back words, bitmaps: cleared per call
+  char* d_zero = nullptr;        // counters, histograms, bitmaps: cleared per call
   size_t zero_bytes = 0;
   uint32_t* d_first = nullptr;   // first-occurrence tables: set to 0xFF per call
   size_t first_entries = 0;
@@ -86,7 +86,6 @@ struct rtopk_ctx {
   uint64_t launches = 0;                          // kernels launched by this context so far
   int finish_max_clusters[kMaxCluster + 1] = {};  // [cs]: co-resident k_finish clusters of size cs (1..16)
   int stream_blocks[2] = {0, 0};      // persistent grid of k_stream per gradient dtype
-  int exact_blocks = 0;               // cooperative grid of k_exact (all blocks resident)
   // work that does not depend on the data (the k-of-r subset, clearing the dense update) runs on a
   // side stream next to the streaming pass
   cudaStream_t side = nullptr;
@@ -247,7 +246,6 @@ size_t carve_zero(const rtopk_ctx* ctx, const Plan& P, Scratch& s, size_t* early
   s.group_total = (uint32_t*)take((size_t)P.n_groups * sizeof(uint32_t));
   if (early_bytes) *early_bytes = at;
   s.hist = (uint32_t*)take(P.slices.size() * kBins * sizeof(uint32_t));
-  s.look_b = (unsigned long long*)take((size_t)P.n_chunks * 8);
   s.sel = (uint32_t*)take(P.sel_words * sizeof(uint32_t));
   return at;
 }
@@ -256,7 +254,7 @@ size_t zero_region_bytes(size_t slices, size_t chunks, size_t groups, size_t sel
   size_t at = 0;
   auto take = [&](size_t bytes) { at = align_up(at + bytes, 256); };
   take(16); take(slices * 4); take(slices * 4); take(groups * 4);
-  take(slices * kBins * 4); take(chunks * 8); take(sel_words * 4);
+  take(slices * kBins * 4); take(sel_words * 4);
   return at;
 }
 
@@ -274,63 +272,53 @@ int check_common(const rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t
   return RTOPK_OK;
 }
 
-// Passes first_pass..2 of the full-vector radix select plus the ordered collect, as one cooperative
-// launch (its blocks meet at grid barriers, so all of them must be resident).
-int launch_exact(rtopk_ctx* ctx, const Plan& P, const Launch& L, int first_pass, cudaStream_t st) {
-  Launch Lc = L;
-  int fp = first_pass;
-  uint32_t nh = P.n_hist_blocks, nc = P.n_chunks;
-  void* args[] = {&Lc, &fp, &nh, &nc};
-  RTOPK_CUDA(ctx, cudaLaunchCooperativeKernel((const void*)k_exact, dim3((unsigned)ctx->exact_blocks), dim3(kThreads),
-                                              args, 0, st));
-  ++ctx->launches;
-  return RTOPK_OK;
-}
-
 template <typename GradT>
 int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st, cudaEvent_t join,
                   float* clear_out, size_t clear_bytes) {
   const uint32_t n = (uint32_t)P.slices.size();
   int rc = RTOPK_OK;
+  auto stream_pass = [&]() -> int {
+    mark(ctx, RTOPK_PHASE_STREAM, st);
+    const uint32_t per = (uint32_t)((P.slices[0].head + (uint64_t)P.slices[0].len + kChunk - 1) / kChunk);
+    const uint32_t uniform = P.uniform ? per : 0u;
+    const int blocks = ctx->stream_blocks[sizeof(GradT) == 4 ? 0 : 1];
+    if (ctx->test_giveup) k_stream<GradT, true><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
+    else k_stream<GradT, false><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
+    ++ctx->launches;
+    if (clear_out) {
+      // the streaming pass saturates the memory system and the kernels after it do not: the dense
+      // update is cleared on the side stream once the pass has ended
+      RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_streamed, st));
+      RTOPK_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_streamed, 0));
+      RTOPK_CUDA(ctx, cudaMemsetAsync(clear_out, 0, clear_bytes, ctx->side));
+      RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_cleared, ctx->side));
+    }
+    mark(ctx, RTOPK_PHASE_ORDER, st);
+    mark(ctx, RTOPK_PHASE_EXACT, st);
+    return RTOPK_OK;
+  };
   if (ctx->select_path == 0) {
     mark(ctx, RTOPK_PHASE_THRESHOLD, st);
     k_sample<GradT><<<n, kSampleThreads, kSampleSmemBytes, st>>>(L);
     ++ctx->launches;
-    mark(ctx, RTOPK_PHASE_STREAM, st);
-    {
-      const uint32_t per = (uint32_t)((P.slices[0].head + (uint64_t)P.slices[0].len + kChunk - 1) / kChunk);
-      const uint32_t uniform = P.uniform ? per : 0u;
-      const int blocks = ctx->stream_blocks[sizeof(GradT) == 4 ? 0 : 1];
-      k_stream<GradT, false><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
-      ++ctx->launches;
-      if (clear_out) {
-        // the streaming pass saturates the memory system and the kernels after it do not: the dense
-        // update is cleared on the side stream once the pass has ended
-        RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_streamed, st));
-        RTOPK_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_streamed, 0));
-        RTOPK_CUDA(ctx, cudaMemsetAsync(clear_out, 0, clear_bytes, ctx->side));
-        RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_cleared, ctx->side));
-      }
-      mark(ctx, RTOPK_PHASE_ORDER, st);
-    }
-    mark(ctx, RTOPK_PHASE_EXACT, st);
+    rc = stream_pass();
+    if (rc) return rc;
     // k_finish needs the subset (side stream); a slice whose bracket missed is selected exactly inside
     // its k_finish cluster, so no kernel of the exact path is launched here
     if (join) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, join, 0));
   } else {
+    // the bracket from a histogram over the full vector; from there on as above
     mark(ctx, RTOPK_PHASE_THRESHOLD, st);
-    k_init_state<<<(n + 127) / 128, 128, 0, st>>>(L, 1u);
+    k_init_state<<<(n + 127) / 128, 128, 0, st>>>(L, 0u);
     ++ctx->launches;
-    mark(ctx, RTOPK_PHASE_STREAM, st);
-    const uint32_t hgrid = std::min<uint32_t>(P.n_hist_blocks, (uint32_t)ctx->sms * 8u);
-    k_hist<GradT, true><<<hgrid, kThreads, 0, st>>>(L, 0, P.n_hist_blocks);
-    ++ctx->launches;
-    mark(ctx, RTOPK_PHASE_ORDER, st);
-    mark(ctx, RTOPK_PHASE_EXACT, st);
     if (P.any_select) {
-      rc = launch_exact(ctx, P, L, 1, st);
-      if (rc) return rc;
+      const uint32_t hgrid = std::min<uint32_t>(P.n_hist_blocks, (uint32_t)ctx->sms * 8u);
+      k_bracket<GradT><<<hgrid, kThreads, 0, st>>>(L, P.n_hist_blocks);
+      ++ctx->launches;
     }
+    rc = stream_pass();
+    if (rc) return rc;
+    if (join) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, join, 0));
   }
   return RTOPK_OK;
 }
@@ -392,12 +380,10 @@ int bind_launch(rtopk_ctx* ctx, const Plan& P, const void* grad, float* residual
   L.s.fin = ctx->d_fin; L.s.list = ctx->d_list;
   L.grad = grad; L.residual = residual; L.msg_idx = msg_idx; L.msg_val = msg_val;
   L.msg_stride = 1;
-  L.lookback_limit = ctx->lookback_limit;
   L.n_slices = (uint32_t)P.slices.size();
   L.worker_base = (uint32_t)worker_base;
   L.seed_lo = (uint32_t)seed; L.seed_hi = (uint32_t)(seed >> 32);
   L.step = step;
-  L.general_primary = ctx->select_path == 1 ? 1u : 0u;
   L.step_ptr = ctx->device_step ? ctx->d_step : nullptr;
   return RTOPK_OK;
 }
@@ -440,7 +426,7 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   }
   mark(ctx, RTOPK_PHASE_SUBSET, st);
   // The sampling kernels clear the leading counters of the zeroed region themselves; the exact
-  // primary path has no such kernel.  The rest (exact-path histograms and look-back words, the
+  // primary path has no such kernel.  The rest (the histograms, the
   // selection bitmap) is first touched by the sampler and the exact path, both behind the fork.
   const bool late_on_side = ctx->select_path == 0;
   if (!late_on_side) RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero, 0, zbytes, st));
@@ -467,12 +453,10 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   rc = grad_dtype == RTOPK_F32 ? launch_select<float>(ctx, P, L, st, join, clear_late, clear_bytes)
                                : launch_select<__nv_bfloat16>(ctx, P, L, st, join, clear_late, clear_bytes);
   if (rc) return rc;
-  // (on the sampled path launch_select has made the stream wait for the side stream before its last kernel)
-  const bool joined = forked && ctx->select_path == 0;
-  if (forked && !joined) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0));
+  // (launch_select has made the stream wait for the side stream behind the streaming pass)
   mark(ctx, RTOPK_PHASE_FINISH, st);
   const bool from_runs = ctx->finish_path == 2 || (ctx->finish_path == 0 && P.n_chunks >= (1u << 15));
-  if (P.any_select && ctx->select_path == 0 && from_runs && L.n_slices <= 65535u) {
+  if (P.any_select && from_runs && L.n_slices <= 65535u) {
     // the usual case is finished straight from the streaming pass's runs, all slices side by side; what
     // these kernels leave (a missed bracket, heavy ties) is flagged for k_finish
     // about one wave of blocks over all slices together (8 blocks of 256 threads per SM)
@@ -822,14 +806,10 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
     if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<float>));
     if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<__nv_bfloat16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<__nv_bfloat16>));
     if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<__nv_bfloat16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<__nv_bfloat16>));
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_f32, k_stream<float, true>, kStreamThreads, sizeof(StreamSmem<float>));
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_bf16, k_stream<__nv_bfloat16, true>, kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>));
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_f32, k_stream<float, false>, kStreamThreads, sizeof(StreamSmem<float>));
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_bf16, k_stream<__nv_bfloat16, false>, kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>));
     if (e == cudaSuccess && (per_f32 < 1 || per_bf16 < 1)) e = cudaErrorLaunchOutOfResources;
     ctx->sms = sms;
-    int per_exact = 0;
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_exact, k_exact, kThreads, 0);
-    if (e == cudaSuccess && per_exact < 1) e = cudaErrorLaunchOutOfResources;
-    ctx->exact_blocks = sms * std::min(per_exact, 4);
     ctx->stream_blocks[0] = sms * per_f32;
     ctx->stream_blocks[1] = sms * per_bf16;
   }
@@ -882,7 +862,7 @@ int rtopk_set_option(rtopk_ctx* ctx, int option, int64_t value) {
   }
   if (option == RTOPK_OPT_DEVICE_STEP && (value == 0 || value == 1)) { ctx->device_step = (int)value; return RTOPK_OK; }
   if (option == RTOPK_OPT_FINISH_PATH && value >= 0 && value <= 2) { ctx->finish_path = (int)value; return RTOPK_OK; }
-  if (option == RTOPK_OPT_TEST_LOOKBACK_LIMIT && value >= 0 && value <= kLookSpinLimit) { ctx->lookback_limit = (int)value; return RTOPK_OK; }
+  if (option == RTOPK_OPT_TEST_STREAM_GIVEUP && (value == 0 || value == 1)) { ctx->test_giveup = (int)value; return RTOPK_OK; }
   if (option == RTOPK_OPT_THRESHOLD_SIGNS && (value == 0 || value == 1)) { ctx->threshold_signs = (int)value; return RTOPK_OK; }
   if (option == RTOPK_OPT_PROFILE && (value == 0 || value == 1)) {
     ctx->profile = (int)value;

@@ -4,10 +4,8 @@
 //   k_sample        brackets the r-th largest key of every slice from a strided sample of a = g + m
 //                   (or, with threshold reuse, from the slice's last exact thresholds) and clears
 //                   the counters of the streaming pass (k_stream, stream.cuh)
-//   k_exact         the exact path over the full vector, one cooperative launch: three radix histogram
-//                   passes (hist_body) and an index-ordered collect (collect_body, ballot-free
-//                   prefix compaction + bounded look-back); the main path behind k_hist (fused add in
-//                   pass 0) when the caller asks for it
+//   k_bracket       the same bracket from a histogram of the 11 leading key bits over the whole slice
+//                   instead of a sample, when the caller asks for it (one more pass over g and m)
 //   k_finish        one cluster per slice: candidate runs -> index order, exact r-th largest key
 //                   among the candidates, then a walk over the candidates in index order that
 //                   numbers the members of the top-r set and writes the ones the k-of-r sampler
@@ -54,6 +52,7 @@ __global__ void k_init_state(Launch L, uint32_t general) {
   if (S.r == S.len) { st.resolved = 31; st.stage = STAGE_DONE; st.flags = 0; }   // top-r is everything
   else { st.resolved = 0; st.stage = STAGE_PASS0; st.flags = general ? FLAG_GENERAL : 0u; }
   L.s.state[s] = st;
+  L.s.fin[s].list_n = 0; L.s.fin[s].done1 = 0; L.s.fin[s].done2 = 0; L.s.fin[s].b_ok = 0;
 }
 
 // ----------------------------------------------------------------------------- sampled threshold
@@ -276,155 +275,6 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample(Launch L) {
   if (tid == 0) L.s.state[sl] = st;
 }
 
-// ----------------------------------------------------------------------------- collect
-// TIES = false: candidates are the keys >= tau_lo.  TIES = true: keys > tau_lo and the first
-// eq_quota keys == tau_lo in index order.  The candidate list keeps index order: inside a block by
-// ballot-free packed prefix sums, across blocks by the look-back on (count above, count equal).
-template <typename GradT, bool FUSE, bool TIES>
-__device__ __forceinline__ void collect_body(const Launch& L, uint32_t total_tiles) {
-  __shared__ uint32_t s_tile, s_wA[kWarps], s_wB[kWarps], s_ex[2];
-  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const Slice* slices = L.s.slices;
-  // persistent blocks; tiles are handed out by ticket so that the look-back only ever waits on
-  // tiles whose blocks are already running
-  while (true) {
-  __syncthreads();
-  if (tid == 0) s_tile = atomicAdd(&L.s.tickets[FUSE ? 0 : 1], 1u);
-  __syncthreads();
-  const uint32_t tile = s_tile;
-  if (tile >= total_tiles) return;
-  const uint32_t sl = find_slice(L.n_slices, tile, [&](uint32_t i) { return slices[i].chunk_begin; });
-  const Slice S = slices[sl];
-  volatile SelState* st = &L.s.state[sl];   // other blocks update it inside one launch: no L1
-  if (!FUSE) {
-    if (!((st->flags & FLAG_GENERAL) && st->stage == STAGE_COLLECT)) continue;
-  }
-  const uint32_t tau = st->tau_lo;
-  const uint32_t quota = TIES ? st->eq_quota : kNoQuota;
-  const uint32_t c = tile - S.chunk_begin;
-  const uint32_t span = S.head + S.len;
-  const int64_t base_g = S.g_off - S.head, base_m = S.m_off - S.head;
-  const uint32_t e_w = c * (uint32_t)kChunk + warp * (uint32_t)kWarpSpan;
-
-  float a[kIter][4];
-  uint32_t maskA = 0, maskB = 0;
-#pragma unroll
-  for (int it = 0; it < kIter; ++it) {
-    const uint32_t e = e_w + it * 128u + lane * 4u;
-    const uint32_t valid = load_vec<GradT, FUSE>(L.grad, L.residual, base_g, base_m, e, S.head, span, a[it]);
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const uint32_t key = mag_key(a[it][j]);
-      const bool ok = (valid >> j) & 1u;
-      if (TIES) {
-        maskA |= (uint32_t)(ok && key > tau) << (it * 4 + j);
-        maskB |= (uint32_t)(ok && key == tau) << (it * 4 + j);
-      } else {
-        maskA |= (uint32_t)(ok && key >= tau) << (it * 4 + j);
-      }
-    }
-  }
-  // per-iteration counts packed one byte each (a byte holds at most 32 lanes x 4 = 128)
-  uint32_t packA = 0, packB = 0;
-#pragma unroll
-  for (int it = 0; it < kIter; ++it) {
-    packA |= (uint32_t)__popc((maskA >> (it * 4)) & 0xFu) << (it * 8);
-    if (TIES) packB |= (uint32_t)__popc((maskB >> (it * 4)) & 0xFu) << (it * 8);
-  }
-  const uint32_t inclA = warp_incl_scan(packA);
-  const uint32_t inclB = TIES ? warp_incl_scan(packB) : 0u;
-  const uint32_t totA = __shfl_sync(0xFFFFFFFFu, inclA, 31), totB = __shfl_sync(0xFFFFFFFFu, inclB, 31);
-  const uint32_t exLaneA = inclA - packA, exLaneB = inclB - packB;
-  uint32_t wA = 0, wB = 0;
-#pragma unroll
-  for (int it = 0; it < kIter; ++it) { wA += (totA >> (it * 8)) & 0xFFu; wB += (totB >> (it * 8)) & 0xFFu; }
-  if (lane == 0) { s_wA[warp] = wA; s_wB[warp] = wB; }
-  __syncthreads();
-  if (warp == 0) {
-    uint32_t bA = 0, bB = 0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) { bA += s_wA[w]; bB += s_wB[w]; }
-    uint32_t exA, exB;
-    unsigned long long* words = L.s.look_b + S.chunk_begin;
-    lookback_exclusive(words, c, bA, bB, exA, exB, L.s.error, L.lookback_limit);
-    if (lane == 0) {
-      s_ex[0] = exA; s_ex[1] = exB;
-      if (c + 1 == slice_chunks(S)) {      // last tile of the slice: publish the total
-        const uint32_t n = exA + bA + min(exB + bB, quota);
-        st->n_cand = n;
-        if (FUSE) st->n_cand_first = n;
-      }
-    }
-  }
-  __syncthreads();
-  if ((maskA | maskB) == 0) continue;
-  uint32_t gt_before = s_ex[0], eq_before = s_ex[1];
-  for (uint32_t w = 0; w < warp; ++w) { gt_before += s_wA[w]; eq_before += s_wB[w]; }
-  uint32_t* cidx = L.s.cand_idx + S.cand_off;
-  float* cval = L.s.cand_val + S.cand_off;
-#pragma unroll
-  for (int it = 0; it < kIter; ++it) {
-    uint32_t bitsA = (maskA >> (it * 4)) & 0xFu, bitsB = (maskB >> (it * 4)) & 0xFu;
-    if (bitsA | bitsB) {
-      uint32_t g = gt_before + ((exLaneA >> (it * 8)) & 0xFFu);
-      uint32_t q = eq_before + ((exLaneB >> (it * 8)) & 0xFFu);
-      const uint32_t e = e_w + it * 128u + lane * 4u;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const bool isA = (bitsA >> j) & 1u, isB = (bitsB >> j) & 1u;
-        if (isA || (isB && q < quota)) {
-          const uint32_t pos = g + min(q, quota);
-          if (pos < S.cand_cap) { cidx[pos] = e + j - S.head; cval[pos] = a[it][j]; }
-        }
-        g += isA; q += isB;
-      }
-    }
-    gt_before += (totA >> (it * 8)) & 0xFFu;
-    eq_before += (totB >> (it * 8)) & 0xFFu;
-  }
-  }
-}
-
-// ----------------------------------------------------------------------------- radix passes
-// Runs in the last block of a slice's histogram pass: turns the finished histogram into the next
-// digit of the r-th largest key.  `full_vector` passes also decide whether the bucket is small
-// enough to collect (or, with all 31 bits resolved, fix the exact threshold and tie quota).
-__device__ __forceinline__ void finish_pass(const Launch& L, uint32_t sl, const Slice& S, int pass,
-                                            bool full_vector, bool fell_back, uint32_t* hist_s,
-                                            uint32_t* scratch) {
-  const int bits = digit_bits(pass);
-  uint32_t* gh = L.s.hist + (size_t)sl * kBins;
-  for (uint32_t b = threadIdx.x; b < (uint32_t)kBins; b += blockDim.x) {
-    hist_s[b] = __ldcg(gh + b);
-    gh[b] = 0;
-  }
-  __syncthreads();
-  volatile SelState* st = &L.s.state[sl];   // other blocks update it inside one launch: no L1
-  const uint32_t need = st->need;
-  uint32_t D, above;
-  const bool ok = pick_digit(hist_s, 1 << bits, need, scratch, D, above);
-  if (threadIdx.x == 0) {
-    L.s.done[sl] = 0;
-    if (!ok) {
-      atomicOr(L.s.error, ERR_SELECT_INCONSISTENT);
-      st->stage = STAGE_DONE;
-      st->resolved = 32;     // blocks the later passes of this slice
-    } else {
-      const uint32_t n_gt = st->n_gt + above, need2 = need - above;
-      const uint32_t prefix = (st->prefix << bits) | D;
-      const uint32_t resolved = st->resolved + bits;
-      st->n_gt = n_gt; st->need = need2; st->prefix = prefix; st->resolved = resolved;
-      if (full_vector) {
-        const uint32_t n_ge = n_gt + hist_s[D];
-        if (n_ge <= S.cand_cap) { st->tau_lo = prefix << (31 - resolved); st->eq_quota = kNoQuota; st->stage = STAGE_COLLECT; }
-        else if (resolved == 31) { st->tau_lo = prefix; st->eq_quota = need2; st->stage = STAGE_COLLECT; }
-        else st->stage = pass + 1;
-        st->flags |= FLAG_GENERAL | (fell_back ? FLAG_FELL_BACK : 0u);
-      }
-    }
-  }
-}
-
 __device__ __forceinline__ bool is_last_block(uint32_t* counter, uint32_t nblocks) {
   __shared__ uint32_t s_last;
   __syncthreads();
@@ -443,27 +293,24 @@ __device__ __forceinline__ bool first_pass_missed(uint32_t n_gathered, const Sli
   return S.r < S.len && (n_gathered < S.r || n_gathered > S.cand_cap);
 }
 
-// Histogram of one digit over the whole slice.  FUSE (pass 0 of the exact path) also performs the
-// add and the write-back; otherwise a is read from the residual buffer.  Pass p > 0 counts only keys
-// whose higher bits equal the resolved prefix.
-template <typename GradT, bool FUSE>
-__device__ __forceinline__ void hist_body(const Launch& L, int pass, uint32_t total_blocks) {
+// The bracket of the r-th largest key from a histogram instead of a sample (RTOPK_OPT_SELECT_PATH = 1): one
+// pass reads g and m, forms a = g + m (nothing is stored: the streaming pass does that) and counts the 11
+// leading bits of every key; the last block of a slice picks the bucket that holds the r-th largest key, and
+// the bucket's bounds are the bracket.  It cannot miss; the streaming pass then gathers the keys of this
+// bucket and above -- more than a sampled bracket would let through, and more than the candidate list
+// holds when very many keys share 11 leading bits, which the finishing kernels repair like any overflow.
+// grid: up to total_blocks blocks; a unit is kHistChunks chunks of one slice.
+template <typename GradT>
+__global__ void __launch_bounds__(kThreads) k_bracket(Launch L, uint32_t total_blocks) {
   __shared__ uint32_t hist_s[kBins];
   __shared__ uint32_t scratch[kWarps + 2];
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const Slice* slices = L.s.slices;
-  const int bits = digit_bits(pass), shift = digit_shift(pass);
   for (uint32_t unit = blockIdx.x; unit < total_blocks; unit += gridDim.x) {
     __syncthreads();                                   // hist_s / scratch of the previous unit are free
     const uint32_t sl = find_slice(L.n_slices, unit, [&](uint32_t i) { return slices[i].hist_begin; });
     const Slice S = slices[sl];
-    volatile SelState* st = &L.s.state[sl];   // other blocks update it inside one launch: no L1
-    const uint32_t flags = st->flags;
-    const bool fell_back = !(flags & FLAG_GENERAL) && !FUSE && pass == 0 && first_pass_missed(L.s.cursor[sl], S);
-    const bool counting = (flags & FLAG_GENERAL) ? st->stage == (uint32_t)pass : fell_back;
-    const bool add_only = FUSE && S.r == S.len;      // nothing to select, but a = g + m is still due
-    if (!counting && !add_only) continue;
-    const uint32_t prefix = st->prefix;
+    if (S.r == S.len) continue;                        // nothing to select
     for (uint32_t b = tid; b < (uint32_t)kBins; b += kThreads) hist_s[b] = 0;
     __syncthreads();
     const uint32_t nchunks = slice_chunks(S);
@@ -477,76 +324,36 @@ __device__ __forceinline__ void hist_body(const Launch& L, int pass, uint32_t to
       uint32_t valid[kIter];
 #pragma unroll
       for (int it = 0; it < kIter; ++it)
-        valid[it] = load_vec<GradT, FUSE>(L.grad, L.residual, base_g, base_m, e_w + it * 128u + lane * 4u,
-                                          S.head, span, a[it]);
-      if (counting) {
+        valid[it] = load_vec<GradT, true, false>(L.grad, L.residual, base_g, base_m, e_w + it * 128u + lane * 4u,
+                                                 S.head, span, a[it]);
 #pragma unroll
-        for (int it = 0; it < kIter; ++it)
+      for (int it = 0; it < kIter; ++it)
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const uint32_t key = mag_key(a[it][j]);
-            if (((valid[it] >> j) & 1u) && (pass == 0 || (key >> (shift + bits)) == prefix))
-              atomicAdd(&hist_s[(key >> shift) & ((1u << bits) - 1u)], 1u);
-          }
-      }
+        for (int j = 0; j < 4; ++j)
+          if ((valid[it] >> j) & 1u) atomicAdd(&hist_s[mag_key(a[it][j]) >> 20], 1u);
     }
-    if (!counting) continue;
     __syncthreads();
     uint32_t* gh = L.s.hist + (size_t)sl * kBins;
-    for (uint32_t b = tid; b < (1u << bits); b += kThreads) {
+    for (uint32_t b = tid; b < (uint32_t)kBins; b += kThreads) {
       const uint32_t v = hist_s[b];
       if (v) atomicAdd(gh + b, v);
     }
     const uint32_t nblocks = (nchunks + kHistChunks - 1) / kHistChunks;
-    if (is_last_block(&L.s.done[sl], nblocks)) finish_pass(L, sl, S, pass, true, fell_back, hist_s, scratch);
-  }
-}
-
-template <typename GradT, bool FUSE>
-__global__ void __launch_bounds__(kThreads) k_hist(Launch L, int pass, uint32_t total_blocks) {
-  hist_body<GradT, FUSE>(L, pass, total_blocks);
-}
-
-// Grid-wide barrier of a cooperative launch (all blocks resident).  `target` = blocks * barriers
-// passed so far.  Bounded: on expiry the error flag is raised and false is returned to every thread
-// of the block, which then leaves the kernel; the other blocks run into the same limit.
-constexpr int kGridSpinLimit = 1 << 22;
-__device__ __forceinline__ bool grid_barrier(uint32_t* counter, uint32_t target, uint32_t* error) {
-  __shared__ uint32_t s_ok;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    __threadfence();
-    atomicAdd(counter, 1u);
-    uint32_t ok = 1;
-    int spins = 0;
-    while (*reinterpret_cast<volatile uint32_t*>(counter) < target) {
-      if (++spins > kGridSpinLimit) { ok = 0; atomicOr(error, ERR_LOOKBACK_TIMEOUT); break; }
-      __nanosleep(100);
+    if (!is_last_block(&L.s.done[sl], nblocks)) continue;
+    for (uint32_t b = tid; b < (uint32_t)kBins; b += kThreads) {
+      hist_s[b] = __ldcg(gh + b);
+      gh[b] = 0;                                         // the run kernels' histogram starts from zero
     }
-    __threadfence();
-    s_ok = ok;
+    __syncthreads();
+    uint32_t D, above;
+    const bool ok = pick_digit(hist_s, kBins, S.r, scratch, D, above);
+    if (tid == 0) {
+      L.s.done[sl] = 0;
+      SelState* st = &L.s.state[sl];
+      if (ok) { st->tau_lo = D << 20; st->tau_hi = (D << 20) | 0xFFFFFu; }
+      else atomicOr(L.s.error, ERR_SELECT_INCONSISTENT);   // fewer than r keys: cannot happen for a valid slice
+    }
   }
-  __syncthreads();
-  return s_ok != 0;
-}
-
-// The whole exact path in one cooperative launch: the remaining radix passes over the full vector
-// (each ends with the per-slice digit pick in the last block that finishes that slice), a grid
-// barrier after each, then the ordered collect.  When no slice needs the exact path -- the usual
-// case after the sampled pass -- every block returns at once, so the idle cost is one launch.
-__global__ void __launch_bounds__(kThreads) k_exact(Launch L, int first_pass, uint32_t n_hist_blocks, uint32_t n_chunks) {
-  if (!L.general_primary) {
-    bool missed = false;
-    for (uint32_t s = threadIdx.x; s < L.n_slices; s += kThreads)
-      missed |= first_pass_missed(L.s.cursor[s], L.s.slices[s]);
-    if (!__syncthreads_or(missed)) return;          // the same answer in every block
-  }
-  uint32_t passed = 0;
-  for (int pass = first_pass; pass < 3; ++pass) {
-    hist_body<float, false>(L, pass, n_hist_blocks);
-    if (!grid_barrier(&L.s.tickets[2], gridDim.x * (++passed), L.s.error)) return;
-  }
-  collect_body<float, false, true>(L, n_chunks);
 }
 
 // ----------------------------------------------------------------------------- finish

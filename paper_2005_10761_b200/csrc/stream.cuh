@@ -59,8 +59,8 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t 
   return ok != 0;
 }
 // Bounded wait for the phase with the given parity to complete.
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity) {
-  for (int i = 0; i < kWaitLimit; ++i)
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, int limit = kWaitLimit) {
+  for (int i = 0; i < limit; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }
@@ -120,10 +120,11 @@ template <> struct SmemGrad<__nv_bfloat16> {
   }
 };
 
-// HIST: the candidates are also counted into the slice's histogram over its bracket -- 2047 equal buckets
-// over [tau_lo, tau_hi] (bracket_shift) and one bucket for the keys above -- which the run kernels
-// (finish.cuh) start from; the keys above the bracket, most of the candidates, are counted per block.
-template <typename GradT, bool HIST>
+// GIVEUP is the instance the test of the give-up path runs (RTOPK_OPT_TEST_STREAM_GIVEUP): its consumers
+// treat their first wait as run out and its producer waits only briefly for them, so every block takes the
+// exit a real expiry would take -- error flag, a last bounded wait for the bulk copies still on their way
+// into the block's shared memory, return -- while all copies do arrive.
+template <typename GradT, bool GIVEUP>
 __global__ void __launch_bounds__(kStreamThreads, 3) k_stream(Launch L, uint32_t total_tiles, uint32_t uniform_chunks) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   StreamSmem<GradT>& sm = *reinterpret_cast<StreamSmem<GradT>*>(smem_raw);
@@ -146,7 +147,14 @@ __global__ void __launch_bounds__(kStreamThreads, 3) k_stream(Launch L, uint32_t
     for (uint32_t i = 0;; ++i) {
       const uint32_t stage = i % kStages, phase = (i / kStages) & 1u;
       const uint32_t next_tile = tile < total_tiles ? gridDim.x + atomicAdd(&L.s.tickets[3], 1u) : tile;
-      if (!mbar_wait(&sm.empty[stage], phase ^ 1u)) { atomicOr(L.s.error, ERR_LOOKBACK_TIMEOUT); return; }
+      if (!mbar_wait(&sm.empty[stage], phase ^ 1u, GIVEUP ? kDrainLimit : kWaitLimit)) {
+        // the consumers never freed the stage: give up, but not before the copies issued into the two stages
+        // (iterations i - 1 and i - 2) have landed in this block's shared memory
+        atomicOr(L.s.error, ERR_WAIT_TIMEOUT);
+        if (i >= 1) mbar_drain(&sm.full[(i - 1) % kStages], ((i - 1) / kStages) & 1u);
+        if (i >= 2) mbar_drain(&sm.full[(i - 2) % kStages], ((i - 2) / kStages) & 1u);
+        return;
+      }
       if (tile >= total_tiles) {
         sm.desc[stage].valid = 0;
         mbar_arrive(&sm.full[stage]);
@@ -173,12 +181,12 @@ __global__ void __launch_bounds__(kStreamThreads, 3) k_stream(Launch L, uint32_t
   const unsigned long long keep = l2_policy_evict_last();
   uint32_t cur_slice = 0xFFFFFFFFu;
   Slice S;
-  uint32_t tau = 0x80000000u, tau_hi = 0x7FFFFFFFu, hshift = 0;
+  uint32_t tau = 0x80000000u;
   for (uint32_t i = 0;; ++i) {
     const uint32_t stage = i % kStages, phase = (i / kStages) & 1u, buf = i & 1u;
-    const bool arrived = mbar_wait(&sm.full[stage], phase);
+    const bool arrived = GIVEUP ? false : mbar_wait(&sm.full[stage], phase);
     if (consumer_any(!arrived)) {                 // every consumer leaves together
-      if (tid == 0) atomicOr(L.s.error, ERR_LOOKBACK_TIMEOUT);
+      if (tid == 0) atomicOr(L.s.error, ERR_WAIT_TIMEOUT);
       // ... but not while a bulk copy into this block's shared memory may still be on its way: the copies
       // the producer has issued into both stages get one more (bounded) wait before the block ends
       mbar_drain(&sm.full[stage], phase);
@@ -191,10 +199,6 @@ __global__ void __launch_bounds__(kStreamThreads, 3) k_stream(Launch L, uint32_t
       cur_slice = d.slice;
       S = slices[cur_slice];
       tau = L.s.state[cur_slice].tau_lo;
-      if (HIST) {
-        tau_hi = max(tau, L.s.state[cur_slice].tau_hi);
-        hshift = bracket_shift(tau, tau_hi);
-      }
     }
     const uint32_t head = S.head, span = head + S.len;
     const uint32_t e_w = d.chunk * (uint32_t)kChunk + warp * (uint32_t)kWarpSpan;   // element on the slice's grid
@@ -238,31 +242,16 @@ __global__ void __launch_bounds__(kStreamThreads, 3) k_stream(Launch L, uint32_t
     uint32_t wA = 0;
 #pragma unroll
     for (int it = 0; it < kIter; ++it) wA += (totA >> (it * 8)) & 0xFFu;
-    if (HIST) {
-      // candidates above the bracket: counted here, added to their one bucket once per chunk
-      uint32_t n_hi = 0;
-      if (maskA) {
-#pragma unroll
-        for (int it = 0; it < kIter; ++it)
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            n_hi += ((maskA >> (it * 4 + j)) & 1u) && mag_key(a[it][j]) > tau_hi;
-      }
-      wA |= warp_sum(n_hi) << 16;                                  // both counts are at most 512 per warp
-    }
     if (lane == 0) sm.wA[buf][warp] = wA;
     consumer_sync();
     if (tid == 0) {
       uint32_t bA = 0;
 #pragma unroll
       for (int w = 0; w < kWarps; ++w) bA += sm.wA[buf][w];
-      const uint32_t bHi = bA >> 16;
-      bA &= 0xFFFFu;
       uint32_t start = 0;
       if (bA) {
         start = atomicAdd(&L.s.cursor[cur_slice], bA);
         atomicAdd(&L.s.group_total[S.group_begin + (d.chunk >> S.gshift)], bA);
-        if (HIST && bHi) atomicAdd(&L.s.hist[(size_t)cur_slice * kBins + (kBins - 1)], bHi);
       }
       const uint32_t tile = S.chunk_begin + d.chunk;
       L.s.chunk_start[tile] = start;
@@ -272,7 +261,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) k_stream(Launch L, uint32_t
     consumer_sync();
     if (maskA) {
       uint32_t before = sm.ex[buf];
-      for (uint32_t w = 0; w < warp; ++w) before += sm.wA[buf][w] & 0xFFFFu;
+      for (uint32_t w = 0; w < warp; ++w) before += sm.wA[buf][w];
       uint32_t* cidx = L.s.raw_idx + S.cand_off;
       float* cval = L.s.raw_val + S.cand_off;
 #pragma unroll
@@ -286,10 +275,6 @@ __global__ void __launch_bounds__(kStreamThreads, 3) k_stream(Launch L, uint32_t
             if ((bits >> j) & 1u) {
               if (pos < S.cand_cap) { st_hint(cidx + pos, e + j - head, keep); st_hint(reinterpret_cast<uint32_t*>(cval) + pos, __float_as_uint(a[it][j]), keep); }
               ++pos;
-              if (HIST) {
-                const uint32_t key = mag_key(a[it][j]);
-                if (key <= tau_hi) atomicAdd(&L.s.hist[(size_t)cur_slice * kBins + ((key - tau) >> hshift)], 1u);
-              }
             }
         }
         before += (totA >> (it * 8)) & 0xFFu;

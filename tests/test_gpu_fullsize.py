@@ -32,6 +32,14 @@ def lib():
     return pkg
 
 
+def _free_bytes() -> int:
+    """Free device memory once this process has given back what its allocator only caches."""
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    return torch.cuda.mem_get_info()[0]
+
+
 def _bits(t: torch.Tensor) -> torch.Tensor:
     return t.view(torch.int32)
 
@@ -158,7 +166,7 @@ def test_c4_per_tensor_lstm_shapes(lib):
 
 def test_c5_quarter_billion_coordinates(lib):
     cfg = wl.configs()["c5_W4_r100_k10"]
-    free, _ = torch.cuda.mem_get_info()
+    free = _free_bytes()
     if free < 24e9:
         pytest.skip("not enough free device memory on this (shared) GPU")
     _run_config(lib, cfg, 1, [2])
@@ -170,7 +178,7 @@ def test_c5_sweep_points_many_workers(lib, name, rows):
     # the remaining corners of the d = 2^28 sweep: W in {16, 32}, r / d = 0.1 %, k / r = 1 / 4.  Properties on
     # every row, the oracle on four sampled rows, the update against the oracle's aggregate of all messages.
     cfg = wl.configs()[name]
-    free, _ = torch.cuda.mem_get_info()
+    free = _free_bytes()
     need = cfg.W * cfg.ld * 4 * 2.3 + 8e9            # g, m, scratch, temporaries of the checks
     if free < need:
         pytest.skip(f"not enough free device memory on this (shared) GPU: {free / 1e9:.0f} GB of {need / 1e9:.0f} GB")
@@ -180,7 +188,7 @@ def test_c5_sweep_points_many_workers(lib, name, rows):
 def test_slice_longer_than_2_to_28_uses_wider_chunk_groups(lib):
     # above 2^28 coordinates a slice has more than 2048 x 32 chunks and k_finish takes its
     # group-walking layout path; properties only (the oracle's sort of such a row takes minutes)
-    free, _ = torch.cuda.mem_get_info()
+    free = _free_bytes()
     if free < 16e9:
         pytest.skip("not enough free device memory on this (shared) GPU")
     import dataclasses
@@ -190,7 +198,7 @@ def test_slice_longer_than_2_to_28_uses_wider_chunk_groups(lib):
 
 
 def test_c5_limits_topk_and_randomk(lib):
-    free, _ = torch.cuda.mem_get_info()
+    free = _free_bytes()
     if free < 16e9:
         pytest.skip("not enough free device memory on this (shared) GPU")
     # k = r (Definition 1): every member of the top-r set is sent -- properties on the device

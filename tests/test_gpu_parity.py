@@ -761,16 +761,18 @@ def test_fallback_is_taken_and_exact_when_the_sample_misleads(lib):
 
 
 def test_a_wait_that_gives_up_is_reported_and_leaves_the_context_usable(lib):
-    # The waits inside the kernels are bounded.  The look-back of the full-vector radix select is made to
-    # give up at once (a test-only option: no GPU fault, no hang is involved): the call returns, nothing
-    # outside the caller's buffers is written (canaries around the messages and the residual), the status
-    # poll reports the internal error, and the same context then serves a normal call correctly.
-    from paper_2005_10761_b200.binding import OPT_TEST_LOOKBACK_LIMIT
+    # The waits inside the kernels are bounded (the streaming pass's waits for its bulk copies and for free
+    # stages are the only ones).  A test-only option makes every block of that pass take the exit of a wait
+    # that ran out (no GPU fault, no hang is involved; the copies all arrive and are waited for): the call
+    # returns, nothing outside the caller's buffers is written (canaries around the messages and the
+    # residual), the status poll reports the internal error, and the same context then serves a normal
+    # call correctly.
+    from paper_2005_10761_b200.binding import OPT_TEST_STREAM_GIVEUP
     rng = np.random.default_rng(77)
-    W, d, r, k = 2, 20000, 5000, 500                 # five tiles per row; the last tile alone cannot hold r candidates
+    W, d, r, k = 2, 20000, 5000, 500                 # five chunks per row
     g = _pad(_spiky(rng, W, d))
     ld = g.shape[1]
-    ctx = _ctx(lib, d, W, r, k, path=EXACT)
+    ctx = _ctx(lib, d, W, r, k)
     tg = torch.from_numpy(g).cuda()
     pad = 4096
     res_buf = torch.full((W * ld + 2 * pad,), 123.0, dtype=torch.float32, device="cuda")
@@ -780,7 +782,7 @@ def test_a_wait_that_gives_up_is_reported_and_leaves_the_context_usable(lib):
     tm.zero_()
     idx = idx_buf[pad:pad + W * k].view(W, k)
     val = val_buf[pad:pad + W * k].view(W, k)
-    ctx.set_option(OPT_TEST_LOOKBACK_LIMIT, 0)
+    ctx.set_option(OPT_TEST_STREAM_GIVEUP, 1)
     ctx.sparsify(tg, tm, d, r, k, 5, 0, idx, val)
     torch.cuda.synchronize()
     with pytest.raises(lib.RTopKError) as e:
@@ -790,8 +792,8 @@ def test_a_wait_that_gives_up_is_reported_and_leaves_the_context_usable(lib):
         assert bool((buf[:pad] == fill).all()) and bool((buf[-pad:] == fill).all())
     assert bool((tm[:, d:] == 0).all())                              # padding columns untouched
     ctx.poll_status()                                                # the flag was cleared by the failed poll
-    # back to the normal limit: the same context gives the oracle's result
-    ctx.set_option(OPT_TEST_LOOKBACK_LIMIT, 1 << 22)
+    # back to normal: the same context gives the oracle's result
+    ctx.set_option(OPT_TEST_STREAM_GIVEUP, 0)
     tm.zero_()
     m_or = np.zeros_like(g)
     ctx.sparsify(tg, tm, d, r, k, 5, 1, idx, val)
