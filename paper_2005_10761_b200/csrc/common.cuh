@@ -14,7 +14,7 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kIter = 4;                      // 4-element vectors per thread per chunk
 constexpr int kWarpSpan = 32 * kIter * 4;     // 512 consecutive elements per warp
 constexpr int kChunk = kWarps * kWarpSpan;    // 4096 elements per block of the collect kernels
-constexpr int kHistChunks = 16;               // chunks per block of the histogram kernels
+constexpr int kHistChunks = 4;                // chunks per unit of work of the histogram pass (k_bracket)
 constexpr int kGroupsMax = 2048;              // chunk groups per slice (two per thread of k_finish)
 
 // radix digits of the 31-bit magnitude key, most significant first: 11 + 11 + 9 bits

@@ -301,7 +301,7 @@ __device__ __forceinline__ bool first_pass_missed(uint32_t n_gathered, const Sli
 // holds when very many keys share 11 leading bits, which the finishing kernels repair like any overflow.
 // grid: up to total_blocks blocks; a unit is kHistChunks chunks of one slice.
 template <typename GradT>
-__global__ void __launch_bounds__(kThreads) k_bracket(Launch L, uint32_t total_blocks) {
+__global__ void __launch_bounds__(kThreads, 8) k_bracket(Launch L, uint32_t total_blocks) {
   __shared__ uint32_t hist_s[kBins];
   __shared__ uint32_t scratch[kWarps + 2];
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
