@@ -158,7 +158,8 @@ def config_dict(cfg, args, world: int) -> dict:
             "variant": ("rtopk_step_apply (fused master update)" if args.apply else
                         f"rtopk_step_threshold (theta = {args.threshold})" if args.threshold is not None
                         else "rtopk_step"),
-            "select_path": args.select_path, "reuse_threshold": bool(args.reuse_threshold)}
+            "select_path": args.select_path, "finish_path": getattr(args, "finish_path", "auto"),
+            "reuse_threshold": bool(args.reuse_threshold)}
 
 
 # ------------------------------------------------------------------------------------ CPU oracle legs
@@ -252,6 +253,8 @@ class Round:
             self.ctx.set_option(B.OPT_REUSE_THRESHOLD, 1)
         if args.select_path == "exact":
             self.ctx.set_option(B.OPT_SELECT_PATH, 1)
+        if getattr(args, "finish_path", "auto") != "auto":
+            self.ctx.set_option(B.OPT_FINISH_PATH, {"cluster": 1, "runs": 2}[args.finish_path])
         if grads is None:
             n_batches = n_batches or resident_batches(cfg, args.steps, args.warmup)
             shard_cfg = cfg if world == 1 else dataclasses.replace(cfg, W=self.W_total)
@@ -579,6 +582,8 @@ def main():
                     help="1 (default, one GPU): also run the other configurations briefly and print them as `sweep`")
     ap.add_argument("--select-path", default="sampled", choices=["sampled", "exact"],
                     help="exact: the multi-pass radix select over the full vector (RTOPK_OPT_SELECT_PATH = 1)")
+    ap.add_argument("--finish-path", default="auto", choices=["auto", "cluster", "runs"],
+                    help="RTOPK_OPT_FINISH_PATH: which kernels turn the candidates into messages (same result)")
     ap.add_argument("--apply", action="store_true",
                     help="time rtopk_step_apply (master update fused into the aggregation; plain workloads, 1 GPU)")
     ap.add_argument("--threshold", type=float, default=None,

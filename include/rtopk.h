@@ -99,14 +99,14 @@ enum {
                                 with rtopk_set_device_step; it starts at 0).  A caller that captures one round
                                 in a CUDA graph can then replay the graph round after round and still draw a
                                 fresh subset each time.  0 = off (default): `step` is the argument */
-  RTOPK_OPT_FINISH_PATH = 5,    /* how the sampled path turns the candidates of the streaming pass into messages
-                                (the result is the same): 1 = one thread-block cluster per slice, which lays
-                                the candidate runs out in index order first; 2 = three grid-wide launches over
-                                all slices that walk the candidate list as the streaming pass left it (a
-                                histogram over the bracket, a count, the emission), with the cluster kernel
-                                behind them for what they leave (a missed bracket, heavy ties); 0 (default) =
-                                2 for calls over 2^27 coordinates or more in all (rows x slice lengths), where
-                                the clusters' serial steps no longer hide behind one another, else 1 */
+  RTOPK_OPT_FINISH_PATH = 5,    /* how the candidates of the streaming pass become messages (the result is the
+                                same): 0 (default) or 2 = three grid-wide launches over all slices that walk
+                                the candidate list as the streaming pass left it (a histogram over the
+                                bracket, a count, the emission; the k-of-r subset is drawn beside the first
+                                two), with the cluster kernel behind them for what they leave (a missed
+                                bracket, heavy ties); 1 = the cluster kernel alone: one thread-block cluster
+                                per slice, which lays the candidate runs out in index order first (the subset
+                                is then drawn beside the start of the streaming pass) */
   RTOPK_OPT_TEST_STREAM_GIVEUP = 6 /* for tests of the give-up path only: 1 = every block of the streaming pass
                                 behaves as if its first bounded wait had run out (consumers at once, the
                                 producer after a short wait for them).  The call still returns, all copies in

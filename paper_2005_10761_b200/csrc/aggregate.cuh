@@ -58,6 +58,7 @@ struct AggOut {
   float eta, mu;
   float* velocity;
   uint32_t* sent;
+  uint32_t clear;     // 1: `out` receives the average and holds anything: the block clears its tile first
   __device__ __forceinline__ void store(uint32_t idx, float ghat) const {
     if (velocity != nullptr) {
       const float v = (float)((double)mu * (double)velocity[idx] + (double)ghat);
@@ -339,8 +340,9 @@ template <typename M>
 __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const uint32_t* __restrict__ starts, uint32_t d,
                                                                   uint32_t W, uint32_t K, AggScale sc,
                                                                   float eta, float* __restrict__ out, float mu,
-                                                                  float* __restrict__ velocity, uint32_t* __restrict__ sent) {
-  const AggOut dst = {out, eta, mu, velocity, sent};
+                                                                  float* __restrict__ velocity, uint32_t* __restrict__ sent,
+                                                                  uint32_t clear) {
+  const AggOut dst = {out, eta, mu, velocity, sent, clear};
   __shared__ uint32_t s_beg[kAggMaxW], s_pre[kAggMaxW + 1], s_cnt[kAggSearchW];
   __shared__ uint32_t st_idx[kAggSparseStage];
   __shared__ float st_val[kAggSparseStage];
@@ -352,6 +354,13 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
   const uint32_t lo = blockIdx.x * (uint32_t)kAggSparseTile;
   const uint32_t span_lo = lo - lo % kTiledSpan;
   if (tid == 0) s_carry = 0;
+  if (clear) {
+    // the update is zero wherever no worker sent anything: the tile is cleared here (asynchronous stores
+    // beside the loads that follow; the barriers below order them before the block's own results)
+    const uint32_t hi = min(d, lo + (uint32_t)kAggSparseTile), full = lo + ((hi - lo) & ~3u);
+    for (uint32_t i = lo + tid * 4u; i < full; i += kAggThreads * 4u) __stcs(reinterpret_cast<float4*>(out + i), make_float4(0.f, 0.f, 0.f, 0.f));
+    for (uint32_t i = full + tid; i < hi; i += kAggThreads) out[i] = 0.f;
+  }
   __syncthreads();
   if (starts == nullptr) {
     // no table of run starts: a warp per worker finds the run of this tile in the worker's sorted

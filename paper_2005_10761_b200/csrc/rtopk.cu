@@ -39,7 +39,8 @@ struct rtopk_ctx {
   SelState* d_state = nullptr;
   char* d_zero = nullptr;        // counters, histograms, bitmaps: cleared per call
   size_t zero_bytes = 0;
-  uint32_t* d_first = nullptr;   // first-occurrence tables: set to 0xFF per call
+  uint32_t* d_first = nullptr;   // first-occurrence tables: all 0xFF before the subset kernels run
+  size_t first_clean = 0;        // leading entries that a call has left at 0xFF for the next one
   size_t first_entries = 0;
   uint32_t* d_cand_idx = nullptr;
   float* d_cand_val = nullptr;
@@ -91,6 +92,7 @@ struct rtopk_ctx {
   cudaStream_t side = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   cudaEvent_t ev_streamed = nullptr, ev_cleared = nullptr;   // the dense update is cleared beside the finishing kernels
+  cudaEvent_t ev_zeroed = nullptr;                           // the side stream has cleared the late part of the zeroed region
   int profile = 0;
   cudaEvent_t ev[RTOPK_N_PHASES + 1] = {};
   bool ev_valid[RTOPK_N_PHASES + 1] = {};
@@ -272,9 +274,14 @@ int check_common(const rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t
   return RTOPK_OK;
 }
 
+int run_sampler(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st, bool clear_first);
+
+// `late.on`: the side stream draws the k-of-r subset only once the streaming pass has ended (see
+// sparsify_impl); the stream does not wait for it here.
+struct LateSide { bool on; };
+
 template <typename GradT>
-int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st, cudaEvent_t join,
-                  float* clear_out, size_t clear_bytes) {
+int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st, cudaEvent_t join, LateSide late) {
   const uint32_t n = (uint32_t)P.slices.size();
   int rc = RTOPK_OK;
   auto stream_pass = [&]() -> int {
@@ -285,12 +292,22 @@ int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t s
     if (ctx->test_giveup) k_stream<GradT, true><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
     else k_stream<GradT, false><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
     ++ctx->launches;
-    if (clear_out) {
-      // the streaming pass saturates the memory system and the kernels after it do not: the dense
-      // update is cleared on the side stream once the pass has ended
+    if (late.on) {
+      // the streaming pass saturates the memory system and fills every SM, the kernels after it do neither:
+      // what does not depend on the data runs on the side stream once the pass has ended
       RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_streamed, st));
       RTOPK_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_streamed, 0));
-      RTOPK_CUDA(ctx, cudaMemsetAsync(clear_out, 0, clear_bytes, ctx->side));
+      {
+        RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_zeroed, 0));      // (recorded long ago: see sparsify_impl)
+        const int rs = run_sampler(ctx, P, L, ctx->side, true);
+        if (rs) return rs;
+        RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_join, ctx->side));
+        // behind the subset, off the path of the kernel that waits for it: the round counter, and the
+        // first-occurrence tables put back to 0xFF for the next call
+        if (ctx->device_step) { k_step_bump<<<1, 32, 0, ctx->side>>>(ctx->d_step); ++ctx->launches; }
+        RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_first, 0xFF, P.first_entries * sizeof(uint32_t), ctx->side));
+        ctx->first_clean = P.first_entries;
+      }
       RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_cleared, ctx->side));
     }
     mark(ctx, RTOPK_PHASE_ORDER, st);
@@ -344,10 +361,12 @@ int upload_slices(rtopk_ctx* ctx, const Plan& P, cudaStream_t st) {
   return RTOPK_OK;
 }
 
-int run_sampler(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st, bool clear_first = true) {
+int run_sampler(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st, bool clear_first) {
   if (!P.any_sampler) return RTOPK_OK;
   const uint32_t n = (uint32_t)P.slices.size();
-  if (clear_first) RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_first, 0xFF, P.first_entries * sizeof(uint32_t), st));
+  if (clear_first && P.first_entries > ctx->first_clean)
+    RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_first, 0xFF, P.first_entries * sizeof(uint32_t), st));
+  ctx->first_clean = 0;                                // used from here on
   const dim3 grid((P.k_draw_max + kDrawThreads - 1) / kDrawThreads, n);
   k_draw<<<grid, kDrawThreads, 0, st>>>(L);
   ++ctx->launches;
@@ -391,7 +410,7 @@ int bind_launch(rtopk_ctx* ctx, const Plan& P, const void* grad, float* residual
 int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
                   int64_t d, int32_t W, int32_t worker_base, int32_t S, const int64_t* seg_off,
                   const int64_t* seg_r, const int64_t* seg_k, uint64_t seed, uint32_t step, uint32_t* msg_idx,
-                  float* msg_val, cudaStream_t st, uint32_t* K_out, float* clear_out = nullptr, uint32_t msg_stride = 1) {
+                  float* msg_val, cudaStream_t st, uint32_t* K_out, uint32_t msg_stride = 1) {
   int rc = check_common(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, msg_idx, msg_val);
   if (rc) return rc;
   if (S < 1 || S > ctx->S_max || !seg_off || !seg_r || !seg_k) return RTOPK_ERR_INVALID_ARG;
@@ -430,33 +449,41 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   // selection bitmap) is first touched by the sampler and the exact path, both behind the fork.
   const bool late_on_side = ctx->select_path == 0;
   if (!late_on_side) RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero, 0, zbytes, st));
-  const bool forked = P.any_sampler || clear_out != nullptr;
+  // Calls that are finished by the run kernels need the subset only for the last of them, and those kernels
+  // leave most of every SM idle, whereas the streaming pass wants all of it from its first microsecond: there
+  // the subset is drawn beside the run kernels, not beside the start of the pass.
+  const bool from_runs = P.any_select && L.n_slices <= 65535u &&
+                         ctx->finish_path != 1;
+  const bool sampler_late = from_runs && late_on_side && P.any_sampler;
+  const bool forked = P.any_sampler && !sampler_late;
   if (forked) {
-    // work that does not depend on the data runs beside the streaming pass: the k-of-r subset and,
-    // for a step call, the clearing of the dense update
+    // work that does not depend on the data runs beside the streaming pass: the k-of-r subset
     RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_fork, st));
     RTOPK_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
     if (late_on_side) RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero + early_bytes, 0, zbytes - early_bytes, ctx->side));
-    rc = run_sampler(ctx, P, L, ctx->side);
+    rc = run_sampler(ctx, P, L, ctx->side, true);
     if (rc) return rc;
     // the subset kernels are the only readers of the round counter: it advances right behind them
     if (ctx->device_step) { k_step_bump<<<1, 32, 0, ctx->side>>>(ctx->d_step); ++ctx->launches; }
-    const bool clear_now = clear_out && !late_on_side;
-    if (clear_now) RTOPK_CUDA(ctx, cudaMemsetAsync(clear_out, 0, (size_t)d * sizeof(float), ctx->side));
     RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_join, ctx->side));
+  } else if (sampler_late) {
+    // the rest of the zeroed region (a few hundred KB) is cleared beside the start of the streaming pass, so
+    // that nothing stands between the end of the pass and the first run kernel
+    RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_fork, st));
+    RTOPK_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
+    RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero + early_bytes, 0, zbytes - early_bytes, ctx->side));
+    RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_zeroed, ctx->side));
   } else if (late_on_side) {
     RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero + early_bytes, 0, zbytes - early_bytes, st));
   }
   cudaEvent_t join = forked ? ctx->ev_join : nullptr;
-  float* clear_late = late_on_side ? clear_out : nullptr;
-  const size_t clear_bytes = (size_t)d * sizeof(float);
-  rc = grad_dtype == RTOPK_F32 ? launch_select<float>(ctx, P, L, st, join, clear_late, clear_bytes)
-                               : launch_select<__nv_bfloat16>(ctx, P, L, st, join, clear_late, clear_bytes);
+  const LateSide late = {sampler_late};
+  rc = grad_dtype == RTOPK_F32 ? launch_select<float>(ctx, P, L, st, join, late)
+                               : launch_select<__nv_bfloat16>(ctx, P, L, st, join, late);
   if (rc) return rc;
   // (launch_select has made the stream wait for the side stream behind the streaming pass)
   mark(ctx, RTOPK_PHASE_FINISH, st);
-  const bool from_runs = ctx->finish_path == 2 || (ctx->finish_path == 0 && P.n_chunks >= (1u << 15));
-  if (P.any_select && from_runs && L.n_slices <= 65535u) {
+  if (from_runs) {
     // the usual case is finished straight from the streaming pass's runs, all slices side by side; what
     // these kernels leave (a missed bracket, heavy ties) is flagged for k_finish
     // about one wave of blocks over all slices together (8 blocks of 256 threads per SM)
@@ -467,6 +494,7 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
     const uint32_t per_slice_run = std::max<uint32_t>(1u, ((uint32_t)ctx->sms * 4u + L.n_slices - 1u) / L.n_slices);
     const dim3 rgrid(std::min((P.cap_max + kRunTile - 1) / (uint32_t)kRunTile, per_slice_run), L.n_slices);
     k_run_count<<<rgrid, kRunThreads, 0, st>>>(L);
+    if (sampler_late) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0));   // the emission needs the subset
     const uint32_t per_slice_emit = std::max<uint32_t>(1u, ((uint32_t)ctx->sms * 5u + L.n_slices - 1u) / L.n_slices);
     const dim3 egrid(std::min((P.cap_max + kRunTile - 1) / (uint32_t)kRunTile, per_slice_emit), L.n_slices);
     k_run_emit<<<egrid, kRunThreads, 0, st>>>(L);
@@ -494,8 +522,8 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
     k_emit_all<<<grid, kThreads, 0, st>>>(L, P.words_all_max);
     ++ctx->launches;
   }
-  if (clear_late) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_cleared, 0));
-  if (ctx->device_step && !forked) { k_step_bump<<<1, 32, 0, st>>>(ctx->d_step); ++ctx->launches; }
+  if (sampler_late) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_cleared, 0));   // the side stream's last work
+  if (ctx->device_step && !forked && !sampler_late) { k_step_bump<<<1, 32, 0, st>>>(ctx->d_step); ++ctx->launches; }
   mark(ctx, RTOPK_PHASE_AGGREGATE, st);
   ctx->ev_valid[RTOPK_N_PHASES] = false;   // closed by the aggregate of a step call, if any
   RTOPK_CUDA(ctx, cudaGetLastError());
@@ -506,11 +534,9 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
 
 // The threshold-then-subsample encoder (proof of Theorem 1) for W rows: the streaming pass gathers
 // the coordinates above theta, then the sizes, the subset and the messages follow on the device.
-// `clear_out`: a dense update to clear beside the kernels that follow the streaming pass.
 int threshold_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
                    int64_t d, int32_t W, int32_t worker_base, float theta, int64_t k, uint64_t seed, uint32_t step,
-                   uint32_t* msg_idx, float* msg_val, uint32_t* msg_count, uint32_t* msg_ones, cudaStream_t st,
-                   float* clear_out) {
+                   uint32_t* msg_idx, float* msg_val, uint32_t* msg_count, uint32_t* msg_ones, cudaStream_t st) {
   int rc = check_common(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, msg_idx, msg_val);
   if (rc) return rc;
   if (!msg_count || !msg_ones || ((uintptr_t)msg_count & 3u) || ((uintptr_t)msg_ones & 3u)) return RTOPK_ERR_INVALID_ARG;
@@ -560,12 +586,6 @@ int threshold_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_
   else
     k_stream<__nv_bfloat16, false><<<ctx->stream_blocks[1], kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>), st>>>(L, P.n_chunks, per);
   ++ctx->launches;
-  if (clear_out) {
-    RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_streamed, st));
-    RTOPK_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_streamed, 0));
-    RTOPK_CUDA(ctx, cudaMemsetAsync(clear_out, 0, (size_t)d * sizeof(float), ctx->side));
-    RTOPK_CUDA(ctx, cudaEventRecord(ctx->ev_cleared, ctx->side));
-  }
   mark(ctx, RTOPK_PHASE_ORDER, st);
   k_thr_sizes<<<L.n_slices, kThrSizeThreads, 0, st>>>(L, (uint32_t)limit, (uint32_t)k, msg_count, msg_ones);
   ++ctx->launches;
@@ -577,7 +597,6 @@ int threshold_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_
   const dim3 egrid((P.chunks_max + kThrThreads / 32 - 1) / (kThrThreads / 32), L.n_slices);
   k_thr_emit<<<egrid, kThrThreads, 0, st>>>(L, ctx->threshold_signs ? 1u : 0u, M);
   ++ctx->launches;
-  if (clear_out) RTOPK_CUDA(ctx, cudaStreamWaitEvent(st, ctx->ev_cleared, 0));
   if (ctx->device_step) { k_step_bump<<<1, 32, 0, st>>>(ctx->d_step); ++ctx->launches; }
   mark(ctx, RTOPK_PHASE_AGGREGATE, st);
   ctx->ev_valid[RTOPK_N_PHASES] = false;
@@ -586,8 +605,7 @@ int threshold_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_
 }
 
 int aggregate_threshold_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, const uint32_t* msg_count,
-                             const uint32_t* msg_ones, int64_t d, int32_t W, int64_t k, float* out, cudaStream_t st,
-                             bool out_cleared);
+                             const uint32_t* msg_ones, int64_t d, int32_t W, int64_t k, float* out, cudaStream_t st);
 
 bool scale_mode_known(int m) {
   return m == RTOPK_SCALE_MEAN || m == RTOPK_SCALE_SUM || m == RTOPK_SCALE_UNBIASED || m == RTOPK_SCALE_COUNT;
@@ -597,14 +615,12 @@ bool aggregate_is_sparse(int64_t d, int32_t W, int64_t k) {
   return W <= kAggMaxW && (uint64_t)W * (uint64_t)k * 16ull <= (uint64_t)d;   // <= 1024 entries per tile on average
 }
 
-// `out_cleared`: the caller has already zeroed `out` in stream order (the step calls do it beside
-// the streaming pass).
 // eta < 0: `out` receives the average.  eta >= 0: `out` holds weights and receives w - eta * average
 // (only the coordinates some worker sent change, so nothing is cleared).
 // `velocity` not null: heavy-ball momentum, `out` holds the weights (eta >= 0), every coordinate changes.
 template <typename M>
 int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_t k, int scale_mode, float* out,
-                     cudaStream_t st, bool out_cleared, float eta, int64_t r, float mu = 0.0f,
+                     cudaStream_t st, float eta, int64_t r, float mu = 0.0f,
                      float* velocity = nullptr) {
   if (!ctx || !out) return RTOPK_ERR_INVALID_ARG;
   if (d < 1 || d > ctx->d_max || W < 1 || W > ctx->W_max || k < 1 || k > d) return RTOPK_ERR_INVALID_ARG;
@@ -639,13 +655,13 @@ int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_
   else if (scale_mode == RTOPK_SCALE_UNBIASED) { sc.num = (double)r; sc.den = (double)W * (double)k; }
   else if (scale_mode == RTOPK_SCALE_COUNT) sc.by_count = 1;
   if (sparse) {
-    // few coordinates are touched: clear the update, then compute only what was sent
-    if (!out_cleared && eta < 0.0f) RTOPK_CUDA(ctx, cudaMemsetAsync(out, 0, (size_t)d * sizeof(float), st));
+    // few coordinates are touched: every block clears its tile of the update and computes only what was sent
+    const uint32_t clear = (eta < 0.0f && velocity == nullptr) ? 1u : 0u;
     // momentum: the sent coordinates are updated here and marked, the others by a plain pass behind it
     if (velocity) RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_sent, 0, ((size_t)d + 31) / 32 * sizeof(uint32_t), st));
     k_aggregate_sparse<M><<<ntiles, kAggThreads, 0, st>>>(msgs, own_search ? nullptr : starts, (uint32_t)d,
                                                           (uint32_t)W, (uint32_t)k, sc, eta, out, mu, velocity,
-                                                          ctx->d_sent);
+                                                          ctx->d_sent, clear);
     ++ctx->launches;
     if (velocity) {
       const uint32_t groups = (uint32_t)((d + 3) / 4);
@@ -668,23 +684,22 @@ int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_
 }
 
 int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
-                   int scale_mode, float* out, cudaStream_t st, bool out_cleared = false, float eta = -1.0f,
+                   int scale_mode, float* out, cudaStream_t st, float eta = -1.0f,
                    int64_t r = 0, uint32_t msg_stride = 1, float mu = 0.0f, float* velocity = nullptr) {
   if (!msg_idx || !msg_val || ((uintptr_t)msg_idx & 3u) || ((uintptr_t)msg_val & 3u)) return RTOPK_ERR_INVALID_ARG;
   if (k < 1 || k > 0xFFFFFFFFll) return RTOPK_ERR_INVALID_ARG;
   const PlainMsgs msgs = {msg_idx, msg_val, (uint32_t)k, msg_stride};
-  return aggregate_launch(ctx, msgs, d, W, k, scale_mode, out, st, out_cleared, eta, r, mu, velocity);
+  return aggregate_launch(ctx, msgs, d, W, k, scale_mode, out, st, eta, r, mu, velocity);
 }
 
 int aggregate_threshold_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, const uint32_t* msg_count,
-                             const uint32_t* msg_ones, int64_t d, int32_t W, int64_t k, float* out, cudaStream_t st,
-                             bool out_cleared) {
+                             const uint32_t* msg_ones, int64_t d, int32_t W, int64_t k, float* out, cudaStream_t st) {
   if (!msg_idx || !msg_val || !msg_count || !msg_ones) return RTOPK_ERR_INVALID_ARG;
   if (((uintptr_t)msg_idx & 3u) || ((uintptr_t)msg_val & 3u) || ((uintptr_t)msg_count & 3u) || ((uintptr_t)msg_ones & 3u))
     return RTOPK_ERR_INVALID_ARG;
   if (k < 1 || k > 0xFFFFFFFFll) return RTOPK_ERR_INVALID_ARG;
   const ThresholdMsgs msgs = {msg_idx, msg_val, (uint32_t)k, msg_count, msg_ones};
-  return aggregate_launch(ctx, msgs, d, W, k, RTOPK_SCALE_MEAN, out, st, out_cleared, -1.0f, 0);
+  return aggregate_launch(ctx, msgs, d, W, k, RTOPK_SCALE_MEAN, out, st, -1.0f, 0);
 }
 
 // ceil(log2 d) index bits (at least 1) and the smallest row strides of the packed format: index
@@ -783,6 +798,7 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_streamed, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_cleared, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&ctx->ev_zeroed, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFinishSmemBytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(k_finish, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
   for (int c = 1; c <= kMaxCluster && e == cudaSuccess; ++c) {
@@ -840,6 +856,7 @@ int rtopk_destroy(rtopk_ctx* ctx) {
   if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
   if (ctx->ev_streamed) cudaEventDestroy(ctx->ev_streamed);
   if (ctx->ev_cleared) cudaEventDestroy(ctx->ev_cleared);
+  if (ctx->ev_zeroed) cudaEventDestroy(ctx->ev_zeroed);
   if (ctx->side) cudaStreamDestroy(ctx->side);
   if (ctx->copy_in) { cudaStreamSynchronize(ctx->copy_in); cudaStreamDestroy(ctx->copy_in); }
   if (ctx->copy_out) { cudaStreamSynchronize(ctx->copy_out); cudaStreamDestroy(ctx->copy_out); }
@@ -900,7 +917,7 @@ int rtopk_sparsify_pairs(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64
   const int64_t off[2] = {0, d};
   uint32_t* words = reinterpret_cast<uint32_t*>(msg_pairs);
   return sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed, step,
-                       words, reinterpret_cast<float*>(words + 1), (cudaStream_t)stream, nullptr, nullptr, 2);
+                       words, reinterpret_cast<float*>(words + 1), (cudaStream_t)stream, nullptr, 2);
 }
 
 int rtopk_aggregate_pairs(rtopk_ctx* ctx, const uint64_t* msg_pairs, int64_t d, int32_t W, int64_t k, int scale_mode,
@@ -908,12 +925,12 @@ int rtopk_aggregate_pairs(rtopk_ctx* ctx, const uint64_t* msg_pairs, int64_t d, 
   if (!msg_pairs || ((uintptr_t)msg_pairs & 7u)) return RTOPK_ERR_INVALID_ARG;
   const uint32_t* words = reinterpret_cast<const uint32_t*>(msg_pairs);
   return aggregate_impl(ctx, words, reinterpret_cast<const float*>(words + 1), d, W, k, scale_mode, out,
-                        (cudaStream_t)stream, false, -1.0f, 0, 2);
+                        (cudaStream_t)stream, -1.0f, 0, 2);
 }
 
 int rtopk_aggregate_unbiased(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W,
                              int64_t k, int64_t r, float* out, void* stream) {
-  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, RTOPK_SCALE_UNBIASED, out, (cudaStream_t)stream, false, -1.0f, r);
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, RTOPK_SCALE_UNBIASED, out, (cudaStream_t)stream, -1.0f, r);
 }
 
 int rtopk_warmup_sizes(int64_t d, int32_t n_workers, double initial_density, double final_density,
@@ -974,7 +991,7 @@ int rtopk_aggregate_packed(rtopk_ctx* ctx, const uint32_t* packed_idx, int64_t l
     return RTOPK_ERR_INVALID_ARG;
   if (scale_mode == RTOPK_SCALE_UNBIASED) return RTOPK_ERR_INVALID_ARG;   // needs r: scale the result by r / k instead
   const PackedMsgs msgs = {packed_idx, packed_val, (uint32_t)ld_words, (uint32_t)ld_halves, (uint32_t)bits};
-  return aggregate_launch(ctx, msgs, d, W, k, scale_mode, out, (cudaStream_t)stream, false, -1.0f, 0);
+  return aggregate_launch(ctx, msgs, d, W, k, scale_mode, out, (cudaStream_t)stream, -1.0f, 0);
 }
 
 int rtopk_tiled_layout(int64_t d, int64_t k, int64_t* spans, int64_t* ld_low, int64_t* ld_halves) {
@@ -1022,7 +1039,7 @@ int rtopk_aggregate_tiled(rtopk_ctx* ctx, const uint32_t* span_tab, const uint16
   if (ld_low < k || ld_halves < k || ld_low > 0xFFFFFFFFll || ld_halves > 0xFFFFFFFFll) return RTOPK_ERR_INVALID_ARG;
   if (scale_mode == RTOPK_SCALE_UNBIASED) return RTOPK_ERR_INVALID_ARG;   // needs r: scale the result by r / k instead
   const TiledMsgs msgs = {span_tab, low_idx, packed_val, (uint32_t)spans, (uint32_t)ld_low, (uint32_t)ld_halves};
-  return aggregate_launch(ctx, msgs, d, W, k, scale_mode, out, (cudaStream_t)stream, false, -1.0f, 0);
+  return aggregate_launch(ctx, msgs, d, W, k, scale_mode, out, (cudaStream_t)stream, -1.0f, 0);
 }
 
 namespace {
@@ -1036,7 +1053,7 @@ int rtopk_apply_momentum(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* m
                          int64_t k, int scale_mode, int64_t r, float eta, float mu, float* velocity, float* weights,
                          void* stream) {
   if (!momentum_args_ok(eta, mu, velocity, weights)) return RTOPK_ERR_INVALID_ARG;
-  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, false, eta, r, 1, mu,
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, eta, r, 1, mu,
                         velocity);
 }
 
@@ -1048,16 +1065,16 @@ int rtopk_step_momentum(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_
   if (!ctx || d < 1 || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
   const int64_t off[2] = {0, d};
   const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed,
-                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, nullptr);
+                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr);
   if (rc) return rc;
-  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, false, eta, r, 1, mu,
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, eta, r, 1, mu,
                         velocity);
 }
 
 int rtopk_apply_update(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W,
                        int64_t k, int scale_mode, float eta, float* weights, void* stream) {
   if (!(eta >= 0.0f) || eta > 3.0e38f) return RTOPK_ERR_INVALID_ARG;
-  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, false, eta);
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, eta);
 }
 
 int rtopk_step_apply(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
@@ -1069,9 +1086,9 @@ int rtopk_step_apply(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t l
   if (!ctx || d < 1 || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
   const int64_t off[2] = {0, d};
   const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed,
-                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, nullptr);
+                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr);
   if (rc) return rc;
-  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, false, eta, r);
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, eta, r);
 }
 
 int rtopk_step(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
@@ -1079,12 +1096,11 @@ int rtopk_step(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, f
                int scale_mode, uint32_t* msg_idx, float* msg_val, float* out, void* stream) {
   if (!out || ((uintptr_t)out & 15u) || !scale_mode_known(scale_mode)) return RTOPK_ERR_INVALID_ARG;
   if (!ctx || d < 1 || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
-  const bool sparse = W >= 1 && k >= 1 && aggregate_is_sparse(d, W, k);
   const int64_t off[2] = {0, d};
   const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed,
-                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, sparse ? out : nullptr);
+                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr);
   if (rc) return rc;
-  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, out, (cudaStream_t)stream, sparse, -1.0f, r);
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, out, (cudaStream_t)stream, -1.0f, r);
 }
 
 int rtopk_step_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,
@@ -1096,12 +1112,11 @@ int rtopk_step_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64
   if (!ctx || d < 1 || d > ctx->d_max || S < 1 || S > ctx->S_max || !seg_k) return RTOPK_ERR_INVALID_ARG;
   int64_t Ksum = 0;
   for (int s = 0; s < S; ++s) Ksum += seg_k[s] > 0 ? seg_k[s] : 0;
-  const bool sparse = W >= 1 && Ksum >= 1 && aggregate_is_sparse(d, W, Ksum);
   uint32_t K = 0;
   const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, S, seg_off, seg_r,
-                               seg_k, seed, step, msg_idx, msg_val, (cudaStream_t)stream, &K, sparse ? out : nullptr);
+                               seg_k, seed, step, msg_idx, msg_val, (cudaStream_t)stream, &K);
   if (rc) return rc;
-  return aggregate_impl(ctx, msg_idx, msg_val, d, W, K, scale_mode, out, (cudaStream_t)stream, sparse);
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, K, scale_mode, out, (cudaStream_t)stream);
 }
 
 int rtopk_sparsify_threshold(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,
@@ -1109,12 +1124,12 @@ int rtopk_sparsify_threshold(rtopk_ctx* ctx, const void* grad, int grad_dtype, i
                              uint64_t seed, uint32_t step, uint32_t* msg_idx, float* msg_val, uint32_t* msg_count,
                              uint32_t* msg_ones, void* stream) {
   return threshold_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, theta, k, seed, step, msg_idx,
-                        msg_val, msg_count, msg_ones, (cudaStream_t)stream, nullptr);
+                        msg_val, msg_count, msg_ones, (cudaStream_t)stream);
 }
 
 int rtopk_aggregate_threshold(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, const uint32_t* msg_count,
                               const uint32_t* msg_ones, int64_t d, int32_t W, int64_t k, float* out, void* stream) {
-  return aggregate_threshold_impl(ctx, msg_idx, msg_val, msg_count, msg_ones, d, W, k, out, (cudaStream_t)stream, false);
+  return aggregate_threshold_impl(ctx, msg_idx, msg_val, msg_count, msg_ones, d, W, k, out, (cudaStream_t)stream);
 }
 
 int rtopk_step_threshold(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
@@ -1123,11 +1138,10 @@ int rtopk_step_threshold(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64
                          float* out, void* stream) {
   if (!out || ((uintptr_t)out & 15u)) return RTOPK_ERR_INVALID_ARG;
   if (!ctx || d < 1 || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
-  const bool sparse = W >= 1 && k >= 1 && aggregate_is_sparse(d, W, k);
   const int rc = threshold_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, theta, k, seed, step,
-                                msg_idx, msg_val, msg_count, msg_ones, (cudaStream_t)stream, sparse ? out : nullptr);
+                                msg_idx, msg_val, msg_count, msg_ones, (cudaStream_t)stream);
   if (rc) return rc;
-  return aggregate_threshold_impl(ctx, msg_idx, msg_val, msg_count, msg_ones, d, W, k, out, (cudaStream_t)stream, sparse);
+  return aggregate_threshold_impl(ctx, msg_idx, msg_val, msg_count, msg_ones, d, W, k, out, (cudaStream_t)stream);
 }
 
 int rtopk_step_host(rtopk_ctx* ctx, const void* h_grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
@@ -1233,7 +1247,7 @@ int rtopk_sample_positions(rtopk_ctx* ctx, int64_t r, int64_t k, uint64_t seed, 
   int rc = upload_slices(ctx, P, st);
   if (rc) return rc;
   RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero, 0, zbytes, st));
-  rc = run_sampler(ctx, P, L, st);
+  rc = run_sampler(ctx, P, L, st, true);
   if (rc) return rc;
   const uint32_t nwords = (uint32_t)((r + 31) / 32);
   k_positions<<<(nwords + kThreads - 1) / kThreads, kThreads, 0, st>>>(L, pos);
