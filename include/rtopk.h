@@ -118,7 +118,8 @@ enum {
 /* Phases of one call, in stream order.  STREAM is the single pass over the full vectors that
  * performs a = g + m, writes it back and gathers the coordinates above the threshold. */
 enum {
-  RTOPK_PHASE_SUBSET = 0,    /* scratch clearing; the k-of-r subset itself runs beside the stream pass */
+  RTOPK_PHASE_SUBSET = 0,    /* scratch clearing; the k-of-r subset itself runs on a stream of the context, beside
+                                the kernels that follow the stream pass */
   RTOPK_PHASE_THRESHOLD = 1, /* first bracket of the r-th largest magnitude (sample, history or histogram pass) */
   RTOPK_PHASE_STREAM = 2,    /* the one kernel over W x d elements: add, write-back, candidate gathering */
   RTOPK_PHASE_ORDER = 3,     /* candidate runs laid out in index order; count check */

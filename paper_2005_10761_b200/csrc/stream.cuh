@@ -8,8 +8,9 @@
 // flag the keys >= the sampled threshold, and append them -- in index order inside the chunk
 // (packed prefix sums) -- to a run of the slice's raw candidate buffer reserved with one atomicAdd
 // per chunk.  The run's start and length go into a per-chunk table and its length is also added to
-// the total of its chunk group; k_finish then lays the runs out in chunk order, which makes the
-// final list independent of the order in which chunks happened to reserve their runs.  No block
+// the total of its chunk group; the finishing kernels number the members of the top-r set by chunk and
+// by place inside the run (finish.cuh) or lay the runs out in chunk order first (k_finish), so the
+// result does not depend on the order in which chunks happened to reserve their runs.  No block
 // ever waits on another block.
 //
 // The only waits are on the block's own mbarriers; they are bounded, and on expiry the error flag
