@@ -341,7 +341,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
                                                                   uint32_t W, uint32_t K, AggScale sc,
                                                                   float eta, float* __restrict__ out, float mu,
                                                                   float* __restrict__ velocity, uint32_t* __restrict__ sent,
-                                                                  uint32_t clear) {
+                                                                  uint32_t clear, const uint32_t* __restrict__ run_cnt) {
   const AggOut dst = {out, eta, mu, velocity, sent, clear};
   __shared__ uint32_t s_beg[kAggMaxW], s_pre[kAggMaxW + 1], s_cnt[kAggSearchW];
   __shared__ uint32_t st_idx[kAggSparseStage];
@@ -351,6 +351,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t ntiles = gridDim.x;
   static_assert(kTiledSpan % kAggSparseTile == 0, "a tile lies inside one span");
+  static_assert(kRunTableTile == (uint32_t)kAggSparseTile, "the sparsifier's run table is kept per tile of this kernel");
   const uint32_t lo = blockIdx.x * (uint32_t)kAggSparseTile;
   const uint32_t span_lo = lo - lo % kTiledSpan;
   if (tid == 0) s_carry = 0;
@@ -378,7 +379,14 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     const uint32_t w = w0 + tid;
     uint32_t cnt = 0;
     if (w < W) {
-      if (starts != nullptr) {
+      if (run_cnt != nullptr) {
+        // the run table the sparsifier kept while it wrote the messages: `starts` holds the complement of the
+        // run's first place (0 where the tile got nothing), run_cnt its length
+        const size_t at = (size_t)w * ntiles + blockIdx.x;
+        const uint32_t b = min(K, ~__ldg(starts + at));
+        s_beg[w] = b;
+        cnt = min(K - b, __ldg(run_cnt + at));
+      } else if (starts != nullptr) {
         const uint32_t* st = starts + (size_t)w * (ntiles + 1) + blockIdx.x;
         const uint32_t b = min(K, __ldg(st)), e = min(K, __ldg(st + 1));
         s_beg[w] = b;

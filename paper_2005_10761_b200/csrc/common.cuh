@@ -114,6 +114,8 @@ struct Scratch {
   TauHistory* history;    // [slices] threshold history across calls
   Fin* fin;               // [slices] state of the run kernels
   uint32_t* list;         // [slices][2 * kListMax]: keys, then indices, of the candidates inside the bucket
+  uint32_t* tile_inv;     // run table of the messages (Launch::tile_inv / tile_cnt), in the zeroed region
+  uint32_t* tile_cnt;
 };
 
 struct Launch {
@@ -129,7 +131,24 @@ struct Launch {
   uint32_t step;
   const uint32_t* step_ptr;   // not null: the round number is read from this device word instead of `step`
   uint32_t reuse;             // 1: brackets may be predicted from the slices' threshold history
+  // Run table of the messages, for the aggregation that follows in a step call (null otherwise): per local
+  // worker row and tile of kRunTableTile coordinates, the first place in the row of a message of that tile,
+  // kept as the maximum of its complement so that the table starts from zero, and how many there are.
+  uint32_t* tile_inv;
+  uint32_t* tile_cnt;
+  uint32_t tiles_per_row;
+  uint32_t K_row;             // messages per worker row
 };
+constexpr uint32_t kRunTableTile = 16384;
+
+// Called by whoever writes message `slot` of slice S for coordinate `index` (counted in the whole vector).
+__device__ __forceinline__ void note_message(const Launch& L, const Slice& S, uint32_t slot, uint32_t index) {
+  if (L.tile_inv == nullptr) return;
+  const uint32_t place = S.msg_off - S.row * L.K_row + slot;
+  const size_t at = (size_t)S.row * L.tiles_per_row + index / kRunTableTile;
+  atomicMax(L.tile_inv + at, ~place);
+  atomicAdd(L.tile_cnt + at, 1u);
+}
 
 // ----------------------------------------------------------------------------- small helpers
 __device__ __forceinline__ uint32_t lane_id() { return threadIdx.x & 31; }

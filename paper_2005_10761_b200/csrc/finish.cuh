@@ -489,6 +489,7 @@ __global__ void __launch_bounds__(kRunThreads, 5) k_run_emit(Launch L) {
         L.msg_idx[(size_t)(S.msg_off + slot) * L.msg_stride] = S.idx_base + idx;
         L.msg_val[(size_t)(S.msg_off + slot) * L.msg_stride] = q_val[warp][q];
         L.residual[S.m_off + idx] = 0.0f;
+        note_message(L, S, slot, S.idx_base + idx);
       }
     }
     __syncwarp();

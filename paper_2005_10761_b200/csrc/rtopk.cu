@@ -41,6 +41,8 @@ struct rtopk_ctx {
   size_t zero_bytes = 0;
   uint32_t* d_first = nullptr;   // first-occurrence tables: all 0xFF before the subset kernels run
   size_t first_clean = 0;        // leading entries that a call has left at 0xFF for the next one
+  const uint32_t* run_inv = nullptr;   // run table of the messages of the last sparsify call that kept one
+  const uint32_t* run_cnt = nullptr;
   size_t first_entries = 0;
   uint32_t* d_cand_idx = nullptr;
   float* d_cand_val = nullptr;
@@ -151,6 +153,8 @@ struct Plan {
   std::vector<Slice> slices;
   uint32_t n_chunks = 0, n_hist_blocks = 0, n_groups = 0;
   size_t cand_entries = 0, draw_entries = 0, first_entries = 0, sel_words = 0;
+  size_t table_words = 0;             // rows x tiles of the messages' run table
+  uint32_t tiles_per_row = 0;
   uint32_t k_draw_max = 0, words_all_max = 0, cap_max = 0, chunks_max = 0, sel_words_max = 0;
   bool any_select = false, any_sampler = false, any_all = false;
   bool uniform = false;               // every slice has the same number of chunks (plain calls)
@@ -173,6 +177,8 @@ int make_plan(const rtopk_ctx* ctx, int64_t ld_g, int64_t ld_m, int64_t d, int32
   if ((int64_t)K > ctx->k_max || (int64_t)R > ctx->r_max) return RTOPK_ERR_INVALID_ARG;
   if (K * (uint64_t)W >= (1ull << 32)) return RTOPK_ERR_INVALID_ARG;
   P.K_row = (uint32_t)K;
+  P.tiles_per_row = (uint32_t)((d + kRunTableTile - 1) / kRunTableTile);
+  P.table_words = (size_t)W * P.tiles_per_row;
   P.uniform = (S == 1);
   P.slices.resize((size_t)W * (size_t)S);
   uint64_t chunks = 0, hblocks = 0, groups = 0, cand = 0, draws = 0, first = 0, selw = 0;
@@ -249,14 +255,17 @@ size_t carve_zero(const rtopk_ctx* ctx, const Plan& P, Scratch& s, size_t* early
   if (early_bytes) *early_bytes = at;
   s.hist = (uint32_t*)take(P.slices.size() * kBins * sizeof(uint32_t));
   s.sel = (uint32_t*)take(P.sel_words * sizeof(uint32_t));
+  s.tile_inv = (uint32_t*)take(P.table_words * sizeof(uint32_t));
+  s.tile_cnt = (uint32_t*)take(P.table_words * sizeof(uint32_t));
   return at;
 }
 
-size_t zero_region_bytes(size_t slices, size_t chunks, size_t groups, size_t sel_words) {
+size_t zero_region_bytes(size_t slices, size_t chunks, size_t groups, size_t sel_words, size_t table_words) {
   size_t at = 0;
   auto take = [&](size_t bytes) { at = align_up(at + bytes, 256); };
   take(16); take(slices * 4); take(slices * 4); take(groups * 4);
-  take(slices * kBins * 4); take(sel_words * 4);
+  take(slices * kBins * 4); take(sel_words * 4); take(table_words * 4); take(table_words * 4);
+  (void)chunks;
   return at;
 }
 
@@ -399,6 +408,8 @@ int bind_launch(rtopk_ctx* ctx, const Plan& P, const void* grad, float* residual
   L.s.fin = ctx->d_fin; L.s.list = ctx->d_list;
   L.grad = grad; L.residual = residual; L.msg_idx = msg_idx; L.msg_val = msg_val;
   L.msg_stride = 1;
+  L.tile_inv = nullptr; L.tile_cnt = nullptr;            // set by the step calls (sparsify_impl)
+  L.tiles_per_row = P.tiles_per_row; L.K_row = P.K_row;
   L.n_slices = (uint32_t)P.slices.size();
   L.worker_base = (uint32_t)worker_base;
   L.seed_lo = (uint32_t)seed; L.seed_hi = (uint32_t)(seed >> 32);
@@ -410,7 +421,8 @@ int bind_launch(rtopk_ctx* ctx, const Plan& P, const void* grad, float* residual
 int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
                   int64_t d, int32_t W, int32_t worker_base, int32_t S, const int64_t* seg_off,
                   const int64_t* seg_r, const int64_t* seg_k, uint64_t seed, uint32_t step, uint32_t* msg_idx,
-                  float* msg_val, cudaStream_t st, uint32_t* K_out, uint32_t msg_stride = 1) {
+                  float* msg_val, cudaStream_t st, uint32_t* K_out, uint32_t msg_stride = 1,
+                  bool keep_run_table = false) {
   int rc = check_common(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, msg_idx, msg_val);
   if (rc) return rc;
   if (S < 1 || S > ctx->S_max || !seg_off || !seg_r || !seg_k) return RTOPK_ERR_INVALID_ARG;
@@ -428,6 +440,12 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   if (rc) return rc;
 
   L.msg_stride = msg_stride;
+  ctx->run_inv = nullptr; ctx->run_cnt = nullptr;
+  if (keep_run_table) {
+    // the aggregation of a step call finds every worker's entries of an output tile without searching
+    L.tile_inv = L.s.tile_inv; L.tile_cnt = L.s.tile_cnt;
+    ctx->run_inv = L.s.tile_inv; ctx->run_cnt = L.s.tile_cnt;
+  }
   rc = upload_slices(ctx, P, st);
   if (rc) return rc;
   ctx->last_n_slices = L.n_slices;
@@ -621,7 +639,7 @@ bool aggregate_is_sparse(int64_t d, int32_t W, int64_t k) {
 template <typename M>
 int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_t k, int scale_mode, float* out,
                      cudaStream_t st, float eta, int64_t r, float mu = 0.0f,
-                     float* velocity = nullptr) {
+                     float* velocity = nullptr, const uint32_t* run_inv = nullptr, const uint32_t* run_cnt = nullptr) {
   if (!ctx || !out) return RTOPK_ERR_INVALID_ARG;
   if (d < 1 || d > ctx->d_max || W < 1 || W > ctx->W_max || k < 1 || k > d) return RTOPK_ERR_INVALID_ARG;
   if (!scale_mode_known(scale_mode)) return RTOPK_ERR_INVALID_ARG;
@@ -639,6 +657,8 @@ int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_
   if constexpr (std::is_same<M, TiledMsgs>::value) {
     if (sparse) { starts = msgs.tab; have_starts = true; }
   }
+  if (!sparse) run_cnt = nullptr;
+  if (run_cnt) { starts = run_inv; have_starts = true; }     // kept by the sparsifier while it wrote the messages
   if (!have_starts && (size_t)W * (ntiles + 1) > ctx->agg_start_entries) return RTOPK_ERR_INVALID_ARG;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return RTOPK_ERR_CUDA;
@@ -661,7 +681,7 @@ int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_
     if (velocity) RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_sent, 0, ((size_t)d + 31) / 32 * sizeof(uint32_t), st));
     k_aggregate_sparse<M><<<ntiles, kAggThreads, 0, st>>>(msgs, own_search ? nullptr : starts, (uint32_t)d,
                                                           (uint32_t)W, (uint32_t)k, sc, eta, out, mu, velocity,
-                                                          ctx->d_sent, clear);
+                                                          ctx->d_sent, clear, run_cnt);
     ++ctx->launches;
     if (velocity) {
       const uint32_t groups = (uint32_t)((d + 3) / 4);
@@ -685,11 +705,15 @@ int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_
 
 int aggregate_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W, int64_t k,
                    int scale_mode, float* out, cudaStream_t st, float eta = -1.0f,
-                   int64_t r = 0, uint32_t msg_stride = 1, float mu = 0.0f, float* velocity = nullptr) {
+                   int64_t r = 0, uint32_t msg_stride = 1, float mu = 0.0f, float* velocity = nullptr,
+                   bool from_step = false) {
   if (!msg_idx || !msg_val || ((uintptr_t)msg_idx & 3u) || ((uintptr_t)msg_val & 3u)) return RTOPK_ERR_INVALID_ARG;
   if (k < 1 || k > 0xFFFFFFFFll) return RTOPK_ERR_INVALID_ARG;
   const PlainMsgs msgs = {msg_idx, msg_val, (uint32_t)k, msg_stride};
-  return aggregate_launch(ctx, msgs, d, W, k, scale_mode, out, st, eta, r, mu, velocity);
+  // `from_step`: the messages are the ones the context's last sparsify call wrote, with their run table
+  const bool tab = from_step && ctx && ctx->run_cnt != nullptr;
+  return aggregate_launch(ctx, msgs, d, W, k, scale_mode, out, st, eta, r, mu, velocity, tab ? ctx->run_inv : nullptr,
+                          tab ? ctx->run_cnt : nullptr);
 }
 
 int aggregate_threshold_impl(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, const uint32_t* msg_count,
@@ -762,7 +786,7 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   ctx->cand_entries = W * cand_row;
   ctx->first_entries = W * (std::min<size_t>((size_t)r_max, 16 * (size_t)k_max) + 128 * S);
   ctx->sel_words = W * ((size_t)r_max / 32 + S + 1);
-  ctx->zero_bytes = zero_region_bytes(slices, chunks, groups, ctx->sel_words);
+  ctx->zero_bytes = zero_region_bytes(slices, chunks, groups, ctx->sel_words, W * (((size_t)d_max + kRunTableTile - 1) / kRunTableTile));
   ctx->agg_start_entries = W * ((size_t)(d_max + kAggTile - 1) / kAggTile + 2);
   if (ctx->cand_entries >= (1ull << 32) || ctx->first_entries >= (1ull << 32)) { delete ctx; return RTOPK_ERR_INVALID_ARG; }
   cudaError_t e = cudaSuccess;
@@ -1065,10 +1089,10 @@ int rtopk_step_momentum(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_
   if (!ctx || d < 1 || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
   const int64_t off[2] = {0, d};
   const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed,
-                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr);
+                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, 1, true);
   if (rc) return rc;
   return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, eta, r, 1, mu,
-                        velocity);
+                        velocity, true);
 }
 
 int rtopk_apply_update(rtopk_ctx* ctx, const uint32_t* msg_idx, const float* msg_val, int64_t d, int32_t W,
@@ -1086,9 +1110,10 @@ int rtopk_step_apply(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t l
   if (!ctx || d < 1 || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
   const int64_t off[2] = {0, d};
   const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed,
-                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr);
+                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, 1, true);
   if (rc) return rc;
-  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, eta, r);
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, eta, r, 1, 0.0f,
+                        nullptr, true);
 }
 
 int rtopk_step(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual, int64_t ld_m,
@@ -1098,9 +1123,10 @@ int rtopk_step(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, f
   if (!ctx || d < 1 || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
   const int64_t off[2] = {0, d};
   const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed,
-                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr);
+                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, 1, true);
   if (rc) return rc;
-  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, out, (cudaStream_t)stream, -1.0f, r);
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, out, (cudaStream_t)stream, -1.0f, r, 1, 0.0f,
+                        nullptr, true);
 }
 
 int rtopk_step_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,
@@ -1114,9 +1140,10 @@ int rtopk_step_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64
   for (int s = 0; s < S; ++s) Ksum += seg_k[s] > 0 ? seg_k[s] : 0;
   uint32_t K = 0;
   const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, S, seg_off, seg_r,
-                               seg_k, seed, step, msg_idx, msg_val, (cudaStream_t)stream, &K);
+                               seg_k, seed, step, msg_idx, msg_val, (cudaStream_t)stream, &K, 1, true);
   if (rc) return rc;
-  return aggregate_impl(ctx, msg_idx, msg_val, d, W, K, scale_mode, out, (cudaStream_t)stream);
+  return aggregate_impl(ctx, msg_idx, msg_val, d, W, K, scale_mode, out, (cudaStream_t)stream, -1.0f, 0, 1, 0.0f,
+                        nullptr, true);
 }
 
 int rtopk_sparsify_threshold(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, float* residual,

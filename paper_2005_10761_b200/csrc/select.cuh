@@ -1003,6 +1003,7 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
               L.msg_idx[(size_t)(S.msg_off + slot) * L.msg_stride] = S.idx_base + idx;
               L.msg_val[(size_t)(S.msg_off + slot) * L.msg_stride] = v[j];
               L.residual[S.m_off + idx] = 0.0f;
+              note_message(L, S, slot, S.idx_base + idx);
             }
           }
           ++o;
@@ -1038,6 +1039,7 @@ __global__ void __launch_bounds__(kThreads) k_emit_all(Launch L, uint32_t words_
       L.msg_idx[(size_t)(S.msg_off + pre) * L.msg_stride] = S.idx_base + p;
       L.msg_val[(size_t)(S.msg_off + pre) * L.msg_stride] = L.residual[S.m_off + p];
       L.residual[S.m_off + p] = 0.0f;
+      note_message(L, S, pre, S.idx_base + p);
     }
     ++pre;
   }
