@@ -62,6 +62,16 @@ def run_gpu(lib, g, m0, d, r, k, seed, step, worker_base=0, path=AUTO, ctx=None,
     ctx.sparsify(tg, tm, d, r, k, seed, step, idx, val, worker_base=worker_base)
     ctx.poll_status()
     stats = [ctx.stats(w) for w in range(W)]
+    # the same round as one fused call (its aggregation works from the run table the sparsifier keeps): the
+    # messages must come out the same, and the update is returned for the comparison with the oracle's average
+    tm2 = torch.from_numpy(m0.copy()).cuda()
+    idx2, val2 = torch.full_like(idx, -1), torch.full_like(val, float("nan"))
+    out = torch.full((g.shape[1],), float("nan"), dtype=torch.float32, device="cuda")
+    ctx.step(tg, tm2, d, r, k, seed, step, idx2, val2, out, worker_base=worker_base)
+    ctx.poll_status()
+    assert torch.equal(idx2, idx) and torch.equal(val2.view(torch.int32), val.view(torch.int32))
+    assert torch.equal(tm2.view(torch.int32), tm.view(torch.int32))
+    run_gpu.last_update = out.cpu().numpy()[:d]
     if own:
         ctx.close()
     return idx.cpu().numpy().view(np.uint32), val.cpu().numpy(), tm.cpu().numpy(), stats
@@ -85,6 +95,10 @@ def check_against_oracle(lib, g, m0, d, r, k, seed=1, step=0, worker_base=0, pat
             f"residual differs: worker {w}, at {np.flatnonzero(_bits(g_m[w, :d]) != _bits(m_or[w, :d]))[:5]}")
         # padding columns are neither read nor written
         assert np.array_equal(_bits(g_m[w, d:]), _bits(m0[w, d:]))
+    _, want = oracle.aggregate(o_idx, o_val, d)
+    got = run_gpu.last_update
+    both_nan = np.isnan(got) & np.isnan(want)          # (IEEE 754 leaves the payload of a NaN sum open)
+    assert np.array_equal(_bits(got)[~both_nan], _bits(want)[~both_nan]), "update of the fused call differs"
     return stats
 
 
