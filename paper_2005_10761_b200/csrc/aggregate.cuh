@@ -451,7 +451,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
       const uint32_t idx = st_idx[q], local = idx - lo;
       if (local >= (uint32_t)kAggSparseTile || idx >= d) continue;   // malformed row: ignore
       if (!((s_shared[local >> 5] >> (local & 31u)) & 1u)) {
-        const double v = msgs.term(st_w[q], st_val[q]);
+        const double v = 0.0 + msgs.term(st_w[q], st_val[q]);          // (the sum starts from +0: a lone -0 gives +0)
         dst.store(idx, (float)agg_scaled(v, 1u, sc));
       }
     }

@@ -554,6 +554,26 @@ def test_momentum_update_against_oracle(lib):
     ctx.close()
 
 
+def test_aggregate_of_signed_zeros_and_cancelling_values(lib):
+    # The sum of a coordinate starts from +0 (as the oracle's accumulator does): a lone -0 gives +0, values that
+    # cancel give +0, and both hold for coordinates with one sender and with several.
+    d, W, k = 70_000, 3, 4
+    idx = np.array([[5, 100, 20_000, 60_000], [5, 101, 20_000, 60_001], [6, 102, 20_000, 60_002]], dtype=np.uint32)
+    val = np.array([[-0.0, -0.0, 1.5, -0.0], [-0.0, 2.0, -1.5, 0.0], [-0.0, -2.0, -0.0, -3.0]], dtype=np.float32)
+    ctx = _ctx(lib, d, W, k, k)
+    out = torch.full((wl.round_up(d, 4),), float("nan"), dtype=torch.float32, device="cuda")
+    t_idx, t_val = torch.from_numpy(idx.view(np.int32)).cuda(), torch.from_numpy(val).cuda()
+    for mode, omode in ((lib.SCALE_MEAN, oracle.SCALE_MEAN), (lib.SCALE_SUM, oracle.SCALE_SUM),
+                        (lib.SCALE_COUNT, oracle.SCALE_COUNT)):
+        ctx.aggregate(t_idx, t_val, d, out, scale_mode=mode)
+        _, want = oracle.aggregate(idx, val, d, omode)
+        assert np.array_equal(_bits(out.cpu().numpy()[:d]), _bits(want)), mode
+    w = torch.zeros_like(out)
+    ctx.apply_update(t_idx, t_val, d, 0.5, w)
+    assert np.array_equal(_bits(w.cpu().numpy()[:d]), _bits(oracle.apply_update(idx, val, d, 0.5, np.zeros(d, dtype=np.float32))))
+    ctx.close()
+
+
 def test_threshold_reuse_changes_nothing_but_the_path(lib):
     """RTOPK_OPT_REUSE_THRESHOLD: consecutive rounds predict the first threshold from the last exact
     ones.  Messages, residual and update stay bit-equal to the oracle; the brackets are predicted
