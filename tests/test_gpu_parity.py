@@ -230,6 +230,39 @@ def test_segmented_per_tensor_selection(lib):
         ctx.close()
 
 
+@pytest.mark.parametrize("case", range(16))
+def test_random_segmented_steps(lib, case):
+    # Seeded random tensor layouts (1 to 8 tensors of 1 to 60,000 coordinates, unaligned cuts), per-tensor r and
+    # k, every finishing path: messages, residual and the update of the fused call against the oracle.
+    rng = np.random.default_rng(50000 + case)
+    S, W = int(rng.integers(1, 9)), int(rng.integers(1, 5))
+    sizes = [int(rng.choice([rng.integers(1, 40), rng.integers(40, 9000), rng.integers(9000, 60000)])) for _ in range(S)]
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    d = int(off[-1])
+    seg_r = [int(rng.integers(1, n + 1)) if rng.random() < 0.3 else max(1, n // int(rng.choice([3, 20, 100]))) for n in sizes]
+    seg_k = [int(rng.integers(1, r + 1)) if rng.random() < 0.4 else max(1, r // int(rng.choice([2, 4, 10]))) for r in seg_r]
+    K = sum(seg_k)
+    g = _pad(_spiky(rng, W, d, p=float(rng.choice([0.0, 0.02, 0.2]))))
+    m0 = _pad(_spiky(rng, W, d) * 0.5)
+    if rng.random() < 0.3:                             # many equal magnitudes, signed zeros
+        g = (np.round(g * 5) / 5).astype(np.float32)
+    m_or = m0.copy()
+    seed, step, wb = int(rng.integers(0, 2**40)), int(rng.integers(0, 99)), int(rng.integers(0, 9))
+    o_idx, o_val = oracle.sparsify_segmented(g, m_or, d, off, seg_r, seg_k, seed=seed, step=step, worker_base=wb)
+    ctx = _ctx(lib, d, W, sum(seg_r), K, S=S, path=int(rng.choice([AUTO, EXACT, RUNS])))
+    tg, tm = torch.from_numpy(g).cuda(), torch.from_numpy(m0.copy()).cuda()
+    idx = torch.zeros((W, K), dtype=torch.int32, device="cuda")
+    val = torch.zeros((W, K), dtype=torch.float32, device="cuda")
+    out = torch.full((wl.round_up(d, 4),), float("nan"), dtype=torch.float32, device="cuda")
+    ctx.step_segmented(tg, tm, d, off, seg_r, seg_k, seed, step, idx, val, out, worker_base=wb)
+    ctx.poll_status()
+    assert np.array_equal(idx.cpu().numpy().view(np.uint32), o_idx)
+    assert np.array_equal(_bits(val.cpu().numpy()), _bits(o_val))
+    assert np.array_equal(_bits(tm.cpu().numpy()[:, :d]), _bits(m_or[:, :d]))
+    assert np.array_equal(_bits(out.cpu().numpy()[:d]), _bits(oracle.aggregate(o_idx, o_val, d)[1]))
+    ctx.close()
+
+
 @pytest.mark.parametrize("W,d,k", [(1, 1000, 10), (4, 4096, 400), (5, 100001, 2000), (16, 300000, 3000),
                                    (32, 50000, 50000 // 3), (300, 20000, 50)])
 def test_aggregate_against_oracle(lib, W, d, k):
