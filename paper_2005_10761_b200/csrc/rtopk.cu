@@ -635,6 +635,13 @@ bool aggregate_is_sparse(int64_t d, int32_t W, int64_t k) {
 
 // eta < 0: `out` receives the average.  eta >= 0: `out` holds weights and receives w - eta * average
 // (only the coordinates some worker sent change, so nothing is cleared).
+// Whether a step call keeps the run table of its messages: the table costs two reductions per message and
+// saves the aggregation one search per worker and output tile, so it pays while a tile holds few messages of
+// a worker (at most 64), and it is only read by the sparse kernel.
+bool run_table_pays(int64_t d, int32_t W, int64_t k) {
+  return W >= 1 && k >= 1 && aggregate_is_sparse(d, W, k) && (uint64_t)k * 256ull <= (uint64_t)d;
+}
+
 // `velocity` not null: heavy-ball momentum, `out` holds the weights (eta >= 0), every coordinate changes.
 template <typename M>
 int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_t k, int scale_mode, float* out,
@@ -1089,7 +1096,8 @@ int rtopk_step_momentum(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_
   if (!ctx || d < 1 || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
   const int64_t off[2] = {0, d};
   const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed,
-                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, 1, true);
+                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, 1,
+                               run_table_pays(d, W, k));
   if (rc) return rc;
   return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, eta, r, 1, mu,
                         velocity, true);
@@ -1110,7 +1118,8 @@ int rtopk_step_apply(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t l
   if (!ctx || d < 1 || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
   const int64_t off[2] = {0, d};
   const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed,
-                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, 1, true);
+                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, 1,
+                               run_table_pays(d, W, k));
   if (rc) return rc;
   return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, weights, (cudaStream_t)stream, eta, r, 1, 0.0f,
                         nullptr, true);
@@ -1123,7 +1132,8 @@ int rtopk_step(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g, f
   if (!ctx || d < 1 || d > ctx->d_max) return RTOPK_ERR_INVALID_ARG;
   const int64_t off[2] = {0, d};
   const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, 1, off, &r, &k, seed,
-                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, 1, true);
+                               step, msg_idx, msg_val, (cudaStream_t)stream, nullptr, 1,
+                               run_table_pays(d, W, k));
   if (rc) return rc;
   return aggregate_impl(ctx, msg_idx, msg_val, d, W, k, scale_mode, out, (cudaStream_t)stream, -1.0f, r, 1, 0.0f,
                         nullptr, true);
@@ -1140,7 +1150,8 @@ int rtopk_step_segmented(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64
   for (int s = 0; s < S; ++s) Ksum += seg_k[s] > 0 ? seg_k[s] : 0;
   uint32_t K = 0;
   const int rc = sparsify_impl(ctx, grad, grad_dtype, ld_g, residual, ld_m, d, W, worker_base, S, seg_off, seg_r,
-                               seg_k, seed, step, msg_idx, msg_val, (cudaStream_t)stream, &K, 1, true);
+                               seg_k, seed, step, msg_idx, msg_val, (cudaStream_t)stream, &K, 1,
+                               run_table_pays(d, W, Ksum));
   if (rc) return rc;
   return aggregate_impl(ctx, msg_idx, msg_val, d, W, K, scale_mode, out, (cudaStream_t)stream, -1.0f, 0, 1, 0.0f,
                         nullptr, true);
