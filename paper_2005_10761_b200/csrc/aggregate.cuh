@@ -336,7 +336,9 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(M msgs, const uint32_
 // A block stages the entries of its tile (all workers' runs, in worker order); the entry of the
 // lowest worker that holds a coordinate owns it and sums that coordinate over the workers in
 // ascending order (binary search in each staged run): the same fixed-order sum as k_aggregate.
-template <typename M>
+// TILE: output coordinates per block: kAggSparseTile for sparse messages, kAggTile where a tile of that size
+// would hold more entries than the stage (the bitmaps and slot tables are laid out for the larger one).
+template <typename M, int TILE>
 __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const uint32_t* __restrict__ starts, uint32_t d,
                                                                   uint32_t W, uint32_t K, AggScale sc,
                                                                   float eta, float* __restrict__ out, float mu,
@@ -351,14 +353,16 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t ntiles = gridDim.x;
   static_assert(kTiledSpan % kAggSparseTile == 0, "a tile lies inside one span");
-  static_assert(kRunTableTile == (uint32_t)kAggSparseTile, "the sparsifier's run table is kept per tile of this kernel");
-  const uint32_t lo = blockIdx.x * (uint32_t)kAggSparseTile;
+  static_assert(kRunTableTile == (uint32_t)kAggSparseTile, "the sparsifier's run table is kept per tile of the larger size");
+  static_assert(TILE == kAggSparseTile || TILE == kAggTile, "two tile sizes");
+  constexpr uint32_t kTile = (uint32_t)TILE;
+  const uint32_t lo = blockIdx.x * kTile;
   const uint32_t span_lo = lo - lo % kTiledSpan;
   if (tid == 0) s_carry = 0;
   if (clear) {
     // the update is zero wherever no worker sent anything: the tile is cleared here (asynchronous stores
     // beside the loads that follow; the barriers below order them before the block's own results)
-    const uint32_t hi = min(d, lo + (uint32_t)kAggSparseTile), full = lo + ((hi - lo) & ~3u);
+    const uint32_t hi = min(d, lo + kTile), full = lo + ((hi - lo) & ~3u);
     for (uint32_t i = lo + tid * 4u; i < full; i += kAggThreads * 4u) __stcs(reinterpret_cast<float4*>(out + i), make_float4(0.f, 0.f, 0.f, 0.f));
     for (uint32_t i = full + tid; i < hi; i += kAggThreads) out[i] = 0.f;
   }
@@ -367,7 +371,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     // no table of run starts: a warp per worker finds the run of this tile in the worker's sorted
     // row, half the warp searching for each end (16-way search: a few dependent loads)
     for (uint32_t w = warp; w < W; w += kAggThreads / 32) {
-      const uint32_t end = lo > 0xFFFFFFFFu - (uint32_t)kAggSparseTile ? 0xFFFFFFFFu : lo + (uint32_t)kAggSparseTile;
+      const uint32_t end = lo > 0xFFFFFFFFu - kTile ? 0xFFFFFFFFu : lo + kTile;
       const uint32_t key = lane < 16 ? lo : end;                 // every index is below 2^32 - 1
       const uint32_t at = half_warp_lower_bound(msgs, w, K, key, lane);
       const uint32_t e = __shfl_sync(0xFFFFFFFFu, at, 16);
@@ -440,7 +444,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     bool any_shared = false;
     for (uint32_t q = tid; q < total; q += kAggThreads) {
       const uint32_t local = st_idx[q] - lo;
-      if (local < (uint32_t)kAggSparseTile) {
+      if (local < kTile) {
         const uint32_t bit = 1u << (local & 31u);
         if (atomicOr(&s_seen[local >> 5], bit) & bit) { atomicOr(&s_shared[local >> 5], bit); any_shared = true; }
       }
@@ -449,7 +453,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     // a sole sender's coordinate: the sum is the value
     for (uint32_t q = tid; q < total; q += kAggThreads) {
       const uint32_t idx = st_idx[q], local = idx - lo;
-      if (local >= (uint32_t)kAggSparseTile || idx >= d) continue;   // malformed row: ignore
+      if (local >= kTile || idx >= d) continue;                      // malformed row: ignore
       if (!((s_shared[local >> 5] >> (local & 31u)) & 1u)) {
         const double v = 0.0 + msgs.term(st_w[q], st_val[q]);          // (the sum starts from +0: a lone -0 gives +0)
         dst.store(idx, (float)agg_scaled(v, 1u, sc));
@@ -479,7 +483,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     auto slot_of = [&](uint32_t local) { return s_slot[local >> 5] + __popc(s_shared[local >> 5] & ((1u << (local & 31u)) - 1u)); };
     for (uint32_t q = tid; q < total; q += kAggThreads) {            // entries per slot
       const uint32_t local = st_idx[q] - lo;
-      if (local < (uint32_t)kAggSparseTile && st_idx[q] < d && ((s_shared[local >> 5] >> (local & 31u)) & 1u))
+      if (local < kTile && st_idx[q] < d && ((s_shared[local >> 5] >> (local & 31u)) & 1u))
         atomicAdd(&s_cur[slot_of(local)], 1u);
     }
     __syncthreads();
@@ -501,7 +505,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     }
     for (uint32_t q = tid; q < total; q += kAggThreads) {            // scatter the stage positions
       const uint32_t local = st_idx[q] - lo;
-      if (local < (uint32_t)kAggSparseTile && st_idx[q] < d && ((s_shared[local >> 5] >> (local & 31u)) & 1u)) {
+      if (local < kTile && st_idx[q] < d && ((s_shared[local >> 5] >> (local & 31u)) & 1u)) {
         const uint32_t sl = slot_of(local);
         s_pool[s_off[sl] + atomicAdd(&s_cur[sl], 1u)] = (uint16_t)q;
       }
@@ -532,7 +536,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
   for (uint32_t q = tid; q < total; q += kAggThreads) {
     const uint32_t w = worker_of(q);
     const uint32_t idx = idx_at(w, q - s_pre[w]);
-    if (idx - lo >= (uint32_t)kAggSparseTile || idx >= d) continue;   // malformed row: ignore
+    if (idx - lo >= kTile || idx >= d) continue;                      // malformed row: ignore
     double sum = 0.0;
     uint32_t senders = 0;
     bool owner = true;

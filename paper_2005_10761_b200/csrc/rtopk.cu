@@ -654,24 +654,29 @@ int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_
   if (scale_mode == RTOPK_SCALE_COUNT && W > 65535) return RTOPK_ERR_UNSUPPORTED;
   if ((uintptr_t)out & 15u) return RTOPK_ERR_INVALID_ARG;
   if ((uint64_t)k * (uint64_t)W >= (1ull << 32)) return RTOPK_ERR_INVALID_ARG;
-  const bool sparse = aggregate_is_sparse(d, W, k);
-  const uint32_t tile = sparse ? (uint32_t)kAggSparseTile : (uint32_t)kAggTile;
+  // three regimes by the entries an output tile holds on average: up to 1024 per 16384 coordinates (the
+  // paper's densities): the sparse kernel; up to 1536 per 4096 coordinates: the same kernel on small tiles;
+  // beyond: the dense kernel, which adds the workers' runs one after the other into a tile of sums
+  const bool sparse16 = aggregate_is_sparse(d, W, k);
+  const bool sparse4 = !sparse16 && W <= kAggMaxW && (uint64_t)W * (uint64_t)k * 8ull <= 3ull * (uint64_t)d;
+  const bool sparse = sparse16 || sparse4;
+  const uint32_t tile = sparse16 ? (uint32_t)kAggSparseTile : (uint32_t)kAggTile;
   const uint32_t ntiles = (uint32_t)((d + tile - 1) / tile);
   // the span-table format brings the sparse kernel's table of run starts along
   static_assert(kAggSparseTile == (int)kTiledSpan, "the spans of the format are the sparse kernel's tiles");
   const uint32_t* starts = ctx->d_agg_starts;
   bool have_starts = false;
   if constexpr (std::is_same<M, TiledMsgs>::value) {
-    if (sparse) { starts = msgs.tab; have_starts = true; }
+    if (sparse16) { starts = msgs.tab; have_starts = true; }
   }
-  if (!sparse) run_cnt = nullptr;
+  if (!sparse16) run_cnt = nullptr;
   if (run_cnt) { starts = run_inv; have_starts = true; }     // kept by the sparsifier while it wrote the messages
   if (!have_starts && (size_t)W * (ntiles + 1) > ctx->agg_start_entries) return RTOPK_ERR_INVALID_ARG;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return RTOPK_ERR_CUDA;
   // with few workers and tiles the sparse kernel finds every tile's runs itself (one launch fewer);
   // otherwise a table of run starts is built first, all searches side by side
-  const bool own_search = !have_starts && sparse && W <= kAggSearchW && (uint64_t)ntiles * (uint64_t)((W + 7) / 8) <= 4096u;
+  const bool own_search = !have_starts && sparse16 && W <= kAggSearchW && (uint64_t)ntiles * (uint64_t)((W + 7) / 8) <= 4096u;
   if (!own_search && !have_starts) {
     const dim3 sgrid((ntiles + 1 + kAggThreads - 1) / kAggThreads, (uint32_t)W);
     k_agg_starts<M><<<sgrid, kAggThreads, 0, st>>>(msgs, (uint32_t)W, (uint32_t)k, ntiles, tile, ctx->d_agg_starts);
@@ -686,9 +691,14 @@ int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_
     const uint32_t clear = (eta < 0.0f && velocity == nullptr) ? 1u : 0u;
     // momentum: the sent coordinates are updated here and marked, the others by a plain pass behind it
     if (velocity) RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_sent, 0, ((size_t)d + 31) / 32 * sizeof(uint32_t), st));
-    k_aggregate_sparse<M><<<ntiles, kAggThreads, 0, st>>>(msgs, own_search ? nullptr : starts, (uint32_t)d,
-                                                          (uint32_t)W, (uint32_t)k, sc, eta, out, mu, velocity,
-                                                          ctx->d_sent, clear, run_cnt);
+    if (sparse16)
+      k_aggregate_sparse<M, kAggSparseTile><<<ntiles, kAggThreads, 0, st>>>(msgs, own_search ? nullptr : starts, (uint32_t)d,
+                                                                            (uint32_t)W, (uint32_t)k, sc, eta, out, mu,
+                                                                            velocity, ctx->d_sent, clear, run_cnt);
+    else
+      k_aggregate_sparse<M, kAggTile><<<ntiles, kAggThreads, 0, st>>>(msgs, starts, (uint32_t)d, (uint32_t)W, (uint32_t)k,
+                                                                      sc, eta, out, mu, velocity, ctx->d_sent, clear,
+                                                                      nullptr);
     ++ctx->launches;
     if (velocity) {
       const uint32_t groups = (uint32_t)((d + 3) / 4);
