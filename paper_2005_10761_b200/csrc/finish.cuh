@@ -24,9 +24,11 @@
 //                 the chunks before (the prefix) plus those before it in its own run (a segmented prefix
 //                 over the tile; for the one run that may reach back into earlier tiles, at most 4095
 //                 entries, the block counts the members among them again).  The members the subset
-//                 chose become messages and their residual slots are zeroed.
-// A block walks several tiles and fetches the next one while it works on the current one: these kernels
-// are chains of dependent memory round trips, and one wave of blocks pays the slice's set-up once.
+//                 chose go through a per-warp queue and become messages; their residual slots are
+//                 zeroed; in a step call the run table of the messages is kept for the aggregation.
+// A block walks several tiles (k_run_count fetches the next one while it works on the current one):
+// these kernels are chains of dependent memory round trips, and one wave of blocks pays the slice's
+// set-up once.
 //
 // Whatever does not fit this scheme -- the first bracket missed (too few or too many candidates), the
 // r-th largest key lies above the bracket, or more than kListMax candidates share the bucket (heavy
