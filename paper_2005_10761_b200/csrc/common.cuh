@@ -77,17 +77,12 @@ struct TauHistory { uint32_t tau1, tau2; float err; uint32_t valid; };
 
 // Where the run kernels (finish.cuh) stand with one slice.
 constexpr int kListMax = 2048;        // the histogram bucket that holds the r-th largest key is resolved on a list of up to this many candidates
-struct alignas(64) Fin {
+struct alignas(32) Fin {
   uint32_t tau, cut;         // the exact r-th largest key; a key equal to it is a member up to this index
   uint32_t ok;
   uint32_t list_n;           // entries of the slice's short list
-  uint32_t done1, done2;     // blocks of k_run_hist / k_run_count that have completed
-  // the bucket of the bracket's histogram that holds the r-th largest key (k_run_hist's last block):
-  uint32_t b_lo, b_hi;       // keys lo <= key < hi
-  uint32_t b_above;          // candidates above it
-  uint32_t b_n;              // candidates inside it
-  uint32_t b_ok;             // 0: the run kernels do not go on with this slice
-  uint32_t pad[5];
+  uint32_t done2;            // blocks of k_run_count that have completed
+  uint32_t pad[3];
 };
 
 struct Scratch {

@@ -12,8 +12,8 @@
 // work is spread evenly however unevenly the candidates are spread over the chunks:
 //
 //   k_run_hist    the histogram (block-local first, the keys above the bracket counted in registers);
-//                 clears the chunks' member counts; the last block of a slice picks the bucket.
-//   k_run_count   the sure members are counted per chunk (a thread adds its eight entries to their
+//                 clears the chunks' member counts.
+//   k_run_count   every block picks the bucket for itself while its first tile is on its way.  The sure members are counted per chunk (a thread adds its eight entries to their
 //                 chunks' counts, one addition per chunk it meets), the candidates inside the bucket go
 //                 to a short list.  The last block of a slice finds the r-th element of the whole order
 //                 -- larger magnitude first, then lower index -- on the list: its key is the exact
@@ -94,7 +94,6 @@ __device__ __forceinline__ void run_pick(const uint32_t* hist, uint32_t need, ui
 // grid: (blocks per slice, n_slices); a block takes tile after tile of kRunThreads * kHistPer candidates
 __global__ void __launch_bounds__(kRunThreads) k_run_hist(Launch L) {
   __shared__ uint32_t hist[kBins];
-  __shared__ uint32_t s[16];
   const uint32_t sl = blockIdx.y, tid = threadIdx.x, lane = tid & 31u;
   const Slice S = L.s.slices[sl];
   const uint32_t n_cand = L.s.cursor[sl];
@@ -132,30 +131,6 @@ __global__ void __launch_bounds__(kRunThreads) k_run_hist(Launch L) {
   __syncthreads();
   uint32_t* gh = L.s.hist + (size_t)sl * kBins;
   for (uint32_t b = tid; b < (uint32_t)kBins; b += kRunThreads) { const uint32_t c = hist[b]; if (c) atomicAdd(gh + b, c); }
-  // the last block of the slice picks the bucket that holds the r-th largest key
-  Fin* F = L.s.fin + sl;
-  __syncthreads();
-  if (tid == 0) {
-    __threadfence();
-    s[15] = atomicAdd(&F->done1, 1u) == nblocks - 1u;
-    if (s[15]) __threadfence();
-  }
-  __syncthreads();
-  if (!s[15]) return;
-#pragma unroll
-  for (int i = 0; i < kBins / kRunThreads; ++i) hist[tid + i * kRunThreads] = __ldcg(gh + tid + i * kRunThreads);
-  __syncthreads();
-  uint32_t D, above;
-  run_pick(hist, S.r, s, D, above);
-  if (tid != 0) return;
-  const bool in_bracket = D < (uint32_t)(kBins - 1);              // else: the r-th largest key lies above the bracket
-  const uint32_t n = in_bracket ? hist[D] : 0u;
-  const uint32_t lo = tau_lo + (D << sh);
-  F->b_lo = lo;
-  F->b_hi = min(tau_hi + 1u, lo + (1u << sh));
-  F->b_above = above;
-  F->b_n = n;
-  F->b_ok = in_bracket && n <= (uint32_t)kListMax;                // else: heavy ties
 }
 
 // Eight consecutive entries of a slice's candidate list, starting at entry i0 (a multiple of 8; the
@@ -185,9 +160,10 @@ __global__ void __launch_bounds__(kRunThreads, 4) k_run_count(Launch L) {
   const uint32_t sl = blockIdx.y, tid = threadIdx.x;
   const Slice S = L.s.slices[sl];
   const uint32_t n_cand = L.s.cursor[sl];
+  const uint32_t tau_lo = L.s.state[sl].tau_lo, tau_hi = max(tau_lo, L.s.state[sl].tau_hi);
   Fin* F = L.s.fin + sl;
-  const uint32_t b_ok = F->b_ok, b_lo = F->b_lo, b_hi = F->b_hi, b_above = F->b_above, b_n = F->b_n;
-  if (S.r == S.len || !b_ok) return;                               // (the same in every block of the slice)
+  if (S.r == S.len) return;
+  if (n_cand < S.r || n_cand > S.cand_cap) return;               // the bracket missed: left to k_finish
   const uint32_t n_tiles = (n_cand + kRunTile - 1) / kRunTile;
   const uint32_t nblocks = min(gridDim.x, n_tiles);
   if (blockIdx.x >= nblocks) return;
@@ -196,10 +172,25 @@ __global__ void __launch_bounds__(kRunThreads, 4) k_run_count(Launch L) {
   const uint32_t* ri = L.s.raw_idx + S.cand_off;
   uint32_t* lkey = L.s.list + (size_t)sl * 2 * kListMax;
   uint32_t* lidx = lkey + kListMax;
-  const uint32_t width = b_hi - b_lo;
   float v[kRunPer], vn[kRunPer];
   uint32_t ix[kRunPer], ixn[kRunPer];
   run_load8(rv, ri, blockIdx.x * (uint32_t)kRunTile + tid * (uint32_t)kRunPer, n_cand, v, ix);
+  // While the first tile is on its way: the bucket of the bracket's histogram that holds the r-th largest
+  // key.  Every block picks it for itself (8 KB of histogram and one block scan cost less than a launch, or
+  // a last-block hand-over, of their own); the answer is the same in every block of the slice.
+  const uint32_t* gh = L.s.hist + (size_t)sl * kBins;
+#pragma unroll
+  for (int i = 0; i < kBins / kRunThreads; ++i) hist[tid + i * kRunThreads] = __ldcg(gh + tid + i * kRunThreads);
+  __syncthreads();
+  uint32_t D, b_above;
+  run_pick(hist, S.r, s, D, b_above);
+  if (D >= (uint32_t)(kBins - 1)) return;                         // the r-th largest key lies above the bracket (or is missing)
+  const uint32_t b_n = hist[D];
+  if (b_n > (uint32_t)kListMax) return;                            // heavy ties
+  const uint32_t sh = bracket_shift(tau_lo, tau_hi);
+  const uint32_t b_lo = tau_lo + (D << sh), b_hi = min(tau_hi + 1u, b_lo + (1u << sh));
+  const uint32_t width = b_hi - b_lo;
+  __syncthreads();                                                 // (hist is used again by the last block)
   for (uint32_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
     const uint32_t i0 = tile * (uint32_t)kRunTile + tid * (uint32_t)kRunPer;
     const uint32_t nx = tile + gridDim.x;                          // the next tile is under way while this one is counted
@@ -341,8 +332,8 @@ __global__ void __launch_bounds__(kRunThreads, 4) k_run_count(Launch L) {
     }
   }
   if (tid != 0) return;
-  Fin f;
-  f.tau = tau; f.cut = cut; f.ok = 1; f.list_n = 0; f.done2 = 0;
+  Fin f = {};
+  f.tau = tau; f.cut = cut; f.ok = 1;
   L.s.fin[sl] = f;
   // what rtopk_get_stats reports, and the threshold history
   st->prefix = tau; st->resolved = 31; st->n_gt = n_gt; st->need = quota;

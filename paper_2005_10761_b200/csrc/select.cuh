@@ -35,7 +35,7 @@ __device__ __forceinline__ void clear_slice_counters(const Launch& L, uint32_t s
   const uint32_t nchunks = slice_chunks(S);
   const uint32_t ngroups = (nchunks + (1u << S.gshift) - 1u) >> S.gshift;
   for (uint32_t g = t; g < ngroups; g += nt) L.s.group_total[S.group_begin + g] = 0;
-  if (t == 0) { L.s.cursor[sl] = 0; L.s.done[sl] = 0; L.s.fin[sl].list_n = 0; L.s.fin[sl].done1 = 0; L.s.fin[sl].done2 = 0; L.s.fin[sl].b_ok = 0; }
+  if (t == 0) { L.s.cursor[sl] = 0; L.s.done[sl] = 0; L.s.fin[sl].list_n = 0; L.s.fin[sl].done2 = 0; }
   if (sl == 0 && t < 4u) L.s.tickets[t] = 0;
 }
 
@@ -52,7 +52,7 @@ __global__ void k_init_state(Launch L, uint32_t general) {
   if (S.r == S.len) { st.resolved = 31; st.stage = STAGE_DONE; st.flags = 0; }   // top-r is everything
   else { st.resolved = 0; st.stage = STAGE_PASS0; st.flags = general ? FLAG_GENERAL : 0u; }
   L.s.state[s] = st;
-  L.s.fin[s].list_n = 0; L.s.fin[s].done1 = 0; L.s.fin[s].done2 = 0; L.s.fin[s].b_ok = 0;
+  L.s.fin[s].list_n = 0; L.s.fin[s].done2 = 0;
 }
 
 // ----------------------------------------------------------------------------- sampled threshold
