@@ -654,11 +654,14 @@ int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_
   if (scale_mode == RTOPK_SCALE_COUNT && W > 65535) return RTOPK_ERR_UNSUPPORTED;
   if ((uintptr_t)out & 15u) return RTOPK_ERR_INVALID_ARG;
   if ((uint64_t)k * (uint64_t)W >= (1ull << 32)) return RTOPK_ERR_INVALID_ARG;
-  // three regimes by the entries an output tile holds on average: up to 1024 per 16384 coordinates (the
-  // paper's densities): the sparse kernel; up to 1536 per 4096 coordinates: the same kernel on small tiles;
-  // beyond: the dense kernel, which adds the workers' runs one after the other into a tile of sums
+  // Three regimes.  Up to 1024 entries per 16384 coordinates on average (the paper's densities): the sparse
+  // kernel.  Beyond: the same kernel on tiles of 4096 while such a tile holds at most 1536 entries and a worker
+  // sends at most d / 64 of them -- the dense kernel, which adds the workers' runs one after the other into a
+  // tile of sums, pays one block barrier per worker and tile (about 1.3 ns x tiles x W in all) but then
+  // takes 120 entries per ns against the sparse kernel's 45, so it wins once the rows are denser than that.
   const bool sparse16 = aggregate_is_sparse(d, W, k);
-  const bool sparse4 = !sparse16 && W <= kAggMaxW && (uint64_t)W * (uint64_t)k * 8ull <= 3ull * (uint64_t)d;
+  const bool sparse4 = !sparse16 && W <= kAggMaxW && (uint64_t)W * (uint64_t)k * 8ull <= 3ull * (uint64_t)d &&
+                       (uint64_t)k * 64ull <= (uint64_t)d;
   const bool sparse = sparse16 || sparse4;
   const uint32_t tile = sparse16 ? (uint32_t)kAggSparseTile : (uint32_t)kAggTile;
   const uint32_t ntiles = (uint32_t)((d + tile - 1) / tile);
