@@ -290,9 +290,26 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(M msgs, const uint32_
         }
       }
     } else {
+      // worker after worker, a block barrier between them (two workers may hold the same coordinate).  The
+      // first entry of every thread for the next worker is fetched before the barrier of the current one, so
+      // that the barrier does not stand in front of a memory round trip.
+      uint32_t nxt_i = 0;
+      float nxt_v = 0.f;
+      bool nxt_ok = false;
+      auto fetch = [&](uint32_t w) {
+        const uint32_t n = s_pre[w + 1] - s_pre[w];
+        nxt_ok = tid < n;
+        if (nxt_ok) { nxt_i = msgs.index_in(w0 + w, s_beg[w] + tid, span_lo) - lo; nxt_v = msgs.value(w0 + w, s_beg[w] + tid); }
+      };
+      fetch(0);
       for (uint32_t w = 0; w < nw; ++w) {
         const uint32_t b = s_beg[w], n = s_pre[w + 1] - s_pre[w];
-        for (uint32_t q = tid; q < n; q += kAggThreads) {
+        const bool ok = nxt_ok;
+        const uint32_t i0 = nxt_i;
+        const float v0 = nxt_v;
+        if (w + 1 < nw) fetch(w + 1);
+        if (ok && i0 < (uint32_t)kAggTile) { acc[i0] += msgs.term(w0 + w, v0); if (COUNT) ++senders[i0]; }
+        for (uint32_t q = tid + kAggThreads; q < n; q += kAggThreads) {
           const uint32_t i = msgs.index_in(w0 + w, b + q, span_lo) - lo;
           if (i < (uint32_t)kAggTile) { acc[i] += msgs.term(w0 + w, msgs.value(w0 + w, b + q)); if (COUNT) ++senders[i]; }
         }
