@@ -462,16 +462,16 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
     ctx->history_stale = true;
   }
   mark(ctx, RTOPK_PHASE_SUBSET, st);
-  // The sampling kernels clear the leading counters of the zeroed region themselves; the exact
-  // primary path has no such kernel.  The rest (the histograms, the
-  // selection bitmap) is first touched by the sampler and the exact path, both behind the fork.
+  // k_sample clears the leading counters of the zeroed region itself; with the bracket from the histogram
+  // pass there is no such kernel and the whole region is cleared here.  The rest (the histograms, the
+  // selection bitmap, the run table of the messages) is first touched behind the streaming pass or by the
+  // subset kernels: it is cleared on the side stream.
   const bool late_on_side = ctx->select_path == 0;
   if (!late_on_side) RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero, 0, zbytes, st));
   // Calls that are finished by the run kernels need the subset only for the last of them, and those kernels
   // leave most of every SM idle, whereas the streaming pass wants all of it from its first microsecond: there
   // the subset is drawn beside the run kernels, not beside the start of the pass.
-  const bool from_runs = P.any_select && L.n_slices <= 65535u &&
-                         ctx->finish_path != 1;
+  const bool from_runs = P.any_select && L.n_slices <= 65535u && ctx->finish_path != 1;
   const bool sampler_late = from_runs && late_on_side && P.any_sampler;
   const bool forked = P.any_sampler && !sampler_late;
   if (forked) {
@@ -499,7 +499,8 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   rc = grad_dtype == RTOPK_F32 ? launch_select<float>(ctx, P, L, st, join, late)
                                : launch_select<__nv_bfloat16>(ctx, P, L, st, join, late);
   if (rc) return rc;
-  // (launch_select has made the stream wait for the side stream behind the streaming pass)
+  // (a subset drawn beside the streaming pass has been waited for by launch_select; one drawn beside the run
+  // kernels is waited for in front of the emission below)
   mark(ctx, RTOPK_PHASE_FINISH, st);
   if (from_runs) {
     // the usual case is finished straight from the streaming pass's runs, all slices side by side; what
