@@ -223,3 +223,61 @@ def test_c5_limits_topk_and_randomk(lib):
     assert torch.equal(_bits(out[i]), _bits(val[0]))                  # W = 1: the update is the message
     assert int((out != 0).sum()) <= cfg.k
     ctx.close()
+
+
+def test_c3_message_formats_and_master_updates_at_full_size(lib):
+    # The messages of one c3_f32 round through everything that follows the sparsifier: the bit-packed and the
+    # span-table format (encoder outputs against the oracle's, the aggregation with the decoder fused in against
+    # the oracle's average of the decoded messages), the master update and the momentum update of all 25.6 M
+    # coordinates, bit for bit.
+    cfg = wl.configs()["c3_f32"]
+    d, W, k = cfg.d, cfg.W, cfg.k
+    ctx = lib.RTopK(d_max=d, W_max=W, r_max=cfg.r, k_max=k)
+    g = wl.gradient(cfg, 0, "cuda")
+    m = wl.zero_residual(cfg, "cuda")
+    idx = torch.zeros((W, k), dtype=torch.int32, device="cuda")
+    val = torch.zeros((W, k), dtype=torch.float32, device="cuda")
+    out = torch.empty(wl.round_up(d, 4), dtype=torch.float32, device="cuda")
+    ctx.step(g, m, d, cfg.r, k, cfg.seed, 0, idx, val, out)
+    del g, m
+    idx_h, val_h = idx.cpu().numpy().view(np.uint32), val.cpu().numpy()
+    # span table
+    spans, ll, lh = lib.tiled_layout(d, k)
+    tab = torch.zeros((W, spans + 1), dtype=torch.int32, device="cuda")
+    low = torch.zeros((W, ll), dtype=torch.int16, device="cuda")
+    qv = torch.zeros((W, lh), dtype=torch.int16, device="cuda")
+    ctx.encode_tiled(idx, val, d, tab, low, qv)
+    o_tab, o_low, o_qv = oracle.encode_tiled(idx_h, val_h, d)
+    assert np.array_equal(tab.cpu().numpy().view(np.uint32), o_tab)
+    assert np.array_equal(low.cpu().numpy().view(np.uint16)[:, :k], o_low)
+    assert np.array_equal(qv.cpu().numpy().view(np.uint16)[:, :k], o_qv)
+    d_idx, d_val = oracle.decode_tiled(o_tab, o_low, o_qv, d, k)
+    assert np.array_equal(d_idx, idx_h)
+    want = oracle.aggregate(d_idx, d_val, d)[1]
+    ctx.aggregate_tiled(tab, low, qv, d, k, out)
+    assert np.array_equal(out.cpu().numpy()[:d].view(np.uint32), want.view(np.uint32))
+    # bit-packed
+    bits, lw, lh = lib.packed_layout(d, k)
+    pi = torch.zeros((W, lw), dtype=torch.int32, device="cuda")
+    pv = torch.zeros((W, lh), dtype=torch.int16, device="cuda")
+    ctx.encode(idx, val, d, pi, pv)
+    o_pi, o_pv = oracle.encode(idx_h, val_h, d)
+    assert np.array_equal(pi.cpu().numpy().view(np.uint32)[:, :o_pi.shape[1]], o_pi)
+    ctx.aggregate_packed(pi, pv, d, k, out)
+    assert np.array_equal(out.cpu().numpy()[:d].view(np.uint32), want.view(np.uint32))
+    # master updates
+    rng = np.random.default_rng(3)
+    w0 = rng.standard_normal(d).astype(np.float32)
+    v0 = (rng.standard_normal(d) * 0.1).astype(np.float32)
+    w, v = torch.zeros_like(out), torch.zeros_like(out)
+    w[:d] = torch.from_numpy(w0).cuda()
+    v[:d] = torch.from_numpy(v0).cuda()
+    ctx.apply_momentum(idx, val, d, 0.05, 0.9, v, w)
+    o_v, o_w = oracle.apply_momentum(idx_h, val_h, d, 0.05, 0.9, v0, w0)
+    assert np.array_equal(v.cpu().numpy()[:d].view(np.uint32), o_v.view(np.uint32))
+    assert np.array_equal(w.cpu().numpy()[:d].view(np.uint32), o_w.view(np.uint32))
+    w[:d] = torch.from_numpy(w0).cuda()
+    ctx.apply_update(idx, val, d, 0.05, w)
+    assert np.array_equal(w.cpu().numpy()[:d].view(np.uint32), oracle.apply_update(idx_h, val_h, d, 0.05, w0).view(np.uint32))
+    ctx.poll_status()
+    ctx.close()
