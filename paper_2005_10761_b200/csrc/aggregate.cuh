@@ -5,8 +5,8 @@
 // (k_agg_starts).  Sums run in double precision in worker order (0, 1, ...) and are rounded once, so
 // the result is bit-reproducible.
 //
-//   k_aggregate_sparse  (W * k << d, the usual case): the output has been cleared by a memset and
-//                       only the coordinates that some worker sent are computed;
+//   k_aggregate_sparse  (W * k << d, the usual case): a block clears its tile of the output (or the caller
+//                       has) and only the coordinates that some worker sent are computed;
 //   k_aggregate         (dense messages): a block adds the runs worker by worker into a shared
 //                       tile of doubles and writes the tile once (zero fill and scatter in one pass).
 #pragma once
@@ -376,13 +376,16 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
   const uint32_t lo = blockIdx.x * kTile;
   const uint32_t span_lo = lo - lo % kTiledSpan;
   if (tid == 0) s_carry = 0;
-  if (clear) {
-    // the update is zero wherever no worker sent anything: the tile is cleared here (asynchronous stores
-    // beside the loads that follow; the barriers below order them before the block's own results)
+  // The update is zero wherever no worker sent anything, and the block clears its tile itself.  The stores are
+  // issued once the tile's entries have arrived in shared memory, so that no load of the block queues behind
+  // them; they drain while the block works in shared memory, and a block barrier orders them before the
+  // block's own results.
+  auto clear_tile = [&]() {
+    if (!clear) return;
     const uint32_t hi = min(d, lo + kTile), full = lo + ((hi - lo) & ~3u);
     for (uint32_t i = lo + tid * 4u; i < full; i += kAggThreads * 4u) __stcs(reinterpret_cast<float4*>(out + i), make_float4(0.f, 0.f, 0.f, 0.f));
     for (uint32_t i = full + tid; i < hi; i += kAggThreads) out[i] = 0.f;
-  }
+  };
   __syncthreads();
   if (starts == nullptr) {
     // no table of run starts: a warp per worker finds the run of this tile in the worker's sorted
@@ -427,7 +430,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     __syncthreads();
   }
   const uint32_t total = s_carry;
-  if (total == 0) return;
+  if (total == 0) { clear_tile(); return; }
   if (tid == 0) s_pre[W] = total;
   const bool staged = total <= (uint32_t)kAggSparseStage;
   __syncthreads();
@@ -458,6 +461,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     // not: the second entry that sets a coordinate's "seen" bit also sets its "shared" bit.
     for (uint32_t i = tid; i < (uint32_t)(kAggSparseTile / 32); i += kAggThreads) { s_seen[i] = 0; s_shared[i] = 0; }
     __syncthreads();
+    clear_tile();                                                     // (ordered before the results by the barrier below)
     bool any_shared = false;
     for (uint32_t q = tid; q < total; q += kAggThreads) {
       const uint32_t local = st_idx[q] - lo;
@@ -548,6 +552,8 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
   // ---- a crowded tile (more entries than the stage holds): every entry looks the other workers' runs
   // up in global memory; the entry of the lowest worker that holds a coordinate owns it and sums that
   // coordinate over the workers in ascending order
+  clear_tile();
+  __syncthreads();
   auto idx_at = [&](uint32_t w, uint32_t j) { return msgs.index_in(w, s_beg[w] + j, span_lo); };
   auto val_at = [&](uint32_t w, uint32_t j) { return msgs.value(w, s_beg[w] + j); };
   for (uint32_t q = tid; q < total; q += kAggThreads) {

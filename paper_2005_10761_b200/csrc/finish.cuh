@@ -4,16 +4,16 @@
 // The streaming pass leaves the candidates of a slice in one dense list: per chunk of 4096 coordinates
 // a run of (index, value) entries in index order, the runs one behind the other in the order in which
 // the chunks were finished, and per chunk where its run starts.  It also leaves the sampled or predicted
-// bracket [tau_lo, tau_hi] of the r-th largest key.  A histogram of the candidates over the bracket --
-// 2047 equal buckets plus one for the keys above -- gives the bucket that holds the r-th largest key, and
-// that bucket splits the candidates: those above it are members of the top-r set for sure, those below
-// it are not, and the few dozen inside it are decided exactly.  Three grid-wide launches over all slices
-// at once; each walks the LIST in tiles of 2048 entries, eight consecutive entries per thread, so the
-// work is spread evenly however unevenly the candidates are spread over the chunks:
+// bracket [tau_lo, tau_hi] of the r-th largest key and, counted while the candidates were written, their
+// histogram over the bracket: 2047 equal buckets (the keys above the bracket are the rest of the list).
+// The bucket that holds the r-th largest key splits the candidates: those above it are members of the
+// top-r set for sure, those below it are not, and the few dozen inside it are decided exactly.  Two
+// grid-wide launches over all slices at once; each walks the LIST in tiles of 2048 entries, eight
+// consecutive entries per thread, so the work is spread evenly however unevenly the candidates are
+// spread over the chunks:
 //
-//   k_run_hist    the histogram (block-local first, the keys above the bracket counted in registers);
-//                 clears the chunks' member counts.
-//   k_run_count   every block picks the bucket for itself while its first tile is on its way.  The sure members are counted per chunk (a thread adds its eight entries to their
+//   k_run_count   every block picks the bucket for itself while its first tile is on its way.  The sure
+//                 members are counted per chunk (a thread adds its eight entries to their
 //                 chunks' counts, one addition per chunk it meets), the candidates inside the bucket go
 //                 to a short list.  The last block of a slice finds the r-th element of the whole order
 //                 -- larger magnitude first, then lower index -- on the list: its key is the exact
@@ -44,7 +44,6 @@ constexpr int kRunThreads = 256;
 constexpr int kRunWarps = kRunThreads / 32;
 constexpr int kRunPer = 8;                                   // consecutive list entries per thread
 constexpr int kRunTile = kRunThreads * kRunPer;              // list entries per tile
-constexpr int kHistPer = 8;                                  // candidates per thread and tile of k_run_hist
 constexpr int kScanPer = 16;                                 // loads in flight per thread of the prefix over the chunks
 constexpr int kRankMax = 512;                                // lists up to this length are ranked by counting
 
@@ -89,48 +88,6 @@ __device__ __forceinline__ void run_pick(const uint32_t* hist, uint32_t need, ui
   __syncthreads();
   D = s[8]; above = s[9];
   __syncthreads();
-}
-
-// grid: (blocks per slice, n_slices); a block takes tile after tile of kRunThreads * kHistPer candidates
-__global__ void __launch_bounds__(kRunThreads) k_run_hist(Launch L) {
-  __shared__ uint32_t hist[kBins];
-  const uint32_t sl = blockIdx.y, tid = threadIdx.x, lane = tid & 31u;
-  const Slice S = L.s.slices[sl];
-  const uint32_t n_cand = L.s.cursor[sl];
-  const uint32_t tau_lo = L.s.state[sl].tau_lo, tau_hi = max(tau_lo, L.s.state[sl].tau_hi);
-  if (S.r == S.len) return;
-  if (n_cand < S.r || n_cand > S.cand_cap) return;               // the bracket missed: left to k_finish
-  {
-    uint32_t* cm = L.s.chunk_pre + S.chunk_begin;                  // members per chunk: counted by k_run_count
-    const uint32_t nchunks = slice_chunks(S);
-    for (uint32_t c = blockIdx.x * kRunThreads + tid; c < nchunks; c += gridDim.x * kRunThreads) cm[c] = 0;
-  }
-  constexpr uint32_t kTile = kRunThreads * kHistPer;
-  const uint32_t nblocks = min(gridDim.x, (n_cand + kTile - 1u) / kTile);
-  if (blockIdx.x >= nblocks) return;
-  const uint32_t sh = bracket_shift(tau_lo, tau_hi);
-  for (uint32_t b = tid; b < (uint32_t)kBins; b += kRunThreads) hist[b] = 0;
-  __syncthreads();
-  const float* rv = L.s.raw_val + S.cand_off;
-  uint32_t n_hi = 0;                                               // the keys above the bracket share one bucket
-  for (uint32_t i0 = blockIdx.x * kTile; i0 < n_cand; i0 += gridDim.x * kTile) {
-    float v[kHistPer];
-#pragma unroll
-    for (int u = 0; u < kHistPer; ++u) { const uint32_t i = i0 + u * kRunThreads + tid; v[u] = i < n_cand ? rv[i] : 0.f; }
-#pragma unroll
-    for (int u = 0; u < kHistPer; ++u) {
-      const uint32_t key = mag_key(v[u]);
-      if (i0 + u * kRunThreads + tid < n_cand) {
-        if (key > tau_hi) ++n_hi;
-        else if (key >= tau_lo) atomicAdd(&hist[(key - tau_lo) >> sh], 1u);
-      }
-    }
-  }
-  n_hi = warp_sum(n_hi);
-  if (lane == 0 && n_hi) atomicAdd(&hist[kBins - 1], n_hi);
-  __syncthreads();
-  uint32_t* gh = L.s.hist + (size_t)sl * kBins;
-  for (uint32_t b = tid; b < (uint32_t)kBins; b += kRunThreads) { const uint32_t c = hist[b]; if (c) atomicAdd(gh + b, c); }
 }
 
 // Eight consecutive entries of a slice's candidate list, starting at entry i0 (a multiple of 8; the
@@ -179,8 +136,11 @@ __global__ void __launch_bounds__(kRunThreads, 4) k_run_count(Launch L) {
   // key.  Every block picks it for itself (8 KB of histogram and one block scan cost less than a launch, or
   // a last-block hand-over, of their own); the answer is the same in every block of the slice.
   const uint32_t* gh = L.s.hist + (size_t)sl * kBins;
+  uint32_t part = 0, inside;
 #pragma unroll
-  for (int i = 0; i < kBins / kRunThreads; ++i) hist[tid + i * kRunThreads] = __ldcg(gh + tid + i * kRunThreads);
+  for (int i = 0; i < kBins / kRunThreads; ++i) { const uint32_t h = __ldcg(gh + tid + i * kRunThreads); hist[tid + i * kRunThreads] = h; part += h; }
+  run_block_scan(part, s, inside);
+  if (tid == 0) hist[kBins - 1] = n_cand - inside;                 // the keys above the bracket: the rest of the list
   __syncthreads();
   uint32_t D, b_above;
   run_pick(hist, S.r, s, D, b_above);

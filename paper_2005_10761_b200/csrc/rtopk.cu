@@ -252,8 +252,8 @@ size_t carve_zero(const rtopk_ctx* ctx, const Plan& P, Scratch& s, size_t* early
   s.done = (uint32_t*)take(P.slices.size() * sizeof(uint32_t));
   s.cursor = (uint32_t*)take(P.slices.size() * sizeof(uint32_t));
   s.group_total = (uint32_t*)take((size_t)P.n_groups * sizeof(uint32_t));
-  if (early_bytes) *early_bytes = at;
   s.hist = (uint32_t*)take(P.slices.size() * kBins * sizeof(uint32_t));
+  if (early_bytes) *early_bytes = at;
   s.sel = (uint32_t*)take(P.sel_words * sizeof(uint32_t));
   s.tile_inv = (uint32_t*)take(P.table_words * sizeof(uint32_t));
   s.tile_cnt = (uint32_t*)take(P.table_words * sizeof(uint32_t));
@@ -286,8 +286,9 @@ int check_common(const rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t
 int run_sampler(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st, bool clear_first);
 
 // `late.on`: the side stream draws the k-of-r subset only once the streaming pass has ended (see
-// sparsify_impl); the stream does not wait for it here.
-struct LateSide { bool on; };
+// sparsify_impl); the stream does not wait for it here.  `late.hist`: the run kernels follow, so the
+// streaming pass also counts the candidates' histogram over the bracket.
+struct LateSide { bool on, hist; };
 
 template <typename GradT>
 int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st, cudaEvent_t join, LateSide late) {
@@ -298,8 +299,9 @@ int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t s
     const uint32_t per = (uint32_t)((P.slices[0].head + (uint64_t)P.slices[0].len + kChunk - 1) / kChunk);
     const uint32_t uniform = P.uniform ? per : 0u;
     const int blocks = ctx->stream_blocks[sizeof(GradT) == 4 ? 0 : 1];
-    if (ctx->test_giveup) k_stream<GradT, true><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
-    else k_stream<GradT, false><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
+    if (ctx->test_giveup) k_stream<GradT, true, false><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
+    else if (late.hist) k_stream<GradT, false, true><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
+    else k_stream<GradT, false, false><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
     ++ctx->launches;
     if (late.on) {
       // the streaming pass saturates the memory system and fills every SM, the kernels after it do neither:
@@ -495,7 +497,7 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
     RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero + early_bytes, 0, zbytes - early_bytes, st));
   }
   cudaEvent_t join = forked ? ctx->ev_join : nullptr;
-  const LateSide late = {sampler_late};
+  const LateSide late = {sampler_late, from_runs};
   rc = grad_dtype == RTOPK_F32 ? launch_select<float>(ctx, P, L, st, join, late)
                                : launch_select<__nv_bfloat16>(ctx, P, L, st, join, late);
   if (rc) return rc;
@@ -505,11 +507,6 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   if (from_runs) {
     // the usual case is finished straight from the streaming pass's runs, all slices side by side; what
     // these kernels leave (a missed bracket, heavy ties) is flagged for k_finish
-    // about one wave of blocks over all slices together (8 blocks of 256 threads per SM)
-    const uint32_t per_slice = std::max<uint32_t>(1u, ((uint32_t)ctx->sms * 8u + L.n_slices - 1u) / L.n_slices);
-    const uint32_t tiles = (P.cap_max + kRunThreads * kHistPer - 1) / (kRunThreads * kHistPer);
-    const dim3 hgrid(std::min(tiles, per_slice), L.n_slices);
-    k_run_hist<<<hgrid, kRunThreads, 0, st>>>(L);
     const uint32_t per_slice_run = std::max<uint32_t>(1u, ((uint32_t)ctx->sms * 4u + L.n_slices - 1u) / L.n_slices);
     const dim3 rgrid(std::min((P.cap_max + kRunTile - 1) / (uint32_t)kRunTile, per_slice_run), L.n_slices);
     k_run_count<<<rgrid, kRunThreads, 0, st>>>(L);
@@ -517,7 +514,7 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
     const uint32_t per_slice_emit = std::max<uint32_t>(1u, ((uint32_t)ctx->sms * 5u + L.n_slices - 1u) / L.n_slices);
     const dim3 egrid(std::min((P.cap_max + kRunTile - 1) / (uint32_t)kRunTile, per_slice_emit), L.n_slices);
     k_run_emit<<<egrid, kRunThreads, 0, st>>>(L);
-    ctx->launches += 3;
+    ctx->launches += 2;
   }
   if (P.any_select) {
     // the largest cluster size that still lets every slice's cluster be resident at once
@@ -601,9 +598,9 @@ int threshold_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_
   mark(ctx, RTOPK_PHASE_STREAM, st);
   const uint32_t per = (uint32_t)((P.slices[0].head + (uint64_t)P.slices[0].len + kChunk - 1) / kChunk);
   if (grad_dtype == RTOPK_F32)
-    k_stream<float, false><<<ctx->stream_blocks[0], kStreamThreads, sizeof(StreamSmem<float>), st>>>(L, P.n_chunks, per);
+    k_stream<float, false, false><<<ctx->stream_blocks[0], kStreamThreads, sizeof(StreamSmem<float>), st>>>(L, P.n_chunks, per);
   else
-    k_stream<__nv_bfloat16, false><<<ctx->stream_blocks[1], kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>), st>>>(L, P.n_chunks, per);
+    k_stream<__nv_bfloat16, false, false><<<ctx->stream_blocks[1], kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>), st>>>(L, P.n_chunks, per);
   ++ctx->launches;
   mark(ctx, RTOPK_PHASE_ORDER, st);
   k_thr_sizes<<<L.n_slices, kThrSizeThreads, 0, st>>>(L, (uint32_t)limit, (uint32_t)k, msg_count, msg_ones);
@@ -863,12 +860,14 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
   if (e == cudaSuccess) {
     int sms = 0, per_f32 = 0, per_bf16 = 0;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<float>));
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<float>));
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<__nv_bfloat16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<__nv_bfloat16>));
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<__nv_bfloat16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<__nv_bfloat16>));
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_f32, k_stream<float, false>, kStreamThreads, sizeof(StreamSmem<float>));
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_bf16, k_stream<__nv_bfloat16, false>, kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<float, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<float>));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<float, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<float>));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<float, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<float>));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<__nv_bfloat16, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<__nv_bfloat16>));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<__nv_bfloat16, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<__nv_bfloat16>));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<__nv_bfloat16, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<__nv_bfloat16>));
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_f32, k_stream<float, false, true>, kStreamThreads, sizeof(StreamSmem<float>));
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_bf16, k_stream<__nv_bfloat16, false, true>, kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>));
     if (e == cudaSuccess && (per_f32 < 1 || per_bf16 < 1)) e = cudaErrorLaunchOutOfResources;
     ctx->sms = sms;
     ctx->stream_blocks[0] = sms * per_f32;

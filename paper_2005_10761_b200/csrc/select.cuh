@@ -27,7 +27,8 @@ __device__ __forceinline__ uint32_t slice_chunks(const Slice& S) {
 }
 
 // Clears the counters of slice `sl` that the streaming pass, the run kernels and the exact path expect
-// to be zero (run cursor, block counter, list length, chunk-group totals; plus the launch-wide tickets).  The sampling
+// to be zero (run cursor, block counter, list length, chunk-group totals, the histogram over the bracket;
+// plus the launch-wide tickets).  The sampling
 // kernels do this instead of a memset node in front of them; `part` of `nparts` thread blocks of
 // blockDim.x threads share the work.
 __device__ __forceinline__ void clear_slice_counters(const Launch& L, uint32_t sl, const Slice& S, uint32_t part, uint32_t nparts) {
@@ -35,6 +36,7 @@ __device__ __forceinline__ void clear_slice_counters(const Launch& L, uint32_t s
   const uint32_t nchunks = slice_chunks(S);
   const uint32_t ngroups = (nchunks + (1u << S.gshift) - 1u) >> S.gshift;
   for (uint32_t g = t; g < ngroups; g += nt) L.s.group_total[S.group_begin + g] = 0;
+  for (uint32_t b = t; b < (uint32_t)kBins; b += nt) L.s.hist[(size_t)sl * kBins + b] = 0;
   if (t == 0) { L.s.cursor[sl] = 0; L.s.done[sl] = 0; L.s.fin[sl].list_n = 0; L.s.fin[sl].done2 = 0; }
   if (sl == 0 && t < 4u) L.s.tickets[t] = 0;
 }

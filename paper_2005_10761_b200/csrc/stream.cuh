@@ -125,7 +125,12 @@ template <> struct SmemGrad<__nv_bfloat16> {
 // treat their first wait as run out and its producer waits only briefly for them, so every block takes the
 // exit a real expiry would take -- error flag, a last bounded wait for the bulk copies still on their way
 // into the block's shared memory, return -- while all copies do arrive.
-template <typename GradT, bool GIVEUP>
+// HIST: the call is finished by the run kernels (finish.cuh).  Every candidate inside the bracket
+// [tau_lo, tau_hi] is then also counted in the slice's histogram over the bracket (one reduction into
+// global memory per such candidate: a third of the candidates, 0.4 % of the coordinates; the keys above
+// the bracket need no counting, their number is the rest of the list), and the chunk's member count is
+// cleared for k_run_count.  The table was cleared by the kernel in front of this one.
+template <typename GradT, bool GIVEUP, bool HIST>
 __global__ void __launch_bounds__(kStreamThreads, 3) k_stream(Launch L, uint32_t total_tiles, uint32_t uniform_chunks) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   StreamSmem<GradT>& sm = *reinterpret_cast<StreamSmem<GradT>*>(smem_raw);
@@ -182,7 +187,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) k_stream(Launch L, uint32_t
   const unsigned long long keep = l2_policy_evict_last();
   uint32_t cur_slice = 0xFFFFFFFFu;
   Slice S;
-  uint32_t tau = 0x80000000u;
+  uint32_t tau = 0x80000000u, tau_hi = 0x80000000u, sh = 0;
   for (uint32_t i = 0;; ++i) {
     const uint32_t stage = i % kStages, phase = (i / kStages) & 1u, buf = i & 1u;
     const bool arrived = GIVEUP ? false : mbar_wait(&sm.full[stage], phase);
@@ -200,6 +205,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) k_stream(Launch L, uint32_t
       cur_slice = d.slice;
       S = slices[cur_slice];
       tau = L.s.state[cur_slice].tau_lo;
+      if (HIST) { tau_hi = max(tau, L.s.state[cur_slice].tau_hi); sh = bracket_shift(tau, tau_hi); }
     }
     const uint32_t head = S.head, span = head + S.len;
     const uint32_t e_w = d.chunk * (uint32_t)kChunk + warp * (uint32_t)kWarpSpan;   // element on the slice's grid
@@ -257,6 +263,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) k_stream(Launch L, uint32_t
       const uint32_t tile = S.chunk_begin + d.chunk;
       L.s.chunk_start[tile] = start;
       L.s.chunk_count[tile] = bA;
+      if (HIST) L.s.chunk_pre[tile] = 0;
       sm.ex[buf] = start;
     }
     consumer_sync();
@@ -265,6 +272,7 @@ __global__ void __launch_bounds__(kStreamThreads, 3) k_stream(Launch L, uint32_t
       for (uint32_t w = 0; w < warp; ++w) before += sm.wA[buf][w];
       uint32_t* cidx = L.s.raw_idx + S.cand_off;
       float* cval = L.s.raw_val + S.cand_off;
+      uint32_t* gh = L.s.hist + (size_t)cur_slice * kBins;
 #pragma unroll
       for (int it = 0; it < kIter; ++it) {
         const uint32_t bits = (maskA >> (it * 4)) & 0xFu;
@@ -276,6 +284,10 @@ __global__ void __launch_bounds__(kStreamThreads, 3) k_stream(Launch L, uint32_t
             if ((bits >> j) & 1u) {
               if (pos < S.cand_cap) { st_hint(cidx + pos, e + j - head, keep); st_hint(reinterpret_cast<uint32_t*>(cval) + pos, __float_as_uint(a[it][j]), keep); }
               ++pos;
+              if (HIST) {
+                const uint32_t key = mag_key(a[it][j]);
+                if (key <= tau_hi) atomicAdd(gh + ((key - tau) >> sh), 1u);
+              }
             }
         }
         before += (totA >> (it * 8)) & 0xFFu;
