@@ -385,8 +385,10 @@ int run_sampler(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t st,
   ++ctx->launches;
   const dim3 sgrid((P.sel_words_max + kSelChunk - 1) / kSelChunk, n);
   if ((size_t)sgrid.x * n > ctx->sel_blk_entries) return RTOPK_ERR_INVALID_ARG;
-  k_sel_count<<<sgrid, kScanThreads, 0, st>>>(L);
-  ++ctx->launches;
+  if (sgrid.x > 1) {                                   // (a bitmap of one chunk has no chunks before it to add up)
+    k_sel_count<<<sgrid, kScanThreads, 0, st>>>(L);
+    ++ctx->launches;
+  }
   k_sel_scan<<<sgrid, kScanThreads, 0, st>>>(L);
   ++ctx->launches;
   return RTOPK_OK;

@@ -82,8 +82,8 @@ __global__ void __launch_bounds__(kDrawThreads) k_resolve(Launch L) {
 }
 
 // Exclusive prefix of the bitmap's popcounts.  A block owns kSelChunk consecutive words of one slice:
-// k_sel_count sums the chunk's popcounts, k_sel_scan adds the totals of the earlier chunks and scans
-// inside the chunk (8 consecutive words per thread).
+// k_sel_count sums the chunk's popcounts (not launched while every bitmap is a single chunk, r <= 262144),
+// k_sel_scan adds the totals of the earlier chunks and scans inside the chunk (8 consecutive words per thread).
 // grid of both: (ceil(most bitmap words of a slice / kSelChunk), n_slices); blk_tot is [n_slices][gridDim.x]
 constexpr int kScanThreads = 1024;
 constexpr int kSelPer = 8;
