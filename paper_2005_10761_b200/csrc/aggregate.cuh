@@ -350,6 +350,18 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate(M msgs, const uint32_
   }
 }
 
+// Bulk asynchronous copy shared -> global (TMA): both addresses 16-byte aligned, the size a multiple of 16 bytes.
+__device__ __forceinline__ void agg_bulk_store(void* dst, const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+               ::"l"(__cvta_generic_to_global(dst)), "r"((uint32_t)__cvta_generic_to_shared(src)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void agg_bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// ... until every bulk copy of the calling thread has been written to its destination
+__device__ __forceinline__ void agg_bulk_wait() {
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  asm volatile("fence.proxy.async;" ::: "memory");                 // the block's own stores to the same words come later
+}
+
 // A block stages the entries of its tile (all workers' runs, in worker order); the entry of the
 // lowest worker that holds a coordinate owns it and sums that coordinate over the workers in
 // ascending order (binary search in each staged run): the same fixed-order sum as k_aggregate.
@@ -376,17 +388,29 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
   const uint32_t lo = blockIdx.x * kTile;
   const uint32_t span_lo = lo - lo % kTiledSpan;
   if (tid == 0) s_carry = 0;
-  // The update is zero wherever no worker sent anything, and the block clears its tile itself.  The stores are
-  // issued once the tile's entries have arrived in shared memory, so that no load of the block queues behind
-  // them; they drain while the block works in shared memory, and a block barrier orders them before the
-  // block's own results.
-  auto clear_tile = [&]() {
-    if (!clear) return;
-    const uint32_t hi = min(d, lo + kTile), full = lo + ((hi - lo) & ~3u);
-    for (uint32_t i = lo + tid * 4u; i < full; i += kAggThreads * 4u) __stcs(reinterpret_cast<float4*>(out + i), make_float4(0.f, 0.f, 0.f, 0.f));
-    for (uint32_t i = full + tid; i < hi; i += kAggThreads) out[i] = 0.f;
-  };
+  // The update is zero wherever no worker sent anything, and the block clears its tile itself: one thread hands
+  // the tile to the copy engine, 4 KB of zeros from shared memory at a time, so that no thread waits while the
+  // 64 KB leave the SM (plain stores held every warp of the block for 3 to 6 us there).  The zeros lie where the
+  // pool of the shared coordinates' entries goes later; the thread waits for the copies right before the
+  // block's first result, and a block barrier orders every result behind that.
+  __shared__ __align__(128) uint16_t s_pool[kAggSparseStage];
+  static_assert(sizeof(uint16_t) * kAggSparseStage == 16 * kAggThreads, "one 16-byte vector of zeros per thread");
+  constexpr uint32_t kZeroBytes = sizeof(uint16_t) * kAggSparseStage;
+  if (clear) {
+    reinterpret_cast<uint4*>(s_pool)[tid] = make_uint4(0u, 0u, 0u, 0u);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // (the copy engine reads what the threads wrote)
+  }
   __syncthreads();
+  if (clear) {
+    const uint32_t hi = min(d, lo + kTile), full = (hi - lo) & ~3u;
+    if (tid == 0) {
+      for (uint32_t b = 0; b < full * 4u; b += kZeroBytes)
+        agg_bulk_store(reinterpret_cast<char*>(out + lo) + b, s_pool, min(kZeroBytes, full * 4u - b));
+      agg_bulk_commit();
+    }
+    if (lo + full + tid < hi) out[lo + full + tid] = 0.f;              // (the last words of an update that is no multiple of 4)
+  }
+  auto clear_wait = [&]() { if (clear && tid == 0) agg_bulk_wait(); };
   if (starts == nullptr) {
     // no table of run starts: a warp per worker finds the run of this tile in the worker's sorted
     // row, half the warp searching for each end (16-way search: a few dependent loads)
@@ -430,7 +454,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     __syncthreads();
   }
   const uint32_t total = s_carry;
-  if (total == 0) { clear_tile(); return; }
+  if (total == 0) { clear_wait(); return; }
   if (tid == 0) s_pre[W] = total;
   const bool staged = total <= (uint32_t)kAggSparseStage;
   __syncthreads();
@@ -443,7 +467,6 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     // ---- the usual case: the tile's entries fit the stage
     __shared__ uint16_t st_w[kAggSparseStage];                       // worker of every staged entry
     __shared__ uint32_t s_seen[kAggSparseTile / 32], s_shared[kAggSparseTile / 32];
-    __shared__ uint16_t s_pool[kAggSparseStage];
     // (the run tables are not needed once the entries are staged with their workers, nor is the "seen"
     // bitmap once the shared coordinates are marked: the slot tables take their place)
     static_assert(kAggSparseStage / 2 <= kAggMaxW, "the slot tables fit the run tables");
@@ -461,7 +484,6 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     // not: the second entry that sets a coordinate's "seen" bit also sets its "shared" bit.
     for (uint32_t i = tid; i < (uint32_t)(kAggSparseTile / 32); i += kAggThreads) { s_seen[i] = 0; s_shared[i] = 0; }
     __syncthreads();
-    clear_tile();                                                     // (ordered before the results by the barrier below)
     bool any_shared = false;
     for (uint32_t q = tid; q < total; q += kAggThreads) {
       const uint32_t local = st_idx[q] - lo;
@@ -470,6 +492,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
         if (atomicOr(&s_seen[local >> 5], bit) & bit) { atomicOr(&s_shared[local >> 5], bit); any_shared = true; }
       }
     }
+    clear_wait();                                                     // (the barrier orders the results behind the clearing)
     any_shared = __syncthreads_or(any_shared);
     // a sole sender's coordinate: the sum is the value
     for (uint32_t q = tid; q < total; q += kAggThreads) {
@@ -552,7 +575,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
   // ---- a crowded tile (more entries than the stage holds): every entry looks the other workers' runs
   // up in global memory; the entry of the lowest worker that holds a coordinate owns it and sums that
   // coordinate over the workers in ascending order
-  clear_tile();
+  clear_wait();
   __syncthreads();
   auto idx_at = [&](uint32_t w, uint32_t j) { return msgs.index_in(w, s_beg[w] + j, span_lo); };
   auto val_at = [&](uint32_t w, uint32_t j) { return msgs.value(w, s_beg[w] + j); };
