@@ -362,13 +362,29 @@ __device__ __forceinline__ void agg_bulk_wait() {
   asm volatile("fence.proxy.async;" ::: "memory");                 // the block's own stores to the same words come later
 }
 
+// Named barriers of k_aggregate_sparse: its eight working warps meet on barrier 1; the clearing warp joins them
+// on barrier 2.
+template <int ID, int N> __device__ __forceinline__ void agg_bar_sync() { asm volatile("bar.sync %0, %1;" ::"n"(ID), "n"(N) : "memory"); }
+template <int ID, int N> __device__ __forceinline__ void agg_bar_arrive() { asm volatile("bar.arrive %0, %1;" ::"n"(ID), "n"(N) : "memory"); }
+template <int ID, int N> __device__ __forceinline__ bool agg_bar_or(bool flag) {
+  uint32_t out;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.or.pred p, %2, %3, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(out) : "r"((uint32_t)flag), "n"(ID), "n"(N) : "memory");
+  return out != 0;
+}
+constexpr int kAggSparseThreads = kAggThreads + 32;                 // eight working warps and the clearing warp
+
 // A block stages the entries of its tile (all workers' runs, in worker order); the entry of the
 // lowest worker that holds a coordinate owns it and sums that coordinate over the workers in
 // ascending order (binary search in each staged run): the same fixed-order sum as k_aggregate.
 // TILE: output coordinates per block: kAggSparseTile for sparse messages, kAggTile where a tile of that size
 // would hold more entries than the stage (the bitmaps and slot tables are laid out for the larger one).
 template <typename M, int TILE>
-__global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const uint32_t* __restrict__ starts, uint32_t d,
+__global__ void __launch_bounds__(kAggSparseThreads) k_aggregate_sparse(M msgs, const uint32_t* __restrict__ starts, uint32_t d,
                                                                   uint32_t W, uint32_t K, AggScale sc,
                                                                   float eta, float* __restrict__ out, float mu,
                                                                   float* __restrict__ velocity, uint32_t* __restrict__ sent,
@@ -388,29 +404,38 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
   const uint32_t lo = blockIdx.x * kTile;
   const uint32_t span_lo = lo - lo % kTiledSpan;
   if (tid == 0) s_carry = 0;
-  // The update is zero wherever no worker sent anything, and the block clears its tile itself: one thread hands
-  // the tile to the copy engine, 4 KB of zeros from shared memory at a time, so that no thread waits while the
-  // 64 KB leave the SM (plain stores held every warp of the block for 3 to 6 us there).  The zeros lie where the
-  // pool of the shared coordinates' entries goes later; the thread waits for the copies right before the
-  // block's first result, and a block barrier orders every result behind that.
-  __shared__ __align__(128) uint16_t s_pool[kAggSparseStage];
-  static_assert(sizeof(uint16_t) * kAggSparseStage == 16 * kAggThreads, "one 16-byte vector of zeros per thread");
-  constexpr uint32_t kZeroBytes = sizeof(uint16_t) * kAggSparseStage;
-  if (clear) {
-    reinterpret_cast<uint4*>(s_pool)[tid] = make_uint4(0u, 0u, 0u, 0u);
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // (the copy engine reads what the threads wrote)
-  }
-  __syncthreads();
-  if (clear) {
+  // The update is zero wherever no worker sent anything, and the block clears its tile itself.  That is the
+  // ninth warp's only work: one of its lanes hands the tile to the copy engine, 4 KB of zeros from shared memory
+  // at a time, and waits until they are written, while the eight working warps fetch and sort the tile's entries
+  // (plain stores held every warp of the block for 3 to 6 us, and so did the copies' issue by a working thread:
+  // the clearing runs at the speed at which HBM takes the zeros).  The working warps meet the clearing warp right
+  // before the block's results.  (Starting the copies only once the entries have arrived, so that no load
+  // queues behind them, was 1 to 3 us slower per launch.)
+  constexpr uint32_t kZeroBytes = 4096;
+  __shared__ __align__(128) unsigned char s_zero[kZeroBytes];
+  if (warp == (uint32_t)(kAggThreads / 32)) {
+    if (!clear) return;
+    for (uint32_t i = lane; i < kZeroBytes / 16u; i += 32u) reinterpret_cast<uint4*>(s_zero)[i] = make_uint4(0u, 0u, 0u, 0u);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // (the copy engine reads what the lanes wrote)
+    __syncwarp();
     const uint32_t hi = min(d, lo + kTile), full = (hi - lo) & ~3u;
-    if (tid == 0) {
+    if (lane == 0) {
       for (uint32_t b = 0; b < full * 4u; b += kZeroBytes)
-        agg_bulk_store(reinterpret_cast<char*>(out + lo) + b, s_pool, min(kZeroBytes, full * 4u - b));
+        agg_bulk_store(reinterpret_cast<char*>(out + lo) + b, s_zero, min(kZeroBytes, full * 4u - b));
       agg_bulk_commit();
+      agg_bulk_wait();
     }
-    if (lo + full + tid < hi) out[lo + full + tid] = 0.f;              // (the last words of an update that is no multiple of 4)
+    if (lo + full + lane < hi) out[lo + full + lane] = 0.f;           // (the last words of an update that is no multiple of 4)
+    __syncwarp();
+    agg_bar_sync<2, kAggSparseThreads>();                           // the results may follow
+    return;
   }
-  auto clear_wait = [&]() { if (clear && tid == 0) agg_bulk_wait(); };
+  // every working warp passes this exactly once, on every path through the kernel
+  auto tile_cleared = [&](bool wait) {
+    if (!clear) return;
+    if (wait) agg_bar_sync<2, kAggSparseThreads>(); else agg_bar_arrive<2, kAggSparseThreads>();
+  };
+  auto sync_w = [&]() { agg_bar_sync<1, kAggThreads>(); };
   if (starts == nullptr) {
     // no table of run starts: a warp per worker finds the run of this tile in the worker's sorted
     // row, half the warp searching for each end (16-way search: a few dependent loads)
@@ -421,7 +446,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
       const uint32_t e = __shfl_sync(0xFFFFFFFFu, at, 16);
       if (lane == 0) { s_beg[w] = at; s_cnt[w] = e - at; }
     }
-    __syncthreads();
+    sync_w();
   }
   for (uint32_t w0 = 0; w0 < W; w0 += kAggThreads) {
     const uint32_t w = w0 + tid;
@@ -445,19 +470,19 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     }
     const uint32_t incl = warp_incl_scan(cnt);
     if (lane == 31) s_warp[warp] = incl;
-    __syncthreads();
+    sync_w();
     uint32_t woff = s_carry;
     for (uint32_t x = 0; x < warp; ++x) woff += s_warp[x];
     if (w < W) s_pre[w] = woff + incl - cnt;
-    __syncthreads();
+    sync_w();
     if (tid == kAggThreads - 1) s_carry = woff + incl;
-    __syncthreads();
+    sync_w();
   }
   const uint32_t total = s_carry;
-  if (total == 0) { clear_wait(); return; }
+  if (total == 0) { tile_cleared(false); return; }
   if (tid == 0) s_pre[W] = total;
   const bool staged = total <= (uint32_t)kAggSparseStage;
-  __syncthreads();
+  sync_w();
   auto worker_of = [&](uint32_t q) {                 // last worker with s_pre[w] <= q
     uint32_t a = 0, b = W;
     while (b - a > 1) { const uint32_t mid = (a + b) >> 1; if (s_pre[mid] <= q) a = mid; else b = mid; }
@@ -467,6 +492,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     // ---- the usual case: the tile's entries fit the stage
     __shared__ uint16_t st_w[kAggSparseStage];                       // worker of every staged entry
     __shared__ uint32_t s_seen[kAggSparseTile / 32], s_shared[kAggSparseTile / 32];
+    __shared__ uint16_t s_pool[kAggSparseStage];
     // (the run tables are not needed once the entries are staged with their workers, nor is the "seen"
     // bitmap once the shared coordinates are marked: the slot tables take their place)
     static_assert(kAggSparseStage / 2 <= kAggMaxW, "the slot tables fit the run tables");
@@ -483,7 +509,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
     // Most coordinates are sent by a single worker.  Two bitmaps over the tile find the ones that are
     // not: the second entry that sets a coordinate's "seen" bit also sets its "shared" bit.
     for (uint32_t i = tid; i < (uint32_t)(kAggSparseTile / 32); i += kAggThreads) { s_seen[i] = 0; s_shared[i] = 0; }
-    __syncthreads();
+    sync_w();
     bool any_shared = false;
     for (uint32_t q = tid; q < total; q += kAggThreads) {
       const uint32_t local = st_idx[q] - lo;
@@ -492,10 +518,62 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
         if (atomicOr(&s_seen[local >> 5], bit) & bit) { atomicOr(&s_shared[local >> 5], bit); any_shared = true; }
       }
     }
-    clear_wait();                                                     // (the barrier orders the results behind the clearing)
-    any_shared = __syncthreads_or(any_shared);
-    // a sole sender's coordinate: the sum is the value
-    for (uint32_t q = tid; q < total; q += kAggThreads) {
+    any_shared = agg_bar_or<1, kAggThreads>(any_shared);                        // (block-uniform)
+    // Shared coordinates (at most half the stage: each has two entries or more) get consecutive slots
+    // in index order; a counting sort by slot brings every coordinate's entries together, and since
+    // the stage is in worker order, taking a slot's entries by ascending stage position sums them in
+    // worker order -- the same fixed-order double sum as everywhere else.
+    static_assert(kAggSparseTile / 32 == 2 * kAggThreads, "two bitmap words per thread");
+    uint32_t n_slots = 0;
+    auto slot_of = [&](uint32_t local) { return s_slot[local >> 5] + __popc(s_shared[local >> 5] & ((1u << (local & 31u)) - 1u)); };
+    if (any_shared) {
+      for (uint32_t i = tid; i < (uint32_t)(kAggSparseStage / 2); i += kAggThreads) s_cur[i] = 0;
+      {
+        const uint32_t c0 = __popc(s_shared[2 * tid]), c1 = __popc(s_shared[2 * tid + 1]);
+        const uint32_t incl = warp_incl_scan(c0 + c1);
+        if (lane == 31) s_warp[warp] = incl;
+        sync_w();
+        uint32_t woff = 0, all = 0;
+        for (uint32_t x = 0; x < (uint32_t)(kAggThreads / 32); ++x) { if (x < warp) woff += s_warp[x]; all += s_warp[x]; }
+        s_slot[2 * tid] = woff + incl - c0 - c1;
+        s_slot[2 * tid + 1] = woff + incl - c1;
+        n_slots = all;
+        sync_w();
+      }
+      for (uint32_t q = tid; q < total; q += kAggThreads) {            // entries per slot
+        const uint32_t local = st_idx[q] - lo;
+        if (local < kTile && st_idx[q] < d && ((s_shared[local >> 5] >> (local & 31u)) & 1u))
+          atomicAdd(&s_cur[slot_of(local)], 1u);
+      }
+      sync_w();
+      {                                                                 // exclusive prefix over the slots (up to 1024)
+        constexpr int kPer = kAggSparseStage / 2 / kAggThreads;
+        uint32_t c[kPer], sum = 0;
+#pragma unroll
+        for (int u = 0; u < kPer; ++u) { c[u] = s_cur[tid * kPer + u]; sum += c[u]; }
+        const uint32_t incl = warp_incl_scan(sum);
+        sync_w();
+        if (lane == 31) s_warp[warp] = incl;
+        sync_w();
+        uint32_t run = incl - sum;
+        for (uint32_t x = 0; x < warp; ++x) run += s_warp[x];
+#pragma unroll
+        for (int u = 0; u < kPer; ++u) { s_off[tid * kPer + u] = run; s_cur[tid * kPer + u] = 0; run += c[u]; }
+        if (tid == kAggThreads - 1) s_off[kAggSparseStage / 2] = run;
+        sync_w();
+      }
+      for (uint32_t q = tid; q < total; q += kAggThreads) {            // scatter the stage positions
+        const uint32_t local = st_idx[q] - lo;
+        if (local < kTile && st_idx[q] < d && ((s_shared[local >> 5] >> (local & 31u)) & 1u)) {
+          const uint32_t sl = slot_of(local);
+          s_pool[s_off[sl] + atomicAdd(&s_cur[sl], 1u)] = (uint16_t)q;
+        }
+      }
+    }
+    // the results, behind the clearing of the tile
+    sync_w();                                                         // (the pool is complete)
+    tile_cleared(true);
+    for (uint32_t q = tid; q < total; q += kAggThreads) {              // a sole sender's coordinate: the sum is the value
       const uint32_t idx = st_idx[q], local = idx - lo;
       if (local >= kTile || idx >= d) continue;                      // malformed row: ignore
       if (!((s_shared[local >> 5] >> (local & 31u)) & 1u)) {
@@ -503,58 +581,6 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
         dst.store(idx, (float)agg_scaled(v, 1u, sc));
       }
     }
-    if (!any_shared) return;                                          // (block-uniform)
-    for (uint32_t i = tid; i < (uint32_t)(kAggSparseStage / 2); i += kAggThreads) s_cur[i] = 0;
-    // Shared coordinates (at most half the stage: each has two entries or more) get consecutive slots
-    // in index order; a counting sort by slot brings every coordinate's entries together, and since
-    // the stage is in worker order, taking a slot's entries by ascending stage position sums them in
-    // worker order -- the same fixed-order double sum as everywhere else.
-    static_assert(kAggSparseTile / 32 == 2 * kAggThreads, "two bitmap words per thread");
-    uint32_t n_slots;
-    {
-      const uint32_t c0 = __popc(s_shared[2 * tid]), c1 = __popc(s_shared[2 * tid + 1]);
-      const uint32_t incl = warp_incl_scan(c0 + c1);
-      if (lane == 31) s_warp[warp] = incl;
-      __syncthreads();
-      uint32_t woff = 0, all = 0;
-      for (uint32_t x = 0; x < (uint32_t)(kAggThreads / 32); ++x) { if (x < warp) woff += s_warp[x]; all += s_warp[x]; }
-      s_slot[2 * tid] = woff + incl - c0 - c1;
-      s_slot[2 * tid + 1] = woff + incl - c1;
-      n_slots = all;
-      __syncthreads();
-    }
-    if (n_slots == 0) return;                                         // (block-uniform)
-    auto slot_of = [&](uint32_t local) { return s_slot[local >> 5] + __popc(s_shared[local >> 5] & ((1u << (local & 31u)) - 1u)); };
-    for (uint32_t q = tid; q < total; q += kAggThreads) {            // entries per slot
-      const uint32_t local = st_idx[q] - lo;
-      if (local < kTile && st_idx[q] < d && ((s_shared[local >> 5] >> (local & 31u)) & 1u))
-        atomicAdd(&s_cur[slot_of(local)], 1u);
-    }
-    __syncthreads();
-    {                                                                 // exclusive prefix over the slots (up to 1024)
-      constexpr int kPer = kAggSparseStage / 2 / kAggThreads;
-      uint32_t c[kPer], sum = 0;
-#pragma unroll
-      for (int u = 0; u < kPer; ++u) { c[u] = s_cur[tid * kPer + u]; sum += c[u]; }
-      const uint32_t incl = warp_incl_scan(sum);
-      __syncthreads();
-      if (lane == 31) s_warp[warp] = incl;
-      __syncthreads();
-      uint32_t run = incl - sum;
-      for (uint32_t x = 0; x < warp; ++x) run += s_warp[x];
-#pragma unroll
-      for (int u = 0; u < kPer; ++u) { s_off[tid * kPer + u] = run; s_cur[tid * kPer + u] = 0; run += c[u]; }
-      if (tid == kAggThreads - 1) s_off[kAggSparseStage / 2] = run;
-      __syncthreads();
-    }
-    for (uint32_t q = tid; q < total; q += kAggThreads) {            // scatter the stage positions
-      const uint32_t local = st_idx[q] - lo;
-      if (local < kTile && st_idx[q] < d && ((s_shared[local >> 5] >> (local & 31u)) & 1u)) {
-        const uint32_t sl = slot_of(local);
-        s_pool[s_off[sl] + atomicAdd(&s_cur[sl], 1u)] = (uint16_t)q;
-      }
-    }
-    __syncthreads();
     for (uint32_t sl = tid; sl < n_slots; sl += kAggThreads) {       // one thread per shared coordinate
       const uint32_t b = s_off[sl], e = s_off[sl + 1];
       if (e == b) continue;                                           // (only entries of a malformed row)
@@ -575,8 +601,7 @@ __global__ void __launch_bounds__(kAggThreads) k_aggregate_sparse(M msgs, const 
   // ---- a crowded tile (more entries than the stage holds): every entry looks the other workers' runs
   // up in global memory; the entry of the lowest worker that holds a coordinate owns it and sums that
   // coordinate over the workers in ascending order
-  clear_wait();
-  __syncthreads();
+  tile_cleared(true);
   auto idx_at = [&](uint32_t w, uint32_t j) { return msgs.index_in(w, s_beg[w] + j, span_lo); };
   auto val_at = [&](uint32_t w, uint32_t j) { return msgs.value(w, s_beg[w] + j); };
   for (uint32_t q = tid; q < total; q += kAggThreads) {

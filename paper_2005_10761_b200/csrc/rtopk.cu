@@ -695,11 +695,11 @@ int aggregate_launch(rtopk_ctx* ctx, const M& msgs, int64_t d, int32_t W, int64_
     // momentum: the sent coordinates are updated here and marked, the others by a plain pass behind it
     if (velocity) RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_sent, 0, ((size_t)d + 31) / 32 * sizeof(uint32_t), st));
     if (sparse16)
-      k_aggregate_sparse<M, kAggSparseTile><<<ntiles, kAggThreads, 0, st>>>(msgs, own_search ? nullptr : starts, (uint32_t)d,
+      k_aggregate_sparse<M, kAggSparseTile><<<ntiles, kAggSparseThreads, 0, st>>>(msgs, own_search ? nullptr : starts, (uint32_t)d,
                                                                             (uint32_t)W, (uint32_t)k, sc, eta, out, mu,
                                                                             velocity, ctx->d_sent, clear, run_cnt);
     else
-      k_aggregate_sparse<M, kAggTile><<<ntiles, kAggThreads, 0, st>>>(msgs, starts, (uint32_t)d, (uint32_t)W, (uint32_t)k,
+      k_aggregate_sparse<M, kAggTile><<<ntiles, kAggSparseThreads, 0, st>>>(msgs, starts, (uint32_t)d, (uint32_t)W, (uint32_t)k,
                                                                       sc, eta, out, mu, velocity, ctx->d_sent, clear,
                                                                       nullptr);
     ++ctx->launches;
