@@ -4,8 +4,9 @@
 // The streaming pass leaves the candidates of a slice in one dense list: per chunk of 4096 coordinates
 // a run of (index, value) entries in index order, the runs one behind the other in the order in which
 // the chunks were finished, and per chunk where its run starts.  It also leaves the sampled or predicted
-// bracket [tau_lo, tau_hi] of the r-th largest key and, counted while the candidates were written, their
-// histogram over the bracket: 2047 equal buckets (the keys above the bracket are the rest of the list).
+// bracket [tau_lo, tau_hi] of the r-th largest key and, counted while the candidates were written (f32
+// gradients; k_run_hist below otherwise), their histogram over the bracket: 2047 equal buckets (the keys above
+// the bracket are the rest of the list).
 // The bucket that holds the r-th largest key splits the candidates: those above it are members of the
 // top-r set for sure, those below it are not, and the few dozen inside it are decided exactly.  Two
 // grid-wide launches over all slices at once; each walks the LIST in tiles of 2048 entries, eight
@@ -88,6 +89,46 @@ __device__ __forceinline__ void run_pick(const uint32_t* hist, uint32_t need, ui
   __syncthreads();
   D = s[8]; above = s[9];
   __syncthreads();
+}
+
+// The histogram over the bracket where the streaming pass has not counted it (bf16 gradients: that pass is
+// bound by instruction issue there, and the counting cost it more than this launch takes); also clears the
+// chunks' member counts.  The keys above the bracket are not counted: their number is the rest of the list.
+// grid: (blocks per slice, n_slices); a block takes tile after tile of kRunThreads * kHistPer candidates
+constexpr int kHistPer = 8;
+__global__ void __launch_bounds__(kRunThreads) k_run_hist(Launch L) {
+  __shared__ uint32_t hist[kBins];
+  const uint32_t sl = blockIdx.y, tid = threadIdx.x;
+  const Slice S = L.s.slices[sl];
+  const uint32_t n_cand = L.s.cursor[sl];
+  const uint32_t tau_lo = L.s.state[sl].tau_lo, tau_hi = max(tau_lo, L.s.state[sl].tau_hi);
+  if (S.r == S.len) return;
+  if (n_cand < S.r || n_cand > S.cand_cap) return;               // the bracket missed: left to k_finish
+  {
+    uint32_t* cm = L.s.chunk_pre + S.chunk_begin;                  // members per chunk: counted by k_run_count
+    const uint32_t nchunks = slice_chunks(S);
+    for (uint32_t c = blockIdx.x * kRunThreads + tid; c < nchunks; c += gridDim.x * kRunThreads) cm[c] = 0;
+  }
+  constexpr uint32_t kTile = kRunThreads * kHistPer;
+  const uint32_t nblocks = min(gridDim.x, (n_cand + kTile - 1u) / kTile);
+  if (blockIdx.x >= nblocks) return;
+  const uint32_t sh = bracket_shift(tau_lo, tau_hi);
+  for (uint32_t b = tid; b < (uint32_t)kBins; b += kRunThreads) hist[b] = 0;
+  __syncthreads();
+  const float* rv = L.s.raw_val + S.cand_off;
+  for (uint32_t i0 = blockIdx.x * kTile; i0 < n_cand; i0 += gridDim.x * kTile) {
+    float v[kHistPer];
+#pragma unroll
+    for (int u = 0; u < kHistPer; ++u) { const uint32_t i = i0 + u * kRunThreads + tid; v[u] = i < n_cand ? rv[i] : 0.f; }
+#pragma unroll
+    for (int u = 0; u < kHistPer; ++u) {
+      const uint32_t key = mag_key(v[u]);
+      if (i0 + u * kRunThreads + tid < n_cand && key >= tau_lo && key <= tau_hi) atomicAdd(&hist[(key - tau_lo) >> sh], 1u);
+    }
+  }
+  __syncthreads();
+  uint32_t* gh = L.s.hist + (size_t)sl * kBins;
+  for (uint32_t b = tid; b < (uint32_t)kBins; b += kRunThreads) { const uint32_t c = hist[b]; if (c) atomicAdd(gh + b, c); }
 }
 
 // Eight consecutive entries of a slice's candidate list, starting at entry i0 (a multiple of 8; the

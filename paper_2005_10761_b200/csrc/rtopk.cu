@@ -300,7 +300,7 @@ int launch_select(rtopk_ctx* ctx, const Plan& P, const Launch& L, cudaStream_t s
     const uint32_t uniform = P.uniform ? per : 0u;
     const int blocks = ctx->stream_blocks[sizeof(GradT) == 4 ? 0 : 1];
     if (ctx->test_giveup) k_stream<GradT, true, false><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
-    else if (late.hist) k_stream<GradT, false, true><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
+    else if (sizeof(GradT) == 4 && late.hist) k_stream<float, false, true><<<blocks, kStreamThreads, sizeof(StreamSmem<float>), st>>>(L, P.n_chunks, uniform);
     else k_stream<GradT, false, false><<<blocks, kStreamThreads, sizeof(StreamSmem<GradT>), st>>>(L, P.n_chunks, uniform);
     ++ctx->launches;
     if (late.on) {
@@ -499,7 +499,9 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
     RTOPK_CUDA(ctx, cudaMemsetAsync(ctx->d_zero + early_bytes, 0, zbytes - early_bytes, st));
   }
   cudaEvent_t join = forked ? ctx->ev_join : nullptr;
-  const LateSide late = {sampler_late, from_runs};
+  // (f32 gradients: the streaming pass counts the candidates' histogram itself; bf16: k_run_hist does)
+  const bool hist_in_stream = from_runs && grad_dtype == RTOPK_F32 && !ctx->test_giveup;
+  const LateSide late = {sampler_late, hist_in_stream};
   rc = grad_dtype == RTOPK_F32 ? launch_select<float>(ctx, P, L, st, join, late)
                                : launch_select<__nv_bfloat16>(ctx, P, L, st, join, late);
   if (rc) return rc;
@@ -509,6 +511,12 @@ int sparsify_impl(rtopk_ctx* ctx, const void* grad, int grad_dtype, int64_t ld_g
   if (from_runs) {
     // the usual case is finished straight from the streaming pass's runs, all slices side by side; what
     // these kernels leave (a missed bracket, heavy ties) is flagged for k_finish
+    if (!hist_in_stream) {
+      const uint32_t per_slice = std::max<uint32_t>(1u, ((uint32_t)ctx->sms * 8u + L.n_slices - 1u) / L.n_slices);
+      const uint32_t tiles = (P.cap_max + kRunThreads * kHistPer - 1) / (kRunThreads * kHistPer);
+      k_run_hist<<<dim3(std::min(tiles, per_slice), L.n_slices), kRunThreads, 0, st>>>(L);
+      ++ctx->launches;
+    }
     const uint32_t per_slice_run = std::max<uint32_t>(1u, ((uint32_t)ctx->sms * 4u + L.n_slices - 1u) / L.n_slices);
     const dim3 rgrid(std::min((P.cap_max + kRunTile - 1) / (uint32_t)kRunTile, per_slice_run), L.n_slices);
     k_run_count<<<rgrid, kRunThreads, 0, st>>>(L);
@@ -867,9 +875,8 @@ int rtopk_create(rtopk_ctx** out, int device, int64_t d_max, int32_t W_max, int6
     if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<float, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<float>));
     if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<__nv_bfloat16, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<__nv_bfloat16>));
     if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<__nv_bfloat16, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<__nv_bfloat16>));
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_stream<__nv_bfloat16, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(StreamSmem<__nv_bfloat16>));
     if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_f32, k_stream<float, false, true>, kStreamThreads, sizeof(StreamSmem<float>));
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_bf16, k_stream<__nv_bfloat16, false, true>, kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>));
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_bf16, k_stream<__nv_bfloat16, false, false>, kStreamThreads, sizeof(StreamSmem<__nv_bfloat16>));
     if (e == cudaSuccess && (per_f32 < 1 || per_bf16 < 1)) e = cudaErrorLaunchOutOfResources;
     ctx->sms = sms;
     ctx->stream_blocks[0] = sms * per_f32;

@@ -125,7 +125,7 @@ template <> struct SmemGrad<__nv_bfloat16> {
 // treat their first wait as run out and its producer waits only briefly for them, so every block takes the
 // exit a real expiry would take -- error flag, a last bounded wait for the bulk copies still on their way
 // into the block's shared memory, return -- while all copies do arrive.
-// HIST: the call is finished by the run kernels (finish.cuh).  Every candidate inside the bracket
+// HIST (f32 gradients): the call is finished by the run kernels (finish.cuh).  Every candidate inside the bracket
 // [tau_lo, tau_hi] is then also counted in the slice's histogram over the bracket (one reduction into
 // global memory per such candidate: a third of the candidates, 0.4 % of the coordinates; the keys above
 // the bracket need no counting, their number is the rest of the list), and the chunk's member count is
