@@ -269,11 +269,12 @@ class Round:
         self.out = torch.zeros(wl.round_up(self.d, 4), dtype=torch.float32, device=dev)
         self.cnt = torch.zeros(self.W, dtype=torch.int32, device=dev)
         self.ones = torch.zeros(self.W, dtype=torch.int32, device=dev)
-        if world > 1:
+        self.sharded = world > 1 or bool(getattr(args, "exchange_path", False))
+        if self.sharded:
             if self.seg:
                 raise SystemExit("the sharded run covers the plain (whole-vector) workloads")
             from paper_2005_10761_b200 import sharded
-            self.exchange = sharded.Exchange(self.W_total, self.K, world, rank, dev)
+            self.exchange = sharded.Exchange(self.W_total, self.K, world, rank, dev, always_collective=True)
         self.t_next = 0
 
     @property
@@ -283,7 +284,7 @@ class Round:
     def step(self, t: int):
         cfg, ctx, args = self.cfg, self.ctx, self.args
         g = self.grads[t % self.n_batches]
-        if self.world == 1:
+        if not self.sharded:
             if self.seg:
                 ctx.step_segmented(g, self.residual, self.d, cfg.seg_off, cfg.seg_r, cfg.seg_k, cfg.seed, t,
                                    self.idx, self.val, self.out)
@@ -309,7 +310,7 @@ class Round:
     def sync_all(self):
         import torch
         torch.cuda.synchronize()
-        if self.world > 1:
+        if self.sharded:
             import torch.distributed as dist
             dist.barrier()
             torch.cuda.synchronize()
@@ -325,7 +326,7 @@ class Round:
         e1.record()
         self.sync_all()
         ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=self.dev)
-        if self.world > 1:
+        if self.sharded:
             import torch.distributed as dist
             dist.all_reduce(ms, op=dist.ReduceOp.MAX)
         return float(ms.item())
@@ -339,7 +340,7 @@ class Round:
         for _ in range(warmup):
             self.step(self.t_next); self.t_next += 1
         self.sync_all()
-        graphed = graph and self.world == 1 and not self.thr   # (the threshold call re-uploads its slice table)
+        graphed = graph and not self.sharded and not self.thr   # (the threshold call re-uploads its slice table)
         per_region, launches = [], 0
         if graphed:
             ctx.set_option(B.OPT_DEVICE_STEP, 1)
@@ -415,10 +416,12 @@ class Round:
         self.ctx.close()
 
 
-def sweep_point(name, args, dev, peak, grads=None, steps=10, warmup=5, repeats=3, select_path=None, cold_l2=False):
+def sweep_point(name, args, dev, peak, grads=None, steps=10, warmup=5, repeats=3, select_path=None, cold_l2=False,
+                workers=0):
     """One short run of another configuration: the metric "vs d, W, r, k"."""
     import torch
-    cfg = pick_workload(name)
+    cfg = pick_workload(name, workers=workers)
+    name = cfg.name
     a = argparse.Namespace(**vars(args))
     a.apply, a.threshold = False, None
     a.select_path = select_path or "sampled"
@@ -525,6 +528,9 @@ def run_sweep(args, dev, peak):
             out.append(sweep_point(name, args, dev, peak, steps=20, warmup=10))
     for name in ("c2", "c3_f32"):
         out.append(sweep_point(name, args, dev, peak, steps=10, warmup=3, select_path="exact"))
+    # one worker row: what each GPU of a job with one worker per GPU runs before the all-gather
+    for name in ("c2", "c3_f32", "c3_bf16", "c4"):
+        out.append(sweep_point(name, args, dev, peak, steps=50, warmup=10, workers=1))
     for name in ("c2", "c3_f32"):
         out.append(message_and_master_point(name, args, dev))
     # c5: d = 2^28; one gradient batch of the largest row count is generated once and shared (every
@@ -593,6 +599,9 @@ def main():
                     help="1 (default): the timed rounds are replays of a CUDA graph that holds one round per resident "
                          "gradient batch (the round counter lives on the device, RTOPK_OPT_DEVICE_STEP, so every "
                          "replayed round still draws its own subset); 1 GPU")
+    ap.add_argument("--exchange-path", action="store_true",
+                    help="one GPU under torch.distributed.run with one rank: run the calls of the sharded job "
+                         "(messages as pairs, the NCCL all-gather, in-place aggregation) instead of rtopk_step")
     ap.add_argument("--reuse-threshold", type=int, default=1, choices=[0, 1],
                     help="1 (default): the rounds of the loop predict their first threshold from the previous "
                          "rounds (RTOPK_OPT_REUSE_THRESHOLD; results are the same); 0: every round samples")
@@ -616,17 +625,20 @@ def main():
         raise SystemExit(f"rank {rank}: no CUDA device {local} ({torch.cuda.device_count()} visible)")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
+    if args.exchange_path and "WORLD_SIZE" not in os.environ:
+        raise SystemExit("--exchange-path needs a process group: start bench.py under torch.distributed.run")
+    grouped = world > 1 or args.exchange_path
+    if grouped:
         dist.init_process_group("nccl", device_id=dev)
     if rank == 0:
         build.build()
-    if world > 1:
+    if grouped:
         dist.barrier()
 
     cfg = pick_workload(args.workload, args.scale_d, args.workers)
     seg = cfg.seg_off is not None
     thr = args.threshold is not None
-    if (args.apply or thr) and (seg or world > 1):
+    if (args.apply or thr) and (seg or grouped):
         raise SystemExit("--apply and --threshold cover the plain single-GPU workloads")
     if args.select_path == "exact" and thr:
         raise SystemExit("--threshold runs on the sampled path only")
@@ -659,7 +671,7 @@ def main():
 
     # end to end: host gradient in, host messages + update out, through rtopk_step_host
     e2e = None
-    if not args.no_e2e and world == 1 and not seg and not args.apply and not thr:
+    if not args.no_e2e and not grouped and not seg and not args.apply and not thr:
         h_grad = rd.grads[0].cpu().pin_memory()
         h_idx = torch.zeros((W, K), dtype=torch.int32).pin_memory()
         h_val = torch.zeros((W, K), dtype=torch.float32).pin_memory()
@@ -681,7 +693,7 @@ def main():
     torch.cuda.empty_cache()
 
     sweep = None
-    if args.sweep and world == 1 and rank == 0 and not (args.apply or thr or args.scale_d or args.workers):
+    if args.sweep and not grouped and rank == 0 and not (args.apply or thr or args.scale_d or args.workers):
         sweep = run_sweep(args, dev, peak)
 
     cpu = None
@@ -706,7 +718,7 @@ def main():
             "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": config_dict(cfg, args, world),
-            "launch": launch_mode if world == 1 else launch_mode + "; per round one NCCL all-gather of W*k 8-byte pairs",
+            "launch": launch_mode if not grouped else launch_mode + "; per round one NCCL all-gather of W*k 8-byte pairs",
             "elements_per_s": W * world * d / (ms_per_step * 1e-3),
             "step_roofline_frac": step_frac, "step_roofline_frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS if world == 1 else None,
             "step_algorithmic_bytes": step_bytes,
@@ -715,7 +727,7 @@ def main():
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": gpu_launches,
             "clocks": clocks, "sweep": sweep,
         }))
-    if world > 1:
+    if grouped:
         dist.destroy_process_group()
 
 

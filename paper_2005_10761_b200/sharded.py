@@ -39,12 +39,15 @@ class Exchange:
     """The buffers of the one all-gather, allocated once: ``send`` [c, k] pairs of this rank (rows beyond
     its shard stay zero and are never read), ``recv`` [world * c, k] pairs of everybody."""
 
-    def __init__(self, W_total: int, k: int, world: int, rank: int, device, group=None):
+    def __init__(self, W_total: int, k: int, world: int, rank: int, device, group=None, always_collective=False):
+        """``always_collective``: issue the all-gather even in a group of one rank (it then copies ``send``
+        to ``recv``), so that a single process runs exactly the calls of a sharded job."""
         self.W_total, self.k, self.world, self.rank, self.group = W_total, k, world, rank, group
         self.c = shard_block(W_total, world)
         self.begin, self.rows = shard_rows(W_total, world, rank)
+        self.collective = world > 1 or always_collective
         self.send = torch.zeros((self.c, k), dtype=torch.int64, device=device)
-        self.recv = self.send if world == 1 else torch.zeros((world * self.c, k), dtype=torch.int64, device=device)
+        self.recv = torch.zeros((world * self.c, k), dtype=torch.int64, device=device) if self.collective else self.send
 
     def local_pairs(self) -> torch.Tensor:
         """Where this rank's sparsify call writes its messages: [rows, k] pairs."""
@@ -52,7 +55,7 @@ class Exchange:
 
     def gather(self) -> torch.Tensor:
         """All ranks' messages, [W_total, k] pairs in global worker order (a view of ``recv``)."""
-        if self.world > 1:
+        if self.collective:
             dist.all_gather_into_tensor(self.recv, self.send, group=self.group)
         return self.recv[: self.W_total]
 

@@ -106,8 +106,10 @@ def configs() -> dict:
 
 
 def scaled(cfg: Workload, d: int, W: Optional[int] = None, name: Optional[str] = None) -> Workload:
-    """The same recipe and ratios at another length (for small parity cases)."""
-    assert cfg.seg_off is None
+    """The same recipe and ratios at another length (for small parity cases), or with another row count."""
+    if cfg.seg_off is not None:                       # per-tensor sizes are tied to the length: only the rows change
+        assert d == cfg.d
+        return replace(cfg, W=W or cfg.W, name=name or cfg.name)
     r = max(1, cfg.r * d // cfg.d)
     k = max(1, min(r, cfg.k * d // cfg.d))
     return replace(cfg, d=d, W=W or cfg.W, r=r, k=k, name=name or f"{cfg.name}_d{d}")
