@@ -275,20 +275,20 @@ __global__ void __launch_bounds__(kStreamThreads, 3) k_stream(Launch L, uint32_t
       uint32_t* gh = L.s.hist + (size_t)cur_slice * kBins;
 #pragma unroll
       for (int it = 0; it < kIter; ++it) {
-        const uint32_t bits = (maskA >> (it * 4)) & 0xFu;
-        if (bits) {
-          uint32_t pos = before + ((exLaneA >> (it * 8)) & 0xFFu);
-          const uint32_t e = e_w + it * 128u + lane * 4u;
-#pragma unroll
-          for (int j = 0; j < 4; ++j)
-            if ((bits >> j) & 1u) {
-              if (pos < S.cand_cap) { st_hint(cidx + pos, e + j - head, keep); st_hint(reinterpret_cast<uint32_t*>(cval) + pos, __float_as_uint(a[it][j]), keep); }
-              ++pos;
-              if (HIST) {
-                const uint32_t key = mag_key(a[it][j]);
-                if (key <= tau_hi) atomicAdd(gh + ((key - tau) >> sh), 1u);
-              }
-            }
+        uint32_t bits = (maskA >> (it * 4)) & 0xFu;
+        uint32_t pos = before + ((exLaneA >> (it * 8)) & 0xFFu);
+        const uint32_t e = e_w + it * 128u + lane * 4u - head;
+        while (bits) {                                             // (a candidate or two per warp and vector)
+          const uint32_t j = (uint32_t)__ffs(bits) - 1u;
+          bits &= bits - 1u;
+          const float lo2 = j & 1u ? a[it][1] : a[it][0], hi2 = j & 1u ? a[it][3] : a[it][2];
+          const uint32_t vb = __float_as_uint(j & 2u ? hi2 : lo2);
+          if (pos < S.cand_cap) { st_hint(cidx + pos, e + j, keep); st_hint(reinterpret_cast<uint32_t*>(cval) + pos, vb, keep); }
+          ++pos;
+          if (HIST) {
+            const uint32_t key = vb & 0x7FFFFFFFu;
+            if (key <= tau_hi) atomicAdd(gh + ((key - tau) >> sh), 1u);
+          }
         }
         before += (totA >> (it * 8)) & 0xFFu;
       }
