@@ -73,3 +73,21 @@ def test_warmup_sizes_host_function_matches_the_oracle():
     import pytest
     with pytest.raises(rt.RTopKError):
         rt.warmup_sizes(100, 4, 0.001, 0.01, 5, 0)
+
+
+def test_workload_recipes_scale_by_length_and_by_rows():
+    """The seeded input recipes: another length keeps the ratios r / d and k / r (floor, at least 1), another
+    row count keeps everything else; the per-tensor workload is tied to its tensor sizes, so only its rows
+    may change."""
+    from paper_2005_10761_b200 import workloads as wl
+    cfgs = wl.configs()
+    c3 = cfgs["c3_f32"]
+    s = wl.scaled(c3, d=1_000_000, W=3)
+    assert (s.d, s.W, s.r, s.k) == (1_000_000, 3, c3.r * 1_000_000 // c3.d, c3.k * 1_000_000 // c3.d)
+    assert wl.scaled(c3, d=10).r == 1 and wl.scaled(c3, d=10).k == 1
+    c4 = cfgs["c4"]
+    one = wl.scaled(c4, d=c4.d, W=1, name="c4_W1")
+    assert one.W == 1 and one.name == "c4_W1"
+    assert (one.seg_off, one.seg_r, one.seg_k, one.d) == (c4.seg_off, c4.seg_r, c4.seg_k, c4.d)
+    with pytest.raises(AssertionError):
+        wl.scaled(c4, d=c4.d // 2)
