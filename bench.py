@@ -687,6 +687,28 @@ def main():
         e2e = {"value": W * d * gsz / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms,
                "h2d_bytes_per_step": W * rd.ld * gsz, "d2h_bytes_per_step": 8 * W * K + 4 * d}
         del h_grad, h_idx, h_val, h_out
+    elif not args.no_e2e and grouped and not seg:
+        # the sharded job end to end: every rank uploads its rows' gradients from pinned host memory, runs the
+        # round (sparsify into pairs, the all-gather, aggregation) and downloads the dense update
+        h_grad = rd.grads[0].cpu().pin_memory()
+        g_dev = torch.empty_like(rd.grads[0])
+        h_out = torch.zeros(rd.out.numel(), dtype=torch.float32).pin_memory()
+        kept = rd.grads
+
+        def host_step(t: int):
+            g_dev.copy_(h_grad, non_blocking=True)
+            rd.step(t)
+            h_out.copy_(rd.out, non_blocking=True)
+        rd.grads, rd.n_batches = [g_dev], 1
+        for _ in range(3):
+            host_step(rd.t_next); rd.t_next += 1
+        n_e2e = max(3, min(args.steps, 10))
+        ms = rd.timed(host_step, rd.t_next, n_e2e) / n_e2e
+        rd.t_next += n_e2e
+        rd.grads, rd.n_batches = kept, len(kept)
+        e2e = {"value": rd.W_total * d * gsz / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms,
+               "h2d_bytes_per_step": W * rd.ld * gsz * world, "d2h_bytes_per_step": 4 * rd.out.numel() * world}
+        del h_grad, g_dev, h_out
     rd.ctx.poll_status()
     rd.close()
     del rd
