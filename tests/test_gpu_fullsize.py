@@ -281,3 +281,47 @@ def test_c3_message_formats_and_master_updates_at_full_size(lib):
     assert np.array_equal(w.cpu().numpy()[:d].view(np.uint32), oracle.apply_update(idx_h, val_h, d, 0.05, w0).view(np.uint32))
     ctx.poll_status()
     ctx.close()
+
+
+def test_eight_rank_job_of_c3_run_rank_by_rank_on_one_gpu(lib):
+    # The sharded job bench.py runs with --gpus 8 (16 rows of c3_f32 per GPU, 128 workers), as one process
+    # over all ranks' data: every rank's rows are sparsified in turn with that rank's worker_base into its
+    # block of the gathered pair buffer (what the all-gather leaves on every GPU), then the buffer is
+    # aggregated in place.  Two sampled workers per rank position against the oracle with their global
+    # worker ids, the average of all 128 messages against the oracle's, bit for bit.
+    import dataclasses
+    from paper_2005_10761_b200 import sharded
+    base = wl.configs()["c3_f32"]
+    world, c = 8, base.W
+    W_total = world * c
+    if _free_bytes() < 12e9:
+        pytest.skip("not enough free device memory")
+    cfg = dataclasses.replace(base, W=W_total)
+    d, r, k = cfg.d, cfg.r, cfg.k
+    ctx = lib.RTopK(d_max=d, W_max=W_total, r_max=r, k_max=k)
+    pairs_all = torch.zeros((W_total, k), dtype=torch.int64, device="cuda")
+    sampled = {0: [3], 3: [0, 15], 7: [9]}             # rank -> local rows followed by the oracle
+    for p in range(world):
+        begin, rows = sharded.shard_rows(W_total, world, p)
+        assert (begin, rows) == (p * c, c)
+        g = wl.gradient(cfg, 0, "cuda", workers=range(begin, begin + rows))
+        m = wl.zero_residual(base, "cuda")
+        ctx.sparsify_pairs(g, m, d, r, k, cfg.seed, 0, pairs_all[begin:begin + rows], worker_base=begin)
+        ctx.poll_status()
+        idx_p, val_p = sharded.unpack_pairs(pairs_all[begin:begin + rows])
+        for w in sampled.get(p, []):
+            m_or = np.zeros((1, cfg.ld), dtype=np.float32)
+            o_idx, o_val = oracle.sparsify(_host_grad(cfg, g[w:w + 1]), m_or, d, r, k, cfg.seed, 0, worker_base=begin + w)
+            assert np.array_equal(idx_p[w].cpu().numpy().view(np.uint32), o_idx[0]), f"rank {p} row {w}: indices"
+            assert np.array_equal(val_p[w].cpu().numpy().view(np.uint32), o_val[0].view(np.uint32)), f"rank {p} row {w}: values"
+            assert np.array_equal(m[w].cpu().numpy().view(np.uint32), m_or[0].view(np.uint32)), f"rank {p} row {w}: residual"
+        del g, m
+    out = torch.empty(wl.round_up(d, 4), dtype=torch.float32, device="cuda")
+    ctx.aggregate_pairs(pairs_all, d, out)
+    ctx.poll_status()
+    idx_all, val_all = sharded.unpack_pairs(pairs_all)
+    idx_h, val_h = idx_all.cpu().numpy().view(np.uint32), val_all.cpu().numpy()
+    assert bool((idx_h[:, 1:] > idx_h[:, :-1]).all()) and int(idx_h.max()) < d
+    o64, o32 = oracle.aggregate(idx_h, val_h, d)
+    assert np.array_equal(out.cpu().numpy()[:d].view(np.uint32), o32.view(np.uint32))
+    ctx.close()
