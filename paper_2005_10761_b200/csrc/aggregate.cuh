@@ -384,7 +384,7 @@ constexpr int kAggSparseThreads = kAggThreads + 32;                 // eight wor
 // TILE: output coordinates per block: kAggSparseTile for sparse messages, kAggTile where a tile of that size
 // would hold more entries than the stage (the bitmaps and slot tables are laid out for the larger one).
 template <typename M, int TILE>
-__global__ void __launch_bounds__(kAggSparseThreads) k_aggregate_sparse(M msgs, const uint32_t* __restrict__ starts, uint32_t d,
+__global__ void __launch_bounds__(kAggSparseThreads, 5) k_aggregate_sparse(M msgs, const uint32_t* __restrict__ starts, uint32_t d,
                                                                   uint32_t W, uint32_t K, AggScale sc,
                                                                   float eta, float* __restrict__ out, float mu,
                                                                   float* __restrict__ velocity, uint32_t* __restrict__ sent,
@@ -481,18 +481,21 @@ __global__ void __launch_bounds__(kAggSparseThreads) k_aggregate_sparse(M msgs, 
   const uint32_t total = s_carry;
   if (total == 0) { tile_cleared(false); return; }
   if (tid == 0) s_pre[W] = total;
-  const bool staged = total <= (uint32_t)kAggSparseStage;
   sync_w();
   auto worker_of = [&](uint32_t q) {                 // last worker with s_pre[w] <= q
     uint32_t a = 0, b = W;
     while (b - a > 1) { const uint32_t mid = (a + b) >> 1; if (s_pre[mid] <= q) a = mid; else b = mid; }
     return a;
   };
-  if (staged) {
-    // ---- the usual case: the tile's entries fit the stage
-    __shared__ uint16_t st_w[kAggSparseStage];                       // worker of every staged entry
-    __shared__ uint32_t s_seen[kAggSparseTile / 32], s_shared[kAggSparseTile / 32];
-    __shared__ uint16_t s_pool[kAggSparseStage];
+  __shared__ uint16_t st_w[kAggSparseStage];                         // worker of every staged entry
+  __shared__ uint32_t s_seen[kAggSparseTile / 32], s_shared[kAggSparseTile / 32];
+  __shared__ uint16_t s_pool[kAggSparseStage];
+  bool cleared = false;                                               // (block-uniform among the working warps)
+  auto results_may_follow = [&]() { if (!cleared) { tile_cleared(true); cleared = true; } };
+  // The entries with coordinates in [lo, lo + kTile) -- the tile, or a part of a crowded tile -- whose runs
+  // s_beg / s_pre describe, `total` of them, at most the stage.
+  auto staged_range = [&](const uint32_t lo, const uint32_t kTile, const uint32_t total) {
+    // ---- the usual case: the entries fit the stage
     // (the run tables are not needed once the entries are staged with their workers, nor is the "seen"
     // bitmap once the shared coordinates are marked: the slot tables take their place)
     static_assert(kAggSparseStage / 2 <= kAggMaxW, "the slot tables fit the run tables");
@@ -572,7 +575,7 @@ __global__ void __launch_bounds__(kAggSparseThreads) k_aggregate_sparse(M msgs, 
     }
     // the results, behind the clearing of the tile
     sync_w();                                                         // (the pool is complete)
-    tile_cleared(true);
+    results_may_follow();
     for (uint32_t q = tid; q < total; q += kAggThreads) {              // a sole sender's coordinate: the sum is the value
       const uint32_t idx = st_idx[q], local = idx - lo;
       if (local >= kTile || idx >= d) continue;                      // malformed row: ignore
@@ -596,14 +599,14 @@ __global__ void __launch_bounds__(kAggSparseThreads) k_aggregate_sparse(M msgs, 
       }
       dst.store(idx, (float)agg_scaled(sum, e - b, sc));
     }
-    return;
-  }
-  // ---- a crowded tile (more entries than the stage holds): every entry looks the other workers' runs
-  // up in global memory; the entry of the lowest worker that holds a coordinate owns it and sums that
-  // coordinate over the workers in ascending order
-  tile_cleared(true);
+  };
+  // ---- more entries than the stage holds, in a range that cannot be split further: every entry looks the
+  // other workers' runs up in global memory; the entry of the lowest worker that holds a coordinate owns it
+  // and sums that coordinate over the workers in ascending order
   auto idx_at = [&](uint32_t w, uint32_t j) { return msgs.index_in(w, s_beg[w] + j, span_lo); };
   auto val_at = [&](uint32_t w, uint32_t j) { return msgs.value(w, s_beg[w] + j); };
+  auto searched_range = [&](const uint32_t lo, const uint32_t kTile, const uint32_t total) {
+  results_may_follow();
   for (uint32_t q = tid; q < total; q += kAggThreads) {
     const uint32_t w = worker_of(q);
     const uint32_t idx = idx_at(w, q - s_pre[w]);
@@ -626,6 +629,66 @@ __global__ void __launch_bounds__(kAggSparseThreads) k_aggregate_sparse(M msgs, 
       dst.store(idx, (float)agg_scaled(sum, senders, sc));
     }
   }
+  };
+  if (total <= (uint32_t)kAggSparseStage) { staged_range(lo, kTile, total); return; }
+  // ---- a crowded tile (messages that concentrate on a part of the vector): the tile is taken in equal parts
+  // small enough that a part's entries are expected to fill half the stage; a thread keeps the tile's runs of
+  // its workers and finds every part's end in them by binary search (the start is the last part's end)
+  constexpr int kMine = kAggMaxW / kAggThreads;
+  uint32_t t_beg[kMine], t_cnt[kMine], t_cur[kMine];
+#pragma unroll
+  for (int i = 0; i < kMine; ++i) {
+    const uint32_t w = (uint32_t)i * kAggThreads + tid;
+    t_beg[i] = w < W ? s_beg[w] : 0u;
+    t_cnt[i] = w < W ? s_pre[w + 1] - s_pre[w] : 0u;
+    t_cur[i] = 0;
+  }
+  uint32_t parts = 2;
+  while (parts < kTile / 32u && total / parts > (uint32_t)(kAggSparseStage / 2)) parts *= 2;
+  const uint32_t part_len = kTile / parts;
+  sync_w();
+  for (uint32_t p = 0; p < parts; ++p) {
+    const uint32_t p_lo = lo + p * part_len;
+    const bool last_part = p + 1 == parts;
+    if (tid == 0) s_carry = 0;
+    sync_w();
+#pragma unroll
+    for (int i = 0; i < kMine; ++i) {
+      if ((uint32_t)i * kAggThreads >= W) break;                        // (block-uniform)
+      const uint32_t w = (uint32_t)i * kAggThreads + tid;
+      uint32_t cnt = 0;
+      if (w < W) {
+        uint32_t a = t_cur[i], b = t_cnt[i];
+        if (!last_part) {
+          const uint32_t end = p_lo + part_len;                         // first entry of the run at or above it
+          while (a < b) { const uint32_t mid = (a + b) >> 1; if (msgs.index_in(w, t_beg[i] + mid, span_lo) < end) a = mid + 1; else b = mid; }
+        } else {
+          a = b;
+        }
+        s_beg[w] = t_beg[i] + t_cur[i];
+        cnt = a - t_cur[i];
+        t_cur[i] = a;
+      }
+      const uint32_t incl = warp_incl_scan(cnt);
+      if (lane == 31) s_warp[warp] = incl;
+      sync_w();
+      uint32_t woff = s_carry;
+      for (uint32_t x = 0; x < warp; ++x) woff += s_warp[x];
+      if (w < W) s_pre[w] = woff + incl - cnt;
+      sync_w();
+      if (tid == kAggThreads - 1) s_carry = woff + incl;
+      sync_w();
+    }
+    const uint32_t part_total = s_carry;
+    if (tid == 0) s_pre[W] = part_total;
+    sync_w();
+    if (part_total != 0) {
+      if (part_total <= (uint32_t)kAggSparseStage) staged_range(p_lo, part_len, part_total);
+      else searched_range(p_lo, part_len, part_total);
+    }
+    sync_w();                                                           // (the run tables are rebuilt for the next part)
+  }
+  if (!cleared) tile_cleared(false);
 }
 
 }  // namespace rtopk

@@ -300,6 +300,24 @@ def test_aggregate_sparse_path_many_workers_and_crowded_tiles(lib):
     d, W, k = 1_000_000, 5, 40                         # runs that end exactly at tile borders
     edge = np.sort(np.concatenate([np.arange(16_380, 16_400), np.arange(32_758, 32_778)]))
     cases.append((d, np.stack([edge] * W)))
+    # Messages that concentrate on a part of the vector: tiles with several times the entries the stage holds,
+    # taken in parts.  (a) 80 % of every row inside 20000 coordinates, the rest anywhere; (b) a tile border in the
+    # middle of the hot range, and rows that differ in how much they send there; (c) 200 workers that all send
+    # the same 96 neighbouring coordinates: no part of 32 coordinates fits the stage, the searched path runs.
+    d, W, k = 2_000_000, 12, 6000
+    hot = [np.sort(np.concatenate([rng.choice(20_000, 4800, replace=False),
+                                   20_000 + rng.choice(d - 20_000, 1200, replace=False)])) for _ in range(W)]
+    cases.append((d, np.stack(hot)))
+    d, W, k = 1_500_000, 9, 5000
+    rows = []
+    for w in range(W):
+        n_hot = 500 * w + 500
+        rows.append(np.sort(np.concatenate([10_000 + rng.choice(12_000, n_hot, replace=False),
+                                            30_000 + rng.choice(d - 30_000, k - n_hot, replace=False)])))
+    cases.append((d, np.stack(rows)))
+    d, W, k = 400_000, 200, 100
+    same = np.concatenate([np.arange(50_000, 50_096), np.array([123_456, 200_000, 300_001, 399_999])])
+    cases.append((d, np.stack([same] * W)))
     for d, idx in cases:
         idx = idx.astype(np.uint32)
         W, k = idx.shape
