@@ -844,7 +844,11 @@ __global__ void __launch_bounds__(kFinishThreads) k_finish(Launch L) {
       TauHistory h = L.s.history[sl];
       const uint32_t pred = st->pred;
       if (pred != 0 && (st->flags & FLAG_FELL_BACK)) {        // the predicted bracket missed: sample next time
-        h.err = fminf(fmaxf(2.0f * h.err, 0.05f), 0.2f);
+        // A bracket that began above the threshold (too few candidates) was too narrow: the next ones are
+        // wider.  One that let more candidates through than the list holds reached too far down: on data
+        // with a steep tail (a Gaussian bulk) a wider bracket would overflow again, so the next ones are narrower.
+        if (st->n_cand_first > S.cand_cap) h.err = fmaxf(0.5f * h.err, 0.002f);
+        else h.err = fminf(fmaxf(2.0f * h.err, 0.05f), 0.2f);
         h.tau1 = tau; h.tau2 = 0; h.valid = 0;
       } else {
         if (pred != 0) {
