@@ -1166,3 +1166,39 @@ def test_exact_selection_inside_the_finishing_cluster(lib, bf16):
         fell.append(sum(ctx.stats(w)["used_fallback"] for w in range(W)))
     assert max(fell) == W                      # in some round every slice took the exact path
     ctx.close()
+
+
+def test_reused_thresholds_settle_on_a_gaussian_gradient(lib):
+    # A plain Gaussian bulk has a steep tail: a predicted bracket at its widest lets about three times r
+    # candidates through and overflows the list.  Such a miss has to narrow the next brackets (widening them
+    # made every third round miss for ever).  Thirty rounds with a fresh gradient each, residual carried: the
+    # brackets of nearly all rounds are predicted and at most three of the sixty slices-rounds are repaired.
+    from paper_2005_10761_b200 import binding as B
+    d, W = 4_000_000, 2
+    r, k = d // 100, d // 1000
+    ctx = _ctx(lib, d, W, r, k)
+    ctx.set_option(B.OPT_REUSE_THRESHOLD, 1)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(11)
+    m = torch.zeros((W, d), device="cuda")
+    idx = torch.zeros((W, k), dtype=torch.int32, device="cuda")
+    val = torch.zeros((W, k), device="cuda")
+    out = torch.zeros(d, device="cuda")
+    repaired = predicted = 0
+    for t in range(30):
+        g = torch.randn((W, d), generator=gen, device="cuda") * 1e-3
+        a = g + m
+        ctx.step(g, m, d, r, k, 7, t, idx, val, out)
+        ctx.poll_status()
+        for w in range(W):
+            st = ctx.stats(w)
+            repaired += st["used_fallback"]
+            predicted += st["bracket_predicted"]
+            i = idx[w].to(torch.int64)                     # whatever the path, the round is a valid one
+            back = m[w].clone()
+            back[i] = val[w]
+            assert torch.equal(back.view(torch.int32), a[w].view(torch.int32))
+            key = a[w].view(torch.int32) & 0x7FFFFFFF
+            assert int((key > st["tau_key"]).sum()) == st["n_greater"] < r
+    assert predicted >= 40 and repaired <= 3, (predicted, repaired)
+    ctx.close()
